@@ -1,0 +1,164 @@
+"""Pins for the oracle's budget allocation, top-k selection and compaction."""
+import numpy as np
+import pytest
+
+from oracle import flashcache_oracle as O
+
+
+# ---------------------------------------------------------------- allocation
+def test_total_budget_rounding_and_clamps():
+    assert O.total_budget(1024, 1, 0.2, 1) == 205        # floor(204.8 + .5)
+    assert O.total_budget(10, 4, 0.25, 1) == 10
+    assert O.total_budget(10, 4, 0.0, 1) == 4            # at least min_keep per layer
+    assert O.total_budget(10, 4, 0.0, 50) == 40          # min_keep itself is capped at N
+    assert O.total_budget(10, 4, 3.0, 1) == 40           # never more than everything
+
+
+def test_single_layer_gets_the_whole_budget():
+    assert list(O.allocate_budgets_one([0.37], 1024, 0.2)) == [205]
+
+
+def test_rho_one_keeps_everything():
+    assert list(O.allocate_budgets_one([0.1, 0.5, 0.9], 77, 1.0)) == [77, 77, 77]
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_budget_invariants_random(seed):
+    rng = np.random.default_rng(seed)
+    L = int(rng.integers(1, 40))
+    N = int(rng.integers(1, 5000))
+    rho = float(rng.choice([0.05, 0.1, 0.2, 0.5, 0.9]))
+    min_keep = int(rng.choice([0, 1, 4, 64]))
+    R = rng.random(L) ** 3 * 2.0
+    if seed % 5 == 0:
+        R[rng.integers(0, L)] = 0.0
+    b = O.allocate_budgets_one(R, N, rho, min_keep)
+    assert b.sum() == O.total_budget(N, L, rho, min_keep)
+    assert b.min() >= min(min_keep, N) and b.max() <= N
+    order = np.argsort(R, kind="stable")
+    assert all(b[order[i]] <= b[order[i + 1]] + 1 for i in range(L - 1))   # monotone up to rounding
+    for i in range(L):
+        for j in range(L):
+            if R[i] > R[j]:
+                assert b[i] >= b[j] - 1
+
+
+def test_equal_ratios_give_equal_budgets_up_to_one():
+    b = O.allocate_budgets_one([0.3] * 7, 1000, 0.2)
+    assert b.sum() == 1400 and b.max() - b.min() <= 1
+    assert list(b) == [200] * 7
+    b = O.allocate_budgets_one([0.3] * 7, 1001, 0.2)      # 1401.4 -> 1401 = 7*200 + 1
+    assert b.sum() == 1401 and sorted(b) == [200] * 6 + [201]
+    assert b[0] == 201                                    # tie on the remainder: lower layer first
+
+
+def test_zero_or_bad_ratios_fall_back_to_uniform():
+    for R in ([0.0, 0.0, 0.0, 0.0], [float("nan"), 1.0, 1.0, 1.0], [float("inf"), 1.0, 1.0, 1.0]):
+        b = O.allocate_budgets_one(R, 100, 0.5)
+        assert list(b) == [50, 50, 50, 50]
+
+
+def test_shares_are_proportional_when_no_cap_binds():
+    R = np.array([1.0, 2.0, 3.0, 4.0])
+    b = O.allocate_budgets_one(R, 10000, 0.1, 1)           # total 4000 -> 400, 800, 1200, 1600
+    assert list(b) == [400, 800, 1200, 1600]
+
+
+def test_upper_cap_binds_and_the_rest_is_reshared():
+    # total = round(0.5*100*3) = 150; raw shares 0.8/0.1/0.1 -> 120, 15, 15.
+    # Layer 0 is capped at N = 100 and the other two split the remaining 50 equally.
+    b = O.allocate_budgets_one([0.8, 0.1, 0.1], 100, 0.5, 1)
+    assert list(b) == [100, 25, 25]
+
+
+def test_lower_cap_binds():
+    # total = 30; raw shares 0, 10, 20 -> layer 0 is lifted to min_keep = 6 and
+    # the other two share the remaining 24 in ratio 1:2.
+    b = O.allocate_budgets_one([0.0, 1.0, 2.0], 100, 0.1, 6)
+    assert list(b) == [6, 8, 16]
+
+
+def test_allocate_budgets_batches_and_offsets():
+    rng = np.random.default_rng(0)
+    L, B = 5, 3
+    energy = rng.random((L, B, 4)) + 0.1
+    energy[..., 1] += energy[..., 0]
+    energy[..., 3] += energy[..., 2]
+    seqlens = [100, 0, 37]
+    budgets, offsets = O.allocate_budgets(energy, seqlens, 0.2, 1)
+    assert budgets.shape == (L, B) and offsets.shape == (L, B + 1)
+    for b in range(B):
+        R = [O.energy_ratio(energy[l, b]) for l in range(L)]
+        np.testing.assert_array_equal(budgets[:, b], O.allocate_budgets_one(R, seqlens[b], 0.2, 1))
+    assert (budgets[:, 1] == 0).all()
+    np.testing.assert_array_equal(offsets[:, 0], 0)
+    np.testing.assert_array_equal(offsets[:, 1:], np.cumsum(budgets, axis=1))
+
+
+# ---------------------------------------------------------------- selection
+def _brute_force_topk(dev, k):
+    """Repeated arg-max, lowest index first among equals: independent of sorting."""
+    key = [float("inf") if x != x else float(x) for x in dev]
+    alive = list(range(len(key)))
+    out = []
+    for _ in range(k):
+        best = alive[0]
+        for x in alive[1:]:
+            if key[x] > key[best]:
+                best = x
+        out.append(best)
+        alive.remove(best)
+    return sorted(out)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_topk_matches_brute_force(seed):
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(1, 40))
+    dev = rng.integers(0, 6, n).astype(np.float64)        # many duplicates, also at the threshold
+    if seed % 3 == 0:
+        dev[rng.integers(0, n)] = np.nan
+    for k in {0, 1, n // 2, max(0, n - 1), n}:
+        assert list(O.select_topk(dev, k)) == _brute_force_topk(dev, k)
+
+
+def test_topk_special_cases():
+    assert list(O.select_topk([1.0, 1.0, 1.0, 1.0], 2)) == [0, 1]          # all equal: lowest indices
+    assert list(O.select_topk([0.0, 5.0, 5.0, 1.0, 5.0], 2)) == [1, 2]     # tie at the cut
+    assert list(O.select_topk([3.0, np.nan, 9.0], 1)) == [1]               # NaN ranks as +inf
+    assert list(O.select_topk([3.0, 2.0], 0)) == []
+    assert list(O.select_topk([3.0, 2.0], 2)) == [0, 1]
+
+
+def test_compaction_is_a_bit_copy():
+    rng = np.random.default_rng(1)
+    X = rng.standard_normal((9, 4)).astype(np.float32)
+    X[3, 1] = np.nan
+    out = O.compact_rows(X, [7, 3, 3])
+    assert out.tobytes() == np.stack([X[7], X[3], X[3]]).tobytes()
+
+
+def test_compress_end_to_end_small():
+    rng = np.random.default_rng(2)
+    L, H, d = 3, 2, 8
+    lens = [24, 9]
+    cu = [0, 24, 33]
+    Ks = [rng.standard_normal((33, H, d)).astype(np.float32) for _ in range(L)]
+    Vs = [rng.standard_normal((33, H, d)).astype(np.float32) for _ in range(L)]
+    Ks[1][5] += 30.0                                        # a planted outlier row, all heads, layer 1
+    res = O.compress(Ks, Vs, cu, 0.25, 0.5, 1, tier="literal")
+    assert res["budgets"].sum(axis=0).tolist() == [O.total_budget(24, L, 0.5, 1), O.total_budget(9, L, 0.5, 1)]
+    for l in range(L):
+        rows = int(res["offsets"][l, -1])
+        assert res["out_k"][l].shape == (rows, H, d)
+        for h in range(H):
+            for b in range(2):
+                sel = res["idx"][l][h][b]
+                assert len(sel) == res["budgets"][l, b]
+                assert list(sel) == sorted(set(sel.tolist()))
+                o = int(res["offsets"][l, b])
+                got = res["out_k"][l][o:o + len(sel), h]
+                assert got.tobytes() == Ks[l][cu[b] + sel, h].tobytes()
+                got = res["out_v"][l][o:o + len(sel), h]
+                assert got.tobytes() == Vs[l][cu[b] + sel, h].tobytes()
+    assert 5 in res["idx"][1][0][0] and 5 in res["idx"][1][1][0]
