@@ -1,0 +1,161 @@
+/*
+ * flashcache.h -- C ABI of the B200 FlashCache compression path.
+ *
+ * The library runs the prefill-time KV-cache compressor of "Revisiting
+ * Multimodal KV Cache Compression: A Frequency-Domain-Guided
+ * Outlier-KV-Aware Approach" (FlashCache) on one GPU:
+ *
+ *     fc_score_layer      x L   Outlier KV Recognition Module   (Sec. 3.2.1, Eq. 5-10)
+ *                               + the energy sums of Eq. 11-12  (Sec. 3.2.2)
+ *     fc_allocate_budgets x 1   Dynamic Budget Allocation       (Sec. 3.2.2, last paragraph)
+ *     fc_select_compact   x L   keep the Outlier KVs by budget  (Sec. 3.2.1, last sentence)
+ *
+ * Conventions
+ *   - Every pointer is marked HOST or DEVICE.  The caller owns every buffer;
+ *     the library allocates device memory only in fc_create and never frees or
+ *     writes caller inputs.
+ *   - All work is enqueued on the caller's stream (a cudaStream_t passed as
+ *     void*); no entry point except fc_last_device_status synchronises.
+ *   - Argument errors are found on the host before anything is launched and
+ *     are returned as fc_status; nothing traps or aborts.
+ *   - One handle serves one stream at a time.
+ *   - KV layout: element [t][h][c] at  base + t*stride_token + h*stride_head + c
+ *     (strides in elements, channel stride 1).  The sequences of a batch are
+ *     packed along t; sequence b owns tokens [cu_seqlens[b], cu_seqlens[b+1]).
+ *     Base pointers and row strides must be 16-byte aligned; head_dim must be
+ *     a multiple of 64.
+ */
+#ifndef FLASHCACHE_H_
+#define FLASHCACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FC_OK = 0,
+  FC_ERR_INVALID_ARG = 1,   /* null pointer, bad size, bad alignment, bad cu_seqlens */
+  FC_ERR_UNSUPPORTED = 2,   /* dtype / head_dim / sequence length outside what was built */
+  FC_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or smaller than the query says */
+  FC_ERR_CUDA = 4,          /* a CUDA runtime call failed */
+  FC_ERR_TIMEOUT = 5,       /* reserved: a bounded device-side wait ran out */
+  FC_ERR_INTERNAL = 6       /* a device-side self check failed (see fc_last_device_status) */
+} fc_status;
+
+typedef enum { FC_F32 = 0, FC_F16 = 1, FC_BF16 = 2 } fc_dtype;
+
+typedef struct fc_handle fc_handle;   /* opaque: twiddle table, status word, launch counter */
+typedef void *fc_stream;              /* a cudaStream_t */
+
+/* One layer's K and V (Eq. 5: K^l = [k_0 .. k_{N-1}], V^l likewise), all KV heads,
+ * all sequences of the batch packed along the token axis. */
+typedef struct {
+  const void *k;              /* DEVICE */
+  const void *v;              /* DEVICE */
+  int64_t stride_token;       /* elements between consecutive tokens          */
+  int64_t stride_head;        /* elements between consecutive heads           */
+  int32_t dtype;              /* fc_dtype                                     */
+  int32_t num_heads;          /* KV heads H                                   */
+  int32_t head_dim;           /* channels per head d                          */
+  int32_t batch;              /* number of sequences B                        */
+  const int32_t *cu_seqlens;  /* HOST int32[B+1], cu[0] = 0, non-decreasing   */
+} fc_kv_view;
+
+/* Create a handle on `device`.  max_seqlen bounds every N_b later passed in
+ * (1 <= max_seqlen <= 131072; lengths that are not a power of two, or below 16,
+ * are limited to 65536).  Allocates the twiddle table (8 bytes * 4 * next power of two of
+ * max_seqlen) and a status word.  Returns FC_ERR_CUDA if the device cannot be
+ * used, FC_ERR_UNSUPPORTED if max_seqlen is out of range. */
+fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen);
+void fc_destroy(fc_handle *h);
+const char *fc_status_string(fc_status s);
+
+/* Synchronises `stream`, then returns FC_OK or the error the kernels recorded in
+ * the handle's device status word since the last call (and clears it). */
+fc_status fc_last_device_status(fc_handle *h, fc_stream stream);
+
+/* Number of kernels this handle has launched since fc_create (diagnostic). */
+uint64_t fc_launch_count(const fc_handle *h);
+
+/* Target size in bytes of the transform intermediates processed per kernel group
+ * (kept below the L2 capacity so they are re-read from cache, not HBM).
+ * Default 32 MiB.  Affects speed only. */
+fc_status fc_set_group_bytes(fc_handle *h, size_t bytes);
+
+/* Workspace sizes (bytes) the next two calls need for this view.  0 on bad input. */
+size_t fc_score_workspace_bytes(const fc_handle *h, const fc_kv_view *kv);
+size_t fc_select_workspace_bytes(const fc_handle *h, const fc_kv_view *kv);
+
+/*
+ * Outlier KV Recognition Module for one layer (Sec. 3.2.1).
+ * For every sequence b (length N), head h and channel c, K and V are taken along
+ * the token axis through the orthonormal DCT of Eq. 6-7, low-pass filtered with
+ * omega = min(N-1, floor(gamma*N)), bins 0..omega kept (Eq. 8), transformed back
+ * (Eq. 9), and every token is scored by
+ *     Dev[x] = mean_c (K[x,c]-K_base[x,c])^2 + mean_c (V[x,c]-V_base[x,c])^2   (Eq. 10).
+ * Arithmetic is fp32 on the stored values.
+ *
+ *   gamma      cutoff factor, 0 <= gamma <= 1.
+ *   scores     DEVICE float[num_heads][T], T = cu_seqlens[B]; written for every token.
+ *   energy     DEVICE double[B][4] = (hiK, totK, hiV, totV) per sequence: the sums of the
+ *              power spectrum P[m] = |C[m]|^2 (Eq. 11) over m > omega and over all m, over
+ *              every head and channel of the layer -- numerators and denominators of
+ *              Eq. 12.  By Parseval (the orthonormal transform of Eq. 6-7) they are
+ *              accumulated as d*sum Dev_k and sum K^2 without storing a spectrum.
+ *   workspace  DEVICE, 256-byte aligned, >= fc_score_workspace_bytes(); scratch only.
+ * Errors: FC_ERR_INVALID_ARG, FC_ERR_UNSUPPORTED (dtype, head_dim % 64, N_b > max_seqlen),
+ * FC_ERR_WORKSPACE, FC_ERR_CUDA (launch failure).
+ */
+fc_status fc_score_layer(fc_handle *h, const fc_kv_view *kv, double gamma,
+                         float *scores, double *energy,
+                         void *workspace, size_t workspace_bytes, fc_stream stream);
+
+/*
+ * Dynamic Budget Allocation Module (Sec. 3.2.2): R^l = hiK/totK + hiV/totV (Eq. 12)
+ * per layer and sequence, normalised to weights, the total budget
+ * B_tot = clamp(floor(rho*N*L + 1/2), L*lo, L*N), lo = min(min_keep, N), shared out as
+ * q_l = clamp(lambda*w_l, lo, N) with sum q_l = B_tot, made integer by largest
+ * remainder (ties: lower layer first).  All in fp64 on the device.
+ *
+ *   energy           DEVICE double[L][B][4] (the per-layer outputs of fc_score_layer).
+ *   cu_seqlens_host  HOST int32[B+1].
+ *   budgets          DEVICE int32[L][B]: tokens kept per head in layer l, sequence b.
+ *   out_offsets      DEVICE int64[L][B+1]: exclusive prefix sum of budgets[l][.]
+ *                    (first row of sequence b in layer l's compacted cache; [B] = rows).
+ * Limits: 1 <= L <= 1024.  Errors: FC_ERR_INVALID_ARG, FC_ERR_UNSUPPORTED, FC_ERR_CUDA.
+ */
+fc_status fc_allocate_budgets(fc_handle *h, const double *energy, int32_t num_layers,
+                              int32_t batch, const int32_t *cu_seqlens_host,
+                              double rho, int32_t min_keep,
+                              int32_t *budgets, int64_t *out_offsets, fc_stream stream);
+
+/*
+ * Keep the Outlier KVs of one layer (Sec. 3.2.1, last sentence; compacted cache of
+ * Fig. 2): for every sequence b and head h the budgets[b] tokens with the largest
+ * score (order: score descending, token index ascending; NaN ranks as +inf) are
+ * written as ascending sequence-local token indices, and their K and V rows are
+ * copied bit for bit.
+ *
+ *   scores       DEVICE float[num_heads][T]           (from fc_score_layer)
+ *   budgets      DEVICE int32[B]                      (layer l's slice)
+ *   out_offsets  DEVICE int64[B+1]                    (layer l's slice)
+ *   out_idx      DEVICE int32[num_heads][out_capacity_rows]; entry [h][out_offsets[b]+j]
+ *   out_k,out_v  DEVICE, dtype of the input, dense [row][h][c], out_capacity_rows rows;
+ *                row out_offsets[b]+j, head h = input row cu[b]+out_idx[h][..], head h.
+ *   out_capacity_rows  rows available; a sequence whose rows would pass it is
+ *                skipped and FC_ERR_INTERNAL is recorded in the status word.
+ *   workspace    DEVICE, 256-byte aligned, >= fc_select_workspace_bytes().
+ */
+fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const float *scores,
+                            const int32_t *budgets, const int64_t *out_offsets,
+                            void *out_k, void *out_v, int32_t *out_idx,
+                            int64_t out_capacity_rows,
+                            void *workspace, size_t workspace_bytes, fc_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLASHCACHE_H_ */

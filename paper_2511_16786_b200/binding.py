@@ -1,0 +1,275 @@
+"""ctypes binding of libflashcache.so: argument marshalling only.
+
+Every function here has the name and the meaning of the C entry point declared
+in include/flashcache.h; tensors are passed as device pointers, the current
+torch CUDA stream is passed as the stream.  All arithmetic happens in the CUDA
+library.  There is no fallback: if the library has not been built this module
+raises on import.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_double, c_int, c_int32, c_int64, c_size_t, c_uint64, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libflashcache.so")
+
+FC_OK = 0
+FC_F32, FC_F16, FC_BF16 = 0, 1, 2
+_DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
+
+EXPORTS = (
+    "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count",
+    "fc_set_group_bytes", "fc_score_workspace_bytes", "fc_select_workspace_bytes",
+    "fc_score_layer", "fc_allocate_budgets", "fc_select_compact",
+)
+
+
+class fc_kv_view(ctypes.Structure):
+    _fields_ = [
+        ("k", c_void_p), ("v", c_void_p),
+        ("stride_token", c_int64), ("stride_head", c_int64),
+        ("dtype", c_int32), ("num_heads", c_int32), ("head_dim", c_int32), ("batch", c_int32),
+        ("cu_seqlens", POINTER(c_int32)),
+    ]
+
+
+class FlashCacheError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: %s (fc_status %d)" % (where, status_string(code), code))
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            "libflashcache.so is missing at %s: build it with "
+            "`python -m paper_2511_16786_b200.build` (needs nvcc); there is no CPU fallback" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    lib.fc_create.argtypes = [POINTER(c_void_p), c_int, c_int32]
+    lib.fc_create.restype = c_int
+    lib.fc_destroy.argtypes = [c_void_p]
+    lib.fc_destroy.restype = None
+    lib.fc_status_string.argtypes = [c_int]
+    lib.fc_status_string.restype = c_char_p
+    lib.fc_last_device_status.argtypes = [c_void_p, c_void_p]
+    lib.fc_last_device_status.restype = c_int
+    lib.fc_launch_count.argtypes = [c_void_p]
+    lib.fc_launch_count.restype = c_uint64
+    lib.fc_set_group_bytes.argtypes = [c_void_p, c_size_t]
+    lib.fc_set_group_bytes.restype = c_int
+    lib.fc_score_workspace_bytes.argtypes = [c_void_p, POINTER(fc_kv_view)]
+    lib.fc_score_workspace_bytes.restype = c_size_t
+    lib.fc_select_workspace_bytes.argtypes = [c_void_p, POINTER(fc_kv_view)]
+    lib.fc_select_workspace_bytes.restype = c_size_t
+    lib.fc_score_layer.argtypes = [c_void_p, POINTER(fc_kv_view), c_double, c_void_p, c_void_p,
+                                   c_void_p, c_size_t, c_void_p]
+    lib.fc_score_layer.restype = c_int
+    lib.fc_allocate_budgets.argtypes = [c_void_p, c_void_p, c_int32, c_int32, POINTER(c_int32),
+                                        c_double, c_int32, c_void_p, c_void_p, c_void_p]
+    lib.fc_allocate_budgets.restype = c_int
+    lib.fc_select_compact.argtypes = [c_void_p, POINTER(fc_kv_view), c_void_p, c_void_p, c_void_p,
+                                      c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_size_t, c_void_p]
+    lib.fc_select_compact.restype = c_int
+    return lib
+
+
+_lib = _load()
+
+
+def status_string(code: int) -> str:
+    return _lib.fc_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != FC_OK:
+        raise FlashCacheError(code, where)
+
+
+def _stream() -> c_void_p:
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _cu_array(cu_seqlens):
+    vals = [int(x) for x in cu_seqlens]
+    return (c_int32 * len(vals))(*vals)
+
+
+def make_view(k: torch.Tensor, v: torch.Tensor, cu_arr) -> fc_kv_view:
+    """View of K, V [T, H, d] tensors (channel stride 1; V must share K's strides)."""
+    if k.dim() != 3 or v.shape != k.shape or v.dtype != k.dtype:
+        raise ValueError("k and v must be [T, H, d] tensors of one dtype")
+    if k.stride(2) != 1 or v.stride() != k.stride():
+        raise ValueError("channel stride must be 1 and v must be laid out like k")
+    if k.dtype not in _DTYPE:
+        raise ValueError("unsupported dtype %s" % k.dtype)
+    return fc_kv_view(c_void_p(k.data_ptr()), c_void_p(v.data_ptr()), k.stride(0), k.stride(1),
+                      _DTYPE[k.dtype], k.shape[1], k.shape[2], len(cu_arr) - 1,
+                      ctypes.cast(cu_arr, POINTER(c_int32)))
+
+
+# ----------------------------------------------------------------------------
+# entry points (same names as the C ABI)
+# ----------------------------------------------------------------------------
+def fc_create(device: int = 0, max_seqlen: int = 65536) -> c_void_p:
+    h = c_void_p()
+    _check(_lib.fc_create(byref(h), int(device), int(max_seqlen)), "fc_create")
+    return h
+
+
+def fc_destroy(handle) -> None:
+    _lib.fc_destroy(handle)
+
+
+def fc_last_device_status(handle) -> int:
+    return int(_lib.fc_last_device_status(handle, _stream()))
+
+
+def fc_launch_count(handle) -> int:
+    return int(_lib.fc_launch_count(handle))
+
+
+def fc_set_group_bytes(handle, nbytes: int) -> None:
+    _check(_lib.fc_set_group_bytes(handle, int(nbytes)), "fc_set_group_bytes")
+
+
+def fc_score_workspace_bytes(handle, k, v, cu_seqlens) -> int:
+    cu = _cu_array(cu_seqlens)
+    view = make_view(k, v, cu)
+    return int(_lib.fc_score_workspace_bytes(handle, byref(view)))
+
+
+def fc_select_workspace_bytes(handle, k, v, cu_seqlens) -> int:
+    cu = _cu_array(cu_seqlens)
+    view = make_view(k, v, cu)
+    return int(_lib.fc_select_workspace_bytes(handle, byref(view)))
+
+
+def fc_score_layer(handle, k, v, cu_seqlens, gamma: float, scores, energy, workspace) -> None:
+    """scores: float32 [H, T]; energy: float64 [B, 4]; workspace: uint8 device tensor."""
+    cu = _cu_array(cu_seqlens)
+    view = make_view(k, v, cu)
+    _check(_lib.fc_score_layer(handle, byref(view), float(gamma), c_void_p(scores.data_ptr()),
+                               c_void_p(energy.data_ptr()), c_void_p(workspace.data_ptr()),
+                               workspace.numel() * workspace.element_size(), _stream()), "fc_score_layer")
+
+
+def fc_allocate_budgets(handle, energy, cu_seqlens, rho: float, min_keep: int, budgets, out_offsets) -> None:
+    """energy: float64 [L, B, 4]; budgets: int32 [L, B]; out_offsets: int64 [L, B+1]."""
+    cu = _cu_array(cu_seqlens)
+    L, B = int(energy.shape[0]), int(energy.shape[1])
+    _check(_lib.fc_allocate_budgets(handle, c_void_p(energy.data_ptr()), L, B,
+                                    ctypes.cast(cu, POINTER(c_int32)), float(rho), int(min_keep),
+                                    c_void_p(budgets.data_ptr()), c_void_p(out_offsets.data_ptr()),
+                                    _stream()), "fc_allocate_budgets")
+
+
+def fc_select_compact(handle, k, v, cu_seqlens, scores, budgets, out_offsets, out_k, out_v, out_idx,
+                      workspace) -> None:
+    """budgets: int32 [B], out_offsets: int64 [B+1] (one layer's slices);
+    out_k/out_v: [capacity, H, d]; out_idx: int32 [H, capacity]."""
+    cu = _cu_array(cu_seqlens)
+    view = make_view(k, v, cu)
+    cap = int(out_k.shape[0])
+    _check(_lib.fc_select_compact(handle, byref(view), c_void_p(scores.data_ptr()),
+                                  c_void_p(budgets.data_ptr()), c_void_p(out_offsets.data_ptr()),
+                                  c_void_p(out_k.data_ptr()), c_void_p(out_v.data_ptr()),
+                                  c_void_p(out_idx.data_ptr()), cap, c_void_p(workspace.data_ptr()),
+                                  workspace.numel() * workspace.element_size(), _stream()),
+           "fc_select_compact")
+
+
+# ----------------------------------------------------------------------------
+# convenience: buffers for a whole model and the three-phase pass
+# ----------------------------------------------------------------------------
+class Compressor:
+    """Owns a handle and the device buffers of one workload shape; `compress`
+    issues fc_score_layer x L, fc_allocate_budgets, fc_select_compact x L on the
+    current stream.  Only allocation and call sequencing happen here."""
+
+    def __init__(self, num_layers: int, num_heads: int, head_dim: int, cu_seqlens, dtype, rho: float,
+                 gamma: float = 0.2, min_keep: int = 1, device: int = 0, group_bytes: int | None = None):
+        self.L, self.H, self.d = num_layers, num_heads, head_dim
+        self.cu = [int(x) for x in cu_seqlens]
+        self.B = len(self.cu) - 1
+        self.T = self.cu[-1]
+        self.rho, self.gamma, self.min_keep = float(rho), float(gamma), int(min_keep)
+        self.dtype = dtype
+        self.device = torch.device("cuda", device)
+        seqlens = [self.cu[b + 1] - self.cu[b] for b in range(self.B)]
+        self.handle = fc_create(device, max(1, max(seqlens) if seqlens else 1))
+        if group_bytes:
+            fc_set_group_bytes(self.handle, group_bytes)
+        dev = self.device
+        self.scores = torch.empty((self.L, self.H, max(self.T, 1)), dtype=torch.float32, device=dev)
+        self.energy = torch.empty((self.L, self.B, 4), dtype=torch.float64, device=dev)
+        self.budgets = torch.empty((self.L, self.B), dtype=torch.int32, device=dev)
+        self.offsets = torch.empty((self.L, self.B + 1), dtype=torch.int64, device=dev)
+        # rows any one layer can receive: every sequence is capped at its own length and at its total
+        import math
+        self.capacity = 0
+        for n in seqlens:
+            lo = min(self.min_keep, n)
+            tot = max(self.L * lo, min(self.L * n, int(math.floor(self.rho * n * self.L + 0.5))))
+            self.capacity += min(n, tot)
+        self.capacity = max(self.capacity, 1)
+        self.out_k = None
+        self.out_v = None
+        self.out_idx = None
+        self._ws = None
+
+    def close(self):
+        if self.handle is not None:
+            fc_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _workspace(self, k, v):
+        need = max(fc_score_workspace_bytes(self.handle, k, v, self.cu),
+                   fc_select_workspace_bytes(self.handle, k, v, self.cu))
+        if need == 0:
+            raise FlashCacheError(1, "fc_score_workspace_bytes")
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    def _outputs(self, per_layer_capacity: int):
+        if self.out_k is None or self.out_k.shape[1] < per_layer_capacity:
+            dev = self.device
+            self.out_k = torch.empty((self.L, per_layer_capacity, self.H, self.d), dtype=self.dtype, device=dev)
+            self.out_v = torch.empty_like(self.out_k)
+            self.out_idx = torch.empty((self.L, self.H, per_layer_capacity), dtype=torch.int32, device=dev)
+
+    def score(self, K_layers, V_layers):
+        ws = self._workspace(K_layers[0], V_layers[0])
+        for l in range(self.L):
+            fc_score_layer(self.handle, K_layers[l], V_layers[l], self.cu, self.gamma,
+                           self.scores[l], self.energy[l], ws)
+
+    def allocate(self):
+        fc_allocate_budgets(self.handle, self.energy, self.cu, self.rho, self.min_keep,
+                            self.budgets, self.offsets)
+
+    def select_compact(self, K_layers, V_layers):
+        ws = self._workspace(K_layers[0], V_layers[0])
+        self._outputs(self.capacity)
+        for l in range(self.L):
+            fc_select_compact(self.handle, K_layers[l], V_layers[l], self.cu, self.scores[l],
+                              self.budgets[l], self.offsets[l], self.out_k[l], self.out_v[l],
+                              self.out_idx[l], ws)
+
+    def compress(self, K_layers, V_layers):
+        self.score(K_layers, V_layers)
+        self.allocate()
+        self.select_compact(K_layers, V_layers)
+
+    def check_device_status(self):
+        _check(fc_last_device_status(self.handle), "device status")

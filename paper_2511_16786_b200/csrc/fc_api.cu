@@ -1,0 +1,92 @@
+// Handle life cycle, status reporting and the twiddle table of the FlashCache library.
+#include "fc_common.cuh"
+
+#include <new>
+
+namespace {
+
+// master[i] = exp(-2*pi*j*i/len), evaluated in fp64 and rounded once to fp32.
+__global__ void k_fill_master(float2 *master, int len) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= len) return;
+  double s, c;
+  sincospi(-2.0 * (double)i / (double)len, &s, &c);
+  master[i] = make_float2((float)c, (float)s);
+}
+
+}  // namespace
+
+extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) {
+  if (!out) return FC_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (max_seqlen < 1 || max_seqlen > 131072) return FC_ERR_UNSUPPORTED;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return FC_ERR_CUDA;
+  FC_CUDA_TRY(cudaSetDevice(device));
+  fc_handle *h = new (std::nothrow) fc_handle();
+  if (!h) return FC_ERR_INTERNAL;
+  h->device = device;
+  h->max_seqlen = max_seqlen;
+  int p2 = 64;
+  while (p2 < max_seqlen) p2 <<= 1;
+  h->master_len = 4 * p2;
+  h->master = nullptr;
+  h->status_word = nullptr;
+  h->group_bytes = (size_t)32 << 20;
+  h->launches = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return FC_ERR_CUDA; }
+  h->num_sms = prop.multiProcessorCount;
+  if (cudaMalloc(&h->master, (size_t)h->master_len * sizeof(float2)) != cudaSuccess ||
+      cudaMalloc(&h->status_word, sizeof(int)) != cudaSuccess ||
+      cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess) {
+    fc_destroy(h);
+    return FC_ERR_CUDA;
+  }
+  k_fill_master<<<(h->master_len + 255) / 256, 256>>>(h->master, h->master_len);
+  if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+    fc_destroy(h);
+    return FC_ERR_CUDA;
+  }
+  *out = h;
+  return FC_OK;
+}
+
+extern "C" void fc_destroy(fc_handle *h) {
+  if (!h) return;
+  if (h->master) cudaFree(h->master);
+  if (h->status_word) cudaFree(h->status_word);
+  delete h;
+}
+
+extern "C" const char *fc_status_string(fc_status s) {
+  switch (s) {
+    case FC_OK: return "ok";
+    case FC_ERR_INVALID_ARG: return "invalid argument";
+    case FC_ERR_UNSUPPORTED: return "unsupported dtype, head_dim or sequence length";
+    case FC_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case FC_ERR_CUDA: return "CUDA runtime error";
+    case FC_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case FC_ERR_INTERNAL: return "device-side self check failed";
+    default: return "unknown status";
+  }
+}
+
+extern "C" fc_status fc_last_device_status(fc_handle *h, fc_stream stream) {
+  if (!h) return FC_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FC_CUDA_TRY(cudaStreamSynchronize(st));
+  int word = 0;
+  FC_CUDA_TRY(cudaMemcpy(&word, h->status_word, sizeof(int), cudaMemcpyDeviceToHost));
+  if (word != 0) FC_CUDA_TRY(cudaMemset(h->status_word, 0, sizeof(int)));
+  if (word == 0) return FC_OK;
+  return (word & FC_DEV_FLAG_INTERNAL) ? FC_ERR_INTERNAL : FC_ERR_TIMEOUT;
+}
+
+extern "C" uint64_t fc_launch_count(const fc_handle *h) { return h ? (uint64_t)h->launches : 0; }
+
+extern "C" fc_status fc_set_group_bytes(fc_handle *h, size_t bytes) {
+  if (!h || bytes == 0) return FC_ERR_INVALID_ARG;
+  h->group_bytes = bytes;
+  return FC_OK;
+}

@@ -1,0 +1,270 @@
+// Shared device helpers of the FlashCache kernels: complex arithmetic on float2,
+// register-resident radix-2/4/8/16 DFTs, and the batched in-shared-memory FFT
+// stages.  The transforms here run along the token axis with the channels of a
+// tile spread across the lanes of a warp, so every lane of a warp executes the
+// same butterfly with the same twiddle and shared-memory rows are read with
+// unit stride.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+#include "../../include/flashcache.h"
+
+#define FC_MAX_STAGES 4
+
+// Bits of the device status word.
+#define FC_DEV_FLAG_INTERNAL 1
+#define FC_DEV_FLAG_TIMEOUT 2
+
+struct fc_handle {
+  int device;
+  int max_seqlen;
+  int master_len;          // power of two; master[i] = exp(-2*pi*i*j/master_len)
+  float2 *master;          // DEVICE
+  int *status_word;        // DEVICE
+  size_t group_bytes;
+  int num_sms;
+  unsigned long long launches;
+};
+
+// Radix plan of one power-of-two FFT length: len = prod radix[s].
+struct FftPlan {
+  int len;
+  int nstages;
+  int radix[FC_MAX_STAGES];
+};
+
+__host__ inline FftPlan make_plan(int len) {
+  FftPlan p;
+  p.len = len;
+  int bits = 0;
+  while ((1 << bits) < len) ++bits;
+  p.nstages = (bits + 3) / 4;
+  for (int s = 0; s < FC_MAX_STAGES; ++s) p.radix[s] = 1;
+  int left = bits;
+  for (int s = 0; s < p.nstages; ++s) {
+    int take = (left + (p.nstages - s) - 1) / (p.nstages - s);   // spread the bits evenly, larger first
+    p.radix[s] = 1 << take;
+    left -= take;
+  }
+  return p;
+}
+
+// ------------------------------------------------------------------ complex
+__device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+__device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
+__device__ __forceinline__ float2 cmul(float2 a, float2 w) {
+  return make_float2(a.x * w.x - a.y * w.y, a.x * w.y + a.y * w.x);
+}
+__device__ __forceinline__ float2 cmul_conj(float2 a, float2 w) {   // a * conj(w)
+  return make_float2(a.x * w.x + a.y * w.y, a.y * w.x - a.x * w.y);
+}
+__device__ __forceinline__ float2 cconj(float2 a) { return make_float2(a.x, -a.y); }
+__device__ __forceinline__ float2 cscale(float2 a, float s) { return make_float2(a.x * s, a.y * s); }
+
+// multiply by exp(DIR * j*pi/2): DIR=-1 -> -j, DIR=+1 -> +j
+template <int DIR>
+__device__ __forceinline__ float2 mul_j(float2 a) {
+  return DIR < 0 ? make_float2(a.y, -a.x) : make_float2(-a.y, a.x);
+}
+
+// ------------------------------------------------------------------ small DFTs
+// y[k] = sum_n x[n] exp(DIR*2*pi*j*n*k/R), natural order in and out.
+template <int DIR>
+__device__ __forceinline__ void dft2(float2 &a, float2 &b) {
+  float2 t = a;
+  a = cadd(t, b);
+  b = csub(t, b);
+}
+
+template <int DIR>
+__device__ __forceinline__ void dft4(float2 &a0, float2 &a1, float2 &a2, float2 &a3) {
+  float2 s0 = cadd(a0, a2), d0 = csub(a0, a2);
+  float2 s1 = cadd(a1, a3), d1 = mul_j<DIR>(csub(a1, a3));
+  a0 = cadd(s0, s1);
+  a2 = csub(s0, s1);
+  a1 = cadd(d0, d1);
+  a3 = csub(d0, d1);
+}
+
+template <int DIR>
+__device__ __forceinline__ void dft8(float2 (&x)[8]) {
+  const float h = 0.70710678118654752440f;
+  dft4<DIR>(x[0], x[2], x[4], x[6]);   // even samples -> x[0],x[2],x[4],x[6] = E0..E3
+  dft4<DIR>(x[1], x[3], x[5], x[7]);   // odd samples  -> x[1],x[3],x[5],x[7] = O0..O3
+  float2 e0 = x[0], e1 = x[2], e2 = x[4], e3 = x[6];
+  float2 o0 = x[1], o1 = x[3], o2 = x[5], o3 = x[7];
+  // w8^1 = (1 + DIR*j)/sqrt2, w8^2 = DIR*j, w8^3 = (-1 + DIR*j)/sqrt2
+  float2 t1 = DIR < 0 ? make_float2((o1.x + o1.y) * h, (o1.y - o1.x) * h)
+                      : make_float2((o1.x - o1.y) * h, (o1.x + o1.y) * h);
+  float2 t2 = mul_j<DIR>(o2);
+  float2 t3 = DIR < 0 ? make_float2((o3.y - o3.x) * h, -(o3.x + o3.y) * h)
+                      : make_float2(-(o3.x + o3.y) * h, (o3.x - o3.y) * h);
+  x[0] = cadd(e0, o0); x[4] = csub(e0, o0);
+  x[1] = cadd(e1, t1); x[5] = csub(e1, t1);
+  x[2] = cadd(e2, t2); x[6] = csub(e2, t2);
+  x[3] = cadd(e3, t3); x[7] = csub(e3, t3);
+}
+
+template <int DIR>
+__device__ __forceinline__ void dft16(float2 (&x)[16]) {
+  const float c1 = 0.92387953251128675613f, s1 = 0.38268343236508977173f;
+  const float h = 0.70710678118654752440f;
+  float2 e[8], o[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { e[i] = x[2 * i]; o[i] = x[2 * i + 1]; }
+  dft8<DIR>(e);
+  dft8<DIR>(o);
+  const float sg = DIR < 0 ? -1.f : 1.f;
+  // w16^k = (cos(k*pi/8), DIR*sin(k*pi/8))
+  float2 t[8];
+  t[0] = o[0];
+  t[1] = cmul(o[1], make_float2(c1, sg * s1));
+  t[2] = cmul(o[2], make_float2(h, sg * h));
+  t[3] = cmul(o[3], make_float2(s1, sg * c1));
+  t[4] = mul_j<DIR>(o[4]);
+  t[5] = cmul(o[5], make_float2(-s1, sg * c1));
+  t[6] = cmul(o[6], make_float2(-h, sg * h));
+  t[7] = cmul(o[7], make_float2(-c1, sg * s1));
+#pragma unroll
+  for (int k = 0; k < 8; ++k) { x[k] = cadd(e[k], t[k]); x[k + 8] = csub(e[k], t[k]); }
+}
+
+template <int R, int DIR>
+__device__ __forceinline__ void dft_small(float2 (&x)[R]) {
+  if constexpr (R == 2) dft2<DIR>(x[0], x[1]);
+  else if constexpr (R == 4) dft4<DIR>(x[0], x[1], x[2], x[3]);
+  else if constexpr (R == 8) dft8<DIR>(x);
+  else dft16<DIR>(x);
+}
+
+// ------------------------------------------------------------------ batched stages in shared memory
+// Tile S[len][ncol] (ncol a power of two, column index fastest).  tw[i] =
+// exp(-2*pi*j*i/len).  One radix-R stage over blocks of length Ls:
+//   forward (decimation in frequency): butterfly, then multiply output p by w_Ls^(j*p);
+//   inverse (decimation in time, the exact mirror): multiply input p by conj(w_Ls^(j*p)), butterfly.
+// A forward pass over all stages leaves bin rev(pos) at row pos; the inverse pass
+// takes that order back to natural order.  No 1/len factor is applied.
+template <int R, bool INVERSE>
+__device__ __forceinline__ void fft_stage(float2 *S, int ncol_log2, int len, int Ls,
+                                          const float2 *tw, int tid, int nthreads) {
+  const int sub = Ls / R;
+  const int ncol = 1 << ncol_log2;
+  const int total = (len / R) << ncol_log2;
+  const int twstep = len / Ls;
+  for (int w = tid; w < total; w += nthreads) {
+    const int c = w & (ncol - 1);
+    const int b = w >> ncol_log2;
+    const int block = b / sub;
+    const int j = b - block * sub;
+    float2 *base = S + ((size_t)(block * Ls + j) << ncol_log2) + c;
+    const int stride = sub << ncol_log2;
+    float2 x[R];
+#pragma unroll
+    for (int p = 0; p < R; ++p) x[p] = base[p * stride];
+    if (INVERSE) {
+      if (sub > 1) {
+#pragma unroll
+        for (int p = 1; p < R; ++p) x[p] = cmul_conj(x[p], tw[j * p * twstep]);
+      }
+      dft_small<R, +1>(x);
+    } else {
+      dft_small<R, -1>(x);
+      if (sub > 1) {
+#pragma unroll
+        for (int p = 1; p < R; ++p) x[p] = cmul(x[p], tw[j * p * twstep]);
+      }
+    }
+#pragma unroll
+    for (int p = 0; p < R; ++p) base[p * stride] = x[p];
+  }
+}
+
+template <bool INVERSE>
+__device__ __forceinline__ void fft_stage_dyn(int R, float2 *S, int ncol_log2, int len, int Ls,
+                                              const float2 *tw, int tid, int nthreads) {
+  switch (R) {
+    case 16: fft_stage<16, INVERSE>(S, ncol_log2, len, Ls, tw, tid, nthreads); break;
+    case 8: fft_stage<8, INVERSE>(S, ncol_log2, len, Ls, tw, tid, nthreads); break;
+    case 4: fft_stage<4, INVERSE>(S, ncol_log2, len, Ls, tw, tid, nthreads); break;
+    case 2: fft_stage<2, INVERSE>(S, ncol_log2, len, Ls, tw, tid, nthreads); break;
+    default: break;
+  }
+}
+
+// All forward stages, natural order -> digit-reversed order.  Ends with __syncthreads().
+__device__ __forceinline__ void fft_forward_tile(const FftPlan &plan, float2 *S, int ncol_log2,
+                                                 const float2 *tw, int tid, int nthreads) {
+  int Ls = plan.len;
+  for (int s = 0; s < plan.nstages; ++s) {
+    fft_stage_dyn<false>(plan.radix[s], S, ncol_log2, plan.len, Ls, tw, tid, nthreads);
+    Ls /= plan.radix[s];
+    __syncthreads();
+  }
+}
+
+// All inverse stages, digit-reversed order -> natural order.  Ends with __syncthreads().
+__device__ __forceinline__ void fft_inverse_tile(const FftPlan &plan, float2 *S, int ncol_log2,
+                                                 const float2 *tw, int tid, int nthreads) {
+  int Ls = 1;
+  for (int s = plan.nstages - 1; s >= 0; --s) {
+    Ls *= plan.radix[s];
+    fft_stage_dyn<true>(plan.radix[s], S, ncol_log2, plan.len, Ls, tw, tid, nthreads);
+    __syncthreads();
+  }
+}
+
+// Bin held at row pos after the forward stages.
+__device__ __forceinline__ int digit_rev(const FftPlan &plan, int pos) {
+  int k = 0, mult = 1, rem = plan.len;
+  for (int s = 0; s < plan.nstages; ++s) {
+    const int R = plan.radix[s];
+    const int sub = rem / R;
+    const int p = pos / sub;
+    pos -= p * sub;
+    k += p * mult;
+    mult *= R;
+    rem = sub;
+  }
+  return k;
+}
+
+// Row that holds bin k after the forward stages.
+__device__ __forceinline__ int digit_pos(const FftPlan &plan, int k) {
+  int pos = 0, rem = plan.len;
+  for (int s = 0; s < plan.nstages; ++s) {
+    const int R = plan.radix[s];
+    const int sub = rem / R;
+    const int p = k % R;
+    k /= R;
+    pos += p * sub;
+    rem = sub;
+  }
+  return pos;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Host-side launch bookkeeping shared by the translation units.
+#define FC_CUDA_TRY(expr)                          \
+  do {                                             \
+    cudaError_t e__ = (expr);                      \
+    if (e__ != cudaSuccess) return FC_ERR_CUDA;    \
+  } while (0)
+
+inline fc_status fc_after_launch(fc_handle *h) {
+  h->launches++;
+  return cudaPeekAtLastError() == cudaSuccess ? FC_OK : FC_ERR_CUDA;
+}

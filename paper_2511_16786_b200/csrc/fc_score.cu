@@ -1,0 +1,681 @@
+// fc_score_layer: Outlier KV Recognition Module (Sec. 3.2.1, Eq. 5-10) plus the
+// energy sums of Eq. 11-12, for one layer.
+//
+// How the score is computed.  For one head, channel c, the complex sequence
+// z[i] = K[i,c] + j V[i,c] carries both matrices through one transform (the DCT is a
+// real linear map, so real and imaginary parts never mix).  The orthonormal DCT-II of
+// Eq. 6-7 of a length-N sequence equals Re(exp(-j*pi*m/(2N)) * W[m]) * alpha[m], where W
+// is the N-point DFT of the even/odd reordering  w[n] = z[2n], w[N-1-n] = z[2n+1].
+// Low-pass filtering (Eq. 8) and the inverse DCT (Eq. 9) are linear, so the
+// spectrum of the residual  z - z_base  in that DFT domain is, with P = W[q],
+// Q = W[N-q], u = exp(j*pi*q/N):
+//     E[q] = P - [q <= omega] (P + uQ)/2 - [N-q <= omega] (P - uQ)/2,   E[0] = 0,
+// and the residual itself is the inverse DFT of E.  Dev[x] (Eq. 10) is then
+// (1/d) * sum_c |residual|^2 with the real part belonging to K and the imaginary
+// part to V; K and V are read exactly once and no Base KV is ever stored.
+//
+// The N-point DFT is done in three passes over an intermediate that stays in L2
+// (N = N1*N2, n = n1*N2 + n2, q = k1 + N1*k2):
+//   pass 1  for every n2: DFT over n1                      -> A[k1][n2]
+//   pass 2  for every k1 (with N1-k1, which holds the partner bins N-q):
+//           twiddle, DFT over n2, the filter above, inverse DFT over k2, twiddle -> B[k1][n2]
+//   pass 3  for every n2: inverse DFT over k1, |.|^2 summed over the channels -> scores
+// Lengths that are not a power of two (or are below 16) go through Bluestein's
+// chirp convolution on a power-of-two length M >= 2N-1 with the same three passes.
+#include "fc_common.cuh"
+
+#include <math.h>
+#include <type_traits>
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// ---------------------------------------------------------------------------
+// index helpers
+// ---------------------------------------------------------------------------
+// Reordered index p -> token (w[n] = z[2n] for n < ceil(N/2), w[N-1-n] = z[2n+1]).
+__device__ __forceinline__ int perm_token(int p, int N) {
+  const int half = (N + 1) >> 1;
+  return p < half ? 2 * p : 2 * (N - 1 - p) + 1;
+}
+
+// exp(j*pi*n^2/N), the Bluestein chirp; the phase is reduced exactly in integers.
+__device__ __forceinline__ float2 chirp(int n, int N) {
+  const unsigned long long r = ((unsigned long long)n * (unsigned long long)n) % (2ull * (unsigned long long)N);
+  float s, c;
+  sincospif(__fdiv_rn((float)(unsigned)r, (float)N), &s, &c);
+  return make_float2(c, s);
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int VEC = 4;
+  __device__ static void load(const float *p, float (&out)[4]) {
+    const float4 v = *reinterpret_cast<const float4 *>(p);
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+  }
+};
+template <> struct Elem<__half> {
+  static constexpr int VEC = 8;
+  __device__ static void load(const __half *p, float (&out)[8]) {
+    const uint4 v = *reinterpret_cast<const uint4 *>(p);
+    const __half2 *h = reinterpret_cast<const __half2 *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float2 f = __half22float2(h[i]); out[2 * i] = f.x; out[2 * i + 1] = f.y; }
+  }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int VEC = 8;
+  __device__ static void load(const __nv_bfloat16 *p, float (&out)[8]) {
+    const uint4 v = *reinterpret_cast<const uint4 *>(p);
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float2 f = __bfloat1622float2(h[i]); out[2 * i] = f.x; out[2 * i + 1] = f.y; }
+  }
+};
+
+// ---------------------------------------------------------------------------
+// pass-1 loaders: value of transform input p for VEC consecutive workspace columns
+// ---------------------------------------------------------------------------
+// K/V rows of one sequence.  Column gc of the group maps to head h0 + gc/d, channel gc%d.
+template <typename T, bool BLUE>
+struct KvLoader {
+  static constexpr int VEC = Elem<T>::VEC;
+  const T *k, *v;          // already offset to the first token of the sequence
+  long long stride_token, stride_head;
+  int head0, head_dim, N;
+  float accK, accV;        // running sums of squares (per thread)
+  __device__ void init() { accK = 0.f; accV = 0.f; }
+  __device__ void load(int p, int gc, float2 (&out)[VEC]) {
+    if (BLUE && p >= N) {
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) out[i] = make_float2(0.f, 0.f);
+      return;
+    }
+    const int t = perm_token(p, N);
+    const int h = head0 + gc / head_dim, c = gc % head_dim;
+    const long long off = (long long)t * stride_token + (long long)h * stride_head + c;
+    float a[VEC], b[VEC];
+    Elem<T>::load(k + off, a);
+    Elem<T>::load(v + off, b);
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) { accK = fmaf(a[i], a[i], accK); accV = fmaf(b[i], b[i], accV); }
+    if (BLUE) {
+      const float2 ch = chirp(p, N);
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) out[i] = cmul_conj(make_float2(a[i], b[i]), ch);
+    } else {
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) out[i] = make_float2(a[i], b[i]);
+    }
+  }
+};
+
+// Bluestein, second half: reads the N-point spectrum W[q][col], applies the
+// low-pass residual filter, and feeds conj(E[q]) * conj(chirp) to the forward
+// machinery (an inverse DFT is the conjugate of the forward DFT of the conjugate).
+struct FilterLoader {
+  static constexpr int VEC = 2;
+  const float2 *spec;      // [N][ncol]
+  int ncol, N, omega;
+  __device__ void init() {}
+  __device__ void load(int p, int gc, float2 (&out)[2]) {
+    if (p >= N) { out[0] = out[1] = make_float2(0.f, 0.f); return; }
+    const int q = p, qp = (N - q) % N;
+    const float4 P4 = *reinterpret_cast<const float4 *>(spec + (size_t)q * ncol + gc);
+    const float4 Q4 = *reinterpret_cast<const float4 *>(spec + (size_t)qp * ncol + gc);
+    float s, c;
+    sincospif(__fdiv_rn((float)q, (float)N), &s, &c);
+    const float2 u = make_float2(c, s);
+    const float inL = (q <= omega) ? 0.5f : 0.f;
+    const float inH = (q != 0 && N - q <= omega) ? 0.5f : 0.f;
+    const float2 ch = chirp(p, N);
+    const float2 Pv[2] = {make_float2(P4.x, P4.y), make_float2(P4.z, P4.w)};
+    const float2 Qv[2] = {make_float2(Q4.x, Q4.y), make_float2(Q4.z, Q4.w)};
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const float2 uQ = cmul(Qv[i], u);
+      float2 E = Pv[i];
+      E = csub(E, cscale(cadd(Pv[i], uQ), inL));
+      E = csub(E, cscale(csub(Pv[i], uQ), inH));
+      out[i] = cmul_conj(cconj(E), ch);
+    }
+  }
+};
+
+// Bluestein convolution kernel h[p] = chirp(|p|) wrapped to length M, in column 0.
+struct ChirpKernelLoader {
+  static constexpr int VEC = 2;
+  int N, M;
+  __device__ void init() {}
+  __device__ void load(int p, int gc, float2 (&out)[2]) {
+    out[0] = out[1] = make_float2(0.f, 0.f);
+    if (gc != 0) return;
+    if (p < N) out[0] = chirp(p, N);
+    else if (p > M - N) out[0] = chirp(M - p, N);
+  }
+};
+
+// ---------------------------------------------------------------------------
+// pass 1: DFT over n1 for one n2 and one slice of cs columns
+// grid (N2, ncol_ws/cs)
+// ---------------------------------------------------------------------------
+template <class Loader>
+__global__ void __launch_bounds__(kThreads)
+k_pass1(Loader ld, FftPlan plan, int N2, int ncol_ws, int cs_log2, float2 *__restrict__ ws,
+        const float2 *__restrict__ master, int master_len, double *__restrict__ partial) {
+  extern __shared__ float2 smem[];
+  const int N1 = plan.len, cs = 1 << cs_log2;
+  float2 *S = smem;
+  float2 *tw = S + (size_t)N1 * cs;
+  int *rev = reinterpret_cast<int *>(tw + N1);
+  const int tid = threadIdx.x;
+  const int n2 = blockIdx.x, gc0 = blockIdx.y * cs;
+
+  for (int i = tid; i < N1; i += kThreads) {
+    tw[i] = master[(size_t)i * (master_len / N1)];
+    rev[i] = digit_rev(plan, i);
+  }
+  ld.init();
+  constexpr int VEC = Loader::VEC;
+  const int vec_per_row = cs / VEC;
+  for (int it = tid; it < N1 * vec_per_row; it += kThreads) {
+    const int row = it / vec_per_row, cv = it - row * vec_per_row;
+    float2 vals[VEC];
+    ld.load(row * N2 + n2, gc0 + cv * VEC, vals);
+    float2 *dst = S + (size_t)row * cs + cv * VEC;
+#pragma unroll
+    for (int i = 0; i < VEC; i += 2)
+      *reinterpret_cast<float4 *>(dst + i) = make_float4(vals[i].x, vals[i].y, vals[i + 1].x, vals[i + 1].y);
+  }
+  __syncthreads();
+  fft_forward_tile(plan, S, cs_log2, tw, tid, kThreads);
+  for (int w = tid; w < N1 * cs; w += kThreads) {
+    const int pos = w >> cs_log2, c = w & (cs - 1);
+    ws[((size_t)rev[pos] * N2 + n2) * ncol_ws + gc0 + c] = S[w];
+  }
+  if constexpr (!std::is_same<Loader, FilterLoader>::value && !std::is_same<Loader, ChirpKernelLoader>::value) {
+    if (partial != nullptr) {
+      __shared__ double red[2][kThreads / 32];
+      double a = warp_sum_d((double)ld.accK), b = warp_sum_d((double)ld.accV);
+      if ((tid & 31) == 0) { red[0][tid >> 5] = a; red[1][tid >> 5] = b; }
+      __syncthreads();
+      if (tid == 0) {
+        double sa = 0, sb = 0;
+        for (int i = 0; i < kThreads / 32; ++i) { sa += red[0][i]; sb += red[1][i]; }
+        const size_t slot = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+        partial[2 * slot] = sa;
+        partial[2 * slot + 1] = sb;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// pass 2: for one k1 (and its partner N1-k1): twiddle, DFT over n2, middle step,
+// inverse DFT over k2, twiddle, scale.  In place in the workspace.
+// MID_DCT   : low-pass residual filter between bins q and N-q   grid (N1/2+1, ncol_ws/cs2)
+// MID_MULH  : pointwise product with the chirp spectrum          grid (N1, ncol_ws/cs2)
+// MID_SPEC  : forward only; column 0 written to hhat[k]          grid (N1, 1)
+// ---------------------------------------------------------------------------
+enum { MID_DCT = 0, MID_MULH = 1, MID_SPEC = 2 };
+
+template <int MID>
+__global__ void __launch_bounds__(kThreads)
+k_pass2(FftPlan plan, int N1, int ncol_ws, int cs2_log2, float2 *__restrict__ ws,
+        const float2 *__restrict__ master, int master_len, int omega,
+        float2 *__restrict__ hhat, float scale) {
+  extern __shared__ float2 smem[];
+  const int N2 = plan.len, cs2 = 1 << cs2_log2;
+  const int Nfft = N1 * N2;
+  const int tid = threadIdx.x;
+  int k1a = blockIdx.x, k1b = blockIdx.x;
+  int halves = 1;
+  if (MID == MID_DCT) {
+    k1b = (N1 - k1a) % N1;
+    halves = (k1b != k1a) ? 2 : 1;
+  }
+  const int ncolT_log2 = cs2_log2 + (halves - 1);
+  const int ncolT = 1 << ncolT_log2;
+  const int gc0 = blockIdx.y * cs2;
+
+  float2 *S = smem;                                    // [N2][2*cs2] at most
+  float2 *tw = S + (size_t)N2 * 2 * cs2;               // [N2]
+  float2 *twN = tw + N2;                               // [2][N2]
+  unsigned short *rev = reinterpret_cast<unsigned short *>(twN + 2 * N2);   // [N2]
+  unsigned short *pos_of = rev + N2;                                       // [N2]
+
+  const int mstepN = master_len / Nfft;
+  for (int i = tid; i < N2; i += kThreads) {
+    tw[i] = master[(size_t)i * (master_len / N2)];
+    twN[i] = master[(size_t)(((long long)i * k1a) % Nfft) * mstepN];
+    twN[N2 + i] = master[(size_t)(((long long)i * k1b) % Nfft) * mstepN];
+    const int k = digit_rev(plan, i);
+    rev[i] = (unsigned short)k;
+    pos_of[k] = (unsigned short)i;
+  }
+  __syncthreads();
+
+  // load with the forward inter-pass twiddle w_N^(n2*k1)
+  for (int w = tid; w < N2 * ncolT; w += kThreads) {
+    const int n2 = w >> ncolT_log2, col = w & (ncolT - 1);
+    const int hf = col >> cs2_log2, c = col & (cs2 - 1);
+    const int k1 = hf ? k1b : k1a;
+    const float2 a = ws[((size_t)k1 * N2 + n2) * ncol_ws + gc0 + c];
+    S[w] = cmul(a, twN[hf * N2 + n2]);
+  }
+  __syncthreads();
+  fft_forward_tile(plan, S, ncolT_log2, tw, tid, kThreads);
+
+  if (MID == MID_SPEC) {
+    for (int pos = tid; pos < N2; pos += kThreads)
+      hhat[k1a + N1 * (int)rev[pos]] = S[(size_t)pos << ncolT_log2];
+    return;
+  }
+  if (MID == MID_MULH) {
+    for (int w = tid; w < N2 * ncolT; w += kThreads) {
+      const int pos = w >> ncolT_log2;
+      S[w] = cmul(S[w], hhat[k1a + N1 * (int)rev[pos]]);
+    }
+  } else {
+    // Every pair {q, N-q} is owned by the thread that meets the smaller bin.
+    const int N = Nfft;
+    const int ustep = master_len / (2 * N);
+    for (int w = tid; w < N2 * ncolT; w += kThreads) {
+      const int pos = w >> ncolT_log2, col = w & (ncolT - 1);
+      const int hf = col >> cs2_log2, c = col & (cs2 - 1);
+      const int k1 = hf ? k1b : k1a;
+      const int q = k1 + N1 * (int)rev[pos];
+      const int qp = (N - q) % N;
+      if (q > qp) continue;
+      const int k1p = qp % N1, k2p = qp / N1;
+      const int hfp = (k1p == k1) ? hf : 1 - hf;
+      const int wp = ((int)pos_of[k2p] << ncolT_log2) + (hfp << cs2_log2) + c;
+      const float2 P = S[w], Q = S[wp];
+      if (q == 0) { S[w] = make_float2(0.f, 0.f); continue; }
+      const float2 u = cconj(master[(size_t)q * ustep]);           // exp(+j*pi*q/N)
+      const float2 uQ = cmul(Q, u);
+      const float inLq = (q <= omega) ? 0.5f : 0.f, inHq = (N - q <= omega) ? 0.5f : 0.f;
+      float2 Eq = P;
+      Eq = csub(Eq, cscale(cadd(P, uQ), inLq));
+      Eq = csub(Eq, cscale(csub(P, uQ), inHq));
+      S[w] = Eq;
+      if (qp != q) {
+        // bin N-q: u' = exp(j*pi*(N-q)/N) = -conj(u)
+        const float2 upP = cscale(cmul_conj(P, u), -1.f);
+        const float inLp = (qp <= omega) ? 0.5f : 0.f, inHp = (q <= omega) ? 0.5f : 0.f;
+        float2 Ep = Q;
+        Ep = csub(Ep, cscale(cadd(Q, upP), inLp));
+        Ep = csub(Ep, cscale(csub(Q, upP), inHp));
+        S[wp] = Ep;
+      }
+    }
+  }
+  __syncthreads();
+  fft_inverse_tile(plan, S, ncolT_log2, tw, tid, kThreads);
+  for (int w = tid; w < N2 * ncolT; w += kThreads) {
+    const int n2 = w >> ncolT_log2, col = w & (ncolT - 1);
+    const int hf = col >> cs2_log2, c = col & (cs2 - 1);
+    const int k1 = hf ? k1b : k1a;
+    const float2 r = cscale(cmul_conj(S[w], twN[hf * N2 + n2]), scale);
+    ws[((size_t)k1 * N2 + n2) * ncol_ws + gc0 + c] = r;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// pass 3: inverse DFT over k1 for one n2.
+// EPI_SCORE : loops over the head's column slices, accumulates sum_c |.|^2 per row,
+//             writes scores and the per-block outlier-energy partials.  grid (N2, heads)
+// EPI_SPEC  : multiplies by conj(chirp) and stores rows p < N of the N-point
+//             spectrum to spec[p][col] (Bluestein, first half).    grid (N2, ncol_ws/cs)
+// ---------------------------------------------------------------------------
+enum { EPI_SCORE = 0, EPI_SPEC = 1 };
+
+template <int EPI, bool BLUE>
+__global__ void __launch_bounds__(kThreads)
+k_pass3(FftPlan plan, int N2, int N, int ncol_ws, int cs_log2, const float2 *__restrict__ ws,
+        const float2 *__restrict__ master, int master_len,
+        float2 *__restrict__ spec, float *__restrict__ scores, int head0, int head_dim,
+        long long score_stride, float inv_scale, double *__restrict__ partial) {
+  extern __shared__ float2 smem[];
+  const int N1 = plan.len, cs = 1 << cs_log2;
+  float2 *S = smem;
+  float2 *tw = S + (size_t)N1 * cs;
+  int *rev = reinterpret_cast<int *>(tw + N1);
+  float *accK = reinterpret_cast<float *>(rev + N1);
+  float *accV = accK + N1;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n2 = blockIdx.x;
+
+  for (int i = tid; i < N1; i += kThreads) {
+    tw[i] = master[(size_t)i * (master_len / N1)];
+    rev[i] = digit_rev(plan, i);
+    accK[i] = 0.f;
+    accV[i] = 0.f;
+  }
+  __syncthreads();
+
+  const int nslices = (EPI == EPI_SCORE) ? head_dim / cs : 1;
+  for (int sl = 0; sl < nslices; ++sl) {
+    const int gc0 = (EPI == EPI_SCORE) ? (blockIdx.y * head_dim + sl * cs) : blockIdx.y * cs;
+    for (int w = tid; w < N1 * cs; w += kThreads) {
+      const int pos = w >> cs_log2, c = w & (cs - 1);
+      S[w] = ws[((size_t)rev[pos] * N2 + n2) * ncol_ws + gc0 + c];
+    }
+    __syncthreads();
+    fft_inverse_tile(plan, S, cs_log2, tw, tid, kThreads);
+    if (EPI == EPI_SPEC) {
+      for (int w = tid; w < N1 * cs; w += kThreads) {
+        const int n1 = w >> cs_log2, c = w & (cs - 1);
+        const int p = n1 * N2 + n2;
+        if (p < N) spec[(size_t)p * ncol_ws + gc0 + c] = cmul_conj(S[w], chirp(p, N));
+      }
+    } else {
+      for (int n1 = warp; n1 < N1; n1 += kThreads / 32) {
+        const int p = n1 * N2 + n2;
+        float sk = 0.f, sv = 0.f;
+        if (!BLUE || p < N) {
+          float2 ch = make_float2(1.f, 0.f);
+          if (BLUE) ch = chirp(p, N);
+          for (int c = lane; c < cs; c += 32) {
+            float2 e = S[((size_t)n1 << cs_log2) + c];
+            if (BLUE) e = cmul_conj(e, ch);
+            sk = fmaf(e.x, e.x, sk);
+            sv = fmaf(e.y, e.y, sv);
+          }
+        }
+        sk = warp_sum(sk);
+        sv = warp_sum(sv);
+        if (lane == 0) { accK[n1] += sk; accV[n1] += sv; }
+      }
+    }
+    __syncthreads();
+  }
+
+  if (EPI == EPI_SCORE) {
+    const int h = head0 + blockIdx.y;
+    double dk = 0.0, dv = 0.0;
+    for (int n1 = tid; n1 < N1; n1 += kThreads) {
+      const int p = n1 * N2 + n2;
+      if (p < N) {
+        const float k = accK[n1] * inv_scale, v = accV[n1] * inv_scale;   // already divided by d
+        scores[(long long)h * score_stride + perm_token(p, N)] = k + v;
+        dk += (double)k;
+        dv += (double)v;
+      }
+    }
+    __shared__ double red[2][kThreads / 32];
+    dk = warp_sum_d(dk);
+    dv = warp_sum_d(dv);
+    if (lane == 0) { red[0][warp] = dk; red[1][warp] = dv; }
+    __syncthreads();
+    if (tid == 0) {
+      double sa = 0, sb = 0;
+      for (int i = 0; i < kThreads / 32; ++i) { sa += red[0][i]; sb += red[1][i]; }
+      const size_t slot = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+      partial[2 * slot] = sa * (double)head_dim;      // d * sum Dev_k = outlier-band energy
+      partial[2 * slot + 1] = sb * (double)head_dim;
+    }
+  }
+}
+
+// Fixed-order reduction of the per-block partial sums of one sequence into
+// energy[4] = (hiK, totK, hiV, totV).  One block.
+__global__ void __launch_bounds__(256)
+k_energy_finalize(const double *__restrict__ part_tot, int n_tot, const double *__restrict__ part_hi,
+                  int n_hi, double *__restrict__ energy) {
+  __shared__ double red[4][256];
+  const int tid = threadIdx.x;
+  double a0 = 0, a1 = 0, b0 = 0, b1 = 0;
+  for (int i = tid; i < n_tot; i += 256) { a0 += part_tot[2 * i]; a1 += part_tot[2 * i + 1]; }
+  for (int i = tid; i < n_hi; i += 256) { b0 += part_hi[2 * i]; b1 += part_hi[2 * i + 1]; }
+  red[0][tid] = b0; red[1][tid] = a0; red[2][tid] = b1; red[3][tid] = a1;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (tid < s)
+      for (int j = 0; j < 4; ++j) red[j][tid] += red[j][tid + s];
+    __syncthreads();
+  }
+  if (tid < 4) energy[tid] = red[tid][0];
+}
+
+__global__ void k_zero_energy(double *energy) {
+  if (threadIdx.x < 4) energy[threadIdx.x] = 0.0;
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+inline int ilog2(int x) { int b = 0; while ((1 << b) < x) ++b; return b; }
+inline bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct SeqPlan {
+  bool bluestein;
+  int N, Nfft, N1, N2;
+  int cs, cs2;               // columns per tile in pass 1/3 and pass 2
+};
+
+SeqPlan plan_sequence(int N) {
+  SeqPlan s;
+  s.N = N;
+  s.bluestein = !(is_pow2(N) && N >= 16);
+  if (s.bluestein) {
+    int M = 64;
+    while (M < 2 * N - 1) M <<= 1;
+    s.Nfft = M;
+  } else {
+    s.Nfft = N;
+  }
+  const int bits = ilog2(s.Nfft);
+  int b1 = bits / 2;
+  if (b1 > 7) b1 = 7;
+  s.N1 = 1 << b1;
+  s.N2 = s.Nfft / s.N1;
+  s.cs = 64;
+  int cs2 = 4096 / s.N2;      // 2*N2*cs2*8 bytes = 64 KiB
+  if (cs2 > 64) cs2 = 64;
+  if (cs2 < 4) cs2 = 4;
+  s.cs2 = cs2;
+  return s;
+}
+
+struct ScoreLayout {
+  size_t off_ws, off_spec, off_hhat, off_hcol, off_part_tot, off_part_hi, total;
+  int heads_per_group;
+};
+
+// Workspace carve-up for one sequence plan (all sequences share the regions; the
+// query takes the maximum over the sequences of the view).
+ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int head_dim) {
+  ScoreLayout L;
+  const size_t per_head = (size_t)sp.Nfft * head_dim * sizeof(float2);
+  int hg = (int)(h->group_bytes / per_head);
+  if (hg < 1) hg = 1;
+  if (hg > num_heads) hg = num_heads;
+  L.heads_per_group = hg;
+  size_t off = 0;
+  L.off_ws = off;       off += align_up(per_head * hg, 256);
+  L.off_spec = off;     off += sp.bluestein ? align_up((size_t)sp.N * head_dim * hg * sizeof(float2), 256) : 0;
+  L.off_hhat = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * sizeof(float2), 256) : 0;
+  L.off_hcol = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * 8 * sizeof(float2), 256) : 0;
+  const size_t slices = (size_t)num_heads * head_dim / sp.cs;
+  L.off_part_tot = off; off += align_up(slices * sp.N2 * 2 * sizeof(double), 256);
+  L.off_part_hi = off;  off += align_up((size_t)num_heads * sp.N2 * 2 * sizeof(double), 256);
+  L.total = off;
+  return L;
+}
+
+fc_status validate_view(const fc_handle *h, const fc_kv_view *kv) {
+  if (!h || !kv || !kv->k || !kv->v || !kv->cu_seqlens) return FC_ERR_INVALID_ARG;
+  if (kv->num_heads <= 0 || kv->head_dim <= 0 || kv->batch < 0) return FC_ERR_INVALID_ARG;
+  if (kv->dtype != FC_F32 && kv->dtype != FC_F16 && kv->dtype != FC_BF16) return FC_ERR_UNSUPPORTED;
+  if (kv->head_dim % 64 != 0) return FC_ERR_UNSUPPORTED;
+  const size_t es = kv->dtype == FC_F32 ? 4 : 2;
+  if (kv->cu_seqlens[0] != 0) return FC_ERR_INVALID_ARG;
+  for (int b = 0; b < kv->batch; ++b) {
+    const long long n = (long long)kv->cu_seqlens[b + 1] - kv->cu_seqlens[b];
+    if (n < 0) return FC_ERR_INVALID_ARG;
+    if (n > h->max_seqlen) return FC_ERR_UNSUPPORTED;
+    if (n > 65536 && !is_pow2((int)n)) return FC_ERR_UNSUPPORTED;
+  }
+  if (kv->stride_token < (long long)kv->head_dim || kv->stride_head < (long long)kv->head_dim)
+    return FC_ERR_INVALID_ARG;
+  if (((uintptr_t)kv->k & 15) || ((uintptr_t)kv->v & 15)) return FC_ERR_INVALID_ARG;
+  if ((kv->stride_token * es) % 16 || (kv->stride_head * es) % 16) return FC_ERR_INVALID_ARG;
+  return FC_OK;
+}
+
+template <class Kern>
+fc_status set_smem(Kern kern, size_t bytes) {
+  if (bytes > 48 * 1024) FC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+  return FC_OK;
+}
+
+size_t smem_pass13(const SeqPlan &sp, int cs) {
+  return (size_t)sp.N1 * cs * sizeof(float2) + sp.N1 * sizeof(float2) + sp.N1 * sizeof(int) + 2 * sp.N1 * sizeof(float);
+}
+size_t smem_pass2(const SeqPlan &sp, int cs2) {
+  return (size_t)sp.N2 * 2 * cs2 * sizeof(float2) + 3 * (size_t)sp.N2 * sizeof(float2) + 2 * (size_t)sp.N2 * sizeof(unsigned short);
+}
+
+template <class Loader>
+fc_status launch_pass1(fc_handle *h, cudaStream_t st, const Loader &ld, const SeqPlan &sp, int ncol_ws, int cs,
+                       float2 *ws, double *partial) {
+  const FftPlan p1 = make_plan(sp.N1);
+  const size_t sm = smem_pass13(sp, cs);
+  fc_status s = set_smem(k_pass1<Loader>, sm);
+  if (s != FC_OK) return s;
+  dim3 grid(sp.N2, ncol_ws / cs);
+  k_pass1<Loader><<<grid, kThreads, sm, st>>>(ld, p1, sp.N2, ncol_ws, ilog2(cs), ws, h->master, h->master_len, partial);
+  return fc_after_launch(h);
+}
+
+template <int MID>
+fc_status launch_pass2(fc_handle *h, cudaStream_t st, const SeqPlan &sp, int ncol_ws, int cs2, float2 *ws,
+                       int omega, float2 *hhat, float scale) {
+  const FftPlan p2 = make_plan(sp.N2);
+  const size_t sm = smem_pass2(sp, cs2);
+  fc_status s = set_smem(k_pass2<MID>, sm);
+  if (s != FC_OK) return s;
+  dim3 grid(MID == MID_DCT ? sp.N1 / 2 + 1 : sp.N1, ncol_ws / cs2);
+  k_pass2<MID><<<grid, kThreads, sm, st>>>(p2, sp.N1, ncol_ws, ilog2(cs2), ws, h->master, h->master_len, omega, hhat, scale);
+  return fc_after_launch(h);
+}
+
+template <typename T>
+fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, int b, double gamma,
+                         float *scores, double *energy, char *wsb) {
+  const int start = kv->cu_seqlens[b];
+  const int N = kv->cu_seqlens[b + 1] - start;
+  const long long total_tokens = kv->cu_seqlens[kv->batch];
+  double *energy_b = energy + 4 * (size_t)b;
+  if (N == 0) {
+    k_zero_energy<<<1, 32, 0, st>>>(energy_b);
+    return fc_after_launch(h);
+  }
+  const int d = kv->head_dim, H = kv->num_heads;
+  const SeqPlan sp = plan_sequence(N);
+  const ScoreLayout L = layout_for(h, sp, H, d);
+  long long om = (long long)floor(gamma * (double)N);
+  if (om > N - 1) om = N - 1;
+  if (om < 0) om = 0;
+  const int omega = (int)om;
+
+  float2 *ws = reinterpret_cast<float2 *>(wsb + L.off_ws);
+  float2 *spec = reinterpret_cast<float2 *>(wsb + L.off_spec);
+  float2 *hhat = reinterpret_cast<float2 *>(wsb + L.off_hhat);
+  float2 *hcol = reinterpret_cast<float2 *>(wsb + L.off_hcol);
+  double *part_tot = reinterpret_cast<double *>(wsb + L.off_part_tot);
+  double *part_hi = reinterpret_cast<double *>(wsb + L.off_part_hi);
+  const T *kp = static_cast<const T *>(kv->k) + (long long)start * kv->stride_token;
+  const T *vp = static_cast<const T *>(kv->v) + (long long)start * kv->stride_token;
+  const FftPlan p1 = make_plan(sp.N1);
+  fc_status s;
+
+  if (sp.bluestein) {
+    // spectrum of the chirp kernel, once per sequence
+    ChirpKernelLoader cl{N, sp.Nfft};
+    if ((s = launch_pass1(h, st, cl, sp, 8, 8, hcol, nullptr)) != FC_OK) return s;
+    if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
+  }
+
+  size_t tot_slots = 0, hi_slots = 0;
+  for (int h0 = 0; h0 < H; h0 += L.heads_per_group) {
+    const int hg = (H - h0 < L.heads_per_group) ? H - h0 : L.heads_per_group;
+    const int ncol_ws = hg * d;
+    double *ptot = part_tot + 2 * tot_slots;
+    double *phi = part_hi + 2 * hi_slots;
+    const size_t sm3 = smem_pass13(sp, sp.cs);
+    if (!sp.bluestein) {
+      KvLoader<T, false> ld{kp, vp, kv->stride_token, kv->stride_head, h0, d, N, 0.f, 0.f};
+      if ((s = launch_pass1(h, st, ld, sp, ncol_ws, sp.cs, ws, ptot)) != FC_OK) return s;
+      if ((s = launch_pass2<MID_DCT>(h, st, sp, ncol_ws, sp.cs2, ws, omega, nullptr, 1.f / (float)N)) != FC_OK) return s;
+      if ((s = set_smem(k_pass3<EPI_SCORE, false>, sm3)) != FC_OK) return s;
+      k_pass3<EPI_SCORE, false><<<dim3(sp.N2, hg), kThreads, sm3, st>>>(
+          p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, nullptr, scores + start, h0, d,
+          total_tokens, 1.f / (float)d, phi);
+      if ((s = fc_after_launch(h)) != FC_OK) return s;
+    } else {
+      const float invM = 1.f / (float)sp.Nfft;
+      KvLoader<T, true> ld{kp, vp, kv->stride_token, kv->stride_head, h0, d, N, 0.f, 0.f};
+      if ((s = launch_pass1(h, st, ld, sp, ncol_ws, sp.cs, ws, ptot)) != FC_OK) return s;
+      if ((s = launch_pass2<MID_MULH>(h, st, sp, ncol_ws, sp.cs2, ws, 0, hhat, invM)) != FC_OK) return s;
+      if ((s = set_smem(k_pass3<EPI_SPEC, true>, sm3)) != FC_OK) return s;
+      k_pass3<EPI_SPEC, true><<<dim3(sp.N2, ncol_ws / sp.cs), kThreads, sm3, st>>>(
+          p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, spec, nullptr, 0, d, 0, 0.f, nullptr);
+      if ((s = fc_after_launch(h)) != FC_OK) return s;
+      FilterLoader fl{spec, ncol_ws, N, omega};
+      if ((s = launch_pass1(h, st, fl, sp, ncol_ws, sp.cs, ws, nullptr)) != FC_OK) return s;
+      if ((s = launch_pass2<MID_MULH>(h, st, sp, ncol_ws, sp.cs2, ws, 0, hhat, invM)) != FC_OK) return s;
+      if ((s = set_smem(k_pass3<EPI_SCORE, true>, sm3)) != FC_OK) return s;
+      const float inv = (float)(1.0 / ((double)N * (double)N * (double)d));
+      k_pass3<EPI_SCORE, true><<<dim3(sp.N2, hg), kThreads, sm3, st>>>(
+          p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, nullptr, scores + start, h0, d,
+          total_tokens, inv, phi);
+      if ((s = fc_after_launch(h)) != FC_OK) return s;
+    }
+    tot_slots += (size_t)sp.N2 * (ncol_ws / sp.cs);
+    hi_slots += (size_t)sp.N2 * hg;
+  }
+  k_energy_finalize<<<1, 256, 0, st>>>(part_tot, (int)tot_slots, part_hi, (int)hi_slots, energy_b);
+  return fc_after_launch(h);
+}
+
+}  // namespace
+
+extern "C" size_t fc_score_workspace_bytes(const fc_handle *h, const fc_kv_view *kv) {
+  if (validate_view(h, kv) != FC_OK) return 0;
+  size_t need = 256;
+  for (int b = 0; b < kv->batch; ++b) {
+    const int N = kv->cu_seqlens[b + 1] - kv->cu_seqlens[b];
+    if (N == 0) continue;
+    const ScoreLayout L = layout_for(h, plan_sequence(N), kv->num_heads, kv->head_dim);
+    if (L.total > need) need = L.total;
+  }
+  return need;
+}
+
+extern "C" fc_status fc_score_layer(fc_handle *h, const fc_kv_view *kv, double gamma, float *scores,
+                                    double *energy, void *workspace, size_t workspace_bytes,
+                                    fc_stream stream) {
+  fc_status s = validate_view(h, kv);
+  if (s != FC_OK) return s;
+  if (!scores || !energy) return FC_ERR_INVALID_ARG;
+  if (!(gamma >= 0.0 && gamma <= 1.0)) return FC_ERR_INVALID_ARG;
+  const size_t need = fc_score_workspace_bytes(h, kv);
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return FC_ERR_WORKSPACE;
+  int dev = -1;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  for (int b = 0; b < kv->batch && s == FC_OK; ++b) {
+    switch (kv->dtype) {
+      case FC_F32: s = score_sequence<float>(h, st, kv, b, gamma, scores, energy, (char *)workspace); break;
+      case FC_F16: s = score_sequence<__half>(h, st, kv, b, gamma, scores, energy, (char *)workspace); break;
+      default: s = score_sequence<__nv_bfloat16>(h, st, kv, b, gamma, scores, energy, (char *)workspace); break;
+    }
+  }
+  return s;
+}

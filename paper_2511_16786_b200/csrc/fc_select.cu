@@ -1,0 +1,381 @@
+// fc_allocate_budgets (Dynamic Budget Allocation Module, Sec. 3.2.2) and
+// fc_select_compact (keep the Outlier KVs by budget, Sec. 3.2.1 last sentence):
+// fp64 budget arithmetic in one small kernel, an exact radix select per
+// (sequence, head) on the fp32 score bits, an ordered compaction of the chosen
+// token indices, and a row gather into the dense compacted cache.
+//
+// This file is compiled with -fmad=false so that the fp64 budget arithmetic is
+// the plain IEEE sequence of multiplies, adds and divides it is written as.
+#include "fc_common.cuh"
+
+#include <math.h>
+
+namespace {
+
+constexpr int kSeqChunk = 64;          // sequences described per launch (kernel-argument table)
+struct SeqTable {
+  int start[kSeqChunk + 1];            // token offsets of the chunk's sequences (cu_seqlens slice)
+};
+
+// ---------------------------------------------------------------------------
+// budgets
+// ---------------------------------------------------------------------------
+__device__ double filled_sum(const double *w, int L, double lam, double lo, double hi) {
+  double s = 0.0;
+  for (int l = 0; l < L; ++l) {
+    double q = lam * w[l];
+    q = q < lo ? lo : (q > hi ? hi : q);
+    s += q;
+  }
+  return s;
+}
+
+// One block per sequence of the chunk.  Shared memory: w[L], cand[2L], fval[2L], frac[L], order[L].
+__global__ void __launch_bounds__(256)
+k_allocate(const double *__restrict__ energy, int L, int B, int b0, SeqTable st, double rho,
+           int min_keep, int *__restrict__ budgets) {
+  extern __shared__ double sh[];
+  double *w = sh;
+  double *cand = w + L;
+  double *fval = cand + 2 * L;
+  double *frac = fval + 2 * L;
+  int *order = reinterpret_cast<int *>(frac + L);
+  __shared__ double s_sum;
+  __shared__ int s_bad;
+  const int tid = threadIdx.x;
+  const int b = b0 + blockIdx.x;
+  const int N = st.start[blockIdx.x + 1] - st.start[blockIdx.x];
+  if (N == 0) {
+    for (int l = tid; l < L; l += blockDim.x) budgets[(size_t)l * B + b] = 0;
+    return;
+  }
+  const double lo = (double)(min_keep < N ? (min_keep < 0 ? 0 : min_keep) : N);
+  const double hi = (double)N;
+  double bt = floor(rho * (double)N * (double)L + 0.5);
+  if (bt < (double)L * lo) bt = (double)L * lo;
+  if (bt > (double)L * hi) bt = (double)L * hi;
+  const long long B_tot = (long long)bt;
+
+  // R^l = hiK/totK + hiV/totV   (Eq. 12)
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+  for (int l = tid; l < L; l += blockDim.x) {
+    const double *e = energy + ((size_t)l * B + b) * 4;
+    const double rk = e[1] > 0.0 ? e[0] / e[1] : 0.0;
+    const double rv = e[3] > 0.0 ? e[2] / e[3] : 0.0;
+    const double R = rk + rv;
+    w[l] = R;
+    if (!(R >= 0.0) || isinf(R)) s_bad = 1;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double s = 0.0;
+    for (int l = 0; l < L; ++l) s += w[l];
+    if (!(s > 0.0) || isinf(s) || isnan(s)) s_bad = 1;
+    s_sum = s;
+  }
+  __syncthreads();
+  const bool uniform = s_bad != 0;
+  const double total = s_sum;
+  __syncthreads();
+  for (int l = tid; l < L; l += blockDim.x) w[l] = uniform ? 1.0 / (double)L : w[l] / total;
+  __syncthreads();
+
+  // kinks of f(lam) = sum clamp(lam*w, lo, hi) and f at each of them
+  for (int i = tid; i < 2 * L; i += blockDim.x) {
+    const double wl = w[i >> 1];
+    cand[i] = wl > 0.0 ? ((i & 1) ? hi / wl : lo / wl) : INFINITY;
+  }
+  __syncthreads();
+  for (int i = tid; i < 2 * L; i += blockDim.x)
+    fval[i] = isinf(cand[i]) ? -1.0 : filled_sum(w, L, cand[i], lo, hi);
+  __syncthreads();
+
+  if (tid == 0) {
+    // smallest kink b* > 0 with f(b*) >= B_tot, and the largest kink a* < b* (0 counts as a kink)
+    double bstar = INFINITY, fb = 0.0, kmax = 0.0;
+    for (int i = 0; i < 2 * L; ++i) {
+      if (isinf(cand[i])) continue;
+      if (cand[i] > kmax) kmax = cand[i];
+      if (cand[i] > 0.0 && fval[i] >= (double)B_tot && cand[i] < bstar) { bstar = cand[i]; fb = fval[i]; }
+    }
+    double lam;
+    if (isinf(bstar)) {
+      lam = kmax;
+    } else {
+      double astar = 0.0;
+      for (int i = 0; i < 2 * L; ++i)
+        if (!isinf(cand[i]) && cand[i] < bstar && cand[i] > astar) astar = cand[i];
+      const double fa = filled_sum(w, L, astar, lo, hi);
+      lam = (fb == fa) ? astar : astar + ((double)B_tot - fa) * (bstar - astar) / (fb - fa);
+    }
+    long long sum = 0;
+    for (int l = 0; l < L; ++l) {
+      double q = lam * w[l];
+      q = q < lo ? lo : (q > hi ? hi : q);
+      const double fl = floor(q);
+      frac[l] = q - fl;
+      budgets[(size_t)l * B + b] = (int)fl;
+      sum += (long long)fl;
+    }
+    s_sum = (double)(B_tot - sum);     // deficit
+  }
+  __syncthreads();
+  // order by (fraction descending, layer ascending)
+  for (int l = tid; l < L; l += blockDim.x) {
+    int rank = 0;
+    const double f = frac[l];
+    for (int m = 0; m < L; ++m) rank += (frac[m] > f || (frac[m] == f && m < l)) ? 1 : 0;
+    order[rank] = l;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    long long deficit = (long long)s_sum;
+    while (deficit > 0) {
+      bool gave = false;
+      for (int r = 0; r < L && deficit > 0; ++r) {
+        int *bl = &budgets[(size_t)order[r] * B + b];
+        if (*bl < N) { *bl += 1; --deficit; gave = true; }
+      }
+      if (!gave) break;
+    }
+  }
+}
+
+__global__ void k_offsets(const int *__restrict__ budgets, int L, int B, long long *__restrict__ out_offsets) {
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= L) return;
+  long long acc = 0;
+  out_offsets[(size_t)l * (B + 1)] = 0;
+  for (int b = 0; b < B; ++b) {
+    acc += budgets[(size_t)l * B + b];
+    out_offsets[(size_t)l * (B + 1) + b + 1] = acc;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// selection
+// ---------------------------------------------------------------------------
+// Monotone map float -> uint32: larger score, larger key.  NaN ranks with +inf, -0 with +0.
+__device__ __forceinline__ unsigned score_key(float x) {
+  if (x != x) return 0xFF800000u;
+  if (x == 0.f) return 0x80000000u;
+  const unsigned u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+constexpr int kSelThreads = 1024;
+
+// Exclusive rank of a 1-bit flag over the block plus the block total.
+__device__ __forceinline__ int block_rank(bool flag, int *wcount, int &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned m = __ballot_sync(0xffffffffu, flag);
+  if (lane == 0) wcount[warp] = __popc(m);
+  __syncthreads();
+  int before = 0, all = 0;
+#pragma unroll
+  for (int i = 0; i < kSelThreads / 32; ++i) {
+    const int c = wcount[i];
+    before += (i < warp) ? c : 0;
+    all += c;
+  }
+  __syncthreads();
+  total = all;
+  return before + __popc(m & ((1u << lane) - 1u));
+}
+
+// grid (sequences in chunk, heads)
+__global__ void __launch_bounds__(kSelThreads)
+k_select(const float *__restrict__ scores, long long T, SeqTable st, int b0,
+         const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
+         int *__restrict__ out_idx, long long cap, int *__restrict__ status) {
+  __shared__ int hist[256];
+  __shared__ int wcount[kSelThreads / 32];
+  __shared__ unsigned s_prefix;
+  __shared__ int s_krem;
+  const int tid = threadIdx.x;
+  const int b = b0 + blockIdx.x, h = blockIdx.y;
+  const int s0 = st.start[blockIdx.x];
+  const int n = st.start[blockIdx.x + 1] - s0;
+  int k = budgets[b];
+  k = k < 0 ? 0 : (k > n ? n : k);
+  const long long off = out_offsets[b];
+  if (k == 0) return;
+  if (off < 0 || off + k > cap) {
+    if (tid == 0) atomicOr(status, FC_DEV_FLAG_INTERNAL);
+    return;
+  }
+  const float *sc = scores + (long long)h * T + s0;
+  int *dst = out_idx + (long long)h * cap + off;
+
+  unsigned tau = 0;
+  int need = 0;            // how many keys equal to tau are kept (lowest indices first)
+  const bool take_all = (k == n);
+  if (!take_all) {
+    unsigned prefix = 0, mask = 0;
+    int krem = k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
+      __syncthreads();
+      for (int i = tid; i < n; i += kSelThreads) {
+        const unsigned key = score_key(sc[i]);
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int cum = 0, dsel = 0;
+        for (int dgt = 255; dgt >= 0; --dgt) {
+          const int c = hist[dgt];
+          if (cum + c >= krem) { dsel = dgt; break; }
+          cum += c;
+        }
+        s_krem = krem - cum;
+        s_prefix = prefix | ((unsigned)dsel << shift);
+      }
+      __syncthreads();
+      krem = s_krem;
+      prefix = s_prefix;
+      mask |= 0xFFu << shift;
+      __syncthreads();
+    }
+    tau = prefix;
+    need = krem;
+  }
+
+  int written = 0, ties_seen = 0;
+  for (int base = 0; base < n; base += kSelThreads) {
+    const int i = base + tid;
+    const bool valid = i < n;
+    const unsigned key = valid ? score_key(sc[i]) : 0u;
+    bool sel = valid;
+    if (!take_all) {
+      const bool is_tie = valid && key == tau;
+      int ties_total;
+      const int tr = block_rank(is_tie, wcount, ties_total);
+      sel = valid && (key > tau || (is_tie && ties_seen + tr < need));
+      ties_seen += ties_total;
+    }
+    int sel_total;
+    const int r = block_rank(sel, wcount, sel_total);
+    if (sel) dst[written + r] = i;
+    written += sel_total;
+  }
+}
+
+// One warp per (compacted row, head): copies the K row and the V row, 16 bytes per lane.
+__global__ void __launch_bounds__(256)
+k_gather(const char *__restrict__ k, const char *__restrict__ v, long long stride_token_b,
+         long long stride_head_b, int row_bytes, int H, SeqTable st, int b0, int nseq,
+         const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
+         const int *__restrict__ out_idx, long long cap, char *__restrict__ out_k,
+         char *__restrict__ out_v) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const long long row_lo = out_offsets[b0], row_hi = out_offsets[b0 + nseq];
+  const long long items = (row_hi - row_lo) * H;
+  const int n16 = row_bytes >> 4;
+  for (long long it = warp; it < items; it += nwarps) {
+    const long long r = row_lo + it / H;
+    const int h = (int)(it % H);
+    if (r >= cap) continue;
+    int bl = 0;
+    while (bl + 1 < nseq && out_offsets[b0 + bl + 1] <= r) ++bl;
+    const int n = st.start[bl + 1] - st.start[bl];
+    int kk = budgets[b0 + bl];
+    kk = kk > n ? n : kk;
+    const long long off_b = out_offsets[b0 + bl];
+    if (r - off_b >= kk || off_b < 0 || off_b + kk > cap) continue;   // same rule as the selection kernel
+    const long long tok = (long long)st.start[bl] + out_idx[(long long)h * cap + r];
+    const long long src = tok * stride_token_b + (long long)h * stride_head_b;
+    const long long dsto = (r * H + h) * (long long)row_bytes;
+    for (int u = lane; u < 2 * n16; u += 32) {
+      const bool isv = u >= n16;
+      const int uu = isv ? u - n16 : u;
+      const uint4 val = *reinterpret_cast<const uint4 *>((isv ? v : k) + src + 16ll * uu);
+      *reinterpret_cast<uint4 *>((isv ? out_v : out_k) + dsto + 16ll * uu) = val;
+    }
+  }
+}
+
+fc_status check_cu(const int32_t *cu, int batch) {
+  if (!cu || batch < 0 || cu[0] != 0) return FC_ERR_INVALID_ARG;
+  for (int b = 0; b < batch; ++b)
+    if (cu[b + 1] < cu[b]) return FC_ERR_INVALID_ARG;
+  return FC_OK;
+}
+
+}  // namespace
+
+extern "C" fc_status fc_allocate_budgets(fc_handle *h, const double *energy, int32_t num_layers,
+                                         int32_t batch, const int32_t *cu_seqlens_host, double rho,
+                                         int32_t min_keep, int32_t *budgets, int64_t *out_offsets,
+                                         fc_stream stream) {
+  if (!h || !energy || !budgets || !out_offsets) return FC_ERR_INVALID_ARG;
+  if (num_layers < 1 || batch < 0 || min_keep < 0) return FC_ERR_INVALID_ARG;
+  if (!(rho >= 0.0) || isinf(rho)) return FC_ERR_INVALID_ARG;
+  if (num_layers > 1024) return FC_ERR_UNSUPPORTED;
+  fc_status s = check_cu(cu_seqlens_host, batch);
+  if (s != FC_OK) return s;
+  int dev = -1;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int L = num_layers;
+  const size_t sm = (size_t)(6 * L) * sizeof(double) + (size_t)L * sizeof(int);
+  for (int b0 = 0; b0 < batch; b0 += kSeqChunk) {
+    const int nseq = batch - b0 < kSeqChunk ? batch - b0 : kSeqChunk;
+    SeqTable tab;
+    for (int i = 0; i <= nseq; ++i) tab.start[i] = cu_seqlens_host[b0 + i];
+    k_allocate<<<nseq, 256, sm, st>>>(energy, L, batch, b0, tab, rho, min_keep, budgets);
+    if ((s = fc_after_launch(h)) != FC_OK) return s;
+  }
+  k_offsets<<<(L + 127) / 128, 128, 0, st>>>(budgets, L, batch, reinterpret_cast<long long *>(out_offsets));
+  return fc_after_launch(h);
+}
+
+extern "C" size_t fc_select_workspace_bytes(const fc_handle *h, const fc_kv_view *kv) {
+  if (!h || !kv) return 0;
+  return 256;   // the selection keeps its state on chip; a token amount so callers can treat both phases alike
+}
+
+extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const float *scores,
+                                       const int32_t *budgets, const int64_t *out_offsets,
+                                       void *out_k, void *out_v, int32_t *out_idx,
+                                       int64_t out_capacity_rows, void *workspace,
+                                       size_t workspace_bytes, fc_stream stream) {
+  if (!h || !kv || !kv->k || !kv->v || !scores || !budgets || !out_offsets || !out_k || !out_v || !out_idx)
+    return FC_ERR_INVALID_ARG;
+  if (kv->num_heads <= 0 || kv->head_dim <= 0 || out_capacity_rows < 0) return FC_ERR_INVALID_ARG;
+  if (kv->dtype != FC_F32 && kv->dtype != FC_F16 && kv->dtype != FC_BF16) return FC_ERR_UNSUPPORTED;
+  const int es = kv->dtype == FC_F32 ? 4 : 2;
+  if ((kv->head_dim * es) % 16) return FC_ERR_UNSUPPORTED;
+  fc_status s = check_cu(kv->cu_seqlens, kv->batch);
+  if (s != FC_OK) return s;
+  if (((uintptr_t)kv->k & 15) || ((uintptr_t)kv->v & 15) || ((uintptr_t)out_k & 15) || ((uintptr_t)out_v & 15))
+    return FC_ERR_INVALID_ARG;
+  if ((kv->stride_token * es) % 16 || (kv->stride_head * es) % 16) return FC_ERR_INVALID_ARG;
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < fc_select_workspace_bytes(h, kv))
+    return FC_ERR_WORKSPACE;
+  int dev = -1;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const long long T = kv->cu_seqlens[kv->batch];
+  for (int b0 = 0; b0 < kv->batch; b0 += kSeqChunk) {
+    const int nseq = kv->batch - b0 < kSeqChunk ? kv->batch - b0 : kSeqChunk;
+    SeqTable tab;
+    for (int i = 0; i <= nseq; ++i) tab.start[i] = kv->cu_seqlens[b0 + i];
+    k_select<<<dim3(nseq, kv->num_heads), kSelThreads, 0, st>>>(
+        scores, T, tab, b0, budgets, reinterpret_cast<const long long *>(out_offsets), out_idx,
+        out_capacity_rows, h->status_word);
+    if ((s = fc_after_launch(h)) != FC_OK) return s;
+    k_gather<<<h->num_sms * 8, 256, 0, st>>>(
+        static_cast<const char *>(kv->k), static_cast<const char *>(kv->v),
+        kv->stride_token * es, kv->stride_head * es, kv->head_dim * es, kv->num_heads, tab, b0, nseq,
+        budgets, reinterpret_cast<const long long *>(out_offsets), out_idx, out_capacity_rows,
+        static_cast<char *>(out_k), static_cast<char *>(out_v));
+    if ((s = fc_after_launch(h)) != FC_OK) return s;
+  }
+  return FC_OK;
+}

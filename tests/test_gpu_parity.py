@@ -1,0 +1,381 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU oracle on
+the same seeded inputs, element by element.
+
+Tolerances (the build's stated bar): score error |g-o| / max(o, 1e-6*e_bar) <= 1e-3
+for fp32 inputs and <= 2e-2 for fp16/bf16 inputs, where e_bar is the head's mean
+of (|k_x|^2+|v_x|^2)/d (so the gamma=1 case, whose true scores are 0, is still
+testable); index sets identical except for tokens whose oracle score is within that
+tolerance of the k-th largest; compacted rows bit-exact given the index set.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import flashcache_oracle as O
+from paper_2511_16786_b200 import synth_kv as S
+
+pytestmark = pytest.mark.gpu
+
+TOL = {torch.float32: 1e-3, torch.float16: 2e-2, torch.bfloat16: 2e-2}
+
+
+@pytest.fixture(scope="module")
+def fc():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    from paper_2511_16786_b200 import binding
+    return binding
+
+
+def _rand_kv(T, H, d, dtype, seed, smooth=True):
+    g = torch.Generator().manual_seed(seed)
+    k = torch.randn((T, H, d), generator=g)
+    v = torch.randn((T, H, d), generator=g)
+    if smooth and T > 1:
+        t = torch.arange(T, dtype=torch.float32)[:, None, None] / T
+        k = 0.3 * k + 3.0 * torch.cos(2.5 * t + torch.randn((1, H, d), generator=g))
+        v = 0.3 * v + 2.0 * t + torch.randn((1, H, d), generator=g)
+    return k.to(dtype), v.to(dtype)
+
+
+def _gpu_scores(fc, k, v, cu, gamma, max_seqlen=None, group_bytes=None):
+    T, H, d = k.shape
+    seqlens = [cu[i + 1] - cu[i] for i in range(len(cu) - 1)]
+    h = fc.fc_create(0, max_seqlen or max(1, max(seqlens, default=1)))
+    try:
+        if group_bytes:
+            fc.fc_set_group_bytes(h, group_bytes)
+        kd, vd = (k if k.is_cuda else k.cuda()), (v if v.is_cuda else v.cuda())
+        scores = torch.full((H, max(T, 1)), -1.0, dtype=torch.float32, device="cuda")
+        energy = torch.full((len(cu) - 1, 4), -1.0, dtype=torch.float64, device="cuda")
+        need = fc.fc_score_workspace_bytes(h, kd, vd, cu)
+        assert need > 0
+        ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        fc.fc_score_layer(h, kd, vd, cu, gamma, scores, energy, ws)
+        assert fc.fc_last_device_status(h) == 0
+        return scores.cpu().numpy().astype(np.float64)[:, :T], energy.cpu().numpy()
+    finally:
+        fc.fc_destroy(h)
+
+
+def _score_errors(g, o, k, v, cu):
+    """max over heads/tokens of |g-o| / max(o, 1e-6*e_bar)."""
+    kk = k.double().numpy()
+    vv = v.double().numpy()
+    worst = 0.0
+    for b in range(len(cu) - 1):
+        s, e = cu[b], cu[b + 1]
+        if e == s:
+            continue
+        for h in range(g.shape[0]):
+            ebar = ((kk[s:e, h] ** 2).sum(1) + (vv[s:e, h] ** 2).sum(1)).mean() / kk.shape[2]
+            den = np.maximum(o[h, s:e], 1e-6 * ebar)
+            worst = max(worst, float((np.abs(g[h, s:e] - o[h, s:e]) / den).max()))
+    return worst
+
+
+def _check_layer(fc, k, v, cu, gamma, **kw):
+    g, en = _gpu_scores(fc, k, v, cu, gamma, **kw)
+    o, eo = O.score_layer(k.double().numpy(), v.double().numpy(), cu, gamma, "fft")
+    err = _score_errors(g, o, k, v, cu)
+    assert err <= TOL[k.dtype], "score error %.3e" % err
+    assert np.all(g >= 0.0)
+    for b in range(len(cu) - 1):
+        if cu[b + 1] == cu[b]:
+            assert not en[b].any()
+            continue
+        tol = 1e-4 if k.dtype == torch.float32 else 2e-2
+        np.testing.assert_allclose(en[b, [1, 3]], eo[b, [1, 3]], rtol=1e-5)
+        scale = eo[b, [1, 3]] * 1e-6
+        assert np.all(np.abs(en[b, [0, 2]] - eo[b, [0, 2]]) <= tol * np.maximum(eo[b, [0, 2]], scale))
+    return g, en
+
+
+# ---------------------------------------------------------------- scores
+@pytest.mark.parametrize("N", [16, 32, 64, 256, 1024, 4096])
+@pytest.mark.parametrize("gamma", [0.2, 1.0])
+def test_scores_power_of_two_fp32(fc, N, gamma):
+    k, v = _rand_kv(N, 2, 128, torch.float32, N)
+    _check_layer(fc, k, v, [0, N], gamma)
+
+
+@pytest.mark.parametrize("N", [1, 2, 3, 5, 8, 17, 100, 257, 1000, 1500, 4099])
+def test_scores_arbitrary_length_fp32(fc, N):
+    k, v = _rand_kv(N, 2, 64, torch.float32, 100 + N)
+    _check_layer(fc, k, v, [0, N], 0.2)
+
+
+@pytest.mark.parametrize("gamma", [0.0, 0.0003, 0.1, 0.5, 0.77, 1.0])
+def test_scores_cutoff_sweep(fc, gamma):
+    k, v = _rand_kv(512, 1, 128, torch.float32, 7)
+    _check_layer(fc, k, v, [0, 512], gamma)
+    k, v = _rand_kv(300, 1, 128, torch.float32, 8)
+    _check_layer(fc, k, v, [0, 300], gamma)
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("N", [2048, 777])
+def test_scores_16bit_inputs(fc, dtype, N):
+    k, v = _rand_kv(N, 3, 128, dtype, 11)
+    _check_layer(fc, k, v, [0, N], 0.2)
+
+
+def test_scores_ragged_batch_with_empty_sequence(fc):
+    lens = [64, 0, 300, 1024, 17, 2048]
+    cu = [0] + list(np.cumsum(lens))
+    cu = [int(x) for x in cu]
+    k, v = _rand_kv(cu[-1], 2, 128, torch.bfloat16, 5)
+    _check_layer(fc, k, v, cu, 0.2, max_seqlen=4096)
+
+
+def test_scores_strided_view_and_small_groups(fc):
+    # K and V live inside a wider buffer (extra heads, padded channels); tiny transform groups
+    N, H, d = 1024, 4, 128
+    big_k, big_v = _rand_kv(N, H + 2, d + 64, torch.float16, 3)
+    k, v = big_k[:, 1:1 + H, :d], big_v[:, 1:1 + H, :d]
+    kd, vd = big_k.cuda()[:, 1:1 + H, :d], big_v.cuda()[:, 1:1 + H, :d]
+    assert not kd.is_contiguous()
+    g1, e1 = _gpu_scores(fc, kd, vd, [0, N], 0.2)
+    g2, e2 = _gpu_scores(fc, k.contiguous(), v.contiguous(), [0, N], 0.2, group_bytes=1 << 20)
+    assert np.array_equal(g1, g2) and np.array_equal(e1, e2)
+    o, _ = O.score_layer(k.double().numpy(), v.double().numpy(), [0, N], 0.2, "fft")
+    assert _score_errors(g1, o, k, v, [0, N]) <= 2e-2
+
+
+def test_scores_are_deterministic(fc):
+    k, v = _rand_kv(4096, 2, 128, torch.bfloat16, 9)
+    a = _gpu_scores(fc, k, v, [0, 4096], 0.2)
+    b = _gpu_scores(fc, k, v, [0, 4096], 0.2)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    k, v = _rand_kv(1234, 2, 128, torch.bfloat16, 9)
+    a = _gpu_scores(fc, k, v, [0, 1234], 0.2)
+    b = _gpu_scores(fc, k, v, [0, 1234], 0.2)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("N", [8192, 32768, 65536])
+def test_scores_long_sequences_sampled_head(fc, N):
+    k, v = _rand_kv(N, 1, 128, torch.bfloat16, N)
+    _check_layer(fc, k, v, [0, N], 0.2)
+
+
+def test_scores_long_arbitrary_length(fc):
+    N = 40961
+    k, v = _rand_kv(N, 1, 64, torch.bfloat16, N)
+    _check_layer(fc, k, v, [0, N], 0.2)
+
+
+# ---------------------------------------------------------------- budgets
+def _gpu_budgets(fc, energy, cu, rho, min_keep):
+    L, B = energy.shape[:2]
+    h = fc.fc_create(0, 1024)
+    try:
+        e = torch.from_numpy(np.ascontiguousarray(energy)).cuda()
+        budgets = torch.full((L, B), -7, dtype=torch.int32, device="cuda")
+        offsets = torch.full((L, B + 1), -7, dtype=torch.int64, device="cuda")
+        fc.fc_allocate_budgets(h, e, cu, rho, min_keep, budgets, offsets)
+        assert fc.fc_last_device_status(h) == 0
+        return budgets.cpu().numpy(), offsets.cpu().numpy()
+    finally:
+        fc.fc_destroy(h)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_budgets_match_oracle(fc, seed):
+    rng = np.random.default_rng(seed)
+    L = int(rng.integers(1, 70))
+    B = int(rng.integers(1, 6))
+    lens = [int(x) for x in rng.integers(0, 5000, B)]
+    cu = [0] + [int(x) for x in np.cumsum(lens)]
+    energy = rng.random((L, B, 4))
+    energy[..., 1] += energy[..., 0]
+    energy[..., 3] += energy[..., 2]
+    if seed % 3 == 0:
+        energy[rng.integers(0, L), :, :] = 0.0
+    rho = float(rng.choice([0.05, 0.1, 0.2, 0.6, 1.0]))
+    min_keep = int(rng.choice([0, 1, 8]))
+    gb, go = _gpu_budgets(fc, energy, cu, rho, min_keep)
+    ob, oo = O.allocate_budgets(energy, lens, rho, min_keep)
+    np.testing.assert_array_equal(gb, ob)
+    np.testing.assert_array_equal(go, oo)
+
+
+def test_budgets_special_cases(fc):
+    e = np.zeros((4, 1, 4))
+    gb, go = _gpu_budgets(fc, e, [0, 100], 0.5, 1)            # all-zero energy: uniform
+    assert gb[:, 0].tolist() == [50, 50, 50, 50]
+    e = np.ones((3, 1, 4))
+    e[:, 0, 0] = [0.8, 0.1, 0.1]
+    e[:, 0, 2] = 0.0
+    gb, _ = _gpu_budgets(fc, e, [0, 100], 0.5, 1)             # upper cap binds, rest re-shared
+    assert gb[:, 0].tolist() == [100, 25, 25]
+    e = np.ones((1, 1, 4))
+    gb, go = _gpu_budgets(fc, e, [0, 1024], 0.2, 1)           # one layer: floor(204.8+.5)
+    assert gb.tolist() == [[205]] and go.tolist() == [[0, 205]]
+
+
+# ---------------------------------------------------------------- selection + compaction
+def _gpu_select(fc, k, v, cu, scores, budgets, offsets, capacity):
+    T, H, d = k.shape
+    h = fc.fc_create(0, 65536)
+    try:
+        kd, vd = k.cuda(), v.cuda()
+        sc = torch.from_numpy(np.ascontiguousarray(scores, dtype=np.float32)).cuda()
+        bd = torch.tensor(budgets, dtype=torch.int32, device="cuda")
+        of = torch.tensor(offsets, dtype=torch.int64, device="cuda")
+        out_k = torch.zeros((capacity, H, d), dtype=k.dtype, device="cuda")
+        out_v = torch.zeros((capacity, H, d), dtype=k.dtype, device="cuda")
+        out_idx = torch.full((H, capacity), -1, dtype=torch.int32, device="cuda")
+        ws = torch.empty(fc.fc_select_workspace_bytes(h, kd, vd, cu), dtype=torch.uint8, device="cuda")
+        fc.fc_select_compact(h, kd, vd, cu, sc, bd, of, out_k, out_v, out_idx, ws)
+        status = fc.fc_last_device_status(h)
+        return out_k.cpu(), out_v.cpu(), out_idx.cpu().numpy(), status
+    finally:
+        fc.fc_destroy(h)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_select_exact_on_given_scores(fc, dtype):
+    rng = np.random.default_rng(0)
+    lens = [1, 37, 0, 1024, 3000, 5]
+    cu = [0] + [int(x) for x in np.cumsum(lens)]
+    T, H, d = cu[-1], 3, 128
+    k, v = _rand_kv(T, H, d, dtype, 1, smooth=False)
+    scores = rng.integers(0, 50, (H, T)).astype(np.float32) / 7.0      # heavy ties
+    scores[0, cu[3] + 5] = np.nan
+    scores[1, cu[4]:cu[4] + 10] = np.inf
+    scores[2, cu[4] + 100:cu[4] + 200] = 0.0
+    budgets = [1, 11, 0, 205, 2999, 5]
+    offsets = [0] + [int(x) for x in np.cumsum(budgets)]
+    out_k, out_v, out_idx, status = _gpu_select(fc, k, v, cu, scores, budgets, offsets, offsets[-1] + 3)
+    assert status == 0
+    for h in range(H):
+        for b, n in enumerate(lens):
+            want = O.select_topk(scores[h, cu[b]:cu[b + 1]], budgets[b])
+            got = out_idx[h, offsets[b]:offsets[b + 1]]
+            np.testing.assert_array_equal(got, want)
+            rows = slice(offsets[b], offsets[b + 1])
+            assert torch.equal(out_k[rows, h].view(torch.uint8), k[cu[b] + want, h].contiguous().view(torch.uint8))
+            assert torch.equal(out_v[rows, h].view(torch.uint8), v[cu[b] + want, h].contiguous().view(torch.uint8))
+    assert (out_idx[:, offsets[-1]:] == -1).all()                          # nothing past the last row
+
+
+def test_select_capacity_overflow_is_reported_not_written(fc):
+    k, v = _rand_kv(64, 1, 128, torch.float32, 2, smooth=False)
+    scores = np.arange(64, dtype=np.float32)[None]
+    _, _, out_idx, status = _gpu_select(fc, k, v, [0, 64], scores, [10], [0, 10], 4)
+    assert status != 0
+    assert (out_idx == -1).all()
+
+
+# ---------------------------------------------------------------- whole pass
+def _compare_compress(fc, cfg, layers=None, sample_heads=None, tier="fft"):
+    from paper_2511_16786_b200.binding import Compressor
+    L = cfg.num_layers
+    Ks, Vs = [], []
+    for l in range(L):
+        k, v = S.make_layer(cfg, l, "cpu")
+        Ks.append(k)
+        Vs.append(v)
+    comp = Compressor(L, cfg.num_heads, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho,
+                      cfg.gamma, cfg.min_keep)
+    Kd, Vd = [k.cuda() for k in Ks], [v.cuda() for v in Vs]
+    comp.compress(Kd, Vd)
+    comp.check_device_status()
+    tol = TOL[cfg.torch_dtype]
+    cu = cfg.cu_seqlens
+    g_scores = comp.scores.cpu().numpy().astype(np.float64)
+    g_energy = comp.energy.cpu().numpy()
+    g_budgets = comp.budgets.cpu().numpy()
+    g_offsets = comp.offsets.cpu().numpy()
+    g_idx = comp.out_idx.cpu().numpy()
+    o_energy = np.zeros_like(g_energy)
+    o_scores = []
+    for l in range(L):
+        o, e = O.score_layer(Ks[l].double().numpy(), Vs[l].double().numpy(), cu, cfg.gamma, tier)
+        o_scores.append(o)
+        o_energy[l] = e
+        assert _score_errors(g_scores[l], o, Ks[l], Vs[l], cu) <= tol
+    ob, oo = O.allocate_budgets(o_energy, list(cfg.seqlens), cfg.rho, cfg.min_keep)
+    # budgets: identical, or +-1 swaps where the largest-remainder fractions nearly tie
+    assert g_budgets.sum(axis=0).tolist() == ob.sum(axis=0).tolist()
+    assert np.abs(g_budgets - ob).max() <= 1
+    # the device budgets are exactly what the oracle rule gives on the device's own energies
+    ob2, oo2 = O.allocate_budgets(g_energy, list(cfg.seqlens), cfg.rho, cfg.min_keep)
+    np.testing.assert_array_equal(g_budgets, ob2)
+    np.testing.assert_array_equal(g_offsets, oo2)
+    for l in range(L):
+        for h in range(cfg.num_heads):
+            for b, n in enumerate(cfg.seqlens):
+                kb = int(g_budgets[l, b])
+                got = g_idx[l, h, g_offsets[l, b]:g_offsets[l, b] + kb]
+                assert np.all(np.diff(got) > 0) and (kb == 0 or (got[0] >= 0 and got[-1] < n))
+                osc = o_scores[l][h, cu[b]:cu[b + 1]]
+                want = O.select_topk(osc, kb)
+                diff = np.setxor1d(got, want)
+                if len(diff) and kb > 0:
+                    tau = np.sort(osc)[::-1][kb - 1]
+                    assert np.all(np.abs(osc[diff] - tau) <= tol * tau), "index sets differ away from the threshold"
+                rows = slice(int(g_offsets[l, b]), int(g_offsets[l, b]) + kb)
+                gk = comp.out_k[l][rows, h].cpu().view(torch.uint8)
+                gv = comp.out_v[l][rows, h].cpu().view(torch.uint8)
+                assert torch.equal(gk, Ks[l][cu[b] + got, h].contiguous().view(torch.uint8))
+                assert torch.equal(gv, Vs[l][cu[b] + got, h].contiguous().view(torch.uint8))
+    comp.close()
+    return g_budgets
+
+
+def test_config1_full(fc):
+    cfg = S.paper_configs()["cfg1"]
+    b = _compare_compress(fc, cfg, tier="literal")
+    assert b.tolist() == [[205]]
+
+
+def test_config2_shape_reduced(fc):
+    base = S.paper_configs()["cfg2"]
+    cfg = S.scaled(base, "cfg2_small", num_layers=6, seqlens=(2048,))
+    b = _compare_compress(fc, cfg)
+    assert len(set(b[:, 0].tolist())) > 1        # per-layer outlier fractions give different budgets
+
+
+def test_config4_shape_reduced(fc):
+    base = S.paper_configs()["cfg4"]
+    cfg = S.scaled(base, "cfg4_small", num_layers=3, num_heads=8, seqlens=(1024,))
+    _compare_compress(fc, cfg)
+
+
+def test_config5_shape_reduced_ragged(fc):
+    base = S.paper_configs()["cfg5"]
+    cfg = S.scaled(base, "cfg5_small", num_layers=4, seqlens=(517, 1024, 64, 1999, 333, 4096, 100, 2311))
+    _compare_compress(fc, cfg)
+
+
+# ---------------------------------------------------------------- ABI error paths (host-side checks only)
+def test_abi_rejects_bad_arguments(fc):
+    h = fc.fc_create(0, 1024)
+    try:
+        k, v = _rand_kv(128, 2, 128, torch.float32, 0)
+        kd, vd = k.cuda(), v.cuda()
+        scores = torch.empty((2, 128), dtype=torch.float32, device="cuda")
+        energy = torch.empty((1, 4), dtype=torch.float64, device="cuda")
+        ws = torch.empty(fc.fc_score_workspace_bytes(h, kd, vd, [0, 128]), dtype=torch.uint8, device="cuda")
+        with pytest.raises(fc.FlashCacheError) as e:
+            fc.fc_score_layer(h, kd, vd, [0, 128], 1.5, scores, energy, ws)          # gamma out of range
+        assert e.value.code == 1
+        with pytest.raises(fc.FlashCacheError) as e:
+            fc.fc_score_layer(h, kd, vd, [0, 128], 0.2, scores, energy, ws[:64])     # workspace too small
+        assert e.value.code == 3
+        with pytest.raises(fc.FlashCacheError) as e:
+            fc.fc_score_layer(h, kd, vd, [0, 200, 128], 0.2, scores, energy, ws)     # decreasing cu_seqlens
+        assert e.value.code == 1
+        k2, v2 = _rand_kv(2048, 1, 128, torch.float32, 0)
+        assert fc.fc_score_workspace_bytes(h, k2.cuda(), v2.cuda(), [0, 2048]) == 0  # longer than max_seqlen
+        k3, v3 = _rand_kv(64, 1, 96, torch.float32, 0)
+        assert fc.fc_score_workspace_bytes(h, k3.cuda(), v3.cuda(), [0, 64]) == 0    # head_dim not a multiple of 64
+        assert fc.fc_last_device_status(h) == 0
+    finally:
+        fc.fc_destroy(h)
+    with pytest.raises(fc.FlashCacheError):
+        fc.fc_create(0, 0)
