@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the FlashCache compression pass (score + allocate + select + compact).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg3] [--impl reference]
+
+A step is one pass of the whole hot path over all layers of the workload, inputs
+resident in HBM.  Prints ONE JSON line (rank 0): KV tokens compressed per second,
+the roofline of the dominant kernel measured with CUDA events inside the timed
+region, the same metric end to end from pinned host buffers, the fp64 CPU oracle
+timed on a bounded sample of the same workload, and the SM clocks sampled during
+the timed region.  With N > 1 (launched by torch.distributed.run) every rank
+runs an independent replica of the workload on its own GPU; nothing is exchanged.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "kv_tokens_compressed_per_s"
+UNIT = "tokens/s"
+FP32_LANES_PER_SM = 128          # FP32 FMA lanes per SM on B200
+DEFAULT_CONFIG = "cfg3"          # the 32k-token workload the target fraction is quoted on
+
+# DRAM traffic per launch of the dominant kernel from the committed ncu capture
+# (profiles/), bytes; None until a capture of that kernel and workload exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, sm_max_mhz=1965.0, source="fallback")
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int, period_ms: int = 25):
+        self.out = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=timestamp," + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", str(period_ms)],
+                stdout=self.out, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self, t0_wall: float, t1_wall: float):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"], samples=0)
+        time.sleep(0.05)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.out.flush()
+        self.out.seek(0)
+        import datetime
+        rows = []
+        for line in self.out.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]), parts[4:9]))
+            except ValueError:
+                continue
+        os.unlink(self.out.name)
+        inside = [r for r in rows if t0_wall - 0.02 <= r[0] <= t1_wall + 0.02] or rows
+        if not inside:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"], samples=0)
+        sm = sorted(r[1] for r in inside)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = set()
+        for r in inside:
+            for name, val in zip(names, r[3][1:]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=sm[len(sm) // 2], sm_max_mhz=inside[0][2], reasons=sorted(reasons),
+                    samples=len(inside))
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    ids = [x.strip() for x in vis.split(",") if x.strip()]
+    if local_rank < len(ids) and ids[local_rank].isdigit():
+        return int(ids[local_rank])
+    return local_rank
+
+
+# --------------------------------------------------------------------------- accounting
+def step_accounting(binding, handle, cfg):
+    """Algorithmic flops and HBM bytes of one step, per kernel class (what the shipped
+    algorithm has to compute and move, not what the hardware happened to do)."""
+    d, H, L = cfg.head_dim, cfg.num_heads, cfg.num_layers
+    s = 4 if cfg.dtype == "f32" else 2
+    acc = {k: dict(flops=0.0, bytes=0.0) for k in ("pass1", "pass2", "pass3", "select", "gather")}
+    rows = 0
+    for N in cfg.seqlens:
+        if N == 0:
+            continue
+        plan = binding.fc_describe_plan(handle, N)
+        M, n1, n2 = plan["nfft"], plan["n1"], plan["n2"]
+        cols = H * d * L                       # complex columns (K + jV) of this sequence
+        reps = 2 if plan["bluestein"] else 1   # chirp path: two convolutions, each a forward+inverse transform
+        acc["pass1"]["flops"] += reps * cols * M * 5.0 * math.log2(n1)
+        acc["pass2"]["flops"] += reps * cols * M * (10.0 * math.log2(n2) + 8.0)
+        acc["pass3"]["flops"] += reps * cols * M * 5.0 * math.log2(n1) + cols * N * 4.0
+        acc["pass1"]["bytes"] += N * H * L * 2.0 * d * s               # K and V rows, read once
+        acc["pass3"]["bytes"] += N * H * L * 4.0                       # score write
+        acc["select"]["bytes"] += N * H * L * 4.0                      # score read
+        acc["gather"]["bytes"] += cfg.rho * N * H * L * (4.0 * d * s + 4.0)
+        rows += N * H * L
+    return acc, rows
+
+
+# --------------------------------------------------------------------------- CPU baseline (oracle)
+def oracle_sample(cfg, Ks_host, Vs_host, budget_s: float):
+    """Times the fp64 oracle ("fft" tier, as it stands) on whole layers of the workload until
+    about budget_s seconds are used; returns tokens/s scaled to the full layer count."""
+    import numpy as np
+    from oracle import flashcache_oracle as O
+    L = cfg.num_layers
+    t0 = time.perf_counter()
+    used, scores, energy = 0, [], []
+    while used < len(Ks_host):
+        s, e = O.score_layer(Ks_host[used], Vs_host[used], cfg.cu_seqlens, cfg.gamma, "fft")
+        scores.append(s)
+        energy.append(e)
+        used += 1
+        el = time.perf_counter() - t0
+        if el + el / used > budget_s:
+            break
+    budgets, offsets = O.allocate_budgets(np.stack(energy), list(cfg.seqlens), cfg.rho, cfg.min_keep)
+    cu = cfg.cu_seqlens
+    for l in range(used):
+        for h in range(cfg.num_heads):
+            for b, n in enumerate(cfg.seqlens):
+                idx = O.select_topk(scores[l][h, cu[b]:cu[b + 1]], int(budgets[l, b]))
+                O.compact_rows(Ks_host[l][cu[b]:cu[b + 1], h], idx)
+                O.compact_rows(Vs_host[l][cu[b]:cu[b + 1], h], idx)
+    el = time.perf_counter() - t0
+    tokens_per_s = cfg.total_tokens / (el * L / used)
+    return tokens_per_s, used, el
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, each step a bounded sample (one layer)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2511_16786_b200 import synth_kv as S
+    cfg = S.paper_configs()[args.config]
+    torch.set_num_threads(max(1, os.cpu_count() or 1))
+    K, V = S.make_layer(cfg, 0, "cpu")
+    Ks, Vs = [K.float().numpy()], [V.float().numpy()]
+    times = []
+    for i in range(args.warmup + args.steps):
+        tps, used, el = oracle_sample(cfg, Ks, Vs, budget_s=1e9)
+        if i >= args.warmup:
+            times.append(el)
+    ms = 1000.0 * sum(times) / len(times)
+    value = cfg.total_tokens / ((ms / 1000.0) * cfg.num_layers)
+    sample = "1 of %d layers (all %d heads, all sequences) per step, scaled by the layer count" % (
+        cfg.num_layers, cfg.num_heads)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name + ": " + cfg.note, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# --------------------------------------------------------------------------- main arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", default=DEFAULT_CONFIG)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--group-mib", type=int, default=0, help="transform group size override (MiB)")
+    ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first LAYERS layers")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-budget-s", type=float, default=15.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2511_16786_b200 import binding, synth_kv as S
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if max(args.warmup, 0) < 3:
+        args.warmup = 3
+
+    peaks = load_peaks()
+    cfg = S.paper_configs()[args.config]
+    if args.layers:
+        cfg = S.scaled(cfg, cfg.name, num_layers=args.layers, note=cfg.note + " (first %d layers only)" % args.layers)
+    dev = torch.device("cuda", local_rank)
+    L = cfg.num_layers
+    Kd, Vd = [], []
+    for l in range(L):
+        k, v = S.make_layer(cfg, l, dev)
+        Kd.append(k)
+        Vd.append(v)
+    comp = binding.Compressor(L, cfg.num_heads, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho,
+                              cfg.gamma, cfg.min_keep, device=local_rank,
+                              group_bytes=(args.group_mib << 20) if args.group_mib else None)
+    input_bytes = sum(k.numel() * k.element_size() * 2 for k in Kd)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    t_load0 = time.time()
+    for _ in range(args.warmup):
+        comp.compress(Kd, Vd)
+    torch.cuda.synchronize()
+    comp.check_device_status()
+
+    # which kernel class dominates: one profiled (untimed) step per class
+    shares = {}
+    for name, cls in binding.KERNEL_CLASSES.items():
+        binding.fc_profile_begin(comp.handle, cls)
+        comp.compress(Kd, Vd)
+        ms, n = binding.fc_profile_end(comp.handle)
+        shares[name] = dict(ms=ms, launches=n)
+    dominant = max((k for k in shares if k != "other"), key=lambda k: shares[k]["ms"])
+
+    # timed region
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    launches0 = binding.fc_launch_count(comp.handle)
+    binding.fc_profile_begin(comp.handle, binding.KERNEL_CLASSES[dominant],
+                             max(1, shares[dominant]["launches"]) * args.steps + 8)
+    t_wall0 = time.time()
+    ev0.record()
+    for _ in range(args.steps):
+        comp.compress(Kd, Vd)
+    ev1.record()
+    barrier()
+    t_wall1 = time.time()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    dom_ms, dom_launches = binding.fc_profile_end(comp.handle)
+    launches = binding.fc_launch_count(comp.handle) - launches0
+    clocks = sampler.stop(t_wall0, t_wall1)
+    comp.check_device_status()
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    tokens = cfg.total_tokens
+    value = tokens * world / (ms_per_step / 1000.0)
+
+    # roofline of the dominant kernel and of the whole step
+    acc, rows = step_accounting(binding, comp.handle, cfg)
+    props = torch.cuda.get_device_properties(dev)
+    alu_peak = props.multi_processor_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # TFLOP/s
+    d_acc = acc[dominant]
+    dom_s = dom_ms / 1000.0 / max(1, args.steps)            # device seconds of that class per step
+    t_alu = d_acc["flops"] / (alu_peak * 1e12)
+    t_hbm = d_acc["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    if t_alu >= t_hbm:
+        roof = dict(bound="alu", achieved=d_acc["flops"] / dom_s / 1e12, peak=alu_peak, unit="TFLOP/s")
+    else:
+        roof = dict(bound="hbm", achieved=d_acc["bytes"] / dom_s / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((args.config, dominant))
+    roof.update(kernel=dominant, launches_per_step=dom_launches / max(1, args.steps),
+                avg_launch_us=1000.0 * dom_ms / max(1, dom_launches), peak_source=(
+                    "%d SMs x %d FP32 lanes x 2 x %.0f MHz" % (props.multi_processor_count, FP32_LANES_PER_SM,
+                                                              peaks["sm_max_mhz"])
+                    if roof["bound"] == "alu" else "MEASURED_PEAKS.json hbm_gbs (%s)" % peaks["source"]),
+                share_of_step=dom_s / (ms_per_step / 1000.0),
+                class_ms_per_step={k: v["ms"] for k, v in shares.items()})
+    s = 4 if cfg.dtype == "f32" else 2
+    step_bytes = rows * (2.0 * cfg.head_dim * s + 8.0 + cfg.rho * (4.0 * cfg.head_dim * s + 4.0))
+    step_flops = sum(v["flops"] for v in acc.values())
+    t_bound = max(step_bytes / (peaks["hbm_gbs"] * 1e9), step_flops / (alu_peak * 1e12))
+    roof_step = dict(bound="alu" if step_flops / (alu_peak * 1e12) >= step_bytes / (peaks["hbm_gbs"] * 1e9) else "hbm",
+                     t_bound_ms=1000.0 * t_bound, frac=t_bound / (ms_per_step / 1000.0),
+                     gflop=step_flops / 1e9, gbytes=step_bytes / 1e9)
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg.name + ": " + cfg.note, "layers": L, "kv_heads": cfg.num_heads,
+                   "head_dim": cfg.head_dim, "seqlens": list(cfg.seqlens), "storage_dtype": cfg.dtype,
+                   "rho": cfg.rho, "gamma": cfg.gamma, "replicas": world,
+                   "l2_policy": "inputs (%.2f GB) exceed L2; no flush" % (input_bytes / 1e9)},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "roofline": roof, "roofline_step": roof_step,
+    }
+
+    # end to end from pinned host buffers (H2D of K,V and D2H of the compacted cache inside the timing)
+    if not args.no_e2e:
+        hostK = [k.cpu().pin_memory() for k in Kd]
+        hostV = [v.cpu().pin_memory() for v in Vd]
+        copy_stream = torch.cuda.Stream(device=dev)
+        evs = [torch.cuda.Event() for _ in range(L)]
+        cap = comp.capacity
+        hk = torch.empty((L, cap, cfg.num_heads, cfg.head_dim), dtype=cfg.torch_dtype).pin_memory()
+        hv = torch.empty_like(hk).pin_memory()
+        hidx = torch.empty((L, cfg.num_heads, cap), dtype=torch.int32).pin_memory()
+        hoff = torch.empty((L, len(cfg.seqlens) + 1), dtype=torch.int64).pin_memory()
+
+        def e2e_step():
+            cur = torch.cuda.current_stream()
+            start = torch.cuda.Event()
+            start.record(cur)
+            copy_stream.wait_event(start)
+            with torch.cuda.stream(copy_stream):
+                for l in range(L):
+                    Kd[l].copy_(hostK[l], non_blocking=True)
+                    Vd[l].copy_(hostV[l], non_blocking=True)
+                    evs[l].record(copy_stream)
+            ws = comp._workspace(Kd[0], Vd[0])
+            for l in range(L):
+                cur.wait_event(evs[l])
+                binding.fc_score_layer(comp.handle, Kd[l], Vd[l], comp.cu, comp.gamma, comp.scores[l],
+                                       comp.energy[l], ws)
+            comp.allocate()
+            comp.select_compact(Kd, Vd)
+            hoff.copy_(comp.offsets, non_blocking=True)
+            cur.synchronize()
+            d2h = hoff.numel() * 8
+            for l in range(L):
+                r = int(hoff[l, -1])
+                hk[l, :r].copy_(comp.out_k[l, :r], non_blocking=True)
+                hv[l, :r].copy_(comp.out_v[l, :r], non_blocking=True)
+                hidx[l, :, :r].copy_(comp.out_idx[l, :, :r], non_blocking=True)
+                d2h += 2 * r * cfg.num_heads * cfg.head_dim * s + r * cfg.num_heads * 4
+            cur.synchronize()
+            return d2h
+
+        for _ in range(2):
+            d2h_bytes = e2e_step()
+        n_e2e = max(3, min(10, args.steps))
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            d2h_bytes = e2e_step()
+        barrier()
+        e2e_ms = 1000.0 * (time.perf_counter() - t0) / n_e2e
+        if dist is not None:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        out["e2e"] = {"value": tokens * world / (e2e_ms / 1000.0), "unit": UNIT,
+                      "h2d_bytes_per_step": int(input_bytes), "d2h_bytes_per_step": int(d2h_bytes),
+                      "ms_per_step": e2e_ms, "steps": n_e2e}
+        del hostK, hostV, hk, hv
+
+    # CPU baseline: the oracle on this machine's host cores, bounded sample (rank 0, single-GPU run only)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_layers_host = min(L, 4)
+        Ks_host = [Kd[l].float().cpu().numpy() for l in range(n_layers_host)]
+        Vs_host = [Vd[l].float().cpu().numpy() for l in range(n_layers_host)]
+        tps, used, el = oracle_sample(cfg, Ks_host, Vs_host, args.cpu_budget_s)
+        out["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": 1, "kind": "oracle",
+                               "host_cores": os.cpu_count(),
+                               "sample": "%d of %d layers (all heads, all sequences), %.1f s, scaled by the layer count"
+                                         % (used, L, el)}
+    comp.close()
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -80,10 +80,25 @@ fc_status fc_last_device_status(fc_handle *h, fc_stream stream);
 /* Number of kernels this handle has launched since fc_create (diagnostic). */
 uint64_t fc_launch_count(const fc_handle *h);
 
+/* Per-kernel timing (diagnostic; the paper has no counterpart).  Between
+ * fc_profile_begin and fc_profile_end every launch of the given kernel class
+ * (1 transform pass 1, 2 transform pass 2, 3 transform pass 3 + scoring,
+ * 4 top-k selection, 5 row gather, 6 other small kernels) is bracketed by a CUDA
+ * event pair on the launching stream, at most max_launches of them.
+ * fc_profile_end waits for the recorded events and returns the summed device
+ * time in milliseconds and the number of launches timed. */
+fc_status fc_profile_begin(fc_handle *h, int32_t kernel_class, int32_t max_launches);
+fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *launches);
+
 /* Target size in bytes of the transform intermediates processed per kernel group
  * (kept below the L2 capacity so they are re-read from cache, not HBM).
  * Default 32 MiB.  Affects speed only. */
 fc_status fc_set_group_bytes(fc_handle *h, size_t bytes);
+
+/* How a sequence of length seqlen is transformed (diagnostic, used for flop
+ * accounting): out = { chirp-convolution path (1) or direct power-of-two path (0),
+ * transform length, first factor N1, second factor N2 }. */
+fc_status fc_describe_plan(const fc_handle *h, int32_t seqlen, int32_t out[4]);
 
 /* Workspace sizes (bytes) the next two calls need for this view.  0 on bad input. */
 size_t fc_score_workspace_bytes(const fc_handle *h, const fc_kv_view *kv);

@@ -23,7 +23,8 @@ _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
     "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count",
-    "fc_set_group_bytes", "fc_score_workspace_bytes", "fc_select_workspace_bytes",
+    "fc_set_group_bytes", "fc_profile_begin", "fc_profile_end", "fc_describe_plan",
+    "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact",
 )
 
@@ -61,6 +62,12 @@ def _load() -> ctypes.CDLL:
     lib.fc_launch_count.restype = c_uint64
     lib.fc_set_group_bytes.argtypes = [c_void_p, c_size_t]
     lib.fc_set_group_bytes.restype = c_int
+    lib.fc_profile_begin.argtypes = [c_void_p, c_int32, c_int32]
+    lib.fc_profile_begin.restype = c_int
+    lib.fc_profile_end.argtypes = [c_void_p, POINTER(c_double), POINTER(c_uint64)]
+    lib.fc_profile_end.restype = c_int
+    lib.fc_describe_plan.argtypes = [c_void_p, c_int32, POINTER(c_int32)]
+    lib.fc_describe_plan.restype = c_int
     lib.fc_score_workspace_bytes.argtypes = [c_void_p, POINTER(fc_kv_view)]
     lib.fc_score_workspace_bytes.restype = c_size_t
     lib.fc_select_workspace_bytes.argtypes = [c_void_p, POINTER(fc_kv_view)]
@@ -134,6 +141,26 @@ def fc_launch_count(handle) -> int:
 
 def fc_set_group_bytes(handle, nbytes: int) -> None:
     _check(_lib.fc_set_group_bytes(handle, int(nbytes)), "fc_set_group_bytes")
+
+
+KERNEL_CLASSES = {"pass1": 1, "pass2": 2, "pass3": 3, "select": 4, "gather": 5, "other": 6}
+
+
+def fc_profile_begin(handle, kernel_class: int, max_launches: int = 16384) -> None:
+    _check(_lib.fc_profile_begin(handle, int(kernel_class), int(max_launches)), "fc_profile_begin")
+
+
+def fc_profile_end(handle):
+    """-> (total_ms, launches) of the kernel class given to fc_profile_begin."""
+    ms, n = c_double(0.0), c_uint64(0)
+    _check(_lib.fc_profile_end(handle, byref(ms), byref(n)), "fc_profile_end")
+    return float(ms.value), int(n.value)
+
+
+def fc_describe_plan(handle, seqlen: int) -> dict:
+    out = (c_int32 * 4)()
+    _check(_lib.fc_describe_plan(handle, int(seqlen), out), "fc_describe_plan")
+    return dict(bluestein=bool(out[0]), nfft=int(out[1]), n1=int(out[2]), n2=int(out[3]))
 
 
 def fc_score_workspace_bytes(handle, k, v, cu_seqlens) -> int:

@@ -34,6 +34,10 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->status_word = nullptr;
   h->group_bytes = (size_t)32 << 20;
   h->launches = 0;
+  h->prof_class = FC_K_NONE;
+  h->prof_events = nullptr;
+  h->prof_cap = 0;
+  h->prof_used = 0;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return FC_ERR_CUDA; }
   h->num_sms = prop.multiProcessorCount;
@@ -52,8 +56,55 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   return FC_OK;
 }
 
+static void free_prof(fc_handle *h) {
+  if (h->prof_events) {
+    for (int i = 0; i < 2 * h->prof_cap; ++i) cudaEventDestroy(h->prof_events[i]);
+    delete[] h->prof_events;
+  }
+  h->prof_events = nullptr;
+  h->prof_cap = h->prof_used = 0;
+  h->prof_class = FC_K_NONE;
+}
+
+extern "C" fc_status fc_profile_begin(fc_handle *h, int32_t kernel_class, int32_t max_launches) {
+  if (!h || kernel_class < FC_K_PASS1 || kernel_class > FC_K_OTHER || max_launches < 1) return FC_ERR_INVALID_ARG;
+  free_prof(h);
+  h->prof_events = new (std::nothrow) cudaEvent_t[2 * (size_t)max_launches];
+  if (!h->prof_events) return FC_ERR_INTERNAL;
+  for (int i = 0; i < 2 * max_launches; ++i) {
+    if (cudaEventCreate(&h->prof_events[i]) != cudaSuccess) {
+      h->prof_cap = i / 2;
+      free_prof(h);
+      return FC_ERR_CUDA;
+    }
+  }
+  h->prof_cap = max_launches;
+  h->prof_used = 0;
+  h->prof_class = kernel_class;
+  return FC_OK;
+}
+
+extern "C" fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *launches) {
+  if (!h || !total_ms || !launches) return FC_ERR_INVALID_ARG;
+  double sum = 0.0;
+  for (int i = 0; i < h->prof_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(h->prof_events[2 * i + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, h->prof_events[2 * i], h->prof_events[2 * i + 1]) != cudaSuccess) {
+      free_prof(h);
+      return FC_ERR_CUDA;
+    }
+    sum += (double)ms;
+  }
+  *total_ms = sum;
+  *launches = (uint64_t)h->prof_used;
+  free_prof(h);
+  return FC_OK;
+}
+
 extern "C" void fc_destroy(fc_handle *h) {
   if (!h) return;
+  free_prof(h);
   if (h->master) cudaFree(h->master);
   if (h->status_word) cudaFree(h->status_word);
   delete h;

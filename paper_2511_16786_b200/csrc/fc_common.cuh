@@ -27,6 +27,30 @@ struct fc_handle {
   size_t group_bytes;
   int num_sms;
   unsigned long long launches;
+  // optional per-kernel-class timing (fc_profile_begin / fc_profile_end)
+  int prof_class;
+  cudaEvent_t *prof_events;   // pairs
+  int prof_cap, prof_used;
+};
+
+// Kernel classes for fc_profile_begin.
+enum { FC_K_NONE = 0, FC_K_PASS1 = 1, FC_K_PASS2 = 2, FC_K_PASS3 = 3, FC_K_SELECT = 4, FC_K_GATHER = 5, FC_K_OTHER = 6 };
+
+// Brackets one launch with an event pair when its class is being profiled.
+struct ProfScope {
+  fc_handle *h;
+  cudaStream_t st;
+  bool on;
+  ProfScope(fc_handle *h_, int cls, cudaStream_t st_) : h(h_), st(st_) {
+    on = h->prof_class == cls && h->prof_used < h->prof_cap;
+    if (on) cudaEventRecord(h->prof_events[2 * h->prof_used], st);
+  }
+  ~ProfScope() {
+    if (on) {
+      cudaEventRecord(h->prof_events[2 * h->prof_used + 1], st);
+      h->prof_used++;
+    }
+  }
 };
 
 // Radix plan of one power-of-two FFT length: len = prod radix[s].

@@ -23,6 +23,7 @@
 // Lengths that are not a power of two (or are below 16) go through Bluestein's
 // chirp convolution on a power-of-two length M >= 2N-1 with the same three passes.
 #include "fc_common.cuh"
+#include "fc_score_fast.cuh"
 
 #include <math.h>
 #include <type_traits>
@@ -453,6 +454,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct SeqPlan {
   bool bluestein;
+  bool fast;                 // specialised kernels (power-of-two N in [1024, 65536])
   int N, Nfft, N1, N2;
   int cs, cs2;               // columns per tile in pass 1/3 and pass 2
 };
@@ -469,8 +471,9 @@ SeqPlan plan_sequence(int N) {
     s.Nfft = N;
   }
   const int bits = ilog2(s.Nfft);
+  s.fast = !s.bluestein && N >= 1024 && N <= 65536;
   int b1 = bits / 2;
-  if (b1 > 7) b1 = 7;
+  if (b1 > 7 && !s.fast) b1 = 7;
   s.N1 = 1 << b1;
   s.N2 = s.Nfft / s.N1;
   s.cs = 64;
@@ -548,6 +551,7 @@ fc_status launch_pass1(fc_handle *h, cudaStream_t st, const Loader &ld, const Se
   fc_status s = set_smem(k_pass1<Loader>, sm);
   if (s != FC_OK) return s;
   dim3 grid(sp.N2, ncol_ws / cs);
+  ProfScope ps(h, FC_K_PASS1, st);
   k_pass1<Loader><<<grid, kThreads, sm, st>>>(ld, p1, sp.N2, ncol_ws, ilog2(cs), ws, h->master, h->master_len, partial);
   return fc_after_launch(h);
 }
@@ -560,8 +564,56 @@ fc_status launch_pass2(fc_handle *h, cudaStream_t st, const SeqPlan &sp, int nco
   fc_status s = set_smem(k_pass2<MID>, sm);
   if (s != FC_OK) return s;
   dim3 grid(MID == MID_DCT ? sp.N1 / 2 + 1 : sp.N1, ncol_ws / cs2);
+  ProfScope ps(h, FC_K_PASS2, st);
   k_pass2<MID><<<grid, kThreads, sm, st>>>(p2, sp.N1, ncol_ws, ilog2(cs2), ws, h->master, h->master_len, omega, hhat, scale);
   return fc_after_launch(h);
+}
+
+// The three specialised launches for one head group of a power-of-two sequence.
+template <typename T, int R1B, int R2B>
+fc_status launch_fast_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp,
+                           const SeqPlan &sp, int h0, int hg, int omega, float2 *ws, double *ptot,
+                           double *phi, float *scores, long long total_tokens) {
+  constexpr int N1 = 16 * R1B, N2 = 16 * R2B;
+  const int d = kv->head_dim, ncol_ws = hg * d;
+  const size_t sm1 = (size_t)N1 * 32 * sizeof(float4) + N1 * sizeof(float2);
+  const size_t sm2 = (size_t)2 * N2 * 8 * sizeof(float4) + 3 * N2 * sizeof(float2);
+  fc_status s;
+  if ((s = set_smem(fast::k_p1<T, R1B>, sm1)) != FC_OK) return s;
+  {
+    ProfScope ps(h, FC_K_PASS1, st);
+    fast::k_p1<T, R1B><<<dim3(N2, ncol_ws / 64), 32 * R1B, sm1, st>>>(
+        kp, vp, kv->stride_token, kv->stride_head, h0, d, sp.N, N2, ncol_ws, ws, h->master, h->master_len, ptot);
+  }
+  if ((s = fc_after_launch(h)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p2<R2B>, sm2)) != FC_OK) return s;
+  {
+    ProfScope ps(h, FC_K_PASS2, st);
+    fast::k_p2<R2B><<<dim3(N1 / 2 + 1, ncol_ws / 16), 16 * R2B, sm2, st>>>(N1, ncol_ws, ws, h->master,
+                                                                          h->master_len, omega);
+  }
+  if ((s = fc_after_launch(h)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p3<R1B>, sm1)) != FC_OK) return s;
+  {
+    ProfScope ps(h, FC_K_PASS3, st);
+    const float inv = (float)(1.0 / ((double)sp.N * (double)sp.N * (double)d));
+    fast::k_p3<R1B><<<dim3(N2, hg), 32 * R1B, sm1, st>>>(sp.N, N2, ncol_ws, ws, h->master, h->master_len, scores,
+                                                         h0, d, total_tokens, inv, phi);
+  }
+  return fc_after_launch(h);
+}
+
+template <typename T>
+fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp,
+                      const SeqPlan &sp, int h0, int hg, int omega, float2 *ws, double *ptot, double *phi,
+                      float *scores, long long total_tokens) {
+#define FC_FAST_CASE(A, B)                                                                                  \
+  if (sp.N1 == 16 * A && sp.N2 == 16 * B)                                                                   \
+    return launch_fast_impl<T, A, B>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores, total_tokens);
+  FC_FAST_CASE(2, 2) FC_FAST_CASE(2, 4) FC_FAST_CASE(4, 4) FC_FAST_CASE(4, 8)
+  FC_FAST_CASE(8, 8) FC_FAST_CASE(8, 16) FC_FAST_CASE(16, 16)
+#undef FC_FAST_CASE
+  return FC_ERR_INTERNAL;
 }
 
 template <typename T>
@@ -608,14 +660,20 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     double *ptot = part_tot + 2 * tot_slots;
     double *phi = part_hi + 2 * hi_slots;
     const size_t sm3 = smem_pass13(sp, sp.cs);
-    if (!sp.bluestein) {
+    if (sp.fast) {
+      if ((s = launch_fast<T>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores + start,
+                              total_tokens)) != FC_OK) return s;
+    } else if (!sp.bluestein) {
       KvLoader<T, false> ld{kp, vp, kv->stride_token, kv->stride_head, h0, d, N, 0.f, 0.f};
       if ((s = launch_pass1(h, st, ld, sp, ncol_ws, sp.cs, ws, ptot)) != FC_OK) return s;
       if ((s = launch_pass2<MID_DCT>(h, st, sp, ncol_ws, sp.cs2, ws, omega, nullptr, 1.f / (float)N)) != FC_OK) return s;
       if ((s = set_smem(k_pass3<EPI_SCORE, false>, sm3)) != FC_OK) return s;
-      k_pass3<EPI_SCORE, false><<<dim3(sp.N2, hg), kThreads, sm3, st>>>(
-          p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, nullptr, scores + start, h0, d,
-          total_tokens, 1.f / (float)d, phi);
+      {
+        ProfScope ps(h, FC_K_PASS3, st);
+        k_pass3<EPI_SCORE, false><<<dim3(sp.N2, hg), kThreads, sm3, st>>>(
+            p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, nullptr, scores + start, h0, d,
+            total_tokens, 1.f / (float)d, phi);
+      }
       if ((s = fc_after_launch(h)) != FC_OK) return s;
     } else {
       const float invM = 1.f / (float)sp.Nfft;
@@ -623,27 +681,47 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       if ((s = launch_pass1(h, st, ld, sp, ncol_ws, sp.cs, ws, ptot)) != FC_OK) return s;
       if ((s = launch_pass2<MID_MULH>(h, st, sp, ncol_ws, sp.cs2, ws, 0, hhat, invM)) != FC_OK) return s;
       if ((s = set_smem(k_pass3<EPI_SPEC, true>, sm3)) != FC_OK) return s;
-      k_pass3<EPI_SPEC, true><<<dim3(sp.N2, ncol_ws / sp.cs), kThreads, sm3, st>>>(
-          p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, spec, nullptr, 0, d, 0, 0.f, nullptr);
+      {
+        ProfScope ps(h, FC_K_PASS3, st);
+        k_pass3<EPI_SPEC, true><<<dim3(sp.N2, ncol_ws / sp.cs), kThreads, sm3, st>>>(
+            p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, spec, nullptr, 0, d, 0, 0.f, nullptr);
+      }
       if ((s = fc_after_launch(h)) != FC_OK) return s;
       FilterLoader fl{spec, ncol_ws, N, omega};
       if ((s = launch_pass1(h, st, fl, sp, ncol_ws, sp.cs, ws, nullptr)) != FC_OK) return s;
       if ((s = launch_pass2<MID_MULH>(h, st, sp, ncol_ws, sp.cs2, ws, 0, hhat, invM)) != FC_OK) return s;
       if ((s = set_smem(k_pass3<EPI_SCORE, true>, sm3)) != FC_OK) return s;
       const float inv = (float)(1.0 / ((double)N * (double)N * (double)d));
-      k_pass3<EPI_SCORE, true><<<dim3(sp.N2, hg), kThreads, sm3, st>>>(
-          p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, nullptr, scores + start, h0, d,
-          total_tokens, inv, phi);
+      {
+        ProfScope ps(h, FC_K_PASS3, st);
+        k_pass3<EPI_SCORE, true><<<dim3(sp.N2, hg), kThreads, sm3, st>>>(
+            p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, nullptr, scores + start, h0, d,
+            total_tokens, inv, phi);
+      }
       if ((s = fc_after_launch(h)) != FC_OK) return s;
     }
     tot_slots += (size_t)sp.N2 * (ncol_ws / sp.cs);
     hi_slots += (size_t)sp.N2 * hg;
   }
-  k_energy_finalize<<<1, 256, 0, st>>>(part_tot, (int)tot_slots, part_hi, (int)hi_slots, energy_b);
+  {
+    ProfScope ps(h, FC_K_OTHER, st);
+    k_energy_finalize<<<1, 256, 0, st>>>(part_tot, (int)tot_slots, part_hi, (int)hi_slots, energy_b);
+  }
   return fc_after_launch(h);
 }
 
 }  // namespace
+
+extern "C" fc_status fc_describe_plan(const fc_handle *h, int32_t seqlen, int32_t out[4]) {
+  if (!h || !out || seqlen < 1) return FC_ERR_INVALID_ARG;
+  if (seqlen > h->max_seqlen || (seqlen > 65536 && !is_pow2(seqlen))) return FC_ERR_UNSUPPORTED;
+  const SeqPlan sp = plan_sequence(seqlen);
+  out[0] = sp.bluestein ? 1 : 0;
+  out[1] = sp.Nfft;
+  out[2] = sp.N1;
+  out[3] = sp.N2;
+  return FC_OK;
+}
 
 extern "C" size_t fc_score_workspace_bytes(const fc_handle *h, const fc_kv_view *kv) {
   if (validate_view(h, kv) != FC_OK) return 0;

@@ -1,0 +1,394 @@
+// Specialised kernels of the three transform passes for power-of-two sequence
+// lengths N = N1*N2 with N1 = 16*R1B and N2 = 16*R2B (R1B, R2B in {2,4,8,16}),
+// i.e. N from 1024 to 65536.  Same mathematics as the generic kernels in
+// fc_score.cu (see the header comment there); what differs is the mapping:
+//
+//  * every thread owns two adjacent channels (one float4 = two complex values),
+//    so all shared-memory and workspace accesses are 128-bit and a twiddle is
+//    loaded once for two butterflies;
+//  * a thread keeps a whole radix-16 butterfly (16 points x 2 channels) in
+//    registers; the first stage of pass 1 is fed straight from the K/V rows in
+//    global memory and the last stage of each pass is written straight to global
+//    memory, so a tile crosses shared memory once per exchange;
+//  * all strides are compile-time constants.
+//
+// The transform is left unnormalised (factor N); pass 3 folds 1/N^2 into the score.
+#pragma once
+#include "fc_common.cuh"
+
+namespace fast {
+
+__device__ __forceinline__ int perm_token(int p, int N) {
+  const int half = (N + 1) >> 1;
+  return p < half ? 2 * p : 2 * (N - 1 - p) + 1;
+}
+
+// two adjacent channels of one row
+template <typename T> struct Load2;
+template <> struct Load2<float> {
+  __device__ static float2 ld(const float *p) { return __ldg(reinterpret_cast<const float2 *>(p)); }
+};
+template <> struct Load2<__half> {
+  __device__ static float2 ld(const __half *p) {
+    const unsigned u = __ldg(reinterpret_cast<const unsigned *>(p));
+    return __half22float2(*reinterpret_cast<const __half2 *>(&u));
+  }
+};
+template <> struct Load2<__nv_bfloat16> {
+  __device__ static float2 ld(const __nv_bfloat16 *p) {
+    const unsigned u = __ldg(reinterpret_cast<const unsigned *>(p));
+    return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+  }
+};
+
+template <int R>
+__device__ __forceinline__ void dft_fwd(float2 (&x)[R]) { dft_small<R, -1>(x); }
+template <int R>
+__device__ __forceinline__ void dft_inv(float2 (&x)[R]) { dft_small<R, +1>(x); }
+
+// ---------------------------------------------------------------------------
+// pass 1: grid (N2, group columns / 64), block 32*R1B.
+// Thread (cp = lane, j = warp): channels 2cp, 2cp+1 of the slice; first stage
+// points n1 = j + R1B*p, p = 0..15, loaded from the K/V rows.
+// ---------------------------------------------------------------------------
+template <typename T, int R1B>
+__global__ void __launch_bounds__(32 * R1B)
+k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, long long stride_head,
+     int head0, int head_dim, int N, int N2, int ncol_ws, float2 *__restrict__ ws,
+     const float2 *__restrict__ master, int master_len, double *__restrict__ partial) {
+  constexpr int N1 = 16 * R1B, NT = 32 * R1B, IT = 16 / R1B;
+  extern __shared__ float4 smem4[];
+  float4 *S = smem4;                                        // [N1][32]
+  float2 *tw = reinterpret_cast<float2 *>(S + N1 * 32);     // [N1]
+  __shared__ double red[2][R1B];
+  const int tid = threadIdx.x, cp = tid & 31, j = tid >> 5;
+  const int n2 = blockIdx.x, gc0 = blockIdx.y * 64;
+  const int h = head0 + gc0 / head_dim, c = gc0 % head_dim + 2 * cp;
+  const T *kb = k + (long long)h * stride_head + c;
+  const T *vb = v + (long long)h * stride_head + c;
+
+  float2 x0[16], x1[16];
+  float accK = 0.f, accV = 0.f;
+#pragma unroll
+  for (int p = 0; p < 16; ++p) {
+    const int tok = perm_token((j + R1B * p) * N2 + n2, N);
+    const long long off = (long long)tok * stride_token;
+    const float2 kk = Load2<T>::ld(kb + off), vv = Load2<T>::ld(vb + off);
+    x0[p] = make_float2(kk.x, vv.x);
+    x1[p] = make_float2(kk.y, vv.y);
+  }
+  for (int i = tid; i < N1; i += NT) tw[i] = master[(size_t)i * (master_len / N1)];
+  __syncthreads();
+#pragma unroll
+  for (int p = 0; p < 16; ++p) {
+    accK = fmaf(x0[p].x, x0[p].x, fmaf(x1[p].x, x1[p].x, accK));
+    accV = fmaf(x0[p].y, x0[p].y, fmaf(x1[p].y, x1[p].y, accV));
+  }
+  dft_fwd<16>(x0);
+  dft_fwd<16>(x1);
+#pragma unroll
+  for (int p = 0; p < 16; ++p) {
+    if (p > 0) {
+      const float2 w = tw[j * p];
+      x0[p] = cmul(x0[p], w);
+      x1[p] = cmul(x1[p], w);
+    }
+    S[(j + R1B * p) * 32 + cp] = make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
+  }
+  __syncthreads();
+  // second stage: radix R1B inside sub-block pp; bin k1 = pp + 16*q
+#pragma unroll
+  for (int it = 0; it < IT; ++it) {
+    const int pp = j + R1B * it;
+    float2 y0[R1B], y1[R1B];
+#pragma unroll
+    for (int q = 0; q < R1B; ++q) {
+      const float4 t = S[(q + R1B * pp) * 32 + cp];
+      y0[q] = make_float2(t.x, t.y);
+      y1[q] = make_float2(t.z, t.w);
+    }
+    dft_fwd<R1B>(y0);
+    dft_fwd<R1B>(y1);
+#pragma unroll
+    for (int q = 0; q < R1B; ++q) {
+      const int k1 = pp + 16 * q;
+      float4 *dst = reinterpret_cast<float4 *>(ws + ((size_t)k1 * N2 + n2) * ncol_ws + gc0 + 2 * cp);
+      *dst = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
+    }
+  }
+  // per-block sums of squares (total energy of Eq. 12, by Parseval)
+  const double a = warp_sum_d((double)accK), b = warp_sum_d((double)accV);
+  if (cp == 0) { red[0][j] = a; red[1][j] = b; }
+  __syncthreads();
+  if (tid == 0) {
+    double sa = 0, sb = 0;
+#pragma unroll
+    for (int i = 0; i < R1B; ++i) { sa += red[0][i]; sb += red[1][i]; }
+    const size_t slot = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+    partial[2 * slot] = sa;
+    partial[2 * slot + 1] = sb;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// pass 2: grid (N1/2 + 1, group columns / 16), block 16*R2B.
+// Thread (cp = tid&7, hf = (tid>>3)&1, j = tid>>4): channel pair cp of the
+// 16-column slice, half hf (k1 = blockIdx.x or N1 - blockIdx.x), first-stage
+// points n2 = j + R2B*p.
+// ---------------------------------------------------------------------------
+template <int R2B>
+__global__ void __launch_bounds__(16 * R2B, (R2B >= 16 ? 2 : 4))
+k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ master, int master_len,
+     int omega) {
+  constexpr int N2 = 16 * R2B, NT = 16 * R2B, IT = 16 / R2B;
+  extern __shared__ float4 smem4[];
+  float4 *S = smem4;                                         // [2][N2][8]
+  float2 *tw = reinterpret_cast<float2 *>(S + 2 * N2 * 8);   // [N2]   w_N2^i
+  float2 *twN = tw + N2;                                     // [2][N2] w_N^(n2*k1)
+  const int tid = threadIdx.x, cp = tid & 7, hf = (tid >> 3) & 1, j = tid >> 4;
+  const int k1a = blockIdx.x, k1b = (N1 - k1a) % N1;
+  const bool self = (k1a == k1b);
+  const int k1 = hf ? k1b : k1a;
+  const int N = N1 * N2;
+  const int gc0 = blockIdx.y * 16;
+  const bool active = !(self && hf);
+
+  {
+    const int mstepN = master_len / N;
+    for (int i = tid; i < N2; i += NT) {
+      tw[i] = master[(size_t)i * (master_len / N2)];
+      twN[i] = master[(size_t)(((long long)i * k1a) % N) * mstepN];
+      twN[N2 + i] = master[(size_t)(((long long)i * k1b) % N) * mstepN];
+    }
+  }
+  float4 *Sh = S + hf * (N2 * 8);
+  float2 x0[16], x1[16];
+  float2 *base = ws + ((size_t)k1 * N2) * ncol_ws + gc0 + 2 * cp;
+  if (active) {
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const float4 t = *reinterpret_cast<const float4 *>(base + (size_t)(j + R2B * p) * ncol_ws);
+      x0[p] = make_float2(t.x, t.y);
+      x1[p] = make_float2(t.z, t.w);
+    }
+  }
+  __syncthreads();
+  if (active) {
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const float2 w = twN[hf * N2 + j + R2B * p];
+      x0[p] = cmul(x0[p], w);
+      x1[p] = cmul(x1[p], w);
+    }
+    dft_fwd<16>(x0);
+    dft_fwd<16>(x1);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      if (p > 0) {
+        const float2 w = tw[j * p];
+        x0[p] = cmul(x0[p], w);
+        x1[p] = cmul(x1[p], w);
+      }
+      Sh[(j + R2B * p) * 8 + cp] = make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
+    }
+  }
+  __syncthreads();
+  // second forward stage, written back in place (each sub-block is touched by one thread only);
+  // registers keep bins k2 = pp + 16*q at index it*R2B + q
+  if (active) {
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R2B * it;
+      float2 y0[R2B], y1[R2B];
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) {
+        const float4 t = Sh[(q + R2B * pp) * 8 + cp];
+        y0[q] = make_float2(t.x, t.y);
+        y1[q] = make_float2(t.z, t.w);
+      }
+      dft_fwd<R2B>(y0);
+      dft_fwd<R2B>(y1);
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) {
+        x0[it * R2B + q] = y0[q];
+        x1[it * R2B + q] = y1[q];
+        Sh[(q + R2B * pp) * 8 + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
+      }
+    }
+  }
+  __syncthreads();       // full spectra of both halves are in shared memory
+  if (active) {
+    const float4 *Sp = S + (self ? hf : 1 - hf) * (N2 * 8);
+    const int ustep = master_len / (2 * N);
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R2B * it;
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) {
+        const int k2 = pp + 16 * q;
+        const int bin = k1 + N1 * k2;
+        const bool inL = bin <= omega, inH = (N - bin) <= omega;
+        float2 &P0 = x0[it * R2B + q], &P1 = x1[it * R2B + q];
+        if (bin == 0 || (inL && inH)) {
+          P0 = make_float2(0.f, 0.f);
+          P1 = make_float2(0.f, 0.f);
+        } else if (inL || inH) {
+          const int k2p = (k1 == 0) ? ((N2 - k2) & (N2 - 1)) : (N2 - 1 - k2);
+          const float4 t = Sp[((k2p >> 4) + R2B * (k2p & 15)) * 8 + cp];
+          float2 u = __ldg(master + (size_t)bin * ustep);          // exp(-j*pi*bin/N)
+          const float sgn = inL ? -0.5f : 0.5f;                   // E = (P -/+ uQ)/2 with u = exp(+j*pi*bin/N)
+          u = make_float2(u.x * sgn, -u.y * sgn);
+          const float2 q0 = make_float2(t.x, t.y), q1 = make_float2(t.z, t.w);
+          P0 = make_float2(fmaf(q0.x, u.x, fmaf(-q0.y, u.y, 0.5f * P0.x)),
+                           fmaf(q0.x, u.y, fmaf(q0.y, u.x, 0.5f * P0.y)));
+          P1 = make_float2(fmaf(q1.x, u.x, fmaf(-q1.y, u.y, 0.5f * P1.x)),
+                           fmaf(q1.x, u.y, fmaf(q1.y, u.x, 0.5f * P1.y)));
+        }
+      }
+    }
+    // first inverse stage (mirror of the second forward stage)
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      float2 y0[R2B], y1[R2B];
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) { y0[q] = x0[it * R2B + q]; y1[q] = x1[it * R2B + q]; }
+      dft_inv<R2B>(y0);
+      dft_inv<R2B>(y1);
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) { x0[it * R2B + q] = y0[q]; x1[it * R2B + q] = y1[q]; }
+    }
+  }
+  __syncthreads();       // all partner reads are done
+  if (active) {
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R2B * it;
+#pragma unroll
+      for (int q = 0; q < R2B; ++q)
+        Sh[(q + R2B * pp) * 8 + cp] = make_float4(x0[it * R2B + q].x, x0[it * R2B + q].y,
+                                                  x1[it * R2B + q].x, x1[it * R2B + q].y);
+    }
+  }
+  __syncthreads();
+  if (active) {
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const float4 t = Sh[(j + R2B * p) * 8 + cp];
+      x0[p] = make_float2(t.x, t.y);
+      x1[p] = make_float2(t.z, t.w);
+      if (p > 0) {
+        const float2 w = tw[j * p];
+        x0[p] = cmul_conj(x0[p], w);
+        x1[p] = cmul_conj(x1[p], w);
+      }
+    }
+    dft_inv<16>(x0);
+    dft_inv<16>(x1);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const float2 w = twN[hf * N2 + j + R2B * p];
+      const float2 a = cmul_conj(x0[p], w), b = cmul_conj(x1[p], w);
+      *reinterpret_cast<float4 *>(base + (size_t)(j + R2B * p) * ncol_ws) = make_float4(a.x, a.y, b.x, b.y);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// pass 3: grid (N2, heads of the group), block 32*R1B.  Inverse DFT over k1,
+// squared magnitude summed over the channels of the head, scores and the
+// per-block outlier-energy partial sums.
+// ---------------------------------------------------------------------------
+template <int R1B>
+__global__ void __launch_bounds__(32 * R1B)
+k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__restrict__ master,
+     int master_len, float *__restrict__ scores, int head0, int head_dim, long long score_stride,
+     float inv_scale, double *__restrict__ partial) {
+  constexpr int N1 = 16 * R1B, NT = 32 * R1B, IT = 16 / R1B;
+  extern __shared__ float4 smem4[];
+  float4 *S = smem4;                                        // [N1][32]
+  float2 *tw = reinterpret_cast<float2 *>(S + N1 * 32);     // [N1]
+  __shared__ double red[2][R1B];
+  const int tid = threadIdx.x, cp = tid & 31, j = tid >> 5;
+  const int n2 = blockIdx.x, hh = blockIdx.y;
+  for (int i = tid; i < N1; i += NT) tw[i] = master[(size_t)i * (master_len / N1)];
+
+  float acc[32];            // [0..15] K part of rows j + R1B*p, [16..31] V part
+#pragma unroll
+  for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+
+  const int nslices = head_dim / 64;
+  for (int sl = 0; sl < nslices; ++sl) {
+    const int gc0 = hh * head_dim + sl * 64;
+    // inverse radix-R1B stage on bins k1 = pp + 16*q, straight from the workspace
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R1B * it;
+      float2 y0[R1B], y1[R1B];
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) {
+        const float4 t = *reinterpret_cast<const float4 *>(
+            ws + ((size_t)(pp + 16 * q) * N2 + n2) * ncol_ws + gc0 + 2 * cp);
+        y0[q] = make_float2(t.x, t.y);
+        y1[q] = make_float2(t.z, t.w);
+      }
+      dft_inv<R1B>(y0);
+      dft_inv<R1B>(y1);
+#pragma unroll
+      for (int q = 0; q < R1B; ++q)
+        S[(q + R1B * pp) * 32 + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
+    }
+    __syncthreads();
+    float2 x0[16], x1[16];
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const float4 t = S[(j + R1B * p) * 32 + cp];
+      x0[p] = make_float2(t.x, t.y);
+      x1[p] = make_float2(t.z, t.w);
+      if (p > 0) {
+        const float2 w = tw[j * p];
+        x0[p] = cmul_conj(x0[p], w);
+        x1[p] = cmul_conj(x1[p], w);
+      }
+    }
+    dft_inv<16>(x0);
+    dft_inv<16>(x1);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      acc[p] = fmaf(x0[p].x, x0[p].x, fmaf(x1[p].x, x1[p].x, acc[p]));
+      acc[16 + p] = fmaf(x0[p].y, x0[p].y, fmaf(x1[p].y, x1[p].y, acc[16 + p]));
+    }
+    __syncthreads();
+  }
+  // transposed warp reduction: lane l ends with the sum over all lanes of acc[l]
+  const int lane = cp;
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) {
+#pragma unroll
+    for (int i = 0; i < s; ++i) {
+      const bool up = (lane & s) != 0;
+      const float send = up ? acc[i] : acc[i + s];
+      const float keep = up ? acc[i + s] : acc[i];
+      acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+    }
+  }
+  const float mine = acc[0] * inv_scale;                           // K part (lane < 16) or V part of row p = lane & 15
+  const float other = __shfl_xor_sync(0xffffffffu, mine, 16);
+  if (lane < 16) {
+    const int p = (j + R1B * lane) * N2 + n2;
+    scores[(long long)(head0 + hh) * score_stride + perm_token(p, N)] = mine + other;
+  }
+  const double dk = warp_sum_d(lane < 16 ? (double)mine : 0.0);
+  const double dv = warp_sum_d(lane < 16 ? 0.0 : (double)mine);
+  if (lane == 0) { red[0][j] = dk; red[1][j] = dv; }
+  __syncthreads();
+  if (tid == 0) {
+    double sa = 0, sb = 0;
+#pragma unroll
+    for (int i = 0; i < R1B; ++i) { sa += red[0][i]; sb += red[1][i]; }
+    const size_t slot = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+    partial[2 * slot] = sa * (double)head_dim;
+    partial[2 * slot + 1] = sb * (double)head_dim;
+  }
+}
+
+}  // namespace fast

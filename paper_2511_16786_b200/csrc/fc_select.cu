@@ -366,15 +366,21 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
     const int nseq = kv->batch - b0 < kSeqChunk ? kv->batch - b0 : kSeqChunk;
     SeqTable tab;
     for (int i = 0; i <= nseq; ++i) tab.start[i] = kv->cu_seqlens[b0 + i];
-    k_select<<<dim3(nseq, kv->num_heads), kSelThreads, 0, st>>>(
-        scores, T, tab, b0, budgets, reinterpret_cast<const long long *>(out_offsets), out_idx,
-        out_capacity_rows, h->status_word);
+    {
+      ProfScope ps(h, FC_K_SELECT, st);
+      k_select<<<dim3(nseq, kv->num_heads), kSelThreads, 0, st>>>(
+          scores, T, tab, b0, budgets, reinterpret_cast<const long long *>(out_offsets), out_idx,
+          out_capacity_rows, h->status_word);
+    }
     if ((s = fc_after_launch(h)) != FC_OK) return s;
-    k_gather<<<h->num_sms * 8, 256, 0, st>>>(
-        static_cast<const char *>(kv->k), static_cast<const char *>(kv->v),
-        kv->stride_token * es, kv->stride_head * es, kv->head_dim * es, kv->num_heads, tab, b0, nseq,
-        budgets, reinterpret_cast<const long long *>(out_offsets), out_idx, out_capacity_rows,
-        static_cast<char *>(out_k), static_cast<char *>(out_v));
+    {
+      ProfScope ps(h, FC_K_GATHER, st);
+      k_gather<<<h->num_sms * 8, 256, 0, st>>>(
+          static_cast<const char *>(kv->k), static_cast<const char *>(kv->v),
+          kv->stride_token * es, kv->stride_head * es, kv->head_dim * es, kv->num_heads, tab, b0, nseq,
+          budgets, reinterpret_cast<const long long *>(out_offsets), out_idx, out_capacity_rows,
+          static_cast<char *>(out_k), static_cast<char *>(out_v));
+    }
     if ((s = fc_after_launch(h)) != FC_OK) return s;
   }
   return FC_OK;
