@@ -8,6 +8,7 @@
 // the plain IEEE sequence of multiplies, adds and divides it is written as.
 #include "fc_common.cuh"
 
+#include <cooperative_groups.h>
 #include <math.h>
 
 namespace {
@@ -164,135 +165,193 @@ __device__ __forceinline__ unsigned score_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-constexpr int kSelThreads = 1024;
+constexpr int kSelThreads = 1024;   // threads per block of the selection kernel
+constexpr int kSelCluster = 8;      // blocks (one cluster) per (sequence, head)
+constexpr int kSelKpt = 16;         // scores per thread: 8 * 1024 * 16 = 131072 tokens at most
 
-// Exclusive rank of a 1-bit flag over the block plus the block total.
-__device__ __forceinline__ int block_rank(bool flag, int *wcount, int &total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const unsigned m = __ballot_sync(0xffffffffu, flag);
-  if (lane == 0) wcount[warp] = __popc(m);
-  __syncthreads();
-  int before = 0, all = 0;
-#pragma unroll
-  for (int i = 0; i < kSelThreads / 32; ++i) {
-    const int c = wcount[i];
-    before += (i < warp) ? c : 0;
-    all += c;
-  }
-  __syncthreads();
-  total = all;
-  return before + __popc(m & ((1u << lane) - 1u));
-}
-
-// grid (sequences in chunk, heads)
-__global__ void __launch_bounds__(kSelThreads)
-k_select(const float *__restrict__ scores, long long T, SeqTable st, int b0,
-         const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
-         int *__restrict__ out_idx, long long cap, int *__restrict__ status) {
-  __shared__ int hist[256];
-  __shared__ int wcount[kSelThreads / 32];
+// Selection + compaction + row gather for one (sequence, head), by one cluster of
+// kSelCluster blocks.  Block r of the cluster owns the contiguous token range
+// [r*chunk, (r+1)*chunk) and keeps its score keys in registers.  The k-th largest
+// key is found by a 4-pass MSB-first radix select whose 256-bin histograms are
+// summed across the cluster through distributed shared memory; the chosen tokens
+// are then ranked in token order (block prefix + cluster prefix), written as
+// ascending indices, and their K/V rows are copied by the same block.
+// grid (kSelCluster * sequences in chunk, heads), cluster (kSelCluster, 1, 1).
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
+k_select_gather(const float *__restrict__ scores, long long T, SeqTable st, int b0,
+                const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
+                int *__restrict__ out_idx, long long cap, int *__restrict__ status,
+                const char *__restrict__ kin, const char *__restrict__ vin, long long stride_token_b,
+                long long stride_head_b, int row_bytes, int H, char *__restrict__ out_k,
+                char *__restrict__ out_v) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ int lhist[256];
+  __shared__ int ghist[4][256];          // cluster-wide histograms, one buffer per pass
+  __shared__ unsigned tot[kSelCluster];  // (ties << 16 | greater) of every block of the cluster
+  __shared__ unsigned wsum[kSelThreads / 32];
   __shared__ unsigned s_prefix;
   __shared__ int s_krem;
-  const int tid = threadIdx.x;
-  const int b = b0 + blockIdx.x, h = blockIdx.y;
-  const int s0 = st.start[blockIdx.x];
-  const int n = st.start[blockIdx.x + 1] - s0;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned r = cluster.block_rank();
+  const int bl = blockIdx.x / kSelCluster;
+  const int b = b0 + bl, h = blockIdx.y;
+  const int s0 = st.start[bl];
+  const int n = st.start[bl + 1] - s0;
   int k = budgets[b];
   k = k < 0 ? 0 : (k > n ? n : k);
   const long long off = out_offsets[b];
-  if (k == 0) return;
+  if (k == 0) return;                                    // same decision in every block of the cluster
   if (off < 0 || off + k > cap) {
-    if (tid == 0) atomicOr(status, FC_DEV_FLAG_INTERNAL);
+    if (tid == 0 && r == 0) atomicOr(status, FC_DEV_FLAG_INTERNAL);
     return;
   }
   const float *sc = scores + (long long)h * T + s0;
   int *dst = out_idx + (long long)h * cap + off;
 
+  const int chunk = (n + kSelCluster - 1) / kSelCluster;
+  const int lo = (int)r * chunk;
+  const int hi = lo + chunk < n ? lo + chunk : n;
+  const int base = lo + tid * kSelKpt;
+  int nv = hi - base;
+  nv = nv < 0 ? 0 : (nv > kSelKpt ? kSelKpt : nv);
+  unsigned key[kSelKpt];
+#pragma unroll
+  for (int i = 0; i < kSelKpt; ++i) key[i] = (i < nv) ? score_key(sc[base + i]) : 0u;
+
+  for (int i = tid; i < 4 * 256; i += kSelThreads) (&ghist[0][0])[i] = 0;
   unsigned tau = 0;
-  int need = 0;            // how many keys equal to tau are kept (lowest indices first)
+  int need = 0;
   const bool take_all = (k == n);
   if (!take_all) {
+    cluster.sync();                                      // histograms are zero everywhere before remote adds
     unsigned prefix = 0, mask = 0;
     int krem = k;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-      for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
+#pragma unroll 1
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (tid < 256) lhist[tid] = 0;
       __syncthreads();
-      for (int i = tid; i < n; i += kSelThreads) {
-        const unsigned key = score_key(sc[i]);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+#pragma unroll
+      for (int i = 0; i < kSelKpt; ++i) {
+        const bool m = (i < nv) && ((key[i] & mask) == prefix);
+        const unsigned act = __ballot_sync(0xffffffffu, m);
+        if (m) {
+          const unsigned dgt = (key[i] >> shift) & 255u;
+          const unsigned peers = __match_any_sync(act, dgt);
+          if (lane == __ffs(peers) - 1) atomicAdd(&lhist[dgt], __popc(peers));
+        }
       }
       __syncthreads();
-      if (tid == 0) {
-        int cum = 0, dsel = 0;
-        for (int dgt = 255; dgt >= 0; --dgt) {
-          const int c = hist[dgt];
-          if (cum + c >= krem) { dsel = dgt; break; }
-          cum += c;
+      if (tid < 256) {
+        const int v = lhist[tid];
+        if (v != 0) {
+#pragma unroll
+          for (unsigned rr = 0; rr < kSelCluster; ++rr)
+            atomicAdd(cluster.map_shared_rank(&ghist[pass][tid], rr), v);
         }
-        s_krem = krem - cum;
-        s_prefix = prefix | ((unsigned)dsel << shift);
+      }
+      cluster.sync();                                    // every block now holds the full histogram
+      if (warp == 0) {
+        // lane l owns bins 8l..8l+7; find the bin where the count from the top reaches krem
+        int mine = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mine += ghist[pass][8 * lane + i];
+        int above = mine;                                // inclusive suffix sum over lanes >= l
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_down_sync(0xffffffffu, above, o);
+          if (lane + o < 32) above += t;
+        }
+        const int strictly_above = above - mine;
+        if (strictly_above < krem && krem <= above) {
+          int cum = strictly_above, dsel = 8 * lane;
+          for (int i = 7; i >= 0; --i) {
+            const int c = ghist[pass][8 * lane + i];
+            if (cum + c >= krem) { dsel = 8 * lane + i; break; }
+            cum += c;
+          }
+          s_krem = krem - cum;
+          s_prefix = prefix | ((unsigned)dsel << shift);
+        }
       }
       __syncthreads();
       krem = s_krem;
       prefix = s_prefix;
       mask |= 0xFFu << shift;
-      __syncthreads();
     }
     tau = prefix;
     need = krem;
   }
 
-  int written = 0, ties_seen = 0;
-  for (int base = 0; base < n; base += kSelThreads) {
-    const int i = base + tid;
-    const bool valid = i < n;
-    const unsigned key = valid ? score_key(sc[i]) : 0u;
-    bool sel = valid;
-    if (!take_all) {
-      const bool is_tie = valid && key == tau;
-      int ties_total;
-      const int tr = block_rank(is_tie, wcount, ties_total);
-      sel = valid && (key > tau || (is_tie && ties_seen + tr < need));
-      ties_seen += ties_total;
-    }
-    int sel_total;
-    const int r = block_rank(sel, wcount, sel_total);
-    if (sel) dst[written + r] = i;
-    written += sel_total;
+  // per-thread counts, block exclusive scan of (ties << 16 | greater)
+  unsigned cnt = 0;
+#pragma unroll
+  for (int i = 0; i < kSelKpt; ++i)
+    if (i < nv) cnt += (key[i] > tau ? 1u : 0u) + (key[i] == tau ? 0x10000u : 0u);
+  unsigned incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
   }
-}
+  if (lane == 31) wsum[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const unsigned v = wsum[lane];
+    unsigned wi = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned t = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += t;
+    }
+    wsum[lane] = wi - v;                                 // exclusive prefix of the warp totals
+    if (lane == 31) {
+#pragma unroll
+      for (unsigned rr = 0; rr < kSelCluster; ++rr) *cluster.map_shared_rank(&tot[r], rr) = wi;
+    }
+  }
+  cluster.sync();                                        // also orders wsum for the block
+  const unsigned excl = wsum[warp] + incl - cnt;
+  int gt_before = 0, tie_before = 0, my_gt = 0, my_tie = 0;
+#pragma unroll
+  for (unsigned rr = 0; rr < kSelCluster; ++rr) {
+    const unsigned t = tot[rr];
+    if (rr < r) { gt_before += (int)(t & 0xFFFFu); tie_before += (int)(t >> 16); }
+    if (rr == r) { my_gt = (int)(t & 0xFFFFu); my_tie = (int)(t >> 16); }
+  }
+  // (a block holds at most 16384 scores, so neither 16-bit field can overflow)
+  int g = gt_before + (int)(excl & 0xFFFFu);
+  int ti = tie_before + (int)(excl >> 16);
+#pragma unroll
+  for (int i = 0; i < kSelKpt; ++i) {
+    if (i < nv) {
+      if (key[i] > tau) {
+        dst[g + (ti < need ? ti : need)] = base + i;
+        ++g;
+      } else if (key[i] == tau) {
+        if (ti < need) dst[g + ti] = base + i;
+        ++ti;
+      }
+    }
+  }
+  __syncthreads();                                       // this block's indices are visible to its warps
 
-// One warp per (compacted row, head): copies the K row and the V row, 16 bytes per lane.
-__global__ void __launch_bounds__(256)
-k_gather(const char *__restrict__ k, const char *__restrict__ v, long long stride_token_b,
-         long long stride_head_b, int row_bytes, int H, SeqTable st, int b0, int nseq,
-         const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
-         const int *__restrict__ out_idx, long long cap, char *__restrict__ out_k,
-         char *__restrict__ out_v) {
-  const int lane = threadIdx.x & 31;
-  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
-  const long long row_lo = out_offsets[b0], row_hi = out_offsets[b0 + nseq];
-  const long long items = (row_hi - row_lo) * H;
+  // gather the rows this block selected: ranks [first, first + count)
+  const int first = gt_before + (tie_before < need ? tie_before : need);
+  int tie_take = need - tie_before;
+  tie_take = tie_take < 0 ? 0 : (tie_take > my_tie ? my_tie : tie_take);
+  const int count = my_gt + tie_take;
   const int n16 = row_bytes >> 4;
-  for (long long it = warp; it < items; it += nwarps) {
-    const long long r = row_lo + it / H;
-    const int h = (int)(it % H);
-    if (r >= cap) continue;
-    int bl = 0;
-    while (bl + 1 < nseq && out_offsets[b0 + bl + 1] <= r) ++bl;
-    const int n = st.start[bl + 1] - st.start[bl];
-    int kk = budgets[b0 + bl];
-    kk = kk > n ? n : kk;
-    const long long off_b = out_offsets[b0 + bl];
-    if (r - off_b >= kk || off_b < 0 || off_b + kk > cap) continue;   // same rule as the selection kernel
-    const long long tok = (long long)st.start[bl] + out_idx[(long long)h * cap + r];
+  for (int rr = warp; rr < count; rr += kSelThreads / 32) {
+    const long long row = off + first + rr;
+    const long long tok = (long long)s0 + dst[first + rr];
     const long long src = tok * stride_token_b + (long long)h * stride_head_b;
-    const long long dsto = (r * H + h) * (long long)row_bytes;
+    const long long dsto = (row * H + h) * (long long)row_bytes;
     for (int u = lane; u < 2 * n16; u += 32) {
       const bool isv = u >= n16;
       const int uu = isv ? u - n16 : u;
-      const uint4 val = *reinterpret_cast<const uint4 *>((isv ? v : k) + src + 16ll * uu);
+      const uint4 val = *reinterpret_cast<const uint4 *>((isv ? vin : kin) + src + 16ll * uu);
       *reinterpret_cast<uint4 *>((isv ? out_v : out_k) + dsto + 16ll * uu) = val;
     }
   }
@@ -352,6 +411,8 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
   if ((kv->head_dim * es) % 16) return FC_ERR_UNSUPPORTED;
   fc_status s = check_cu(kv->cu_seqlens, kv->batch);
   if (s != FC_OK) return s;
+  for (int b = 0; b < kv->batch; ++b)
+    if (kv->cu_seqlens[b + 1] - kv->cu_seqlens[b] > kSelCluster * kSelThreads * kSelKpt) return FC_ERR_UNSUPPORTED;
   if (((uintptr_t)kv->k & 15) || ((uintptr_t)kv->v & 15) || ((uintptr_t)out_k & 15) || ((uintptr_t)out_v & 15))
     return FC_ERR_INVALID_ARG;
   if ((kv->stride_token * es) % 16 || (kv->stride_head * es) % 16) return FC_ERR_INVALID_ARG;
@@ -368,18 +429,11 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
     for (int i = 0; i <= nseq; ++i) tab.start[i] = kv->cu_seqlens[b0 + i];
     {
       ProfScope ps(h, FC_K_SELECT, st);
-      k_select<<<dim3(nseq, kv->num_heads), kSelThreads, 0, st>>>(
+      k_select_gather<<<dim3(kSelCluster * nseq, kv->num_heads), kSelThreads, 0, st>>>(
           scores, T, tab, b0, budgets, reinterpret_cast<const long long *>(out_offsets), out_idx,
-          out_capacity_rows, h->status_word);
-    }
-    if ((s = fc_after_launch(h)) != FC_OK) return s;
-    {
-      ProfScope ps(h, FC_K_GATHER, st);
-      k_gather<<<h->num_sms * 8, 256, 0, st>>>(
-          static_cast<const char *>(kv->k), static_cast<const char *>(kv->v),
-          kv->stride_token * es, kv->stride_head * es, kv->head_dim * es, kv->num_heads, tab, b0, nseq,
-          budgets, reinterpret_cast<const long long *>(out_offsets), out_idx, out_capacity_rows,
-          static_cast<char *>(out_k), static_cast<char *>(out_v));
+          out_capacity_rows, h->status_word, static_cast<const char *>(kv->k),
+          static_cast<const char *>(kv->v), kv->stride_token * es, kv->stride_head * es,
+          kv->head_dim * es, kv->num_heads, static_cast<char *>(out_k), static_cast<char *>(out_v));
     }
     if ((s = fc_after_launch(h)) != FC_OK) return s;
   }
