@@ -34,6 +34,8 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->status_word = nullptr;
   h->group_bytes = (size_t)32 << 20;
   h->launches = 0;
+  h->aux[0] = h->aux[1] = nullptr;
+  h->ev_fork = h->ev_join[0] = h->ev_join[1] = nullptr;
   h->prof_class = FC_K_NONE;
   h->prof_events = nullptr;
   h->prof_cap = 0;
@@ -43,7 +45,12 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->num_sms = prop.multiProcessorCount;
   if (cudaMalloc(&h->master, (size_t)h->master_len * sizeof(float2)) != cudaSuccess ||
       cudaMalloc(&h->status_word, sizeof(int)) != cudaSuccess ||
-      cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess) {
+      cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&h->aux[0], cudaStreamNonBlocking) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&h->aux[1], cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_join[0], cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_join[1], cudaEventDisableTiming) != cudaSuccess) {
     fc_destroy(h);
     return FC_ERR_CUDA;
   }
@@ -105,6 +112,11 @@ extern "C" fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *la
 extern "C" void fc_destroy(fc_handle *h) {
   if (!h) return;
   free_prof(h);
+  for (int i = 0; i < 2; ++i) {
+    if (h->aux[i]) cudaStreamDestroy(h->aux[i]);
+    if (h->ev_join[i]) cudaEventDestroy(h->ev_join[i]);
+  }
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
   if (h->master) cudaFree(h->master);
   if (h->status_word) cudaFree(h->status_word);
   delete h;

@@ -27,6 +27,10 @@ struct fc_handle {
   size_t group_bytes;
   int num_sms;
   unsigned long long launches;
+  // two internal streams: consecutive head groups of one fc_score_layer call are
+  // transformed concurrently on alternating streams and workspace halves
+  cudaStream_t aux[2];
+  cudaEvent_t ev_fork, ev_join[2];
   // optional per-kernel-class timing (fc_profile_begin / fc_profile_end)
   int prof_class;
   cudaEvent_t *prof_events;   // pairs

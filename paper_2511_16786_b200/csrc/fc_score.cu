@@ -486,6 +486,7 @@ SeqPlan plan_sequence(int N) {
 
 struct ScoreLayout {
   size_t off_ws, off_spec, off_hhat, off_hcol, off_part_tot, off_part_hi, total;
+  size_t ws_buf_bytes;       // one group buffer; the fast path keeps two and alternates
   int heads_per_group;
 };
 
@@ -497,9 +498,13 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   int hg = (int)(h->group_bytes / per_head);
   if (hg < 1) hg = 1;
   if (hg > num_heads) hg = num_heads;
+  int groups = (num_heads + hg - 1) / hg;
+  if (sp.fast && groups < 2 && num_heads >= 2) groups = 2;     // keep both internal streams busy
+  hg = (num_heads + groups - 1) / groups;                      // balanced groups
   L.heads_per_group = hg;
+  L.ws_buf_bytes = align_up(per_head * hg, 256);
   size_t off = 0;
-  L.off_ws = off;       off += align_up(per_head * hg, 256);
+  L.off_ws = off;       off += L.ws_buf_bytes * (sp.fast ? 2 : 1);
   L.off_spec = off;     off += sp.bluestein ? align_up((size_t)sp.N * head_dim * hg * sizeof(float2), 256) : 0;
   L.off_hhat = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * sizeof(float2), 256) : 0;
   L.off_hcol = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * 8 * sizeof(float2), 256) : 0;
@@ -653,16 +658,23 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
   }
 
+  if (sp.fast) {
+    FC_CUDA_TRY(cudaEventRecord(h->ev_fork, st));
+    FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[0], h->ev_fork, 0));
+    FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[1], h->ev_fork, 0));
+  }
   size_t tot_slots = 0, hi_slots = 0;
-  for (int h0 = 0; h0 < H; h0 += L.heads_per_group) {
+  int group = 0;
+  for (int h0 = 0; h0 < H; h0 += L.heads_per_group, ++group) {
     const int hg = (H - h0 < L.heads_per_group) ? H - h0 : L.heads_per_group;
     const int ncol_ws = hg * d;
     double *ptot = part_tot + 2 * tot_slots;
     double *phi = part_hi + 2 * hi_slots;
     const size_t sm3 = smem_pass13(sp, sp.cs);
     if (sp.fast) {
-      if ((s = launch_fast<T>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores + start,
-                              total_tokens)) != FC_OK) return s;
+      float2 *wsg = reinterpret_cast<float2 *>(wsb + L.off_ws + (size_t)(group & 1) * L.ws_buf_bytes);
+      if ((s = launch_fast<T>(h, h->aux[group & 1], kv, kp, vp, sp, h0, hg, omega, wsg, ptot, phi,
+                              scores + start, total_tokens)) != FC_OK) return s;
     } else if (!sp.bluestein) {
       KvLoader<T, false> ld{kp, vp, kv->stride_token, kv->stride_head, h0, d, N, 0.f, 0.f};
       if ((s = launch_pass1(h, st, ld, sp, ncol_ws, sp.cs, ws, ptot)) != FC_OK) return s;
@@ -702,6 +714,12 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     }
     tot_slots += (size_t)sp.N2 * (ncol_ws / sp.cs);
     hi_slots += (size_t)sp.N2 * hg;
+  }
+  if (sp.fast) {
+    for (int i = 0; i < 2; ++i) {
+      FC_CUDA_TRY(cudaEventRecord(h->ev_join[i], h->aux[i]));
+      FC_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_join[i], 0));
+    }
   }
   {
     ProfScope ps(h, FC_K_OTHER, st);
