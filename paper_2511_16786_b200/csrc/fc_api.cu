@@ -32,6 +32,7 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->master_len = 4 * p2;
   h->master = nullptr;
   h->status_word = nullptr;
+  h->done_counter = nullptr;
   h->group_bytes = (size_t)32 << 20;
   h->launches = 0;
   h->aux[0] = h->aux[1] = nullptr;
@@ -46,6 +47,8 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   if (cudaMalloc(&h->master, (size_t)h->master_len * sizeof(float2)) != cudaSuccess ||
       cudaMalloc(&h->status_word, sizeof(int)) != cudaSuccess ||
       cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess ||
+      cudaMalloc(&h->done_counter, sizeof(unsigned)) != cudaSuccess ||
+      cudaMemset(h->done_counter, 0, sizeof(unsigned)) != cudaSuccess ||
       cudaStreamCreateWithFlags(&h->aux[0], cudaStreamNonBlocking) != cudaSuccess ||
       cudaStreamCreateWithFlags(&h->aux[1], cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
@@ -119,6 +122,7 @@ extern "C" void fc_destroy(fc_handle *h) {
   if (h->ev_fork) cudaEventDestroy(h->ev_fork);
   if (h->master) cudaFree(h->master);
   if (h->status_word) cudaFree(h->status_word);
+  if (h->done_counter) cudaFree(h->done_counter);
   delete h;
 }
 

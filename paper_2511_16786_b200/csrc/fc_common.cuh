@@ -24,6 +24,7 @@ struct fc_handle {
   int master_len;          // power of two; master[i] = exp(-2*pi*i*j/master_len)
   float2 *master;          // DEVICE
   int *status_word;        // DEVICE
+  unsigned *done_counter;  // DEVICE, zero between calls (the last block of a sequence resets it)
   size_t group_bytes;
   int num_sms;
   unsigned long long launches;

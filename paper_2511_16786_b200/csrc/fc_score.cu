@@ -578,7 +578,8 @@ fc_status launch_pass2(fc_handle *h, cudaStream_t st, const SeqPlan &sp, int nco
 template <typename T, int R1B, int R2B>
 fc_status launch_fast_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp,
                            const SeqPlan &sp, int h0, int hg, int omega, float2 *ws, double *ptot,
-                           double *phi, float *scores, long long total_tokens) {
+                           double *phi, float *scores, long long total_tokens, const double *part_tot,
+                           const double *part_hi, double *energy_b) {
   constexpr int N1 = 16 * R1B, N2 = 16 * R2B;
   const int d = kv->head_dim, ncol_ws = hg * d;
   const size_t sm1 = (size_t)N1 * 32 * sizeof(float4) + N1 * sizeof(float2);
@@ -602,8 +603,10 @@ fc_status launch_fast_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, 
   {
     ProfScope ps(h, FC_K_PASS3, st);
     const float inv = (float)(1.0 / ((double)sp.N * (double)sp.N * (double)d));
-    fast::k_p3<R1B><<<dim3(N2, hg), 32 * R1B, sm1, st>>>(sp.N, N2, ncol_ws, ws, h->master, h->master_len, scores,
-                                                         h0, d, total_tokens, inv, phi);
+    const int H = kv->num_heads;
+    fast::k_p3<R1B><<<dim3(N2, hg), 32 * R1B, sm1, st>>>(
+        sp.N, N2, ncol_ws, ws, h->master, h->master_len, scores, h0, d, total_tokens, inv, phi,
+        h->done_counter, (unsigned)(N2 * H), part_tot, N2 * (H * d / 64), part_hi, N2 * H, energy_b);
   }
   return fc_after_launch(h);
 }
@@ -611,10 +614,12 @@ fc_status launch_fast_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, 
 template <typename T>
 fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp,
                       const SeqPlan &sp, int h0, int hg, int omega, float2 *ws, double *ptot, double *phi,
-                      float *scores, long long total_tokens) {
+                      float *scores, long long total_tokens, const double *part_tot, const double *part_hi,
+                      double *energy_b) {
 #define FC_FAST_CASE(A, B)                                                                                  \
   if (sp.N1 == 16 * A && sp.N2 == 16 * B)                                                                   \
-    return launch_fast_impl<T, A, B>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores, total_tokens);
+    return launch_fast_impl<T, A, B>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores, total_tokens, \
+                                     part_tot, part_hi, energy_b);
   FC_FAST_CASE(2, 2) FC_FAST_CASE(2, 4) FC_FAST_CASE(4, 4) FC_FAST_CASE(4, 8)
   FC_FAST_CASE(8, 8) FC_FAST_CASE(8, 16) FC_FAST_CASE(16, 16)
 #undef FC_FAST_CASE
@@ -674,7 +679,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     if (sp.fast) {
       float2 *wsg = reinterpret_cast<float2 *>(wsb + L.off_ws + (size_t)(group & 1) * L.ws_buf_bytes);
       if ((s = launch_fast<T>(h, h->aux[group & 1], kv, kp, vp, sp, h0, hg, omega, wsg, ptot, phi,
-                              scores + start, total_tokens)) != FC_OK) return s;
+                              scores + start, total_tokens, part_tot, part_hi, energy_b)) != FC_OK) return s;
     } else if (!sp.bluestein) {
       KvLoader<T, false> ld{kp, vp, kv->stride_token, kv->stride_head, h0, d, N, 0.f, 0.f};
       if ((s = launch_pass1(h, st, ld, sp, ncol_ws, sp.cs, ws, ptot)) != FC_OK) return s;
@@ -721,6 +726,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       FC_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_join[i], 0));
     }
   }
+  if (sp.fast) return FC_OK;          // the last pass-3 block of the sequence has written the energy sums
   {
     ProfScope ps(h, FC_K_OTHER, st);
     k_energy_finalize<<<1, 256, 0, st>>>(part_tot, (int)tot_slots, part_hi, (int)hi_slots, energy_b);

@@ -302,7 +302,9 @@ template <int R1B>
 __global__ void __launch_bounds__(32 * R1B)
 k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__restrict__ master,
      int master_len, float *__restrict__ scores, int head0, int head_dim, long long score_stride,
-     float inv_scale, double *__restrict__ partial) {
+     float inv_scale, double *__restrict__ partial, unsigned *__restrict__ done_counter,
+     unsigned total_blocks, const double *__restrict__ part_tot, int n_tot,
+     const double *__restrict__ part_hi, int n_hi, double *__restrict__ energy) {
   constexpr int N1 = 16 * R1B, NT = 32 * R1B, IT = 16 / R1B;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                        // [N1][32]
@@ -389,6 +391,30 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
     partial[2 * slot] = sa * (double)head_dim;
     partial[2 * slot + 1] = sb * (double)head_dim;
   }
+  // The last block of the sequence (over all head groups, on either stream) adds up the
+  // per-block partial sums in a fixed order: energy = (hiK, totK, hiV, totV).
+  __shared__ bool is_last;
+  if (tid == 0) {
+    __threadfence();
+    const unsigned prev = atomicAdd(done_counter, 1u);
+    is_last = (prev + 1u == total_blocks);
+    if (is_last) *done_counter = 0u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  double *redd = reinterpret_cast<double *>(smem4);        // [4][NT], the tile is no longer needed
+  double a0 = 0, a1 = 0, b0 = 0, b1 = 0;
+  for (int i = tid; i < n_tot; i += NT) { a0 += __ldcg(part_tot + 2 * i); a1 += __ldcg(part_tot + 2 * i + 1); }
+  for (int i = tid; i < n_hi; i += NT) { b0 += __ldcg(part_hi + 2 * i); b1 += __ldcg(part_hi + 2 * i + 1); }
+  redd[tid] = b0; redd[NT + tid] = a0; redd[2 * NT + tid] = b1; redd[3 * NT + tid] = a1;
+  __syncthreads();
+  for (int st = NT / 2; st > 0; st >>= 1) {
+    if (tid < st)
+      for (int q = 0; q < 4; ++q) redd[q * NT + tid] += redd[q * NT + tid + st];
+    __syncthreads();
+  }
+  if (tid < 4) energy[tid] = redd[tid * NT];
 }
 
 }  // namespace fast
