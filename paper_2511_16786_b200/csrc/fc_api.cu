@@ -2,6 +2,7 @@
 #include "fc_common.cuh"
 
 #include <new>
+#include <stdlib.h>
 
 namespace {
 
@@ -34,6 +35,11 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->status_word = nullptr;
   h->done_counter = nullptr;
   h->group_bytes = (size_t)32 << 20;
+  // Developer tuning knobs (tile widths in channel pairs); the defaults are the measured best.
+  h->tune_cpw = 32;
+  h->tune_cp = 8;
+  if (const char *e = getenv("FC_TUNE_CPW")) { const int v = atoi(e); if (v == 16 || v == 32) h->tune_cpw = v; }
+  if (const char *e = getenv("FC_TUNE_CP")) { const int v = atoi(e); if (v == 4 || v == 8) h->tune_cp = v; }
   h->launches = 0;
   h->aux[0] = h->aux[1] = nullptr;
   h->ev_fork = h->ev_join[0] = h->ev_join[1] = nullptr;

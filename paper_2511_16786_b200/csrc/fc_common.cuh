@@ -26,6 +26,7 @@ struct fc_handle {
   int *status_word;        // DEVICE
   unsigned *done_counter;  // DEVICE, zero between calls (the last block of a sequence resets it)
   size_t group_bytes;
+  int tune_cpw, tune_cp;   // tile widths of the specialised kernels (channel pairs), see fc_create
   int num_sms;
   unsigned long long launches;
   // two internal streams: consecutive head groups of one fc_score_layer call are

@@ -508,7 +508,7 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   L.off_spec = off;     off += sp.bluestein ? align_up((size_t)sp.N * head_dim * hg * sizeof(float2), 256) : 0;
   L.off_hhat = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * sizeof(float2), 256) : 0;
   L.off_hcol = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * 8 * sizeof(float2), 256) : 0;
-  const size_t slices = (size_t)num_heads * head_dim / sp.cs;
+  const size_t slices = (size_t)num_heads * head_dim / 32;   // finest slicing any kernel variant uses
   L.off_part_tot = off; off += align_up(slices * sp.N2 * 2 * sizeof(double), 256);
   L.off_part_hi = off;  off += align_up((size_t)num_heads * sp.N2 * 2 * sizeof(double), 256);
   L.total = off;
@@ -538,6 +538,8 @@ fc_status validate_view(const fc_handle *h, const fc_kv_view *kv) {
 template <class Kern>
 fc_status set_smem(Kern kern, size_t bytes) {
   if (bytes > 48 * 1024) FC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+  // as much of the L1/shared array as shared memory as the device offers: these kernels do not rely on L1
+  FC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
   return FC_OK;
 }
 
@@ -575,40 +577,56 @@ fc_status launch_pass2(fc_handle *h, cudaStream_t st, const SeqPlan &sp, int nco
 }
 
 // The three specialised launches for one head group of a power-of-two sequence.
-template <typename T, int R1B, int R2B>
+// CPW: channel pairs per block in passes 1 and 3; CP: channel pairs per half tile in pass 2.
+template <typename T, int R1B, int R2B, int CPW, int CP>
 fc_status launch_fast_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp,
                            const SeqPlan &sp, int h0, int hg, int omega, float2 *ws, double *ptot,
                            double *phi, float *scores, long long total_tokens, const double *part_tot,
                            const double *part_hi, double *energy_b) {
   constexpr int N1 = 16 * R1B, N2 = 16 * R2B;
   const int d = kv->head_dim, ncol_ws = hg * d;
-  const size_t sm1 = (size_t)N1 * 32 * sizeof(float4) + N1 * sizeof(float2);
-  const size_t sm2 = (size_t)2 * N2 * 8 * sizeof(float4) + 3 * N2 * sizeof(float2);
+  const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
+  const size_t sm2 = (size_t)2 * N2 * CP * sizeof(float4) + 5 * N2 * sizeof(float2);
   fc_status s;
-  if ((s = set_smem(fast::k_p1<T, R1B>, sm1)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p1<T, R1B, CPW>, sm1)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS1, st);
-    fast::k_p1<T, R1B><<<dim3(N2, ncol_ws / 64), 32 * R1B, sm1, st>>>(
+    fast::k_p1<T, R1B, CPW><<<dim3(N2, ncol_ws / (2 * CPW)), CPW * R1B, sm1, st>>>(
         kp, vp, kv->stride_token, kv->stride_head, h0, d, sp.N, N2, ncol_ws, ws, h->master, h->master_len, ptot);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
-  if ((s = set_smem(fast::k_p2<R2B>, sm2)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p2<R2B, CP>, sm2)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS2, st);
-    fast::k_p2<R2B><<<dim3(N1 / 2 + 1, ncol_ws / 16), 16 * R2B, sm2, st>>>(N1, ncol_ws, ws, h->master,
-                                                                          h->master_len, omega);
+    fast::k_p2<R2B, CP><<<dim3(N1 / 2 + 1, ncol_ws / (2 * CP)), 2 * CP * R2B, sm2, st>>>(
+        N1, ncol_ws, ws, h->master, h->master_len, omega);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
-  if ((s = set_smem(fast::k_p3<R1B>, sm1)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p3<R1B, CPW>, sm1)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS3, st);
     const float inv = (float)(1.0 / ((double)sp.N * (double)sp.N * (double)d));
     const int H = kv->num_heads;
-    fast::k_p3<R1B><<<dim3(N2, hg), 32 * R1B, sm1, st>>>(
+    fast::k_p3<R1B, CPW><<<dim3(N2, hg), CPW * R1B, sm1, st>>>(
         sp.N, N2, ncol_ws, ws, h->master, h->master_len, scores, h0, d, total_tokens, inv, phi,
-        h->done_counter, (unsigned)(N2 * H), part_tot, N2 * (H * d / 64), part_hi, N2 * H, energy_b);
+        h->done_counter, (unsigned)(N2 * H), part_tot, N2 * (H * d / (2 * CPW)), part_hi, N2 * H, energy_b);
   }
   return fc_after_launch(h);
+}
+
+template <typename T, int CPW, int CP>
+fc_status launch_fast_tuned(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp,
+                            const SeqPlan &sp, int h0, int hg, int omega, float2 *ws, double *ptot, double *phi,
+                            float *scores, long long total_tokens, const double *part_tot,
+                            const double *part_hi, double *energy_b) {
+#define FC_FAST_CASE(A, B)                                                                                \
+  if (sp.N1 == 16 * A && sp.N2 == 16 * B)                                                                 \
+    return launch_fast_impl<T, A, B, CPW, CP>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores, \
+                                              total_tokens, part_tot, part_hi, energy_b);
+  FC_FAST_CASE(2, 2) FC_FAST_CASE(2, 4) FC_FAST_CASE(4, 4) FC_FAST_CASE(4, 8)
+  FC_FAST_CASE(8, 8) FC_FAST_CASE(8, 16) FC_FAST_CASE(16, 16)
+#undef FC_FAST_CASE
+  return FC_ERR_INTERNAL;
 }
 
 template <typename T>
@@ -616,13 +634,12 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
                       const SeqPlan &sp, int h0, int hg, int omega, float2 *ws, double *ptot, double *phi,
                       float *scores, long long total_tokens, const double *part_tot, const double *part_hi,
                       double *energy_b) {
-#define FC_FAST_CASE(A, B)                                                                                  \
-  if (sp.N1 == 16 * A && sp.N2 == 16 * B)                                                                   \
-    return launch_fast_impl<T, A, B>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores, total_tokens, \
-                                     part_tot, part_hi, energy_b);
-  FC_FAST_CASE(2, 2) FC_FAST_CASE(2, 4) FC_FAST_CASE(4, 4) FC_FAST_CASE(4, 8)
-  FC_FAST_CASE(8, 8) FC_FAST_CASE(8, 16) FC_FAST_CASE(16, 16)
-#undef FC_FAST_CASE
+#define FC_TUNE_CASE(W, C)                                                                              \
+  if (h->tune_cpw == W && h->tune_cp == C)                                                              \
+    return launch_fast_tuned<T, W, C>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores,       \
+                                      total_tokens, part_tot, part_hi, energy_b);
+  FC_TUNE_CASE(32, 8) FC_TUNE_CASE(32, 4) FC_TUNE_CASE(16, 8) FC_TUNE_CASE(16, 4)
+#undef FC_TUNE_CASE
   return FC_ERR_INTERNAL;
 }
 
@@ -717,7 +734,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       }
       if ((s = fc_after_launch(h)) != FC_OK) return s;
     }
-    tot_slots += (size_t)sp.N2 * (ncol_ws / sp.cs);
+    tot_slots += (size_t)sp.N2 * (ncol_ws / (sp.fast ? 2 * h->tune_cpw : sp.cs));
     hi_slots += (size_t)sp.N2 * hg;
   }
   if (sp.fast) {

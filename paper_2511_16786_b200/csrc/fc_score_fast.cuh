@@ -47,22 +47,22 @@ template <int R>
 __device__ __forceinline__ void dft_inv(float2 (&x)[R]) { dft_small<R, +1>(x); }
 
 // ---------------------------------------------------------------------------
-// pass 1: grid (N2, group columns / 64), block 32*R1B.
-// Thread (cp = lane, j = warp): channels 2cp, 2cp+1 of the slice; first stage
-// points n1 = j + R1B*p, p = 0..15, loaded from the K/V rows.
+// pass 1: grid (N2, group columns / (2*CPW)), block CPW*R1B.
+// Thread (cp = tid % CPW, j = tid / CPW): channels 2cp, 2cp+1 of the slice; first
+// stage points n1 = j + R1B*p, p = 0..15, loaded from the K/V rows.
 // ---------------------------------------------------------------------------
-template <typename T, int R1B>
-__global__ void __launch_bounds__(32 * R1B)
+template <typename T, int R1B, int CPW>
+__global__ void __launch_bounds__(CPW * R1B)
 k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, long long stride_head,
      int head0, int head_dim, int N, int N2, int ncol_ws, float2 *__restrict__ ws,
      const float2 *__restrict__ master, int master_len, double *__restrict__ partial) {
-  constexpr int N1 = 16 * R1B, NT = 32 * R1B, IT = 16 / R1B;
+  constexpr int N1 = 16 * R1B, NT = CPW * R1B, IT = 16 / R1B, NW = (NT + 31) / 32;
   extern __shared__ float4 smem4[];
-  float4 *S = smem4;                                        // [N1][32]
-  float2 *tw = reinterpret_cast<float2 *>(S + N1 * 32);     // [N1]
-  __shared__ double red[2][R1B];
-  const int tid = threadIdx.x, cp = tid & 31, j = tid >> 5;
-  const int n2 = blockIdx.x, gc0 = blockIdx.y * 64;
+  float4 *S = smem4;                                        // [N1][CPW]
+  float2 *tw = reinterpret_cast<float2 *>(S + N1 * CPW);    // [N1]
+  __shared__ double red[2][NW];
+  const int tid = threadIdx.x, cp = tid % CPW, j = tid / CPW;
+  const int n2 = blockIdx.x, gc0 = blockIdx.y * (2 * CPW);
   const int h = head0 + gc0 / head_dim, c = gc0 % head_dim + 2 * cp;
   const T *kb = k + (long long)h * stride_head + c;
   const T *vb = v + (long long)h * stride_head + c;
@@ -93,7 +93,7 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
       x0[p] = cmul(x0[p], w);
       x1[p] = cmul(x1[p], w);
     }
-    S[(j + R1B * p) * 32 + cp] = make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
+    S[(j + R1B * p) * CPW + cp] = make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
   }
   __syncthreads();
   // second stage: radix R1B inside sub-block pp; bin k1 = pp + 16*q
@@ -103,7 +103,7 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
     float2 y0[R1B], y1[R1B];
 #pragma unroll
     for (int q = 0; q < R1B; ++q) {
-      const float4 t = S[(q + R1B * pp) * 32 + cp];
+      const float4 t = S[(q + R1B * pp) * CPW + cp];
       y0[q] = make_float2(t.x, t.y);
       y1[q] = make_float2(t.z, t.w);
     }
@@ -118,12 +118,12 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
   }
   // per-block sums of squares (total energy of Eq. 12, by Parseval)
   const double a = warp_sum_d((double)accK), b = warp_sum_d((double)accV);
-  if (cp == 0) { red[0][j] = a; red[1][j] = b; }
+  if ((tid & 31) == 0) { red[0][tid >> 5] = a; red[1][tid >> 5] = b; }
   __syncthreads();
   if (tid == 0) {
     double sa = 0, sb = 0;
 #pragma unroll
-    for (int i = 0; i < R1B; ++i) { sa += red[0][i]; sb += red[1][i]; }
+    for (int i = 0; i < NW; ++i) { sa += red[0][i]; sb += red[1][i]; }
     const size_t slot = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
     partial[2 * slot] = sa;
     partial[2 * slot + 1] = sb;
@@ -131,37 +131,40 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
 }
 
 // ---------------------------------------------------------------------------
-// pass 2: grid (N1/2 + 1, group columns / 16), block 16*R2B.
-// Thread (cp = tid&7, hf = (tid>>3)&1, j = tid>>4): channel pair cp of the
-// 16-column slice, half hf (k1 = blockIdx.x or N1 - blockIdx.x), first-stage
-// points n2 = j + R2B*p.
+// pass 2: grid (N1/2 + 1, group columns / (2*CP)), block 2*CP*R2B.
+// Thread (cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2*CP)): channel pair cp of
+// the slice, half hf (k1 = blockIdx.x or N1 - blockIdx.x), first-stage points
+// n2 = j + R2B*p.
 // ---------------------------------------------------------------------------
-template <int R2B>
-__global__ void __launch_bounds__(16 * R2B, (R2B >= 16 ? 2 : 4))
+template <int R2B, int CP>
+__global__ void __launch_bounds__(2 * CP * R2B, 512 / (2 * CP * R2B > 32 ? 2 * CP * R2B : 32))
 k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ master, int master_len,
      int omega) {
-  constexpr int N2 = 16 * R2B, NT = 16 * R2B, IT = 16 / R2B;
+  constexpr int N2 = 16 * R2B, NT = 2 * CP * R2B, IT = 16 / R2B;
   extern __shared__ float4 smem4[];
-  float4 *S = smem4;                                         // [2][N2][8]
-  float2 *tw = reinterpret_cast<float2 *>(S + 2 * N2 * 8);   // [N2]   w_N2^i
+  float4 *S = smem4;                                         // [2][N2][CP]
+  float2 *tw = reinterpret_cast<float2 *>(S + 2 * N2 * CP);  // [N2]   w_N2^i
   float2 *twN = tw + N2;                                     // [2][N2] w_N^(n2*k1)
-  const int tid = threadIdx.x, cp = tid & 7, hf = (tid >> 3) & 1, j = tid >> 4;
-  const int k1a = blockIdx.x, k1b = (N1 - k1a) % N1;
+  float2 *uT = twN + 2 * N2;                                 // [2][N2] exp(-j*pi*(k1 + N1*k2)/N)
+  const int tid = threadIdx.x, cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
+  const int k1a = blockIdx.x, k1b = (N1 - k1a) & (N1 - 1);
   const bool self = (k1a == k1b);
   const int k1 = hf ? k1b : k1a;
   const int N = N1 * N2;
-  const int gc0 = blockIdx.y * 16;
+  const int gc0 = blockIdx.y * (2 * CP);
   const bool active = !(self && hf);
 
   {
-    const int mstepN = master_len / N;
+    const int mstepN = master_len / N, ustep = master_len / (2 * N);
     for (int i = tid; i < N2; i += NT) {
       tw[i] = master[(size_t)i * (master_len / N2)];
-      twN[i] = master[(size_t)(((long long)i * k1a) % N) * mstepN];
-      twN[N2 + i] = master[(size_t)(((long long)i * k1b) % N) * mstepN];
+      twN[i] = master[(size_t)((i * k1a) & (N - 1)) * mstepN];
+      twN[N2 + i] = master[(size_t)((i * k1b) & (N - 1)) * mstepN];
+      uT[i] = master[(size_t)(k1a + N1 * i) * ustep];
+      uT[N2 + i] = master[(size_t)(k1b + N1 * i) * ustep];
     }
   }
-  float4 *Sh = S + hf * (N2 * 8);
+  float4 *Sh = S + hf * (N2 * CP);
   float2 x0[16], x1[16];
   float2 *base = ws + ((size_t)k1 * N2) * ncol_ws + gc0 + 2 * cp;
   if (active) {
@@ -189,7 +192,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
         x0[p] = cmul(x0[p], w);
         x1[p] = cmul(x1[p], w);
       }
-      Sh[(j + R2B * p) * 8 + cp] = make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
+      Sh[(j + R2B * p) * CP + cp] = make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
     }
   }
   __syncthreads();
@@ -202,7 +205,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       float2 y0[R2B], y1[R2B];
 #pragma unroll
       for (int q = 0; q < R2B; ++q) {
-        const float4 t = Sh[(q + R2B * pp) * 8 + cp];
+        const float4 t = Sh[(q + R2B * pp) * CP + cp];
         y0[q] = make_float2(t.x, t.y);
         y1[q] = make_float2(t.z, t.w);
       }
@@ -212,14 +215,13 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       for (int q = 0; q < R2B; ++q) {
         x0[it * R2B + q] = y0[q];
         x1[it * R2B + q] = y1[q];
-        Sh[(q + R2B * pp) * 8 + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
+        Sh[(q + R2B * pp) * CP + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
       }
     }
   }
   __syncthreads();       // full spectra of both halves are in shared memory
   if (active) {
-    const float4 *Sp = S + (self ? hf : 1 - hf) * (N2 * 8);
-    const int ustep = master_len / (2 * N);
+    const float4 *Sp = S + (self ? hf : 1 - hf) * (N2 * CP);
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
       const int pp = j + R2B * it;
@@ -234,8 +236,8 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
           P1 = make_float2(0.f, 0.f);
         } else if (inL || inH) {
           const int k2p = (k1 == 0) ? ((N2 - k2) & (N2 - 1)) : (N2 - 1 - k2);
-          const float4 t = Sp[((k2p >> 4) + R2B * (k2p & 15)) * 8 + cp];
-          float2 u = __ldg(master + (size_t)bin * ustep);          // exp(-j*pi*bin/N)
+          const float4 t = Sp[((k2p >> 4) + R2B * (k2p & 15)) * CP + cp];
+          float2 u = uT[hf * N2 + k2];                             // exp(-j*pi*bin/N)
           const float sgn = inL ? -0.5f : 0.5f;                   // E = (P -/+ uQ)/2 with u = exp(+j*pi*bin/N)
           u = make_float2(u.x * sgn, -u.y * sgn);
           const float2 q0 = make_float2(t.x, t.y), q1 = make_float2(t.z, t.w);
@@ -265,7 +267,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       const int pp = j + R2B * it;
 #pragma unroll
       for (int q = 0; q < R2B; ++q)
-        Sh[(q + R2B * pp) * 8 + cp] = make_float4(x0[it * R2B + q].x, x0[it * R2B + q].y,
+        Sh[(q + R2B * pp) * CP + cp] = make_float4(x0[it * R2B + q].x, x0[it * R2B + q].y,
                                                   x1[it * R2B + q].x, x1[it * R2B + q].y);
     }
   }
@@ -273,7 +275,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   if (active) {
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
-      const float4 t = Sh[(j + R2B * p) * 8 + cp];
+      const float4 t = Sh[(j + R2B * p) * CP + cp];
       x0[p] = make_float2(t.x, t.y);
       x1[p] = make_float2(t.z, t.w);
       if (p > 0) {
@@ -294,33 +296,34 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
 }
 
 // ---------------------------------------------------------------------------
-// pass 3: grid (N2, heads of the group), block 32*R1B.  Inverse DFT over k1,
+// pass 3: grid (N2, heads of the group), block CPW*R1B.  Inverse DFT over k1,
 // squared magnitude summed over the channels of the head, scores and the
 // per-block outlier-energy partial sums.
 // ---------------------------------------------------------------------------
-template <int R1B>
-__global__ void __launch_bounds__(32 * R1B)
+template <int R1B, int CPW>
+__global__ void __launch_bounds__(CPW * R1B)
 k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__restrict__ master,
      int master_len, float *__restrict__ scores, int head0, int head_dim, long long score_stride,
      float inv_scale, double *__restrict__ partial, unsigned *__restrict__ done_counter,
      unsigned total_blocks, const double *__restrict__ part_tot, int n_tot,
      const double *__restrict__ part_hi, int n_hi, double *__restrict__ energy) {
-  constexpr int N1 = 16 * R1B, NT = 32 * R1B, IT = 16 / R1B;
+  constexpr int N1 = 16 * R1B, NT = CPW * R1B, IT = 16 / R1B, NW = (NT + 31) / 32;
   extern __shared__ float4 smem4[];
-  float4 *S = smem4;                                        // [N1][32]
-  float2 *tw = reinterpret_cast<float2 *>(S + N1 * 32);     // [N1]
-  __shared__ double red[2][R1B];
-  const int tid = threadIdx.x, cp = tid & 31, j = tid >> 5;
+  float4 *S = smem4;                                        // [N1][CPW]
+  float2 *tw = reinterpret_cast<float2 *>(S + N1 * CPW);    // [N1]
+  __shared__ double red[2][NW];
+  const int tid = threadIdx.x, cp = tid % CPW, j = tid / CPW;
   const int n2 = blockIdx.x, hh = blockIdx.y;
   for (int i = tid; i < N1; i += NT) tw[i] = master[(size_t)i * (master_len / N1)];
 
-  float acc[32];            // [0..15] K part of rows j + R1B*p, [16..31] V part
+  float acc[16];            // |residual|^2 of rows j + R1B*p summed over this thread's channels (K and V)
 #pragma unroll
-  for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+  for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+  float totK = 0.f, totV = 0.f;
 
-  const int nslices = head_dim / 64;
+  const int nslices = head_dim / (2 * CPW);
   for (int sl = 0; sl < nslices; ++sl) {
-    const int gc0 = hh * head_dim + sl * 64;
+    const int gc0 = hh * head_dim + sl * (2 * CPW);
     // inverse radix-R1B stage on bins k1 = pp + 16*q, straight from the workspace
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
@@ -337,13 +340,13 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
       dft_inv<R1B>(y1);
 #pragma unroll
       for (int q = 0; q < R1B; ++q)
-        S[(q + R1B * pp) * 32 + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
+        S[(q + R1B * pp) * CPW + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
     }
     __syncthreads();
     float2 x0[16], x1[16];
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
-      const float4 t = S[(j + R1B * p) * 32 + cp];
+      const float4 t = S[(j + R1B * p) * CPW + cp];
       x0[p] = make_float2(t.x, t.y);
       x1[p] = make_float2(t.z, t.w);
       if (p > 0) {
@@ -356,37 +359,48 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
     dft_inv<16>(x1);
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
-      acc[p] = fmaf(x0[p].x, x0[p].x, fmaf(x1[p].x, x1[p].x, acc[p]));
-      acc[16 + p] = fmaf(x0[p].y, x0[p].y, fmaf(x1[p].y, x1[p].y, acc[16 + p]));
+      const float ek = fmaf(x0[p].x, x0[p].x, x1[p].x * x1[p].x);
+      const float ev = fmaf(x0[p].y, x0[p].y, x1[p].y * x1[p].y);
+      totK += ek;
+      totV += ev;
+      acc[p] += ek + ev;
     }
     __syncthreads();
   }
-  // transposed warp reduction: lane l ends with the sum over all lanes of acc[l]
-  const int lane = cp;
+  // transposed reduction over the CPW lanes that share j: the 16 row sums are halved at every
+  // step until one is left, further steps are plain adds; row p = cp >> log2(CPW/16)
+  {
+    int count = 16;
 #pragma unroll
-  for (int s = 16; s >= 1; s >>= 1) {
+    for (int s = CPW / 2; s >= 1; s >>= 1) {
+      if (count > 1) {
+        const int half = count / 2;
 #pragma unroll
-    for (int i = 0; i < s; ++i) {
-      const bool up = (lane & s) != 0;
-      const float send = up ? acc[i] : acc[i + s];
-      const float keep = up ? acc[i + s] : acc[i];
-      acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        for (int i = 0; i < half; ++i) {
+          const bool up = (cp & s) != 0;
+          const float send = up ? acc[i] : acc[i + half];
+          const float keep = up ? acc[i + half] : acc[i];
+          acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        }
+        count = half;
+      } else {
+        acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], s);
+      }
     }
   }
-  const float mine = acc[0] * inv_scale;                           // K part (lane < 16) or V part of row p = lane & 15
-  const float other = __shfl_xor_sync(0xffffffffu, mine, 16);
-  if (lane < 16) {
-    const int p = (j + R1B * lane) * N2 + n2;
-    scores[(long long)(head0 + hh) * score_stride + perm_token(p, N)] = mine + other;
+  constexpr int DUP = CPW / 16;                             // lanes that end with the same row sum
+  if ((cp & (DUP - 1)) == 0) {
+    const int p = (j + R1B * (cp / DUP)) * N2 + n2;
+    scores[(long long)(head0 + hh) * score_stride + perm_token(p, N)] = acc[0] * inv_scale;
   }
-  const double dk = warp_sum_d(lane < 16 ? (double)mine : 0.0);
-  const double dv = warp_sum_d(lane < 16 ? 0.0 : (double)mine);
-  if (lane == 0) { red[0][j] = dk; red[1][j] = dv; }
+  const double dk = warp_sum_d((double)(totK * inv_scale));
+  const double dv = warp_sum_d((double)(totV * inv_scale));
+  if ((tid & 31) == 0) { red[0][tid >> 5] = dk; red[1][tid >> 5] = dv; }
   __syncthreads();
   if (tid == 0) {
     double sa = 0, sb = 0;
 #pragma unroll
-    for (int i = 0; i < R1B; ++i) { sa += red[0][i]; sb += red[1][i]; }
+    for (int i = 0; i < NW; ++i) { sa += red[0][i]; sb += red[1][i]; }
     const size_t slot = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
     partial[2 * slot] = sa * (double)head_dim;
     partial[2 * slot + 1] = sb * (double)head_dim;

@@ -167,7 +167,7 @@ __device__ __forceinline__ unsigned score_key(float x) {
 
 constexpr int kSelThreads = 1024;   // threads per block of the selection kernel
 constexpr int kSelCluster = 8;      // blocks (one cluster) per (sequence, head)
-constexpr int kSelKpt = 16;         // scores per thread: 8 * 1024 * 16 = 131072 tokens at most
+constexpr int kSelKptMax = 16;      // scores per thread: 8 * 1024 * 16 = 131072 tokens at most
 
 // Selection + compaction + row gather for one (sequence, head), by one cluster of
 // kSelCluster blocks.  Block r of the cluster owns the contiguous token range
@@ -177,6 +177,7 @@ constexpr int kSelKpt = 16;         // scores per thread: 8 * 1024 * 16 = 131072
 // are then ranked in token order (block prefix + cluster prefix), written as
 // ascending indices, and their K/V rows are copied by the same block.
 // grid (kSelCluster * sequences in chunk, heads), cluster (kSelCluster, 1, 1).
+template <int kSelKpt>
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 k_select_gather(const float *__restrict__ scores, long long T, SeqTable st, int b0,
                 const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
@@ -412,7 +413,7 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
   fc_status s = check_cu(kv->cu_seqlens, kv->batch);
   if (s != FC_OK) return s;
   for (int b = 0; b < kv->batch; ++b)
-    if (kv->cu_seqlens[b + 1] - kv->cu_seqlens[b] > kSelCluster * kSelThreads * kSelKpt) return FC_ERR_UNSUPPORTED;
+    if (kv->cu_seqlens[b + 1] - kv->cu_seqlens[b] > kSelCluster * kSelThreads * kSelKptMax) return FC_ERR_UNSUPPORTED;
   if (((uintptr_t)kv->k & 15) || ((uintptr_t)kv->v & 15) || ((uintptr_t)out_k & 15) || ((uintptr_t)out_v & 15))
     return FC_ERR_INVALID_ARG;
   if ((kv->stride_token * es) % 16 || (kv->stride_head * es) % 16) return FC_ERR_INVALID_ARG;
@@ -427,13 +428,22 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
     const int nseq = kv->batch - b0 < kSeqChunk ? kv->batch - b0 : kSeqChunk;
     SeqTable tab;
     for (int i = 0; i <= nseq; ++i) tab.start[i] = kv->cu_seqlens[b0 + i];
+    int nmax = 0;
+    for (int i = 0; i < nseq; ++i) nmax = tab.start[i + 1] - tab.start[i] > nmax ? tab.start[i + 1] - tab.start[i] : nmax;
+    const int per_thread = (nmax + kSelCluster * kSelThreads - 1) / (kSelCluster * kSelThreads);
     {
       ProfScope ps(h, FC_K_SELECT, st);
-      k_select_gather<<<dim3(kSelCluster * nseq, kv->num_heads), kSelThreads, 0, st>>>(
-          scores, T, tab, b0, budgets, reinterpret_cast<const long long *>(out_offsets), out_idx,
-          out_capacity_rows, h->status_word, static_cast<const char *>(kv->k),
-          static_cast<const char *>(kv->v), kv->stride_token * es, kv->stride_head * es,
-          kv->head_dim * es, kv->num_heads, static_cast<char *>(out_k), static_cast<char *>(out_v));
+#define FC_SEL_LAUNCH(KPT)                                                                              \
+  k_select_gather<KPT><<<dim3(kSelCluster * nseq, kv->num_heads), kSelThreads, 0, st>>>(                \
+      scores, T, tab, b0, budgets, reinterpret_cast<const long long *>(out_offsets), out_idx,           \
+      out_capacity_rows, h->status_word, static_cast<const char *>(kv->k),                              \
+      static_cast<const char *>(kv->v), kv->stride_token * es, kv->stride_head * es, kv->head_dim * es, \
+      kv->num_heads, static_cast<char *>(out_k), static_cast<char *>(out_v))
+      if (per_thread <= 2) FC_SEL_LAUNCH(2);
+      else if (per_thread <= 4) FC_SEL_LAUNCH(4);
+      else if (per_thread <= 8) FC_SEL_LAUNCH(8);
+      else FC_SEL_LAUNCH(16);
+#undef FC_SEL_LAUNCH
     }
     if ((s = fc_after_launch(h)) != FC_OK) return s;
   }
