@@ -170,6 +170,47 @@ fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const float *sco
                             int64_t out_capacity_rows,
                             void *workspace, size_t workspace_bytes, fc_stream stream);
 
+/*
+ * fc_score_layer without any allocation (the paper has no counterpart: this is a
+ * packaging variant of the same computation, added for integration reasons).
+ *
+ * Who needs it: code that is not allowed to obtain device memory at the point where it
+ * wants to score a layer -- for example a serving process whose whole device memory is
+ * handed to a framework's pool at start-up, a plug-in interface that forbids allocation
+ * after initialisation, or a real-time path where the implicit device synchronisation
+ * of cudaMalloc/cudaFree is not acceptable.  Such callers cannot use fc_create (it
+ * allocates the twiddle table) nor provide the workspace of fc_score_layer.
+ *
+ * This entry point needs no handle and no workspace.  Its twiddle table and all of its
+ * scratch live in arrays that are part of the library image: FC_STATIC_SCRATCH_BYTES
+ * (8 MiB) of scratch plus a 128 KiB table, held by every GPU that has loaded the library
+ * until the process exits.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ * Inputs and outputs are the caller's, exactly as for fc_score_layer:
+ *
+ *   kv, gamma, scores, energy, stream   as in fc_score_layer (same layout, same results
+ *                                       up to fp32 rounding: it runs the library's generic
+ *                                       transform kernels for every length).
+ *
+ * Limits: every sequence length <= 4096 (else FC_ERR_UNSUPPORTED), and the scratch the view
+ * needs (what fc_score_workspace_bytes would report with one head per transform group)
+ * <= FC_STATIC_SCRATCH_BYTES (else FC_ERR_WORKSPACE).  At head_dim 128 that admits
+ * power-of-two lengths up to 4096 and any other length up to 2048.
+ *
+ * First call on a device: looks up the device addresses of the arrays, fills the twiddle
+ * table and waits for the device once (cudaDeviceSynchronize).  Make that first call with
+ * the device current and before any stream capture begins.  Later calls only enqueue
+ * kernels on `stream`.
+ *
+ * Sharing: all calls on one device use the same scratch, which keeps the previous call's
+ * contents (every region is rewritten before it is read, nothing needs clearing).  Two
+ * calls that can overlap on the GPU (different streams, or different host threads without
+ * ordering between their streams) race on it; order them.
+ */
+#define FC_STATIC_SCRATCH_BYTES ((size_t)8 << 20)
+size_t fc_static_scratch_bytes(void);
+fc_status fc_score_layer_static(const fc_kv_view *kv, double gamma, float *scores,
+                                double *energy, fc_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

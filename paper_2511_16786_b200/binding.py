@@ -26,6 +26,7 @@ EXPORTS = (
     "fc_set_group_bytes", "fc_profile_begin", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact",
+    "fc_static_scratch_bytes", "fc_score_layer_static",
 )
 
 
@@ -81,6 +82,10 @@ def _load() -> ctypes.CDLL:
     lib.fc_select_compact.argtypes = [c_void_p, POINTER(fc_kv_view), c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_size_t, c_void_p]
     lib.fc_select_compact.restype = c_int
+    lib.fc_static_scratch_bytes.argtypes = []
+    lib.fc_static_scratch_bytes.restype = c_size_t
+    lib.fc_score_layer_static.argtypes = [POINTER(fc_kv_view), c_double, c_void_p, c_void_p, c_void_p]
+    lib.fc_score_layer_static.restype = c_int
     return lib
 
 
@@ -182,6 +187,20 @@ def fc_score_layer(handle, k, v, cu_seqlens, gamma: float, scores, energy, works
     _check(_lib.fc_score_layer(handle, byref(view), float(gamma), c_void_p(scores.data_ptr()),
                                c_void_p(energy.data_ptr()), c_void_p(workspace.data_ptr()),
                                workspace.numel() * workspace.element_size(), _stream()), "fc_score_layer")
+
+
+def fc_static_scratch_bytes() -> int:
+    return int(_lib.fc_static_scratch_bytes())
+
+
+def fc_score_layer_static(k, v, cu_seqlens, gamma: float, scores, energy) -> None:
+    """fc_score_layer for callers that may not allocate device memory: no handle, no
+    workspace; the scratch is a fixed array inside the library (see include/flashcache.h
+    for the size limits and the sharing rule).  scores: float32 [H, T]; energy: float64 [B, 4]."""
+    cu = _cu_array(cu_seqlens)
+    view = make_view(k, v, cu)
+    _check(_lib.fc_score_layer_static(byref(view), float(gamma), c_void_p(scores.data_ptr()),
+                                      c_void_p(energy.data_ptr()), _stream()), "fc_score_layer_static")
 
 
 def fc_allocate_budgets(handle, energy, cu_seqlens, rho: float, min_keep: int, budgets, out_offsets) -> None:

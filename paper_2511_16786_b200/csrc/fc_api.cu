@@ -47,6 +47,7 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->prof_events = nullptr;
   h->prof_cap = 0;
   h->prof_used = 0;
+  h->generic_only = false;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return FC_ERR_CUDA; }
   h->num_sms = prop.multiProcessorCount;

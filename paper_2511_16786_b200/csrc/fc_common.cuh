@@ -37,6 +37,9 @@ struct fc_handle {
   int prof_class;
   cudaEvent_t *prof_events;   // pairs
   int prof_cap, prof_used;
+  // true only for the stack handle of fc_score_layer_static: every length takes the generic
+  // single-stream kernels (no internal streams or events exist there)
+  bool generic_only;
 };
 
 // Kernel classes for fc_profile_begin.

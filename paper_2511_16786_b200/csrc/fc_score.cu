@@ -26,6 +26,7 @@
 #include "fc_score_fast.cuh"
 
 #include <math.h>
+#include <mutex>
 #include <type_traits>
 
 namespace {
@@ -459,7 +460,7 @@ struct SeqPlan {
   int cs, cs2;               // columns per tile in pass 1/3 and pass 2
 };
 
-SeqPlan plan_sequence(int N) {
+SeqPlan plan_sequence(int N, bool allow_fast = true) {
   SeqPlan s;
   s.N = N;
   s.bluestein = !(is_pow2(N) && N >= 16);
@@ -471,7 +472,7 @@ SeqPlan plan_sequence(int N) {
     s.Nfft = N;
   }
   const int bits = ilog2(s.Nfft);
-  s.fast = !s.bluestein && N >= 1024 && N <= 65536;
+  s.fast = allow_fast && !s.bluestein && N >= 1024 && N <= 65536;
   int b1 = bits / 2;
   if (b1 > 7 && !s.fast) b1 = 7;
   s.N1 = 1 << b1;
@@ -655,7 +656,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     return fc_after_launch(h);
   }
   const int d = kv->head_dim, H = kv->num_heads;
-  const SeqPlan sp = plan_sequence(N);
+  const SeqPlan sp = plan_sequence(N, !h->generic_only);
   const ScoreLayout L = layout_for(h, sp, H, d);
   long long om = (long long)floor(gamma * (double)N);
   if (om > N - 1) om = N - 1;
@@ -770,7 +771,7 @@ extern "C" size_t fc_score_workspace_bytes(const fc_handle *h, const fc_kv_view 
   for (int b = 0; b < kv->batch; ++b) {
     const int N = kv->cu_seqlens[b + 1] - kv->cu_seqlens[b];
     if (N == 0) continue;
-    const ScoreLayout L = layout_for(h, plan_sequence(N), kv->num_heads, kv->head_dim);
+    const ScoreLayout L = layout_for(h, plan_sequence(N, !h->generic_only), kv->num_heads, kv->head_dim);
     if (L.total > need) need = L.total;
   }
   return need;
@@ -794,6 +795,116 @@ extern "C" fc_status fc_score_layer(fc_handle *h, const fc_kv_view *kv, double g
       case FC_F32: s = score_sequence<float>(h, st, kv, b, gamma, scores, energy, (char *)workspace); break;
       case FC_F16: s = score_sequence<__half>(h, st, kv, b, gamma, scores, energy, (char *)workspace); break;
       default: s = score_sequence<__nv_bfloat16>(h, st, kv, b, gamma, scores, energy, (char *)workspace); break;
+    }
+  }
+  return s;
+}
+
+// ---------------------------------------------------------------------------
+// fc_score_layer_static: the same scoring with every byte of scratch in arrays that are
+// part of the loaded library image, for callers that must not allocate device memory.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxSeqlen = 4096;                       // longest sequence accepted
+constexpr int kStaticMasterLen = 4 * kStaticMaxSeqlen;       // same sizing rule as fc_create's table
+constexpr size_t kStaticScratchBytes = FC_STATIC_SCRATCH_BYTES;
+
+// Scratch shared by every call of fc_score_layer_static on a device; it keeps whatever the
+// last call left there.  The kernels below write each region before they read it, so
+// nothing has to be cleared between calls.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+static __device__ __align__(256) float2 g_static_master[kStaticMasterLen];
+static __device__ int g_static_status;
+static __device__ unsigned g_static_counter;
+
+// exp(-2*pi*j*i/len) in fp64, rounded once to fp32 (same definition as the handle's table).
+__global__ void k_fill_static_master(float2 *master, int len) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= len) return;
+  double s, c;
+  sincospi(-2.0 * (double)i / (double)len, &s, &c);
+  master[i] = make_float2((float)c, (float)s);
+}
+
+// Device addresses of the arrays above, looked up once per device.  In host code the
+// array names stand for the symbols, not for device memory: they must never be passed
+// to a kernel; cudaGetSymbolAddress gives the pointer a kernel can use.
+struct StaticSetup {
+  bool ready;
+  unsigned char *scratch;
+  float2 *master;
+  int *status;
+  unsigned *counter;
+};
+constexpr int kMaxDevices = 64;
+StaticSetup g_setup[kMaxDevices];
+std::mutex g_setup_mutex;
+
+fc_status static_setup(int dev, StaticSetup *out) {
+  if (dev < 0 || dev >= kMaxDevices) return FC_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
+  StaticSetup &s = g_setup[dev];
+  if (!s.ready) {
+    void *p_scratch = nullptr, *p_master = nullptr, *p_status = nullptr, *p_counter = nullptr;
+    FC_CUDA_TRY(cudaGetSymbolAddress(&p_scratch, g_static_scratch));
+    FC_CUDA_TRY(cudaGetSymbolAddress(&p_master, g_static_master));
+    FC_CUDA_TRY(cudaGetSymbolAddress(&p_status, g_static_status));
+    FC_CUDA_TRY(cudaGetSymbolAddress(&p_counter, g_static_counter));
+    k_fill_static_master<<<(kStaticMasterLen + 255) / 256, 256>>>(static_cast<float2 *>(p_master), kStaticMasterLen);
+    FC_CUDA_TRY(cudaGetLastError());
+    FC_CUDA_TRY(cudaDeviceSynchronize());
+    s.scratch = static_cast<unsigned char *>(p_scratch);
+    s.master = static_cast<float2 *>(p_master);
+    s.status = static_cast<int *>(p_status);
+    s.counter = static_cast<unsigned *>(p_counter);
+    s.ready = true;
+  }
+  *out = s;
+  return FC_OK;
+}
+
+}  // namespace
+
+extern "C" size_t fc_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+extern "C" fc_status fc_score_layer_static(const fc_kv_view *kv, double gamma, float *scores,
+                                           double *energy, fc_stream stream) {
+  if (!kv || !scores || !energy) return FC_ERR_INVALID_ARG;
+  if (!(gamma >= 0.0 && gamma <= 1.0)) return FC_ERR_INVALID_ARG;
+  int dev = -1;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  StaticSetup su;
+  fc_status s = static_setup(dev, &su);
+  if (s != FC_OK) return s;
+  // A handle that lives on this stack frame and owns nothing: its table, status word and
+  // counter are the static arrays, and it is restricted to the single-stream kernels.
+  fc_handle hs = {};
+  hs.device = dev;
+  hs.max_seqlen = kStaticMaxSeqlen;
+  hs.master_len = kStaticMasterLen;
+  hs.master = su.master;
+  hs.status_word = su.status;
+  hs.done_counter = su.counter;
+  hs.group_bytes = 1;                 // one head per transform group: the smallest workspace
+  hs.tune_cpw = 32;
+  hs.tune_cp = 8;
+  hs.prof_class = FC_K_NONE;
+  hs.generic_only = true;
+  cudaDeviceProp prop;
+  FC_CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+  hs.num_sms = prop.multiProcessorCount;
+  s = validate_view(&hs, kv);         // lengths above kStaticMaxSeqlen come back as FC_ERR_UNSUPPORTED
+  if (s != FC_OK) return s;
+  const size_t need = fc_score_workspace_bytes(&hs, kv);
+  if (need == 0) return FC_ERR_INVALID_ARG;
+  if (need > kStaticScratchBytes) return FC_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  for (int b = 0; b < kv->batch && s == FC_OK; ++b) {
+    switch (kv->dtype) {
+      case FC_F32: s = score_sequence<float>(&hs, st, kv, b, gamma, scores, energy, (char *)su.scratch); break;
+      case FC_F16: s = score_sequence<__half>(&hs, st, kv, b, gamma, scores, energy, (char *)su.scratch); break;
+      default: s = score_sequence<__nv_bfloat16>(&hs, st, kv, b, gamma, scores, energy, (char *)su.scratch); break;
     }
   }
   return s;
