@@ -148,7 +148,7 @@ def fc_set_group_bytes(handle, nbytes: int) -> None:
     _check(_lib.fc_set_group_bytes(handle, int(nbytes)), "fc_set_group_bytes")
 
 
-KERNEL_CLASSES = {"pass1": 1, "pass2": 2, "pass3": 3, "select": 4, "gather": 5, "other": 6}
+KERNEL_CLASSES = {"pass1": 1, "pass2": 2, "pass3": 3, "select": 4, "gather": 5, "other": 6, "fused": 7}
 
 
 def fc_profile_begin(handle, kernel_class: int, max_launches: int = 16384) -> None:

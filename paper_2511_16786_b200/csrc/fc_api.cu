@@ -1,5 +1,6 @@
 // Handle life cycle, status reporting and the twiddle table of the FlashCache library.
 #include "fc_common.cuh"
+#include "fc_score_fused.cuh"
 
 #include <new>
 #include <stdlib.h>
@@ -48,6 +49,11 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->prof_cap = 0;
   h->prof_used = 0;
   h->generic_only = false;
+  h->fused_sched = nullptr;
+  h->fused_enabled = 0;   // the separate-launch kernels are still faster; FC_FUSED=1 switches the fused kernel on
+  h->fused_blocks_per_sm = 0;
+  if (const char *e = getenv("FC_FUSED")) { h->fused_enabled = atoi(e) != 0 ? 1 : 0; }
+  if (const char *e = getenv("FC_FUSED_BPS")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_blocks_per_sm = v; }
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return FC_ERR_CUDA; }
   h->num_sms = prop.multiProcessorCount;
@@ -56,6 +62,8 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
       cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess ||
       cudaMalloc(&h->done_counter, sizeof(unsigned)) != cudaSuccess ||
       cudaMemset(h->done_counter, 0, sizeof(unsigned)) != cudaSuccess ||
+      cudaMalloc(&h->fused_sched, sizeof(fused::Sched)) != cudaSuccess ||
+      cudaMemset(h->fused_sched, 0, sizeof(fused::Sched)) != cudaSuccess ||
       cudaStreamCreateWithFlags(&h->aux[0], cudaStreamNonBlocking) != cudaSuccess ||
       cudaStreamCreateWithFlags(&h->aux[1], cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
@@ -84,7 +92,7 @@ static void free_prof(fc_handle *h) {
 }
 
 extern "C" fc_status fc_profile_begin(fc_handle *h, int32_t kernel_class, int32_t max_launches) {
-  if (!h || kernel_class < FC_K_PASS1 || kernel_class > FC_K_OTHER || max_launches < 1) return FC_ERR_INVALID_ARG;
+  if (!h || kernel_class < FC_K_PASS1 || kernel_class > FC_K_FUSED || max_launches < 1) return FC_ERR_INVALID_ARG;
   free_prof(h);
   h->prof_events = new (std::nothrow) cudaEvent_t[2 * (size_t)max_launches];
   if (!h->prof_events) return FC_ERR_INTERNAL;
@@ -130,6 +138,7 @@ extern "C" void fc_destroy(fc_handle *h) {
   if (h->master) cudaFree(h->master);
   if (h->status_word) cudaFree(h->status_word);
   if (h->done_counter) cudaFree(h->done_counter);
+  if (h->fused_sched) cudaFree(h->fused_sched);
   delete h;
 }
 

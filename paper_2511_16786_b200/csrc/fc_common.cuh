@@ -40,10 +40,14 @@ struct fc_handle {
   // true only for the stack handle of fc_score_layer_static: every length takes the generic
   // single-stream kernels (no internal streams or events exist there)
   bool generic_only;
+  // scheduler state of the fused persistent kernel (DEVICE, all zero between launches) and knobs
+  void *fused_sched;
+  int fused_enabled;       // 1 enables the fused kernel (developer knob FC_FUSED)
+  int fused_blocks_per_sm; // 0 = as many as fit
 };
 
 // Kernel classes for fc_profile_begin.
-enum { FC_K_NONE = 0, FC_K_PASS1 = 1, FC_K_PASS2 = 2, FC_K_PASS3 = 3, FC_K_SELECT = 4, FC_K_GATHER = 5, FC_K_OTHER = 6 };
+enum { FC_K_NONE = 0, FC_K_PASS1 = 1, FC_K_PASS2 = 2, FC_K_PASS3 = 3, FC_K_SELECT = 4, FC_K_GATHER = 5, FC_K_OTHER = 6, FC_K_FUSED = 7 };
 
 // Brackets one launch with an event pair when its class is being profiled.
 struct ProfScope {

@@ -24,6 +24,7 @@
 // chirp convolution on a power-of-two length M >= 2N-1 with the same three passes.
 #include "fc_common.cuh"
 #include "fc_score_fast.cuh"
+#include "fc_score_fused.cuh"
 
 #include <math.h>
 #include <mutex>
@@ -485,6 +486,44 @@ SeqPlan plan_sequence(int N, bool allow_fast = true) {
   return s;
 }
 
+// Plan of the fused persistent kernel for one power-of-two sequence (see fc_score_fused.cuh).
+struct FusedPlan {
+  bool ok;
+  int r1b, r2b;                 // N1 = 16*r1b, N2 = 16*r2b
+  int UC, upd, U, R;
+  int n1t, n2t, n3t, ncb1, ncb2;
+  size_t ring_bytes, part_tot_bytes, part_hi_bytes;
+};
+
+FusedPlan plan_fused(const fc_handle *h, const SeqPlan &sp, int H, int d) {
+  FusedPlan f = {};
+  if (!sp.fast || !h->fused_enabled || sp.N < 4096 || sp.N > 65536) return f;
+  f.r1b = sp.N1 / 16;
+  f.r2b = sp.N2 / 16;
+  const int cpw = fused::NT / f.r1b, cp = fused::NT / (2 * f.r2b);
+  const int min_uc = 2 * cpw > 2 * cp ? 2 * cpw : 2 * cp;
+  int uc = (1 << 20) / sp.N;                       // about 8 MB of intermediate per unit
+  if (uc < min_uc) uc = min_uc;
+  while (uc > min_uc && (uc > d || d % uc != 0)) uc >>= 1;
+  if (uc > d || d % uc != 0 || uc % (2 * cpw) != 0 || uc % (2 * cp) != 0) return f;
+  f.UC = uc;
+  f.upd = d / uc;
+  f.U = H * f.upd;
+  if (f.U > 1024 || H > 1024) return f;
+  f.R = f.upd + 3;                                  // a slot is rewritten at least two stages after its last reader was handed out
+  if (f.R > f.U) f.R = f.U;
+  f.ncb1 = uc / (2 * cpw);
+  f.ncb2 = uc / (2 * cp);
+  f.n1t = sp.N2 * f.ncb1;
+  f.n2t = (sp.N1 / 2) * f.ncb2;
+  f.n3t = sp.N2;
+  f.ring_bytes = align_up((size_t)f.R * sp.N * uc * sizeof(float2), 256);
+  f.part_tot_bytes = align_up((size_t)f.U * f.n1t * 2 * sizeof(double), 256);
+  f.part_hi_bytes = align_up((size_t)H * f.n3t * 2 * sizeof(double), 256);
+  f.ok = true;
+  return f;
+}
+
 struct ScoreLayout {
   size_t off_ws, off_spec, off_hhat, off_hcol, off_part_tot, off_part_hi, total;
   size_t ws_buf_bytes;       // one group buffer; the fast path keeps two and alternates
@@ -495,6 +534,19 @@ struct ScoreLayout {
 // query takes the maximum over the sequences of the view).
 ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int head_dim) {
   ScoreLayout L;
+  {
+    const FusedPlan f = plan_fused(h, sp, num_heads, head_dim);
+    if (f.ok) {                                      // ring | pass-1 partial sums | pass-3 partial sums
+      L = ScoreLayout{};
+      L.off_ws = 0;
+      L.off_part_tot = f.ring_bytes;
+      L.off_part_hi = f.ring_bytes + f.part_tot_bytes;
+      L.total = f.ring_bytes + f.part_tot_bytes + f.part_hi_bytes;
+      L.ws_buf_bytes = f.ring_bytes;
+      L.heads_per_group = num_heads;
+      return L;
+    }
+  }
   const size_t per_head = (size_t)sp.Nfft * head_dim * sizeof(float2);
   int hg = (int)(h->group_bytes / per_head);
   if (hg < 1) hg = 1;
@@ -644,6 +696,37 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
   return FC_ERR_INTERNAL;
 }
 
+template <typename T, int R1B, int R2B>
+fc_status launch_fused_impl(fc_handle *h, cudaStream_t st, const fused::Params &P) {
+  auto kern = fused::k_fused<T, R1B, R2B>;
+  const size_t sm = fused::Smem<R1B, R2B>::bytes;
+  fc_status s = set_smem(kern, sm);
+  if (s != FC_OK) return s;
+  static int blocks_per_sm = 0;                     // per instantiation; the answer does not change
+  if (blocks_per_sm == 0) {
+    int n = 0;
+    FC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, fused::NT, sm));
+    if (n < 1) return FC_ERR_INTERNAL;
+    blocks_per_sm = n;
+  }
+  int bps = blocks_per_sm;
+  if (h->fused_blocks_per_sm > 0 && h->fused_blocks_per_sm < bps) bps = h->fused_blocks_per_sm;
+  unsigned grid = (unsigned)(h->num_sms * bps);
+  if (grid > P.total_tiles) grid = P.total_tiles;
+  ProfScope ps(h, FC_K_FUSED, st);
+  kern<<<grid, fused::NT, sm, st>>>(P);
+  return fc_after_launch(h);
+}
+
+template <typename T>
+fc_status launch_fused(fc_handle *h, cudaStream_t st, const FusedPlan &f, const fused::Params &P) {
+#define FC_FUSED_CASE(A, B) \
+  if (f.r1b == A && f.r2b == B) return launch_fused_impl<T, A, B>(h, st, P);
+  FC_FUSED_CASE(4, 4) FC_FUSED_CASE(4, 8) FC_FUSED_CASE(8, 8) FC_FUSED_CASE(8, 16) FC_FUSED_CASE(16, 16)
+#undef FC_FUSED_CASE
+  return FC_ERR_INTERNAL;
+}
+
 template <typename T>
 fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, int b, double gamma,
                          float *scores, double *energy, char *wsb) {
@@ -673,6 +756,31 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   const T *vp = static_cast<const T *>(kv->v) + (long long)start * kv->stride_token;
   const FftPlan p1 = make_plan(sp.N1);
   fc_status s;
+
+  {
+    const FusedPlan f = plan_fused(h, sp, H, d);
+    if (f.ok) {
+      const int es = (int)sizeof(T);
+      fused::Params P = {};
+      P.k = kp; P.v = vp;
+      P.stride_token_b = (long long)kv->stride_token * es;
+      P.stride_head_b = (long long)kv->stride_head * es;
+      P.N = N; P.omega = omega; P.head_dim = d; P.num_heads = H;
+      P.UC = f.UC; P.upd = f.upd; P.U = f.U; P.R = f.R;
+      P.n1t = f.n1t; P.n2t = f.n2t; P.n3t = f.n3t; P.ncb1 = f.ncb1; P.ncb2 = f.ncb2;
+      P.total_tiles = (unsigned)((long long)f.U * (f.n1t + f.n2t) + (long long)H * f.n3t);
+      P.ws = ws;
+      P.master = h->master; P.master_len = h->master_len;
+      P.scores = scores + start; P.score_stride = total_tokens;
+      P.inv_scale = (float)(1.0 / ((double)N * (double)N * (double)d));
+      P.part_tot = part_tot; P.part_hi = part_hi;
+      P.energy = energy_b;
+      P.sched = static_cast<fused::Sched *>(h->fused_sched);
+      P.status = h->status_word;
+      P.spin_limit = 1u << 22;
+      return launch_fused<T>(h, st, f, P);
+    }
+  }
 
   if (sp.bluestein) {
     // spectrum of the chirp kernel, once per sequence

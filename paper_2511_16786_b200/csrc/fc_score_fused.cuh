@@ -1,0 +1,783 @@
+// Fused, persistent form of the three transform passes for power-of-two sequence
+// lengths N = N1*N2 from 4096 to 65536 (N1 = 16*R1B, N2 = 16*R2B).  Same mathematics
+// as fc_score.cu (see the header comment there); what differs:
+//
+//  * ONE launch scores a whole (layer, sequence).  The columns of the layer are cut into
+//    units of UC complex columns (about 8 MB of intermediate each); the tiles of
+//    pass 1 of unit s, pass 2 of unit s-1 and pass 3 of the head completed at s-2 form
+//    stage s.  Persistent blocks take tiles in stage order from an atomic counter and
+//    wait (bounded) on per-unit completion counters, so a tile only ever waits for
+//    tiles that were handed out before it.  The intermediates live in a ring of unit
+//    slots that stays in L2.
+//  * every tile is 2048 float4 (32 KB), processed by 128 threads; the next tile is
+//    fetched into the second shared-memory buffer with cp.async while the current one
+//    is transformed in place.
+//  * a thread owns two adjacent channels as ONE packed value per component:
+//    float4 = (re_a, re_b, im_a, im_b), and all butterflies run on the packed
+//    fp32x2 add/mul/fma instructions of sm_100, halving the issue slots of the
+//    arithmetic.
+//
+// The transform is unnormalised (factor N); pass 3 folds 1/N^2 into the score.
+#pragma once
+#include "fc_common.cuh"
+
+namespace fused {
+
+constexpr int NT = 128;        // threads per block
+constexpr int TILE4 = 2048;    // float4 per tile buffer
+
+// Scheduler state in global memory (owned by the handle, all zero between launches).
+struct Sched {
+  unsigned tile_counter;
+  unsigned exit_counter;
+  unsigned abort_flag;
+  unsigned pad;
+  unsigned done1[1024];   // pass-1 tiles finished per unit
+  unsigned done2[1024];   // pass-2 tiles finished per unit
+  unsigned done3[1024];   // pass-3 tiles finished per head
+};
+
+struct Params {
+  const void *k, *v;               // first token of the sequence
+  long long stride_token_b, stride_head_b;   // bytes
+  int N, omega, head_dim, num_heads;
+  int UC, upd, U, R;               // unit columns, units per head, units, ring slots
+  int n1t, n2t, n3t, ncb1, ncb2;   // tiles per unit (pass 1, 2), per head (pass 3); column blocks per unit
+  unsigned total_tiles;
+  float2 *ws;                      // ring of R unit slots, each [N1*N2][UC] float2 (stored as planar pairs)
+  const float2 *master;
+  int master_len;
+  float *scores;                   // already offset to the sequence's first token
+  long long score_stride;          // tokens in the packed batch
+  float inv_scale;                 // 1 / (N^2 d)
+  double *part_tot, *part_hi;      // per-tile energy partial sums
+  double *energy;                  // [4]
+  Sched *sched;
+  int *status;
+  unsigned spin_limit;
+};
+
+// ------------------------------------------------------------------ packed arithmetic
+// Two complex numbers a and b (adjacent channels): r = (re_a, re_b), i = (im_a, im_b).
+struct c2 { float2 r, i; };
+
+__device__ __forceinline__ float2 padd(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ float2 psub(float2 a, float2 b) { return __ffma2_rn(b, make_float2(-1.f, -1.f), a); }
+__device__ __forceinline__ float2 pmul(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 pfma(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 bc(float s) { return make_float2(s, s); }
+
+__device__ __forceinline__ c2 cadd2(const c2 &a, const c2 &b) { return {padd(a.r, b.r), padd(a.i, b.i)}; }
+__device__ __forceinline__ c2 csub2(const c2 &a, const c2 &b) { return {psub(a.r, b.r), psub(a.i, b.i)}; }
+__device__ __forceinline__ c2 from4(float4 t) { return {make_float2(t.x, t.y), make_float2(t.z, t.w)}; }
+__device__ __forceinline__ float4 to4(const c2 &a) { return make_float4(a.r.x, a.r.y, a.i.x, a.i.y); }
+
+// a * w and a * conj(w) for one twiddle w given as a broadcast float4 (wr, wr, wi, wi).
+__device__ __forceinline__ c2 cmul_b(const c2 &a, float4 w) {
+  const float2 wr = make_float2(w.x, w.y), wi = make_float2(w.z, w.w);
+  const float2 nwi = pmul(wi, make_float2(-1.f, -1.f));
+  return {pfma(a.i, nwi, pmul(a.r, wr)), pfma(a.i, wr, pmul(a.r, wi))};
+}
+__device__ __forceinline__ c2 cmulc_b(const c2 &a, float4 w) {
+  const float2 wr = make_float2(w.x, w.y), wi = make_float2(w.z, w.w);
+  const float2 nwi = pmul(wi, make_float2(-1.f, -1.f));
+  return {pfma(a.i, wi, pmul(a.r, wr)), pfma(a.r, nwi, pmul(a.i, wr))};
+}
+// product of two broadcast twiddles, still broadcast
+__device__ __forceinline__ float4 wmul_b(float4 a, float4 b) {
+  const float2 ar = make_float2(a.x, a.y), ai = make_float2(a.z, a.w);
+  const float2 br = make_float2(b.x, b.y), bi = make_float2(b.z, b.w);
+  const float2 nbi = pmul(bi, make_float2(-1.f, -1.f));
+  const float2 r = pfma(ai, nbi, pmul(ar, br)), i = pfma(ai, br, pmul(ar, bi));
+  return make_float4(r.x, r.y, i.x, i.y);
+}
+__device__ __forceinline__ float4 bcast4(float2 w) { return make_float4(w.x, w.x, w.y, w.y); }
+
+// ------------------------------------------------------------------ small DFTs on c2
+// y[k] = sum_n x[n] exp(DIR*2*pi*j*n*k/R), natural order in and out.
+template <int DIR>
+__device__ __forceinline__ void dft2p(c2 &a, c2 &b) {
+  const c2 t = a;
+  a = cadd2(t, b);
+  b = csub2(t, b);
+}
+
+// multiply-by-(DIR*j) is folded into the adds: DIR=-1: -j*(tr,ti) = (ti,-tr); DIR=+1: (-ti, tr)
+template <int DIR>
+__device__ __forceinline__ void dft4p(c2 &a0, c2 &a1, c2 &a2, c2 &a3) {
+  const c2 s0 = cadd2(a0, a2), d0 = csub2(a0, a2);
+  const c2 s1 = cadd2(a1, a3), t = csub2(a1, a3);
+  a0 = cadd2(s0, s1);
+  a2 = csub2(s0, s1);
+  if (DIR < 0) {
+    a1 = {padd(d0.r, t.i), psub(d0.i, t.r)};
+    a3 = {psub(d0.r, t.i), padd(d0.i, t.r)};
+  } else {
+    a1 = {psub(d0.r, t.i), padd(d0.i, t.r)};
+    a3 = {padd(d0.r, t.i), psub(d0.i, t.r)};
+  }
+}
+
+template <int DIR>
+__device__ __forceinline__ void dft8p(c2 (&x)[8]) {
+  const float2 h = bc(0.70710678118654752440f), nh = bc(-0.70710678118654752440f);
+  dft4p<DIR>(x[0], x[2], x[4], x[6]);   // even samples -> E0..E3 at x[0],x[2],x[4],x[6]
+  dft4p<DIR>(x[1], x[3], x[5], x[7]);   // odd samples  -> O0..O3 at x[1],x[3],x[5],x[7]
+  const c2 e0 = x[0], e1 = x[2], e2 = x[4], e3 = x[6];
+  const c2 o0 = x[1], o1 = x[3], o2 = x[5], o3 = x[7];
+  x[0] = cadd2(e0, o0);
+  x[4] = csub2(e0, o0);
+  // k = 2: t = DIR*j*o2
+  if (DIR < 0) {
+    x[2] = {padd(e2.r, o2.i), psub(e2.i, o2.r)};
+    x[6] = {psub(e2.r, o2.i), padd(e2.i, o2.r)};
+  } else {
+    x[2] = {psub(e2.r, o2.i), padd(e2.i, o2.r)};
+    x[6] = {padd(e2.r, o2.i), psub(e2.i, o2.r)};
+  }
+  // k = 1: w = (1 + DIR*j)/sqrt2 ; k = 3: w = (-1 + DIR*j)/sqrt2.  With s = or+oi, d = oi-or:
+  //   DIR=-1: o*w8^1 = h*(s, d)       o*w8^3 = h*(d, -s)
+  //   DIR=+1: o*w8^1 = h*(-d, s)      o*w8^3 = h*(-s, -d)
+  {
+    const float2 s = padd(o1.r, o1.i), d = psub(o1.i, o1.r);
+    if (DIR < 0) {
+      x[1] = {pfma(s, h, e1.r), pfma(d, h, e1.i)};
+      x[5] = {pfma(s, nh, e1.r), pfma(d, nh, e1.i)};
+    } else {
+      x[1] = {pfma(d, nh, e1.r), pfma(s, h, e1.i)};
+      x[5] = {pfma(d, h, e1.r), pfma(s, nh, e1.i)};
+    }
+  }
+  {
+    const float2 s = padd(o3.r, o3.i), d = psub(o3.i, o3.r);
+    if (DIR < 0) {
+      x[3] = {pfma(d, h, e3.r), pfma(s, nh, e3.i)};
+      x[7] = {pfma(d, nh, e3.r), pfma(s, h, e3.i)};
+    } else {
+      x[3] = {pfma(s, nh, e3.r), pfma(d, nh, e3.i)};
+      x[7] = {pfma(s, h, e3.r), pfma(d, h, e3.i)};
+    }
+  }
+}
+
+// t = o * (c + DIR*j*s), then (e + t, e - t)
+template <int DIR>
+__device__ __forceinline__ void bfly_w(const c2 &e, const c2 &o, float c, float s, c2 &lo, c2 &hi) {
+  const float sg = DIR < 0 ? -1.f : 1.f;
+  const float2 wr = bc(c), wi = bc(sg * s), nwi = bc(-sg * s);
+  const c2 t = {pfma(o.i, nwi, pmul(o.r, wr)), pfma(o.i, wr, pmul(o.r, wi))};
+  lo = cadd2(e, t);
+  hi = csub2(e, t);
+}
+
+template <int DIR>
+__device__ __forceinline__ void dft16p(c2 (&x)[16]) {
+  const float c1 = 0.92387953251128675613f, s1 = 0.38268343236508977173f;
+  const float h = 0.70710678118654752440f;
+  c2 e[8], o[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { e[i] = x[2 * i]; o[i] = x[2 * i + 1]; }
+  dft8p<DIR>(e);
+  dft8p<DIR>(o);
+  x[0] = cadd2(e[0], o[0]);
+  x[8] = csub2(e[0], o[0]);
+  bfly_w<DIR>(e[1], o[1], c1, s1, x[1], x[9]);
+  bfly_w<DIR>(e[2], o[2], h, h, x[2], x[10]);
+  bfly_w<DIR>(e[3], o[3], s1, c1, x[3], x[11]);
+  if (DIR < 0) {
+    x[4] = {padd(e[4].r, o[4].i), psub(e[4].i, o[4].r)};
+    x[12] = {psub(e[4].r, o[4].i), padd(e[4].i, o[4].r)};
+  } else {
+    x[4] = {psub(e[4].r, o[4].i), padd(e[4].i, o[4].r)};
+    x[12] = {padd(e[4].r, o[4].i), psub(e[4].i, o[4].r)};
+  }
+  bfly_w<DIR>(e[5], o[5], -s1, c1, x[5], x[13]);
+  bfly_w<DIR>(e[6], o[6], -h, h, x[6], x[14]);
+  bfly_w<DIR>(e[7], o[7], -c1, s1, x[7], x[15]);
+}
+
+template <int R, int DIR>
+__device__ __forceinline__ void dftp(c2 (&x)[R]) {
+  if constexpr (R == 2) dft2p<DIR>(x[0], x[1]);
+  else if constexpr (R == 4) dft4p<DIR>(x[0], x[1], x[2], x[3]);
+  else if constexpr (R == 8) dft8p<DIR>(x);
+  else dft16p<DIR>(x);
+}
+
+// ------------------------------------------------------------------ memory helpers
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+__device__ __forceinline__ int perm_token(int p, int N) {
+  const int half = N >> 1;                       // N is even here
+  return p < half ? 2 * p : 2 * (N - 1 - p) + 1;
+}
+
+// input element pair -> packed float2 (two adjacent channels)
+template <typename T> struct Pair;
+template <> struct Pair<float> {
+  static constexpr int ES = 4;
+  __device__ static float2 ld(const char *s) { return *reinterpret_cast<const float2 *>(s); }
+};
+template <> struct Pair<__half> {
+  static constexpr int ES = 2;
+  __device__ static float2 ld(const char *s) { return __half22float2(*reinterpret_cast<const __half2 *>(s)); }
+};
+template <> struct Pair<__nv_bfloat16> {
+  static constexpr int ES = 2;
+  __device__ static float2 ld(const char *s) {
+    const unsigned u = *reinterpret_cast<const unsigned *>(s);
+    return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+  }
+};
+
+// ------------------------------------------------------------------ tile descriptors
+enum { PH_NONE = 0, PH_P1 = 1, PH_P2 = 2, PH_P3 = 3 };
+struct Tile {
+  int phase;   // PH_*
+  int unit;    // unit (pass 1, 2) or head (pass 3)
+  int a;       // n2 (pass 1, 3) or k1 pair index x (pass 2)
+  int cb;      // column block inside the unit (pass 1, 2)
+  int ready;   // dependencies were already satisfied when the tile was fetched
+};
+
+// Stage walk kept by thread 0: tiles are fetched in increasing order, so it only moves forward.
+struct Walk { int stage; unsigned start; };
+
+__device__ __forceinline__ void stage_counts(const Params &P, int s, int &c1, int &c2, int &c3) {
+  c1 = (s < P.U) ? P.n1t : 0;
+  c2 = (s >= 1 && s <= P.U) ? P.n2t : 0;
+  c3 = (s >= 2 && s - 2 < P.U && (s - 2) % P.upd == P.upd - 1) ? P.n3t : 0;
+}
+
+__device__ __forceinline__ Tile decode_tile(const Params &P, Walk &w, unsigned t) {
+  Tile tl;
+  tl.ready = 0;
+  if (t >= P.total_tiles) { tl.phase = PH_NONE; tl.unit = tl.a = tl.cb = 0; return tl; }
+  int c1, c2, c3;
+  stage_counts(P, w.stage, c1, c2, c3);
+  while (t >= w.start + (unsigned)(c1 + c2 + c3)) {
+    w.start += (unsigned)(c1 + c2 + c3);
+    ++w.stage;
+    stage_counts(P, w.stage, c1, c2, c3);
+  }
+  int i = (int)(t - w.start);
+  if (i < c3) {
+    tl.phase = PH_P3; tl.unit = (w.stage - 2) / P.upd; tl.a = i; tl.cb = 0;
+    return tl;
+  }
+  i -= c3;
+  const int m = c1 < c2 ? c1 : c2;
+  int idx, ph;
+  if (i < 2 * m) { ph = (i & 1) ? PH_P1 : PH_P2; idx = i >> 1; }
+  else { idx = m + (i - 2 * m); ph = (c1 > c2) ? PH_P1 : PH_P2; }
+  tl.phase = ph;
+  if (ph == PH_P1) { tl.unit = w.stage; tl.a = idx / P.ncb1; tl.cb = idx - tl.a * P.ncb1; }
+  else { tl.unit = w.stage - 1; tl.a = idx / P.ncb2; tl.cb = idx - tl.a * P.ncb2; }
+  return tl;
+}
+
+// Are the tiles this one depends on finished?  (thread 0 only)
+__device__ __forceinline__ bool deps_ok(const Params &P, const Tile &tl) {
+  const Sched *sc = P.sched;
+  if (tl.phase == PH_P1) {
+    if (tl.unit < P.R) return true;
+    return ld_acquire(&sc->done3[(tl.unit - P.R) / P.upd]) >= (unsigned)P.n3t;   // the ring slot was read out
+  }
+  if (tl.phase == PH_P2) return ld_acquire(&sc->done1[tl.unit]) >= (unsigned)P.n1t;
+  if (tl.phase == PH_P3) {
+    for (int u = tl.unit * P.upd; u < (tl.unit + 1) * P.upd; ++u)
+      if (ld_acquire(&sc->done2[u]) < (unsigned)P.n2t) return false;
+    return true;
+  }
+  return true;
+}
+
+// Bounded wait (thread 0 only).  false: gave up or another block gave up.
+__device__ __forceinline__ bool wait_deps(const Params &P, const Tile &tl) {
+  for (unsigned it = 0; it < P.spin_limit; ++it) {
+    if (deps_ok(P, tl)) return true;
+    if (ld_acquire(&P.sched->abort_flag) != 0u) return false;
+    __nanosleep(200);
+  }
+  atomicExch(&P.sched->abort_flag, 1u);
+  atomicOr(P.status, FC_DEV_FLAG_TIMEOUT);
+  return false;
+}
+
+__device__ __forceinline__ void signal_done(const Params &P, const Tile &tl) {   // thread 0, after a block barrier
+  __threadfence();
+  Sched *sc = P.sched;
+  unsigned *c = tl.phase == PH_P1 ? &sc->done1[tl.unit] : (tl.phase == PH_P2 ? &sc->done2[tl.unit] : &sc->done3[tl.unit]);
+  atomicAdd(c, 1u);
+}
+
+__device__ __forceinline__ float2 *slot_base(const Params &P, int unit) {
+  return P.ws + (size_t)(unit % P.R) * (size_t)P.N * (size_t)P.UC;
+}
+
+// ------------------------------------------------------------------ pass 1
+// Tile (unit, n2, cb): DFT over n1 of 2*CPW channels.  Thread (cp = tid % CPW, j = tid / CPW).
+template <typename T, int R1B>
+struct Pass1 {
+  static constexpr int N1 = 16 * R1B, CPW = NT / R1B, IT = 16 / R1B, ES = Pair<T>::ES;
+  static constexpr int ROWB = 2 * CPW * ES, CPR = ROWB / 16;   // bytes and 16-byte chunks per input row slice
+
+  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, int tid) {
+    const int N2 = P.N / N1;
+    const int gcol = tl.unit * P.UC + tl.cb * 2 * CPW;
+    const int head = gcol / P.head_dim, c = gcol - head * P.head_dim;
+    const long long hoff = (long long)head * P.stride_head_b + (long long)c * ES;
+    const char *kb = static_cast<const char *>(P.k) + hoff;
+    const char *vb = static_cast<const char *>(P.v) + hoff;
+    char *dst0 = reinterpret_cast<char *>(buf);
+#pragma unroll
+    for (int idx = tid; idx < 2 * N1 * CPR; idx += NT) {
+      const int m = idx / (N1 * CPR), rem = idx - m * (N1 * CPR);
+      const int row = rem / CPR, q = rem - row * CPR;
+      const int tok = perm_token(row * N2 + tl.a, P.N);
+      const char *src = (m ? vb : kb) + (long long)tok * P.stride_token_b + 16 * q;
+      cp_async16(dst0 + (m * N1 + row) * ROWB + 16 * q, src);
+    }
+  }
+
+  __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
+                                 double (*red)[4], int tid) {
+    const int N2 = P.N / N1;
+    const int cp = tid % CPW, j = tid / CPW;
+    const char *in = reinterpret_cast<const char *>(buf);
+    c2 x[16];
+    float2 aK = make_float2(0.f, 0.f), aV = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const int row = j + R1B * p;
+      x[p].r = Pair<T>::ld(in + row * ROWB + cp * 2 * ES);
+      x[p].i = Pair<T>::ld(in + (N1 + row) * ROWB + cp * 2 * ES);
+      aK = pfma(x[p].r, x[p].r, aK);
+      aV = pfma(x[p].i, x[p].i, aV);
+    }
+    {
+      const double a = warp_sum_d((double)(aK.x + aK.y)), b = warp_sum_d((double)(aV.x + aV.y));
+      if ((tid & 31) == 0) { red[0][tid >> 5] = a; red[1][tid >> 5] = b; }
+    }
+    __syncthreads();                       // every thread has its inputs; the buffer becomes the exchange area
+    dftp<16, -1>(x);
+    const int tstep = ntab / N1;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      if (p > 0) x[p] = cmul_b(x[p], twb[j * p * tstep]);
+      buf[(j + R1B * p) * CPW + cp] = to4(x[p]);
+    }
+    __syncthreads();
+    float2 *slot = slot_base(P, tl.unit);
+    const int col = tl.cb * 2 * CPW + 2 * cp;
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R1B * it;
+      c2 y[R1B];
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) y[q] = from4(buf[(q + R1B * pp) * CPW + cp]);
+      dftp<R1B, -1>(y);
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) {
+        const int k1 = pp + 16 * q;
+        float4 *dst = reinterpret_cast<float4 *>(slot + ((size_t)k1 * N2 + tl.a) * P.UC + col);
+        __stcg(dst, to4(y[q]));
+      }
+    }
+    if (tid == 0) {
+      const size_t s = (size_t)tl.unit * P.n1t + (size_t)tl.a * P.ncb1 + tl.cb;
+      P.part_tot[2 * s] = red[0][0] + red[0][1] + red[0][2] + red[0][3];
+      P.part_tot[2 * s + 1] = red[1][0] + red[1][1] + red[1][2] + red[1][3];
+    }
+  }
+};
+
+// ------------------------------------------------------------------ pass 2
+// Tile (unit, x, cb): bins k1a = x and k1b = N1 - x (x = 0: k1 = 0 and k1 = N1/2, each its own
+// partner) of 2*CP channels.  Thread (cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2*CP)).
+template <int R2B>
+struct Pass2 {
+  static constexpr int N2 = 16 * R2B, CP = NT / (2 * R2B), IT = 16 / R2B, NAB = R2B + 16;
+
+  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, float4 *ab, float2 *chf, int tid) {
+    const int N1 = P.N / N2;
+    const int k1a = tl.a, k1b = tl.a == 0 ? N1 / 2 : N1 - tl.a;
+    const float2 *slot = slot_base(P, tl.unit);
+    const int col = tl.cb * 2 * CP;
+#pragma unroll
+    for (int idx = tid; idx < 2 * N2 * CP; idx += NT) {
+      const int hf = idx / (N2 * CP), rem = idx - hf * (N2 * CP);
+      const int n2 = rem / CP, cpi = rem - n2 * CP;
+      const int k1 = hf ? k1b : k1a;
+      cp_async16(buf + idx, slot + ((size_t)k1 * N2 + n2) * P.UC + col + 2 * cpi);
+    }
+    // per-tile twiddle factors: w_N^(k1*n2) = A[j] * B[p] for n2 = j + R2B*p
+    const int ms = P.master_len / P.N;
+    if (tid < 2 * NAB) {
+      const int hf = tid / NAB, r = tid - hf * NAB;
+      const int k1 = hf ? k1b : k1a;
+      const int m = (r < R2B ? k1 * r : k1 * R2B * (r - R2B)) & (P.N - 1);
+      ab[hf * NAB + r] = bcast4(__ldg(P.master + (size_t)m * ms));
+    } else if (tid < 2 * NAB + 2) {
+      const int hf = tid - 2 * NAB;
+      const int k1 = hf ? k1b : k1a;
+      chf[hf] = __ldg(P.master + (size_t)k1 * (P.master_len / (2 * P.N)));      // exp(-j*pi*k1/N)
+    }
+  }
+
+  __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
+                                 const float2 *t2, const float4 *ab, const float2 *chf, int tid) {
+    const int N1 = P.N / N2, N = P.N;
+    const int cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
+    const bool self = tl.a == 0;
+    const int k1 = hf ? (self ? N1 / 2 : N1 - tl.a) : tl.a;
+    float4 *Sh = buf + hf * (N2 * CP);
+    const float4 *Sp = buf + (self ? hf : 1 - hf) * (N2 * CP);
+    const float4 A = ab[hf * NAB + j];
+    const float4 *B = ab + hf * NAB + R2B;
+    const int tstep = ntab / N2;
+    c2 x[16];
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      x[p] = from4(Sh[(j + R2B * p) * CP + cp]);
+      x[p] = cmul_b(x[p], wmul_b(A, B[p]));
+    }
+    dftp<16, -1>(x);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      if (p > 0) x[p] = cmul_b(x[p], twb[j * p * tstep]);
+      Sh[(j + R2B * p) * CP + cp] = to4(x[p]);        // same cell this thread read: no barrier needed before
+    }
+    __syncthreads();
+    // second forward stage; registers keep bin k2 = pp + 16*q at index it*R2B + q, shared memory the same
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R2B * it;
+      c2 y[R2B];
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) y[q] = from4(Sh[(q + R2B * pp) * CP + cp]);
+      dftp<R2B, -1>(y);
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) {
+        x[it * R2B + q] = y[q];
+        Sh[(q + R2B * pp) * CP + cp] = to4(y[q]);
+      }
+    }
+    __syncthreads();                       // full spectra of both halves are in shared memory
+    const float2 ch = chf[hf];
+    const float2 half2 = bc(0.5f);
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R2B * it;
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) {
+        const int k2 = pp + 16 * q;
+        const int bin = k1 + N1 * k2;
+        const bool inL = bin <= P.omega, inH = (N - bin) <= P.omega;
+        c2 &Pv = x[it * R2B + q];
+        if (bin == 0 || (inL && inH)) {
+          Pv.r = make_float2(0.f, 0.f);
+          Pv.i = make_float2(0.f, 0.f);
+        } else if (inL || inH) {
+          const int k2p = (k1 == 0) ? ((N2 - k2) & (N2 - 1)) : (N2 - 1 - k2);
+          const c2 Q = from4(Sp[((k2p >> 4) + R2B * (k2p & 15)) * CP + cp]);
+          const float2 tt = t2[k2];
+          const float sgn = inL ? -0.5f : 0.5f;                  // E = (P -/+ uQ)/2, u = exp(+j*pi*bin/N)
+          const float er = ch.x * tt.x - ch.y * tt.y, ei = ch.x * tt.y + ch.y * tt.x;   // exp(-j*pi*bin/N)
+          const float2 ur = bc(er * sgn), ui = bc(-ei * sgn), nui = bc(ei * sgn);
+          Pv.r = pfma(Q.i, nui, pfma(Q.r, ur, pmul(Pv.r, half2)));
+          Pv.i = pfma(Q.i, ur, pfma(Q.r, ui, pmul(Pv.i, half2)));
+        }
+      }
+    }
+    // first inverse stage (mirror of the second forward stage), in registers
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      c2 y[R2B];
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) y[q] = x[it * R2B + q];
+      dftp<R2B, +1>(y);
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) x[it * R2B + q] = y[q];
+    }
+    __syncthreads();                       // all partner reads are done
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R2B * it;
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) Sh[(q + R2B * pp) * CP + cp] = to4(x[it * R2B + q]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      x[p] = from4(Sh[(j + R2B * p) * CP + cp]);
+      if (p > 0) x[p] = cmulc_b(x[p], twb[j * p * tstep]);
+    }
+    dftp<16, +1>(x);
+    float2 *base = slot_base(P, tl.unit) + (size_t)k1 * N2 * P.UC + tl.cb * 2 * CP + 2 * cp;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const c2 o = cmulc_b(x[p], wmul_b(A, B[p]));
+      __stcg(reinterpret_cast<float4 *>(base + (size_t)(j + R2B * p) * P.UC), to4(o));
+    }
+  }
+};
+
+// ------------------------------------------------------------------ pass 3
+// Tile (head, n2): inverse DFT over k1 of every channel of the head, slice by slice
+// (2*CPW channels per slice), |.|^2 summed over the channels -> one score per row.
+// Thread (cp = tid % CPW, j = tid / CPW).
+template <int CNT, int S>
+struct RowReduce {     // halves the CNT row sums across lanes cp ^ S, then continues with S/2
+  __device__ static void run(float (&acc)[16], int cp, int &prow) {
+    if constexpr (S >= 1) {
+      if constexpr (CNT > 1) {
+        constexpr int H = CNT / 2;
+        const bool up = (cp & S) != 0;
+#pragma unroll
+        for (int i = 0; i < H; ++i) {
+          const float send = up ? acc[i] : acc[i + H];
+          const float keep = up ? acc[i + H] : acc[i];
+          acc[i] = keep + __shfl_xor_sync(0xffffffffu, send, S);
+        }
+        if (up) prow += H;
+        RowReduce<H, S / 2>::run(acc, cp, prow);
+      } else {
+        acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], S);
+        RowReduce<1, S / 2>::run(acc, cp, prow);
+      }
+    }
+  }
+};
+
+template <int R1B>
+struct Pass3 {
+  static constexpr int N1 = 16 * R1B, CPW = NT / R1B, IT = 16 / R1B;
+  static constexpr int LEFT = CPW >= 16 ? 1 : 16 / CPW;       // row sums a lane ends up with
+  static constexpr int DUP = CPW > 16 ? CPW / 16 : 1;         // lanes that end up with the same row sum
+
+  __device__ static void issue(const Params &P, const Tile &tl, int slice, float4 *buf, int tid) {
+    const int N2 = P.N / N1;
+    const int gc = slice * 2 * CPW;
+    const int unit = tl.unit * P.upd + gc / P.UC, col = gc % P.UC;
+    const float2 *slot = slot_base(P, unit);
+#pragma unroll
+    for (int idx = tid; idx < N1 * CPW; idx += NT) {
+      const int k1 = idx / CPW, cpi = idx - k1 * CPW;
+      cp_async16(buf + idx, slot + ((size_t)k1 * N2 + tl.a) * P.UC + col + 2 * cpi);
+    }
+  }
+
+  // one slice, data already in buf; adds to acc / totK / totV
+  __device__ static void slice(float4 *buf, const float4 *twb, int tstep, int cp, int j,
+                               float (&acc)[16], float2 &totK, float2 &totV) {
+    c2 x[16];
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R1B * it;
+      c2 y[R1B];
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) y[q] = from4(buf[(pp + 16 * q) * CPW + cp]);
+      dftp<R1B, +1>(y);
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) x[it * R1B + q] = y[q];
+    }
+    __syncthreads();                       // all bins read; the buffer becomes the exchange area
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R1B * it;
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) buf[(q + R1B * pp) * CPW + cp] = to4(x[it * R1B + q]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      x[p] = from4(buf[(j + R1B * p) * CPW + cp]);
+      if (p > 0) x[p] = cmulc_b(x[p], twb[j * p * tstep]);
+    }
+    dftp<16, +1>(x);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const float2 t = pfma(x[p].i, x[p].i, pmul(x[p].r, x[p].r));
+      acc[p] += t.x + t.y;
+      totK = pfma(x[p].r, x[p].r, totK);
+      totV = pfma(x[p].i, x[p].i, totV);
+    }
+  }
+
+  __device__ static void finish(const Params &P, const Tile &tl, float (&acc)[16], float2 totK, float2 totV,
+                                double (*red)[4], int tid) {
+    const int N2 = P.N / N1;
+    const int cp = tid % CPW, j = tid / CPW;
+    int prow = 0;
+    RowReduce<16, CPW / 2>::run(acc, cp, prow);
+    if ((cp & (DUP - 1)) == 0) {
+#pragma unroll
+      for (int i = 0; i < LEFT; ++i) {
+        const int p = (j + R1B * (prow + i)) * N2 + tl.a;
+        P.scores[(long long)tl.unit * P.score_stride + perm_token(p, P.N)] = acc[i] * P.inv_scale;
+      }
+    }
+    const double dk = warp_sum_d((double)((totK.x + totK.y) * P.inv_scale));
+    const double dv = warp_sum_d((double)((totV.x + totV.y) * P.inv_scale));
+    if ((tid & 31) == 0) { red[0][tid >> 5] = dk; red[1][tid >> 5] = dv; }
+    __syncthreads();
+    if (tid == 0) {
+      const size_t s = (size_t)tl.unit * P.n3t + tl.a;
+      P.part_hi[2 * s] = (red[0][0] + red[0][1] + red[0][2] + red[0][3]) * (double)P.head_dim;   // d * sum Dev_k
+      P.part_hi[2 * s + 1] = (red[1][0] + red[1][1] + red[1][2] + red[1][3]) * (double)P.head_dim;
+    }
+  }
+};
+
+// ------------------------------------------------------------------ the kernel
+template <int R1B, int R2B>
+struct Smem {
+  static constexpr int N1 = 16 * R1B, N2 = 16 * R2B, NTAB = N1 > N2 ? N1 : N2, NAB = R2B + 16;
+  static constexpr size_t bytes = (size_t)2 * TILE4 * sizeof(float4) + NTAB * sizeof(float4) + N2 * sizeof(float2) +
+                                  2 * 2 * NAB * sizeof(float4) + 2 * 2 * sizeof(float2);
+};
+
+template <typename T, int R1B, int R2B>
+__global__ void __launch_bounds__(NT, 3) k_fused(const __grid_constant__ Params P) {
+  using SM = Smem<R1B, R2B>;
+  using P1 = Pass1<T, R1B>;
+  using P2 = Pass2<R2B>;
+  using P3 = Pass3<R1B>;
+  constexpr int NTAB = SM::NTAB, N2 = SM::N2, NAB = SM::NAB;
+  extern __shared__ float4 smem4[];
+  float4 *bufs = smem4;                                           // [2][TILE4]
+  float4 *twb = smem4 + 2 * TILE4;                                // [NTAB] exp(-2*pi*j*i/NTAB), broadcast
+  float2 *t2 = reinterpret_cast<float2 *>(twb + NTAB);            // [N2]   exp(-j*pi*k2/N2)
+  float4 *ab = reinterpret_cast<float4 *>(t2 + N2);               // [2 buffers][2 halves][NAB]
+  float2 *chf = reinterpret_cast<float2 *>(ab + 2 * 2 * NAB);     // [2 buffers][2 halves]
+  __shared__ Tile desc[2];
+  __shared__ double red[2][4];
+  __shared__ int s_ok;
+  const int tid = threadIdx.x;
+  Sched *sc = P.sched;
+
+  for (int i = tid; i < NTAB; i += NT) twb[i] = bcast4(__ldg(P.master + (size_t)i * (P.master_len / NTAB)));
+  for (int i = tid; i < N2; i += NT) t2[i] = __ldg(P.master + (size_t)i * (P.master_len / (2 * N2)));
+
+  Walk walk = {0, 0u};
+  if (tid == 0) {
+    Tile first;
+    if (ld_acquire(&sc->abort_flag) != 0u) { first.phase = PH_NONE; first.unit = first.a = first.cb = first.ready = 0; }
+    else first = decode_tile(P, walk, atomicAdd(&sc->tile_counter, 1u));
+    desc[0] = first;
+  }
+  __syncthreads();
+  Tile cur = desc[0];
+  int b = 0;
+  bool issued = false;
+
+  while (cur.phase != PH_NONE) {
+    if (tid == 0) {
+      int ok = 1;
+      if (!issued) ok = wait_deps(P, cur) ? 1 : 0;
+      Tile nx;
+      nx.phase = PH_NONE; nx.unit = nx.a = nx.cb = nx.ready = 0;
+      if (ok && ld_acquire(&sc->abort_flag) == 0u) {
+        nx = decode_tile(P, walk, atomicAdd(&sc->tile_counter, 1u));
+        if (nx.phase != PH_NONE) nx.ready = deps_ok(P, nx) ? 1 : 0;
+      }
+      desc[b ^ 1] = nx;
+      s_ok = ok;
+    }
+    __syncthreads();
+    if (!s_ok) break;
+    const Tile nxt = desc[b ^ 1];
+    bool nxt_issued = false;
+
+    // loads of the tile after this one go to the buffer this tile does not end in
+    auto prefetch = [&](int nb) {
+      if (nxt.phase != PH_NONE && nxt.ready) {
+        float4 *dst = bufs + nb * TILE4;
+        if (nxt.phase == PH_P1) P1::issue(P, nxt, dst, tid);
+        else if (nxt.phase == PH_P2) P2::issue(P, nxt, dst, ab + nb * 2 * NAB, chf + nb * 2, tid);
+        else P3::issue(P, nxt, 0, dst, tid);
+        cp_async_commit();
+        nxt_issued = true;
+      }
+    };
+
+    if (cur.phase == PH_P3) {
+      const int nsl = P.head_dim / (2 * P3::CPW);
+      if (!issued) { P3::issue(P, cur, 0, bufs + b * TILE4, tid); cp_async_commit(); }
+      float acc[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+      float2 totK = make_float2(0.f, 0.f), totV = make_float2(0.f, 0.f);
+      const int cp = tid % P3::CPW, j = tid / P3::CPW;
+      for (int s = 0; s < nsl; ++s) {
+        bool more = false;
+        if (s + 1 < nsl) { P3::issue(P, cur, s + 1, bufs + (b ^ 1) * TILE4, tid); cp_async_commit(); more = true; }
+        else { prefetch(b ^ 1); more = nxt_issued; }
+        if (more) cp_async_wait<1>(); else cp_async_wait<0>();
+        __syncthreads();
+        P3::slice(bufs + b * TILE4, twb, NTAB / P3::N1, cp, j, acc, totK, totV);
+        b ^= 1;
+      }
+      P3::finish(P, cur, acc, totK, totV, red, tid);
+    } else {
+      if (cur.phase == PH_P1) {
+        if (!issued) { P1::issue(P, cur, bufs + b * TILE4, tid); cp_async_commit(); }
+      } else {
+        if (!issued) { P2::issue(P, cur, bufs + b * TILE4, ab + b * 2 * NAB, chf + b * 2, tid); cp_async_commit(); }
+      }
+      prefetch(b ^ 1);
+      if (nxt_issued) cp_async_wait<1>(); else cp_async_wait<0>();
+      __syncthreads();
+      if (cur.phase == PH_P1) P1::compute(P, cur, bufs + b * TILE4, twb, NTAB, red, tid);
+      else P2::compute(P, cur, bufs + b * TILE4, twb, NTAB, t2, ab + b * 2 * NAB, chf + b * 2, tid);
+      b ^= 1;
+    }
+    __syncthreads();                       // every store of the tile has been issued
+    if (tid == 0) signal_done(P, cur);
+    cur = nxt;
+    issued = nxt_issued;
+  }
+
+  // ---- exit: the last block to leave adds up the energy partial sums in a fixed order and
+  // returns the scheduler state to all-zero
+  cp_async_wait<0>();
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    const unsigned prev = atomicAdd(&sc->exit_counter, 1u);
+    s_ok = (prev + 1u == gridDim.x) ? 1 : 0;
+  }
+  __syncthreads();
+  if (!s_ok) return;
+  __threadfence();
+  double *redd = reinterpret_cast<double *>(smem4);        // [4][NT]
+  const int n_tot = P.U * P.n1t, n_hi = P.num_heads * P.n3t;
+  double a0 = 0, a1 = 0, b0 = 0, b1 = 0;
+  for (int i = tid; i < n_tot; i += NT) { a0 += __ldcg(P.part_tot + 2 * i); a1 += __ldcg(P.part_tot + 2 * i + 1); }
+  for (int i = tid; i < n_hi; i += NT) { b0 += __ldcg(P.part_hi + 2 * i); b1 += __ldcg(P.part_hi + 2 * i + 1); }
+  redd[tid] = b0; redd[NT + tid] = a0; redd[2 * NT + tid] = b1; redd[3 * NT + tid] = a1;
+  __syncthreads();
+  for (int st = NT / 2; st > 0; st >>= 1) {
+    if (tid < st)
+      for (int q = 0; q < 4; ++q) redd[q * NT + tid] += redd[q * NT + tid + st];
+    __syncthreads();
+  }
+  if (tid < 4) P.energy[tid] = redd[tid * NT];
+  for (int i = tid; i < 1024; i += NT) { sc->done1[i] = 0u; sc->done2[i] = 0u; sc->done3[i] = 0u; }
+  if (tid == 0) { sc->tile_counter = 0u; sc->exit_counter = 0u; sc->abort_flag = 0u; }
+}
+
+}  // namespace fused
