@@ -90,6 +90,12 @@ uint64_t fc_launch_count(const fc_handle *h);
 fc_status fc_profile_begin(fc_handle *h, int32_t kernel_class, int32_t max_launches);
 fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *launches);
 
+/* Running totals of the fused transform kernel since fc_create (diagnostic; synchronises the
+ * device): out = { tiles processed, tiles whose inputs were not finished when they were looked
+ * at one tile ahead, cycles spent reporting finished tiles, clock cycles (thread 0 of every block, summed) inside
+ * pass-1, pass-2 and pass-3 tiles, cycles waiting for tile data, cycles inside the tile loop }. */
+fc_status fc_fused_stats(fc_handle *h, uint64_t out[8]);
+
 /* Target size in bytes of the transform intermediates processed per kernel group
  * (kept below the L2 capacity so they are re-read from cache, not HBM).
  * Default 32 MiB.  Affects speed only. */

@@ -52,6 +52,8 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->fused_sched = nullptr;
   h->fused_enabled = 0;   // the separate-launch kernels are still faster; FC_FUSED=1 switches the fused kernel on
   h->fused_blocks_per_sm = 0;
+  h->fused_lag = 1;
+  if (const char *e = getenv("FC_FUSED_LAG")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_lag = v; }
   if (const char *e = getenv("FC_FUSED")) { h->fused_enabled = atoi(e) != 0 ? 1 : 0; }
   if (const char *e = getenv("FC_FUSED_BPS")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_blocks_per_sm = v; }
   cudaDeviceProp prop;
@@ -164,6 +166,14 @@ extern "C" fc_status fc_last_device_status(fc_handle *h, fc_stream stream) {
   if (word != 0) FC_CUDA_TRY(cudaMemset(h->status_word, 0, sizeof(int)));
   if (word == 0) return FC_OK;
   return (word & FC_DEV_FLAG_INTERNAL) ? FC_ERR_INTERNAL : FC_ERR_TIMEOUT;
+}
+
+extern "C" fc_status fc_fused_stats(fc_handle *h, uint64_t out[8]) {
+  if (!h || !out || !h->fused_sched) return FC_ERR_INVALID_ARG;
+  FC_CUDA_TRY(cudaDeviceSynchronize());
+  const fused::Sched *sc = static_cast<const fused::Sched *>(h->fused_sched);
+  FC_CUDA_TRY(cudaMemcpy(out, sc->stats, 8 * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+  return FC_OK;
 }
 
 extern "C" uint64_t fc_launch_count(const fc_handle *h) { return h ? (uint64_t)h->launches : 0; }

@@ -44,6 +44,7 @@ struct fc_handle {
   void *fused_sched;
   int fused_enabled;       // 1 enables the fused kernel (developer knob FC_FUSED)
   int fused_blocks_per_sm; // 0 = as many as fit
+  int fused_lag;           // stages between pass 1, pass 2 and pass 3 of a unit
 };
 
 // Kernel classes for fc_profile_begin.

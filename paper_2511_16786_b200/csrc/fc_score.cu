@@ -490,9 +490,8 @@ SeqPlan plan_sequence(int N, bool allow_fast = true) {
 struct FusedPlan {
   bool ok;
   int r1b, r2b;                 // N1 = 16*r1b, N2 = 16*r2b
-  int UC, upd, U, R;
-  int n1t, n2t, n3t, ncb1, ncb2;
-  size_t ring_bytes, part_tot_bytes, part_hi_bytes;
+  int UC, U, R, lag, TPU, ncb1, ncb2, nparts;
+  size_t ring_bytes, part_bytes, partial_bytes;
 };
 
 FusedPlan plan_fused(const fc_handle *h, const SeqPlan &sp, int H, int d) {
@@ -507,19 +506,20 @@ FusedPlan plan_fused(const fc_handle *h, const SeqPlan &sp, int H, int d) {
   while (uc > min_uc && (uc > d || d % uc != 0)) uc >>= 1;
   if (uc > d || d % uc != 0 || uc % (2 * cpw) != 0 || uc % (2 * cp) != 0) return f;
   f.UC = uc;
-  f.upd = d / uc;
-  f.U = H * f.upd;
-  if (f.U > 1024 || H > 1024) return f;
-  f.R = f.upd + 3;                                  // a slot is rewritten at least two stages after its last reader was handed out
+  f.U = H * (d / uc);
+  f.nparts = d / (2 * cpw);
+  if (f.U > 1024 || (f.nparts > 1 && (long long)H * sp.N2 > fused::kMaxCnt3)) return f;
+  // pass 3 of unit u-R is handed out in stage u-R+2*lag; pass 1 of unit u rewrites its slot in stage u:
+  // R = 2*lag + 3 puts three stages between them
+  f.lag = h->fused_lag;
+  f.R = 2 * f.lag + 3;
   if (f.R > f.U) f.R = f.U;
+  f.TPU = (int)((long long)sp.N * uc / 4096);
   f.ncb1 = uc / (2 * cpw);
   f.ncb2 = uc / (2 * cp);
-  f.n1t = sp.N2 * f.ncb1;
-  f.n2t = (sp.N1 / 2) * f.ncb2;
-  f.n3t = sp.N2;
   f.ring_bytes = align_up((size_t)f.R * sp.N * uc * sizeof(float2), 256);
-  f.part_tot_bytes = align_up((size_t)f.U * f.n1t * 2 * sizeof(double), 256);
-  f.part_hi_bytes = align_up((size_t)H * f.n3t * 2 * sizeof(double), 256);
+  f.part_bytes = align_up((size_t)f.U * f.TPU * 2 * sizeof(double), 256);
+  f.partial_bytes = f.nparts > 1 ? align_up((size_t)f.nparts * H * sp.N * sizeof(float), 256) : 0;
   f.ok = true;
   return f;
 }
@@ -536,12 +536,13 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   ScoreLayout L;
   {
     const FusedPlan f = plan_fused(h, sp, num_heads, head_dim);
-    if (f.ok) {                                      // ring | pass-1 partial sums | pass-3 partial sums
+    if (f.ok) {                                      // ring | pass-1 energy sums | pass-3 energy sums | partial scores
       L = ScoreLayout{};
       L.off_ws = 0;
       L.off_part_tot = f.ring_bytes;
-      L.off_part_hi = f.ring_bytes + f.part_tot_bytes;
-      L.total = f.ring_bytes + f.part_tot_bytes + f.part_hi_bytes;
+      L.off_part_hi = f.ring_bytes + f.part_bytes;
+      L.off_spec = f.ring_bytes + 2 * f.part_bytes;
+      L.total = f.ring_bytes + 2 * f.part_bytes + f.partial_bytes;
       L.ws_buf_bytes = f.ring_bytes;
       L.heads_per_group = num_heads;
       return L;
@@ -766,10 +767,11 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       P.stride_token_b = (long long)kv->stride_token * es;
       P.stride_head_b = (long long)kv->stride_head * es;
       P.N = N; P.omega = omega; P.head_dim = d; P.num_heads = H;
-      P.UC = f.UC; P.upd = f.upd; P.U = f.U; P.R = f.R;
-      P.n1t = f.n1t; P.n2t = f.n2t; P.n3t = f.n3t; P.ncb1 = f.ncb1; P.ncb2 = f.ncb2;
-      P.total_tiles = (unsigned)((long long)f.U * (f.n1t + f.n2t) + (long long)H * f.n3t);
+      P.UC = f.UC; P.U = f.U; P.R = f.R; P.lag = f.lag;
+      P.TPU = f.TPU; P.ncb1 = f.ncb1; P.ncb2 = f.ncb2; P.nparts = f.nparts;
+      P.total_tiles = (unsigned)(3ll * f.U * f.TPU);
       P.ws = ws;
+      P.partial = reinterpret_cast<float *>(spec);
       P.master = h->master; P.master_len = h->master_len;
       P.scores = scores + start; P.score_stride = total_tokens;
       P.inv_scale = (float)(1.0 / ((double)N * (double)N * (double)d));

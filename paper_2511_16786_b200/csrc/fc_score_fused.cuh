@@ -3,15 +3,19 @@
 // as fc_score.cu (see the header comment there); what differs:
 //
 //  * ONE launch scores a whole (layer, sequence).  The columns of the layer are cut into
-//    units of UC complex columns (about 8 MB of intermediate each); the tiles of
-//    pass 1 of unit s, pass 2 of unit s-1 and pass 3 of the head completed at s-2 form
-//    stage s.  Persistent blocks take tiles in stage order from an atomic counter and
+//    units of UC complex columns (about 8 MB of intermediate each); stage s consists of
+//    the pass-1 tiles of unit s, then the pass-2 tiles of unit s-1, then the pass-3 tiles
+//    of unit s-2.  Persistent blocks take tiles in that order from an atomic counter and
 //    wait (bounded) on per-unit completion counters, so a tile only ever waits for
-//    tiles that were handed out before it.  The intermediates live in a ring of unit
-//    slots that stays in L2.
-//  * every tile is 2048 float4 (32 KB), processed by 128 threads; the next tile is
-//    fetched into the second shared-memory buffer with cp.async while the current one
-//    is transformed in place.
+//    tiles that were handed out before it; a producer and its first consumer are three
+//    tile blocks apart, more than the blocks in flight, so the wait is normally over
+//    before it starts.  The intermediates live in a ring of unit slots that stays in L2.
+//  * every tile is 4096 complex points = 2048 float4 (32 KB), processed by 128 threads;
+//    the next tile is fetched into the second shared-memory buffer with cp.async while the
+//    current one is transformed in place.  Thread 0 asks for tile indices and reads
+//    completion counters one step ahead, so those round trips are off the critical path.
+//  * pass 3 writes one partial score per 2*CPW channels; the block that delivers the last
+//    partial of a (head, row set) adds them in a fixed order (deterministic).
 //  * a thread owns two adjacent channels as ONE packed value per component:
 //    float4 = (re_a, re_b, im_a, im_b), and all butterflies run on the packed
 //    fp32x2 add/mul/fma instructions of sm_100, halving the issue slots of the
@@ -24,7 +28,8 @@
 namespace fused {
 
 constexpr int NT = 128;        // threads per block
-constexpr int TILE4 = 2048;    // float4 per tile buffer
+constexpr int TILE4 = 2048;    // float4 per tile
+constexpr int BUF4 = TILE4 + 16; // float4 per shared-memory buffer (room for the pass-2 bank padding)
 
 // Scheduler state in global memory (owned by the handle, all zero between launches).
 struct Sched {
@@ -34,19 +39,27 @@ struct Sched {
   unsigned pad;
   unsigned done1[1024];   // pass-1 tiles finished per unit
   unsigned done2[1024];   // pass-2 tiles finished per unit
-  unsigned done3[1024];   // pass-3 tiles finished per head
+  unsigned done3[1024];   // pass-3 tiles finished per unit
+  unsigned cnt3[65536];   // partial scores delivered per (head, n2); the last deliverer resets its entry
+  // running totals since the handle was created (diagnostic, see fc_fused_stats): tiles, tiles whose
+  // dependencies were not finished at look-ahead time, wait iterations, clock cycles of thread 0 inside
+  // pass-1 / pass-2 / pass-3 tiles, cycles waiting for tile data, cycles in the tile loop
+  unsigned long long stats[8];
 };
+constexpr int kMaxCnt3 = 65536;
 
 struct Params {
   const void *k, *v;               // first token of the sequence
   long long stride_token_b, stride_head_b;   // bytes
   int N, omega, head_dim, num_heads;
-  int UC, upd, U, R;               // unit columns, units per head, units, ring slots
-  int n1t, n2t, n3t, ncb1, ncb2;   // tiles per unit (pass 1, 2), per head (pass 3); column blocks per unit
+  int UC, U, R, lag;               // unit columns, units, ring slots, stages between the passes of a unit
+  int TPU, ncb1, ncb2;             // tiles per unit and pass; column blocks per unit in pass 1/3 and in pass 2
+  int nparts;                      // partial scores per (head, token) = head_dim / (2*CPW)
   unsigned total_tiles;
   float2 *ws;                      // ring of R unit slots, each [N1*N2][UC] float2 (stored as planar pairs)
   const float2 *master;
   int master_len;
+  float *partial;                  // [nparts][num_heads][N] partial scores (used when nparts > 1)
   float *scores;                   // already offset to the sequence's first token
   long long score_stride;          // tokens in the packed batch
   float inv_scale;                 // 1 / (N^2 d)
@@ -242,74 +255,69 @@ template <> struct Pair<__nv_bfloat16> {
   }
 };
 
+
 // ------------------------------------------------------------------ tile descriptors
 enum { PH_NONE = 0, PH_P1 = 1, PH_P2 = 2, PH_P3 = 3 };
 struct Tile {
   int phase;   // PH_*
-  int unit;    // unit (pass 1, 2) or head (pass 3)
+  int unit;
   int a;       // n2 (pass 1, 3) or k1 pair index x (pass 2)
-  int cb;      // column block inside the unit (pass 1, 2)
-  int ready;   // dependencies were already satisfied when the tile was fetched
+  int cb;      // column block inside the unit
+  int idx;     // tile number inside its (unit, pass)
+  int ready;   // the tiles it depends on had finished when thread 0 looked
 };
 
 // Stage walk kept by thread 0: tiles are fetched in increasing order, so it only moves forward.
 struct Walk { int stage; unsigned start; };
 
-__device__ __forceinline__ void stage_counts(const Params &P, int s, int &c1, int &c2, int &c3) {
-  c1 = (s < P.U) ? P.n1t : 0;
-  c2 = (s >= 1 && s <= P.U) ? P.n2t : 0;
-  c3 = (s >= 2 && s - 2 < P.U && (s - 2) % P.upd == P.upd - 1) ? P.n3t : 0;
+__device__ __forceinline__ int stage_blocks(const Params &P, int s) {
+  const int l = P.lag;
+  return (s < P.U ? 1 : 0) + ((s >= l && s < P.U + l) ? 1 : 0) + ((s >= 2 * l && s < P.U + 2 * l) ? 1 : 0);
 }
 
 __device__ __forceinline__ Tile decode_tile(const Params &P, Walk &w, unsigned t) {
   Tile tl;
-  tl.ready = 0;
-  if (t >= P.total_tiles) { tl.phase = PH_NONE; tl.unit = tl.a = tl.cb = 0; return tl; }
-  int c1, c2, c3;
-  stage_counts(P, w.stage, c1, c2, c3);
-  while (t >= w.start + (unsigned)(c1 + c2 + c3)) {
-    w.start += (unsigned)(c1 + c2 + c3);
+  tl.phase = PH_NONE; tl.unit = tl.a = tl.cb = tl.idx = tl.ready = 0;
+  if (t >= P.total_tiles) return tl;
+  unsigned cnt = (unsigned)(stage_blocks(P, w.stage) * P.TPU);
+  while (t >= w.start + cnt) {
+    w.start += cnt;
     ++w.stage;
-    stage_counts(P, w.stage, c1, c2, c3);
+    cnt = (unsigned)(stage_blocks(P, w.stage) * P.TPU);
   }
-  int i = (int)(t - w.start);
-  if (i < c3) {
-    tl.phase = PH_P3; tl.unit = (w.stage - 2) / P.upd; tl.a = i; tl.cb = 0;
-    return tl;
-  }
-  i -= c3;
-  const int m = c1 < c2 ? c1 : c2;
-  int idx, ph;
-  if (i < 2 * m) { ph = (i & 1) ? PH_P1 : PH_P2; idx = i >> 1; }
-  else { idx = m + (i - 2 * m); ph = (c1 > c2) ? PH_P1 : PH_P2; }
-  tl.phase = ph;
-  if (ph == PH_P1) { tl.unit = w.stage; tl.a = idx / P.ncb1; tl.cb = idx - tl.a * P.ncb1; }
-  else { tl.unit = w.stage - 1; tl.a = idx / P.ncb2; tl.cb = idx - tl.a * P.ncb2; }
+  const int s = w.stage;
+  const int i = (int)(t - w.start);
+  int blk = i / P.TPU;
+  tl.idx = i - blk * P.TPU;
+  // blocks present in stage s, in order: pass 1 of unit s, pass 2 of unit s-lag, pass 3 of unit s-2*lag
+  const int l = P.lag;
+  if (s >= P.U) ++blk;                                  // no pass-1 block
+  if (blk >= 1 && !(s >= l && s < P.U + l)) ++blk;      // no pass-2 block
+  if (blk == 0) { tl.phase = PH_P1; tl.unit = s; tl.a = tl.idx / P.ncb1; tl.cb = tl.idx - tl.a * P.ncb1; }
+  else if (blk == 1) { tl.phase = PH_P2; tl.unit = s - l; tl.a = tl.idx / P.ncb2; tl.cb = tl.idx - tl.a * P.ncb2; }
+  else { tl.phase = PH_P3; tl.unit = s - 2 * l; tl.a = tl.idx / P.ncb1; tl.cb = tl.idx - tl.a * P.ncb1; }
   return tl;
 }
 
-// Are the tiles this one depends on finished?  (thread 0 only)
-__device__ __forceinline__ bool deps_ok(const Params &P, const Tile &tl) {
+// The one completion counter a tile waits for (nullptr: none).  It must reach P.TPU.
+__device__ __forceinline__ const unsigned *dep_counter(const Params &P, const Tile &tl) {
   const Sched *sc = P.sched;
-  if (tl.phase == PH_P1) {
-    if (tl.unit < P.R) return true;
-    return ld_acquire(&sc->done3[(tl.unit - P.R) / P.upd]) >= (unsigned)P.n3t;   // the ring slot was read out
-  }
-  if (tl.phase == PH_P2) return ld_acquire(&sc->done1[tl.unit]) >= (unsigned)P.n1t;
-  if (tl.phase == PH_P3) {
-    for (int u = tl.unit * P.upd; u < (tl.unit + 1) * P.upd; ++u)
-      if (ld_acquire(&sc->done2[u]) < (unsigned)P.n2t) return false;
-    return true;
-  }
-  return true;
+  if (tl.phase == PH_P1) return tl.unit >= P.R ? &sc->done3[tl.unit - P.R] : nullptr;   // ring slot read out
+  if (tl.phase == PH_P2) return &sc->done1[tl.unit];
+  if (tl.phase == PH_P3) return &sc->done2[tl.unit];
+  return nullptr;
 }
 
-// Bounded wait (thread 0 only).  false: gave up or another block gave up.
+// Bounded wait (thread 0 only).  false: gave up, or another block gave up.
 __device__ __forceinline__ bool wait_deps(const Params &P, const Tile &tl) {
+  const unsigned *c = dep_counter(P, tl);
+  if (c == nullptr) return true;
   for (unsigned it = 0; it < P.spin_limit; ++it) {
-    if (deps_ok(P, tl)) return true;
+    if (ld_acquire(c) >= (unsigned)P.TPU) {
+      return true;
+    }
     if (ld_acquire(&P.sched->abort_flag) != 0u) return false;
-    __nanosleep(200);
+    __nanosleep(100);
   }
   atomicExch(&P.sched->abort_flag, 1u);
   atomicOr(P.status, FC_DEV_FLAG_TIMEOUT);
@@ -329,6 +337,7 @@ __device__ __forceinline__ float2 *slot_base(const Params &P, int unit) {
 
 // ------------------------------------------------------------------ pass 1
 // Tile (unit, n2, cb): DFT over n1 of 2*CPW channels.  Thread (cp = tid % CPW, j = tid / CPW).
+// In every pass `pre` runs just before the first block barrier of the tile and `post` just after it.
 template <typename T, int R1B>
 struct Pass1 {
   static constexpr int N1 = 16 * R1B, CPW = NT / R1B, IT = 16 / R1B, ES = Pair<T>::ES;
@@ -352,8 +361,9 @@ struct Pass1 {
     }
   }
 
+  template <class Pre, class Post>
   __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
-                                 double (*red)[4], int tid) {
+                                 double (*red)[4], int tid, Pre pre, Post post) {
     const int N2 = P.N / N1;
     const int cp = tid % CPW, j = tid / CPW;
     const char *in = reinterpret_cast<const char *>(buf);
@@ -371,7 +381,9 @@ struct Pass1 {
       const double a = warp_sum_d((double)(aK.x + aK.y)), b = warp_sum_d((double)(aV.x + aV.y));
       if ((tid & 31) == 0) { red[0][tid >> 5] = a; red[1][tid >> 5] = b; }
     }
+    pre();
     __syncthreads();                       // every thread has its inputs; the buffer becomes the exchange area
+    post();
     dftp<16, -1>(x);
     const int tstep = ntab / N1;
 #pragma unroll
@@ -397,7 +409,7 @@ struct Pass1 {
       }
     }
     if (tid == 0) {
-      const size_t s = (size_t)tl.unit * P.n1t + (size_t)tl.a * P.ncb1 + tl.cb;
+      const size_t s = (size_t)tl.unit * P.TPU + tl.idx;
       P.part_tot[2 * s] = red[0][0] + red[0][1] + red[0][2] + red[0][3];
       P.part_tot[2 * s + 1] = red[1][0] + red[1][1] + red[1][2] + red[1][3];
     }
@@ -407,9 +419,12 @@ struct Pass1 {
 // ------------------------------------------------------------------ pass 2
 // Tile (unit, x, cb): bins k1a = x and k1b = N1 - x (x = 0: k1 = 0 and k1 = N1/2, each its own
 // partner) of 2*CP channels.  Thread (cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2*CP)).
+// The second half starts PAD float4 later so that the two halves of a quarter warp fall into
+// different banks when a row is only 64 bytes.
 template <int R2B>
 struct Pass2 {
   static constexpr int N2 = 16 * R2B, CP = NT / (2 * R2B), IT = 16 / R2B, NAB = R2B + 16;
+  static constexpr int PAD = CP < 8 ? 4 : 0, HALF = N2 * CP + PAD;
 
   __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, float4 *ab, float2 *chf, int tid) {
     const int N1 = P.N / N2;
@@ -421,7 +436,7 @@ struct Pass2 {
       const int hf = idx / (N2 * CP), rem = idx - hf * (N2 * CP);
       const int n2 = rem / CP, cpi = rem - n2 * CP;
       const int k1 = hf ? k1b : k1a;
-      cp_async16(buf + idx, slot + ((size_t)k1 * N2 + n2) * P.UC + col + 2 * cpi);
+      cp_async16(buf + hf * HALF + rem, slot + ((size_t)k1 * N2 + n2) * P.UC + col + 2 * cpi);
     }
     // per-tile twiddle factors: w_N^(k1*n2) = A[j] * B[p] for n2 = j + R2B*p
     const int ms = P.master_len / P.N;
@@ -437,14 +452,15 @@ struct Pass2 {
     }
   }
 
+  template <class Pre, class Post>
   __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
-                                 const float2 *t2, const float4 *ab, const float2 *chf, int tid) {
+                                 const float2 *t2, const float4 *ab, const float2 *chf, int tid, Pre pre, Post post) {
     const int N1 = P.N / N2, N = P.N;
     const int cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
     const bool self = tl.a == 0;
     const int k1 = hf ? (self ? N1 / 2 : N1 - tl.a) : tl.a;
-    float4 *Sh = buf + hf * (N2 * CP);
-    const float4 *Sp = buf + (self ? hf : 1 - hf) * (N2 * CP);
+    float4 *Sh = buf + hf * HALF;
+    const float4 *Sp = buf + (self ? hf : 1 - hf) * HALF;
     const float4 A = ab[hf * NAB + j];
     const float4 *B = ab + hf * NAB + R2B;
     const int tstep = ntab / N2;
@@ -460,7 +476,9 @@ struct Pass2 {
       if (p > 0) x[p] = cmul_b(x[p], twb[j * p * tstep]);
       Sh[(j + R2B * p) * CP + cp] = to4(x[p]);        // same cell this thread read: no barrier needed before
     }
+    pre();
     __syncthreads();
+    post();
     // second forward stage; registers keep bin k2 = pp + 16*q at index it*R2B + q, shared memory the same
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
@@ -536,9 +554,8 @@ struct Pass2 {
 };
 
 // ------------------------------------------------------------------ pass 3
-// Tile (head, n2): inverse DFT over k1 of every channel of the head, slice by slice
-// (2*CPW channels per slice), |.|^2 summed over the channels -> one score per row.
-// Thread (cp = tid % CPW, j = tid / CPW).
+// Tile (unit, n2, cb): inverse DFT over k1 of 2*CPW channels, |.|^2 summed over them -> one
+// partial score per row.  Thread (cp = tid % CPW, j = tid / CPW).
 template <int CNT, int S>
 struct RowReduce {     // halves the CNT row sums across lanes cp ^ S, then continues with S/2
   __device__ static void run(float (&acc)[16], int cp, int &prow) {
@@ -568,11 +585,10 @@ struct Pass3 {
   static constexpr int LEFT = CPW >= 16 ? 1 : 16 / CPW;       // row sums a lane ends up with
   static constexpr int DUP = CPW > 16 ? CPW / 16 : 1;         // lanes that end up with the same row sum
 
-  __device__ static void issue(const Params &P, const Tile &tl, int slice, float4 *buf, int tid) {
+  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, int tid) {
     const int N2 = P.N / N1;
-    const int gc = slice * 2 * CPW;
-    const int unit = tl.unit * P.upd + gc / P.UC, col = gc % P.UC;
-    const float2 *slot = slot_base(P, unit);
+    const float2 *slot = slot_base(P, tl.unit);
+    const int col = tl.cb * 2 * CPW;
 #pragma unroll
     for (int idx = tid; idx < N1 * CPW; idx += NT) {
       const int k1 = idx / CPW, cpi = idx - k1 * CPW;
@@ -580,9 +596,12 @@ struct Pass3 {
     }
   }
 
-  // one slice, data already in buf; adds to acc / totK / totV
-  __device__ static void slice(float4 *buf, const float4 *twb, int tstep, int cp, int j,
-                               float (&acc)[16], float2 &totK, float2 &totV) {
+  template <class Pre, class Post>
+  __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
+                                 double (*red)[4], int *s_last, int tid, Pre pre, Post post) {
+    const int N2 = P.N / N1;
+    const int cp = tid % CPW, j = tid / CPW;
+    const int tstep = ntab / N1;
     c2 x[16];
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
@@ -594,7 +613,9 @@ struct Pass3 {
 #pragma unroll
       for (int q = 0; q < R1B; ++q) x[it * R1B + q] = y[q];
     }
+    pre();
     __syncthreads();                       // all bins read; the buffer becomes the exchange area
+    post();
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
       const int pp = j + R1B * it;
@@ -608,36 +629,57 @@ struct Pass3 {
       if (p > 0) x[p] = cmulc_b(x[p], twb[j * p * tstep]);
     }
     dftp<16, +1>(x);
+    float acc[16];
+    float2 totK = make_float2(0.f, 0.f), totV = make_float2(0.f, 0.f);
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
       const float2 t = pfma(x[p].i, x[p].i, pmul(x[p].r, x[p].r));
-      acc[p] += t.x + t.y;
+      acc[p] = t.x + t.y;
       totK = pfma(x[p].r, x[p].r, totK);
       totV = pfma(x[p].i, x[p].i, totV);
     }
-  }
-
-  __device__ static void finish(const Params &P, const Tile &tl, float (&acc)[16], float2 totK, float2 totV,
-                                double (*red)[4], int tid) {
-    const int N2 = P.N / N1;
-    const int cp = tid % CPW, j = tid / CPW;
     int prow = 0;
     RowReduce<16, CPW / 2>::run(acc, cp, prow);
+    const int gcol = tl.unit * P.UC + tl.cb * 2 * CPW;
+    const int head = gcol / P.head_dim, part = (gcol - head * P.head_dim) / (2 * CPW);
+    float *dstp = P.nparts > 1 ? P.partial + ((size_t)part * P.num_heads + head) * (size_t)P.N
+                               : P.scores + (long long)head * P.score_stride;
     if ((cp & (DUP - 1)) == 0) {
 #pragma unroll
       for (int i = 0; i < LEFT; ++i) {
         const int p = (j + R1B * (prow + i)) * N2 + tl.a;
-        P.scores[(long long)tl.unit * P.score_stride + perm_token(p, P.N)] = acc[i] * P.inv_scale;
+        __stcg(dstp + perm_token(p, P.N), acc[i] * P.inv_scale);
       }
     }
     const double dk = warp_sum_d((double)((totK.x + totK.y) * P.inv_scale));
     const double dv = warp_sum_d((double)((totV.x + totV.y) * P.inv_scale));
     if ((tid & 31) == 0) { red[0][tid >> 5] = dk; red[1][tid >> 5] = dv; }
-    __syncthreads();
+    __syncthreads();                       // partial scores of the tile are issued, warp sums are visible
     if (tid == 0) {
-      const size_t s = (size_t)tl.unit * P.n3t + tl.a;
+      const size_t s = (size_t)tl.unit * P.TPU + tl.idx;
       P.part_hi[2 * s] = (red[0][0] + red[0][1] + red[0][2] + red[0][3]) * (double)P.head_dim;   // d * sum Dev_k
       P.part_hi[2 * s + 1] = (red[1][0] + red[1][1] + red[1][2] + red[1][3]) * (double)P.head_dim;
+    }
+    if (P.nparts > 1) {
+      // the block that delivers the last partial of (head, n2) adds all of them in a fixed order
+      if (tid == 0) {
+        __threadfence();
+        unsigned *c = &P.sched->cnt3[head * N2 + tl.a];
+        const unsigned old = atomicAdd(c, 1u);
+        const int last = (old + 1u == (unsigned)P.nparts) ? 1 : 0;
+        if (last) *c = 0u;
+        *s_last = last;
+      }
+      __syncthreads();
+      if (*s_last) {
+        __threadfence();
+        for (int n1 = tid; n1 < N1; n1 += NT) {
+          const int tok = perm_token(n1 * N2 + tl.a, P.N);
+          float sum = 0.f;
+          for (int q = 0; q < P.nparts; ++q) sum += __ldcg(P.partial + ((size_t)q * P.num_heads + head) * (size_t)P.N + tok);
+          P.scores[(long long)head * P.score_stride + tok] = sum;
+        }
+      }
     }
   }
 };
@@ -646,128 +688,156 @@ struct Pass3 {
 template <int R1B, int R2B>
 struct Smem {
   static constexpr int N1 = 16 * R1B, N2 = 16 * R2B, NTAB = N1 > N2 ? N1 : N2, NAB = R2B + 16;
-  static constexpr size_t bytes = (size_t)2 * TILE4 * sizeof(float4) + NTAB * sizeof(float4) + N2 * sizeof(float2) +
+  static constexpr size_t bytes = (size_t)2 * BUF4 * sizeof(float4) + NTAB * sizeof(float4) + N2 * sizeof(float2) +
                                   2 * 2 * NAB * sizeof(float4) + 2 * 2 * sizeof(float2);
 };
 
+#ifndef FC_FUSED_MINB
+#define FC_FUSED_MINB 3
+#endif
 template <typename T, int R1B, int R2B>
-__global__ void __launch_bounds__(NT, 3) k_fused(const __grid_constant__ Params P) {
+__global__ void __launch_bounds__(NT, FC_FUSED_MINB) k_fused(const __grid_constant__ Params P) {
   using SM = Smem<R1B, R2B>;
   using P1 = Pass1<T, R1B>;
   using P2 = Pass2<R2B>;
   using P3 = Pass3<R1B>;
   constexpr int NTAB = SM::NTAB, N2 = SM::N2, NAB = SM::NAB;
   extern __shared__ float4 smem4[];
-  float4 *bufs = smem4;                                           // [2][TILE4]
-  float4 *twb = smem4 + 2 * TILE4;                                // [NTAB] exp(-2*pi*j*i/NTAB), broadcast
+  float4 *bufs = smem4;                                           // [2][BUF4]
+  float4 *twb = smem4 + 2 * BUF4;                                 // [NTAB] exp(-2*pi*j*i/NTAB), broadcast
   float2 *t2 = reinterpret_cast<float2 *>(twb + NTAB);            // [N2]   exp(-j*pi*k2/N2)
   float4 *ab = reinterpret_cast<float4 *>(t2 + N2);               // [2 buffers][2 halves][NAB]
   float2 *chf = reinterpret_cast<float2 *>(ab + 2 * 2 * NAB);     // [2 buffers][2 halves]
   __shared__ Tile desc[2];
   __shared__ double red[2][4];
-  __shared__ int s_ok;
+  __shared__ int s_ok, s_last;
   const int tid = threadIdx.x;
   Sched *sc = P.sched;
 
   for (int i = tid; i < NTAB; i += NT) twb[i] = bcast4(__ldg(P.master + (size_t)i * (P.master_len / NTAB)));
   for (int i = tid; i < N2; i += NT) t2[i] = __ldg(P.master + (size_t)i * (P.master_len / (2 * N2)));
 
+  auto issue = [&](const Tile &tl, int nb) {
+    float4 *dst = bufs + nb * BUF4;
+    if (tl.phase == PH_P1) P1::issue(P, tl, dst, tid);
+    else if (tl.phase == PH_P2) P2::issue(P, tl, dst, ab + nb * 2 * NAB, chf + nb * 2, tid);
+    else P3::issue(P, tl, dst, tid);
+    cp_async_commit();
+  };
+
+  // thread 0 keeps the stage walk and one tile index that was asked for but not yet looked at
   Walk walk = {0, 0u};
+  unsigned t_ahead = 0u;
   if (tid == 0) {
-    Tile first;
-    if (ld_acquire(&sc->abort_flag) != 0u) { first.phase = PH_NONE; first.unit = first.a = first.cb = first.ready = 0; }
-    else first = decode_tile(P, walk, atomicAdd(&sc->tile_counter, 1u));
+    const unsigned t0 = atomicAdd(&sc->tile_counter, 1u);
+    t_ahead = atomicAdd(&sc->tile_counter, 1u);
+    Tile first = decode_tile(P, walk, t0);
+    int ok = 1;
+    if (first.phase != PH_NONE) ok = wait_deps(P, first) ? 1 : 0;
     desc[0] = first;
+    s_ok = ok;
   }
   __syncthreads();
   Tile cur = desc[0];
+  Tile prev = cur;
+  bool have_prev = false, issued = false, finished = false;
   int b = 0;
-  bool issued = false;
-
-  while (cur.phase != PH_NONE) {
-    if (tid == 0) {
-      int ok = 1;
-      if (!issued) ok = wait_deps(P, cur) ? 1 : 0;
-      Tile nx;
-      nx.phase = PH_NONE; nx.unit = nx.a = nx.cb = nx.ready = 0;
-      if (ok && ld_acquire(&sc->abort_flag) == 0u) {
-        nx = decode_tile(P, walk, atomicAdd(&sc->tile_counter, 1u));
-        if (nx.phase != PH_NONE) nx.ready = deps_ok(P, nx) ? 1 : 0;
-      }
-      desc[b ^ 1] = nx;
-      s_ok = ok;
-    }
-    __syncthreads();
-    if (!s_ok) break;
-    const Tile nxt = desc[b ^ 1];
-    bool nxt_issued = false;
-
-    // loads of the tile after this one go to the buffer this tile does not end in
-    auto prefetch = [&](int nb) {
-      if (nxt.phase != PH_NONE && nxt.ready) {
-        float4 *dst = bufs + nb * TILE4;
-        if (nxt.phase == PH_P1) P1::issue(P, nxt, dst, tid);
-        else if (nxt.phase == PH_P2) P2::issue(P, nxt, dst, ab + nb * 2 * NAB, chf + nb * 2, tid);
-        else P3::issue(P, nxt, 0, dst, tid);
-        cp_async_commit();
-        nxt_issued = true;
-      }
-    };
-
-    if (cur.phase == PH_P3) {
-      const int nsl = P.head_dim / (2 * P3::CPW);
-      if (!issued) { P3::issue(P, cur, 0, bufs + b * TILE4, tid); cp_async_commit(); }
-      float acc[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) acc[i] = 0.f;
-      float2 totK = make_float2(0.f, 0.f), totV = make_float2(0.f, 0.f);
-      const int cp = tid % P3::CPW, j = tid / P3::CPW;
-      for (int s = 0; s < nsl; ++s) {
-        bool more = false;
-        if (s + 1 < nsl) { P3::issue(P, cur, s + 1, bufs + (b ^ 1) * TILE4, tid); cp_async_commit(); more = true; }
-        else { prefetch(b ^ 1); more = nxt_issued; }
-        if (more) cp_async_wait<1>(); else cp_async_wait<0>();
+  unsigned long long st_tiles = 0, st_slow = 0, st_ph[4] = {0, 0, 0, 0}, st_wait = 0;
+  const long long clk_begin = clock64();
+  if (cur.phase != PH_NONE && s_ok) {
+    issue(cur, 0);
+    issued = true;
+    while (true) {
+      const long long clk_top = clock64();
+      if (!issued) ++st_slow;
+      if (!issued) {                       // its dependencies were not finished when thread 0 looked ahead
+        __syncthreads();                   // the previous tile is stored: report it first, this tile may wait for it
+        if (tid == 0) {
+          if (have_prev) signal_done(P, prev);
+          s_ok = wait_deps(P, cur) ? 1 : 0;
+        }
+        have_prev = false;
         __syncthreads();
-        P3::slice(bufs + b * TILE4, twb, NTAB / P3::N1, cp, j, acc, totK, totV);
-        b ^= 1;
+        if (!s_ok) break;
+        issue(cur, b);
       }
-      P3::finish(P, cur, acc, totK, totV, red, tid);
-    } else {
-      if (cur.phase == PH_P1) {
-        if (!issued) { P1::issue(P, cur, bufs + b * TILE4, tid); cp_async_commit(); }
-      } else {
-        if (!issued) { P2::issue(P, cur, bufs + b * TILE4, ab + b * 2 * NAB, chf + b * 2, tid); cp_async_commit(); }
+      Tile nx;
+      nx.phase = PH_NONE; nx.unit = nx.a = nx.cb = nx.idx = nx.ready = 0;
+      unsigned depv = 0u;
+      if (tid == 0) {
+        nx = decode_tile(P, walk, t_ahead);
+        t_ahead = atomicAdd(&sc->tile_counter, 1u);       // answer is needed one tile from now
+        const unsigned *dc = dep_counter(P, nx);
+        depv = dc != nullptr ? ld_acquire(dc) : (unsigned)P.TPU;   // looked at in pre()
       }
-      prefetch(b ^ 1);
-      if (nxt_issued) cp_async_wait<1>(); else cp_async_wait<0>();
-      __syncthreads();
-      if (cur.phase == PH_P1) P1::compute(P, cur, bufs + b * TILE4, twb, NTAB, red, tid);
-      else P2::compute(P, cur, bufs + b * TILE4, twb, NTAB, t2, ab + b * 2 * NAB, chf + b * 2, tid);
+      cp_async_wait<0>();
+      __syncthreads();                     // this tile's data is in shared memory; the previous tile is stored
+      const long long clk_sig = clock64();
+      if (tid == 0 && have_prev) signal_done(P, prev);
+      const long long clk_data = clock64();
+      st_ph[0] += (unsigned long long)(clk_data - clk_sig);
+      Tile nxt;
+      nxt.phase = PH_NONE; nxt.unit = nxt.a = nxt.cb = nxt.idx = nxt.ready = 0;
+      bool nxt_issued = false;
+      auto pre = [&]() {
+        if (tid == 0) {
+          nx.ready = depv >= (unsigned)P.TPU ? 1 : 0;
+          desc[b ^ 1] = nx;
+        }
+      };
+      auto post = [&]() {
+        nxt = desc[b ^ 1];
+        if (nxt.phase != PH_NONE && nxt.ready) { issue(nxt, b ^ 1); nxt_issued = true; }
+      };
+      float4 *buf = bufs + b * BUF4;
+      if (cur.phase == PH_P1) P1::compute(P, cur, buf, twb, NTAB, red, tid, pre, post);
+      else if (cur.phase == PH_P2) P2::compute(P, cur, buf, twb, NTAB, t2, ab + b * 2 * NAB, chf + b * 2, tid, pre, post);
+      else P3::compute(P, cur, buf, twb, NTAB, red, &s_last, tid, pre, post);
+      {
+        const long long clk_end = clock64();
+        ++st_tiles;
+        st_wait += (unsigned long long)(clk_data - clk_top);
+        st_ph[cur.phase] += (unsigned long long)(clk_end - clk_data);
+      }
+      prev = cur;
+      have_prev = true;
+      cur = nxt;
+      issued = nxt_issued;
       b ^= 1;
+      if (cur.phase == PH_NONE) { finished = true; break; }
     }
-    __syncthreads();                       // every store of the tile has been issued
-    if (tid == 0) signal_done(P, cur);
-    cur = nxt;
-    issued = nxt_issued;
+  }
+  cp_async_wait<0>();
+  __syncthreads();
+  if (tid == 0 && finished && have_prev) signal_done(P, prev);
+  if (tid == 0) {
+    atomicAdd(&sc->stats[0], st_tiles);
+    atomicAdd(&sc->stats[1], st_slow);
+    atomicAdd(&sc->stats[2], st_ph[0]);      // cycles thread 0 spent reporting finished tiles
+    atomicAdd(&sc->stats[3], st_ph[PH_P1]);
+    atomicAdd(&sc->stats[4], st_ph[PH_P2]);
+    atomicAdd(&sc->stats[5], st_ph[PH_P3]);
+    atomicAdd(&sc->stats[6], st_wait);
+    atomicAdd(&sc->stats[7], (unsigned long long)(clock64() - clk_begin));
   }
 
   // ---- exit: the last block to leave adds up the energy partial sums in a fixed order and
   // returns the scheduler state to all-zero
-  cp_async_wait<0>();
-  __syncthreads();
   if (tid == 0) {
     __threadfence();
-    const unsigned prev = atomicAdd(&sc->exit_counter, 1u);
-    s_ok = (prev + 1u == gridDim.x) ? 1 : 0;
+    const unsigned old = atomicAdd(&sc->exit_counter, 1u);
+    s_ok = (old + 1u == gridDim.x) ? 1 : 0;
   }
   __syncthreads();
   if (!s_ok) return;
   __threadfence();
   double *redd = reinterpret_cast<double *>(smem4);        // [4][NT]
-  const int n_tot = P.U * P.n1t, n_hi = P.num_heads * P.n3t;
+  const int n_part = P.U * P.TPU;
   double a0 = 0, a1 = 0, b0 = 0, b1 = 0;
-  for (int i = tid; i < n_tot; i += NT) { a0 += __ldcg(P.part_tot + 2 * i); a1 += __ldcg(P.part_tot + 2 * i + 1); }
-  for (int i = tid; i < n_hi; i += NT) { b0 += __ldcg(P.part_hi + 2 * i); b1 += __ldcg(P.part_hi + 2 * i + 1); }
+  for (int i = tid; i < n_part; i += NT) {
+    a0 += __ldcg(P.part_tot + 2 * i); a1 += __ldcg(P.part_tot + 2 * i + 1);
+    b0 += __ldcg(P.part_hi + 2 * i);  b1 += __ldcg(P.part_hi + 2 * i + 1);
+  }
   redd[tid] = b0; redd[NT + tid] = a0; redd[2 * NT + tid] = b1; redd[3 * NT + tid] = a1;
   __syncthreads();
   for (int st = NT / 2; st > 0; st >>= 1) {
@@ -776,7 +846,9 @@ __global__ void __launch_bounds__(NT, 3) k_fused(const __grid_constant__ Params 
     __syncthreads();
   }
   if (tid < 4) P.energy[tid] = redd[tid * NT];
-  for (int i = tid; i < 1024; i += NT) { sc->done1[i] = 0u; sc->done2[i] = 0u; sc->done3[i] = 0u; }
+  for (int i = tid; i < P.U; i += NT) { sc->done1[i] = 0u; sc->done2[i] = 0u; sc->done3[i] = 0u; }
+  const int ncnt = P.nparts > 1 ? P.num_heads * (P.N / (16 * R1B)) : 0;
+  for (int i = tid; i < ncnt; i += NT) sc->cnt3[i] = 0u;
   if (tid == 0) { sc->tile_counter = 0u; sc->exit_counter = 0u; sc->abort_flag = 0u; }
 }
 
