@@ -90,9 +90,17 @@ uint64_t fc_launch_count(const fc_handle *h);
 fc_status fc_profile_begin(fc_handle *h, int32_t kernel_class, int32_t max_launches);
 fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *launches);
 
+/* Chooses how power-of-two sequences of 4096..65536 tokens are transformed: enabled = 0 (default)
+ * runs the three passes as separate launches per head group, enabled = 1 runs ONE persistent
+ * kernel per (layer, sequence) that hands out tiles of all three passes in dependency order;
+ * stage_lag (1..4) is the distance, in units of about 8 MB of intermediate, between the passes
+ * of a unit.  Same results up to fp32 rounding; affects speed and workspace size only, so call
+ * it before fc_score_workspace_bytes. */
+fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_lag);
+
 /* Running totals of the fused transform kernel since fc_create (diagnostic; synchronises the
  * device): out = { tiles processed, tiles whose inputs were not finished when they were looked
- * at one tile ahead, cycles spent reporting finished tiles, clock cycles (thread 0 of every block, summed) inside
+ * when the scheduler warp first looked, unused, clock cycles (thread 0 of every block, summed) inside
  * pass-1, pass-2 and pass-3 tiles, cycles waiting for tile data, cycles inside the tile loop }. */
 fc_status fc_fused_stats(fc_handle *h, uint64_t out[8]);
 

@@ -23,7 +23,7 @@ _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
     "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count",
-    "fc_set_group_bytes", "fc_fused_stats", "fc_profile_begin", "fc_profile_end", "fc_describe_plan",
+    "fc_set_group_bytes", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact",
     "fc_static_scratch_bytes", "fc_score_layer_static",
@@ -63,6 +63,8 @@ def _load() -> ctypes.CDLL:
     lib.fc_launch_count.restype = c_uint64
     lib.fc_set_group_bytes.argtypes = [c_void_p, c_size_t]
     lib.fc_set_group_bytes.restype = c_int
+    lib.fc_set_fused.argtypes = [c_void_p, c_int32, c_int32]
+    lib.fc_set_fused.restype = c_int
     lib.fc_fused_stats.argtypes = [c_void_p, POINTER(c_uint64)]
     lib.fc_fused_stats.restype = c_int
     lib.fc_profile_begin.argtypes = [c_void_p, c_int32, c_int32]
@@ -150,10 +152,14 @@ def fc_set_group_bytes(handle, nbytes: int) -> None:
     _check(_lib.fc_set_group_bytes(handle, int(nbytes)), "fc_set_group_bytes")
 
 
+def fc_set_fused(handle, enabled: bool, stage_lag: int = 2) -> None:
+    _check(_lib.fc_set_fused(handle, 1 if enabled else 0, int(stage_lag)), "fc_set_fused")
+
+
 def fc_fused_stats(handle) -> dict:
     out = (c_uint64 * 8)()
     _check(_lib.fc_fused_stats(handle, out), "fc_fused_stats")
-    keys = ("tiles", "late_tiles", "cycles_signal", "cycles_pass1", "cycles_pass2", "cycles_pass3",
+    keys = ("tiles", "late_tiles", "unused", "cycles_pass1", "cycles_pass2", "cycles_pass3",
             "cycles_data_wait", "cycles_loop")
     return {k: int(v) for k, v in zip(keys, out)}
 

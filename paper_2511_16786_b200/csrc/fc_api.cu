@@ -178,6 +178,13 @@ extern "C" fc_status fc_fused_stats(fc_handle *h, uint64_t out[8]) {
 
 extern "C" uint64_t fc_launch_count(const fc_handle *h) { return h ? (uint64_t)h->launches : 0; }
 
+extern "C" fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_lag) {
+  if (!h || stage_lag < 1 || stage_lag > 4) return FC_ERR_INVALID_ARG;
+  h->fused_enabled = enabled ? 1 : 0;
+  h->fused_lag = stage_lag;
+  return FC_OK;
+}
+
 extern "C" fc_status fc_set_group_bytes(fc_handle *h, size_t bytes) {
   if (!h || bytes == 0) return FC_ERR_INVALID_ARG;
   h->group_bytes = bytes;

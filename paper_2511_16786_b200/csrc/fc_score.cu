@@ -706,7 +706,7 @@ fc_status launch_fused_impl(fc_handle *h, cudaStream_t st, const fused::Params &
   static int blocks_per_sm = 0;                     // per instantiation; the answer does not change
   if (blocks_per_sm == 0) {
     int n = 0;
-    FC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, fused::NT, sm));
+    FC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, fused::NTH, sm));
     if (n < 1) return FC_ERR_INTERNAL;
     blocks_per_sm = n;
   }
@@ -715,7 +715,7 @@ fc_status launch_fused_impl(fc_handle *h, cudaStream_t st, const fused::Params &
   unsigned grid = (unsigned)(h->num_sms * bps);
   if (grid > P.total_tiles) grid = P.total_tiles;
   ProfScope ps(h, FC_K_FUSED, st);
-  kern<<<grid, fused::NT, sm, st>>>(P);
+  kern<<<grid, fused::NTH, sm, st>>>(P);
   return fc_after_launch(h);
 }
 

@@ -226,6 +226,9 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
+// barrier of the four compute warps (the scheduler warp never joins it)
+__device__ __forceinline__ void bar_compute() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
+
 __device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(v) : "l"(p) : "memory");
@@ -337,13 +340,12 @@ __device__ __forceinline__ float2 *slot_base(const Params &P, int unit) {
 
 // ------------------------------------------------------------------ pass 1
 // Tile (unit, n2, cb): DFT over n1 of 2*CPW channels.  Thread (cp = tid % CPW, j = tid / CPW).
-// In every pass `pre` runs just before the first block barrier of the tile and `post` just after it.
 template <typename T, int R1B>
 struct Pass1 {
   static constexpr int N1 = 16 * R1B, CPW = NT / R1B, IT = 16 / R1B, ES = Pair<T>::ES;
   static constexpr int ROWB = 2 * CPW * ES, CPR = ROWB / 16;   // bytes and 16-byte chunks per input row slice
 
-  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, int tid) {
+  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, int lane) {
     const int N2 = P.N / N1;
     const int gcol = tl.unit * P.UC + tl.cb * 2 * CPW;
     const int head = gcol / P.head_dim, c = gcol - head * P.head_dim;
@@ -351,8 +353,8 @@ struct Pass1 {
     const char *kb = static_cast<const char *>(P.k) + hoff;
     const char *vb = static_cast<const char *>(P.v) + hoff;
     char *dst0 = reinterpret_cast<char *>(buf);
-#pragma unroll
-    for (int idx = tid; idx < 2 * N1 * CPR; idx += NT) {
+#pragma unroll 8
+    for (int idx = lane; idx < 2 * N1 * CPR; idx += 32) {
       const int m = idx / (N1 * CPR), rem = idx - m * (N1 * CPR);
       const int row = rem / CPR, q = rem - row * CPR;
       const int tok = perm_token(row * N2 + tl.a, P.N);
@@ -361,9 +363,8 @@ struct Pass1 {
     }
   }
 
-  template <class Pre, class Post>
   __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
-                                 double (*red)[4], int tid, Pre pre, Post post) {
+                                 double (*red)[4], int tid) {
     const int N2 = P.N / N1;
     const int cp = tid % CPW, j = tid / CPW;
     const char *in = reinterpret_cast<const char *>(buf);
@@ -381,9 +382,7 @@ struct Pass1 {
       const double a = warp_sum_d((double)(aK.x + aK.y)), b = warp_sum_d((double)(aV.x + aV.y));
       if ((tid & 31) == 0) { red[0][tid >> 5] = a; red[1][tid >> 5] = b; }
     }
-    pre();
-    __syncthreads();                       // every thread has its inputs; the buffer becomes the exchange area
-    post();
+    bar_compute();                         // every thread has its inputs; the buffer becomes the exchange area
     dftp<16, -1>(x);
     const int tstep = ntab / N1;
 #pragma unroll
@@ -391,7 +390,7 @@ struct Pass1 {
       if (p > 0) x[p] = cmul_b(x[p], twb[j * p * tstep]);
       buf[(j + R1B * p) * CPW + cp] = to4(x[p]);
     }
-    __syncthreads();
+    bar_compute();
     float2 *slot = slot_base(P, tl.unit);
     const int col = tl.cb * 2 * CPW + 2 * cp;
 #pragma unroll
@@ -426,13 +425,13 @@ struct Pass2 {
   static constexpr int N2 = 16 * R2B, CP = NT / (2 * R2B), IT = 16 / R2B, NAB = R2B + 16;
   static constexpr int PAD = CP < 8 ? 4 : 0, HALF = N2 * CP + PAD;
 
-  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, float4 *ab, float2 *chf, int tid) {
+  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, float4 *ab, float2 *chf, int lane) {
     const int N1 = P.N / N2;
     const int k1a = tl.a, k1b = tl.a == 0 ? N1 / 2 : N1 - tl.a;
     const float2 *slot = slot_base(P, tl.unit);
     const int col = tl.cb * 2 * CP;
-#pragma unroll
-    for (int idx = tid; idx < 2 * N2 * CP; idx += NT) {
+#pragma unroll 8
+    for (int idx = lane; idx < 2 * N2 * CP; idx += 32) {
       const int hf = idx / (N2 * CP), rem = idx - hf * (N2 * CP);
       const int n2 = rem / CP, cpi = rem - n2 * CP;
       const int k1 = hf ? k1b : k1a;
@@ -440,21 +439,22 @@ struct Pass2 {
     }
     // per-tile twiddle factors: w_N^(k1*n2) = A[j] * B[p] for n2 = j + R2B*p
     const int ms = P.master_len / P.N;
-    if (tid < 2 * NAB) {
-      const int hf = tid / NAB, r = tid - hf * NAB;
-      const int k1 = hf ? k1b : k1a;
-      const int m = (r < R2B ? k1 * r : k1 * R2B * (r - R2B)) & (P.N - 1);
-      ab[hf * NAB + r] = bcast4(__ldg(P.master + (size_t)m * ms));
-    } else if (tid < 2 * NAB + 2) {
-      const int hf = tid - 2 * NAB;
-      const int k1 = hf ? k1b : k1a;
-      chf[hf] = __ldg(P.master + (size_t)k1 * (P.master_len / (2 * P.N)));      // exp(-j*pi*k1/N)
+    for (int e = lane; e < 2 * NAB + 2; e += 32) {
+      if (e < 2 * NAB) {
+        const int hf = e / NAB, r = e - hf * NAB;
+        const int k1 = hf ? k1b : k1a;
+        const int m = (r < R2B ? k1 * r : k1 * R2B * (r - R2B)) & (P.N - 1);
+        ab[hf * NAB + r] = bcast4(__ldg(P.master + (size_t)m * ms));
+      } else {
+        const int hf = e - 2 * NAB;
+        const int k1 = hf ? k1b : k1a;
+        chf[hf] = __ldg(P.master + (size_t)k1 * (P.master_len / (2 * P.N)));      // exp(-j*pi*k1/N)
+      }
     }
   }
 
-  template <class Pre, class Post>
   __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
-                                 const float2 *t2, const float4 *ab, const float2 *chf, int tid, Pre pre, Post post) {
+                                 const float2 *t2, const float4 *ab, const float2 *chf, int tid) {
     const int N1 = P.N / N2, N = P.N;
     const int cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
     const bool self = tl.a == 0;
@@ -476,9 +476,7 @@ struct Pass2 {
       if (p > 0) x[p] = cmul_b(x[p], twb[j * p * tstep]);
       Sh[(j + R2B * p) * CP + cp] = to4(x[p]);        // same cell this thread read: no barrier needed before
     }
-    pre();
-    __syncthreads();
-    post();
+    bar_compute();
     // second forward stage; registers keep bin k2 = pp + 16*q at index it*R2B + q, shared memory the same
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
@@ -493,7 +491,7 @@ struct Pass2 {
         Sh[(q + R2B * pp) * CP + cp] = to4(y[q]);
       }
     }
-    __syncthreads();                       // full spectra of both halves are in shared memory
+    bar_compute();                       // full spectra of both halves are in shared memory
     const float2 ch = chf[hf];
     const float2 half2 = bc(0.5f);
 #pragma unroll
@@ -530,14 +528,14 @@ struct Pass2 {
 #pragma unroll
       for (int q = 0; q < R2B; ++q) x[it * R2B + q] = y[q];
     }
-    __syncthreads();                       // all partner reads are done
+    bar_compute();                       // all partner reads are done
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
       const int pp = j + R2B * it;
 #pragma unroll
       for (int q = 0; q < R2B; ++q) Sh[(q + R2B * pp) * CP + cp] = to4(x[it * R2B + q]);
     }
-    __syncthreads();
+    bar_compute();
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
       x[p] = from4(Sh[(j + R2B * p) * CP + cp]);
@@ -585,20 +583,19 @@ struct Pass3 {
   static constexpr int LEFT = CPW >= 16 ? 1 : 16 / CPW;       // row sums a lane ends up with
   static constexpr int DUP = CPW > 16 ? CPW / 16 : 1;         // lanes that end up with the same row sum
 
-  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, int tid) {
+  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, int lane) {
     const int N2 = P.N / N1;
     const float2 *slot = slot_base(P, tl.unit);
     const int col = tl.cb * 2 * CPW;
-#pragma unroll
-    for (int idx = tid; idx < N1 * CPW; idx += NT) {
+#pragma unroll 8
+    for (int idx = lane; idx < N1 * CPW; idx += 32) {
       const int k1 = idx / CPW, cpi = idx - k1 * CPW;
       cp_async16(buf + idx, slot + ((size_t)k1 * N2 + tl.a) * P.UC + col + 2 * cpi);
     }
   }
 
-  template <class Pre, class Post>
   __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
-                                 double (*red)[4], int *s_last, int tid, Pre pre, Post post) {
+                                 double (*red)[4], int tid) {
     const int N2 = P.N / N1;
     const int cp = tid % CPW, j = tid / CPW;
     const int tstep = ntab / N1;
@@ -613,16 +610,14 @@ struct Pass3 {
 #pragma unroll
       for (int q = 0; q < R1B; ++q) x[it * R1B + q] = y[q];
     }
-    pre();
-    __syncthreads();                       // all bins read; the buffer becomes the exchange area
-    post();
+    bar_compute();                         // all bins read; the buffer becomes the exchange area
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
       const int pp = j + R1B * it;
 #pragma unroll
       for (int q = 0; q < R1B; ++q) buf[(q + R1B * pp) * CPW + cp] = to4(x[it * R1B + q]);
     }
-    __syncthreads();
+    bar_compute();
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
       x[p] = from4(buf[(j + R1B * p) * CPW + cp]);
@@ -654,37 +649,52 @@ struct Pass3 {
     const double dk = warp_sum_d((double)((totK.x + totK.y) * P.inv_scale));
     const double dv = warp_sum_d((double)((totV.x + totV.y) * P.inv_scale));
     if ((tid & 31) == 0) { red[0][tid >> 5] = dk; red[1][tid >> 5] = dv; }
-    __syncthreads();                       // partial scores of the tile are issued, warp sums are visible
+    bar_compute();                       // partial scores of the tile are issued, warp sums are visible
     if (tid == 0) {
       const size_t s = (size_t)tl.unit * P.TPU + tl.idx;
       P.part_hi[2 * s] = (red[0][0] + red[0][1] + red[0][2] + red[0][3]) * (double)P.head_dim;   // d * sum Dev_k
       P.part_hi[2 * s + 1] = (red[1][0] + red[1][1] + red[1][2] + red[1][3]) * (double)P.head_dim;
     }
-    if (P.nparts > 1) {
-      // the block that delivers the last partial of (head, n2) adds all of them in a fixed order
-      if (tid == 0) {
-        __threadfence();
-        unsigned *c = &P.sched->cnt3[head * N2 + tl.a];
-        const unsigned old = atomicAdd(c, 1u);
-        const int last = (old + 1u == (unsigned)P.nparts) ? 1 : 0;
-        if (last) *c = 0u;
-        *s_last = last;
-      }
-      __syncthreads();
-      if (*s_last) {
-        __threadfence();
-        for (int n1 = tid; n1 < N1; n1 += NT) {
-          const int tok = perm_token(n1 * N2 + tl.a, P.N);
-          float sum = 0.f;
-          for (int q = 0; q < P.nparts; ++q) sum += __ldcg(P.partial + ((size_t)q * P.num_heads + head) * (size_t)P.N + tok);
-          P.scores[(long long)head * P.score_stride + tok] = sum;
-        }
-      }
-    }
   }
 };
 
+// ------------------------------------------------------------------ mbarrier helpers
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"((unsigned)__cvta_generic_to_shared(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
+  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}\n"
+               ::"r"((unsigned)__cvta_generic_to_shared(bar)) : "memory");
+}
+// arrives once all cp.async copies this thread has issued so far have landed (counted in the init value)
+__device__ __forceinline__ void mbar_arrive_after_copies(unsigned long long *bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n"
+               ::"r"((unsigned)__cvta_generic_to_shared(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(unsigned long long *bar, unsigned parity) {
+  unsigned ok;
+  asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"((unsigned)__cvta_generic_to_shared(bar)), "r"(parity) : "memory");
+  return ok != 0u;
+}
+// Bounded wait for a phase of an mbarrier.  false: gave up (and said so), or another block gave up.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, const Params &P) {
+  for (unsigned it = 0; it < P.spin_limit; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    if ((it & 63u) == 63u && ld_acquire(&P.sched->abort_flag) != 0u) return false;
+    __nanosleep(32);
+  }
+  atomicExch(&P.sched->abort_flag, 1u);
+  atomicOr(P.status, FC_DEV_FLAG_TIMEOUT);
+  return false;
+}
+
 // ------------------------------------------------------------------ the kernel
+// Block = 4 compute warps + 1 scheduler warp.  The scheduler warp takes tile numbers, waits for
+// the tiles they depend on, fills one of two shared-memory buffers with cp.async and reports
+// finished tiles; the compute warps only ever wait for a full buffer.
+constexpr int NTH = NT + 32;
+
 template <int R1B, int R2B>
 struct Smem {
   static constexpr int N1 = 16 * R1B, N2 = 16 * R2B, NTAB = N1 > N2 ? N1 : N2, NAB = R2B + 16;
@@ -692,11 +702,40 @@ struct Smem {
                                   2 * 2 * NAB * sizeof(float4) + 2 * 2 * sizeof(float2);
 };
 
+// Scheduler warp: report a finished tile (all 32 lanes call it).
+template <int R1B>
+__device__ __forceinline__ void report_tile(const Params &P, const Tile &tl, int lane) {
+  constexpr int N1 = 16 * R1B, CPW = NT / R1B;
+  if (lane == 0) signal_done(P, tl);
+  if (tl.phase == PH_P3 && P.nparts > 1) {
+    // the block that delivers the last partial score of (head, n2) adds all of them in a fixed order
+    const int N2 = P.N / N1;
+    const int gcol = tl.unit * P.UC + tl.cb * 2 * CPW;
+    const int head = gcol / P.head_dim;
+    unsigned old = 0u;
+    if (lane == 0) {
+      unsigned *c = &P.sched->cnt3[head * N2 + tl.a];
+      old = atomicAdd(c, 1u);            // after the fence in signal_done
+      if (old + 1u == (unsigned)P.nparts) *c = 0u;
+    }
+    old = __shfl_sync(0xffffffffu, old, 0);
+    if (old + 1u == (unsigned)P.nparts) {
+      __threadfence();
+      for (int n1 = lane; n1 < N1; n1 += 32) {
+        const int tok = perm_token(n1 * N2 + tl.a, P.N);
+        float sum = 0.f;
+        for (int q = 0; q < P.nparts; ++q) sum += __ldcg(P.partial + ((size_t)q * P.num_heads + head) * (size_t)P.N + tok);
+        P.scores[(long long)head * P.score_stride + tok] = sum;
+      }
+    }
+  }
+}
+
 #ifndef FC_FUSED_MINB
 #define FC_FUSED_MINB 3
 #endif
 template <typename T, int R1B, int R2B>
-__global__ void __launch_bounds__(NT, FC_FUSED_MINB) k_fused(const __grid_constant__ Params P) {
+__global__ void __launch_bounds__(NTH, FC_FUSED_MINB) k_fused(const __grid_constant__ Params P) {
   using SM = Smem<R1B, R2B>;
   using P1 = Pass1<T, R1B>;
   using P2 = Pass2<R2B>;
@@ -709,136 +748,151 @@ __global__ void __launch_bounds__(NT, FC_FUSED_MINB) k_fused(const __grid_consta
   float4 *ab = reinterpret_cast<float4 *>(t2 + N2);               // [2 buffers][2 halves][NAB]
   float2 *chf = reinterpret_cast<float2 *>(ab + 2 * 2 * NAB);     // [2 buffers][2 halves]
   __shared__ Tile desc[2];
-  __shared__ double red[2][4];
-  __shared__ int s_ok, s_last;
-  const int tid = threadIdx.x;
+  __shared__ unsigned long long full[2], done[2];
+  __shared__ double red[2][2][4];          // per buffer: a warp may enter the next tile while thread 0 still adds these up
+  __shared__ int s_last;
+  const int tid = threadIdx.x, lane = tid & 31;
   Sched *sc = P.sched;
 
-  for (int i = tid; i < NTAB; i += NT) twb[i] = bcast4(__ldg(P.master + (size_t)i * (P.master_len / NTAB)));
-  for (int i = tid; i < N2; i += NT) t2[i] = __ldg(P.master + (size_t)i * (P.master_len / (2 * N2)));
-
-  auto issue = [&](const Tile &tl, int nb) {
-    float4 *dst = bufs + nb * BUF4;
-    if (tl.phase == PH_P1) P1::issue(P, tl, dst, tid);
-    else if (tl.phase == PH_P2) P2::issue(P, tl, dst, ab + nb * 2 * NAB, chf + nb * 2, tid);
-    else P3::issue(P, tl, dst, tid);
-    cp_async_commit();
-  };
-
-  // thread 0 keeps the stage walk and one tile index that was asked for but not yet looked at
-  Walk walk = {0, 0u};
-  unsigned t_ahead = 0u;
+  for (int i = tid; i < NTAB; i += NTH) twb[i] = bcast4(__ldg(P.master + (size_t)i * (P.master_len / NTAB)));
+  for (int i = tid; i < N2; i += NTH) t2[i] = __ldg(P.master + (size_t)i * (P.master_len / (2 * N2)));
   if (tid == 0) {
-    const unsigned t0 = atomicAdd(&sc->tile_counter, 1u);
-    t_ahead = atomicAdd(&sc->tile_counter, 1u);
-    Tile first = decode_tile(P, walk, t0);
-    int ok = 1;
-    if (first.phase != PH_NONE) ok = wait_deps(P, first) ? 1 : 0;
-    desc[0] = first;
-    s_ok = ok;
+    mbar_init(&full[0], 64u); mbar_init(&full[1], 64u);     // per lane: one arrival after its copies, one plain
+    mbar_init(&done[0], (unsigned)NT); mbar_init(&done[1], (unsigned)NT);
   }
   __syncthreads();
-  Tile cur = desc[0];
-  Tile prev = cur;
-  bool have_prev = false, issued = false, finished = false;
-  int b = 0;
-  unsigned long long st_tiles = 0, st_slow = 0, st_ph[4] = {0, 0, 0, 0}, st_wait = 0;
-  const long long clk_begin = clock64();
-  if (cur.phase != PH_NONE && s_ok) {
-    issue(cur, 0);
-    issued = true;
-    while (true) {
-      const long long clk_top = clock64();
-      if (!issued) ++st_slow;
-      if (!issued) {                       // its dependencies were not finished when thread 0 looked ahead
-        __syncthreads();                   // the previous tile is stored: report it first, this tile may wait for it
-        if (tid == 0) {
-          if (have_prev) signal_done(P, prev);
-          s_ok = wait_deps(P, cur) ? 1 : 0;
-        }
-        have_prev = false;
-        __syncthreads();
-        if (!s_ok) break;
-        issue(cur, b);
+
+  if (tid >= NT) {
+    // ------------------------------------------------------------ scheduler warp
+    Walk walk = {0, 0u};
+    unsigned t_next = 0u;
+    if (lane == 0) t_next = atomicAdd(&sc->tile_counter, 1u);
+    Tile held[2];
+    unsigned held_k[2] = {0u, 0u};
+    bool live[2] = {false, false};
+    unsigned long long n_tiles = 0, n_late = 0;
+    bool ok = true;
+    unsigned k = 0;
+    for (;; ++k) {
+      const int b = (int)(k & 1u);
+      if (live[b]) {                       // the tile that used this buffer two steps ago
+        if (!mbar_wait(&done[b], (held_k[b] >> 1) & 1u, P)) { ok = false; break; }
+        report_tile<R1B>(P, held[b], lane);
+        live[b] = false;
       }
-      Tile nx;
-      nx.phase = PH_NONE; nx.unit = nx.a = nx.cb = nx.idx = nx.ready = 0;
-      unsigned depv = 0u;
-      if (tid == 0) {
-        nx = decode_tile(P, walk, t_ahead);
-        t_ahead = atomicAdd(&sc->tile_counter, 1u);       // answer is needed one tile from now
-        const unsigned *dc = dep_counter(P, nx);
-        depv = dc != nullptr ? ld_acquire(dc) : (unsigned)P.TPU;   // looked at in pre()
-      }
-      cp_async_wait<0>();
-      __syncthreads();                     // this tile's data is in shared memory; the previous tile is stored
-      const long long clk_sig = clock64();
-      if (tid == 0 && have_prev) signal_done(P, prev);
-      const long long clk_data = clock64();
-      st_ph[0] += (unsigned long long)(clk_data - clk_sig);
-      Tile nxt;
-      nxt.phase = PH_NONE; nxt.unit = nxt.a = nxt.cb = nxt.idx = nxt.ready = 0;
-      bool nxt_issued = false;
-      auto pre = [&]() {
-        if (tid == 0) {
-          nx.ready = depv >= (unsigned)P.TPU ? 1 : 0;
-          desc[b ^ 1] = nx;
+      const unsigned t = __shfl_sync(0xffffffffu, t_next, 0);
+      const Tile tl = decode_tile(P, walk, t);
+      if (tl.phase == PH_NONE) break;
+      if (lane == 0) t_next = atomicAdd(&sc->tile_counter, 1u);      // answer is needed one tile from now
+      const unsigned *dc = dep_counter(P, tl);
+      if (dc != nullptr) {
+        unsigned it = 0;
+        while (true) {
+          unsigned v = lane == 0 ? ld_acquire(dc) : 0u;
+          v = __shfl_sync(0xffffffffu, v, 0);
+          if (v >= (unsigned)P.TPU) break;
+          if (it == 0) ++n_late;
+          // the tile in the other buffer may be what somebody (even this tile) is waiting for
+          if (live[b ^ 1] && mbar_test(&done[b ^ 1], (held_k[b ^ 1] >> 1) & 1u)) {
+            report_tile<R1B>(P, held[b ^ 1], lane);
+            live[b ^ 1] = false;
+          }
+          unsigned stop = 0u;
+          if (lane == 0) {
+            if (++it > P.spin_limit) { atomicExch(&sc->abort_flag, 1u); atomicOr(P.status, FC_DEV_FLAG_TIMEOUT); stop = 1u; }
+            else if ((it & 15u) == 15u && ld_acquire(&sc->abort_flag) != 0u) stop = 1u;
+          }
+          stop = __shfl_sync(0xffffffffu, stop, 0);
+          if (stop) { ok = false; break; }
+          __nanosleep(64);
         }
-      };
-      auto post = [&]() {
-        nxt = desc[b ^ 1];
-        if (nxt.phase != PH_NONE && nxt.ready) { issue(nxt, b ^ 1); nxt_issued = true; }
-      };
+        if (!ok) break;
+      }
+      float4 *dst = bufs + b * BUF4;
+      if (lane == 0) desc[b] = tl;
+      if (tl.phase == PH_P1) P1::issue(P, tl, dst, lane);
+      else if (tl.phase == PH_P2) P2::issue(P, tl, dst, ab + b * 2 * NAB, chf + b * 2, lane);
+      else P3::issue(P, tl, dst, lane);
+      __syncwarp();
+      __threadfence_block();
+      mbar_arrive_after_copies(&full[b]);
+      mbar_arrive(&full[b]);
+      held[b] = tl;
+      held_k[b] = k;
+      live[b] = true;
+      ++n_tiles;
+    }
+    // drain: older buffer first
+    for (int jj = 0; jj < 2; ++jj) {
+      const int b = (int)((k + jj) & 1u);
+      if (live[b]) {
+        if (ok && !mbar_wait(&done[b], (held_k[b] >> 1) & 1u, P)) ok = false;
+        if (ok) report_tile<R1B>(P, held[b], lane);
+        live[b] = false;
+      }
+    }
+    if (ok) {                              // both buffers are idle: hand the compute warps the end marker
+      const int b = (int)(k & 1u);
+      if (lane == 0) desc[b].phase = PH_NONE;
+      __syncwarp();
+      __threadfence_block();
+      mbar_arrive(&full[b]);
+      mbar_arrive(&full[b]);
+    }
+    cp_async_wait<0>();
+    if (lane == 0) {
+      atomicAdd(&sc->stats[0], n_tiles);
+      atomicAdd(&sc->stats[1], n_late);
+    }
+  } else {
+    // ------------------------------------------------------------ compute warps
+    unsigned long long c_wait = 0, c_ph[4] = {0, 0, 0, 0};
+    const long long c_begin = clock64();
+    for (unsigned k = 0;; ++k) {
+      const int b = (int)(k & 1u);
+      const long long c0 = clock64();
+      if (!mbar_wait(&full[b], (k >> 1) & 1u, P)) break;
+      const Tile tl = desc[b];
+      if (tl.phase == PH_NONE) break;
+      const long long c1 = clock64();
       float4 *buf = bufs + b * BUF4;
-      if (cur.phase == PH_P1) P1::compute(P, cur, buf, twb, NTAB, red, tid, pre, post);
-      else if (cur.phase == PH_P2) P2::compute(P, cur, buf, twb, NTAB, t2, ab + b * 2 * NAB, chf + b * 2, tid, pre, post);
-      else P3::compute(P, cur, buf, twb, NTAB, red, &s_last, tid, pre, post);
-      {
-        const long long clk_end = clock64();
-        ++st_tiles;
-        st_wait += (unsigned long long)(clk_data - clk_top);
-        st_ph[cur.phase] += (unsigned long long)(clk_end - clk_data);
-      }
-      prev = cur;
-      have_prev = true;
-      cur = nxt;
-      issued = nxt_issued;
-      b ^= 1;
-      if (cur.phase == PH_NONE) { finished = true; break; }
+      if (tl.phase == PH_P1) P1::compute(P, tl, buf, twb, NTAB, red[b], tid);
+      else if (tl.phase == PH_P2) P2::compute(P, tl, buf, twb, NTAB, t2, ab + b * 2 * NAB, chf + b * 2, tid);
+      else P3::compute(P, tl, buf, twb, NTAB, red[b], tid);
+      mbar_arrive(&done[b]);               // this thread's part of the tile is stored, the buffer is free
+      c_wait += (unsigned long long)(c1 - c0);
+      c_ph[tl.phase] += (unsigned long long)(clock64() - c1);
+    }
+    if (tid == 0) {
+      atomicAdd(&sc->stats[3], c_ph[PH_P1]);
+      atomicAdd(&sc->stats[4], c_ph[PH_P2]);
+      atomicAdd(&sc->stats[5], c_ph[PH_P3]);
+      atomicAdd(&sc->stats[6], c_wait);
+      atomicAdd(&sc->stats[7], (unsigned long long)(clock64() - c_begin));
     }
   }
-  cp_async_wait<0>();
   __syncthreads();
-  if (tid == 0 && finished && have_prev) signal_done(P, prev);
-  if (tid == 0) {
-    atomicAdd(&sc->stats[0], st_tiles);
-    atomicAdd(&sc->stats[1], st_slow);
-    atomicAdd(&sc->stats[2], st_ph[0]);      // cycles thread 0 spent reporting finished tiles
-    atomicAdd(&sc->stats[3], st_ph[PH_P1]);
-    atomicAdd(&sc->stats[4], st_ph[PH_P2]);
-    atomicAdd(&sc->stats[5], st_ph[PH_P3]);
-    atomicAdd(&sc->stats[6], st_wait);
-    atomicAdd(&sc->stats[7], (unsigned long long)(clock64() - clk_begin));
-  }
 
   // ---- exit: the last block to leave adds up the energy partial sums in a fixed order and
   // returns the scheduler state to all-zero
   if (tid == 0) {
     __threadfence();
     const unsigned old = atomicAdd(&sc->exit_counter, 1u);
-    s_ok = (old + 1u == gridDim.x) ? 1 : 0;
+    s_last = (old + 1u == gridDim.x) ? 1 : 0;
   }
   __syncthreads();
-  if (!s_ok) return;
+  if (!s_last) return;
   __threadfence();
   double *redd = reinterpret_cast<double *>(smem4);        // [4][NT]
   const int n_part = P.U * P.TPU;
   double a0 = 0, a1 = 0, b0 = 0, b1 = 0;
-  for (int i = tid; i < n_part; i += NT) {
-    a0 += __ldcg(P.part_tot + 2 * i); a1 += __ldcg(P.part_tot + 2 * i + 1);
-    b0 += __ldcg(P.part_hi + 2 * i);  b1 += __ldcg(P.part_hi + 2 * i + 1);
+  if (tid < NT) {
+    for (int i = tid; i < n_part; i += NT) {
+      a0 += __ldcg(P.part_tot + 2 * i); a1 += __ldcg(P.part_tot + 2 * i + 1);
+      b0 += __ldcg(P.part_hi + 2 * i);  b1 += __ldcg(P.part_hi + 2 * i + 1);
+    }
+    redd[tid] = b0; redd[NT + tid] = a0; redd[2 * NT + tid] = b1; redd[3 * NT + tid] = a1;
   }
-  redd[tid] = b0; redd[NT + tid] = a0; redd[2 * NT + tid] = b1; redd[3 * NT + tid] = a1;
   __syncthreads();
   for (int st = NT / 2; st > 0; st >>= 1) {
     if (tid < st)
@@ -846,9 +900,9 @@ __global__ void __launch_bounds__(NT, FC_FUSED_MINB) k_fused(const __grid_consta
     __syncthreads();
   }
   if (tid < 4) P.energy[tid] = redd[tid * NT];
-  for (int i = tid; i < P.U; i += NT) { sc->done1[i] = 0u; sc->done2[i] = 0u; sc->done3[i] = 0u; }
+  for (int i = tid; i < P.U; i += NTH) { sc->done1[i] = 0u; sc->done2[i] = 0u; sc->done3[i] = 0u; }
   const int ncnt = P.nparts > 1 ? P.num_heads * (P.N / (16 * R1B)) : 0;
-  for (int i = tid; i < ncnt; i += NT) sc->cnt3[i] = 0u;
+  for (int i = tid; i < ncnt; i += NTH) sc->cnt3[i] = 0u;
   if (tid == 0) { sc->tile_counter = 0u; sc->exit_counter = 0u; sc->abort_flag = 0u; }
 }
 

@@ -40,13 +40,15 @@ def _rand_kv(T, H, d, dtype, seed, smooth=True):
     return k.to(dtype), v.to(dtype)
 
 
-def _gpu_scores(fc, k, v, cu, gamma, max_seqlen=None, group_bytes=None):
+def _gpu_scores(fc, k, v, cu, gamma, max_seqlen=None, group_bytes=None, fused=None):
     T, H, d = k.shape
     seqlens = [cu[i + 1] - cu[i] for i in range(len(cu) - 1)]
     h = fc.fc_create(0, max_seqlen or max(1, max(seqlens, default=1)))
     try:
         if group_bytes:
             fc.fc_set_group_bytes(h, group_bytes)
+        if fused is not None:
+            fc.fc_set_fused(h, True, fused)
         kd, vd = (k if k.is_cuda else k.cuda()), (v if v.is_cuda else v.cuda())
         scores = torch.full((H, max(T, 1)), -1.0, dtype=torch.float32, device="cuda")
         energy = torch.full((len(cu) - 1, 4), -1.0, dtype=torch.float64, device="cuda")
@@ -165,6 +167,24 @@ def test_scores_long_arbitrary_length(fc):
     N = 40961
     k, v = _rand_kv(N, 1, 64, torch.bfloat16, N)
     _check_layer(fc, k, v, [0, N], 0.2)
+
+
+@pytest.mark.parametrize("lag", [1, 2, 3])
+@pytest.mark.parametrize("N,H,dtype", [(4096, 3, torch.float32), (8192, 2, torch.bfloat16), (16384, 1, torch.float16),
+                                       (32768, 2, torch.bfloat16), (65536, 1, torch.bfloat16)])
+def test_scores_fused_persistent_kernel(fc, N, H, dtype, lag):
+    # the one-launch persistent form of the three passes, every supported length and stage distance
+    k, v = _rand_kv(N, H, 128, dtype, N + lag)
+    g, en = _check_layer(fc, k, v, [0, N], 0.2, fused=lag)
+    g2, en2 = _gpu_scores(fc, k, v, [0, N], 0.2, fused=lag)
+    assert np.array_equal(g, g2) and np.array_equal(en, en2)          # deterministic
+
+
+def test_scores_fused_ragged_batch(fc):
+    lens = [4096, 300, 8192, 0, 1024, 4096]
+    cu = [0] + [int(x) for x in np.cumsum(lens)]
+    k, v = _rand_kv(cu[-1], 4, 128, torch.bfloat16, 21)
+    _check_layer(fc, k, v, cu, 0.2, max_seqlen=8192, fused=2)
 
 
 # ---------------------------------------------------------------- budgets
