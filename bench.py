@@ -216,18 +216,13 @@ def main():
         return
 
     import torch
-    from paper_2511_16786_b200 import binding, synth_kv as S
+    from paper_2511_16786_b200 import binding, replicas, synth_kv as S
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local_rank = replicas.world_from_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dist = replicas.init("nccl", torch.device("cuda", local_rank))
     if max(args.warmup, 0) < 3:
         args.warmup = 3
 
@@ -248,9 +243,7 @@ def main():
     input_bytes = sum(k.numel() * k.element_size() * 2 for k in Kd)
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(dist, dev)
 
     sampler = ClockSampler(physical_gpu_index(local_rank))
     t_load0 = time.time()
@@ -286,13 +279,10 @@ def main():
     launches = binding.fc_launch_count(comp.handle) - launches0
     clocks = sampler.stop(t_wall0, t_wall1)
     comp.check_device_status()
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = replicas.max_over_ranks(elapsed_ms, dist, dev)
     ms_per_step = elapsed_ms / args.steps
     tokens = cfg.total_tokens
-    value = tokens * world / (ms_per_step / 1000.0)
+    value = replicas.whole_job_rate(tokens, world, ms_per_step)
 
     # roofline of the dominant kernel and of the whole step
     acc, rows = step_accounting(binding, comp.handle, cfg)
@@ -385,11 +375,8 @@ def main():
             d2h_bytes = e2e_step()
         barrier()
         e2e_ms = 1000.0 * (time.perf_counter() - t0) / n_e2e
-        if dist is not None:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        out["e2e"] = {"value": tokens * world / (e2e_ms / 1000.0), "unit": UNIT,
+        e2e_ms = replicas.max_over_ranks(e2e_ms, dist, dev)
+        out["e2e"] = {"value": replicas.whole_job_rate(tokens, world, e2e_ms), "unit": UNIT,
                       "h2d_bytes_per_step": int(input_bytes), "d2h_bytes_per_step": int(d2h_bytes),
                       "ms_per_step": e2e_ms, "steps": n_e2e}
         del hostK, hostV, hk, hv

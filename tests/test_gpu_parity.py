@@ -372,6 +372,83 @@ def test_config5_shape_reduced_ragged(fc):
     _compare_compress(fc, cfg)
 
 
+# ---------------------------------------------------------------- full-size shapes, sampled
+def _compare_sampled(fc, cfg, samples):
+    """Whole pass at a benchmark configuration's own sizes (same Compressor, same launch
+    configuration as bench.py); the oracle checks the sampled (layer, sequence, head) triples one by
+    one, properties that hold at any size cover the rest."""
+    from paper_2511_16786_b200.binding import Compressor
+    L, H, d = cfg.num_layers, cfg.num_heads, cfg.head_dim
+    Kd, Vd = zip(*(S.make_layer(cfg, l, "cuda") for l in range(L)))
+    comp = Compressor(L, H, d, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho, cfg.gamma, cfg.min_keep)
+    comp.compress(Kd, Vd)
+    comp.check_device_status()
+    tol = TOL[cfg.torch_dtype]
+    cu = cfg.cu_seqlens
+    g_energy = comp.energy.cpu().numpy()
+    g_budgets = comp.budgets.cpu().numpy()
+    g_offsets = comp.offsets.cpu().numpy()
+    # any size: Parseval totals, score/energy identity, the budget rule on the device's own energies
+    for l in range(L):
+        for b, n in enumerate(cfg.seqlens):
+            ks, vs = Kd[l][cu[b]:cu[b + 1]].double(), Vd[l][cu[b]:cu[b + 1]].double()
+            np.testing.assert_allclose(g_energy[l, b, 1], float((ks * ks).sum()), rtol=1e-5)
+            np.testing.assert_allclose(g_energy[l, b, 3], float((vs * vs).sum()), rtol=1e-5)
+            dev_sum = float(comp.scores[l][:, cu[b]:cu[b + 1]].double().sum()) * d
+            np.testing.assert_allclose(g_energy[l, b, 0] + g_energy[l, b, 2], dev_sum, rtol=1e-4)
+    ob, oo = O.allocate_budgets(g_energy, list(cfg.seqlens), cfg.rho, cfg.min_keep)
+    np.testing.assert_array_equal(g_budgets, ob)
+    np.testing.assert_array_equal(g_offsets, oo)
+    for b, n in enumerate(cfg.seqlens):
+        assert int(g_budgets[:, b].sum()) == O.total_budget(n, L, cfg.rho, cfg.min_keep)
+    # sampled triples against the oracle
+    for (l, b, h) in samples:
+        n = cfg.seqlens[b]
+        kh = Kd[l][cu[b]:cu[b + 1], h].cpu()
+        vh = Vd[l][cu[b]:cu[b + 1], h].cpu()
+        o, _ = O.score_head(kh.double().numpy(), vh.double().numpy(), cfg.gamma, "fft")
+        g32 = comp.scores[l][h, cu[b]:cu[b + 1]].cpu().numpy()
+        g = g32.astype(np.float64)
+        ebar = ((kh.double().numpy() ** 2).sum(1) + (vh.double().numpy() ** 2).sum(1)).mean() / d
+        err = float((np.abs(g - o) / np.maximum(o, 1e-6 * ebar)).max())
+        assert err <= tol, "layer %d seq %d head %d: score error %.3e" % (l, b, h, err)
+        kb = int(g_budgets[l, b])
+        off = int(g_offsets[l, b])
+        got = comp.out_idx[l, h, off:off + kb].cpu().numpy()
+        # index work is exact on the fp32 scores both sides see ...
+        np.testing.assert_array_equal(got, O.select_topk(g32, kb))
+        # ... and agrees with the fp64 scores except within the tolerance of the threshold
+        want = O.select_topk(o, kb)
+        diff = np.setxor1d(got, want)
+        if len(diff) and kb > 0:
+            tau = np.sort(o)[::-1][kb - 1]
+            assert np.all(np.abs(o[diff] - tau) <= tol * tau)
+        rows = slice(off, off + kb)
+        assert torch.equal(comp.out_k[l][rows, h].cpu().view(torch.uint8), kh[got].contiguous().view(torch.uint8))
+        assert torch.equal(comp.out_v[l][rows, h].cpu().view(torch.uint8), vh[got].contiguous().view(torch.uint8))
+    comp.close()
+
+
+def test_config2_full_size_sampled(fc):
+    cfg = S.paper_configs()["cfg2"]
+    _compare_sampled(fc, cfg, [(0, 0, 0), (13, 0, 2), (27, 0, 3)])
+
+
+def test_config3_full_size_sampled(fc):
+    cfg = S.paper_configs()["cfg3"]
+    _compare_sampled(fc, cfg, [(0, 0, 1), (27, 0, 3)])
+
+
+def test_config4_shape_full_length_sampled(fc):
+    cfg = S.scaled(S.paper_configs()["cfg4"], "cfg4", num_layers=3)       # 32 heads x 16384 tokens, 3 of the 32 layers
+    _compare_sampled(fc, cfg, [(0, 0, 0), (2, 0, 31)])
+
+
+def test_config5_full_lengths_sampled(fc):
+    cfg = S.scaled(S.paper_configs()["cfg5"], "cfg5", num_layers=2)       # the 8 ragged lengths, 2 of the 28 layers
+    _compare_sampled(fc, cfg, [(0, 6, 0), (1, 7, 3), (1, 3, 2)])
+
+
 # ---------------------------------------------------------------- ABI error paths (host-side checks only)
 def test_abi_rejects_bad_arguments(fc):
     h = fc.fc_create(0, 1024)
