@@ -10,10 +10,11 @@
 //    tiles that were handed out before it; a producer and its first consumer are three
 //    tile blocks apart, more than the blocks in flight, so the wait is normally over
 //    before it starts.  The intermediates live in a ring of unit slots that stays in L2.
-//  * every tile is 4096 complex points = 2048 float4 (32 KB), processed by 128 threads;
-//    the next tile is fetched into the second shared-memory buffer with cp.async while the
-//    current one is transformed in place.  Thread 0 asks for tile indices and reads
-//    completion counters one step ahead, so those round trips are off the critical path.
+//  * every tile is 4096 complex points = 2048 float4 (32 KB), processed by the 128 threads of
+//    four compute warps; a fifth (scheduler) warp asks for tile numbers, waits for the tiles
+//    they depend on, fills the second shared-memory buffer with cp.async while the current
+//    one is transformed in place, and reports finished tiles, so the compute warps only ever
+//    wait for a full buffer (mbarrier).
 //  * pass 3 writes one partial score per 2*CPW channels; the block that delivers the last
 //    partial of a (head, row set) adds them in a fixed order (deterministic).
 //  * a thread owns two adjacent channels as ONE packed value per component:
@@ -42,8 +43,8 @@ struct Sched {
   unsigned done3[1024];   // pass-3 tiles finished per unit
   unsigned cnt3[65536];   // partial scores delivered per (head, n2); the last deliverer resets its entry
   // running totals since the handle was created (diagnostic, see fc_fused_stats): tiles, tiles whose
-  // dependencies were not finished at look-ahead time, wait iterations, clock cycles of thread 0 inside
-  // pass-1 / pass-2 / pass-3 tiles, cycles waiting for tile data, cycles in the tile loop
+  // dependencies were not finished when the scheduler warp first looked, unused, clock cycles of thread 0
+  // inside pass-1 / pass-2 / pass-3 tiles, cycles waiting for a full buffer, cycles in the tile loop
   unsigned long long stats[8];
 };
 constexpr int kMaxCnt3 = 65536;
