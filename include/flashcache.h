@@ -101,8 +101,10 @@ fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_lag);
 /* Running totals of the fused transform kernel since fc_create (diagnostic; synchronises the
  * device): out = { tiles processed, tiles whose inputs were not finished when they were looked
  * when the scheduler warp first looked, unused, clock cycles (thread 0 of every block, summed) inside
- * pass-1, pass-2 and pass-3 tiles, cycles waiting for tile data, cycles inside the tile loop }. */
-fc_status fc_fused_stats(fc_handle *h, uint64_t out[8]);
+ * pass-1, pass-2 and pass-3 tiles, cycles waiting for tile data, cycles inside the tile loop,
+ * scheduler-warp cycles waiting for a buffer to come back, waiting for dependencies, issuing loads,
+ * and compute-warp cycles between the end of an issue and the buffer being full (waits only) }. */
+fc_status fc_fused_stats(fc_handle *h, uint64_t out[12]);
 
 /* Target size in bytes of the transform intermediates processed per kernel group
  * (kept below the L2 capacity so they are re-read from cache, not HBM).

@@ -152,15 +152,17 @@ def fc_set_group_bytes(handle, nbytes: int) -> None:
     _check(_lib.fc_set_group_bytes(handle, int(nbytes)), "fc_set_group_bytes")
 
 
-def fc_set_fused(handle, enabled: bool, stage_lag: int = 2) -> None:
-    _check(_lib.fc_set_fused(handle, 1 if enabled else 0, int(stage_lag)), "fc_set_fused")
+def fc_set_fused(handle, mode, stage_lag: int = 2) -> None:
+    """mode: 0 separate launches, 1 fused kernel with two packed columns per thread, 2 fused kernel
+    with one column per thread."""
+    _check(_lib.fc_set_fused(handle, int(mode), int(stage_lag)), "fc_set_fused")
 
 
 def fc_fused_stats(handle) -> dict:
-    out = (c_uint64 * 8)()
+    out = (c_uint64 * 12)()
     _check(_lib.fc_fused_stats(handle, out), "fc_fused_stats")
     keys = ("tiles", "late_tiles", "unused", "cycles_pass1", "cycles_pass2", "cycles_pass3",
-            "cycles_data_wait", "cycles_loop")
+            "cycles_data_wait", "cycles_loop", "sched_buffer_wait", "sched_dep_wait", "sched_issue", "landing_wait")
     return {k: int(v) for k, v in zip(keys, out)}
 
 

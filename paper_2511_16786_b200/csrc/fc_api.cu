@@ -54,7 +54,7 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->fused_blocks_per_sm = 0;
   h->fused_lag = 1;
   if (const char *e = getenv("FC_FUSED_LAG")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_lag = v; }
-  if (const char *e = getenv("FC_FUSED")) { h->fused_enabled = atoi(e) != 0 ? 1 : 0; }
+  if (const char *e = getenv("FC_FUSED")) { const int v = atoi(e); if (v >= 0 && v <= 2) h->fused_enabled = v; }
   if (const char *e = getenv("FC_FUSED_BPS")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_blocks_per_sm = v; }
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return FC_ERR_CUDA; }
@@ -168,19 +168,19 @@ extern "C" fc_status fc_last_device_status(fc_handle *h, fc_stream stream) {
   return (word & FC_DEV_FLAG_INTERNAL) ? FC_ERR_INTERNAL : FC_ERR_TIMEOUT;
 }
 
-extern "C" fc_status fc_fused_stats(fc_handle *h, uint64_t out[8]) {
+extern "C" fc_status fc_fused_stats(fc_handle *h, uint64_t out[12]) {
   if (!h || !out || !h->fused_sched) return FC_ERR_INVALID_ARG;
   FC_CUDA_TRY(cudaDeviceSynchronize());
   const fused::Sched *sc = static_cast<const fused::Sched *>(h->fused_sched);
-  FC_CUDA_TRY(cudaMemcpy(out, sc->stats, 8 * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+  FC_CUDA_TRY(cudaMemcpy(out, sc->stats, 12 * sizeof(uint64_t), cudaMemcpyDeviceToHost));   // stats and stats2 are adjacent
   return FC_OK;
 }
 
 extern "C" uint64_t fc_launch_count(const fc_handle *h) { return h ? (uint64_t)h->launches : 0; }
 
 extern "C" fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_lag) {
-  if (!h || stage_lag < 1 || stage_lag > 4) return FC_ERR_INVALID_ARG;
-  h->fused_enabled = enabled ? 1 : 0;
+  if (!h || stage_lag < 1 || stage_lag > 4 || enabled < 0 || enabled > 2) return FC_ERR_INVALID_ARG;
+  h->fused_enabled = enabled;
   h->fused_lag = stage_lag;
   return FC_OK;
 }

@@ -42,7 +42,7 @@ struct fc_handle {
   bool generic_only;
   // scheduler state of the fused persistent kernel (DEVICE, all zero between launches) and knobs
   void *fused_sched;
-  int fused_enabled;       // 1 enables the fused kernel (developer knob FC_FUSED)
+  int fused_enabled;       // 0 separate launches, 1 fused kernel (two packed columns per thread), 2 fused, one column per thread
   int fused_blocks_per_sm; // 0 = as many as fit
   int fused_lag;           // stages between pass 1, pass 2 and pass 3 of a unit
 };

@@ -697,16 +697,17 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
   return FC_ERR_INTERNAL;
 }
 
-template <typename T, int R1B, int R2B>
+template <typename T, int R1B, int R2B, int ONE>
 fc_status launch_fused_impl(fc_handle *h, cudaStream_t st, const fused::Params &P) {
-  auto kern = fused::k_fused<T, R1B, R2B>;
-  const size_t sm = fused::Smem<R1B, R2B>::bytes;
+  auto kern = fused::k_fused<T, R1B, R2B, ONE>;
+  const size_t sm = fused::Smem<R1B, R2B, ONE>::bytes;
+  constexpr int threads = fused::Threads<ONE>::all;
   fc_status s = set_smem(kern, sm);
   if (s != FC_OK) return s;
   static int blocks_per_sm = 0;                     // per instantiation; the answer does not change
   if (blocks_per_sm == 0) {
     int n = 0;
-    FC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, fused::NTH, sm));
+    FC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, threads, sm));
     if (n < 1) return FC_ERR_INTERNAL;
     blocks_per_sm = n;
   }
@@ -715,14 +716,20 @@ fc_status launch_fused_impl(fc_handle *h, cudaStream_t st, const fused::Params &
   unsigned grid = (unsigned)(h->num_sms * bps);
   if (grid > P.total_tiles) grid = P.total_tiles;
   ProfScope ps(h, FC_K_FUSED, st);
-  kern<<<grid, fused::NTH, sm, st>>>(P);
+  kern<<<grid, threads, sm, st>>>(P);
   return fc_after_launch(h);
 }
 
 template <typename T>
 fc_status launch_fused(fc_handle *h, cudaStream_t st, const FusedPlan &f, const fused::Params &P) {
+  if (h->fused_enabled == 2 && f.r1b >= 8) {        // one column per thread (needs N1 >= 128)
+#define FC_FUSED_CASE1(A, B) \
+  if (f.r1b == A && f.r2b == B) return launch_fused_impl<T, A, B, 1>(h, st, P);
+    FC_FUSED_CASE1(8, 8) FC_FUSED_CASE1(8, 16) FC_FUSED_CASE1(16, 16)
+#undef FC_FUSED_CASE1
+  }
 #define FC_FUSED_CASE(A, B) \
-  if (f.r1b == A && f.r2b == B) return launch_fused_impl<T, A, B>(h, st, P);
+  if (f.r1b == A && f.r2b == B) return launch_fused_impl<T, A, B, 0>(h, st, P);
   FC_FUSED_CASE(4, 4) FC_FUSED_CASE(4, 8) FC_FUSED_CASE(8, 8) FC_FUSED_CASE(8, 16) FC_FUSED_CASE(16, 16)
 #undef FC_FUSED_CASE
   return FC_ERR_INTERNAL;

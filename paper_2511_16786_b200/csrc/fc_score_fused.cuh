@@ -46,6 +46,9 @@ struct Sched {
   // dependencies were not finished when the scheduler warp first looked, unused, clock cycles of thread 0
   // inside pass-1 / pass-2 / pass-3 tiles, cycles waiting for a full buffer, cycles in the tile loop
   unsigned long long stats[8];
+  // scheduler warp (lane 0, summed): cycles waiting for a buffer to come back, waiting for dependencies,
+  // issuing the loads; compute warps: cycles from the end of the issue to the buffer being full
+  unsigned long long stats2[4];
 };
 constexpr int kMaxCnt3 = 65536;
 
@@ -659,6 +662,250 @@ struct Pass3 {
   }
 };
 
+// ------------------------------------------------------------------ one-column compute variants
+// Same tiles, same shared-memory bytes and the same scheduler-side loads as Pass1/2/3, but 256
+// compute threads per tile, each owning ONE complex column (K + jV of one channel) and 16 points
+// in plain float2 arithmetic: half the registers per thread, twice the resident warps.  The
+// intermediate is then ordinary interleaved complex (re, im) per column.  N1 >= 128 only (the
+// row sums of pass 3 are reduced inside one warp).
+constexpr int NTC1 = 256;
+__device__ __forceinline__ void bar_compute1() { asm volatile("bar.sync 1, 256;\n" ::: "memory"); }
+
+template <typename T> struct One;
+template <> struct One<float> { __device__ static float ld(const char *s) { return *reinterpret_cast<const float *>(s); } };
+template <> struct One<__half> { __device__ static float ld(const char *s) { return __half2float(*reinterpret_cast<const __half *>(s)); } };
+template <> struct One<__nv_bfloat16> {
+  __device__ static float ld(const char *s) {
+    return __uint_as_float((unsigned)(*reinterpret_cast<const unsigned short *>(s)) << 16);
+  }
+};
+
+template <typename T, int R1B>
+struct Pass1S {
+  static constexpr int N1 = 16 * R1B, C = NTC1 / R1B, IT = 16 / R1B, ES = Pair<T>::ES, ROWB = C * ES;
+  __device__ static void compute(const Params &P, const Tile &tl, float4 *buf4, const float2 *tw, int ntab,
+                                 double (*red)[8], int tid) {
+    const int N2 = P.N / N1;
+    const int c = tid % C, j = tid / C;
+    const char *in = reinterpret_cast<const char *>(buf4);
+    float2 *S = reinterpret_cast<float2 *>(buf4);
+    float2 x[16];
+    float aK = 0.f, aV = 0.f;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const int row = j + R1B * p;
+      x[p].x = One<T>::ld(in + row * ROWB + c * ES);
+      x[p].y = One<T>::ld(in + (N1 + row) * ROWB + c * ES);
+      aK = fmaf(x[p].x, x[p].x, aK);
+      aV = fmaf(x[p].y, x[p].y, aV);
+    }
+    {
+      const double a = warp_sum_d((double)aK), b = warp_sum_d((double)aV);
+      if ((tid & 31) == 0) { red[0][tid >> 5] = a; red[1][tid >> 5] = b; }
+    }
+    bar_compute1();                        // every thread has its inputs; the buffer becomes the exchange area
+    dft_small<16, -1>(x);
+    const int tstep = ntab / N1;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      if (p > 0) x[p] = cmul(x[p], tw[j * p * tstep]);
+      S[(j + R1B * p) * C + c] = x[p];
+    }
+    bar_compute1();
+    float2 *slot = slot_base(P, tl.unit);
+    const int col = tl.cb * C + c;
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R1B * it;
+      float2 y[R1B];
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) y[q] = S[(q + R1B * pp) * C + c];
+      dft_small<R1B, -1>(y);
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) {
+        const int k1 = pp + 16 * q;
+        __stcg(slot + ((size_t)k1 * N2 + tl.a) * P.UC + col, y[q]);
+      }
+    }
+    if (tid == 0) {
+      const size_t s = (size_t)tl.unit * P.TPU + tl.idx;
+      double a = 0, b = 0;
+#pragma unroll
+      for (int w = 0; w < NTC1 / 32; ++w) { a += red[0][w]; b += red[1][w]; }
+      P.part_tot[2 * s] = a;
+      P.part_tot[2 * s + 1] = b;
+    }
+  }
+};
+
+// Thread (c = tid % C, j = (tid / C) % R2B, hf = tid / (C * R2B)): consecutive j are consecutive
+// rows, so a half warp reads 128 contiguous bytes.
+template <int R2B>
+struct Pass2S {
+  static constexpr int N2 = 16 * R2B, C = NTC1 / (2 * R2B), IT = 16 / R2B, NAB = R2B + 16;
+  static constexpr int HALF2 = 2 * Pass2<R2B>::HALF;         // float2 per half, as the loads laid it out
+  __device__ static void compute(const Params &P, const Tile &tl, float4 *buf4, const float2 *tw, int ntab,
+                                 const float2 *t2, const float4 *ab, const float2 *chf, int tid) {
+    const int N1 = P.N / N2, N = P.N;
+    const int c = tid % C, j = (tid / C) % R2B, hf = tid / (C * R2B);
+    const bool self = tl.a == 0;
+    const int k1 = hf ? (self ? N1 / 2 : N1 - tl.a) : tl.a;
+    float2 *Sh = reinterpret_cast<float2 *>(buf4) + hf * HALF2;
+    const float2 *Sp = reinterpret_cast<const float2 *>(buf4) + (self ? hf : 1 - hf) * HALF2;
+    const float4 A4 = ab[hf * NAB + j];
+    const float2 A = make_float2(A4.x, A4.z);
+    const float4 *B = ab + hf * NAB + R2B;
+    const int tstep = ntab / N2;
+    float2 x[16];
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const float4 b4 = B[p];
+      x[p] = cmul(Sh[(j + R2B * p) * C + c], cmul(A, make_float2(b4.x, b4.z)));
+    }
+    dft_small<16, -1>(x);
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      if (p > 0) x[p] = cmul(x[p], tw[j * p * tstep]);
+      Sh[(j + R2B * p) * C + c] = x[p];             // same cell this thread read: no barrier needed before
+    }
+    bar_compute1();
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R2B * it;
+      float2 y[R2B];
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) y[q] = Sh[(q + R2B * pp) * C + c];
+      dft_small<R2B, -1>(y);
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) {
+        x[it * R2B + q] = y[q];
+        Sh[(q + R2B * pp) * C + c] = y[q];
+      }
+    }
+    bar_compute1();                        // full spectra of both halves are in shared memory
+    const float2 ch = chf[hf];
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R2B * it;
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) {
+        const int k2 = pp + 16 * q;
+        const int bin = k1 + N1 * k2;
+        const bool inL = bin <= P.omega, inH = (N - bin) <= P.omega;
+        float2 &Pv = x[it * R2B + q];
+        if (bin == 0 || (inL && inH)) {
+          Pv = make_float2(0.f, 0.f);
+        } else if (inL || inH) {
+          const int k2p = (k1 == 0) ? ((N2 - k2) & (N2 - 1)) : (N2 - 1 - k2);
+          const float2 Q = Sp[((k2p >> 4) + R2B * (k2p & 15)) * C + c];
+          const float2 e = cmul(ch, t2[k2]);                      // exp(-j*pi*bin/N)
+          const float sgn = inL ? -0.5f : 0.5f;                   // E = (P -/+ uQ)/2, u = exp(+j*pi*bin/N)
+          const float ur = e.x * sgn, ui = -e.y * sgn;
+          Pv = make_float2(fmaf(Q.x, ur, fmaf(-Q.y, ui, 0.5f * Pv.x)), fmaf(Q.x, ui, fmaf(Q.y, ur, 0.5f * Pv.y)));
+        }
+      }
+    }
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      float2 y[R2B];
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) y[q] = x[it * R2B + q];
+      dft_small<R2B, +1>(y);
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) x[it * R2B + q] = y[q];
+    }
+    bar_compute1();                        // all partner reads are done
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R2B * it;
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) Sh[(q + R2B * pp) * C + c] = x[it * R2B + q];
+    }
+    bar_compute1();
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      x[p] = Sh[(j + R2B * p) * C + c];
+      if (p > 0) x[p] = cmul_conj(x[p], tw[j * p * tstep]);
+    }
+    dft_small<16, +1>(x);
+    float2 *base = slot_base(P, tl.unit) + (size_t)k1 * N2 * P.UC + tl.cb * C + c;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const float4 b4 = B[p];
+      __stcg(base + (size_t)(j + R2B * p) * P.UC, cmul_conj(x[p], cmul(A, make_float2(b4.x, b4.z))));
+    }
+  }
+};
+
+template <int R1B>
+struct Pass3S {
+  static constexpr int N1 = 16 * R1B, C = NTC1 / R1B, IT = 16 / R1B;
+  static constexpr int DUP = C > 16 ? C / 16 : 1;
+  __device__ static void compute(const Params &P, const Tile &tl, float4 *buf4, const float2 *tw, int ntab,
+                                 double (*red)[8], int tid) {
+    const int N2 = P.N / N1;
+    const int c = tid % C, j = tid / C;
+    const int tstep = ntab / N1;
+    float2 *S = reinterpret_cast<float2 *>(buf4);
+    float2 x[16];
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R1B * it;
+      float2 y[R1B];
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) y[q] = S[(pp + 16 * q) * C + c];
+      dft_small<R1B, +1>(y);
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) x[it * R1B + q] = y[q];
+    }
+    bar_compute1();                        // all bins read; the buffer becomes the exchange area
+#pragma unroll
+    for (int it = 0; it < IT; ++it) {
+      const int pp = j + R1B * it;
+#pragma unroll
+      for (int q = 0; q < R1B; ++q) S[(q + R1B * pp) * C + c] = x[it * R1B + q];
+    }
+    bar_compute1();
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      x[p] = S[(j + R1B * p) * C + c];
+      if (p > 0) x[p] = cmul_conj(x[p], tw[j * p * tstep]);
+    }
+    dft_small<16, +1>(x);
+    float acc[16];
+    float totK = 0.f, totV = 0.f;
+#pragma unroll
+    for (int p = 0; p < 16; ++p) {
+      const float ek = x[p].x * x[p].x, ev = x[p].y * x[p].y;
+      acc[p] = ek + ev;
+      totK += ek;
+      totV += ev;
+    }
+    int prow = 0;
+    RowReduce<16, C / 2>::run(acc, c, prow);
+    const int gcol = tl.unit * P.UC + tl.cb * C;
+    const int head = gcol / P.head_dim, part = (gcol - head * P.head_dim) / C;
+    float *dstp = P.nparts > 1 ? P.partial + ((size_t)part * P.num_heads + head) * (size_t)P.N
+                               : P.scores + (long long)head * P.score_stride;
+    if ((c & (DUP - 1)) == 0) {
+      const int p = (j + R1B * prow) * N2 + tl.a;
+      __stcg(dstp + perm_token(p, P.N), acc[0] * P.inv_scale);
+    }
+    const double dk = warp_sum_d((double)(totK * P.inv_scale));
+    const double dv = warp_sum_d((double)(totV * P.inv_scale));
+    if ((tid & 31) == 0) { red[0][tid >> 5] = dk; red[1][tid >> 5] = dv; }
+    bar_compute1();
+    if (tid == 0) {
+      const size_t s = (size_t)tl.unit * P.TPU + tl.idx;
+      double a = 0, b = 0;
+#pragma unroll
+      for (int w = 0; w < NTC1 / 32; ++w) { a += red[0][w]; b += red[1][w]; }
+      P.part_hi[2 * s] = a * (double)P.head_dim;
+      P.part_hi[2 * s + 1] = b * (double)P.head_dim;
+    }
+  }
+};
+
 // ------------------------------------------------------------------ mbarrier helpers
 __device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"((unsigned)__cvta_generic_to_shared(bar)), "r"(count) : "memory");
@@ -694,12 +941,14 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
 // Block = 4 compute warps + 1 scheduler warp.  The scheduler warp takes tile numbers, waits for
 // the tiles they depend on, fills one of two shared-memory buffers with cp.async and reports
 // finished tiles; the compute warps only ever wait for a full buffer.
-constexpr int NTH = NT + 32;
+// ONE = 0: two packed columns per thread, 128 compute threads; ONE = 1: one column per thread, 256.
+template <int ONE> struct Threads { static constexpr int compute = ONE ? NTC1 : NT, all = compute + 32; };
 
-template <int R1B, int R2B>
+template <int R1B, int R2B, int ONE>
 struct Smem {
   static constexpr int N1 = 16 * R1B, N2 = 16 * R2B, NTAB = N1 > N2 ? N1 : N2, NAB = R2B + 16;
-  static constexpr size_t bytes = (size_t)2 * BUF4 * sizeof(float4) + NTAB * sizeof(float4) + N2 * sizeof(float2) +
+  static constexpr size_t tw_bytes = NTAB * (ONE ? sizeof(float2) : sizeof(float4));
+  static constexpr size_t bytes = (size_t)2 * BUF4 * sizeof(float4) + tw_bytes + N2 * sizeof(float2) +
                                   2 * 2 * NAB * sizeof(float4) + 2 * 2 * sizeof(float2);
 };
 
@@ -735,35 +984,41 @@ __device__ __forceinline__ void report_tile(const Params &P, const Tile &tl, int
 #ifndef FC_FUSED_MINB
 #define FC_FUSED_MINB 3
 #endif
-template <typename T, int R1B, int R2B>
-__global__ void __launch_bounds__(NTH, FC_FUSED_MINB) k_fused(const __grid_constant__ Params P) {
-  using SM = Smem<R1B, R2B>;
+template <typename T, int R1B, int R2B, int ONE>
+__global__ void __launch_bounds__(Threads<ONE>::all, FC_FUSED_MINB) k_fused(const __grid_constant__ Params P) {
+  using SM = Smem<R1B, R2B, ONE>;
+  constexpr int NTC = Threads<ONE>::compute, NTH = Threads<ONE>::all;
   using P1 = Pass1<T, R1B>;
   using P2 = Pass2<R2B>;
   using P3 = Pass3<R1B>;
   constexpr int NTAB = SM::NTAB, N2 = SM::N2, NAB = SM::NAB;
   extern __shared__ float4 smem4[];
   float4 *bufs = smem4;                                           // [2][BUF4]
-  float4 *twb = smem4 + 2 * BUF4;                                 // [NTAB] exp(-2*pi*j*i/NTAB), broadcast
-  float2 *t2 = reinterpret_cast<float2 *>(twb + NTAB);            // [N2]   exp(-j*pi*k2/N2)
+  float4 *twb = smem4 + 2 * BUF4;                                 // [NTAB] exp(-2*pi*j*i/NTAB): broadcast float4, or float2 (ONE)
+  float2 *tw1 = reinterpret_cast<float2 *>(twb);
+  float2 *t2 = reinterpret_cast<float2 *>(reinterpret_cast<char *>(twb) + SM::tw_bytes);   // [N2] exp(-j*pi*k2/N2)
   float4 *ab = reinterpret_cast<float4 *>(t2 + N2);               // [2 buffers][2 halves][NAB]
   float2 *chf = reinterpret_cast<float2 *>(ab + 2 * 2 * NAB);     // [2 buffers][2 halves]
   __shared__ Tile desc[2];
   __shared__ unsigned long long full[2], done[2];
-  __shared__ double red[2][2][4];          // per buffer: a warp may enter the next tile while thread 0 still adds these up
+  __shared__ double red[2][2][8];          // per buffer: a warp may enter the next tile while thread 0 still adds these up
   __shared__ int s_last;
+  __shared__ long long stamp[2];
   const int tid = threadIdx.x, lane = tid & 31;
   Sched *sc = P.sched;
 
-  for (int i = tid; i < NTAB; i += NTH) twb[i] = bcast4(__ldg(P.master + (size_t)i * (P.master_len / NTAB)));
+  for (int i = tid; i < NTAB; i += NTH) {
+    const float2 w = __ldg(P.master + (size_t)i * (P.master_len / NTAB));
+    if (ONE) tw1[i] = w; else twb[i] = bcast4(w);
+  }
   for (int i = tid; i < N2; i += NTH) t2[i] = __ldg(P.master + (size_t)i * (P.master_len / (2 * N2)));
   if (tid == 0) {
     mbar_init(&full[0], 64u); mbar_init(&full[1], 64u);     // per lane: one arrival after its copies, one plain
-    mbar_init(&done[0], (unsigned)NT); mbar_init(&done[1], (unsigned)NT);
+    mbar_init(&done[0], (unsigned)NTC); mbar_init(&done[1], (unsigned)NTC);
   }
   __syncthreads();
 
-  if (tid >= NT) {
+  if (tid >= NTC) {
     // ------------------------------------------------------------ scheduler warp
     Walk walk = {0, 0u};
     unsigned t_next = 0u;
@@ -771,16 +1026,18 @@ __global__ void __launch_bounds__(NTH, FC_FUSED_MINB) k_fused(const __grid_const
     Tile held[2];
     unsigned held_k[2] = {0u, 0u};
     bool live[2] = {false, false};
-    unsigned long long n_tiles = 0, n_late = 0;
+    unsigned long long n_tiles = 0, n_late = 0, s_back = 0, s_deps = 0, s_issue = 0;
     bool ok = true;
     unsigned k = 0;
     for (;; ++k) {
       const int b = (int)(k & 1u);
+      const long long q0 = clock64();
       if (live[b]) {                       // the tile that used this buffer two steps ago
         if (!mbar_wait(&done[b], (held_k[b] >> 1) & 1u, P)) { ok = false; break; }
         report_tile<R1B>(P, held[b], lane);
         live[b] = false;
       }
+      const long long q1 = clock64();
       const unsigned t = __shfl_sync(0xffffffffu, t_next, 0);
       const Tile tl = decode_tile(P, walk, t);
       if (tl.phase == PH_NONE) break;
@@ -809,6 +1066,7 @@ __global__ void __launch_bounds__(NTH, FC_FUSED_MINB) k_fused(const __grid_const
         }
         if (!ok) break;
       }
+      const long long q2 = clock64();
       float4 *dst = bufs + b * BUF4;
       if (lane == 0) desc[b] = tl;
       if (tl.phase == PH_P1) P1::issue(P, tl, dst, lane);
@@ -816,8 +1074,12 @@ __global__ void __launch_bounds__(NTH, FC_FUSED_MINB) k_fused(const __grid_const
       else P3::issue(P, tl, dst, lane);
       __syncwarp();
       __threadfence_block();
+      if (lane == 0) stamp[b] = clock64();
       mbar_arrive_after_copies(&full[b]);
       mbar_arrive(&full[b]);
+      s_back += (unsigned long long)(q1 - q0);
+      s_deps += (unsigned long long)(q2 - q1);
+      s_issue += (unsigned long long)(clock64() - q2);
       held[b] = tl;
       held_k[b] = k;
       live[b] = true;
@@ -844,10 +1106,13 @@ __global__ void __launch_bounds__(NTH, FC_FUSED_MINB) k_fused(const __grid_const
     if (lane == 0) {
       atomicAdd(&sc->stats[0], n_tiles);
       atomicAdd(&sc->stats[1], n_late);
+      atomicAdd(&sc->stats2[0], s_back);
+      atomicAdd(&sc->stats2[1], s_deps);
+      atomicAdd(&sc->stats2[2], s_issue);
     }
   } else {
     // ------------------------------------------------------------ compute warps
-    unsigned long long c_wait = 0, c_ph[4] = {0, 0, 0, 0};
+    unsigned long long c_wait = 0, c_land = 0, c_ph[4] = {0, 0, 0, 0};
     const long long c_begin = clock64();
     for (unsigned k = 0;; ++k) {
       const int b = (int)(k & 1u);
@@ -856,10 +1121,17 @@ __global__ void __launch_bounds__(NTH, FC_FUSED_MINB) k_fused(const __grid_const
       const Tile tl = desc[b];
       if (tl.phase == PH_NONE) break;
       const long long c1 = clock64();
+      { const long long l = c1 - stamp[b]; if (c1 - c0 > 64) c_land += (unsigned long long)(l > 0 ? l : 0); }
       float4 *buf = bufs + b * BUF4;
-      if (tl.phase == PH_P1) P1::compute(P, tl, buf, twb, NTAB, red[b], tid);
-      else if (tl.phase == PH_P2) P2::compute(P, tl, buf, twb, NTAB, t2, ab + b * 2 * NAB, chf + b * 2, tid);
-      else P3::compute(P, tl, buf, twb, NTAB, red[b], tid);
+      if constexpr (ONE) {
+        if (tl.phase == PH_P1) Pass1S<T, R1B>::compute(P, tl, buf, tw1, NTAB, red[b], tid);
+        else if (tl.phase == PH_P2) Pass2S<R2B>::compute(P, tl, buf, tw1, NTAB, t2, ab + b * 2 * NAB, chf + b * 2, tid);
+        else Pass3S<R1B>::compute(P, tl, buf, tw1, NTAB, red[b], tid);
+      } else {
+        if (tl.phase == PH_P1) P1::compute(P, tl, buf, twb, NTAB, reinterpret_cast<double (*)[4]>(red[b]), tid);
+        else if (tl.phase == PH_P2) P2::compute(P, tl, buf, twb, NTAB, t2, ab + b * 2 * NAB, chf + b * 2, tid);
+        else P3::compute(P, tl, buf, twb, NTAB, reinterpret_cast<double (*)[4]>(red[b]), tid);
+      }
       mbar_arrive(&done[b]);               // this thread's part of the tile is stored, the buffer is free
       c_wait += (unsigned long long)(c1 - c0);
       c_ph[tl.phase] += (unsigned long long)(clock64() - c1);
@@ -869,6 +1141,7 @@ __global__ void __launch_bounds__(NTH, FC_FUSED_MINB) k_fused(const __grid_const
       atomicAdd(&sc->stats[4], c_ph[PH_P2]);
       atomicAdd(&sc->stats[5], c_ph[PH_P3]);
       atomicAdd(&sc->stats[6], c_wait);
+      atomicAdd(&sc->stats2[3], c_land);
       atomicAdd(&sc->stats[7], (unsigned long long)(clock64() - c_begin));
     }
   }
