@@ -697,6 +697,61 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
   return FC_ERR_INTERNAL;
 }
 
+// cuTensorMapEncodeTiled, looked up through the runtime (no link against the driver library).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+fc_status encode_map(CUtensorMap *m, CUtensorMapDataType dt, int rank, const void *base, const cuuint64_t *dims,
+                     const cuuint64_t *strides_b, const cuuint32_t *box) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return FC_ERR_CUDA;
+  const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+  const CUresult r = fn(m, dt, (cuuint32_t)rank, const_cast<void *>(base), dims, strides_b, box, ones,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? FC_OK : FC_ERR_INTERNAL;
+}
+
+// The four tensor maps of one fused launch (see fused::TmaMaps).
+template <typename T>
+fc_status make_tma_maps(const fused::Params &P, int N1, int N2, int cpw, int cp, fused::TmaMaps *M) {
+  const CUtensorMapDataType dt = sizeof(T) == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                               : (std::is_same<T, __half>::value ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                                 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+  fc_status s;
+  {
+    const cuuint64_t dims[4] = {(cuuint64_t)P.head_dim, (cuuint64_t)P.num_heads, (cuuint64_t)(2 * N2), (cuuint64_t)(N1 / 2)};
+    const cuuint64_t str[3] = {(cuuint64_t)P.stride_head_b, (cuuint64_t)P.stride_token_b,
+                               (cuuint64_t)(2 * N2) * (cuuint64_t)P.stride_token_b};
+    const cuuint32_t box[4] = {(cuuint32_t)(2 * cpw), 1, 1, (cuuint32_t)(N1 / 2)};
+    if ((s = encode_map(&M->k, dt, 4, P.k, dims, str, box)) != FC_OK) return s;
+    if ((s = encode_map(&M->v, dt, 4, P.v, dims, str, box)) != FC_OK) return s;
+  }
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)(2 * P.UC), (cuuint64_t)N2, (cuuint64_t)P.R * (cuuint64_t)N1};
+    const cuuint64_t str[2] = {(cuuint64_t)P.UC * 8, (cuuint64_t)N2 * (cuuint64_t)P.UC * 8};
+    const cuuint32_t box2[3] = {(cuuint32_t)(4 * cp), (cuuint32_t)N2, 1};
+    const cuuint32_t box3[3] = {(cuuint32_t)(4 * cpw), 1, (cuuint32_t)N1};
+    if ((s = encode_map(&M->ws2, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, P.ws, dims, str, box2)) != FC_OK) return s;
+    if ((s = encode_map(&M->ws3, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, P.ws, dims, str, box3)) != FC_OK) return s;
+  }
+  return FC_OK;
+}
+
 template <typename T, int R1B, int R2B, int ONE>
 fc_status launch_fused_impl(fc_handle *h, cudaStream_t st, const fused::Params &P) {
   auto kern = fused::k_fused<T, R1B, R2B, ONE>;
@@ -715,8 +770,10 @@ fc_status launch_fused_impl(fc_handle *h, cudaStream_t st, const fused::Params &
   if (h->fused_blocks_per_sm > 0 && h->fused_blocks_per_sm < bps) bps = h->fused_blocks_per_sm;
   unsigned grid = (unsigned)(h->num_sms * bps);
   if (grid > P.total_tiles) grid = P.total_tiles;
+  fused::TmaMaps M;
+  if ((s = make_tma_maps<T>(P, 16 * R1B, 16 * R2B, fused::NT / R1B, fused::NT / (2 * R2B), &M)) != FC_OK) return s;
   ProfScope ps(h, FC_K_FUSED, st);
-  kern<<<grid, threads, sm, st>>>(P);
+  kern<<<grid, threads, sm, st>>>(P, M);
   return fc_after_launch(h);
 }
 

@@ -24,13 +24,15 @@
 //
 // The transform is unnormalised (factor N); pass 3 folds 1/N^2 into the score.
 #pragma once
+#include <cuda.h>   // CUtensorMap (type only; the encoder is looked up at run time)
+
 #include "fc_common.cuh"
 
 namespace fused {
 
 constexpr int NT = 128;        // threads per block
 constexpr int TILE4 = 2048;    // float4 per tile
-constexpr int BUF4 = TILE4 + 16; // float4 per shared-memory buffer (room for the pass-2 bank padding)
+constexpr int BUF4 = TILE4;     // float4 per shared-memory buffer
 
 // Scheduler state in global memory (owned by the handle, all zero between launches).
 struct Sched {
@@ -73,6 +75,13 @@ struct Params {
   int *status;
   unsigned spin_limit;
 };
+
+// Tensor maps of one launch (encoded on the host, read by the TMA unit):
+//   k, v   K / V of the sequence as [N1/2 groups][2*N2 tokens][heads][channels]; a box is one channel
+//          slice of the N1/2 tokens that share a position inside their group (one half of a pass-1 tile)
+//   ws2    the ring as [R*N1 rows k1][N2][2*UC floats], box = N2 x (4*CP floats): one half of a pass-2 tile
+//   ws3    the same tensor, box = N1 x 1 x (4*CPW floats): a pass-3 tile
+struct TmaMaps { CUtensorMap k, v, ws2, ws3; };
 
 // ------------------------------------------------------------------ packed arithmetic
 // Two complex numbers a and b (adjacent channels): r = (re_a, re_b), i = (im_a, im_b).
@@ -263,6 +272,26 @@ template <> struct Pair<__nv_bfloat16> {
 };
 
 
+// ------------------------------------------------------------------ TMA and mbarrier transaction helpers
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;\n" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes) {
+  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}\n"
+               ::"r"((unsigned)__cvta_generic_to_shared(bar)), "r"(bytes) : "memory");
+}
+// Tiled loads into this block's shared memory; completion is counted in bytes on `bar`.  No multicast.
+__device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *map, int c0, int c1, int c2,
+                                            unsigned long long *bar) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
+               ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)), "l"(reinterpret_cast<unsigned long long>(map)),
+                 "r"(c0), "r"(c1), "r"(c2), "r"((unsigned)__cvta_generic_to_shared(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(void *smem_dst, const CUtensorMap *map, int c0, int c1, int c2, int c3,
+                                            unsigned long long *bar) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n"
+               ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)), "l"(reinterpret_cast<unsigned long long>(map)),
+                 "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"((unsigned)__cvta_generic_to_shared(bar)) : "memory");
+}
+
 // ------------------------------------------------------------------ tile descriptors
 enum { PH_NONE = 0, PH_P1 = 1, PH_P2 = 2, PH_P3 = 3 };
 struct Tile {
@@ -349,22 +378,22 @@ struct Pass1 {
   static constexpr int N1 = 16 * R1B, CPW = NT / R1B, IT = 16 / R1B, ES = Pair<T>::ES;
   static constexpr int ROWB = 2 * CPW * ES, CPR = ROWB / 16;   // bytes and 16-byte chunks per input row slice
 
-  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, int lane) {
+  // Shared-memory rows of a tile: [K even half][K odd half][V even half][V odd half], N1/2 rows of ROWB
+  // bytes each.  Row n1 of the transform input is row n1 of the even half for n1 < N1/2 and row
+  // N1-1-n1 of the odd half otherwise (the odd tokens run backwards).
+  static constexpr unsigned BOXB = (N1 / 2) * ROWB, TILEB = 4 * BOXB;
+  __device__ static int srow(int n1) { return n1 < N1 / 2 ? n1 : N1 / 2 + (N1 - 1 - n1); }
+  __device__ static void issue(const Params &P, const TmaMaps &M, const Tile &tl, float4 *buf, unsigned long long *bar) {
     const int N2 = P.N / N1;
     const int gcol = tl.unit * P.UC + tl.cb * 2 * CPW;
     const int head = gcol / P.head_dim, c = gcol - head * P.head_dim;
-    const long long hoff = (long long)head * P.stride_head_b + (long long)c * ES;
-    const char *kb = static_cast<const char *>(P.k) + hoff;
-    const char *vb = static_cast<const char *>(P.v) + hoff;
-    char *dst0 = reinterpret_cast<char *>(buf);
-#pragma unroll 8
-    for (int idx = lane; idx < 2 * N1 * CPR; idx += 32) {
-      const int m = idx / (N1 * CPR), rem = idx - m * (N1 * CPR);
-      const int row = rem / CPR, q = rem - row * CPR;
-      const int tok = perm_token(row * N2 + tl.a, P.N);
-      const char *src = (m ? vb : kb) + (long long)tok * P.stride_token_b + 16 * q;
-      cp_async16(dst0 + (m * N1 + row) * ROWB + 16 * q, src);
-    }
+    const int r_even = 2 * tl.a, r_odd = 2 * (N2 - 1 - tl.a) + 1;
+    char *dst = reinterpret_cast<char *>(buf);
+    mbar_expect_tx(bar, TILEB);
+    tma_load_4d(dst, &M.k, c, head, r_even, 0, bar);
+    tma_load_4d(dst + BOXB, &M.k, c, head, r_odd, 0, bar);
+    tma_load_4d(dst + 2 * BOXB, &M.v, c, head, r_even, 0, bar);
+    tma_load_4d(dst + 3 * BOXB, &M.v, c, head, r_odd, 0, bar);
   }
 
   __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
@@ -376,7 +405,7 @@ struct Pass1 {
     float2 aK = make_float2(0.f, 0.f), aV = make_float2(0.f, 0.f);
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
-      const int row = j + R1B * p;
+      const int row = srow(j + R1B * p);
       x[p].r = Pair<T>::ld(in + row * ROWB + cp * 2 * ES);
       x[p].i = Pair<T>::ld(in + (N1 + row) * ROWB + cp * 2 * ES);
       aK = pfma(x[p].r, x[p].r, aK);
@@ -421,25 +450,24 @@ struct Pass1 {
 
 // ------------------------------------------------------------------ pass 2
 // Tile (unit, x, cb): bins k1a = x and k1b = N1 - x (x = 0: k1 = 0 and k1 = N1/2, each its own
-// partner) of 2*CP channels.  Thread (cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2*CP)).
-// The second half starts PAD float4 later so that the two halves of a quarter warp fall into
-// different banks when a row is only 64 bytes.
+// partner) of 2*CP channels.  Thread (cp = tid % CP, j = (tid / CP) % R2B, hf = tid / (CP*R2B)): consecutive j
+// are consecutive rows, so a quarter warp reads 128 contiguous bytes even when a row is 64 bytes.
 template <int R2B>
 struct Pass2 {
   static constexpr int N2 = 16 * R2B, CP = NT / (2 * R2B), IT = 16 / R2B, NAB = R2B + 16;
-  static constexpr int PAD = CP < 8 ? 4 : 0, HALF = N2 * CP + PAD;
+  static constexpr int HALF = N2 * CP;
 
-  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, float4 *ab, float2 *chf, int lane) {
+  __device__ static void issue(const Params &P, const TmaMaps &M, const Tile &tl, float4 *buf, float4 *ab, float2 *chf,
+                               unsigned long long *bar, int lane) {
     const int N1 = P.N / N2;
     const int k1a = tl.a, k1b = tl.a == 0 ? N1 / 2 : N1 - tl.a;
-    const float2 *slot = slot_base(P, tl.unit);
-    const int col = tl.cb * 2 * CP;
-#pragma unroll 8
-    for (int idx = lane; idx < 2 * N2 * CP; idx += 32) {
-      const int hf = idx / (N2 * CP), rem = idx - hf * (N2 * CP);
-      const int n2 = rem / CP, cpi = rem - n2 * CP;
-      const int k1 = hf ? k1b : k1a;
-      cp_async16(buf + hf * HALF + rem, slot + ((size_t)k1 * N2 + n2) * P.UC + col + 2 * cpi);
+    if (lane == 0) {
+      const int row0 = (tl.unit % P.R) * N1;                 // first k1 row of the unit's ring slot
+      const int x0 = 2 * tl.cb * 2 * CP;                     // floats
+      fence_proxy_async();                                   // the rows were written through the generic proxy
+      mbar_expect_tx(bar, 2u * N2 * CP * (unsigned)sizeof(float4));
+      tma_load_3d(buf, &M.ws2, x0, 0, row0 + k1a, bar);
+      tma_load_3d(buf + HALF, &M.ws2, x0, 0, row0 + k1b, bar);
     }
     // per-tile twiddle factors: w_N^(k1*n2) = A[j] * B[p] for n2 = j + R2B*p
     const int ms = P.master_len / P.N;
@@ -460,7 +488,7 @@ struct Pass2 {
   __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
                                  const float2 *t2, const float4 *ab, const float2 *chf, int tid) {
     const int N1 = P.N / N2, N = P.N;
-    const int cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
+    const int cp = tid % CP, j = (tid / CP) % R2B, hf = tid / (CP * R2B);
     const bool self = tl.a == 0;
     const int k1 = hf ? (self ? N1 / 2 : N1 - tl.a) : tl.a;
     float4 *Sh = buf + hf * HALF;
@@ -587,15 +615,9 @@ struct Pass3 {
   static constexpr int LEFT = CPW >= 16 ? 1 : 16 / CPW;       // row sums a lane ends up with
   static constexpr int DUP = CPW > 16 ? CPW / 16 : 1;         // lanes that end up with the same row sum
 
-  __device__ static void issue(const Params &P, const Tile &tl, float4 *buf, int lane) {
-    const int N2 = P.N / N1;
-    const float2 *slot = slot_base(P, tl.unit);
-    const int col = tl.cb * 2 * CPW;
-#pragma unroll 8
-    for (int idx = lane; idx < N1 * CPW; idx += 32) {
-      const int k1 = idx / CPW, cpi = idx - k1 * CPW;
-      cp_async16(buf + idx, slot + ((size_t)k1 * N2 + tl.a) * P.UC + col + 2 * cpi);
-    }
+  __device__ static void issue(const Params &P, const TmaMaps &M, const Tile &tl, float4 *buf, unsigned long long *bar) {
+    mbar_expect_tx(bar, (unsigned)(N1 * CPW * sizeof(float4)));
+    tma_load_3d(buf, &M.ws3, 2 * tl.cb * 2 * CPW, tl.a, (tl.unit % P.R) * N1, bar);
   }
 
   __device__ static void compute(const Params &P, const Tile &tl, float4 *buf, const float4 *twb, int ntab,
@@ -693,7 +715,7 @@ struct Pass1S {
     float aK = 0.f, aV = 0.f;
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
-      const int row = j + R1B * p;
+      const int row = Pass1<T, R1B>::srow(j + R1B * p);
       x[p].x = One<T>::ld(in + row * ROWB + c * ES);
       x[p].y = One<T>::ld(in + (N1 + row) * ROWB + c * ES);
       aK = fmaf(x[p].x, x[p].x, aK);
@@ -985,15 +1007,16 @@ __device__ __forceinline__ void report_tile(const Params &P, const Tile &tl, int
 #define FC_FUSED_MINB 3
 #endif
 template <typename T, int R1B, int R2B, int ONE>
-__global__ void __launch_bounds__(Threads<ONE>::all, FC_FUSED_MINB) k_fused(const __grid_constant__ Params P) {
+__global__ void __launch_bounds__(Threads<ONE>::all, FC_FUSED_MINB) k_fused(const __grid_constant__ Params P,
+                                                                             const __grid_constant__ TmaMaps M) {
   using SM = Smem<R1B, R2B, ONE>;
   constexpr int NTC = Threads<ONE>::compute, NTH = Threads<ONE>::all;
   using P1 = Pass1<T, R1B>;
   using P2 = Pass2<R2B>;
   using P3 = Pass3<R1B>;
   constexpr int NTAB = SM::NTAB, N2 = SM::N2, NAB = SM::NAB;
-  extern __shared__ float4 smem4[];
-  float4 *bufs = smem4;                                           // [2][BUF4]
+  extern __shared__ __align__(1024) float4 smem4[];
+  float4 *bufs = smem4;                                           // [2][BUF4], TMA destinations (128-byte aligned)
   float4 *twb = smem4 + 2 * BUF4;                                 // [NTAB] exp(-2*pi*j*i/NTAB): broadcast float4, or float2 (ONE)
   float2 *tw1 = reinterpret_cast<float2 *>(twb);
   float2 *t2 = reinterpret_cast<float2 *>(reinterpret_cast<char *>(twb) + SM::tw_bytes);   // [N2] exp(-j*pi*k2/N2)
@@ -1013,7 +1036,7 @@ __global__ void __launch_bounds__(Threads<ONE>::all, FC_FUSED_MINB) k_fused(cons
   }
   for (int i = tid; i < N2; i += NTH) t2[i] = __ldg(P.master + (size_t)i * (P.master_len / (2 * N2)));
   if (tid == 0) {
-    mbar_init(&full[0], 64u); mbar_init(&full[1], 64u);     // per lane: one arrival after its copies, one plain
+    mbar_init(&full[0], 33u); mbar_init(&full[1], 33u);     // one per scheduler lane + the one that announces the bytes
     mbar_init(&done[0], (unsigned)NTC); mbar_init(&done[1], (unsigned)NTC);
   }
   __syncthreads();
@@ -1029,19 +1052,22 @@ __global__ void __launch_bounds__(Threads<ONE>::all, FC_FUSED_MINB) k_fused(cons
     unsigned long long n_tiles = 0, n_late = 0, s_back = 0, s_deps = 0, s_issue = 0;
     bool ok = true;
     unsigned k = 0;
+    // reports the tile in buffer bb if the compute warps have finished it (never blocks)
+    auto poll_report = [&](int bb) {
+      if (live[bb] && mbar_test(&done[bb], (held_k[bb] >> 1) & 1u)) {
+        report_tile<R1B>(P, held[bb], lane);
+        live[bb] = false;
+      }
+    };
     for (;; ++k) {
       const int b = (int)(k & 1u);
       const long long q0 = clock64();
-      if (live[b]) {                       // the tile that used this buffer two steps ago
-        if (!mbar_wait(&done[b], (held_k[b] >> 1) & 1u, P)) { ok = false; break; }
-        report_tile<R1B>(P, held[b], lane);
-        live[b] = false;
-      }
-      const long long q1 = clock64();
       const unsigned t = __shfl_sync(0xffffffffu, t_next, 0);
       const Tile tl = decode_tile(P, walk, t);
       if (tl.phase == PH_NONE) break;
       if (lane == 0) t_next = atomicAdd(&sc->tile_counter, 1u);      // answer is needed one tile from now
+      // 1. the tiles this one reads must be finished.  While waiting, keep reporting what the compute
+      //    warps finish here: it may be exactly what somebody (even this tile) is waiting for.
       const unsigned *dc = dep_counter(P, tl);
       if (dc != nullptr) {
         unsigned it = 0;
@@ -1050,11 +1076,8 @@ __global__ void __launch_bounds__(Threads<ONE>::all, FC_FUSED_MINB) k_fused(cons
           v = __shfl_sync(0xffffffffu, v, 0);
           if (v >= (unsigned)P.TPU) break;
           if (it == 0) ++n_late;
-          // the tile in the other buffer may be what somebody (even this tile) is waiting for
-          if (live[b ^ 1] && mbar_test(&done[b ^ 1], (held_k[b ^ 1] >> 1) & 1u)) {
-            report_tile<R1B>(P, held[b ^ 1], lane);
-            live[b ^ 1] = false;
-          }
+          poll_report(0);
+          poll_report(1);
           unsigned stop = 0u;
           if (lane == 0) {
             if (++it > P.spin_limit) { atomicExch(&sc->abort_flag, 1u); atomicOr(P.status, FC_DEV_FLAG_TIMEOUT); stop = 1u; }
@@ -1066,19 +1089,31 @@ __global__ void __launch_bounds__(Threads<ONE>::all, FC_FUSED_MINB) k_fused(cons
         }
         if (!ok) break;
       }
+      const long long q1 = clock64();
+      // 2. the buffer must be free: the tile that used it two steps ago is finished (and gets reported)
+      if (live[b]) {
+        if (!mbar_wait(&done[b], (held_k[b] >> 1) & 1u, P)) { ok = false; break; }
+        report_tile<R1B>(P, held[b], lane);
+        live[b] = false;
+      }
       const long long q2 = clock64();
+      // 3. descriptor, per-tile tables, then the tile itself through the TMA unit
       float4 *dst = bufs + b * BUF4;
       if (lane == 0) desc[b] = tl;
-      if (tl.phase == PH_P1) P1::issue(P, tl, dst, lane);
-      else if (tl.phase == PH_P2) P2::issue(P, tl, dst, ab + b * 2 * NAB, chf + b * 2, lane);
-      else P3::issue(P, tl, dst, lane);
+      if (tl.phase == PH_P2) {
+        P2::issue(P, M, tl, dst, ab + b * 2 * NAB, chf + b * 2, &full[b], lane);
+        if (lane == 0) stamp[b] = clock64();
+      } else if (lane == 0) {
+        fence_proxy_async();               // what the counters vouch for was written through the generic proxy
+        if (tl.phase == PH_P1) P1::issue(P, M, tl, dst, &full[b]);
+        else P3::issue(P, M, tl, dst, &full[b]);
+        stamp[b] = clock64();
+      }
       __syncwarp();
       __threadfence_block();
-      if (lane == 0) stamp[b] = clock64();
-      mbar_arrive_after_copies(&full[b]);
-      mbar_arrive(&full[b]);
-      s_back += (unsigned long long)(q1 - q0);
-      s_deps += (unsigned long long)(q2 - q1);
+      mbar_arrive(&full[b]);               // one per lane: descriptor and tables are written
+      s_deps += (unsigned long long)(q1 - q0);
+      s_back += (unsigned long long)(q2 - q1);
       s_issue += (unsigned long long)(clock64() - q2);
       held[b] = tl;
       held_k[b] = k;
@@ -1100,9 +1135,8 @@ __global__ void __launch_bounds__(Threads<ONE>::all, FC_FUSED_MINB) k_fused(cons
       __syncwarp();
       __threadfence_block();
       mbar_arrive(&full[b]);
-      mbar_arrive(&full[b]);
+      if (lane == 0) mbar_arrive(&full[b]);   // stands in for the arrival that announces a tile's bytes
     }
-    cp_async_wait<0>();
     if (lane == 0) {
       atomicAdd(&sc->stats[0], n_tiles);
       atomicAdd(&sc->stats[1], n_late);
@@ -1132,6 +1166,7 @@ __global__ void __launch_bounds__(Threads<ONE>::all, FC_FUSED_MINB) k_fused(cons
         else if (tl.phase == PH_P2) P2::compute(P, tl, buf, twb, NTAB, t2, ab + b * 2 * NAB, chf + b * 2, tid);
         else P3::compute(P, tl, buf, twb, NTAB, reinterpret_cast<double (*)[4]>(red[b]), tid);
       }
+      fence_proxy_async();                 // this thread wrote the buffer; the TMA unit writes it next
       mbar_arrive(&done[b]);               // this thread's part of the tile is stored, the buffer is free
       c_wait += (unsigned long long)(c1 - c0);
       c_ph[tl.phase] += (unsigned long long)(clock64() - c1);
