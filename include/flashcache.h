@@ -98,6 +98,15 @@ fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *launches);
  * it before fc_score_workspace_bytes. */
 fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_lag);
 
+/* enabled = 1: consecutive fc_select_compact calls on one stream may run concurrently (each
+ * uses a fraction of the GPU): a launch may begin once every block of the previous one has
+ * started, and does not finish before the previous one has, so anything enqueued after the
+ * last call still sees all of them complete.  Use it only when (a) nothing else is enqueued on
+ * the stream between the calls, and (b) the scores, budgets and offsets of all of them were
+ * produced before the first call, as in  score x L, allocate, select x L.  Default 0: every
+ * call waits for the one before it. */
+fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled);
+
 /* Running totals of the fused transform kernel since fc_create (diagnostic; synchronises the
  * device): out = { tiles processed, tiles whose inputs were not finished when they were looked
  * when the scheduler warp first looked, unused, clock cycles (thread 0 of every block, summed) inside

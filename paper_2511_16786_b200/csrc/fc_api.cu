@@ -53,6 +53,7 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->fused_enabled = 0;   // the separate-launch kernels are still faster; FC_FUSED=1 switches the fused kernel on
   h->fused_blocks_per_sm = 0;
   h->fused_lag = 1;
+  h->select_overlap = 0;
   if (const char *e = getenv("FC_FUSED_LAG")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_lag = v; }
   if (const char *e = getenv("FC_FUSED")) { const int v = atoi(e); if (v >= 0 && v <= 2) h->fused_enabled = v; }
   if (const char *e = getenv("FC_FUSED_BPS")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_blocks_per_sm = v; }
@@ -182,6 +183,12 @@ extern "C" fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_l
   if (!h || stage_lag < 1 || stage_lag > 4 || enabled < 0 || enabled > 2) return FC_ERR_INVALID_ARG;
   h->fused_enabled = enabled;
   h->fused_lag = stage_lag;
+  return FC_OK;
+}
+
+extern "C" fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled) {
+  if (!h) return FC_ERR_INVALID_ARG;
+  h->select_overlap = enabled ? 1 : 0;
   return FC_OK;
 }
 

@@ -178,8 +178,8 @@ constexpr int kSelKptMax = 16;      // scores per thread: 8 * 1024 * 16 = 131072
 // ascending indices, and their K/V rows are copied by the same block.
 // grid (kSelCluster * sequences in chunk, heads), cluster (kSelCluster, 1, 1).
 template <int kSelKpt>
-__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
-k_select_gather(const float *__restrict__ scores, long long T, SeqTable st, int b0,
+__device__ __forceinline__ void
+select_gather_body(const float *__restrict__ scores, long long T, const SeqTable &st, int b0,
                 const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
                 int *__restrict__ out_idx, long long cap, int *__restrict__ status,
                 const char *__restrict__ kin, const char *__restrict__ vin, long long stride_token_b,
@@ -187,8 +187,8 @@ k_select_gather(const float *__restrict__ scores, long long T, SeqTable st, int 
                 char *__restrict__ out_v) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
-  __shared__ int lhist[256];
-  __shared__ int ghist[4][256];          // cluster-wide histograms, one buffer per pass
+  __shared__ int lhist[4][256];          // this block's histograms, one per pass (read by the whole cluster)
+  __shared__ int ghist[256];             // cluster-wide histogram of the current pass
   __shared__ unsigned tot[kSelCluster];  // (ties << 16 | greater) of every block of the cluster
   __shared__ unsigned wsum[kSelThreads / 32];
   __shared__ unsigned s_prefix;
@@ -220,19 +220,17 @@ k_select_gather(const float *__restrict__ scores, long long T, SeqTable st, int 
 #pragma unroll
   for (int i = 0; i < kSelKpt; ++i) key[i] = (i < nv) ? score_key(sc[base + i]) : 0u;
 
-  for (int i = tid; i < 4 * 256; i += kSelThreads) (&ghist[0][0])[i] = 0;
+  for (int i = tid; i < 4 * 256; i += kSelThreads) (&lhist[0][0])[i] = 0;
   unsigned tau = 0;
   int need = 0;
   const bool take_all = (k == n);
   if (!take_all) {
-    cluster.sync();                                      // histograms are zero everywhere before remote adds
+    __syncthreads();                                     // the local histograms are zero
     unsigned prefix = 0, mask = 0;
     int krem = k;
 #pragma unroll 1
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
-      if (tid < 256) lhist[tid] = 0;
-      __syncthreads();
 #pragma unroll
       for (int i = 0; i < kSelKpt; ++i) {
         const bool m = (i < nv) && ((key[i] & mask) == prefix);
@@ -240,24 +238,22 @@ k_select_gather(const float *__restrict__ scores, long long T, SeqTable st, int 
         if (m) {
           const unsigned dgt = (key[i] >> shift) & 255u;
           const unsigned peers = __match_any_sync(act, dgt);
-          if (lane == __ffs(peers) - 1) atomicAdd(&lhist[dgt], __popc(peers));
+          if (lane == __ffs(peers) - 1) atomicAdd(&lhist[pass][dgt], __popc(peers));
         }
+      }
+      cluster.sync();                                    // every block's histogram of this pass is complete
+      if (tid < 256) {
+        int v = 0;
+#pragma unroll
+        for (unsigned rr = 0; rr < kSelCluster; ++rr) v += *cluster.map_shared_rank(&lhist[pass][tid], rr);
+        ghist[tid] = v;
       }
       __syncthreads();
-      if (tid < 256) {
-        const int v = lhist[tid];
-        if (v != 0) {
-#pragma unroll
-          for (unsigned rr = 0; rr < kSelCluster; ++rr)
-            atomicAdd(cluster.map_shared_rank(&ghist[pass][tid], rr), v);
-        }
-      }
-      cluster.sync();                                    // every block now holds the full histogram
       if (warp == 0) {
         // lane l owns bins 8l..8l+7; find the bin where the count from the top reaches krem
         int mine = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) mine += ghist[pass][8 * lane + i];
+        for (int i = 0; i < 8; ++i) mine += ghist[8 * lane + i];
         int above = mine;                                // inclusive suffix sum over lanes >= l
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -268,7 +264,7 @@ k_select_gather(const float *__restrict__ scores, long long T, SeqTable st, int 
         if (strictly_above < krem && krem <= above) {
           int cum = strictly_above, dsel = 8 * lane;
           for (int i = 7; i >= 0; --i) {
-            const int c = ghist[pass][8 * lane + i];
+            const int c = ghist[8 * lane + i];
             if (cum + c >= krem) { dsel = 8 * lane + i; break; }
             cum += c;
           }
@@ -358,6 +354,24 @@ k_select_gather(const float *__restrict__ scores, long long T, SeqTable st, int 
   }
 }
 
+// The kernel.  overlap != 0 (launched with the programmatic-serialisation attribute): the next
+// launch in the stream may start as soon as every block of this one has begun, and this grid
+// does not finish before its predecessor has, so "the last launch is complete" still means
+// "all of them are".
+template <int kSelKpt>
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
+k_select_gather(const float *__restrict__ scores, long long T, const __grid_constant__ SeqTable st, int b0,
+                const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
+                int *__restrict__ out_idx, long long cap, int *__restrict__ status,
+                const char *__restrict__ kin, const char *__restrict__ vin, long long stride_token_b,
+                long long stride_head_b, int row_bytes, int H, char *__restrict__ out_k,
+                char *__restrict__ out_v, int overlap) {
+  if (overlap) asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+  select_gather_body<kSelKpt>(scores, T, st, b0, budgets, out_offsets, out_idx, cap, status, kin, vin,
+                              stride_token_b, stride_head_b, row_bytes, H, out_k, out_v);
+  if (overlap) asm volatile("griddepcontrol.wait;\n" ::: "memory");
+}
+
 fc_status check_cu(const int32_t *cu, int batch) {
   if (!cu || batch < 0 || cu[0] != 0) return FC_ERR_INVALID_ARG;
   for (int b = 0; b < batch; ++b)
@@ -434,15 +448,29 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
     {
       ProfScope ps(h, FC_K_SELECT, st);
 #define FC_SEL_LAUNCH(KPT)                                                                              \
-  k_select_gather<KPT><<<dim3(kSelCluster * nseq, kv->num_heads), kSelThreads, 0, st>>>(                \
-      scores, T, tab, b0, budgets, reinterpret_cast<const long long *>(out_offsets), out_idx,           \
-      out_capacity_rows, h->status_word, static_cast<const char *>(kv->k),                              \
-      static_cast<const char *>(kv->v), kv->stride_token * es, kv->stride_head * es, kv->head_dim * es, \
-      kv->num_heads, static_cast<char *>(out_k), static_cast<char *>(out_v))
+  do {                                                                                                  \
+    cudaLaunchConfig_t lc = {};                                                                         \
+    lc.gridDim = dim3(kSelCluster * nseq, kv->num_heads);                                               \
+    lc.blockDim = dim3(kSelThreads);                                                                    \
+    lc.stream = st;                                                                                     \
+    cudaLaunchAttribute at[1];                                                                          \
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                      \
+    at[0].val.programmaticStreamSerializationAllowed = 1;                                               \
+    lc.attrs = at;                                                                                      \
+    lc.numAttrs = h->select_overlap ? 1 : 0;                                                            \
+    launch_err = cudaLaunchKernelEx(&lc, k_select_gather<KPT>, scores, (long long)T, tab, b0, budgets,   \
+        reinterpret_cast<const long long *>(out_offsets), out_idx, (long long)out_capacity_rows,        \
+        h->status_word, static_cast<const char *>(kv->k), static_cast<const char *>(kv->v),             \
+        (long long)(kv->stride_token * es), (long long)(kv->stride_head * es), (int)(kv->head_dim * es), \
+        (int)kv->num_heads, static_cast<char *>(out_k), static_cast<char *>(out_v),                     \
+        (int)h->select_overlap);                                                                        \
+  } while (0)
+      cudaError_t launch_err = cudaSuccess;
       if (per_thread <= 2) FC_SEL_LAUNCH(2);
       else if (per_thread <= 4) FC_SEL_LAUNCH(4);
       else if (per_thread <= 8) FC_SEL_LAUNCH(8);
       else FC_SEL_LAUNCH(16);
+      if (launch_err != cudaSuccess) return FC_ERR_CUDA;
 #undef FC_SEL_LAUNCH
     }
     if ((s = fc_after_launch(h)) != FC_OK) return s;
