@@ -98,6 +98,16 @@ fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *launches);
  * it before fc_score_workspace_bytes. */
 fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_lag);
 
+/* enabled = 1: fc_score_layer calls for power-of-two lengths of 1024..65536 tokens leave their
+ * work on the library's two internal streams instead of making `stream` wait for it, so that the
+ * next layer starts while the last kernels of this one drain.  Inputs are still taken in stream
+ * order (the internal streams wait for everything enqueued on `stream` before the call).  The
+ * scores and energies of such calls are ordered on a stream only by the next
+ * fc_allocate_budgets, fc_select_compact or fc_last_device_status call that is given that
+ * stream; read them earlier only after a device-wide synchronisation.  Default 0: every call
+ * is complete in stream order when it returns. */
+fc_status fc_set_score_overlap(fc_handle *h, int32_t enabled);
+
 /* enabled = 1: consecutive fc_select_compact calls on one stream may run concurrently (each
  * uses a fraction of the GPU): a launch may begin once every block of the previous one has
  * started, and does not finish before the previous one has, so anything enqueued after the

@@ -23,7 +23,7 @@ _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
     "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count",
-    "fc_set_group_bytes", "fc_set_select_overlap", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_end", "fc_describe_plan",
+    "fc_set_group_bytes", "fc_set_score_overlap", "fc_set_select_overlap", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact",
     "fc_static_scratch_bytes", "fc_score_layer_static",
@@ -63,6 +63,8 @@ def _load() -> ctypes.CDLL:
     lib.fc_launch_count.restype = c_uint64
     lib.fc_set_group_bytes.argtypes = [c_void_p, c_size_t]
     lib.fc_set_group_bytes.restype = c_int
+    lib.fc_set_score_overlap.argtypes = [c_void_p, c_int32]
+    lib.fc_set_score_overlap.restype = c_int
     lib.fc_set_select_overlap.argtypes = [c_void_p, c_int32]
     lib.fc_set_select_overlap.restype = c_int
     lib.fc_set_fused.argtypes = [c_void_p, c_int32, c_int32]
@@ -152,6 +154,10 @@ def fc_launch_count(handle) -> int:
 
 def fc_set_group_bytes(handle, nbytes: int) -> None:
     _check(_lib.fc_set_group_bytes(handle, int(nbytes)), "fc_set_group_bytes")
+
+
+def fc_set_score_overlap(handle, enabled: bool) -> None:
+    _check(_lib.fc_set_score_overlap(handle, 1 if enabled else 0), "fc_set_score_overlap")
 
 
 def fc_set_select_overlap(handle, enabled: bool) -> None:
@@ -262,7 +268,7 @@ class Compressor:
 
     def __init__(self, num_layers: int, num_heads: int, head_dim: int, cu_seqlens, dtype, rho: float,
                  gamma: float = 0.2, min_keep: int = 1, device: int = 0, group_bytes: int | None = None,
-                 select_overlap: bool = True):
+                 select_overlap: bool = True, score_overlap: bool = True):
         self.L, self.H, self.d = num_layers, num_heads, head_dim
         self.cu = [int(x) for x in cu_seqlens]
         self.B = len(self.cu) - 1
@@ -276,6 +282,8 @@ class Compressor:
             fc_set_group_bytes(self.handle, group_bytes)
         # compress() issues select x L back to back after score x L and allocate: the documented case
         fc_set_select_overlap(self.handle, select_overlap)
+        # score x L is followed by allocate (which joins the internal streams) before anything reads the scores
+        fc_set_score_overlap(self.handle, score_overlap)
         dev = self.device
         self.scores = torch.empty((self.L, self.H, max(self.T, 1)), dtype=torch.float32, device=dev)
         self.energy = torch.empty((self.L, self.B, 4), dtype=torch.float64, device=dev)

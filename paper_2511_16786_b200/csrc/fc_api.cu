@@ -54,6 +54,11 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->fused_blocks_per_sm = 0;
   h->fused_lag = 1;
   h->select_overlap = 0;
+  h->score_overlap = 0;
+  h->step = 0;
+  h->last_sig = -1;
+  h->pending_join = false;
+  for (int a = 0; a < 2; ++a) for (int b = 0; b < 2; ++b) h->ev_done[a][b] = nullptr;
   if (const char *e = getenv("FC_FUSED_LAG")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_lag = v; }
   if (const char *e = getenv("FC_FUSED")) { const int v = atoi(e); if (v >= 0 && v <= 2) h->fused_enabled = v; }
   if (const char *e = getenv("FC_FUSED_BPS")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_blocks_per_sm = v; }
@@ -63,8 +68,12 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   if (cudaMalloc(&h->master, (size_t)h->master_len * sizeof(float2)) != cudaSuccess ||
       cudaMalloc(&h->status_word, sizeof(int)) != cudaSuccess ||
       cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess ||
-      cudaMalloc(&h->done_counter, sizeof(unsigned)) != cudaSuccess ||
-      cudaMemset(h->done_counter, 0, sizeof(unsigned)) != cudaSuccess ||
+      cudaMalloc(&h->done_counter, 2 * sizeof(unsigned)) != cudaSuccess ||
+      cudaMemset(h->done_counter, 0, 2 * sizeof(unsigned)) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_done[0][0], cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_done[0][1], cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_done[1][0], cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_done[1][1], cudaEventDisableTiming) != cudaSuccess ||
       cudaMalloc(&h->fused_sched, sizeof(fused::Sched)) != cudaSuccess ||
       cudaMemset(h->fused_sched, 0, sizeof(fused::Sched)) != cudaSuccess ||
       cudaStreamCreateWithFlags(&h->aux[0], cudaStreamNonBlocking) != cudaSuccess ||
@@ -134,6 +143,8 @@ extern "C" void fc_destroy(fc_handle *h) {
   if (!h) return;
   free_prof(h);
   for (int i = 0; i < 2; ++i) {
+    if (h->aux[i]) cudaStreamSynchronize(h->aux[i]);
+    for (int a = 0; a < 2; ++a) if (h->ev_done[a][i]) cudaEventDestroy(h->ev_done[a][i]);
     if (h->aux[i]) cudaStreamDestroy(h->aux[i]);
     if (h->ev_join[i]) cudaEventDestroy(h->ev_join[i]);
   }
@@ -161,6 +172,10 @@ extern "C" const char *fc_status_string(fc_status s) {
 extern "C" fc_status fc_last_device_status(fc_handle *h, fc_stream stream) {
   if (!h) return FC_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  {
+    const fc_status fs = fc_flush_pending(h, st);
+    if (fs != FC_OK) return fs;
+  }
   FC_CUDA_TRY(cudaStreamSynchronize(st));
   int word = 0;
   FC_CUDA_TRY(cudaMemcpy(&word, h->status_word, sizeof(int), cudaMemcpyDeviceToHost));
@@ -189,6 +204,12 @@ extern "C" fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_l
 extern "C" fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled) {
   if (!h) return FC_ERR_INVALID_ARG;
   h->select_overlap = enabled ? 1 : 0;
+  return FC_OK;
+}
+
+extern "C" fc_status fc_set_score_overlap(fc_handle *h, int32_t enabled) {
+  if (!h) return FC_ERR_INVALID_ARG;
+  h->score_overlap = enabled ? 1 : 0;
   return FC_OK;
 }
 

@@ -46,6 +46,13 @@ struct fc_handle {
   int fused_blocks_per_sm; // 0 = as many as fit
   int fused_lag;           // stages between pass 1, pass 2 and pass 3 of a unit
   int select_overlap;      // 1: consecutive fc_select_compact launches may overlap (fc_set_select_overlap)
+  // fc_set_score_overlap: consecutive fc_score_layer calls keep running on the two internal streams
+  // without rejoining the caller's stream; the join is made by the next call that consumes their results
+  int score_overlap;
+  unsigned step;                 // specialised-path sequences scored so far (parity picks partial-sum buffers)
+  long long last_sig;            // (N, heads, head_dim) of the previous specialised-path step
+  bool pending_join;             // internal streams hold work the caller's stream has not waited for
+  cudaEvent_t ev_done[2][2];     // [step parity][internal stream]: that stream finished that step
 };
 
 // Kernel classes for fc_profile_begin.
@@ -302,6 +309,17 @@ __device__ __forceinline__ double warp_sum_d(double v) {
     cudaError_t e__ = (expr);                      \
     if (e__ != cudaSuccess) return FC_ERR_CUDA;    \
   } while (0)
+
+// Makes `st` wait for everything the internal streams were given (no-op when nothing is pending).
+inline fc_status fc_flush_pending(fc_handle *h, cudaStream_t st) {
+  if (!h->pending_join) return FC_OK;
+  for (int i = 0; i < 2; ++i) {
+    FC_CUDA_TRY(cudaEventRecord(h->ev_join[i], h->aux[i]));
+    FC_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_join[i], 0));
+  }
+  h->pending_join = false;
+  return FC_OK;
+}
 
 inline fc_status fc_after_launch(fc_handle *h) {
   h->launches++;

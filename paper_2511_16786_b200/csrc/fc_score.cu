@@ -526,6 +526,7 @@ FusedPlan plan_fused(const fc_handle *h, const SeqPlan &sp, int H, int d) {
 
 struct ScoreLayout {
   size_t off_ws, off_spec, off_hhat, off_hcol, off_part_tot, off_part_hi, total;
+  size_t part_tot_bytes, part_hi_bytes;   // one copy; the specialised path keeps two and alternates (step parity)
   size_t ws_buf_bytes;       // one group buffer; the fast path keeps two and alternates
   int heads_per_group;
 };
@@ -563,8 +564,10 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   L.off_hhat = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * sizeof(float2), 256) : 0;
   L.off_hcol = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * 8 * sizeof(float2), 256) : 0;
   const size_t slices = (size_t)num_heads * head_dim / 32;   // finest slicing any kernel variant uses
-  L.off_part_tot = off; off += align_up(slices * sp.N2 * 2 * sizeof(double), 256);
-  L.off_part_hi = off;  off += align_up((size_t)num_heads * sp.N2 * 2 * sizeof(double), 256);
+  L.part_tot_bytes = align_up(slices * sp.N2 * 2 * sizeof(double), 256);
+  L.part_hi_bytes = align_up((size_t)num_heads * sp.N2 * 2 * sizeof(double), 256);
+  L.off_part_tot = off; off += L.part_tot_bytes * (sp.fast ? 2 : 1);
+  L.off_part_hi = off;  off += L.part_hi_bytes * (sp.fast ? 2 : 1);
   L.total = off;
   return L;
 }
@@ -663,7 +666,7 @@ fc_status launch_fast_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, 
     const int H = kv->num_heads;
     fast::k_p3<R1B, CPW><<<dim3(N2, hg), CPW * R1B, sm1, st>>>(
         sp.N, N2, ncol_ws, ws, h->master, h->master_len, scores, h0, d, total_tokens, inv, phi,
-        h->done_counter, (unsigned)(N2 * H), part_tot, N2 * (H * d / (2 * CPW)), part_hi, N2 * H, energy_b);
+        h->done_counter + (h->step & 1u), (unsigned)(N2 * H), part_tot, N2 * (H * d / (2 * CPW)), part_hi, N2 * H, energy_b);
   }
   return fc_after_launch(h);
 }
@@ -811,12 +814,20 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   if (om < 0) om = 0;
   const int omega = (int)om;
 
+  fc_status s0 = FC_OK;
   float2 *ws = reinterpret_cast<float2 *>(wsb + L.off_ws);
   float2 *spec = reinterpret_cast<float2 *>(wsb + L.off_spec);
   float2 *hhat = reinterpret_cast<float2 *>(wsb + L.off_hhat);
   float2 *hcol = reinterpret_cast<float2 *>(wsb + L.off_hcol);
   double *part_tot = reinterpret_cast<double *>(wsb + L.off_part_tot);
   double *part_hi = reinterpret_cast<double *>(wsb + L.off_part_hi);
+  const bool separate_fast = sp.fast && !plan_fused(h, sp, H, d).ok;
+  if (separate_fast) {                 // consecutive steps alternate between two copies of the partial sums
+    part_tot = reinterpret_cast<double *>(wsb + L.off_part_tot + (h->step & 1u) * L.part_tot_bytes);
+    part_hi = reinterpret_cast<double *>(wsb + L.off_part_hi + (h->step & 1u) * L.part_hi_bytes);
+  } else {
+    if ((s0 = fc_flush_pending(h, st)) != FC_OK) return s0;   // this path works on the caller's stream
+  }
   const T *kp = static_cast<const T *>(kv->k) + (long long)start * kv->stride_token;
   const T *vp = static_cast<const T *>(kv->v) + (long long)start * kv->stride_token;
   const FftPlan p1 = make_plan(sp.N1);
@@ -856,9 +867,18 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   }
 
   if (sp.fast) {
+    const long long sig = (long long)N + ((long long)H << 20) + ((long long)d << 40);
     FC_CUDA_TRY(cudaEventRecord(h->ev_fork, st));
-    FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[0], h->ev_fork, 0));
-    FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[1], h->ev_fork, 0));
+    for (int i = 0; i < 2; ++i) {
+      FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[i], h->ev_fork, 0));
+      // the partial sums and the block counter of this parity were last used two steps ago: the other
+      // stream must be through with that step (this one is, by stream order)
+      if (h->step >= 2) FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[i], h->ev_done[h->step & 1u][1 - i], 0));
+      // a different shape carves the workspace differently: nothing of the previous step may be in flight
+      if (h->step >= 1 && sig != h->last_sig)
+        FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[i], h->ev_done[(h->step - 1) & 1u][1 - i], 0));
+    }
+    h->last_sig = sig;
   }
   size_t tot_slots = 0, hi_slots = 0;
   int group = 0;
@@ -913,9 +933,11 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     hi_slots += (size_t)sp.N2 * hg;
   }
   if (sp.fast) {
-    for (int i = 0; i < 2; ++i) {
-      FC_CUDA_TRY(cudaEventRecord(h->ev_join[i], h->aux[i]));
-      FC_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_join[i], 0));
+    for (int i = 0; i < 2; ++i) FC_CUDA_TRY(cudaEventRecord(h->ev_done[h->step & 1u][i], h->aux[i]));
+    h->step++;
+    h->pending_join = true;
+    if (!h->score_overlap) {           // default: the caller's stream waits for this call's work right away
+      if ((s = fc_flush_pending(h, st)) != FC_OK) return s;
     }
   }
   if (sp.fast) return FC_OK;          // the last pass-3 block of the sequence has written the energy sums

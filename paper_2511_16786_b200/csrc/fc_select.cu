@@ -395,6 +395,7 @@ extern "C" fc_status fc_allocate_budgets(fc_handle *h, const double *energy, int
   FC_CUDA_TRY(cudaGetDevice(&dev));
   if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if ((s = fc_flush_pending(h, st)) != FC_OK) return s;    // the energies may still be in flight on the internal streams
   const int L = num_layers;
   const size_t sm = (size_t)(6 * L) * sizeof(double) + (size_t)L * sizeof(int);
   for (int b0 = 0; b0 < batch; b0 += kSeqChunk) {
@@ -437,6 +438,7 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
   FC_CUDA_TRY(cudaGetDevice(&dev));
   if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if ((s = fc_flush_pending(h, st)) != FC_OK) return s;
   const long long T = kv->cu_seqlens[kv->batch];
   for (int b0 = 0; b0 < kv->batch; b0 += kSeqChunk) {
     const int nseq = kv->batch - b0 < kSeqChunk ? kv->batch - b0 : kSeqChunk;

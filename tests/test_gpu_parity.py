@@ -375,23 +375,25 @@ def test_config5_shape_reduced_ragged(fc):
     _compare_compress(fc, cfg)
 
 
-def test_overlapping_select_launches_give_the_same_cache(fc):
+def test_overlapping_launches_give_the_same_results(fc):
     from paper_2511_16786_b200.binding import Compressor
     cfg = S.scaled(S.paper_configs()["cfg2"], "cfg2_overlap", num_layers=12, seqlens=(4096, 1000))
     Kd, Vd = zip(*(S.make_layer(cfg, l, "cuda") for l in range(cfg.num_layers)))
     res = []
     for overlap in (False, True):
         comp = Compressor(cfg.num_layers, cfg.num_heads, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho,
-                          cfg.gamma, cfg.min_keep, select_overlap=overlap)
+                          cfg.gamma, cfg.min_keep, select_overlap=overlap, score_overlap=overlap)
         comp.out_k = comp.out_v = comp.out_idx = None
         for _ in range(3):                                    # repeated passes reuse the output buffers
             comp.compress(Kd, Vd)
         comp.check_device_status()
         off = comp.offsets.cpu()
         rows = [int(off[l, -1]) for l in range(cfg.num_layers)]
-        res.append(([comp.out_k[l, :rows[l]].cpu() for l in range(cfg.num_layers)],
+        res.append(([comp.scores.cpu().view(torch.int32)], [comp.energy.cpu().view(torch.int32)],
+                    [comp.budgets.cpu()]))
+        res[-1] = res[-1] + ([comp.out_k[l, :rows[l]].cpu() for l in range(cfg.num_layers)],
                     [comp.out_v[l, :rows[l]].cpu() for l in range(cfg.num_layers)],
-                    [comp.out_idx[l, :, :rows[l]].cpu() for l in range(cfg.num_layers)]))
+                    [comp.out_idx[l, :, :rows[l]].cpu() for l in range(cfg.num_layers)])
         comp.close()
     for a, b in zip(res[0], res[1]):
         for x, y in zip(a, b):
