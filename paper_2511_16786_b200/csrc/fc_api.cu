@@ -53,6 +53,8 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->fused_enabled = 0;   // the separate-launch kernels are still faster; FC_FUSED=1 switches the fused kernel on
   h->fused_blocks_per_sm = 0;
   h->fused_lag = 1;
+  h->fused_unit_shift = 20;
+  if (const char *e = getenv("FC_FUSED_UNIT_SHIFT")) { const int v = atoi(e); if (v >= 18 && v <= 23) h->fused_unit_shift = v; }
   h->select_overlap = 0;
   h->score_overlap = 0;
   h->step = 0;

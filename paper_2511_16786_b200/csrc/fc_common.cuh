@@ -45,6 +45,7 @@ struct fc_handle {
   int fused_enabled;       // 0 separate launches, 1 fused kernel (two packed columns per thread), 2 fused, one column per thread
   int fused_blocks_per_sm; // 0 = as many as fit
   int fused_lag;           // stages between pass 1, pass 2 and pass 3 of a unit
+  int fused_unit_shift;    // log2 of (unit columns x N): 20 = 8 MB units (developer knob FC_FUSED_UNIT_SHIFT)
   int select_overlap;      // 1: consecutive fc_select_compact launches may overlap (fc_set_select_overlap)
   // fc_set_score_overlap: consecutive fc_score_layer calls keep running on the two internal streams
   // without rejoining the caller's stream; the join is made by the next call that consumes their results

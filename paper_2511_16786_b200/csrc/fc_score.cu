@@ -501,7 +501,7 @@ FusedPlan plan_fused(const fc_handle *h, const SeqPlan &sp, int H, int d) {
   f.r2b = sp.N2 / 16;
   const int cpw = fused::NT / f.r1b, cp = fused::NT / (2 * f.r2b);
   const int min_uc = 2 * cpw > 2 * cp ? 2 * cpw : 2 * cp;
-  int uc = (1 << 20) / sp.N;                       // about 8 MB of intermediate per unit
+  int uc = (1 << h->fused_unit_shift) / sp.N;      // 2^20: about 8 MB of intermediate per unit
   if (uc < min_uc) uc = min_uc;
   while (uc > min_uc && (uc > d || d % uc != 0)) uc >>= 1;
   if (uc > d || d % uc != 0 || uc % (2 * cpw) != 0 || uc % (2 * cp) != 0) return f;
