@@ -329,23 +329,54 @@ class Compressor:
             self.out_v = torch.empty_like(self.out_k)
             self.out_idx = torch.empty((self.L, self.H, per_layer_capacity), dtype=torch.int32, device=dev)
 
-    def score(self, K_layers, V_layers):
+    # The per-layer calls below go straight to the C entry points with arguments that are marshalled
+    # once per set of tensors (views, pointers, the cu_seqlens array): the per-call Python work would
+    # otherwise cost more than the selection kernels it launches.
+    def _marshal(self, K_layers, V_layers):
+        key = tuple(k.data_ptr() for k in K_layers) + tuple(v.data_ptr() for v in V_layers)
+        if getattr(self, "_mkey", None) == key and self._m_out == (id(self.out_k), id(self._ws)):
+            return self._m
         ws = self._workspace(K_layers[0], V_layers[0])
+        self._outputs(self.capacity)
+        cu = _cu_array(self.cu)
+        views = [make_view(K_layers[l], V_layers[l], cu) for l in range(self.L)]
+        P = c_void_p
+        m = dict(
+            cu=cu, views=views, refs=[byref(v) for v in views],
+            ws=P(ws.data_ptr()), ws_bytes=ws.numel(),
+            scores=[P(self.scores[l].data_ptr()) for l in range(self.L)],
+            energy=[P(self.energy[l].data_ptr()) for l in range(self.L)],
+            budgets=[P(self.budgets[l].data_ptr()) for l in range(self.L)],
+            offsets=[P(self.offsets[l].data_ptr()) for l in range(self.L)],
+            out_k=[P(self.out_k[l].data_ptr()) for l in range(self.L)],
+            out_v=[P(self.out_v[l].data_ptr()) for l in range(self.L)],
+            out_idx=[P(self.out_idx[l].data_ptr()) for l in range(self.L)],
+            cap=int(self.out_k.shape[1]))
+        self._m, self._mkey, self._m_out = m, key, (id(self.out_k), id(self._ws))
+        return m
+
+    def score(self, K_layers, V_layers):
+        m = self._marshal(K_layers, V_layers)
+        st, h, gamma = _stream(), self.handle, c_double(self.gamma)
+        call = _lib.fc_score_layer
         for l in range(self.L):
-            fc_score_layer(self.handle, K_layers[l], V_layers[l], self.cu, self.gamma,
-                           self.scores[l], self.energy[l], ws)
+            rc = call(h, m["refs"][l], gamma, m["scores"][l], m["energy"][l], m["ws"], m["ws_bytes"], st)
+            if rc != FC_OK:
+                raise FlashCacheError(rc, "fc_score_layer")
 
     def allocate(self):
         fc_allocate_budgets(self.handle, self.energy, self.cu, self.rho, self.min_keep,
                             self.budgets, self.offsets)
 
     def select_compact(self, K_layers, V_layers):
-        ws = self._workspace(K_layers[0], V_layers[0])
-        self._outputs(self.capacity)
+        m = self._marshal(K_layers, V_layers)
+        st, h = _stream(), self.handle
+        call = _lib.fc_select_compact
         for l in range(self.L):
-            fc_select_compact(self.handle, K_layers[l], V_layers[l], self.cu, self.scores[l],
-                              self.budgets[l], self.offsets[l], self.out_k[l], self.out_v[l],
-                              self.out_idx[l], ws)
+            rc = call(h, m["refs"][l], m["scores"][l], m["budgets"][l], m["offsets"][l], m["out_k"][l],
+                      m["out_v"][l], m["out_idx"][l], m["cap"], m["ws"], m["ws_bytes"], st)
+            if rc != FC_OK:
+                raise FlashCacheError(rc, "fc_select_compact")
 
     def compress(self, K_layers, V_layers):
         self.score(K_layers, V_layers)
