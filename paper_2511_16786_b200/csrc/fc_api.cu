@@ -18,6 +18,17 @@ __global__ void k_fill_master(float2 *master, int len) {
 
 }  // namespace
 
+static bool create_streams(fc_handle *h) {
+  for (int i = 0; i < FC_MAX_AUX; ++i) {
+    if (cudaStreamCreateWithFlags(&h->aux[i], cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_join[i], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_done[0][i], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_done[1][i], cudaEventDisableTiming) != cudaSuccess)
+      return false;
+  }
+  return true;
+}
+
 extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) {
   if (!out) return FC_ERR_INVALID_ARG;
   *out = nullptr;
@@ -42,8 +53,10 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   if (const char *e = getenv("FC_TUNE_CPW")) { const int v = atoi(e); if (v == 16 || v == 32) h->tune_cpw = v; }
   if (const char *e = getenv("FC_TUNE_CP")) { const int v = atoi(e); if (v == 4 || v == 8) h->tune_cp = v; }
   h->launches = 0;
-  h->aux[0] = h->aux[1] = nullptr;
-  h->ev_fork = h->ev_join[0] = h->ev_join[1] = nullptr;
+  h->num_aux = 2;
+  if (const char *e = getenv("FC_NUM_AUX")) { const int v = atoi(e); if (v >= 1 && v <= FC_MAX_AUX) h->num_aux = v; }
+  h->ev_fork = nullptr;
+  for (int i = 0; i < FC_MAX_AUX; ++i) { h->aux[i] = nullptr; h->ev_join[i] = nullptr; }
   h->prof_class = FC_K_NONE;
   h->prof_events = nullptr;
   h->prof_cap = 0;
@@ -60,7 +73,7 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->step = 0;
   h->last_sig = -1;
   h->pending_join = false;
-  for (int a = 0; a < 2; ++a) for (int b = 0; b < 2; ++b) h->ev_done[a][b] = nullptr;
+  for (int a = 0; a < 2; ++a) for (int b = 0; b < FC_MAX_AUX; ++b) h->ev_done[a][b] = nullptr;
   if (const char *e = getenv("FC_FUSED_LAG")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_lag = v; }
   if (const char *e = getenv("FC_FUSED")) { const int v = atoi(e); if (v >= 0 && v <= 2) h->fused_enabled = v; }
   if (const char *e = getenv("FC_FUSED_BPS")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_blocks_per_sm = v; }
@@ -72,17 +85,10 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
       cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess ||
       cudaMalloc(&h->done_counter, 2 * sizeof(unsigned)) != cudaSuccess ||
       cudaMemset(h->done_counter, 0, 2 * sizeof(unsigned)) != cudaSuccess ||
-      cudaEventCreateWithFlags(&h->ev_done[0][0], cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&h->ev_done[0][1], cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&h->ev_done[1][0], cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&h->ev_done[1][1], cudaEventDisableTiming) != cudaSuccess ||
       cudaMalloc(&h->fused_sched, sizeof(fused::Sched)) != cudaSuccess ||
       cudaMemset(h->fused_sched, 0, sizeof(fused::Sched)) != cudaSuccess ||
-      cudaStreamCreateWithFlags(&h->aux[0], cudaStreamNonBlocking) != cudaSuccess ||
-      cudaStreamCreateWithFlags(&h->aux[1], cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&h->ev_join[0], cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&h->ev_join[1], cudaEventDisableTiming) != cudaSuccess) {
+      !create_streams(h)) {
     fc_destroy(h);
     return FC_ERR_CUDA;
   }
@@ -144,7 +150,7 @@ extern "C" fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *la
 extern "C" void fc_destroy(fc_handle *h) {
   if (!h) return;
   free_prof(h);
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < FC_MAX_AUX; ++i) {
     if (h->aux[i]) cudaStreamSynchronize(h->aux[i]);
     for (int a = 0; a < 2; ++a) if (h->ev_done[a][i]) cudaEventDestroy(h->ev_done[a][i]);
     if (h->aux[i]) cudaStreamDestroy(h->aux[i]);

@@ -13,6 +13,7 @@
 #include "../../include/flashcache.h"
 
 #define FC_MAX_STAGES 4
+#define FC_MAX_AUX 4     // internal streams a handle may use
 
 // Bits of the device status word.
 #define FC_DEV_FLAG_INTERNAL 1
@@ -29,10 +30,11 @@ struct fc_handle {
   int tune_cpw, tune_cp;   // tile widths of the specialised kernels (channel pairs), see fc_create
   int num_sms;
   unsigned long long launches;
-  // two internal streams: consecutive head groups of one fc_score_layer call are
-  // transformed concurrently on alternating streams and workspace halves
-  cudaStream_t aux[2];
-  cudaEvent_t ev_fork, ev_join[2];
+  // internal streams: consecutive head groups of one fc_score_layer call are transformed
+  // concurrently, round robin over the streams, each with its own workspace buffer
+  cudaStream_t aux[FC_MAX_AUX];
+  int num_aux;             // how many of them are used (2 by default, FC_NUM_AUX)
+  cudaEvent_t ev_fork, ev_join[FC_MAX_AUX];
   // optional per-kernel-class timing (fc_profile_begin / fc_profile_end)
   int prof_class;
   cudaEvent_t *prof_events;   // pairs
@@ -53,7 +55,7 @@ struct fc_handle {
   unsigned step;                 // specialised-path sequences scored so far (parity picks partial-sum buffers)
   long long last_sig;            // (N, heads, head_dim) of the previous specialised-path step
   bool pending_join;             // internal streams hold work the caller's stream has not waited for
-  cudaEvent_t ev_done[2][2];     // [step parity][internal stream]: that stream finished that step
+  cudaEvent_t ev_done[2][FC_MAX_AUX];   // [step parity][internal stream]: that stream finished that step
 };
 
 // Kernel classes for fc_profile_begin.
@@ -314,7 +316,7 @@ __device__ __forceinline__ double warp_sum_d(double v) {
 // Makes `st` wait for everything the internal streams were given (no-op when nothing is pending).
 inline fc_status fc_flush_pending(fc_handle *h, cudaStream_t st) {
   if (!h->pending_join) return FC_OK;
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < h->num_aux; ++i) {
     FC_CUDA_TRY(cudaEventRecord(h->ev_join[i], h->aux[i]));
     FC_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_join[i], 0));
   }

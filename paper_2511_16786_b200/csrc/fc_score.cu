@@ -554,12 +554,12 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   if (hg < 1) hg = 1;
   if (hg > num_heads) hg = num_heads;
   int groups = (num_heads + hg - 1) / hg;
-  if (sp.fast && groups < 2 && num_heads >= 2) groups = 2;     // keep both internal streams busy
+  if (sp.fast && groups < h->num_aux && num_heads >= h->num_aux) groups = h->num_aux;   // keep every internal stream busy
   hg = (num_heads + groups - 1) / groups;                      // balanced groups
   L.heads_per_group = hg;
   L.ws_buf_bytes = align_up(per_head * hg, 256);
   size_t off = 0;
-  L.off_ws = off;       off += L.ws_buf_bytes * (sp.fast ? 2 : 1);
+  L.off_ws = off;       off += L.ws_buf_bytes * (sp.fast ? h->num_aux : 1);
   L.off_spec = off;     off += sp.bluestein ? align_up((size_t)sp.N * head_dim * hg * sizeof(float2), 256) : 0;
   L.off_hhat = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * sizeof(float2), 256) : 0;
   L.off_hcol = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * 8 * sizeof(float2), 256) : 0;
@@ -869,14 +869,17 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   if (sp.fast) {
     const long long sig = (long long)N + ((long long)H << 20) + ((long long)d << 40);
     FC_CUDA_TRY(cudaEventRecord(h->ev_fork, st));
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < h->num_aux; ++i) {
       FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[i], h->ev_fork, 0));
-      // the partial sums and the block counter of this parity were last used two steps ago: the other
-      // stream must be through with that step (this one is, by stream order)
-      if (h->step >= 2) FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[i], h->ev_done[h->step & 1u][1 - i], 0));
-      // a different shape carves the workspace differently: nothing of the previous step may be in flight
-      if (h->step >= 1 && sig != h->last_sig)
-        FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[i], h->ev_done[(h->step - 1) & 1u][1 - i], 0));
+      for (int o = 0; o < h->num_aux; ++o) {
+        if (o == i) continue;
+        // the partial sums and the block counter of this parity were last used two steps ago: the other
+        // streams must be through with that step (this one is, by stream order)
+        if (h->step >= 2) FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[i], h->ev_done[h->step & 1u][o], 0));
+        // a different shape carves the workspace differently: nothing of the previous step may be in flight
+        if (h->step >= 1 && sig != h->last_sig)
+          FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[i], h->ev_done[(h->step - 1) & 1u][o], 0));
+      }
     }
     h->last_sig = sig;
   }
@@ -889,8 +892,9 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     double *phi = part_hi + 2 * hi_slots;
     const size_t sm3 = smem_pass13(sp, sp.cs);
     if (sp.fast) {
-      float2 *wsg = reinterpret_cast<float2 *>(wsb + L.off_ws + (size_t)(group & 1) * L.ws_buf_bytes);
-      if ((s = launch_fast<T>(h, h->aux[group & 1], kv, kp, vp, sp, h0, hg, omega, wsg, ptot, phi,
+      const int si = group % h->num_aux;
+      float2 *wsg = reinterpret_cast<float2 *>(wsb + L.off_ws + (size_t)si * L.ws_buf_bytes);
+      if ((s = launch_fast<T>(h, h->aux[si], kv, kp, vp, sp, h0, hg, omega, wsg, ptot, phi,
                               scores + start, total_tokens, part_tot, part_hi, energy_b)) != FC_OK) return s;
     } else if (!sp.bluestein) {
       KvLoader<T, false> ld{kp, vp, kv->stride_token, kv->stride_head, h0, d, N, 0.f, 0.f};
@@ -933,7 +937,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     hi_slots += (size_t)sp.N2 * hg;
   }
   if (sp.fast) {
-    for (int i = 0; i < 2; ++i) FC_CUDA_TRY(cudaEventRecord(h->ev_done[h->step & 1u][i], h->aux[i]));
+    for (int i = 0; i < h->num_aux; ++i) FC_CUDA_TRY(cudaEventRecord(h->ev_done[h->step & 1u][i], h->aux[i]));
     h->step++;
     h->pending_join = true;
     if (!h->score_overlap) {           // default: the caller's stream waits for this call's work right away
