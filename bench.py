@@ -270,8 +270,11 @@ def main():
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     launches0 = binding.fc_launch_count(comp.handle)
+    # inside the timed region every 7th launch of the dominant kernel is bracketed by an event pair
+    prof_stride = 7
+    binding.fc_profile_stride(comp.handle, prof_stride)
     binding.fc_profile_begin(comp.handle, binding.KERNEL_CLASSES[dominant],
-                             max(1, shares[dominant]["launches"]) * args.steps + 8)
+                             max(1, shares[dominant]["launches"]) * args.steps // prof_stride + 8)
     t_wall0 = time.time()
     ev0.record()
     for _ in range(args.steps):
@@ -294,7 +297,9 @@ def main():
     props = torch.cuda.get_device_properties(dev)
     alu_peak = props.multi_processor_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # TFLOP/s
     d_acc = acc[dominant]
-    dom_s = dom_ms / 1000.0 / max(1, args.steps)            # device seconds of that class per step
+    launches_per_step = max(1, shares[dominant]["launches"])
+    avg_launch_s = dom_ms / 1000.0 / max(1, dom_launches)   # average over the sampled launches of the timed region
+    dom_s = avg_launch_s * launches_per_step                # device seconds of that class per step
     t_alu = d_acc["flops"] / (alu_peak * 1e12)
     t_hbm = d_acc["bytes"] / (peaks["hbm_gbs"] * 1e9)
     if t_alu >= t_hbm:
@@ -303,7 +308,7 @@ def main():
         roof = dict(bound="hbm", achieved=d_acc["bytes"] / dom_s / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((args.config, dominant))
-    roof.update(kernel=dominant, launches_per_step=dom_launches / max(1, args.steps),
+    roof.update(kernel=dominant, launches_per_step=launches_per_step, launches_timed=dom_launches,
                 avg_launch_us=1000.0 * dom_ms / max(1, dom_launches), peak_source=(
                     "%d SMs x %d FP32 lanes x 2 x %.0f MHz" % (props.multi_processor_count, FP32_LANES_PER_SM,
                                                               peaks["sm_max_mhz"])

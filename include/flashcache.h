@@ -88,6 +88,9 @@ uint64_t fc_launch_count(const fc_handle *h);
  * fc_profile_end waits for the recorded events and returns the summed device
  * time in milliseconds and the number of launches timed. */
 fc_status fc_profile_begin(fc_handle *h, int32_t kernel_class, int32_t max_launches);
+/* Time only every stride-th launch of the class (default 1): the event pairs cost a little and keep
+ * neighbouring launches from overlapping, so a sample disturbs a timed region less. */
+fc_status fc_profile_stride(fc_handle *h, int32_t stride);
 fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *launches);
 
 /* Chooses how power-of-two sequences of 4096..65536 tokens are transformed: enabled = 0 (default)

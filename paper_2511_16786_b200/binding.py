@@ -23,7 +23,7 @@ _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
     "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count",
-    "fc_set_group_bytes", "fc_set_score_overlap", "fc_set_select_overlap", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_end", "fc_describe_plan",
+    "fc_set_group_bytes", "fc_set_score_overlap", "fc_set_select_overlap", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact",
     "fc_static_scratch_bytes", "fc_score_layer_static",
@@ -73,6 +73,8 @@ def _load() -> ctypes.CDLL:
     lib.fc_fused_stats.restype = c_int
     lib.fc_profile_begin.argtypes = [c_void_p, c_int32, c_int32]
     lib.fc_profile_begin.restype = c_int
+    lib.fc_profile_stride.argtypes = [c_void_p, c_int32]
+    lib.fc_profile_stride.restype = c_int
     lib.fc_profile_end.argtypes = [c_void_p, POINTER(c_double), POINTER(c_uint64)]
     lib.fc_profile_end.restype = c_int
     lib.fc_describe_plan.argtypes = [c_void_p, c_int32, POINTER(c_int32)]
@@ -183,6 +185,10 @@ KERNEL_CLASSES = {"pass1": 1, "pass2": 2, "pass3": 3, "select": 4, "gather": 5, 
 
 def fc_profile_begin(handle, kernel_class: int, max_launches: int = 16384) -> None:
     _check(_lib.fc_profile_begin(handle, int(kernel_class), int(max_launches)), "fc_profile_begin")
+
+
+def fc_profile_stride(handle, stride: int) -> None:
+    _check(_lib.fc_profile_stride(handle, int(stride)), "fc_profile_stride")
 
 
 def fc_profile_end(handle):

@@ -61,6 +61,8 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->prof_events = nullptr;
   h->prof_cap = 0;
   h->prof_used = 0;
+  h->prof_stride = 1;
+  h->prof_seen = 0;
   h->generic_only = false;
   h->fused_sched = nullptr;
   h->fused_enabled = 0;   // the separate-launch kernels are still faster; FC_FUSED=1 switches the fused kernel on
@@ -125,7 +127,14 @@ extern "C" fc_status fc_profile_begin(fc_handle *h, int32_t kernel_class, int32_
   }
   h->prof_cap = max_launches;
   h->prof_used = 0;
+  h->prof_seen = 0;
   h->prof_class = kernel_class;
+  return FC_OK;
+}
+
+extern "C" fc_status fc_profile_stride(fc_handle *h, int32_t stride) {
+  if (!h || stride < 1) return FC_ERR_INVALID_ARG;
+  h->prof_stride = stride;
   return FC_OK;
 }
 

@@ -39,6 +39,7 @@ struct fc_handle {
   int prof_class;
   cudaEvent_t *prof_events;   // pairs
   int prof_cap, prof_used;
+  int prof_stride, prof_seen;  // every prof_stride-th launch of the class is timed
   // true only for the stack handle of fc_score_layer_static: every length takes the generic
   // single-stream kernels (no internal streams or events exist there)
   bool generic_only;
@@ -67,7 +68,7 @@ struct ProfScope {
   cudaStream_t st;
   bool on;
   ProfScope(fc_handle *h_, int cls, cudaStream_t st_) : h(h_), st(st_) {
-    on = h->prof_class == cls && h->prof_used < h->prof_cap;
+    on = h->prof_class == cls && h->prof_used < h->prof_cap && (h->prof_seen++ % h->prof_stride) == 0;
     if (on) cudaEventRecord(h->prof_events[2 * h->prof_used], st);
   }
   ~ProfScope() {
