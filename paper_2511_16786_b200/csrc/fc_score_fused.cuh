@@ -12,7 +12,7 @@
 //    before it starts.  The intermediates live in a ring of unit slots that stays in L2.
 //  * every tile is 4096 complex points = 2048 float4 (32 KB), processed by the 128 threads of
 //    four compute warps; a fifth (scheduler) warp asks for tile numbers, waits for the tiles
-//    they depend on, fills the second shared-memory buffer with cp.async while the current
+//    they depend on, fills the second shared-memory buffer through the TMA unit while the current
 //    one is transformed in place, and reports finished tiles, so the compute warps only ever
 //    wait for a full buffer (mbarrier).
 //  * pass 3 writes one partial score per 2*CPW channels; the block that delivers the last
@@ -231,14 +231,6 @@ __device__ __forceinline__ void dftp(c2 (&x)[R]) {
 }
 
 // ------------------------------------------------------------------ memory helpers
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
-  const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
-
 // barrier of the four compute warps (the scheduler warp never joins it)
 __device__ __forceinline__ void bar_compute() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
 
@@ -936,11 +928,6 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
   asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}\n"
                ::"r"((unsigned)__cvta_generic_to_shared(bar)) : "memory");
 }
-// arrives once all cp.async copies this thread has issued so far have landed (counted in the init value)
-__device__ __forceinline__ void mbar_arrive_after_copies(unsigned long long *bar) {
-  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n"
-               ::"r"((unsigned)__cvta_generic_to_shared(bar)) : "memory");
-}
 __device__ __forceinline__ bool mbar_test(unsigned long long *bar, unsigned parity) {
   unsigned ok;
   asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
@@ -961,7 +948,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
 
 // ------------------------------------------------------------------ the kernel
 // Block = 4 compute warps + 1 scheduler warp.  The scheduler warp takes tile numbers, waits for
-// the tiles they depend on, fills one of two shared-memory buffers with cp.async and reports
+// the tiles they depend on, fills one of two shared-memory buffers with tiled TMA loads and reports
 // finished tiles; the compute warps only ever wait for a full buffer.
 // ONE = 0: two packed columns per thread, 128 compute threads; ONE = 1: one column per thread, 256.
 template <int ONE> struct Threads { static constexpr int compute = ONE ? NTC1 : NT, all = compute + 32; };
