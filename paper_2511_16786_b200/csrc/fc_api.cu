@@ -82,6 +82,17 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return FC_ERR_CUDA; }
   h->num_sms = prop.multiProcessorCount;
+  h->l2_persist = 1;
+  if (const char *e = getenv("FC_L2_PERSIST")) h->l2_persist = atoi(e) != 0 ? 1 : 0;
+  h->persist_max = (size_t)prop.persistingL2CacheMaxSize;
+  h->window_max = (size_t)prop.accessPolicyMaxWindowSize;
+  for (int i = 0; i < FC_MAX_AUX; ++i) { h->window_base[i] = nullptr; h->window_bytes[i] = 0; }
+  // part of L2 may be set aside for persisting lines: a limit of this process's context, gone with it
+  if (h->l2_persist && h->persist_max > 0 &&
+      cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->persist_max) != cudaSuccess) {
+    cudaGetLastError();
+    h->l2_persist = 0;
+  }
   if (cudaMalloc(&h->master, (size_t)h->master_len * sizeof(float2)) != cudaSuccess ||
       cudaMalloc(&h->status_word, sizeof(int)) != cudaSuccess ||
       cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess ||

@@ -29,6 +29,12 @@ struct fc_handle {
   size_t group_bytes;
   int tune_cpw, tune_cp;   // tile widths of the specialised kernels (channel pairs), see fc_create
   int num_sms;
+  // L2 residency of the transform intermediates: the per-stream workspace buffers are declared a
+  // persisting access window on the internal streams (0 switches it off, FC_L2_PERSIST)
+  int l2_persist;
+  size_t persist_max, window_max;      // device limits (bytes)
+  const void *window_base[FC_MAX_AUX]; // what each internal stream's window was last set to
+  size_t window_bytes[FC_MAX_AUX];
   unsigned long long launches;
   // internal streams: consecutive head groups of one fc_score_layer call are transformed
   // concurrently, round robin over the streams, each with its own workspace buffer

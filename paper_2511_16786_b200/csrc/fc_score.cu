@@ -866,6 +866,28 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
   }
 
+  if (sp.fast && h->l2_persist && L.ws_buf_bytes <= h->window_max &&
+      L.ws_buf_bytes * (size_t)h->num_aux <= h->persist_max) {
+    // keep each stream's intermediate in the persisting part of L2; everything else these streams touch
+    // (the K/V rows, the scores) streams through
+    for (int i = 0; i < h->num_aux; ++i) {
+      const char *base = wsb + L.off_ws + (size_t)i * L.ws_buf_bytes;
+      if (h->window_base[i] == base && h->window_bytes[i] == L.ws_buf_bytes) continue;
+      cudaStreamAttrValue av = {};
+      av.accessPolicyWindow.base_ptr = const_cast<char *>(base);
+      av.accessPolicyWindow.num_bytes = L.ws_buf_bytes;
+      av.accessPolicyWindow.hitRatio = 1.0f;
+      av.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+      av.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+      if (cudaStreamSetAttribute(h->aux[i], cudaStreamAttributeAccessPolicyWindow, &av) != cudaSuccess) {
+        cudaGetLastError();
+        h->l2_persist = 0;               // not supported here: never try again
+        break;
+      }
+      h->window_base[i] = base;
+      h->window_bytes[i] = L.ws_buf_bytes;
+    }
+  }
   if (sp.fast) {
     const long long sig = (long long)N + ((long long)H << 20) + ((long long)d << 40);
     FC_CUDA_TRY(cudaEventRecord(h->ev_fork, st));
