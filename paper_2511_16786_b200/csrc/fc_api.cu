@@ -87,12 +87,7 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->persist_max = (size_t)prop.persistingL2CacheMaxSize;
   h->window_max = (size_t)prop.accessPolicyMaxWindowSize;
   for (int i = 0; i < FC_MAX_AUX; ++i) { h->window_base[i] = nullptr; h->window_bytes[i] = 0; }
-  // part of L2 may be set aside for persisting lines: a limit of this process's context, gone with it
-  if (h->l2_persist && h->persist_max > 0 &&
-      cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->persist_max) != cudaSuccess) {
-    cudaGetLastError();
-    h->l2_persist = 0;
-  }
+  h->persist_on = 0;
   if (cudaMalloc(&h->master, (size_t)h->master_len * sizeof(float2)) != cudaSuccess ||
       cudaMalloc(&h->status_word, sizeof(int)) != cudaSuccess ||
       cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess ||
@@ -170,6 +165,7 @@ extern "C" fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *la
 extern "C" void fc_destroy(fc_handle *h) {
   if (!h) return;
   free_prof(h);
+  if (h->persist_on) { cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, 0); cudaCtxResetPersistingL2Cache(); }
   for (int i = 0; i < FC_MAX_AUX; ++i) {
     if (h->aux[i]) cudaStreamSynchronize(h->aux[i]);
     for (int a = 0; a < 2; ++a) if (h->ev_done[a][i]) cudaEventDestroy(h->ev_done[a][i]);

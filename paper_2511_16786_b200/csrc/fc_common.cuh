@@ -32,6 +32,7 @@ struct fc_handle {
   // L2 residency of the transform intermediates: the per-stream workspace buffers are declared a
   // persisting access window on the internal streams (0 switches it off, FC_L2_PERSIST)
   int l2_persist;
+  int persist_on;                      // the context's persisting-L2 set-aside is currently claimed by this handle
   size_t persist_max, window_max;      // device limits (bytes)
   const void *window_base[FC_MAX_AUX]; // what each internal stream's window was last set to
   size_t window_bytes[FC_MAX_AUX];

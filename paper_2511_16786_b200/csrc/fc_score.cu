@@ -866,8 +866,20 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
   }
 
-  if (sp.fast && h->l2_persist && L.ws_buf_bytes <= h->window_max &&
-      L.ws_buf_bytes * (size_t)h->num_aux <= h->persist_max) {
+  // The persisting part of L2 is a set-aside of this process's context (gone with it): claim it while the
+  // specialised path runs, give it back to ordinary caching when another path takes over.
+  const bool want_persist = separate_fast && h->l2_persist && L.ws_buf_bytes <= h->window_max &&
+                            L.ws_buf_bytes * (size_t)h->num_aux <= h->persist_max;
+  if (want_persist != (h->persist_on != 0)) {
+    if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want_persist ? h->persist_max : 0) != cudaSuccess) {
+      cudaGetLastError();
+      h->l2_persist = 0;
+    } else {
+      h->persist_on = want_persist ? 1 : 0;
+      if (!want_persist) cudaCtxResetPersistingL2Cache();
+    }
+  }
+  if (want_persist && h->persist_on) {
     // keep each stream's intermediate in the persisting part of L2; everything else these streams touch
     // (the K/V rows, the scores) streams through
     for (int i = 0; i < h->num_aux; ++i) {
