@@ -231,8 +231,10 @@ fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const float *sco
  *
  * Limits: every sequence length <= 4096 (else FC_ERR_UNSUPPORTED), and the scratch the view
  * needs (what fc_score_workspace_bytes would report with one head per transform group)
- * <= FC_STATIC_SCRATCH_BYTES (else FC_ERR_WORKSPACE).  At head_dim 128 that admits
- * power-of-two lengths up to 4096 and any other length up to 2048.
+ * <= FC_STATIC_SCRATCH_BYTES (else FC_ERR_WORKSPACE).  A power-of-two length N needs
+ * N * head_dim * 8 bytes plus a few KiB (at head_dim 128: up to 4096; at 256: up to 2048);
+ * any other length up to 4096 fits at every head_dim (a head is transformed 32 columns at a
+ * time).
  *
  * First call on a device: looks up the device addresses of the arrays, fills the twiddle
  * table and waits for the device once (cudaDeviceSynchronize).  Make that first call with

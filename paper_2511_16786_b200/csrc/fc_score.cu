@@ -340,7 +340,11 @@ __global__ void __launch_bounds__(kThreads)
 k_pass3(FftPlan plan, int N2, int N, int ncol_ws, int cs_log2, const float2 *__restrict__ ws,
         const float2 *__restrict__ master, int master_len,
         float2 *__restrict__ spec, float *__restrict__ scores, int head0, int head_dim,
-        long long score_stride, float inv_scale, double *__restrict__ partial) {
+        long long score_stride, float inv_scale, double *__restrict__ partial,
+        float energy_scale, int accumulate) {
+  // EPI_SCORE sums the head_dim columns starting at blockIdx.y * head_dim; when a head is
+  // transformed in several column groups, head_dim is the group width, energy_scale the
+  // true number of channels, and every group after the first adds to the stored score.
   extern __shared__ float2 smem[];
   const int N1 = plan.len, cs = 1 << cs_log2;
   float2 *S = smem;
@@ -403,7 +407,8 @@ k_pass3(FftPlan plan, int N2, int N, int ncol_ws, int cs_log2, const float2 *__r
       const int p = n1 * N2 + n2;
       if (p < N) {
         const float k = accK[n1] * inv_scale, v = accV[n1] * inv_scale;   // already divided by d
-        scores[(long long)h * score_stride + perm_token(p, N)] = k + v;
+        float *dst = scores + (long long)h * score_stride + perm_token(p, N);
+        *dst = accumulate ? *dst + (k + v) : k + v;
         dk += (double)k;
         dv += (double)v;
       }
@@ -417,8 +422,8 @@ k_pass3(FftPlan plan, int N2, int N, int ncol_ws, int cs_log2, const float2 *__r
       double sa = 0, sb = 0;
       for (int i = 0; i < kThreads / 32; ++i) { sa += red[0][i]; sb += red[1][i]; }
       const size_t slot = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
-      partial[2 * slot] = sa * (double)head_dim;      // d * sum Dev_k = outlier-band energy
-      partial[2 * slot + 1] = sb * (double)head_dim;
+      partial[2 * slot] = sa * (double)energy_scale;      // d * sum Dev_k = outlier-band energy
+      partial[2 * slot + 1] = sb * (double)energy_scale;
     }
   }
 }
@@ -529,6 +534,7 @@ struct ScoreLayout {
   size_t part_tot_bytes, part_hi_bytes;   // one copy; the specialised path keeps two and alternates (step parity)
   size_t ws_buf_bytes;       // one group buffer; the fast path keeps two and alternates
   int heads_per_group;
+  int sub_cols;              // chirp path: columns of one head transformed together (head_dim = all of them)
 };
 
 // Workspace carve-up for one sequence plan (all sequences share the regions; the
@@ -557,15 +563,19 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   if (sp.fast && groups < h->num_aux && num_heads >= h->num_aux) groups = h->num_aux;   // keep every internal stream busy
   hg = (num_heads + groups - 1) / groups;                      // balanced groups
   L.heads_per_group = hg;
-  L.ws_buf_bytes = align_up(per_head * hg, 256);
+  int sub = head_dim;
+  if (sp.bluestein && hg == 1)
+    while (sub % 64 == 0 && (size_t)sp.Nfft * sub * sizeof(float2) > h->group_bytes) sub /= 2;
+  L.sub_cols = sub;
+  L.ws_buf_bytes = align_up((size_t)sp.Nfft * sub * hg * sizeof(float2), 256);
   size_t off = 0;
   L.off_ws = off;       off += L.ws_buf_bytes * (sp.fast ? h->num_aux : 1);
-  L.off_spec = off;     off += sp.bluestein ? align_up((size_t)sp.N * head_dim * hg * sizeof(float2), 256) : 0;
+  L.off_spec = off;     off += sp.bluestein ? align_up((size_t)sp.N * sub * hg * sizeof(float2), 256) : 0;
   L.off_hhat = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * sizeof(float2), 256) : 0;
   L.off_hcol = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * 8 * sizeof(float2), 256) : 0;
   const size_t slices = (size_t)num_heads * head_dim / 32;   // finest slicing any kernel variant uses
   L.part_tot_bytes = align_up(slices * sp.N2 * 2 * sizeof(double), 256);
-  L.part_hi_bytes = align_up((size_t)num_heads * sp.N2 * 2 * sizeof(double), 256);
+  L.part_hi_bytes = align_up((size_t)num_heads * (head_dim / sub) * sp.N2 * 2 * sizeof(double), 256);
   L.off_part_tot = off; off += L.part_tot_bytes * (sp.fast ? 2 : 1);
   L.off_part_hi = off;  off += L.part_hi_bytes * (sp.fast ? 2 : 1);
   L.total = off;
@@ -939,33 +949,52 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
         ProfScope ps(h, FC_K_PASS3, st);
         k_pass3<EPI_SCORE, false><<<dim3(sp.N2, hg), kThreads, sm3, st>>>(
             p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, nullptr, scores + start, h0, d,
-            total_tokens, 1.f / (float)d, phi);
+            total_tokens, 1.f / (float)d, phi, (float)d, 0);
       }
       if ((s = fc_after_launch(h)) != FC_OK) return s;
     } else {
+      // One head may be transformed in several column groups (sub < d) so that the padded
+      // length-Nfft intermediates of a group stay within the cache budget; the groups run in
+      // stream order and the last pass adds their contributions to the score in that order.
       const float invM = 1.f / (float)sp.Nfft;
-      KvLoader<T, true> ld{kp, vp, kv->stride_token, kv->stride_head, h0, d, N, 0.f, 0.f};
-      if ((s = launch_pass1(h, st, ld, sp, ncol_ws, sp.cs, ws, ptot)) != FC_OK) return s;
-      if ((s = launch_pass2<MID_MULH>(h, st, sp, ncol_ws, sp.cs2, ws, 0, hhat, invM)) != FC_OK) return s;
-      if ((s = set_smem(k_pass3<EPI_SPEC, true>, sm3)) != FC_OK) return s;
-      {
-        ProfScope ps(h, FC_K_PASS3, st);
-        k_pass3<EPI_SPEC, true><<<dim3(sp.N2, ncol_ws / sp.cs), kThreads, sm3, st>>>(
-            p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, spec, nullptr, 0, d, 0, 0.f, nullptr);
-      }
-      if ((s = fc_after_launch(h)) != FC_OK) return s;
-      FilterLoader fl{spec, ncol_ws, N, omega};
-      if ((s = launch_pass1(h, st, fl, sp, ncol_ws, sp.cs, ws, nullptr)) != FC_OK) return s;
-      if ((s = launch_pass2<MID_MULH>(h, st, sp, ncol_ws, sp.cs2, ws, 0, hhat, invM)) != FC_OK) return s;
-      if ((s = set_smem(k_pass3<EPI_SCORE, true>, sm3)) != FC_OK) return s;
       const float inv = (float)(1.0 / ((double)N * (double)N * (double)d));
-      {
-        ProfScope ps(h, FC_K_PASS3, st);
-        k_pass3<EPI_SCORE, true><<<dim3(sp.N2, hg), kThreads, sm3, st>>>(
-            p1, sp.N2, N, ncol_ws, ilog2(sp.cs), ws, h->master, h->master_len, nullptr, scores + start, h0, d,
-            total_tokens, inv, phi);
+      const int sub = L.sub_cols, cs = (sub % 64 == 0) ? 64 : 32;
+      const int ngroups = (hg == 1) ? d / sub : 1;
+      const int ncol = (hg == 1) ? sub : ncol_ws;
+      int cs2 = sp.cs2;
+      while (ncol % cs2) cs2 >>= 1;
+      const size_t sm3c = smem_pass13(sp, cs);
+      for (int cg = 0; cg < ngroups; ++cg) {
+        const int c0 = cg * sub;
+        double *ptot_c = ptot + 2 * (size_t)cg * sp.N2 * (ncol / cs);
+        double *phi_c = phi + 2 * (size_t)cg * sp.N2 * hg;
+        const int dd = (hg == 1) ? sub : d;           // columns the loader and the last pass see per head
+        KvLoader<T, true> ld{kp + c0, vp + c0, kv->stride_token, kv->stride_head, h0, dd, N, 0.f, 0.f};
+        if ((s = launch_pass1(h, st, ld, sp, ncol, cs, ws, ptot_c)) != FC_OK) return s;
+        if ((s = launch_pass2<MID_MULH>(h, st, sp, ncol, cs2, ws, 0, hhat, invM)) != FC_OK) return s;
+        if ((s = set_smem(k_pass3<EPI_SPEC, true>, sm3c)) != FC_OK) return s;
+        {
+          ProfScope ps(h, FC_K_PASS3, st);
+          k_pass3<EPI_SPEC, true><<<dim3(sp.N2, ncol / cs), kThreads, sm3c, st>>>(
+              p1, sp.N2, N, ncol, ilog2(cs), ws, h->master, h->master_len, spec, nullptr, 0, dd, 0, 0.f, nullptr,
+              0.f, 0);
+        }
+        if ((s = fc_after_launch(h)) != FC_OK) return s;
+        FilterLoader fl{spec, ncol, N, omega};
+        if ((s = launch_pass1(h, st, fl, sp, ncol, cs, ws, nullptr)) != FC_OK) return s;
+        if ((s = launch_pass2<MID_MULH>(h, st, sp, ncol, cs2, ws, 0, hhat, invM)) != FC_OK) return s;
+        if ((s = set_smem(k_pass3<EPI_SCORE, true>, sm3c)) != FC_OK) return s;
+        {
+          ProfScope ps(h, FC_K_PASS3, st);
+          k_pass3<EPI_SCORE, true><<<dim3(sp.N2, hg), kThreads, sm3c, st>>>(
+              p1, sp.N2, N, ncol, ilog2(cs), ws, h->master, h->master_len, nullptr, scores + start, h0, dd,
+              total_tokens, inv, phi_c, (float)d, cg > 0 ? 1 : 0);
+        }
+        if ((s = fc_after_launch(h)) != FC_OK) return s;
       }
-      if ((s = fc_after_launch(h)) != FC_OK) return s;
+      tot_slots += (size_t)sp.N2 * (ncol / cs) * ngroups;
+      hi_slots += (size_t)sp.N2 * hg * ngroups;
+      continue;
     }
     tot_slots += (size_t)sp.N2 * (ncol_ws / (sp.fast ? 2 * h->tune_cpw : sp.cs));
     hi_slots += (size_t)sp.N2 * hg;

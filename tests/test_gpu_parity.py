@@ -169,6 +169,17 @@ def test_scores_long_arbitrary_length(fc):
     _check_layer(fc, k, v, [0, N], 0.2)
 
 
+@pytest.mark.parametrize("d,group_bytes", [(128, 1), (128, 3000 * 64 * 8 * 3), (192, 1), (64, 1)])
+def test_scores_arbitrary_length_in_column_groups(fc, d, group_bytes):
+    # a small cache budget makes the chirp path transform each head in groups of 32..96 columns
+    # and add the groups' contributions to the score one after the other
+    N = 3000
+    k, v = _rand_kv(N, 2, d, torch.float32, 40 + d)
+    g1, _ = _check_layer(fc, k, v, [0, N], 0.2, group_bytes=group_bytes)
+    g2, _ = _check_layer(fc, k, v, [0, N], 0.2)
+    np.testing.assert_allclose(g1, g2, rtol=2e-3, atol=1e-6 * float(g2.max()))
+
+
 @pytest.mark.parametrize("mode", [1, 2])
 @pytest.mark.parametrize("lag", [1, 2, 3])
 @pytest.mark.parametrize("N,H,dtype", [(4096, 3, torch.float32), (8192, 2, torch.bfloat16), (16384, 1, torch.float16),

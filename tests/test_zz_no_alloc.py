@@ -97,8 +97,14 @@ def test_sizes_beyond_the_fixed_scratch_are_refused(fc):
     with pytest.raises(fc.FlashCacheError) as e:
         fc.fc_score_layer_static(k, v, cu, 0.2, scores, energy)          # longer than 4096
     assert e.value.code == 2
-    k, v, cu = _inputs([3000], 1, 128, torch.float32, 4)
-    scores = torch.zeros((1, 3000), dtype=torch.float32, device="cuda")
+    k, v, cu = _inputs([4096], 1, 256, torch.float32, 4)
+    scores = torch.zeros((1, 4096), dtype=torch.float32, device="cuda")
     with pytest.raises(fc.FlashCacheError) as e:
-        fc.fc_score_layer_static(k, v, cu, 0.2, scores, energy)          # chirp path needs more than 8 MiB here
+        fc.fc_score_layer_static(k, v, cu, 0.2, scores, energy)          # 4096 x 256 complex values alone fill 8 MiB
     assert e.value.code == 3
+
+
+def test_other_lengths_up_to_the_limit_fit(fc):
+    # the chirp path transforms a head in 32-column groups here, so every length up to 4096 fits
+    _compare(fc, [3000, 4095], 2, 128, torch.float32, 5)
+    _compare(fc, [2500], 1, 256, torch.bfloat16, 6)
