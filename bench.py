@@ -336,61 +336,38 @@ def main():
         "roofline": roof, "roofline_step": roof_step,
     }
 
-    # end to end from pinned host buffers (H2D of K,V and D2H of the compacted cache inside the timing)
+    # end to end through fc_compress_host: K and V start in page-locked host memory, the compacted caches
+    # end there; every step's copies in and out are inside the timed region (consecutive steps overlap
+    # one step's copies back with the next step's copies in, as a serving loop would)
     if not args.no_e2e:
         hostK = [k.cpu().pin_memory() for k in Kd]
         hostV = [v.cpu().pin_memory() for v in Vd]
-        copy_stream = torch.cuda.Stream(device=dev)
-        evs = [torch.cuda.Event() for _ in range(L)]
-        cap = comp.capacity
-        hk = torch.empty((L, cap, cfg.num_heads, cfg.head_dim), dtype=cfg.torch_dtype).pin_memory()
-        hv = torch.empty_like(hk).pin_memory()
-        hidx = torch.empty((L, cfg.num_heads, cap), dtype=torch.int32).pin_memory()
-        hoff = torch.empty((L, len(cfg.seqlens) + 1), dtype=torch.int64).pin_memory()
+        hc = binding.HostCompressor(L, cfg.num_heads, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho,
+                                    cfg.gamma, cfg.min_keep, device=dev.index)
+        results = [hc.new_result(), hc.new_result()]
 
-        def e2e_step():
-            cur = torch.cuda.current_stream()
-            start = torch.cuda.Event()
-            start.record(cur)
-            copy_stream.wait_event(start)
-            with torch.cuda.stream(copy_stream):
-                for l in range(L):
-                    Kd[l].copy_(hostK[l], non_blocking=True)
-                    Vd[l].copy_(hostV[l], non_blocking=True)
-                    evs[l].record(copy_stream)
-            ws = comp._workspace(Kd[0], Vd[0])
-            for l in range(L):
-                cur.wait_event(evs[l])
-                binding.fc_score_layer(comp.handle, Kd[l], Vd[l], comp.cu, comp.gamma, comp.scores[l],
-                                       comp.energy[l], ws)
-            comp.allocate()
-            comp.select_compact(Kd, Vd)
-            hoff.copy_(comp.offsets, non_blocking=True)
-            cur.synchronize()
-            d2h = hoff.numel() * 8
-            for l in range(L):
-                r = int(hoff[l, -1])
-                hk[l, :r].copy_(comp.out_k[l, :r], non_blocking=True)
-                hv[l, :r].copy_(comp.out_v[l, :r], non_blocking=True)
-                hidx[l, :, :r].copy_(comp.out_idx[l, :, :r], non_blocking=True)
-                d2h += 2 * r * cfg.num_heads * cfg.head_dim * s + r * cfg.num_heads * 4
-            cur.synchronize()
-            return d2h
+        def e2e_steps(n):
+            for i in range(n):
+                hc.compress(hostK, hostV, results[i % 2])
+            torch.cuda.synchronize(dev)
 
-        for _ in range(2):
-            d2h_bytes = e2e_step()
+        e2e_steps(2)
+        hc.check_device_status()
         n_e2e = max(3, min(10, args.steps))
         barrier()
         t0 = time.perf_counter()
-        for _ in range(n_e2e):
-            d2h_bytes = e2e_step()
+        e2e_steps(n_e2e)
         barrier()
         e2e_ms = 1000.0 * (time.perf_counter() - t0) / n_e2e
         e2e_ms = replicas.max_over_ranks(e2e_ms, dist, dev)
+        rows = int(results[0].layer_rows[L])
+        d2h_bytes = (2 * rows * cfg.num_heads * cfg.head_dim * s + rows * cfg.num_heads * 4
+                     + results[0].budgets.numel() * 4 + results[0].offsets.numel() * 8)
         out["e2e"] = {"value": replicas.whole_job_rate(tokens, world, e2e_ms), "unit": UNIT,
                       "h2d_bytes_per_step": int(input_bytes), "d2h_bytes_per_step": int(d2h_bytes),
-                      "ms_per_step": e2e_ms, "steps": n_e2e}
-        del hostK, hostV, hk, hv
+                      "ms_per_step": e2e_ms, "steps": n_e2e, "call": "fc_compress_host"}
+        hc.close()
+        del hostK, hostV, results, hc
 
     # CPU baseline: the oracle on this machine's host cores, bounded sample (rank 0, single-GPU run only)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -251,6 +251,70 @@ size_t fc_static_scratch_bytes(void);
 fc_status fc_score_layer_static(const fc_kv_view *kv, double gamma, float *scores,
                                 double *energy, fc_stream stream);
 
+/*
+ * The whole compressor for one prefill, from HOST memory to HOST memory (Sec. 3.2, Fig. 2):
+ * copies every layer's K and V to the device, scores each layer as soon as its copies have
+ * landed (fc_score_layer), allocates the budgets over all layers (fc_allocate_budgets), keeps
+ * the Outlier KVs of every layer (fc_select_compact) and copies the compacted caches back.
+ * The same kernels as the per-stage entry points, so the same results; what this call adds is
+ * the copy pipeline around them.
+ *
+ * Inputs (HOST; page-locked memory lets the copies overlap the kernels, pageable memory
+ * works but serialises them):
+ *   k_host, v_host   [num_layers] pointers; layer l dense [T][num_heads][head_dim] of `dtype`,
+ *                    T = cu_seqlens[batch].
+ *   cu_seqlens       int32[batch+1], as in fc_kv_view.
+ *   gamma, rho, min_keep   as in fc_score_layer and fc_allocate_budgets.
+ * Device memory (DEVICE, owned by the caller, 256-byte aligned, >= fc_compress_host_arena_bytes):
+ *   arena            staging for the inputs of all layers, scores, energies, budgets, the
+ *                    compacted caches and the kernels' workspace.  Two consecutive calls with
+ *                    the same arena are ordered by the library (the second call's copies wait
+ *                    for the first call's selection, not for its copies back to the host, so
+ *                    they overlap those).  Otherwise the arena must not be in use by work that
+ *                    was enqueued later than the moment `stream` has reached at the call.
+ * Outputs (HOST, valid once `stream` has been synchronised after the call):
+ *   budgets_host     int32[num_layers][batch]     tokens kept per head (layer, sequence)
+ *   offsets_host     int64[num_layers][batch+1]   prefix sums, as fc_allocate_budgets' out_offsets
+ *   layer_rows_host  int64[num_layers+1]          first packed row of every layer; [L] = rows in all
+ *   out_k_host, out_v_host   packed rows [row][num_heads][head_dim]; layer l, sequence b, j-th
+ *                    kept token = row layer_rows[l] + offsets[l][b] + j
+ *   out_idx_host     int32; layer l's indices are the array [num_heads][r_l], r_l =
+ *                    layer_rows[l+1]-layer_rows[l], starting at element num_heads*layer_rows[l];
+ *                    entry [h][offsets[l][b]+j] = sequence-local token index, ascending in j
+ *   out_capacity_rows  rows available in out_k_host / out_v_host (and num_heads times as many
+ *                    index entries); fc_compress_host_rows() gives the number needed.
+ * budgets_host, offsets_host and layer_rows_host are already valid when the call returns: the call
+ * blocks the host once, after the budgets are known, to learn the sizes of the copies back.
+ *
+ * Errors: FC_ERR_INVALID_ARG, FC_ERR_UNSUPPORTED (as fc_score_layer), FC_ERR_WORKSPACE (arena
+ * too small or misaligned; more rows than out_capacity_rows, in which case nothing is copied
+ * back), FC_ERR_CUDA.  Device-side checks report through fc_last_device_status as usual.
+ */
+typedef struct {
+  const void *const *k_host;
+  const void *const *v_host;
+  int32_t num_layers, dtype, num_heads, head_dim, batch, min_keep;
+  const int32_t *cu_seqlens;
+  double gamma, rho;
+  void *arena;
+  size_t arena_bytes;
+  void *out_k_host, *out_v_host;
+  int32_t *out_idx_host;
+  int64_t out_capacity_rows;
+  int32_t *budgets_host;
+  int64_t *offsets_host;
+  int64_t *layer_rows_host;
+} fc_host_job;
+
+/* Rows the compacted caches of all layers hold together: the sum over sequences of
+ * B_tot = clamp(floor(rho*N*L + 1/2), L*lo, L*N) (Sec. 3.2.2), which the budgets add up to. */
+int64_t fc_compress_host_rows(int32_t num_layers, int32_t batch, const int32_t *cu_seqlens,
+                              double rho, int32_t min_keep);
+/* Device bytes fc_compress_host needs for this job (only the shape fields, cu_seqlens, rho and
+ * min_keep are read).  0 on bad input. */
+size_t fc_compress_host_arena_bytes(const fc_handle *h, const fc_host_job *job);
+fc_status fc_compress_host(fc_handle *h, const fc_host_job *job, fc_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

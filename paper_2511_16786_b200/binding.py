@@ -27,6 +27,7 @@ EXPORTS = (
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact",
     "fc_static_scratch_bytes", "fc_score_layer_static",
+    "fc_compress_host_rows", "fc_compress_host_arena_bytes", "fc_compress_host",
 )
 
 
@@ -36,6 +37,20 @@ class fc_kv_view(ctypes.Structure):
         ("stride_token", c_int64), ("stride_head", c_int64),
         ("dtype", c_int32), ("num_heads", c_int32), ("head_dim", c_int32), ("batch", c_int32),
         ("cu_seqlens", POINTER(c_int32)),
+    ]
+
+
+class fc_host_job(ctypes.Structure):
+    _fields_ = [
+        ("k_host", POINTER(c_void_p)), ("v_host", POINTER(c_void_p)),
+        ("num_layers", c_int32), ("dtype", c_int32), ("num_heads", c_int32), ("head_dim", c_int32),
+        ("batch", c_int32), ("min_keep", c_int32),
+        ("cu_seqlens", POINTER(c_int32)),
+        ("gamma", c_double), ("rho", c_double),
+        ("arena", c_void_p), ("arena_bytes", c_size_t),
+        ("out_k_host", c_void_p), ("out_v_host", c_void_p), ("out_idx_host", c_void_p),
+        ("out_capacity_rows", c_int64),
+        ("budgets_host", c_void_p), ("offsets_host", c_void_p), ("layer_rows_host", c_void_p),
     ]
 
 
@@ -96,6 +111,12 @@ def _load() -> ctypes.CDLL:
     lib.fc_static_scratch_bytes.restype = c_size_t
     lib.fc_score_layer_static.argtypes = [POINTER(fc_kv_view), c_double, c_void_p, c_void_p, c_void_p]
     lib.fc_score_layer_static.restype = c_int
+    lib.fc_compress_host_rows.argtypes = [c_int32, c_int32, POINTER(c_int32), c_double, c_int32]
+    lib.fc_compress_host_rows.restype = c_int64
+    lib.fc_compress_host_arena_bytes.argtypes = [c_void_p, POINTER(fc_host_job)]
+    lib.fc_compress_host_arena_bytes.restype = c_size_t
+    lib.fc_compress_host.argtypes = [c_void_p, POINTER(fc_host_job), c_void_p]
+    lib.fc_compress_host.restype = c_int
     return lib
 
 
@@ -237,6 +258,12 @@ def fc_score_layer_static(k, v, cu_seqlens, gamma: float, scores, energy) -> Non
     view = make_view(k, v, cu)
     _check(_lib.fc_score_layer_static(byref(view), float(gamma), c_void_p(scores.data_ptr()),
                                       c_void_p(energy.data_ptr()), _stream()), "fc_score_layer_static")
+
+
+def fc_compress_host_rows(num_layers: int, cu_seqlens, rho: float, min_keep: int) -> int:
+    cu = _cu_array(cu_seqlens)
+    return int(_lib.fc_compress_host_rows(int(num_layers), len(cu) - 1, ctypes.cast(cu, POINTER(c_int32)),
+                                          float(rho), int(min_keep)))
 
 
 def fc_allocate_budgets(handle, energy, cu_seqlens, rho: float, min_keep: int, budgets, out_offsets) -> None:
@@ -391,3 +418,93 @@ class Compressor:
 
     def check_device_status(self):
         _check(fc_last_device_status(self.handle), "device status")
+
+
+class HostResult:
+    """Page-locked host buffers one fc_compress_host call fills (layout: include/flashcache.h)."""
+
+    def __init__(self, num_layers: int, num_heads: int, head_dim: int, batch: int, rows: int, dtype):
+        rows = max(int(rows), 1)
+        self.out_k = torch.empty((rows, num_heads, head_dim), dtype=dtype).pin_memory()
+        self.out_v = torch.empty((rows, num_heads, head_dim), dtype=dtype).pin_memory()
+        self.out_idx = torch.empty((rows * num_heads,), dtype=torch.int32).pin_memory()
+        self._budgets_store = torch.zeros((num_layers * max(batch, 1),), dtype=torch.int32)
+        self.budgets = self._budgets_store[:num_layers * batch].view(num_layers, batch)
+        self.offsets = torch.zeros((num_layers, batch + 1), dtype=torch.int64)
+        self.layer_rows = torch.zeros((num_layers + 1,), dtype=torch.int64)
+        self.capacity = rows
+        self.num_heads = num_heads
+
+    def layer(self, l: int):
+        """(K rows, V rows, indices [H, r]) of layer l; call after the stream has been synchronised."""
+        r0, r1 = int(self.layer_rows[l]), int(self.layer_rows[l + 1])
+        H = self.num_heads
+        return self.out_k[r0:r1], self.out_v[r0:r1], self.out_idx[H * r0:H * r1].view(H, r1 - r0)
+
+
+class HostCompressor:
+    """fc_compress_host for one workload shape: owns the handle and the device arena; `compress`
+    takes per-layer HOST tensors [T, H, d] (page-locked for overlap) and enqueues the whole path on
+    the current stream.  Two HostResult objects used in turn let the copies back of one call overlap
+    the copies in of the next."""
+
+    def __init__(self, num_layers: int, num_heads: int, head_dim: int, cu_seqlens, dtype, rho: float,
+                 gamma: float = 0.2, min_keep: int = 1, device: int = 0):
+        self.L, self.H, self.d = int(num_layers), int(num_heads), int(head_dim)
+        self.cu = [int(x) for x in cu_seqlens]
+        self.B = len(self.cu) - 1
+        self.T = self.cu[-1]
+        self.rho, self.gamma, self.min_keep = float(rho), float(gamma), int(min_keep)
+        self.dtype = dtype
+        self.device = torch.device("cuda", device)
+        seqlens = [self.cu[b + 1] - self.cu[b] for b in range(self.B)]
+        self.handle = fc_create(device, max(1, max(seqlens) if seqlens else 1))
+        self.rows = fc_compress_host_rows(self.L, self.cu, self.rho, self.min_keep)
+        self._cu = _cu_array(self.cu)
+        self._kptr = (c_void_p * self.L)()
+        self._vptr = (c_void_p * self.L)()
+        self._job = fc_host_job(
+            k_host=ctypes.cast(self._kptr, POINTER(c_void_p)), v_host=ctypes.cast(self._vptr, POINTER(c_void_p)),
+            num_layers=self.L, dtype=_DTYPE[dtype], num_heads=self.H, head_dim=self.d, batch=self.B,
+            min_keep=self.min_keep, cu_seqlens=ctypes.cast(self._cu, POINTER(c_int32)),
+            gamma=self.gamma, rho=self.rho)
+        need = int(_lib.fc_compress_host_arena_bytes(self.handle, byref(self._job)))
+        if need == 0:
+            raise FlashCacheError(2, "fc_compress_host_arena_bytes")
+        self.arena = torch.empty(need, dtype=torch.uint8, device=self.device)
+        self._job.arena = self.arena.data_ptr()
+        self._job.arena_bytes = need
+
+    def new_result(self) -> HostResult:
+        return HostResult(self.L, self.H, self.d, self.B, self.rows, self.dtype)
+
+    def compress(self, K_layers, V_layers, result: HostResult) -> None:
+        if len(K_layers) != self.L or len(V_layers) != self.L:
+            raise ValueError("one K and one V tensor per layer")
+        for l in range(self.L):
+            k, v = K_layers[l], V_layers[l]
+            if k.is_cuda or v.is_cuda or not k.is_contiguous() or not v.is_contiguous() or k.dtype != self.dtype \
+                    or v.dtype != self.dtype or tuple(k.shape) != (self.T, self.H, self.d) or k.shape != v.shape:
+                raise ValueError("layer %d: expected contiguous host tensors [T, H, d] of the compressor's dtype" % l)
+            self._kptr[l] = k.data_ptr()
+            self._vptr[l] = v.data_ptr()
+        j = self._job
+        j.out_k_host, j.out_v_host, j.out_idx_host = result.out_k.data_ptr(), result.out_v.data_ptr(), result.out_idx.data_ptr()
+        j.out_capacity_rows = result.capacity
+        j.budgets_host, j.offsets_host = result._budgets_store.data_ptr(), result.offsets.data_ptr()
+        j.layer_rows_host = result.layer_rows.data_ptr()
+        _check(_lib.fc_compress_host(self.handle, byref(j), _stream()), "fc_compress_host")
+
+    def check_device_status(self):
+        _check(fc_last_device_status(self.handle), "device status")
+
+    def close(self):
+        if self.handle is not None:
+            fc_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -173,6 +173,10 @@ extern "C" void fc_destroy(fc_handle *h) {
     if (h->ev_join[i]) cudaEventDestroy(h->ev_join[i]);
   }
   if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+  if (h->host_copy) { cudaStreamSynchronize(h->host_copy); cudaStreamDestroy(h->host_copy); }
+  for (int i = 0; i < h->host_ev_cap; ++i) cudaEventDestroy(h->host_ev[i]);
+  delete[] h->host_ev;
+  if (h->ev_inputs_free) cudaEventDestroy(h->ev_inputs_free);
   if (h->master) cudaFree(h->master);
   if (h->status_word) cudaFree(h->status_word);
   if (h->done_counter) cudaFree(h->done_counter);

@@ -64,6 +64,14 @@ struct fc_handle {
   long long last_sig;            // (N, heads, head_dim) of the previous specialised-path step
   bool pending_join;             // internal streams hold work the caller's stream has not waited for
   cudaEvent_t ev_done[2][FC_MAX_AUX];   // [step parity][internal stream]: that stream finished that step
+  // fc_compress_host (created on its first call): the stream the host-to-device copies run on, one
+  // event per layer (that layer's copies have landed), and the point of the previous job after
+  // which the staged inputs of its arena may be overwritten
+  cudaStream_t host_copy;
+  cudaEvent_t *host_ev;
+  int host_ev_cap;
+  cudaEvent_t ev_inputs_free;
+  const void *host_last_arena;
 };
 
 // Kernel classes for fc_profile_begin.
