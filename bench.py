@@ -215,6 +215,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first LAYERS layers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     args = ap.parse_args()
     if args.impl == "reference":
@@ -335,6 +336,23 @@ def main():
         "clocks": clocks, "gpu_launches": int(launches),
         "roofline": roof, "roofline_step": roof_step,
     }
+
+    # the same step replayed from a CUDA graph (reported beside the headline, which stays the plain call
+    # sequence because only that one carries the per-kernel event timing)
+    if not args.no_graph:
+        graph = comp.capture(Kd, Vd)
+        for _ in range(3):
+            graph.replay()
+        barrier()
+        ev0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        ev1.record()
+        barrier()
+        g_ms = replicas.max_over_ranks(ev0.elapsed_time(ev1), dist, dev) / args.steps
+        comp.check_device_status()
+        out["cuda_graph"] = {"ms_per_step": g_ms, "value": replicas.whole_job_rate(tokens, world, g_ms), "unit": UNIT}
+        del graph
 
     # end to end through fc_compress_host: K and V start in page-locked host memory, the compacted caches
     # end there; every step's copies in and out are inside the timed region (consecutive steps overlap

@@ -120,6 +120,14 @@ fc_status fc_set_score_overlap(fc_handle *h, int32_t enabled);
  * call waits for the one before it. */
 fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled);
 
+/* Forgets the ordering state the handle keeps between calls (which of its internal events the next
+ * call would wait on).  Call it right before cudaStreamBeginCapture and right after
+ * cudaStreamEndCapture when a sequence of calls on this handle is captured into a CUDA graph: an
+ * event recorded outside a capture cannot be waited on inside one, nor the other way round.
+ * Everything enqueued earlier through the handle must already be complete, or be ordered before the
+ * next call by the stream that call is given (a graph launch on that stream is). */
+fc_status fc_reset_ordering(fc_handle *h);
+
 /* Running totals of the fused transform kernel since fc_create (diagnostic; synchronises the
  * device): out = { tiles processed, tiles whose inputs were not finished when they were looked
  * when the scheduler warp first looked, unused, clock cycles (thread 0 of every block, summed) inside

@@ -23,7 +23,7 @@ _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
     "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count",
-    "fc_set_group_bytes", "fc_set_score_overlap", "fc_set_select_overlap", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
+    "fc_set_group_bytes", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact",
     "fc_static_scratch_bytes", "fc_score_layer_static",
@@ -78,6 +78,8 @@ def _load() -> ctypes.CDLL:
     lib.fc_launch_count.restype = c_uint64
     lib.fc_set_group_bytes.argtypes = [c_void_p, c_size_t]
     lib.fc_set_group_bytes.restype = c_int
+    lib.fc_reset_ordering.argtypes = [c_void_p]
+    lib.fc_reset_ordering.restype = c_int
     lib.fc_set_score_overlap.argtypes = [c_void_p, c_int32]
     lib.fc_set_score_overlap.restype = c_int
     lib.fc_set_select_overlap.argtypes = [c_void_p, c_int32]
@@ -266,6 +268,10 @@ def fc_compress_host_rows(num_layers: int, cu_seqlens, rho: float, min_keep: int
                                           float(rho), int(min_keep)))
 
 
+def fc_reset_ordering(handle) -> None:
+    _check(_lib.fc_reset_ordering(handle), "fc_reset_ordering")
+
+
 def fc_allocate_budgets(handle, energy, cu_seqlens, rho: float, min_keep: int, budgets, out_offsets) -> None:
     """energy: float64 [L, B, 4]; budgets: int32 [L, B]; out_offsets: int64 [L, B+1]."""
     cu = _cu_array(cu_seqlens)
@@ -415,6 +421,25 @@ class Compressor:
         self.score(K_layers, V_layers)
         self.allocate()
         self.select_compact(K_layers, V_layers)
+
+    def capture(self, K_layers, V_layers):
+        """The whole `compress` sequence on these tensors as a CUDA graph (torch.cuda.CUDAGraph): one
+        warm-up pass, then a capture on a side stream.  `replay()` reruns it on the tensors' current
+        contents; results land in the same buffers as `compress`.  Worth it for short sequences, where
+        the launches cost more than the kernels."""
+        self.compress(K_layers, V_layers)
+        torch.cuda.synchronize(self.device)
+        self.check_device_status()
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream(device=self.device)
+        side.wait_stream(torch.cuda.current_stream(self.device))
+        fc_reset_ordering(self.handle)
+        try:
+            with torch.cuda.graph(graph, stream=side):
+                self.compress(K_layers, V_layers)
+        finally:
+            fc_reset_ordering(self.handle)
+        return graph
 
     def check_device_status(self):
         _check(fc_last_device_status(self.handle), "device status")

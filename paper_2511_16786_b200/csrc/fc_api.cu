@@ -241,6 +241,15 @@ extern "C" fc_status fc_set_score_overlap(fc_handle *h, int32_t enabled) {
   return FC_OK;
 }
 
+extern "C" fc_status fc_reset_ordering(fc_handle *h) {
+  if (!h) return FC_ERR_INVALID_ARG;
+  h->step = 0;
+  h->last_sig = 0;
+  h->pending_join = false;
+  h->host_last_arena = nullptr;
+  return FC_OK;
+}
+
 extern "C" fc_status fc_set_group_bytes(fc_handle *h, size_t bytes) {
   if (!h || bytes == 0) return FC_ERR_INVALID_ARG;
   h->group_bytes = bytes;

@@ -481,9 +481,12 @@ SeqPlan plan_sequence(int N, bool allow_fast = true) {
   s.fast = allow_fast && !s.bluestein && N >= 1024 && N <= 65536;
   int b1 = bits / 2;
   if (b1 > 7 && !s.fast) b1 = 7;
+  s.cs = 64;
+  // 131072 points: 256 x 512 with 32-column tiles in passes 1 and 3 beats 128 x 1024, whose pass 2 has
+  // room for only 4 columns per block (measured on the chirp path: 461 against 488 ms per step)
+  if (bits == 17) { b1 = 8; s.cs = 32; }
   s.N1 = 1 << b1;
   s.N2 = s.Nfft / s.N1;
-  s.cs = 64;
   int cs2 = 4096 / s.N2;      // 2*N2*cs2*8 bytes = 64 KiB
   if (cs2 > 64) cs2 = 64;
   if (cs2 < 4) cs2 = 4;
@@ -563,9 +566,14 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   if (sp.fast && groups < h->num_aux && num_heads >= h->num_aux) groups = h->num_aux;   // keep every internal stream busy
   hg = (num_heads + groups - 1) / groups;                      // balanced groups
   L.heads_per_group = hg;
+  // Chirp path, one head per group: the head is split into column groups only when its intermediates
+  // pass four times the budget.  Narrower tiles cost time (measured: +2 % at 64 columns, +8 % at 32 for
+  // 131072-point transforms) and the generic kernels do not wait on DRAM, so below that the split
+  // would only save workspace.
   int sub = head_dim;
+  const size_t split_above = h->group_bytes > ((size_t)1 << 60) ? h->group_bytes : 4 * h->group_bytes;
   if (sp.bluestein && hg == 1)
-    while (sub % 64 == 0 && (size_t)sp.Nfft * sub * sizeof(float2) > h->group_bytes) sub /= 2;
+    while (sub % 64 == 0 && (size_t)sp.Nfft * sub * sizeof(float2) > split_above) sub /= 2;
   L.sub_cols = sub;
   L.ws_buf_bytes = align_up((size_t)sp.Nfft * sub * hg * sizeof(float2), 256);
   size_t off = 0;
@@ -580,6 +588,38 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   L.off_part_hi = off;  off += L.part_hi_bytes * (sp.fast ? 2 : 1);
   L.total = off;
   return L;
+}
+
+// The specialised path keeps each internal stream's intermediate buffer in the persisting part of L2.
+bool window_fits(const fc_handle *h, const ScoreLayout &L) {
+  return h->l2_persist && L.ws_buf_bytes <= h->window_max && L.ws_buf_bytes * (size_t)h->num_aux <= h->persist_max;
+}
+
+// The persisting part of L2 is a set-aside of this process's context (gone with it): claimed while calls
+// contain a sequence for the specialised path, given back to ordinary caching when a call has none (the
+// generic kernels lose about a tenth of their speed to a set-aside they do not use).  Decided once per call;
+// left as it is while `st` is being captured into a graph, where device-wide settings cannot change.
+void claim_persisting_l2(fc_handle *h, const fc_kv_view *kv, cudaStream_t st) {
+  if (!h->l2_persist || h->generic_only) return;
+  bool claim = false;
+  for (int b = 0; b < kv->batch && !claim; ++b) {
+    const int N = kv->cu_seqlens[b + 1] - kv->cu_seqlens[b];
+    if (N == 0) continue;
+    const SeqPlan sp = plan_sequence(N);
+    if (!sp.fast || plan_fused(h, sp, kv->num_heads, kv->head_dim).ok) continue;
+    claim = window_fits(h, layout_for(h, sp, kv->num_heads, kv->head_dim));
+  }
+  if (claim == (h->persist_on != 0)) return;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); return; }
+  if (cap != cudaStreamCaptureStatusNone) return;
+  if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, claim ? h->persist_max : 0) != cudaSuccess) {
+    cudaGetLastError();
+    h->l2_persist = 0;
+    return;
+  }
+  h->persist_on = claim ? 1 : 0;
+  if (!claim) cudaCtxResetPersistingL2Cache();
 }
 
 fc_status validate_view(const fc_handle *h, const fc_kv_view *kv) {
@@ -876,19 +916,8 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
   }
 
-  // The persisting part of L2 is a set-aside of this process's context (gone with it): claim it while the
-  // specialised path runs, give it back to ordinary caching when another path takes over.
-  const bool want_persist = separate_fast && h->l2_persist && L.ws_buf_bytes <= h->window_max &&
-                            L.ws_buf_bytes * (size_t)h->num_aux <= h->persist_max;
-  if (want_persist != (h->persist_on != 0)) {
-    if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want_persist ? h->persist_max : 0) != cudaSuccess) {
-      cudaGetLastError();
-      h->l2_persist = 0;
-    } else {
-      h->persist_on = want_persist ? 1 : 0;
-      if (!want_persist) cudaCtxResetPersistingL2Cache();
-    }
-  }
+  // fc_score_layer has claimed the persisting part of L2 if any sequence of the call takes this path
+  const bool want_persist = separate_fast && window_fits(h, L);
   if (want_persist && h->persist_on) {
     // keep each stream's intermediate in the persisting part of L2; everything else these streams touch
     // (the K/V rows, the scores) streams through
@@ -958,7 +987,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       // stream order and the last pass adds their contributions to the score in that order.
       const float invM = 1.f / (float)sp.Nfft;
       const float inv = (float)(1.0 / ((double)N * (double)N * (double)d));
-      const int sub = L.sub_cols, cs = (sub % 64 == 0) ? 64 : 32;
+      const int sub = L.sub_cols, cs = (sub % 64 == 0) ? sp.cs : 32;
       const int ngroups = (hg == 1) ? d / sub : 1;
       const int ncol = (hg == 1) ? sub : ncol_ws;
       int cs2 = sp.cs2;
@@ -1053,6 +1082,7 @@ extern "C" fc_status fc_score_layer(fc_handle *h, const fc_kv_view *kv, double g
   FC_CUDA_TRY(cudaGetDevice(&dev));
   if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  claim_persisting_l2(h, kv, st);
   for (int b = 0; b < kv->batch && s == FC_OK; ++b) {
     switch (kv->dtype) {
       case FC_F32: s = score_sequence<float>(h, st, kv, b, gamma, scores, energy, (char *)workspace); break;
