@@ -300,18 +300,44 @@ def select_topk(dev, k: int) -> np.ndarray:
     return np.array(sorted(order[:k]), dtype=np.int64)
 
 
+def layer_score(dev_heads) -> np.ndarray:
+    """Deviation of a token in the layer-wide formulation, where K^l is N x D with D the
+    whole hidden width (Sec. 3.1, Eq. 5): the mean over the D channels.  With D = H*d it is
+    the mean over the H heads of the per-head deviation (Eq. 10 applied to each head's d
+    channels).  dev_heads: [H, N]."""
+    return np.asarray(dev_heads, dtype=np.float64).mean(axis=0)
+
+
+def select_topk_protected(dev, k: int, protect=None) -> np.ndarray:
+    """select_topk with tokens that must survive (text tokens, attention sinks, a recent window:
+    Sec. 1 speaks of compressing the visual KVs): a token whose `protect` entry is non-zero ranks
+    before every other token; protected tokens are equal among themselves (index ascending), the
+    others keep the order of select_topk.  The budget k still counts them, so with more than k
+    protected tokens the first k of them by index are kept."""
+    dev = np.asarray(dev, dtype=np.float64)
+    if protect is None:
+        return select_topk(dev, k)
+    prot = np.asarray(protect).astype(bool)
+    key = np.where(np.isnan(dev), np.inf, dev)
+    order = sorted(range(dev.shape[0]), key=lambda x: (0, 0.0, x) if prot[x] else (1, -key[x], x))
+    return np.array(sorted(order[:k]), dtype=np.int64)
+
+
 def compact_rows(X: np.ndarray, idx) -> np.ndarray:
     """Rows idx of X[N, ...] in the given order, bit for bit."""
     return np.ascontiguousarray(np.asarray(X)[np.asarray(idx, dtype=np.int64)])
 
 
 def compress(K_layers, V_layers, cu_seqlens, gamma: float, rho: float,
-             min_keep: int = 1, tier: str = "fft"):
+             min_keep: int = 1, tier: str = "fft", per_layer: bool = False, protect=None):
     """The whole pass over L layers.  K_layers[l], V_layers[l]: [T, H, d].
 
     Returns dict(scores[L][H,T], energy[L,B,4], budgets[L,B], offsets[L,B+1],
     idx[l][h] (list over sequences of ascending local token indices),
     out_k[l], out_v[l] ([rows_l, H, d], stored dtype preserved)).
+
+    per_layer: every head of a layer keeps the tokens chosen from layer_score (one index set
+    per layer and sequence) instead of its own.  protect: [T] flags, see select_topk_protected.
     """
     L = len(K_layers)
     B = len(cu_seqlens) - 1
@@ -335,7 +361,10 @@ def compress(K_layers, V_layers, cu_seqlens, gamma: float, rho: float,
             per_seq = []
             for b in range(B):
                 s0 = int(cu_seqlens[b])
-                sel = select_topk(scores[l][h, s0:s0 + seqlens[b]], int(budgets[l, b]))
+                dev = scores[l][:, s0:s0 + seqlens[b]]
+                dev = layer_score(dev) if per_layer else dev[h]
+                prot = None if protect is None else np.asarray(protect)[s0:s0 + seqlens[b]]
+                sel = select_topk_protected(dev, int(budgets[l, b]), prot)
                 per_seq.append(sel)
                 o = int(offsets[l, b])
                 ok[o:o + len(sel), h] = compact_rows(Kl[s0:s0 + seqlens[b], h], sel)

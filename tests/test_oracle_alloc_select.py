@@ -162,3 +162,92 @@ def test_compress_end_to_end_small():
                 got = res["out_v"][l][o:o + len(sel), h]
                 assert got.tobytes() == Vs[l][cu[b] + sel, h].tobytes()
     assert 5 in res["idx"][1][0][0] and 5 in res["idx"][1][1][0]
+
+
+# ---------------------------------------------------------------- layer-wide score, protected tokens
+def _brute_force_protected(dev, k, prot):
+    """Protected tokens first (by index), then repeated arg-max over the rest."""
+    p = [x for x in range(len(dev)) if prot[x]]
+    out = p[:k]
+    if len(out) < k:
+        rest = [x for x in range(len(dev)) if not prot[x]]
+        sub = _brute_force_topk([dev[x] for x in rest], k - len(out))
+        out = out + [rest[i] for i in sub]
+    return sorted(out)
+
+
+def _brute_force_protected_by_rank(dev, k, prot):
+    """The same through repeated arg-max on (protected, score) pairs, lowest index first among equals."""
+    key = [(1, 0.0) if prot[x] else (0, float("inf") if dev[x] != dev[x] else float(dev[x])) for x in range(len(dev))]
+    alive = list(range(len(key)))
+    out = []
+    for _ in range(k):
+        best = alive[0]
+        for x in alive[1:]:
+            if key[x] > key[best]:
+                best = x
+        out.append(best)
+        alive.remove(best)
+    return sorted(out)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_protected_topk_matches_brute_force(seed):
+    rng = np.random.default_rng(100 + seed)
+    n = int(rng.integers(1, 40))
+    dev = rng.integers(0, 6, n).astype(np.float64)
+    if seed % 3 == 0:
+        dev[rng.integers(0, n)] = np.nan                   # a NaN score still ranks below a protected token
+    prot = (rng.random(n) < 0.3).astype(np.uint8)
+    for k in {0, 1, n // 2, max(0, n - 1), n}:
+        got = list(O.select_topk_protected(dev, k, prot))
+        assert got == _brute_force_protected_by_rank(dev, k, prot)
+        assert got == _brute_force_protected(dev, k, prot)
+
+
+def test_protected_topk_special_cases():
+    dev = [9.0, 1.0, 8.0, 0.0, 7.0]
+    assert list(O.select_topk_protected(dev, 2, None)) == [0, 2]
+    assert list(O.select_topk_protected(dev, 2, [0, 0, 0, 0, 0])) == [0, 2]          # empty mask changes nothing
+    assert list(O.select_topk_protected(dev, 2, [0, 1, 0, 0, 0])) == [0, 1]          # the protected token takes a slot
+    assert list(O.select_topk_protected(dev, 2, [0, 1, 0, 1, 1])) == [1, 3]          # more protected than budget: by index
+    assert list(O.select_topk_protected(dev, 5, [0, 1, 0, 1, 1])) == [0, 1, 2, 3, 4]
+    assert list(O.select_topk_protected([np.nan, 1.0], 1, [0, 1])) == [1]            # protection outranks NaN = +inf
+
+
+def test_layer_score_is_the_deviation_over_the_whole_hidden_width():
+    # Eq. 10 on the N x D matrices (D = H*d) equals the mean over heads of Eq. 10 on each head's N x d slice
+    rng = np.random.default_rng(5)
+    N, H, d = 24, 3, 4
+    K = rng.standard_normal((N, H, d))
+    V = rng.standard_normal((N, H, d))
+    per_head = np.stack([O.score_head(K[:, h], V[:, h], 0.25)[0] for h in range(H)])
+    whole = O.score_head(K.reshape(N, H * d), V.reshape(N, H * d), 0.25)[0]
+    np.testing.assert_allclose(O.layer_score(per_head), whole, rtol=1e-12, atol=1e-15)
+    assert O.layer_score(per_head[:1]).tolist() == per_head[0].tolist()               # one head: nothing to average
+
+
+def test_compress_per_layer_and_protected():
+    rng = np.random.default_rng(6)
+    L, H, d = 2, 3, 8
+    cu = [0, 20, 31]
+    T = 31
+    Ks = [rng.standard_normal((T, H, d)).astype(np.float32) for _ in range(L)]
+    Vs = [rng.standard_normal((T, H, d)).astype(np.float32) for _ in range(L)]
+    prot = np.zeros(T, dtype=np.uint8)
+    prot[[0, 1, 19, 20, 30]] = 1                            # sinks and last tokens of both sequences
+    res = O.compress(Ks, Vs, cu, 0.25, 0.5, 3, tier="literal", per_layer=True, protect=prot)
+    base = O.compress(Ks, Vs, cu, 0.25, 0.5, 3, tier="literal")
+    assert np.array_equal(res["budgets"], base["budgets"])  # the options act on the selection only
+    for l in range(L):
+        for b in range(2):
+            sets = [res["idx"][l][h][b].tolist() for h in range(H)]
+            assert sets[0] == sets[1] == sets[2]            # one index set per layer
+            local = [t - cu[b] for t in np.flatnonzero(prot) if cu[b] <= t < cu[b + 1]]
+            assert set(local) <= set(sets[0])               # min_keep 3 >= protected tokens per sequence
+            dev = O.layer_score(res["scores"][l][:, cu[b]:cu[b + 1]])
+            assert sets[0] == list(O.select_topk_protected(dev, int(res["budgets"][l, b]), prot[cu[b]:cu[b + 1]]))
+            o = int(res["offsets"][l, b])
+            for h in range(H):
+                got = res["out_k"][l][o:o + len(sets[0]), h]
+                assert got.tobytes() == Ks[l][np.array(sets[0]) + cu[b], h].tobytes()
