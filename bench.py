@@ -216,6 +216,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
+    ap.add_argument("--per-layer", action="store_true",
+                    help="one index set per layer from the head-averaged score (fc_select_compact_ex)")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     args = ap.parse_args()
     if args.impl == "reference":
@@ -246,7 +248,8 @@ def main():
         Vd.append(v)
     comp = binding.Compressor(L, cfg.num_heads, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho,
                               cfg.gamma, cfg.min_keep, device=local_rank,
-                              group_bytes=(args.group_mib << 20) if args.group_mib else None)
+                              group_bytes=(args.group_mib << 20) if args.group_mib else None,
+                              per_layer=args.per_layer)
     input_bytes = sum(k.numel() * k.element_size() * 2 for k in Kd)
 
     def barrier():
@@ -329,7 +332,8 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": cfg.name + ": " + cfg.note, "layers": L, "kv_heads": cfg.num_heads,
+        "config": {"workload": cfg.name + ": " + cfg.note + (", one index set per layer" if args.per_layer else ""),
+                   "layers": L, "kv_heads": cfg.num_heads,
                    "head_dim": cfg.head_dim, "seqlens": list(cfg.seqlens), "storage_dtype": cfg.dtype,
                    "rho": cfg.rho, "gamma": cfg.gamma, "replicas": world,
                    "l2_policy": "inputs (%.2f GB) exceed L2; no flush" % (input_bytes / 1e9)},

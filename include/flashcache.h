@@ -217,6 +217,33 @@ fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const float *sco
                             void *workspace, size_t workspace_bytes, fc_stream stream);
 
 /*
+ * fc_select_compact with options (opt == NULL: exactly fc_select_compact).
+ *
+ *   per_layer  0: every KV head keeps its own tokens (the default reading: Eq. 10 over the head's
+ *              d channels).  1: the layer-wide reading of Sec. 3.1 / Eq. 5, where K^l is N x D with
+ *              D the whole hidden width: one index set per layer and sequence, ranked by the
+ *              deviation over all H*d channels, i.e. by the mean (here: the sum, same order) over
+ *              the heads of the per-head scores; every head keeps those tokens, out_idx holds the
+ *              same indices for every head.
+ *   protect    DEVICE uint8[T] or NULL.  A non-zero byte marks a token that must survive (text
+ *              tokens, attention sinks, a recent window; the paper compresses the visual KVs,
+ *              Sec. 1): it ranks before every unmarked token, marked tokens rank among themselves
+ *              by index.  The budget still counts them: a sequence with more marked tokens than
+ *              budget keeps the first `budget` of them, so give fc_allocate_budgets a min_keep of
+ *              at least the largest number of marked tokens in a sequence.
+ */
+typedef struct {
+  int32_t per_layer;
+  const void *protect;
+} fc_select_options;
+
+fc_status fc_select_compact_ex(fc_handle *h, const fc_kv_view *kv, const float *scores,
+                               const int32_t *budgets, const int64_t *out_offsets,
+                               void *out_k, void *out_v, int32_t *out_idx,
+                               int64_t out_capacity_rows, const fc_select_options *opt,
+                               void *workspace, size_t workspace_bytes, fc_stream stream);
+
+/*
  * fc_score_layer without any allocation (the paper has no counterpart: this is a
  * packaging variant of the same computation, added for integration reasons).
  *

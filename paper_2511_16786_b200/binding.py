@@ -25,7 +25,7 @@ EXPORTS = (
     "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count",
     "fc_set_group_bytes", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
-    "fc_score_layer", "fc_allocate_budgets", "fc_select_compact",
+    "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
     "fc_static_scratch_bytes", "fc_score_layer_static",
     "fc_compress_host_rows", "fc_compress_host_arena_bytes", "fc_compress_host",
 )
@@ -38,6 +38,10 @@ class fc_kv_view(ctypes.Structure):
         ("dtype", c_int32), ("num_heads", c_int32), ("head_dim", c_int32), ("batch", c_int32),
         ("cu_seqlens", POINTER(c_int32)),
     ]
+
+
+class fc_select_options(ctypes.Structure):
+    _fields_ = [("per_layer", c_int32), ("protect", c_void_p)]
 
 
 class fc_host_job(ctypes.Structure):
@@ -109,6 +113,10 @@ def _load() -> ctypes.CDLL:
     lib.fc_select_compact.argtypes = [c_void_p, POINTER(fc_kv_view), c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_size_t, c_void_p]
     lib.fc_select_compact.restype = c_int
+    lib.fc_select_compact_ex.argtypes = [c_void_p, POINTER(fc_kv_view), c_void_p, c_void_p, c_void_p,
+                                         c_void_p, c_void_p, c_void_p, c_int64, POINTER(fc_select_options),
+                                         c_void_p, c_size_t, c_void_p]
+    lib.fc_select_compact_ex.restype = c_int
     lib.fc_static_scratch_bytes.argtypes = []
     lib.fc_static_scratch_bytes.restype = c_size_t
     lib.fc_score_layer_static.argtypes = [POINTER(fc_kv_view), c_double, c_void_p, c_void_p, c_void_p]
@@ -297,6 +305,26 @@ def fc_select_compact(handle, k, v, cu_seqlens, scores, budgets, out_offsets, ou
            "fc_select_compact")
 
 
+def fc_select_compact_ex(handle, k, v, cu_seqlens, scores, budgets, out_offsets, out_k, out_v, out_idx,
+                         workspace, per_layer: bool = False, protect=None) -> None:
+    """fc_select_compact with options: per_layer (one index set per layer from the head-averaged
+    score) and protect (uint8 [T] on the device, non-zero = always ranked first)."""
+    cu = _cu_array(cu_seqlens)
+    view = make_view(k, v, cu)
+    cap = int(out_k.shape[0])
+    if protect is not None and (protect.dtype != torch.uint8 or not protect.is_cuda or protect.numel() != k.shape[0]
+                                or not protect.is_contiguous()):
+        raise ValueError("protect: contiguous uint8 device tensor with one entry per token")
+    opt = fc_select_options(per_layer=1 if per_layer else 0,
+                            protect=protect.data_ptr() if protect is not None else None)
+    _check(_lib.fc_select_compact_ex(handle, byref(view), c_void_p(scores.data_ptr()),
+                                     c_void_p(budgets.data_ptr()), c_void_p(out_offsets.data_ptr()),
+                                     c_void_p(out_k.data_ptr()), c_void_p(out_v.data_ptr()),
+                                     c_void_p(out_idx.data_ptr()), cap, byref(opt), c_void_p(workspace.data_ptr()),
+                                     workspace.numel() * workspace.element_size(), _stream()),
+           "fc_select_compact_ex")
+
+
 # ----------------------------------------------------------------------------
 # convenience: buffers for a whole model and the three-phase pass
 # ----------------------------------------------------------------------------
@@ -307,8 +335,14 @@ class Compressor:
 
     def __init__(self, num_layers: int, num_heads: int, head_dim: int, cu_seqlens, dtype, rho: float,
                  gamma: float = 0.2, min_keep: int = 1, device: int = 0, group_bytes: int | None = None,
-                 select_overlap: bool = True, score_overlap: bool = True):
+                 select_overlap: bool = True, score_overlap: bool = True, per_layer: bool = False,
+                 protect=None):
         self.L, self.H, self.d = num_layers, num_heads, head_dim
+        # selection options (fc_select_compact_ex): one index set per layer; uint8 [T] device mask of tokens to keep
+        self.per_layer = bool(per_layer)
+        self.protect = protect
+        self._opt = fc_select_options(per_layer=1 if per_layer else 0,
+                                      protect=protect.data_ptr() if protect is not None else None)
         self.cu = [int(x) for x in cu_seqlens]
         self.B = len(self.cu) - 1
         self.T = self.cu[-1]
@@ -410,12 +444,12 @@ class Compressor:
     def select_compact(self, K_layers, V_layers):
         m = self._marshal(K_layers, V_layers)
         st, h = _stream(), self.handle
-        call = _lib.fc_select_compact
+        call, opt = _lib.fc_select_compact_ex, byref(self._opt)
         for l in range(self.L):
             rc = call(h, m["refs"][l], m["scores"][l], m["budgets"][l], m["offsets"][l], m["out_k"][l],
-                      m["out_v"][l], m["out_idx"][l], m["cap"], m["ws"], m["ws_bytes"], st)
+                      m["out_v"][l], m["out_idx"][l], m["cap"], opt, m["ws"], m["ws_bytes"], st)
             if rc != FC_OK:
-                raise FlashCacheError(rc, "fc_select_compact")
+                raise FlashCacheError(rc, "fc_select_compact_ex")
 
     def compress(self, K_layers, V_layers):
         self.score(K_layers, V_layers)

@@ -177,14 +177,18 @@ constexpr int kSelKptMax = 16;      // scores per thread: 8 * 1024 * 16 = 131072
 // are then ranked in token order (block prefix + cluster prefix), written as
 // ascending indices, and their K/V rows are copied by the same block.
 // grid (kSelCluster * sequences in chunk, heads), cluster (kSelCluster, 1, 1).
-template <int kSelKpt>
+// PER_LAYER: one cluster per sequence (grid.y = 1) ranks the tokens by the sum over heads of their
+// scores (the order of the head-averaged deviation), writes the same indices for every head and
+// gathers the rows of all heads.  protect (may be null): a non-zero byte per token of the batch puts
+// that token before every unmarked one.
+template <int kSelKpt, bool PER_LAYER>
 __device__ __forceinline__ void
 select_gather_body(const float *__restrict__ scores, long long T, const SeqTable &st, int b0,
                 const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
                 int *__restrict__ out_idx, long long cap, int *__restrict__ status,
                 const char *__restrict__ kin, const char *__restrict__ vin, long long stride_token_b,
                 long long stride_head_b, int row_bytes, int H, char *__restrict__ out_k,
-                char *__restrict__ out_v) {
+                char *__restrict__ out_v, const unsigned char *__restrict__ protect) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ int lhist[4][256];          // this block's histograms, one per pass (read by the whole cluster)
@@ -196,7 +200,7 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned r = cluster.block_rank();
   const int bl = blockIdx.x / kSelCluster;
-  const int b = b0 + bl, h = blockIdx.y;
+  const int b = b0 + bl, h = PER_LAYER ? 0 : blockIdx.y;
   const int s0 = st.start[bl];
   const int n = st.start[bl + 1] - s0;
   int k = budgets[b];
@@ -218,7 +222,15 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
   nv = nv < 0 ? 0 : (nv > kSelKpt ? kSelKpt : nv);
   unsigned key[kSelKpt];
 #pragma unroll
-  for (int i = 0; i < kSelKpt; ++i) key[i] = (i < nv) ? score_key(sc[base + i]) : 0u;
+  for (int i = 0; i < kSelKpt; ++i) {
+    key[i] = 0u;
+    if (i < nv) {
+      float x = sc[base + i];
+      if (PER_LAYER)
+        for (int hh = 1; hh < H; ++hh) x += sc[(long long)hh * T + base + i];
+      key[i] = (protect && protect[s0 + base + i]) ? 0xFFFFFFFFu : score_key(x);
+    }
+  }
 
   for (int i = tid; i < 4 * 256; i += kSelThreads) (&lhist[0][0])[i] = 0;
   unsigned tau = 0;
@@ -323,12 +335,18 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
 #pragma unroll
   for (int i = 0; i < kSelKpt; ++i) {
     if (i < nv) {
+      int pos = -1;
       if (key[i] > tau) {
-        dst[g + (ti < need ? ti : need)] = base + i;
+        pos = g + (ti < need ? ti : need);
         ++g;
       } else if (key[i] == tau) {
-        if (ti < need) dst[g + ti] = base + i;
+        if (ti < need) pos = g + ti;
         ++ti;
+      }
+      if (pos >= 0) {
+        dst[pos] = base + i;
+        if (PER_LAYER)
+          for (int hh = 1; hh < H; ++hh) dst[(long long)hh * cap + pos] = base + i;
       }
     }
   }
@@ -343,9 +361,12 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
   for (int rr = warp; rr < count; rr += kSelThreads / 32) {
     const long long row = off + first + rr;
     const long long tok = (long long)s0 + dst[first + rr];
-    const long long src = tok * stride_token_b + (long long)h * stride_head_b;
-    const long long dsto = (row * H + h) * (long long)row_bytes;
-    for (int u = lane; u < 2 * n16; u += 32) {
+    const int per_head = 2 * n16;
+    for (int w = lane; w < (PER_LAYER ? H * per_head : per_head); w += 32) {
+      const int hh = PER_LAYER ? w / per_head : h;
+      const int u = PER_LAYER ? w - hh * per_head : w;
+      const long long src = tok * stride_token_b + (long long)hh * stride_head_b;
+      const long long dsto = (row * H + hh) * (long long)row_bytes;
       const bool isv = u >= n16;
       const int uu = isv ? u - n16 : u;
       const uint4 val = *reinterpret_cast<const uint4 *>((isv ? vin : kin) + src + 16ll * uu);
@@ -358,17 +379,17 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
 // launch in the stream may start as soon as every block of this one has begun, and this grid
 // does not finish before its predecessor has, so "the last launch is complete" still means
 // "all of them are".
-template <int kSelKpt>
+template <int kSelKpt, bool PER_LAYER>
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 k_select_gather(const float *__restrict__ scores, long long T, const __grid_constant__ SeqTable st, int b0,
                 const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
                 int *__restrict__ out_idx, long long cap, int *__restrict__ status,
                 const char *__restrict__ kin, const char *__restrict__ vin, long long stride_token_b,
                 long long stride_head_b, int row_bytes, int H, char *__restrict__ out_k,
-                char *__restrict__ out_v, int overlap) {
+                char *__restrict__ out_v, int overlap, const unsigned char *__restrict__ protect) {
   if (overlap) asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
-  select_gather_body<kSelKpt>(scores, T, st, b0, budgets, out_offsets, out_idx, cap, status, kin, vin,
-                              stride_token_b, stride_head_b, row_bytes, H, out_k, out_v);
+  select_gather_body<kSelKpt, PER_LAYER>(scores, T, st, b0, budgets, out_offsets, out_idx, cap, status, kin, vin,
+                                         stride_token_b, stride_head_b, row_bytes, H, out_k, out_v, protect);
   if (overlap) asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
 
@@ -419,6 +440,17 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
                                        void *out_k, void *out_v, int32_t *out_idx,
                                        int64_t out_capacity_rows, void *workspace,
                                        size_t workspace_bytes, fc_stream stream) {
+  return fc_select_compact_ex(h, kv, scores, budgets, out_offsets, out_k, out_v, out_idx, out_capacity_rows,
+                              nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" fc_status fc_select_compact_ex(fc_handle *h, const fc_kv_view *kv, const float *scores,
+                                          const int32_t *budgets, const int64_t *out_offsets,
+                                          void *out_k, void *out_v, int32_t *out_idx,
+                                          int64_t out_capacity_rows, const fc_select_options *opt,
+                                          void *workspace, size_t workspace_bytes, fc_stream stream) {
+  const bool per_layer = opt && opt->per_layer != 0;
+  const unsigned char *protect = opt ? static_cast<const unsigned char *>(opt->protect) : nullptr;
   if (!h || !kv || !kv->k || !kv->v || !scores || !budgets || !out_offsets || !out_k || !out_v || !out_idx)
     return FC_ERR_INVALID_ARG;
   if (kv->num_heads <= 0 || kv->head_dim <= 0 || out_capacity_rows < 0) return FC_ERR_INVALID_ARG;
@@ -449,10 +481,10 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
     const int per_thread = (nmax + kSelCluster * kSelThreads - 1) / (kSelCluster * kSelThreads);
     {
       ProfScope ps(h, FC_K_SELECT, st);
-#define FC_SEL_LAUNCH(KPT)                                                                              \
+#define FC_SEL_LAUNCH(KPT, PL)                                                                          \
   do {                                                                                                  \
     cudaLaunchConfig_t lc = {};                                                                         \
-    lc.gridDim = dim3(kSelCluster * nseq, kv->num_heads);                                               \
+    lc.gridDim = dim3(kSelCluster * nseq, (PL) ? 1 : kv->num_heads);                                    \
     lc.blockDim = dim3(kSelThreads);                                                                    \
     lc.stream = st;                                                                                     \
     cudaLaunchAttribute at[1];                                                                          \
@@ -460,18 +492,25 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
     at[0].val.programmaticStreamSerializationAllowed = 1;                                               \
     lc.attrs = at;                                                                                      \
     lc.numAttrs = h->select_overlap ? 1 : 0;                                                            \
-    launch_err = cudaLaunchKernelEx(&lc, k_select_gather<KPT>, scores, (long long)T, tab, b0, budgets,   \
+    launch_err = cudaLaunchKernelEx(&lc, k_select_gather<KPT, PL>, scores, (long long)T, tab, b0, budgets, \
         reinterpret_cast<const long long *>(out_offsets), out_idx, (long long)out_capacity_rows,        \
         h->status_word, static_cast<const char *>(kv->k), static_cast<const char *>(kv->v),             \
         (long long)(kv->stride_token * es), (long long)(kv->stride_head * es), (int)(kv->head_dim * es), \
         (int)kv->num_heads, static_cast<char *>(out_k), static_cast<char *>(out_v),                     \
-        (int)h->select_overlap);                                                                        \
+        (int)h->select_overlap, protect);                                                               \
   } while (0)
       cudaError_t launch_err = cudaSuccess;
-      if (per_thread <= 2) FC_SEL_LAUNCH(2);
-      else if (per_thread <= 4) FC_SEL_LAUNCH(4);
-      else if (per_thread <= 8) FC_SEL_LAUNCH(8);
-      else FC_SEL_LAUNCH(16);
+      if (per_layer) {
+        if (per_thread <= 2) FC_SEL_LAUNCH(2, true);
+        else if (per_thread <= 4) FC_SEL_LAUNCH(4, true);
+        else if (per_thread <= 8) FC_SEL_LAUNCH(8, true);
+        else FC_SEL_LAUNCH(16, true);
+      } else {
+        if (per_thread <= 2) FC_SEL_LAUNCH(2, false);
+        else if (per_thread <= 4) FC_SEL_LAUNCH(4, false);
+        else if (per_thread <= 8) FC_SEL_LAUNCH(8, false);
+        else FC_SEL_LAUNCH(16, false);
+      }
       if (launch_err != cudaSuccess) return FC_ERR_CUDA;
 #undef FC_SEL_LAUNCH
     }

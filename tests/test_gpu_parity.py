@@ -251,7 +251,7 @@ def test_budgets_special_cases(fc):
 
 
 # ---------------------------------------------------------------- selection + compaction
-def _gpu_select(fc, k, v, cu, scores, budgets, offsets, capacity):
+def _gpu_select(fc, k, v, cu, scores, budgets, offsets, capacity, per_layer=False, protect=None):
     T, H, d = k.shape
     h = fc.fc_create(0, 65536)
     try:
@@ -263,7 +263,12 @@ def _gpu_select(fc, k, v, cu, scores, budgets, offsets, capacity):
         out_v = torch.zeros((capacity, H, d), dtype=k.dtype, device="cuda")
         out_idx = torch.full((H, capacity), -1, dtype=torch.int32, device="cuda")
         ws = torch.empty(fc.fc_select_workspace_bytes(h, kd, vd, cu), dtype=torch.uint8, device="cuda")
-        fc.fc_select_compact(h, kd, vd, cu, sc, bd, of, out_k, out_v, out_idx, ws)
+        if per_layer or protect is not None:
+            pr = None if protect is None else torch.from_numpy(np.ascontiguousarray(protect, dtype=np.uint8)).cuda()
+            fc.fc_select_compact_ex(h, kd, vd, cu, sc, bd, of, out_k, out_v, out_idx, ws, per_layer=per_layer,
+                                    protect=pr)
+        else:
+            fc.fc_select_compact(h, kd, vd, cu, sc, bd, of, out_k, out_v, out_idx, ws)
         status = fc.fc_last_device_status(h)
         return out_k.cpu(), out_v.cpu(), out_idx.cpu().numpy(), status
     finally:
@@ -294,6 +299,84 @@ def test_select_exact_on_given_scores(fc, dtype):
             assert torch.equal(out_k[rows, h].view(torch.uint8), k[cu[b] + want, h].contiguous().view(torch.uint8))
             assert torch.equal(out_v[rows, h].view(torch.uint8), v[cu[b] + want, h].contiguous().view(torch.uint8))
     assert (out_idx[:, offsets[-1]:] == -1).all()                          # nothing past the last row
+
+
+@pytest.mark.parametrize("per_layer", [False, True])
+@pytest.mark.parametrize("with_mask", [False, True])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_select_options_exact_on_given_scores(fc, dtype, with_mask, per_layer):
+    # scores are multiples of 1/8, so their sums over heads are exact in fp32 and the order is the oracle's
+    rng = np.random.default_rng(3)
+    lens = [1, 37, 0, 1024, 3000, 5, 20000]
+    cu = [0] + [int(x) for x in np.cumsum(lens)]
+    T, H, d = cu[-1], 3, 128
+    k, v = _rand_kv(T, H, d, dtype, 4, smooth=False)
+    scores = rng.integers(0, 50, (H, T)).astype(np.float32) / 8.0
+    scores[0, cu[3] + 5] = np.nan
+    scores[1, cu[4]:cu[4] + 10] = np.inf
+    protect = None
+    if with_mask:
+        protect = (rng.random(T) < 0.02).astype(np.uint8)
+        protect[cu[3]:cu[3] + 4] = 1                     # sinks
+        protect[cu[4] - 16:cu[4]] = 1                    # a recent window
+        protect[cu[1]:cu[2]] = 1                         # a whole sequence marked: more marked tokens than budget
+    budgets = [1, 11, 0, 205, 2999, 5, 1234]
+    offsets = [0] + [int(x) for x in np.cumsum(budgets)]
+    out_k, out_v, out_idx, status = _gpu_select(fc, k, v, cu, scores, budgets, offsets, offsets[-1] + 3,
+                                                per_layer=per_layer, protect=protect)
+    assert status == 0
+    for h in range(H):
+        for b, n in enumerate(lens):
+            dev = scores[:, cu[b]:cu[b + 1]].astype(np.float64)
+            dev = O.layer_score(dev) if per_layer else dev[h]
+            pr = None if protect is None else protect[cu[b]:cu[b + 1]]
+            want = O.select_topk_protected(dev, budgets[b], pr)
+            got = out_idx[h, offsets[b]:offsets[b + 1]]
+            np.testing.assert_array_equal(got, want)
+            rows = slice(offsets[b], offsets[b + 1])
+            assert torch.equal(out_k[rows, h].view(torch.uint8), k[cu[b] + want, h].contiguous().view(torch.uint8))
+            assert torch.equal(out_v[rows, h].view(torch.uint8), v[cu[b] + want, h].contiguous().view(torch.uint8))
+    assert (out_idx[:, offsets[-1]:] == -1).all()
+
+
+def test_compress_per_layer_with_protected_tokens_matches_oracle(fc):
+    from paper_2511_16786_b200.binding import Compressor
+    base = S.paper_configs()["cfg2"]
+    cfg = S.scaled(base, "per_layer_small", num_layers=4, seqlens=(2048, 700), min_keep=24)
+    L, cu = cfg.num_layers, cfg.cu_seqlens
+    Ks, Vs = zip(*[S.make_layer(cfg, l, "cpu") for l in range(L)])
+    protect = np.zeros(cu[-1], dtype=np.uint8)
+    for b in range(2):
+        protect[cu[b]:cu[b] + 4] = 1                     # sinks
+        protect[cu[b + 1] - 16:cu[b + 1]] = 1            # recent window
+    comp = Compressor(L, cfg.num_heads, cfg.head_dim, cu, cfg.torch_dtype, cfg.rho, cfg.gamma, cfg.min_keep,
+                      per_layer=True, protect=torch.from_numpy(protect).cuda())
+    comp.compress([k.cuda() for k in Ks], [v.cuda() for v in Vs])
+    comp.check_device_status()
+    budgets, offsets = comp.budgets.cpu().numpy(), comp.offsets.cpu().numpy()
+    idx = comp.out_idx.cpu().numpy()
+    tol = TOL[cfg.torch_dtype]
+    for l in range(L):
+        o, _ = O.score_layer(Ks[l].double().numpy(), Vs[l].double().numpy(), cu, cfg.gamma, "fft")
+        for b, n in enumerate(cfg.seqlens):
+            kb, off = int(budgets[l, b]), int(offsets[l, b])
+            got = idx[l, 0, off:off + kb]
+            for h in range(1, cfg.num_heads):
+                np.testing.assert_array_equal(idx[l, h, off:off + kb], got)       # one index set per layer
+            pr = protect[cu[b]:cu[b + 1]]
+            assert set(np.flatnonzero(pr)) <= set(got.tolist())                    # 20 marked tokens, min_keep 24
+            dev = O.layer_score(o[:, cu[b]:cu[b + 1]])
+            want = O.select_topk_protected(dev, kb, pr)
+            diff = np.setxor1d(got, want)
+            if len(diff):
+                tau = np.sort(dev[pr == 0])[::-1][kb - int(pr.sum()) - 1]
+                assert np.all(np.abs(dev[diff] - tau) <= tol * tau)
+            for h in range(cfg.num_heads):
+                gk = comp.out_k[l][off:off + kb, h].cpu().view(torch.uint8)
+                assert torch.equal(gk, Ks[l][cu[b] + got, h].contiguous().view(torch.uint8))
+                gv = comp.out_v[l][off:off + kb, h].cpu().view(torch.uint8)
+                assert torch.equal(gv, Vs[l][cu[b] + got, h].contiguous().view(torch.uint8))
+    comp.close()
 
 
 def test_select_capacity_overflow_is_reported_not_written(fc):
