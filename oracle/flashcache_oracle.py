@@ -192,6 +192,26 @@ def score_layer(K: np.ndarray, V: np.ndarray, cu_seqlens, gamma: float, tier: st
     return scores, energy
 
 
+def power_spectrum(K: np.ndarray, V: np.ndarray, cu_seqlens, tier: str = "literal") -> np.ndarray:
+    """Power spectrum of one layer (Eq. 11): P[m] = |C[m]|^2 with C[m] the row of DCT
+    coefficients of frequency m over all channels of all heads, for K and for V.
+    Returns [T, 2]: row cu[b] + m holds (P_k[m], P_v[m]) of sequence b."""
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    T = K.shape[0]
+    dct = dct_literal if tier == "literal" else dct_fft
+    out = np.zeros((T, 2), dtype=np.float64)
+    for b in range(len(cu_seqlens) - 1):
+        s, e = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        if e == s:
+            continue
+        Ck = dct(K[s:e].reshape(e - s, -1))
+        Cv = dct(V[s:e].reshape(e - s, -1))
+        out[s:e, 0] = np.sum(Ck * Ck, axis=1)
+        out[s:e, 1] = np.sum(Cv * Cv, axis=1)
+    return out
+
+
 def energy_ratio(energy_row) -> float:
     """R^l = R_k^l + R_v^l of Eq. 12 from (hiK, totK, hiV, totV); a matrix with
     zero total energy contributes 0."""

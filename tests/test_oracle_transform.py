@@ -229,3 +229,50 @@ def test_generator_structure_low_frequency_dominates():
     # rows replaced by N(0, 5) outliers stand far above the noise floor
     top = O.select_topk(dev, 20)
     assert dev[top].min() > 20 * np.median(dev)
+
+
+# ---------------------------------------------------------------- power spectrum (Eq. 11)
+def test_power_spectrum_of_a_single_basis_vector_is_one_line():
+    # x = a * alpha[m0] * phi_N(m0, .) in one channel has C = a * delta[m - m0] (orthonormal rows, Eq. 7),
+    # so P is a^2 at m0 and zero elsewhere
+    N, H, d = 37, 2, 3
+    for m0 in (0, 1, 9, 36):
+        K = np.zeros((N, H, d))
+        V = np.zeros((N, H, d))
+        m1 = (m0 + 5) % N
+        K[:, 1, 2] = 3.0 * O.alpha(N)[m0] * O.phi(N)[m0]
+        V[:, 0, 0] = -2.0 * O.alpha(N)[m1] * O.phi(N)[m1]
+        P = O.power_spectrum(K, V, [0, N])
+        want = np.zeros((N, 2))
+        want[m0, 0] = 9.0
+        want[m1, 1] = 4.0
+        np.testing.assert_allclose(P, want, atol=1e-12)
+
+
+@pytest.mark.parametrize("tier", ["literal", "fft"])
+def test_power_spectrum_parseval_and_band_sums(tier):
+    rng = np.random.default_rng(11)
+    lens = [24, 0, 9, 16]
+    cu = [0] + [int(x) for x in np.cumsum(lens)]
+    K = rng.standard_normal((cu[-1], 2, 4))
+    V = rng.standard_normal((cu[-1], 2, 4)) * 2.0
+    P = O.power_spectrum(K, V, cu, tier)
+    _, energy = O.score_layer(K, V, cu, 0.25, "literal")
+    for b, n in enumerate(lens):
+        if n == 0:
+            continue
+        s, e = cu[b], cu[b + 1]
+        assert np.isclose(P[s:e, 0].sum(), (K[s:e] ** 2).sum(), rtol=1e-12)          # Parseval: orthonormal transform
+        assert np.isclose(P[s:e, 1].sum(), (V[s:e] ** 2).sum(), rtol=1e-12)
+        om = O.cutoff_index(n, 0.25)
+        np.testing.assert_allclose([P[s + om + 1:e, 0].sum(), P[s:e, 0].sum(), P[s + om + 1:e, 1].sum(), P[s:e, 1].sum()],
+                                   energy[b], rtol=1e-10)                            # the sums Eq. 12 is made of
+
+
+def test_power_spectrum_tiers_agree():
+    rng = np.random.default_rng(12)
+    for n in (1, 2, 7, 31, 64):
+        K = rng.standard_normal((n, 1, 5))
+        V = rng.standard_normal((n, 1, 5))
+        np.testing.assert_allclose(O.power_spectrum(K, V, [0, n], "fft"), O.power_spectrum(K, V, [0, n], "literal"),
+                                   rtol=1e-9, atol=1e-12)
