@@ -217,6 +217,22 @@ fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const float *sco
                             void *workspace, size_t workspace_bytes, fc_stream stream);
 
 /*
+ * Spectrum diagnostics (Sec. 3.2.2, Eq. 11; the curves of the paper's energy-distribution figures):
+ * the power spectrum of one layer, P_k[m] = |C_k[m]|^2 and P_v[m] = |C_v[m]|^2, where C[m] is the row of
+ * DCT coefficients (Eq. 6-7) of frequency m over all channels of all KV heads.  Its band sums are the
+ * numerators and denominators of Eq. 12 (what fc_score_layer returns as `energy`), its running sum is
+ * the cumulative-energy curve from which a cutoff gamma can be read.  Not on the compression path:
+ * it runs the generic transform kernels on the caller's stream.
+ *
+ *   spectrum   DEVICE double[T][2]: row cu_seqlens[b] + m = (P_k[m], P_v[m]) of sequence b.
+ *   workspace  DEVICE, 256-byte aligned, >= fc_power_spectrum_workspace_bytes().
+ * Errors: as fc_score_layer.
+ */
+size_t fc_power_spectrum_workspace_bytes(const fc_handle *h, const fc_kv_view *kv);
+fc_status fc_power_spectrum(fc_handle *h, const fc_kv_view *kv, double *spectrum,
+                            void *workspace, size_t workspace_bytes, fc_stream stream);
+
+/*
  * fc_select_compact with options (opt == NULL: exactly fc_select_compact).
  *
  *   per_layer  0: every KV head keeps its own tokens (the default reading: Eq. 10 over the head's

@@ -26,6 +26,7 @@ EXPORTS = (
     "fc_set_group_bytes", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
+    "fc_power_spectrum_workspace_bytes", "fc_power_spectrum",
     "fc_static_scratch_bytes", "fc_score_layer_static",
     "fc_compress_host_rows", "fc_compress_host_arena_bytes", "fc_compress_host",
 )
@@ -117,6 +118,10 @@ def _load() -> ctypes.CDLL:
                                          c_void_p, c_void_p, c_void_p, c_int64, POINTER(fc_select_options),
                                          c_void_p, c_size_t, c_void_p]
     lib.fc_select_compact_ex.restype = c_int
+    lib.fc_power_spectrum_workspace_bytes.argtypes = [c_void_p, POINTER(fc_kv_view)]
+    lib.fc_power_spectrum_workspace_bytes.restype = c_size_t
+    lib.fc_power_spectrum.argtypes = [c_void_p, POINTER(fc_kv_view), c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.fc_power_spectrum.restype = c_int
     lib.fc_static_scratch_bytes.argtypes = []
     lib.fc_static_scratch_bytes.restype = c_size_t
     lib.fc_score_layer_static.argtypes = [POINTER(fc_kv_view), c_double, c_void_p, c_void_p, c_void_p]
@@ -274,6 +279,20 @@ def fc_compress_host_rows(num_layers: int, cu_seqlens, rho: float, min_keep: int
     cu = _cu_array(cu_seqlens)
     return int(_lib.fc_compress_host_rows(int(num_layers), len(cu) - 1, ctypes.cast(cu, POINTER(c_int32)),
                                           float(rho), int(min_keep)))
+
+
+def fc_power_spectrum_workspace_bytes(handle, k, v, cu_seqlens) -> int:
+    cu = _cu_array(cu_seqlens)
+    view = make_view(k, v, cu)
+    return int(_lib.fc_power_spectrum_workspace_bytes(handle, byref(view)))
+
+
+def fc_power_spectrum(handle, k, v, cu_seqlens, spectrum, workspace) -> None:
+    """spectrum: float64 [T, 2] on the device: (P_k[m], P_v[m]) at row cu[b] + m."""
+    cu = _cu_array(cu_seqlens)
+    view = make_view(k, v, cu)
+    _check(_lib.fc_power_spectrum(handle, byref(view), c_void_p(spectrum.data_ptr()), c_void_p(workspace.data_ptr()),
+                                  workspace.numel() * workspace.element_size(), _stream()), "fc_power_spectrum")
 
 
 def fc_reset_ordering(handle) -> None:

@@ -448,6 +448,154 @@ k_energy_finalize(const double *__restrict__ part_tot, int n_tot, const double *
   if (tid < 4) energy[tid] = red[tid][0];
 }
 
+// ---------------------------------------------------------------------------
+// Power spectrum of a layer (Eq. 11): P_k[m], P_v[m] = sum over heads and channels of C[m,c]^2.
+// With z = k + j*v reordered as in pass 1 and Z its unnormalised N-point DFT, the spectra of the two
+// real sequences are Y_k[q] = (Z[q] + conj(Z[N-q]))/2 and Y_v[q] = (Z[q] - conj(Z[N-q]))/(2j), and with
+// w = exp(-j*pi*q/(2N)) * Y[q]:  C[q] = alpha[q]*Re(w),  C[N-q] = -alpha[N-q]*Im(w)  (alpha of Eq. 7).
+// ---------------------------------------------------------------------------
+// (P, Q) = (Z[q], Z[N-q]), t = exp(-j*pi*q/(2N)).  lo = (P_k[q], P_v[q]), hi = (P_k[N-q], P_v[N-q]).
+__device__ __forceinline__ void power_of_pair(float2 P, float2 Q, float2 t, int q, float invN, float2 &lo, float2 &hi) {
+  if (q == 0) {
+    lo = make_float2(P.x * P.x * invN, P.y * P.y * invN);
+    hi = lo;
+    return;
+  }
+  const float2 yk = make_float2(0.5f * (P.x + Q.x), 0.5f * (P.y - Q.y));
+  const float2 yv = make_float2(0.5f * (P.y + Q.y), 0.5f * (Q.x - P.x));
+  const float2 wk = cmul(yk, t), wv = cmul(yv, t);
+  const float a2 = 2.f * invN;
+  lo = make_float2(a2 * wk.x * wk.x, a2 * wv.x * wv.x);
+  hi = make_float2(a2 * wk.y * wk.y, a2 * wv.y * wv.y);
+}
+
+// Power-of-two N: pass 2 without the way back.  grid (N1/2 + 1, NY); block y works through the column
+// slices y, y + NY, ... of the group and writes its sums over them to partial[y][q].
+__global__ void __launch_bounds__(kThreads)
+k_pass2_power(FftPlan plan, int N1, int ncol_ws, int cs2_log2, const float2 *__restrict__ ws,
+              const float2 *__restrict__ master, int master_len, float2 *__restrict__ partial) {
+  extern __shared__ float2 smem[];
+  const int N2 = plan.len, cs2 = 1 << cs2_log2;
+  const int N = N1 * N2;
+  const int tid = threadIdx.x;
+  const int k1a = blockIdx.x, k1b = (N1 - k1a) % N1;
+  const int halves = (k1b != k1a) ? 2 : 1;
+  const int ncolT_log2 = cs2_log2 + (halves - 1);
+  const int ncolT = 1 << ncolT_log2;
+
+  float2 *S = smem;                                    // [N2][2*cs2] at most
+  float2 *tw = S + (size_t)N2 * 2 * cs2;               // [N2]
+  float2 *twN = tw + N2;                               // [2][N2]
+  unsigned short *rev = reinterpret_cast<unsigned short *>(twN + 2 * N2);   // [N2]
+  unsigned short *pos_of = rev + N2;                                       // [N2]
+  float2 *acc = reinterpret_cast<float2 *>(pos_of + N2);                   // [N2][2]: (P_k, P_v) of row (pos, half)
+
+  const int mstepN = master_len / N;
+  for (int i = tid; i < N2; i += kThreads) {
+    tw[i] = master[(size_t)i * (master_len / N2)];
+    twN[i] = master[(size_t)(((long long)i * k1a) % N) * mstepN];
+    twN[N2 + i] = master[(size_t)(((long long)i * k1b) % N) * mstepN];
+    const int k = digit_rev(plan, i);
+    rev[i] = (unsigned short)k;
+    pos_of[k] = (unsigned short)i;
+    acc[2 * i] = make_float2(0.f, 0.f);
+    acc[2 * i + 1] = make_float2(0.f, 0.f);
+  }
+  __syncthreads();
+
+  const int tstep = master_len / (4 * N);
+  const float invN = 1.f / (float)N;
+  for (int sl = blockIdx.y; sl < ncol_ws / cs2; sl += gridDim.y) {
+    const int gc0 = sl * cs2;
+    for (int w = tid; w < N2 * ncolT; w += kThreads) {
+      const int n2 = w >> ncolT_log2, col = w & (ncolT - 1);
+      const int hf = col >> cs2_log2, c = col & (cs2 - 1);
+      const int k1 = hf ? k1b : k1a;
+      S[w] = cmul(ws[((size_t)k1 * N2 + n2) * ncol_ws + gc0 + c], twN[hf * N2 + n2]);
+    }
+    __syncthreads();
+    fft_forward_tile(plan, S, ncolT_log2, tw, tid, kThreads);
+    // every pair {q, N-q} is owned by the thread that meets the smaller bin; each location of S receives
+    // the contribution of its own bin
+    for (int w = tid; w < N2 * ncolT; w += kThreads) {
+      const int pos = w >> ncolT_log2, col = w & (ncolT - 1);
+      const int hf = col >> cs2_log2, c = col & (cs2 - 1);
+      const int k1 = hf ? k1b : k1a;
+      const int q = k1 + N1 * (int)rev[pos];
+      const int qp = (N - q) % N;
+      if (q > qp) continue;
+      const int k1p = qp % N1, k2p = qp / N1;
+      const int hfp = (k1p == k1) ? hf : 1 - hf;
+      const int wp = ((int)pos_of[k2p] << ncolT_log2) + (hfp << cs2_log2) + c;
+      float2 lo, hi;
+      power_of_pair(S[w], S[wp], master[(size_t)q * tstep], q, invN, lo, hi);
+      S[w] = lo;
+      if (qp != q) S[wp] = hi;
+    }
+    __syncthreads();
+    for (int r = tid; r < N2 * halves; r += kThreads) {      // row r = (pos, half): sum its cs2 columns in order
+      const int pos = r / halves, hf = r - pos * halves;
+      const float2 *row = S + ((size_t)pos << ncolT_log2) + (hf << cs2_log2);
+      float2 a = acc[2 * pos + hf];
+      for (int c = 0; c < cs2; ++c) { a.x += row[c].x; a.y += row[c].y; }
+      acc[2 * pos + hf] = a;
+    }
+    __syncthreads();
+  }
+  for (int r = tid; r < N2 * halves; r += kThreads) {
+    const int pos = r / halves, hf = r - pos * halves;
+    const int q = (hf ? k1b : k1a) + N1 * (int)rev[pos];
+    partial[(size_t)blockIdx.y * N + q] = acc[2 * pos + hf];
+  }
+}
+
+// Other N (chirp path): from the N-point spectrum spec[q][col].  grid (N/2 + 1): block q sums the pair
+// {q, N-q} over all columns of the group and writes partial[q], partial[N-q].
+__global__ void __launch_bounds__(kThreads)
+k_spec_power(const float2 *__restrict__ spec, int ncol, int N, float2 *__restrict__ partial) {
+  const int q = blockIdx.x, qp = (N - q) % N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float s, c;
+  sincospif(-__fdiv_rn((float)q, (float)(2 * N)), &s, &c);
+  const float2 t = make_float2(c, s);
+  const float invN = 1.f / (float)N;
+  float a[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int col = tid; col < ncol; col += kThreads) {
+    float2 lo, hi;
+    power_of_pair(spec[(size_t)q * ncol + col], spec[(size_t)qp * ncol + col], t, q, invN, lo, hi);
+    a[0] += lo.x; a[1] += lo.y; a[2] += hi.x; a[3] += hi.y;
+  }
+  __shared__ float red[4][kThreads / 32];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    a[i] = warp_sum(a[i]);
+    if (lane == 0) red[i][warp] = a[i];
+  }
+  __syncthreads();
+  if (tid == 0) {
+    float r[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int w = 0; w < kThreads / 32; ++w)
+      for (int i = 0; i < 4; ++i) r[i] += red[i][w];
+    partial[q] = make_float2(r[0], r[1]);
+    if (qp != q) partial[qp] = make_float2(r[2], r[3]);
+  }
+}
+
+// spectrum[m] (+)= sum over y of partial[y][m], in fp64 and in a fixed order.
+__global__ void k_power_accumulate(const float2 *__restrict__ partial, int ny, int N, double *__restrict__ spectrum,
+                                   int first) {
+  const int m = blockIdx.x * blockDim.x + threadIdx.x;
+  if (m >= N) return;
+  double a = first ? 0.0 : spectrum[2 * m], b = first ? 0.0 : spectrum[2 * m + 1];
+  for (int y = 0; y < ny; ++y) {
+    const float2 p = partial[(size_t)y * N + m];
+    a += (double)p.x;
+    b += (double)p.y;
+  }
+  spectrum[2 * m] = a;
+  spectrum[2 * m + 1] = b;
+}
+
 __global__ void k_zero_energy(double *energy) {
   if (threadIdx.x < 4) energy[threadIdx.x] = 0.0;
 }
@@ -1044,7 +1192,115 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   return fc_after_launch(h);
 }
 
+// Column slices of one launch of k_pass2_power that run side by side (the rest are looped over).
+constexpr int kPowerNY = 16;
+
+size_t power_partial_bytes(int N) { return align_up((size_t)kPowerNY * N * sizeof(float2), 256); }
+
+// Power spectrum of one sequence (Eq. 11) into spectrum[2*m .. 2*m+1], m < N.  Generic kernels, caller's stream.
+template <typename T>
+fc_status power_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, int b, double *spectrum, char *wsb) {
+  const int start = kv->cu_seqlens[b];
+  const int N = kv->cu_seqlens[b + 1] - start;
+  if (N == 0) return FC_OK;
+  const int d = kv->head_dim, H = kv->num_heads;
+  const SeqPlan sp = plan_sequence(N, false);
+  const ScoreLayout L = layout_for(h, sp, H, d);
+  float2 *ws = reinterpret_cast<float2 *>(wsb + L.off_ws);
+  float2 *spec = reinterpret_cast<float2 *>(wsb + L.off_spec);
+  float2 *hhat = reinterpret_cast<float2 *>(wsb + L.off_hhat);
+  float2 *hcol = reinterpret_cast<float2 *>(wsb + L.off_hcol);
+  float2 *partial = reinterpret_cast<float2 *>(wsb + L.total);
+  double *out = spectrum + 2 * (size_t)start;
+  const T *kp = static_cast<const T *>(kv->k) + (long long)start * kv->stride_token;
+  const T *vp = static_cast<const T *>(kv->v) + (long long)start * kv->stride_token;
+  const FftPlan p1 = make_plan(sp.N1);
+  fc_status s;
+  if (sp.bluestein) {
+    ChirpKernelLoader cl{N, sp.Nfft};
+    if ((s = launch_pass1(h, st, cl, sp, 8, 8, hcol, nullptr)) != FC_OK) return s;
+    if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
+  }
+  bool first = true;
+  for (int h0 = 0; h0 < H; h0 += L.heads_per_group) {
+    const int hg = (H - h0 < L.heads_per_group) ? H - h0 : L.heads_per_group;
+    const int ncol_ws = hg * d;
+    if (!sp.bluestein) {
+      KvLoader<T, false> ld{kp, vp, kv->stride_token, kv->stride_head, h0, d, N, 0.f, 0.f};
+      if ((s = launch_pass1(h, st, ld, sp, ncol_ws, sp.cs, ws, nullptr)) != FC_OK) return s;
+      const FftPlan p2 = make_plan(sp.N2);
+      const size_t sm = smem_pass2(sp, sp.cs2) + (size_t)sp.N2 * 2 * sizeof(float2);
+      if ((s = set_smem(k_pass2_power, sm)) != FC_OK) return s;
+      const int slices = ncol_ws / sp.cs2, ny = slices < kPowerNY ? slices : kPowerNY;
+      k_pass2_power<<<dim3(sp.N1 / 2 + 1, ny), kThreads, sm, st>>>(p2, sp.N1, ncol_ws, ilog2(sp.cs2), ws, h->master,
+                                                                   h->master_len, partial);
+      if ((s = fc_after_launch(h)) != FC_OK) return s;
+      k_power_accumulate<<<(N + 255) / 256, 256, 0, st>>>(partial, ny, N, out, first ? 1 : 0);
+      if ((s = fc_after_launch(h)) != FC_OK) return s;
+      first = false;
+      continue;
+    }
+    const float invM = 1.f / (float)sp.Nfft;
+    const int sub = L.sub_cols, cs = (sub % 64 == 0) ? sp.cs : 32;
+    const int ngroups = (hg == 1) ? d / sub : 1;
+    const int ncol = (hg == 1) ? sub : ncol_ws;
+    int cs2 = sp.cs2;
+    while (ncol % cs2) cs2 >>= 1;
+    const size_t sm3c = smem_pass13(sp, cs);
+    for (int cg = 0; cg < ngroups; ++cg) {
+      const int dd = (hg == 1) ? sub : d;
+      KvLoader<T, true> ld{kp + cg * sub, vp + cg * sub, kv->stride_token, kv->stride_head, h0, dd, N, 0.f, 0.f};
+      if ((s = launch_pass1(h, st, ld, sp, ncol, cs, ws, nullptr)) != FC_OK) return s;
+      if ((s = launch_pass2<MID_MULH>(h, st, sp, ncol, cs2, ws, 0, hhat, invM)) != FC_OK) return s;
+      if ((s = set_smem(k_pass3<EPI_SPEC, true>, sm3c)) != FC_OK) return s;
+      k_pass3<EPI_SPEC, true><<<dim3(sp.N2, ncol / cs), kThreads, sm3c, st>>>(
+          p1, sp.N2, N, ncol, ilog2(cs), ws, h->master, h->master_len, spec, nullptr, 0, dd, 0, 0.f, nullptr, 0.f, 0);
+      if ((s = fc_after_launch(h)) != FC_OK) return s;
+      k_spec_power<<<N / 2 + 1, kThreads, 0, st>>>(spec, ncol, N, partial);
+      if ((s = fc_after_launch(h)) != FC_OK) return s;
+      k_power_accumulate<<<(N + 255) / 256, 256, 0, st>>>(partial, 1, N, out, first ? 1 : 0);
+      if ((s = fc_after_launch(h)) != FC_OK) return s;
+      first = false;
+    }
+  }
+  return FC_OK;
+}
+
 }  // namespace
+
+extern "C" size_t fc_power_spectrum_workspace_bytes(const fc_handle *h, const fc_kv_view *kv) {
+  if (validate_view(h, kv) != FC_OK) return 0;
+  size_t need = 256;
+  for (int b = 0; b < kv->batch; ++b) {
+    const int N = kv->cu_seqlens[b + 1] - kv->cu_seqlens[b];
+    if (N == 0) continue;
+    const size_t t = layout_for(h, plan_sequence(N, false), kv->num_heads, kv->head_dim).total + power_partial_bytes(N);
+    if (t > need) need = t;
+  }
+  return need;
+}
+
+extern "C" fc_status fc_power_spectrum(fc_handle *h, const fc_kv_view *kv, double *spectrum, void *workspace,
+                                       size_t workspace_bytes, fc_stream stream) {
+  fc_status s = validate_view(h, kv);
+  if (s != FC_OK) return s;
+  if (!spectrum) return FC_ERR_INVALID_ARG;
+  const size_t need = fc_power_spectrum_workspace_bytes(h, kv);
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return FC_ERR_WORKSPACE;
+  int dev = -1;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if ((s = fc_flush_pending(h, st)) != FC_OK) return s;     // the workspace may still be in use on the internal streams
+  for (int b = 0; b < kv->batch && s == FC_OK; ++b) {
+    switch (kv->dtype) {
+      case FC_F32: s = power_sequence<float>(h, st, kv, b, spectrum, (char *)workspace); break;
+      case FC_F16: s = power_sequence<__half>(h, st, kv, b, spectrum, (char *)workspace); break;
+      default: s = power_sequence<__nv_bfloat16>(h, st, kv, b, spectrum, (char *)workspace); break;
+    }
+  }
+  return s;
+}
 
 extern "C" fc_status fc_describe_plan(const fc_handle *h, int32_t seqlen, int32_t out[4]) {
   if (!h || !out || seqlen < 1) return FC_ERR_INVALID_ARG;

@@ -180,6 +180,48 @@ def test_scores_arbitrary_length_in_column_groups(fc, d, group_bytes):
     np.testing.assert_allclose(g1, g2, rtol=2e-3, atol=1e-6 * float(g2.max()))
 
 
+# ---------------------------------------------------------------- power spectrum (Eq. 11)
+@pytest.mark.parametrize("lens,H,d,dtype", [([16], 1, 64, torch.float32), ([1024], 2, 128, torch.float32),
+                                            ([1, 2, 3, 8, 300, 0, 1000], 2, 64, torch.float32),
+                                            ([4096, 777, 2048], 3, 128, torch.bfloat16),
+                                            ([32768], 1, 128, torch.float16), ([5000], 2, 192, torch.float32)])
+def test_power_spectrum_matches_oracle(fc, lens, H, d, dtype):
+    cu = [0] + [int(x) for x in np.cumsum(lens)]
+    T = cu[-1]
+    k, v = _rand_kv(T, H, d, dtype, 77 + T)
+    h = fc.fc_create(0, max(lens))
+    try:
+        kd, vd = k.cuda(), v.cuda()
+        spec = torch.full((T, 2), -1.0, dtype=torch.float64, device="cuda")
+        ws = torch.empty(fc.fc_power_spectrum_workspace_bytes(h, kd, vd, cu), dtype=torch.uint8, device="cuda")
+        fc.fc_power_spectrum(h, kd, vd, cu, spec, ws)
+        assert fc.fc_last_device_status(h) == 0
+        got = spec.cpu().numpy()
+        # the band sums are what fc_score_layer reports as energies
+        scores = torch.empty((H, T), dtype=torch.float32, device="cuda")
+        energy = torch.empty((len(lens), 4), dtype=torch.float64, device="cuda")
+        ws2 = torch.empty(fc.fc_score_workspace_bytes(h, kd, vd, cu), dtype=torch.uint8, device="cuda")
+        fc.fc_score_layer(h, kd, vd, cu, 0.2, scores, energy, ws2)
+        assert fc.fc_last_device_status(h) == 0
+        en = energy.cpu().numpy()
+    finally:
+        fc.fc_destroy(h)
+    want = O.power_spectrum(k.double().numpy(), v.double().numpy(), cu, "fft")
+    for b, n in enumerate(lens):
+        if n == 0:
+            continue
+        s, e = cu[b], cu[b + 1]
+        for j in range(2):
+            # fp32 transforms: every bin carries an error proportional to the largest bins of the sequence
+            floor = 1e-6 * want[s:e, j].max()
+            err = np.abs(got[s:e, j] - want[s:e, j]) / np.maximum(want[s:e, j], floor)
+            assert err.max() <= 2e-3, "sequence %d matrix %d: %.3e" % (b, j, err.max())
+            np.testing.assert_allclose(got[s:e, j].sum(), want[s:e, j].sum(), rtol=1e-5)          # Parseval
+        om = O.cutoff_index(n, 0.2)
+        np.testing.assert_allclose(got[s + om + 1:e, 0].sum(), en[b, 0], rtol=2e-3, atol=1e-6 * en[b, 1])
+        np.testing.assert_allclose(got[s + om + 1:e, 1].sum(), en[b, 2], rtol=2e-3, atol=1e-6 * en[b, 3])
+
+
 @pytest.mark.parametrize("mode", [1, 2])
 @pytest.mark.parametrize("lag", [1, 2, 3])
 @pytest.mark.parametrize("N,H,dtype", [(4096, 3, torch.float32), (8192, 2, torch.bfloat16), (16384, 1, torch.float16),
