@@ -395,3 +395,40 @@ def compress(K_layers, V_layers, cu_seqlens, gamma: float, rho: float,
         out_v.append(ov)
     return dict(scores=scores, energy=energy, budgets=budgets, offsets=offsets,
                 idx=idx, out_k=out_k, out_v=out_v)
+
+
+# ---------------------------------------------------------------------------
+# Decoding stage on the compacted cache (Sec. 3.1, Eq. 3-4)
+# ---------------------------------------------------------------------------
+def decode_attention(q, cache_k, cache_v, offsets, tail_k=None, tail_v=None, tail_len=None):
+    """Output of one decoding step for one layer: x_out = Softmax(Q_t K^T / sqrt(D)) V (Eq. 4),
+    per head with D = d channels, K and V being the kept rows of the sequence followed by the
+    KV pairs appended since the prefill (Eq. 3), which are never compressed.
+
+    q: [B, Hq, d], Hq a multiple of the H KV heads (query head j reads KV head j // (Hq/H));
+    cache_k, cache_v: [rows, H, d], sequence b owns rows offsets[b] .. offsets[b+1];
+    tail_k, tail_v: [B, cap, H, d] with tail_len[b] valid rows (optional).
+    Returns [B, Hq, d] in fp64; a sequence without any row gives zeros."""
+    q = np.asarray(q, dtype=np.float64)
+    ck = np.asarray(cache_k, dtype=np.float64)
+    cv = np.asarray(cache_v, dtype=np.float64)
+    B, Hq, d = q.shape
+    H = ck.shape[1]
+    G = Hq // H
+    out = np.zeros((B, Hq, d), dtype=np.float64)
+    for b in range(B):
+        lo, hi = int(offsets[b]), int(offsets[b + 1])
+        for j in range(Hq):
+            h = j // G
+            K = ck[lo:hi, h]
+            V = cv[lo:hi, h]
+            if tail_k is not None:
+                n = int(tail_len[b])
+                K = np.concatenate([K, np.asarray(tail_k, dtype=np.float64)[b, :n, h]], axis=0)
+                V = np.concatenate([V, np.asarray(tail_v, dtype=np.float64)[b, :n, h]], axis=0)
+            if K.shape[0] == 0:
+                continue
+            s = K @ q[b, j] / math.sqrt(d)
+            p = np.exp(s - s.max())
+            out[b, j] = (p / p.sum()) @ V
+    return out

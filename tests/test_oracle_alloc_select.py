@@ -1,4 +1,6 @@
 """Pins for the oracle's budget allocation, top-k selection and compaction."""
+import math
+
 import numpy as np
 import pytest
 
@@ -251,3 +253,58 @@ def test_compress_per_layer_and_protected():
             for h in range(H):
                 got = res["out_k"][l][o:o + len(sets[0]), h]
                 assert got.tobytes() == Ks[l][np.array(sets[0]) + cu[b], h].tobytes()
+
+
+# ---------------------------------------------------------------- decoding step on the compacted cache (Eq. 3-4)
+def _attention_by_loops(qv, K, V):
+    """Softmax(q K^T / sqrt(d)) V with explicit sums, no max subtraction (small scores only)."""
+    d = len(qv)
+    w = [math.exp(sum(qv[c] * K[r][c] for c in range(d)) / math.sqrt(d)) for r in range(len(K))]
+    z = sum(w)
+    return [sum(w[r] * V[r][c] for r in range(len(K))) / z for c in range(d)]
+
+
+def test_decode_attention_matches_explicit_sums():
+    rng = np.random.default_rng(21)
+    B, H, G, d = 2, 2, 3, 4
+    offsets = [0, 5, 12]
+    ck = rng.standard_normal((12, H, d))
+    cv = rng.standard_normal((12, H, d))
+    q = rng.standard_normal((B, H * G, d))
+    tk = rng.standard_normal((B, 3, H, d))
+    tv = rng.standard_normal((B, 3, H, d))
+    out = O.decode_attention(q, ck, cv, offsets, tk, tv, [2, 0])
+    for b in range(B):
+        for j in range(H * G):
+            h = j // G
+            K = list(ck[offsets[b]:offsets[b + 1], h]) + list(tk[b, :[2, 0][b], h])
+            V = list(cv[offsets[b]:offsets[b + 1], h]) + list(tv[b, :[2, 0][b], h])
+            np.testing.assert_allclose(out[b, j], _attention_by_loops(q[b, j], K, V), rtol=1e-12, atol=1e-14)
+
+
+def test_decode_attention_closed_forms():
+    rng = np.random.default_rng(22)
+    H, d = 2, 8
+    ck = rng.standard_normal((6, H, d))
+    cv = rng.standard_normal((6, H, d))
+    # a zero query weighs every row equally: the output is the mean of the value rows
+    out = O.decode_attention(np.zeros((1, 4, d)), ck, cv, [0, 6])
+    np.testing.assert_allclose(out[0, 0], cv[:, 0].mean(axis=0), rtol=1e-13)
+    np.testing.assert_allclose(out[0, 3], cv[:, 1].mean(axis=0), rtol=1e-13)
+    # a single row: the output is that value row whatever the query
+    out = O.decode_attention(rng.standard_normal((1, 2, d)) * 50.0, ck[:1], cv[:1], [0, 1])
+    np.testing.assert_allclose(out[0, 1], cv[0, 1], rtol=1e-13)
+    # a query far along one key picks that key's value; large scores do not overflow
+    q = np.zeros((1, 2, d))
+    q[0, 0] = 400.0 * ck[2, 0] / np.linalg.norm(ck[2, 0]) ** 2 * math.sqrt(d) * 10.0
+    out = O.decode_attention(q, ck, cv, [0, 6])
+    assert np.all(np.isfinite(out))
+    s = ck[:, 0] @ q[0, 0]
+    np.testing.assert_allclose(out[0, 0], cv[int(np.argmax(s)), 0], rtol=1e-9, atol=1e-9)
+    # the order of the rows does not matter; an empty sequence gives zeros
+    perm = rng.permutation(6)
+    qq = rng.standard_normal((2, 4, d))
+    a = O.decode_attention(qq, ck, cv, [0, 6, 6])
+    b = O.decode_attention(qq, ck[perm], cv[perm], [0, 6, 6])
+    np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-14)
+    assert not a[1].any()
