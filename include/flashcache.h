@@ -233,6 +233,42 @@ fc_status fc_power_spectrum(fc_handle *h, const fc_kv_view *kv, double *spectrum
                             void *workspace, size_t workspace_bytes, fc_stream stream);
 
 /*
+ * Decoding step on the compacted cache (Sec. 3.1, Eq. 3-4): for every sequence b and query head j
+ *     out[b][j] = Softmax(q[b][j] K^T / sqrt(head_dim)) V
+ * where K and V are, for KV head j / (num_q_heads / num_heads), the rows the compressor kept for
+ * sequence b (rows offsets[b] .. offsets[b+1] of one layer's compacted cache, as written by
+ * fc_select_compact) followed by the KV pairs appended since the prefill, which stay uncompressed
+ * (the `tail`).  Reads every K and V row once; fp32 accumulation; a sequence without rows gives zeros.
+ *
+ *   q            DEVICE [batch][num_q_heads][head_dim], dtype FC_F16 or FC_BF16 (as the cache)
+ *   cache_k/v    DEVICE [cache_rows][num_heads][head_dim] dense, 16-byte aligned
+ *   offsets      DEVICE int64[batch+1] (one layer's slice of fc_allocate_budgets' out_offsets)
+ *   tail_k/v     DEVICE [batch][tail_capacity][num_heads][head_dim] or NULL
+ *   tail_len     DEVICE int32[batch]: valid rows of each sequence's tail (<= tail_capacity)
+ *   max_rows     HOST upper bound of (kept rows + tail rows) of any sequence; sizes the launch only
+ *   out          DEVICE [batch][num_q_heads][head_dim], same dtype
+ *   workspace    DEVICE, 256-byte aligned, >= fc_decode_workspace_bytes()
+ * Limits: head_dim 128, num_q_heads a multiple of num_heads with at most 16 query heads per KV head.
+ * Errors: FC_ERR_INVALID_ARG, FC_ERR_UNSUPPORTED, FC_ERR_WORKSPACE, FC_ERR_CUDA; a bounded wait that
+ * runs out sets FC_ERR_TIMEOUT in the device status word.
+ */
+typedef struct {
+  const void *q;
+  const void *cache_k, *cache_v;
+  int64_t cache_rows;
+  const int64_t *offsets;
+  const void *tail_k, *tail_v;
+  const int32_t *tail_len;
+  int32_t tail_capacity;
+  int32_t dtype, batch, num_heads, num_q_heads, head_dim;
+  int64_t max_rows;
+} fc_decode_args;
+
+size_t fc_decode_workspace_bytes(const fc_handle *h, const fc_decode_args *a);
+fc_status fc_decode_attention(fc_handle *h, const fc_decode_args *a, void *out,
+                              void *workspace, size_t workspace_bytes, fc_stream stream);
+
+/*
  * fc_select_compact with options (opt == NULL: exactly fc_select_compact).
  *
  *   per_layer  0: every KV head keeps its own tokens (the default reading: Eq. 10 over the head's

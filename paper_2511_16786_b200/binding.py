@@ -27,6 +27,7 @@ EXPORTS = (
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
     "fc_power_spectrum_workspace_bytes", "fc_power_spectrum",
+    "fc_decode_workspace_bytes", "fc_decode_attention",
     "fc_static_scratch_bytes", "fc_score_layer_static",
     "fc_compress_host_rows", "fc_compress_host_arena_bytes", "fc_compress_host",
 )
@@ -43,6 +44,15 @@ class fc_kv_view(ctypes.Structure):
 
 class fc_select_options(ctypes.Structure):
     _fields_ = [("per_layer", c_int32), ("protect", c_void_p)]
+
+
+class fc_decode_args(ctypes.Structure):
+    _fields_ = [
+        ("q", c_void_p), ("cache_k", c_void_p), ("cache_v", c_void_p), ("cache_rows", c_int64),
+        ("offsets", c_void_p), ("tail_k", c_void_p), ("tail_v", c_void_p), ("tail_len", c_void_p),
+        ("tail_capacity", c_int32), ("dtype", c_int32), ("batch", c_int32), ("num_heads", c_int32),
+        ("num_q_heads", c_int32), ("head_dim", c_int32), ("max_rows", c_int64),
+    ]
 
 
 class fc_host_job(ctypes.Structure):
@@ -122,6 +132,10 @@ def _load() -> ctypes.CDLL:
     lib.fc_power_spectrum_workspace_bytes.restype = c_size_t
     lib.fc_power_spectrum.argtypes = [c_void_p, POINTER(fc_kv_view), c_void_p, c_void_p, c_size_t, c_void_p]
     lib.fc_power_spectrum.restype = c_int
+    lib.fc_decode_workspace_bytes.argtypes = [c_void_p, POINTER(fc_decode_args)]
+    lib.fc_decode_workspace_bytes.restype = c_size_t
+    lib.fc_decode_attention.argtypes = [c_void_p, POINTER(fc_decode_args), c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.fc_decode_attention.restype = c_int
     lib.fc_static_scratch_bytes.argtypes = []
     lib.fc_static_scratch_bytes.restype = c_size_t
     lib.fc_score_layer_static.argtypes = [POINTER(fc_kv_view), c_double, c_void_p, c_void_p, c_void_p]
@@ -293,6 +307,35 @@ def fc_power_spectrum(handle, k, v, cu_seqlens, spectrum, workspace) -> None:
     view = make_view(k, v, cu)
     _check(_lib.fc_power_spectrum(handle, byref(view), c_void_p(spectrum.data_ptr()), c_void_p(workspace.data_ptr()),
                                   workspace.numel() * workspace.element_size(), _stream()), "fc_power_spectrum")
+
+
+def make_decode_args(q, cache_k, cache_v, offsets, max_rows: int, tail_k=None, tail_v=None, tail_len=None):
+    """q: [B, Hq, d]; cache_k/v: [rows, H, d]; offsets: int64 [B+1] on the device; tail_k/v: [B, cap, H, d];
+    tail_len: int32 [B] on the device.  max_rows bounds kept + tail rows of any sequence."""
+    B, Hq, d = (int(x) for x in q.shape)
+    rows, H, _ = (int(x) for x in cache_k.shape)
+    for t in (q, cache_k, cache_v):
+        if not t.is_cuda or not t.is_contiguous() or t.dtype != q.dtype:
+            raise ValueError("q and the cache must be contiguous device tensors of one dtype")
+    a = fc_decode_args(q=q.data_ptr(), cache_k=cache_k.data_ptr(), cache_v=cache_v.data_ptr(), cache_rows=rows,
+                       offsets=offsets.data_ptr(), dtype=_DTYPE[q.dtype], batch=B, num_heads=H, num_q_heads=Hq,
+                       head_dim=d, max_rows=int(max_rows))
+    if tail_k is not None:
+        if not (tail_k.is_contiguous() and tail_v.is_contiguous() and tail_k.dtype == q.dtype):
+            raise ValueError("tail_k/tail_v: contiguous [B, cap, H, d] of the cache dtype")
+        a.tail_k, a.tail_v, a.tail_len = tail_k.data_ptr(), tail_v.data_ptr(), tail_len.data_ptr()
+        a.tail_capacity = int(tail_k.shape[1])
+    return a
+
+
+def fc_decode_workspace_bytes(handle, args) -> int:
+    return int(_lib.fc_decode_workspace_bytes(handle, byref(args)))
+
+
+def fc_decode_attention(handle, args, out, workspace) -> None:
+    """out: [B, Hq, d] device tensor of the cache dtype."""
+    _check(_lib.fc_decode_attention(handle, byref(args), c_void_p(out.data_ptr()), c_void_p(workspace.data_ptr()),
+                                    workspace.numel() * workspace.element_size(), _stream()), "fc_decode_attention")
 
 
 def fc_reset_ordering(handle) -> None:
