@@ -203,6 +203,89 @@ def run_reference(args):
     }))
 
 
+# --------------------------------------------------------------------------- decoding step on the compacted cache
+def run_decode(args):
+    """Latency of the attention of one decoding step (fc_decode_attention, every layer) against the
+    context length, on the full cache and on caches compressed to 20 % and 10 %: the quantity behind the
+    paper's decoding-latency figure, for the attention part only.  L2 is flushed before every step, so
+    the K and V rows come from HBM; the roofline is their bytes over the measured HBM bandwidth."""
+    import torch
+    from paper_2511_16786_b200 import binding
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    L, H, G, d, B = 28, 4, 7, 128, 1
+    dtype = torch.bfloat16
+    handle = binding.fc_create(0, 1024)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    g = torch.Generator(device=dev).manual_seed(0)
+    points = []
+    lengths = (args.decode_n,) if args.decode_n else (2048, 4096, 8192, 16384, 32768, 65536)
+    ratios = (args.decode_rho,) if args.decode_rho else (1.0, 0.2, 0.1)
+    for N in lengths:
+        base_ms = None
+        for rho in ratios:
+            rows = max(1, int(rho * N + 0.5))
+            ck = torch.randn((L, rows, H, d), generator=g, device=dev, dtype=torch.float32).to(dtype)
+            cv = torch.randn((L, rows, H, d), generator=g, device=dev, dtype=torch.float32).to(dtype)
+            q = torch.randn((B, H * G, d), generator=g, device=dev, dtype=torch.float32).to(dtype)
+            off = torch.tensor([0, rows], dtype=torch.int64, device=dev)
+            out = torch.empty((L, B, H * G, d), dtype=dtype, device=dev)
+            argl = [binding.make_decode_args(q, ck[l], cv[l], off, rows) for l in range(L)]
+            ws = torch.empty(binding.fc_decode_workspace_bytes(handle, argl[0]), dtype=torch.uint8, device=dev)
+
+            def step():
+                for l in range(L):
+                    binding.fc_decode_attention(handle, argl[l], out[l], ws)
+
+            for _ in range(3):
+                step()
+            torch.cuda.synchronize()
+            binding._check(binding.fc_last_device_status(handle), "device status")
+            n_rep = 20
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_rep)]
+            for e0, e1 in ev:
+                flush.zero_()
+                e0.record()
+                step()
+                e1.record()
+            torch.cuda.synchronize()
+            ms = sorted(e0.elapsed_time(e1) for e0, e1 in ev)[n_rep // 2]
+            # the same step replayed from a CUDA graph, as a serving loop would issue it
+            graph = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream(device=dev)
+            side.wait_stream(torch.cuda.current_stream(dev))
+            with torch.cuda.graph(graph, stream=side):
+                step()
+            for e0, e1 in ev:
+                flush.zero_()
+                e0.record()
+                graph.replay()
+                e1.record()
+            torch.cuda.synchronize()
+            ms_graph = sorted(e0.elapsed_time(e1) for e0, e1 in ev)[n_rep // 2]
+            del graph
+            nbytes = 2.0 * L * rows * H * d * 2
+            gbs = nbytes / (ms_graph * 1e-3) / 1e9
+            if base_ms is None:
+                base_ms = ms_graph
+            points.append({"N": N, "rho": rho, "rows_per_layer": rows, "ms_per_step_eager": ms, "ms_per_step": ms_graph,
+                           "gbytes": nbytes / 1e9,
+                           "achieved_gbs": gbs, "frac_of_hbm": gbs / peaks["hbm_gbs"],
+                           "speedup_vs_first_ratio": base_ms / ms_graph})
+            del ck, cv
+    binding.fc_destroy(handle)
+    print(json.dumps({
+        "metric": "decode_attention_ms_per_token", "unit": "ms", "higher_is_better": False, "n_gpus": 1,
+        "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+        "config": {"workload": "attention of one decoding step over the compacted caches of 28 layers, "
+                               "4 KV heads x 7 query heads, head_dim 128, batch 1",
+                   "l2_policy": "256 MB written before every step (flush)", "median_of": 20},
+        "roofline": {"bound": "hbm", "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "peak_source": "MEASURED_PEAKS.json hbm_gbs (%s)" % peaks["source"]},
+        "points": points}))
+
+
 # --------------------------------------------------------------------------- main arm
 def main():
     ap = argparse.ArgumentParser()
@@ -219,9 +302,16 @@ def main():
     ap.add_argument("--per-layer", action="store_true",
                     help="one index set per layer from the head-averaged score (fc_select_compact_ex)")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
+    ap.add_argument("--decode", action="store_true",
+                    help="time the decoding-step attention on full and compressed caches instead of the compressor")
+    ap.add_argument("--decode-n", type=int, default=0, help="--decode: only this context length")
+    ap.add_argument("--decode-rho", type=float, default=0.0, help="--decode: only this cache ratio")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.decode:
+        run_decode(args)
         return
 
     import torch

@@ -3,7 +3,7 @@
 // that read, so the design is about keeping HBM busy:
 //
 //  * grid (splits, KV heads, sequences); a block walks its share of the rows in tiles of 64, filled by
-//    tiled TMA loads (128-byte swizzle) into a two-stage shared-memory ring behind mbarriers;
+//    tiled TMA loads (128-byte swizzle) into a four-stage shared-memory ring behind mbarriers;
 //  * all query heads of a KV head (up to 16) are one 16-row operand of m16n8k16 tensor-core products,
 //    so a K/V tile is read from shared memory once for the whole group; each of the 4 warps owns 16
 //    rows of the tile and keeps its own running maximum, sum and 16 x 128 fp32 output;
@@ -20,7 +20,11 @@ constexpr int kWarps = 4;
 constexpr int kThreadsD = 32 * kWarps;
 constexpr int kBoxBytes = kTile * 128;  // one TMA box: 64 rows x 64 elements of 2 bytes
 constexpr int kStageBytes = 4 * kBoxBytes;   // K low/high halves, V low/high halves
-constexpr unsigned kSpinLimit = 1u << 22;    // polls of ~32 ns: gives up after about a tenth of a second
+// tiles in the shared-memory ring: 4 (one resident block per SM, three tiles in flight) measured best;
+// 2 and 3 (three and two blocks per SM) and 5..7 were slower (1.05, 0.98, 0.84..0.91 against 0.82 ms for
+// 28 layers of 65536 rows)
+constexpr int kStages = 4;
+constexpr unsigned kSpinLimit = 1u << 20;    // blocking tests of an mbarrier before a wait gives up
 
 struct DecodeParams {
   const void *q;
@@ -44,18 +48,17 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned
   asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}\n"
                ::"r"((unsigned)__cvta_generic_to_shared(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_test(unsigned long long *bar, unsigned parity) {
+// One potentially blocking test: the thread sleeps until the phase completes or a hardware time limit passes.
+__device__ __forceinline__ bool mbar_try(unsigned long long *bar, unsigned parity) {
   unsigned ok;
-  asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
                : "=r"(ok) : "r"((unsigned)__cvta_generic_to_shared(bar)), "r"(parity) : "memory");
   return ok != 0u;
 }
 // Bounded wait; false = gave up.
 __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity) {
-  for (unsigned it = 0; it < kSpinLimit; ++it) {
-    if (mbar_test(bar, parity)) return true;
-    __nanosleep(32);
-  }
+  for (unsigned it = 0; it < kSpinLimit; ++it)
+    if (mbar_try(bar, parity)) return true;
   return false;
 }
 // Tiled loads into this block's shared memory; completion is counted in bytes on `bar`.  No multicast.
@@ -124,7 +127,7 @@ __global__ void __launch_bounds__(kThreadsD)
 k_decode_partial(const DecodeParams P, const __grid_constant__ DecodeMaps M) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  unsigned long long *full = reinterpret_cast<unsigned long long *>(smem + 2 * kStageBytes);
+  unsigned long long *full = reinterpret_cast<unsigned long long *>(smem + kStages * kStageBytes);
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -141,8 +144,7 @@ k_decode_partial(const DecodeParams P, const __grid_constant__ DecodeMaps M) {
   const int ntiles = lo < hi ? (hi - lo + kTile - 1) / kTile : 0;
 
   if (tid == 0) {
-    mbar_init(&full[0], 1u);
-    mbar_init(&full[1], 1u);
+    for (int i = 0; i < kStages; ++i) mbar_init(&full[i], 1u);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   __syncthreads();
@@ -189,11 +191,16 @@ k_decode_partial(const DecodeParams P, const __grid_constant__ DecodeMaps M) {
   bool failed = false;
   int issued = 0;
 
-  if (tid == 0 && ntiles > 0) { issue(0, 0); issued = 1; }
+  if (tid == 0)
+    for (int ti = 0; ti < kStages - 1 && ti < ntiles; ++ti) { issue(ti, ti); issued = ti + 1; }
+
   for (int ti = 0; ti < ntiles; ++ti) {
-    const int s = ti & 1;
-    if (tid == 0 && ti + 1 < ntiles) { issue(ti + 1, s ^ 1); issued = ti + 2; }   // that stage was released by the barrier below
-    const bool got = mbar_wait(&full[s], (unsigned)(ti >> 1) & 1u);
+    const int s = ti % kStages;
+    if (tid == 0 && ti + kStages - 1 < ntiles) {          // into the stage that the barrier below released last time round
+      issue(ti + kStages - 1, (ti + kStages - 1) % kStages);
+      issued = ti + kStages;
+    }
+    const bool got = mbar_wait(&full[s], (unsigned)(ti / kStages) & 1u);
     if (__syncthreads_or(got ? 0 : 1)) { failed = true; break; }
     const int row0 = lo + ti * kTile;
     int valid = (row0 < n_main_pad ? n_main : total) - row0;
@@ -266,7 +273,7 @@ k_decode_partial(const DecodeParams P, const __grid_constant__ DecodeMaps M) {
     // (they write this block's shared memory), and report an empty share
     if (tid == 0) {
       atomicOr(P.status, FC_DEV_FLAG_TIMEOUT);
-      for (int ti = 0; ti < issued; ++ti) mbar_wait(&full[ti & 1], (unsigned)(ti >> 1) & 1u);
+      for (int ti = 0; ti < issued; ++ti) mbar_wait(&full[ti % kStages], (unsigned)(ti / kStages) & 1u);
     }
     m[0] = m[1] = -INFINITY;
     l[0] = l[1] = 0.f;
@@ -368,6 +375,23 @@ fc_status encode_rows(CUtensorMap *m, CUtensorMapDataType dt, int rank, const vo
   return r == CUDA_SUCCESS ? FC_OK : FC_ERR_INTERNAL;
 }
 
+constexpr size_t kDecodeSmem = (size_t)kStages * kStageBytes + 64 + 1024;   // ring, barriers, slack to align the ring to 1024 bytes
+
+// Resident blocks of k_decode_partial per SM (the launch is sized to one full wave of them).
+int decode_blocks_per_sm() {
+  static int n = 0;
+  if (n == 0) {
+    int v = 0;
+    if (cudaFuncSetAttribute(k_decode_partial<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecodeSmem) == cudaSuccess &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, k_decode_partial<__half>, kThreadsD, kDecodeSmem) == cudaSuccess && v > 0)
+      n = v;
+    else
+      n = 1;
+    cudaGetLastError();
+  }
+  return n;
+}
+
 struct DecodePlan {
   int nsplit, chunk;
   size_t off_ml, total;
@@ -397,7 +421,7 @@ DecodePlan plan_decode(const fc_handle *h, const fc_decode_args *a) {
   long long tiles = (logical + kTile - 1) / kTile;
   if (tiles < 1) tiles = 1;
   const long long groups = (long long)a->batch * a->num_heads;
-  long long want = (4ll * h->num_sms + groups - 1) / groups;                // about four blocks per SM in flight
+  long long want = (long long)decode_blocks_per_sm() * h->num_sms / groups;           // one full wave of resident blocks
   if (want < 1) want = 1;
   if (want > tiles) want = tiles;
   const long long per = (tiles + want - 1) / want;
@@ -446,7 +470,7 @@ fc_status launch_decode(fc_handle *h, const fc_decode_args *a, const DecodePlan 
   P.tail_cap = a->tail_k ? a->tail_capacity : 0;
   P.has_tail = a->tail_k ? 1 : 0;
   P.scale_log2 = (float)(1.4426950408889634 / sqrt((double)kD));
-  const size_t sm = 2 * (size_t)kStageBytes + 64 + 1024;
+  const size_t sm = kDecodeSmem;
   FC_CUDA_TRY(cudaFuncSetAttribute(k_decode_partial<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
   k_decode_partial<T><<<dim3(pl.nsplit, a->num_heads, a->batch), kThreadsD, sm, st>>>(P, M);
   if ((s = fc_after_launch(h)) != FC_OK) return s;
