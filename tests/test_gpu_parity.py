@@ -538,6 +538,53 @@ def test_overlapping_launches_give_the_same_results(fc):
 
 
 # ---------------------------------------------------------------- full-size shapes, sampled
+def test_head_sharded_pass_equals_the_whole_pass(fc):
+    # two shards of the KV heads, run one after the other on this GPU, with the energy sums added by hand
+    # where the ranks would all-reduce them: budgets, indices and rows equal those of the unsharded pass
+    from paper_2511_16786_b200.binding import Compressor
+    from paper_2511_16786_b200.head_shard import HeadShardedCompressor, shard_heads
+    base = S.paper_configs()["cfg2"]
+    cfg = S.scaled(base, "shard_small", num_layers=4, seqlens=(2048, 500))
+    L, H = cfg.num_layers, cfg.num_heads
+    Kd = [S.make_layer(cfg, l, "cuda")[0] for l in range(L)]
+    Vd = [S.make_layer(cfg, l, "cuda")[1] for l in range(L)]
+    whole = Compressor(L, H, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho, cfg.gamma, cfg.min_keep)
+    whole.compress(Kd, Vd)
+    whole.check_device_status()
+    shards = []
+    for rank in range(2):
+        h0, h1 = shard_heads(H, 2, rank)
+        sc = HeadShardedCompressor(None, rank, 2, L, H, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho,
+                                   cfg.gamma, cfg.min_keep)
+        Kl = [k[:, h0:h1] for k in Kd]
+        Vl = [v[:, h0:h1] for v in Vd]
+        sc.local.score(Kl, Vl)
+        shards.append((sc, Kl, Vl, h0, h1))
+    torch.cuda.synchronize()
+    total = shards[0][0].local.energy + shards[1][0].local.energy
+    np.testing.assert_allclose(total.cpu().numpy(), whole.energy.cpu().numpy(), rtol=1e-12)
+    for sc, Kl, Vl, h0, h1 in shards:
+        sc.local.energy.copy_(total)
+        sc.local.allocate()
+        sc.local.select_compact(Kl, Vl)
+        sc.local.check_device_status()
+        assert torch.equal(sc.local.budgets, whole.budgets)
+        off = whole.offsets.cpu()
+        for l in range(L):
+            r = int(off[l, -1])
+            assert torch.equal(sc.local.out_idx[l, :, :r], whole.out_idx[l, h0:h1, :r])
+            assert torch.equal(sc.local.out_k[l, :r].view(torch.uint8), whole.out_k[l, :r, h0:h1].contiguous().view(torch.uint8))
+        sc.close()
+    # one rank, no group: the wrapper is the plain pass
+    one = HeadShardedCompressor(None, 0, 1, L, H, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho, cfg.gamma,
+                                cfg.min_keep)
+    one.compress(Kd, Vd)
+    one.local.check_device_status()
+    assert torch.equal(one.local.budgets, whole.budgets) and torch.equal(one.local.offsets, whole.offsets)
+    one.close()
+    whole.close()
+
+
 def test_graph_replay_gives_the_same_results(fc):
     # the whole call sequence captured once into a CUDA graph; replays on new contents of the same
     # tensors must equal an eager pass on those contents, and eager calls must still work afterwards
