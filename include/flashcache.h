@@ -352,6 +352,8 @@ fc_status fc_score_layer_static(const fc_kv_view *kv, double gamma, float *score
  *                    T = cu_seqlens[batch].
  *   cu_seqlens       int32[batch+1], as in fc_kv_view.
  *   gamma, rho, min_keep   as in fc_score_layer and fc_allocate_budgets.
+ *   per_layer, protect_host   the options of fc_select_compact_ex; protect_host is a HOST uint8[T]
+ *                    mask (or NULL) that the call copies to the device with the inputs.
  * Device memory (DEVICE, owned by the caller, 256-byte aligned, >= fc_compress_host_arena_bytes):
  *   arena            staging for the inputs of all layers, scores, energies, budgets, the
  *                    compacted caches and the kernels' workspace.  Two consecutive calls with
@@ -391,6 +393,8 @@ typedef struct {
   int32_t *budgets_host;
   int64_t *offsets_host;
   int64_t *layer_rows_host;
+  int32_t per_layer;
+  const uint8_t *protect_host;
 } fc_host_job;
 
 /* Rows the compacted caches of all layers hold together: the sum over sequences of

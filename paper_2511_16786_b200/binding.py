@@ -66,6 +66,7 @@ class fc_host_job(ctypes.Structure):
         ("out_k_host", c_void_p), ("out_v_host", c_void_p), ("out_idx_host", c_void_p),
         ("out_capacity_rows", c_int64),
         ("budgets_host", c_void_p), ("offsets_host", c_void_p), ("layer_rows_host", c_void_p),
+        ("per_layer", c_int32), ("protect_host", c_void_p),
     ]
 
 
@@ -570,8 +571,10 @@ class HostCompressor:
     the copies in of the next."""
 
     def __init__(self, num_layers: int, num_heads: int, head_dim: int, cu_seqlens, dtype, rho: float,
-                 gamma: float = 0.2, min_keep: int = 1, device: int = 0):
+                 gamma: float = 0.2, min_keep: int = 1, device: int = 0, per_layer: bool = False, protect=None):
         self.L, self.H, self.d = int(num_layers), int(num_heads), int(head_dim)
+        # selection options: one index set per layer; protect = uint8 [T] HOST tensor of tokens that must survive
+        self.per_layer, self.protect = bool(per_layer), protect
         self.cu = [int(x) for x in cu_seqlens]
         self.B = len(self.cu) - 1
         self.T = self.cu[-1]
@@ -588,7 +591,11 @@ class HostCompressor:
             k_host=ctypes.cast(self._kptr, POINTER(c_void_p)), v_host=ctypes.cast(self._vptr, POINTER(c_void_p)),
             num_layers=self.L, dtype=_DTYPE[dtype], num_heads=self.H, head_dim=self.d, batch=self.B,
             min_keep=self.min_keep, cu_seqlens=ctypes.cast(self._cu, POINTER(c_int32)),
-            gamma=self.gamma, rho=self.rho)
+            gamma=self.gamma, rho=self.rho, per_layer=1 if per_layer else 0,
+            protect_host=protect.data_ptr() if protect is not None else None)
+        if protect is not None and (protect.is_cuda or protect.dtype != torch.uint8 or protect.numel() != self.T
+                                    or not protect.is_contiguous()):
+            raise ValueError("protect: contiguous uint8 host tensor with one entry per token")
         need = int(_lib.fc_compress_host_arena_bytes(self.handle, byref(self._job)))
         if need == 0:
             raise FlashCacheError(2, "fc_compress_host_arena_bytes")

@@ -20,7 +20,7 @@ inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 struct Arena {
   size_t off_k, off_v, layer_in_bytes;
   size_t off_scores, off_energy, off_budgets, off_offsets;
-  size_t off_out_k, off_out_v, off_out_idx, off_ws;
+  size_t off_out_k, off_out_v, off_out_idx, off_ws, off_protect;
   size_t ws_bytes, total;
   long long T, rows;
   size_t row_bytes;
@@ -77,6 +77,7 @@ Arena carve(const fc_handle *h, const fc_host_job *j) {
   a.off_out_v = off;   off += up256((size_t)R1 * a.row_bytes);
   a.off_out_idx = off; off += up256((size_t)R1 * H * sizeof(int32_t));
   a.off_ws = off;      off += a.ws_bytes > 0 ? a.ws_bytes : 256;
+  a.off_protect = off; off += up256((size_t)T1);
   a.total = off;
   return a;
 }
@@ -181,6 +182,13 @@ extern "C" fc_status fc_compress_host(fc_handle *h, const fc_host_job *job, fc_s
   }
   h->host_last_arena = nullptr;                 // set again only when this job got as far as its selection
 
+  unsigned char *protect = nullptr;
+  if (job->protect_host) {
+    protect = reinterpret_cast<unsigned char *>(base + a.off_protect);
+    FC_CUDA_TRY(cudaMemcpyAsync(protect, job->protect_host, (size_t)a.T, cudaMemcpyHostToDevice, h->host_copy));
+  }
+  const fc_select_options opt = {job->per_layer, protect};
+
   OverlapScope restore(h);
   h->score_overlap = 1;                         // score x L, then allocate joins the internal streams
   h->select_overlap = 1;                        // select x L back to back, all inputs ready before the first
@@ -219,9 +227,9 @@ extern "C" fc_status fc_compress_host(fc_handle *h, const fc_host_job *job, fc_s
     if (r == 0) continue;
     const fc_kv_view kv = view_of(job, base + a.off_k + (size_t)l * a.layer_in_bytes,
                                   base + a.off_v + (size_t)l * a.layer_in_bytes);
-    s = fc_select_compact(h, &kv, scores + (size_t)l * H * a.T, budgets + (size_t)l * B,
-                          offsets + (size_t)l * (B + 1), ok + (size_t)r0 * a.row_bytes, ov + (size_t)r0 * a.row_bytes,
-                          oi + (size_t)r0 * H, r, ws, a.ws_bytes, st);
+    s = fc_select_compact_ex(h, &kv, scores + (size_t)l * H * a.T, budgets + (size_t)l * B,
+                             offsets + (size_t)l * (B + 1), ok + (size_t)r0 * a.row_bytes, ov + (size_t)r0 * a.row_bytes,
+                             oi + (size_t)r0 * H, r, &opt, ws, a.ws_bytes, st);
     if (s != FC_OK) return s;
   }
   FC_CUDA_TRY(cudaEventRecord(h->ev_inputs_free, st));

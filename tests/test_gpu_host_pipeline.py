@@ -31,9 +31,10 @@ def _layers(cfg, pin=True):
     return Ks, Vs
 
 
-def _per_stage(fc, cfg, Ks, Vs):
+def _per_stage(fc, cfg, Ks, Vs, per_layer=False, protect=None):
     comp = fc.Compressor(cfg.num_layers, cfg.num_heads, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho,
-                         cfg.gamma, cfg.min_keep)
+                         cfg.gamma, cfg.min_keep, per_layer=per_layer,
+                         protect=None if protect is None else protect.cuda())
     Kd, Vd = [k.cuda() for k in Ks], [v.cuda() for v in Vs]
     comp.compress(Kd, Vd)
     comp.check_device_status()
@@ -139,4 +140,29 @@ def test_pageable_inputs_and_bad_arguments(fc):
     with pytest.raises(fc.FlashCacheError) as e:
         hc.compress(Ks, Vs, res)
     assert e.value.code == 3
+    hc.close()
+
+
+def test_host_pipeline_with_selection_options(fc):
+    base = S.paper_configs()["cfg2"]
+    cfg = S.scaled(base, "host_options", num_layers=3, seqlens=(1024, 600), min_keep=24)
+    Ks, Vs = _layers(cfg)
+    cu = cfg.cu_seqlens
+    protect = torch.zeros(cu[-1], dtype=torch.uint8)
+    for b in range(2):
+        protect[cu[b]:cu[b] + 4] = 1
+        protect[cu[b + 1] - 16:cu[b + 1]] = 1
+    protect = protect.pin_memory()
+    ref = _per_stage(fc, cfg, Ks, Vs, per_layer=True, protect=protect)
+    hc = fc.HostCompressor(cfg.num_layers, cfg.num_heads, cfg.head_dim, cu, cfg.torch_dtype, cfg.rho, cfg.gamma,
+                           cfg.min_keep, per_layer=True, protect=protect)
+    res = hc.new_result()
+    hc.compress(Ks, Vs, res)
+    torch.cuda.synchronize()
+    hc.check_device_status()
+    _check_against_per_stage(cfg, res, ref)
+    k, v, idx = res.layer(0)
+    assert torch.equal(idx[0], idx[1])                                   # one index set per layer
+    got = set(idx[0, :int(res.budgets[0, 0])].tolist())
+    assert set(range(4)) <= got and set(range(1024 - 16, 1024)) <= got   # the marked tokens of sequence 0 survive
     hc.close()
