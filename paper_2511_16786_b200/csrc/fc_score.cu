@@ -243,8 +243,8 @@ k_pass2(FftPlan plan, int N1, int ncol_ws, int cs2_log2, float2 *__restrict__ ws
   const int ncolT = 1 << ncolT_log2;
   const int gc0 = blockIdx.y * cs2;
 
-  float2 *S = smem;                                    // [N2][2*cs2] at most
-  float2 *tw = S + (size_t)N2 * 2 * cs2;               // [N2]
+  float2 *S = smem;                                    // [N2][2*cs2] for the paired rows of MID_DCT, else [N2][cs2]
+  float2 *tw = S + (size_t)N2 * (MID == MID_DCT ? 2 : 1) * cs2;   // [N2]
   float2 *twN = tw + N2;                               // [2][N2]
   unsigned short *rev = reinterpret_cast<unsigned short *>(twN + 2 * N2);   // [N2]
   unsigned short *pos_of = rev + N2;                                       // [N2]
@@ -801,8 +801,8 @@ fc_status set_smem(Kern kern, size_t bytes) {
 size_t smem_pass13(const SeqPlan &sp, int cs) {
   return (size_t)sp.N1 * cs * sizeof(float2) + sp.N1 * sizeof(float2) + sp.N1 * sizeof(int) + 2 * sp.N1 * sizeof(float);
 }
-size_t smem_pass2(const SeqPlan &sp, int cs2) {
-  return (size_t)sp.N2 * 2 * cs2 * sizeof(float2) + 3 * (size_t)sp.N2 * sizeof(float2) + 2 * (size_t)sp.N2 * sizeof(unsigned short);
+size_t smem_pass2(const SeqPlan &sp, int cs2, int halves = 2) {
+  return (size_t)sp.N2 * halves * cs2 * sizeof(float2) + 3 * (size_t)sp.N2 * sizeof(float2) + 2 * (size_t)sp.N2 * sizeof(unsigned short);
 }
 
 template <class Loader>
@@ -822,7 +822,7 @@ template <int MID>
 fc_status launch_pass2(fc_handle *h, cudaStream_t st, const SeqPlan &sp, int ncol_ws, int cs2, float2 *ws,
                        int omega, float2 *hhat, float scale) {
   const FftPlan p2 = make_plan(sp.N2);
-  const size_t sm = smem_pass2(sp, cs2);
+  const size_t sm = smem_pass2(sp, cs2, MID == MID_DCT ? 2 : 1);
   fc_status s = set_smem(k_pass2<MID>, sm);
   if (s != FC_OK) return s;
   dim3 grid(MID == MID_DCT ? sp.N1 / 2 + 1 : sp.N1, ncol_ws / cs2);
@@ -1138,7 +1138,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       const int sub = L.sub_cols, cs = (sub % 64 == 0) ? sp.cs : 32;
       const int ngroups = (hg == 1) ? d / sub : 1;
       const int ncol = (hg == 1) ? sub : ncol_ws;
-      int cs2 = sp.cs2;
+      int cs2 = 2 * sp.cs2 > 64 ? 64 : 2 * sp.cs2;       // the convolution pass holds single rows: twice the columns fit
       while (ncol % cs2) cs2 >>= 1;
       const size_t sm3c = smem_pass13(sp, cs);
       for (int cg = 0; cg < ngroups; ++cg) {
@@ -1244,7 +1244,7 @@ fc_status power_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     const int sub = L.sub_cols, cs = (sub % 64 == 0) ? sp.cs : 32;
     const int ngroups = (hg == 1) ? d / sub : 1;
     const int ncol = (hg == 1) ? sub : ncol_ws;
-    int cs2 = sp.cs2;
+    int cs2 = 2 * sp.cs2 > 64 ? 64 : 2 * sp.cs2;
     while (ncol % cs2) cs2 >>= 1;
     const size_t sm3c = smem_pass13(sp, cs);
     for (int cg = 0; cg < ngroups; ++cg) {
