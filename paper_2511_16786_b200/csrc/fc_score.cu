@@ -898,6 +898,89 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
   return FC_ERR_INTERNAL;
 }
 
+// The chirp path on the specialised kernels, for transform lengths M = N1*N2 of 1024..65536 (sequence
+// lengths that are not a power of two, up to 32768): two circular convolutions with the chirp kernel, each
+// pass 1 -> pass 2 (multiply by the kernel's spectrum) -> pass 3, on the caller's stream.  Tile widths fixed.
+template <typename T, int R1B, int R2B>
+fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq,
+                            int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
+                            double *phi, float *scores, long long total_tokens) {
+  constexpr int CPW = 32, CP = 8, N1 = 16 * R1B, N2 = 16 * R2B;
+  const int d = kv->head_dim, ncol = hg * d;
+  const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
+  const size_t sm2 = (size_t)2 * N2 * CP * sizeof(float4) + 5 * N2 * sizeof(float2);
+  const float invM = 1.f / (float)(N1 * N2);
+  const dim3 g1(N2, ncol / (2 * CPW)), g2(N1 / 2, ncol / (2 * CP)), g3(N2, hg);
+  fc_status s;
+  if ((s = set_smem(fast::k_p1<T, R1B, CPW, fast::LD_CHIRP>, sm1)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_FILTER>, sm1)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p2<R2B, CP, fast::MID_CONV>, sm2)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SPEC>, sm1)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP>, sm1)) != FC_OK) return s;
+  {
+    ProfScope ps(h, FC_K_PASS1, st);
+    fast::k_p1<T, R1B, CPW, fast::LD_CHIRP><<<g1, CPW * R1B, sm1, st>>>(
+        kp, vp, kv->stride_token, kv->stride_head, h0, d, Nseq, N2, ncol, ws, h->master, h->master_len, ptot);
+  }
+  if ((s = fc_after_launch(h)) != FC_OK) return s;
+  {
+    ProfScope ps(h, FC_K_PASS2, st);
+    fast::k_p2<R2B, CP, fast::MID_CONV><<<g2, 2 * CP * R2B, sm2, st>>>(N1, ncol, ws, h->master, h->master_len, 0, hhat, invM);
+  }
+  if ((s = fc_after_launch(h)) != FC_OK) return s;
+  {
+    ProfScope ps(h, FC_K_PASS3, st);
+    fast::k_p3<R1B, CPW, fast::OUT_SPEC><<<g3, CPW * R1B, sm1, st>>>(
+        Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, h0, d, 0, 0.f, nullptr, nullptr, 0u, nullptr, 0, nullptr, 0,
+        nullptr, spec);
+  }
+  if ((s = fc_after_launch(h)) != FC_OK) return s;
+  {
+    ProfScope ps(h, FC_K_PASS1, st);
+    fast::k_p1<float, R1B, CPW, fast::LD_FILTER><<<g1, CPW * R1B, sm1, st>>>(
+        nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, omega);
+  }
+  if ((s = fc_after_launch(h)) != FC_OK) return s;
+  {
+    ProfScope ps(h, FC_K_PASS2, st);
+    fast::k_p2<R2B, CP, fast::MID_CONV><<<g2, 2 * CP * R2B, sm2, st>>>(N1, ncol, ws, h->master, h->master_len, 0, hhat, invM);
+  }
+  if ((s = fc_after_launch(h)) != FC_OK) return s;
+  {
+    ProfScope ps(h, FC_K_PASS3, st);
+    const float inv = (float)(1.0 / ((double)Nseq * (double)Nseq * (double)d));
+    fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP><<<g3, CPW * R1B, sm1, st>>>(
+        Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, d, total_tokens, inv, phi, nullptr, 0u, nullptr, 0,
+        nullptr, 0, nullptr, nullptr);
+  }
+  return fc_after_launch(h);
+}
+
+// Factors of the specialised kernels for a transform length (0, 0 when it has none).
+inline void fast_factors(int M, int *r1b, int *r2b) {
+  *r1b = *r2b = 0;
+  if (!is_pow2(M) || M < 1024 || M > 65536) return;
+  const int bits = ilog2(M), b1 = bits / 2;
+  *r1b = (1 << b1) / 16;
+  *r2b = (M >> b1) / 16;
+}
+
+template <typename T>
+fc_status launch_chirp(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq, int M,
+                       int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
+                       double *phi, float *scores, long long total_tokens) {
+  int a, b;
+  fast_factors(M, &a, &b);
+#define FC_CHIRP_CASE(A, B)                                                                                  \
+  if (a == A && b == B)                                                                                      \
+    return launch_chirp_impl<T, A, B>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, scores, \
+                                      total_tokens);
+  FC_CHIRP_CASE(2, 2) FC_CHIRP_CASE(2, 4) FC_CHIRP_CASE(4, 4) FC_CHIRP_CASE(4, 8)
+  FC_CHIRP_CASE(8, 8) FC_CHIRP_CASE(8, 16) FC_CHIRP_CASE(16, 16)
+#undef FC_CHIRP_CASE
+  return FC_ERR_INTERNAL;
+}
+
 // cuTensorMapEncodeTiled, looked up through the runtime (no link against the driver library).
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -1133,6 +1216,15 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       // One head may be transformed in several column groups (sub < d) so that the padded
       // length-Nfft intermediates of a group stay within the cache budget; the groups run in
       // stream order and the last pass adds their contributions to the score in that order.
+      int fa, fb;
+      fast_factors(sp.Nfft, &fa, &fb);
+      if (fa != 0 && !h->generic_only && L.sub_cols == d) {      // whole heads, a length the specialised kernels take
+        if ((s = launch_chirp<T>(h, st, kv, kp, vp, N, sp.Nfft, h0, hg, omega, ws, spec, hhat, ptot, phi,
+                                 scores + start, total_tokens)) != FC_OK) return s;
+        tot_slots += (size_t)(16 * fb) * (ncol_ws / 64);
+        hi_slots += (size_t)(16 * fb) * hg;
+        continue;
+      }
       const float invM = 1.f / (float)sp.Nfft;
       const float inv = (float)(1.0 / ((double)N * (double)N * (double)d));
       const int sub = L.sub_cols, cs = (sub % 64 == 0) ? sp.cs : 32;

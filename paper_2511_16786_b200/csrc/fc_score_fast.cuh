@@ -41,6 +41,29 @@ template <> struct Load2<__nv_bfloat16> {
   }
 };
 
+// exp(+j*pi*n*n/N), the chirp of the convolution form of an N-point DFT; n*n is reduced modulo 2N
+// (one period) in integers first.
+__device__ __forceinline__ float2 chirp_f(int n, int N) {
+  const unsigned long long r = ((unsigned long long)n * (unsigned long long)n) % (2ull * (unsigned long long)N);
+  float s, c;
+  sincospif(__fdiv_rn((float)(unsigned)r, (float)N), &s, &c);
+  return make_float2(c, s);
+}
+
+// What pass 1 transforms.
+//   LD_KV     : the K/V rows of a power-of-two sequence (N = N1*N2 points).
+//   LD_CHIRP  : chirp convolution, first half: the N < N1*N2 rows times conj(chirp), zeros behind them.
+//   LD_FILTER : chirp convolution, second half: the N-point spectrum spec[q][col] through the low-pass
+//               residual filter, conjugated (an inverse DFT is the conjugate of the forward DFT of the
+//               conjugate) and times conj(chirp), zeros behind.
+enum { LD_KV = 0, LD_CHIRP = 1, LD_FILTER = 2 };
+// What pass 2 does between its forward and inverse halves: the DCT/low-pass residual filter on paired rows,
+// or a multiplication by the spectrum of the chirp kernel (rows 2x and 2x+1, unrelated).
+enum { MID_FILTER = 0, MID_CONV = 1 };
+// What pass 3 does with the rows it gets back: scores of a power-of-two sequence, the N-point spectrum of
+// the chirp path (rows < N times conj(chirp)), or the scores at the end of the chirp path.
+enum { OUT_SCORE = 0, OUT_SPEC = 1, OUT_SCORE_CHIRP = 2 };
+
 template <int R>
 __device__ __forceinline__ void dft_fwd(float2 (&x)[R]) { dft_small<R, -1>(x); }
 template <int R>
@@ -51,11 +74,12 @@ __device__ __forceinline__ void dft_inv(float2 (&x)[R]) { dft_small<R, +1>(x); }
 // Thread (cp = tid % CPW, j = tid / CPW): channels 2cp, 2cp+1 of the slice; first
 // stage points n1 = j + R1B*p, p = 0..15, loaded from the K/V rows.
 // ---------------------------------------------------------------------------
-template <typename T, int R1B, int CPW>
+template <typename T, int R1B, int CPW, int LD = LD_KV>
 __global__ void __launch_bounds__(CPW * R1B)
 k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, long long stride_head,
      int head0, int head_dim, int N, int N2, int ncol_ws, float2 *__restrict__ ws,
-     const float2 *__restrict__ master, int master_len, double *__restrict__ partial) {
+     const float2 *__restrict__ master, int master_len, double *__restrict__ partial,
+     const float2 *__restrict__ spec = nullptr, int omega = 0) {
   constexpr int N1 = 16 * R1B, NT = CPW * R1B, IT = 16 / R1B, NW = (NT + 31) / 32;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                        // [N1][CPW]
@@ -71,18 +95,52 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
   float accK = 0.f, accV = 0.f;
 #pragma unroll
   for (int p = 0; p < 16; ++p) {
-    const int tok = perm_token((j + R1B * p) * N2 + n2, N);
-    const long long off = (long long)tok * stride_token;
-    const float2 kk = Load2<T>::ld(kb + off), vv = Load2<T>::ld(vb + off);
-    x0[p] = make_float2(kk.x, vv.x);
-    x1[p] = make_float2(kk.y, vv.y);
+    const int n = (j + R1B * p) * N2 + n2;
+    if (LD == LD_KV) {
+      const long long off = (long long)perm_token(n, N) * stride_token;
+      const float2 kk = Load2<T>::ld(kb + off), vv = Load2<T>::ld(vb + off);
+      x0[p] = make_float2(kk.x, vv.x);
+      x1[p] = make_float2(kk.y, vv.y);
+    } else if (LD == LD_CHIRP) {
+      x0[p] = x1[p] = make_float2(0.f, 0.f);
+      if (n < N) {
+        const long long off = (long long)perm_token(n, N) * stride_token;
+        const float2 kk = Load2<T>::ld(kb + off), vv = Load2<T>::ld(vb + off);
+        accK = fmaf(kk.x, kk.x, fmaf(kk.y, kk.y, accK));
+        accV = fmaf(vv.x, vv.x, fmaf(vv.y, vv.y, accV));
+        const float2 ch = chirp_f(n, N);
+        x0[p] = cmul_conj(make_float2(kk.x, vv.x), ch);
+        x1[p] = cmul_conj(make_float2(kk.y, vv.y), ch);
+      }
+    } else {
+      x0[p] = x1[p] = make_float2(0.f, 0.f);
+      if (n < N) {
+        const int q = n, qp = (N - q) % N;
+        const float4 P4 = *reinterpret_cast<const float4 *>(spec + (size_t)q * ncol_ws + gc0 + 2 * cp);
+        const float4 Q4 = *reinterpret_cast<const float4 *>(spec + (size_t)qp * ncol_ws + gc0 + 2 * cp);
+        float sn, cs;
+        sincospif(__fdiv_rn((float)q, (float)N), &sn, &cs);
+        const float2 u = make_float2(cs, sn);
+        const float inL = (q <= omega) ? 0.5f : 0.f;
+        const float inH = (q != 0 && N - q <= omega) ? 0.5f : 0.f;
+        const float2 ch = chirp_f(n, N);
+        const float2 P0 = make_float2(P4.x, P4.y), P1 = make_float2(P4.z, P4.w);
+        const float2 uQ0 = cmul(make_float2(Q4.x, Q4.y), u), uQ1 = cmul(make_float2(Q4.z, Q4.w), u);
+        float2 E0 = csub(csub(P0, cscale(cadd(P0, uQ0), inL)), cscale(csub(P0, uQ0), inH));
+        float2 E1 = csub(csub(P1, cscale(cadd(P1, uQ1), inL)), cscale(csub(P1, uQ1), inH));
+        x0[p] = cmul_conj(cconj(E0), ch);
+        x1[p] = cmul_conj(cconj(E1), ch);
+      }
+    }
   }
   for (int i = tid; i < N1; i += NT) tw[i] = master[(size_t)i * (master_len / N1)];
   __syncthreads();
+  if (LD == LD_KV) {
 #pragma unroll
-  for (int p = 0; p < 16; ++p) {
-    accK = fmaf(x0[p].x, x0[p].x, fmaf(x1[p].x, x1[p].x, accK));
-    accV = fmaf(x0[p].y, x0[p].y, fmaf(x1[p].y, x1[p].y, accV));
+    for (int p = 0; p < 16; ++p) {
+      accK = fmaf(x0[p].x, x0[p].x, fmaf(x1[p].x, x1[p].x, accK));
+      accV = fmaf(x0[p].y, x0[p].y, fmaf(x1[p].y, x1[p].y, accV));
+    }
   }
   dft_fwd<16>(x0);
   dft_fwd<16>(x1);
@@ -116,6 +174,7 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
       *dst = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
     }
   }
+  if (LD == LD_FILTER) return;
   // per-block sums of squares (total energy of Eq. 12, by Parseval)
   const double a = warp_sum_d((double)accK), b = warp_sum_d((double)accV);
   if ((tid & 31) == 0) { red[0][tid >> 5] = a; red[1][tid >> 5] = b; }
@@ -136,10 +195,10 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
 // the slice, half hf (k1 = blockIdx.x or N1 - blockIdx.x), first-stage points
 // n2 = j + R2B*p.
 // ---------------------------------------------------------------------------
-template <int R2B, int CP>
+template <int R2B, int CP, int MID = MID_FILTER>
 __global__ void __launch_bounds__(2 * CP * R2B, 512 / (2 * CP * R2B > 32 ? 2 * CP * R2B : 32))
 k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ master, int master_len,
-     int omega) {
+     int omega, const float2 *__restrict__ hhat = nullptr, float scale = 1.f) {
   constexpr int N2 = 16 * R2B, NT = 2 * CP * R2B, IT = 16 / R2B;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                         // [2][N2][CP]
@@ -147,7 +206,9 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   float2 *twN = tw + N2;                                     // [2][N2] w_N^(n2*k1)
   float2 *uT = twN + 2 * N2;                                 // [2][N2] exp(-j*pi*(k1 + N1*k2)/N)
   const int tid = threadIdx.x, cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
-  const int k1a = blockIdx.x, k1b = (N1 - k1a) & (N1 - 1);
+  // MID_CONV: grid.x = N1/2, the two halves of the block are the unrelated rows 2x and 2x + 1
+  const int k1a = (MID == MID_CONV) ? 2 * blockIdx.x : blockIdx.x;
+  const int k1b = (MID == MID_CONV) ? 2 * blockIdx.x + 1 : ((N1 - k1a) & (N1 - 1));
   const bool self = (k1a == k1b);
   const int k1 = hf ? k1b : k1a;
   const int N = N1 * N2;
@@ -160,8 +221,10 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       tw[i] = master[(size_t)i * (master_len / N2)];
       twN[i] = master[(size_t)((i * k1a) & (N - 1)) * mstepN];
       twN[N2 + i] = master[(size_t)((i * k1b) & (N - 1)) * mstepN];
-      uT[i] = master[(size_t)(k1a + N1 * i) * ustep];
-      uT[N2 + i] = master[(size_t)(k1b + N1 * i) * ustep];
+      if (MID == MID_FILTER) {
+        uT[i] = master[(size_t)(k1a + N1 * i) * ustep];
+        uT[N2 + i] = master[(size_t)(k1b + N1 * i) * ustep];
+      }
     }
   }
   float4 *Sh = S + hf * (N2 * CP);
@@ -229,6 +292,12 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       for (int q = 0; q < R2B; ++q) {
         const int k2 = pp + 16 * q;
         const int bin = k1 + N1 * k2;
+        if (MID == MID_CONV) {
+          const float2 hq = cscale(__ldg(hhat + bin), scale);
+          x0[it * R2B + q] = cmul(x0[it * R2B + q], hq);
+          x1[it * R2B + q] = cmul(x1[it * R2B + q], hq);
+          continue;
+        }
         const bool inL = bin <= omega, inH = (N - bin) <= omega;
         float2 &P0 = x0[it * R2B + q], &P1 = x1[it * R2B + q];
         if (bin == 0 || (inL && inH)) {
@@ -300,13 +369,17 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
 // squared magnitude summed over the channels of the head, scores and the
 // per-block outlier-energy partial sums.
 // ---------------------------------------------------------------------------
-template <int R1B, int CPW>
+// OUT_SPEC and OUT_SCORE_CHIRP: N is the sequence length (< N1*N2), rows at or past it are dropped;
+// OUT_SPEC stores to spec[row][col] and returns; OUT_SCORE_CHIRP is given done_counter == nullptr and
+// leaves the final energy sums to the caller.
+template <int R1B, int CPW, int OUT = OUT_SCORE>
 __global__ void __launch_bounds__(CPW * R1B)
 k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__restrict__ master,
      int master_len, float *__restrict__ scores, int head0, int head_dim, long long score_stride,
      float inv_scale, double *__restrict__ partial, unsigned *__restrict__ done_counter,
      unsigned total_blocks, const double *__restrict__ part_tot, int n_tot,
-     const double *__restrict__ part_hi, int n_hi, double *__restrict__ energy) {
+     const double *__restrict__ part_hi, int n_hi, double *__restrict__ energy,
+     float2 *__restrict__ spec = nullptr) {
   constexpr int N1 = 16 * R1B, NT = CPW * R1B, IT = 16 / R1B, NW = (NT + 31) / 32;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                        // [N1][CPW]
@@ -359,6 +432,18 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
     dft_inv<16>(x1);
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
+      if (OUT != OUT_SCORE) {
+        const int pos = (j + R1B * p) * N2 + n2;
+        if (pos >= N) continue;
+        const float2 ch = chirp_f(pos, N);
+        x0[p] = cmul_conj(x0[p], ch);
+        x1[p] = cmul_conj(x1[p], ch);
+        if (OUT == OUT_SPEC) {
+          *reinterpret_cast<float4 *>(spec + (size_t)pos * ncol_ws + gc0 + 2 * cp) =
+              make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
+          continue;
+        }
+      }
       const float ek = fmaf(x0[p].x, x0[p].x, x1[p].x * x1[p].x);
       const float ev = fmaf(x0[p].y, x0[p].y, x1[p].y * x1[p].y);
       totK += ek;
@@ -367,6 +452,7 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
     }
     __syncthreads();
   }
+  if (OUT == OUT_SPEC) return;
   // transposed reduction over the CPW lanes that share j: the 16 row sums are halved at every
   // step until one is left, further steps are plain adds; row p = cp >> log2(CPW/16)
   {
@@ -391,7 +477,8 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
   constexpr int DUP = CPW / 16;                             // lanes that end with the same row sum
   if ((cp & (DUP - 1)) == 0) {
     const int p = (j + R1B * (cp / DUP)) * N2 + n2;
-    scores[(long long)(head0 + hh) * score_stride + perm_token(p, N)] = acc[0] * inv_scale;
+    if (OUT == OUT_SCORE || p < N)
+      scores[(long long)(head0 + hh) * score_stride + perm_token(p, N)] = acc[0] * inv_scale;
   }
   const double dk = warp_sum_d((double)(totK * inv_scale));
   const double dv = warp_sum_d((double)(totV * inv_scale));
@@ -407,6 +494,7 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
   }
   // The last block of the sequence (over all head groups, on either stream) adds up the
   // per-block partial sums in a fixed order: energy = (hiK, totK, hiV, totV).
+  if (OUT == OUT_SCORE_CHIRP) return;
   __shared__ bool is_last;
   if (tid == 0) {
     __threadfence();
