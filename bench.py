@@ -34,9 +34,9 @@ DEFAULT_CONFIG = "cfg3"          # the 32k-token workload the target fraction is
 # DRAM traffic per launch of the dominant kernel from the committed ncu capture
 # (profiles/), bytes; None until a capture of that kernel and workload exists.
 NCU_TRAFFIC_BYTES = {
-    # profiles/transform_passes_cfg3_dram_and_icache.md (c): 0.69 MB read + 0.70 MB written per launch of k_p2
+    # profiles/transform_passes_cfg3_dram_and_icache.md (d): 0.68 MB read + 0.79 MB written per launch of k_p2
     # (average over 24 launches with the intermediate in the persisting part of L2)
-    ("cfg3", "pass2"): 1.38e6,
+    ("cfg3", "pass2"): 1.47e6,
 }
 
 
