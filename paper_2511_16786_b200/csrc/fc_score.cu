@@ -901,20 +901,22 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
 // The chirp path on the specialised kernels, for transform lengths M = N1*N2 of 1024..65536 (sequence
 // lengths that are not a power of two, up to 32768): two circular convolutions with the chirp kernel, each
 // pass 1 -> pass 2 (multiply by the kernel's spectrum) -> pass 3, on the caller's stream.  Tile widths fixed.
-template <typename T, int R1B, int R2B>
+// DOUBLE: rows of 2 * 16 * R2B points, pass 2 joins two half-length transforms per row (131072 = 256 x 512).
+template <typename T, int R1B, int R2B, bool DOUBLE = false>
 fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq,
                             int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
                             double *phi, float *scores, long long total_tokens) {
-  constexpr int CPW = 32, CP = 8, N1 = 16 * R1B, N2 = 16 * R2B;
+  constexpr int CPW = 32, CP = 8, N1 = 16 * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
+  constexpr int MIDV = DOUBLE ? fast::MID_CONV2 : fast::MID_CONV;
   const int d = kv->head_dim, ncol = hg * d;
   const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
-  const size_t sm2 = (size_t)2 * N2 * CP * sizeof(float4) + 5 * N2 * sizeof(float2);
+  const size_t sm2 = (size_t)2 * (16 * R2B) * CP * sizeof(float4) + 5 * (16 * R2B) * sizeof(float2);
   const float invM = 1.f / (float)(N1 * N2);
-  const dim3 g1(N2, ncol / (2 * CPW)), g2(N1 / 2, ncol / (2 * CP)), g3(N2, hg);
+  const dim3 g1(N2, ncol / (2 * CPW)), g2(DOUBLE ? N1 : N1 / 2, ncol / (2 * CP)), g3(N2, hg);
   fc_status s;
   if ((s = set_smem(fast::k_p1<T, R1B, CPW, fast::LD_CHIRP>, sm1)) != FC_OK) return s;
   if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_FILTER>, sm1)) != FC_OK) return s;
-  if ((s = set_smem(fast::k_p2<R2B, CP, fast::MID_CONV>, sm2)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p2<R2B, CP, MIDV>, sm2)) != FC_OK) return s;
   if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SPEC>, sm1)) != FC_OK) return s;
   if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP>, sm1)) != FC_OK) return s;
   {
@@ -925,7 +927,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS2, st);
-    fast::k_p2<R2B, CP, fast::MID_CONV><<<g2, 2 * CP * R2B, sm2, st>>>(N1, ncol, ws, h->master, h->master_len, 0, hhat, invM);
+    fast::k_p2<R2B, CP, MIDV><<<g2, 2 * CP * R2B, sm2, st>>>(N1, ncol, ws, h->master, h->master_len, 0, hhat, invM);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
@@ -943,7 +945,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS2, st);
-    fast::k_p2<R2B, CP, fast::MID_CONV><<<g2, 2 * CP * R2B, sm2, st>>>(N1, ncol, ws, h->master, h->master_len, 0, hhat, invM);
+    fast::k_p2<R2B, CP, MIDV><<<g2, 2 * CP * R2B, sm2, st>>>(N1, ncol, ws, h->master, h->master_len, 0, hhat, invM);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
@@ -959,6 +961,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
 // Factors of the specialised kernels for a transform length (0, 0 when it has none).
 inline void fast_factors(int M, int *r1b, int *r2b) {
   *r1b = *r2b = 0;
+  if (M == 131072) { *r1b = 16; *r2b = 32; return; }           // 256 x 512: pass 2 takes its rows in two halves
   if (!is_pow2(M) || M < 1024 || M > 65536) return;
   const int bits = ilog2(M), b1 = bits / 2;
   *r1b = (1 << b1) / 16;
@@ -978,6 +981,9 @@ fc_status launch_chirp(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, cons
   FC_CHIRP_CASE(2, 2) FC_CHIRP_CASE(2, 4) FC_CHIRP_CASE(4, 4) FC_CHIRP_CASE(4, 8)
   FC_CHIRP_CASE(8, 8) FC_CHIRP_CASE(8, 16) FC_CHIRP_CASE(16, 16)
 #undef FC_CHIRP_CASE
+  if (a == 16 && b == 32)
+    return launch_chirp_impl<T, 16, 16, true>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, scores,
+                                              total_tokens);
   return FC_ERR_INTERNAL;
 }
 

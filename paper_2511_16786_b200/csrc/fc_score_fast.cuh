@@ -58,8 +58,11 @@ __device__ __forceinline__ float2 chirp_f(int n, int N) {
 //               conjugate) and times conj(chirp), zeros behind.
 enum { LD_KV = 0, LD_CHIRP = 1, LD_FILTER = 2 };
 // What pass 2 does between its forward and inverse halves: the DCT/low-pass residual filter on paired rows,
-// or a multiplication by the spectrum of the chirp kernel (rows 2x and 2x+1, unrelated).
-enum { MID_FILTER = 0, MID_CONV = 1 };
+// or a multiplication by the spectrum of the chirp kernel (rows 2x and 2x+1, unrelated).  MID_CONV2 is the
+// convolution for rows of 2*N2 points: the two halves of the block take the even and the odd samples of ONE
+// row through N2-point transforms, a radix-2 step joins them before the multiplication and splits the
+// product again after it (bins k and k + N2 live in the two halves' threads of equal index).
+enum { MID_FILTER = 0, MID_CONV = 1, MID_CONV2 = 2 };
 // What pass 3 does with the rows it gets back: scores of a power-of-two sequence, the N-point spectrum of
 // the chirp path (rows < N times conj(chirp)), or the scores at the end of the chirp path.
 enum { OUT_SCORE = 0, OUT_SPEC = 1, OUT_SCORE_CHIRP = 2 };
@@ -208,10 +211,12 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   const int tid = threadIdx.x, cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
   // MID_CONV: grid.x = N1/2, the two halves of the block are the unrelated rows 2x and 2x + 1
   const int k1a = (MID == MID_CONV) ? 2 * blockIdx.x : blockIdx.x;
-  const int k1b = (MID == MID_CONV) ? 2 * blockIdx.x + 1 : ((N1 - k1a) & (N1 - 1));
-  const bool self = (k1a == k1b);
+  const int k1b = (MID == MID_CONV) ? 2 * blockIdx.x + 1
+                : (MID == MID_CONV2) ? (int)blockIdx.x : ((N1 - k1a) & (N1 - 1));
+  const bool self = (MID == MID_FILTER) && (k1a == k1b);
   const int k1 = hf ? k1b : k1a;
-  const int N = N1 * N2;
+  constexpr int ROW = (MID == MID_CONV2) ? 2 * N2 : N2;      // points of one row of the workspace
+  const int N = N1 * ROW;
   const int gc0 = blockIdx.y * (2 * CP);
   const bool active = !(self && hf);
 
@@ -219,8 +224,14 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
     const int mstepN = master_len / N, ustep = master_len / (2 * N);
     for (int i = tid; i < N2; i += NT) {
       tw[i] = master[(size_t)i * (master_len / N2)];
-      twN[i] = master[(size_t)((i * k1a) & (N - 1)) * mstepN];
-      twN[N2 + i] = master[(size_t)((i * k1b) & (N - 1)) * mstepN];
+      if (MID == MID_CONV2) {
+        twN[i] = master[(size_t)(((2 * i) * k1a) & (N - 1)) * mstepN];           // even samples: n2 = 2i
+        twN[N2 + i] = master[(size_t)(((2 * i + 1) * k1a) & (N - 1)) * mstepN];   // odd samples: n2 = 2i + 1
+        uT[i] = master[(size_t)i * (master_len / ROW)];                          // w_ROW^k of the radix-2 step
+      } else {
+        twN[i] = master[(size_t)((i * k1a) & (N - 1)) * mstepN];
+        twN[N2 + i] = master[(size_t)((i * k1b) & (N - 1)) * mstepN];
+      }
       if (MID == MID_FILTER) {
         uT[i] = master[(size_t)(k1a + N1 * i) * ustep];
         uT[N2 + i] = master[(size_t)(k1b + N1 * i) * ustep];
@@ -229,11 +240,13 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   }
   float4 *Sh = S + hf * (N2 * CP);
   float2 x0[16], x1[16];
-  float2 *base = ws + ((size_t)k1 * N2) * ncol_ws + gc0 + 2 * cp;
+  // element n2 of the row: MID_CONV2 interleaves the halves (n2 = 2i + hf)
+  float2 *base = ws + ((size_t)k1 * ROW + (MID == MID_CONV2 ? hf : 0)) * ncol_ws + gc0 + 2 * cp;
+  const size_t rstride = (size_t)(MID == MID_CONV2 ? 2 : 1) * ncol_ws;
   if (active) {
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
-      const float4 t = *reinterpret_cast<const float4 *>(base + (size_t)(j + R2B * p) * ncol_ws);
+      const float4 t = *reinterpret_cast<const float4 *>(base + (size_t)(j + R2B * p) * rstride);
       x0[p] = make_float2(t.x, t.y);
       x1[p] = make_float2(t.z, t.w);
     }
@@ -298,6 +311,18 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
           x1[it * R2B + q] = cmul(x1[it * R2B + q], hq);
           continue;
         }
+        if (MID == MID_CONV2) {
+          // this thread holds E[k2] (hf = 0) or O[k2] (hf = 1); A[k2] = E + w O, A[k2 + N2] = E - w O
+          const float4 t = Sp[(q + R2B * pp) * CP + cp];
+          const float2 w = uT[k2];
+          float2 &m0 = x0[it * R2B + q], &m1 = x1[it * R2B + q];
+          const float2 e0 = hf ? make_float2(t.x, t.y) : m0, e1 = hf ? make_float2(t.z, t.w) : m1;
+          const float2 o0 = cmul(hf ? m0 : make_float2(t.x, t.y), w), o1 = cmul(hf ? m1 : make_float2(t.z, t.w), w);
+          const float2 hq = cscale(__ldg(hhat + k1 + N1 * (k2 + hf * N2)), scale);
+          m0 = cmul(hf ? csub(e0, o0) : cadd(e0, o0), hq);
+          m1 = cmul(hf ? csub(e1, o1) : cadd(e1, o1), hq);
+          continue;
+        }
         const bool inL = bin <= omega, inH = (N - bin) <= omega;
         float2 &P0 = x0[it * R2B + q], &P1 = x1[it * R2B + q];
         if (bin == 0 || (inL && inH)) {
@@ -317,6 +342,37 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
         }
       }
     }
+  }
+  if (MID == MID_CONV2) {
+    // B[k2] sits in half 0, B[k2 + N2] in half 1: even samples come back from B_lo + B_hi, odd samples from
+    // (B_lo - B_hi) * conj(w)
+    __syncthreads();                                   // everyone has read its partner's spectrum
+#pragma unroll
+    for (int it = 0; it < IT; ++it)
+#pragma unroll
+      for (int q = 0; q < R2B; ++q)
+        Sh[(q + R2B * (j + R2B * it)) * CP + cp] = make_float4(x0[it * R2B + q].x, x0[it * R2B + q].y,
+                                                               x1[it * R2B + q].x, x1[it * R2B + q].y);
+    __syncthreads();
+    const float4 *Sp = S + (1 - hf) * (N2 * CP);
+#pragma unroll
+    for (int it = 0; it < IT; ++it)
+#pragma unroll
+      for (int q = 0; q < R2B; ++q) {
+        const int pp = j + R2B * it, k2 = pp + 16 * q;
+        const float4 t = Sp[(q + R2B * pp) * CP + cp];
+        float2 &m0 = x0[it * R2B + q], &m1 = x1[it * R2B + q];
+        if (hf == 0) {
+          m0 = cadd(m0, make_float2(t.x, t.y));
+          m1 = cadd(m1, make_float2(t.z, t.w));
+        } else {
+          const float2 w = uT[k2];
+          m0 = cmul_conj(csub(make_float2(t.x, t.y), m0), w);
+          m1 = cmul_conj(csub(make_float2(t.z, t.w), m1), w);
+        }
+      }
+  }
+  if (active) {
     // first inverse stage (mirror of the second forward stage)
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
@@ -359,7 +415,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
     for (int p = 0; p < 16; ++p) {
       const float2 w = twN[hf * N2 + j + R2B * p];
       const float2 a = cmul_conj(x0[p], w), b = cmul_conj(x1[p], w);
-      *reinterpret_cast<float4 *>(base + (size_t)(j + R2B * p) * ncol_ws) = make_float4(a.x, a.y, b.x, b.y);
+      *reinterpret_cast<float4 *>(base + (size_t)(j + R2B * p) * rstride) = make_float4(a.x, a.y, b.x, b.y);
     }
   }
 }
