@@ -905,10 +905,12 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
 template <typename T, int R1B, int R2B, bool DOUBLE = false>
 fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq,
                             int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
-                            double *phi, float *scores, long long total_tokens) {
+                            double *phi, float *scores, long long total_tokens, int dcols, int accumulate) {
   constexpr int CPW = 32, CP = 8, N1 = 16 * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
   constexpr int MIDV = DOUBLE ? fast::MID_CONV2 : fast::MID_CONV;
-  const int d = kv->head_dim, ncol = hg * d;
+  // dcols: columns of a head in this launch (head_dim, or a column group of one head: kp/vp point at its
+  // first channel and hg is 1)
+  const int d = kv->head_dim, ncol = hg * dcols;
   const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
   const size_t sm2 = (size_t)2 * (16 * R2B) * CP * sizeof(float4) + 5 * (16 * R2B) * sizeof(float2);
   const float invM = 1.f / (float)(N1 * N2);
@@ -922,7 +924,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   {
     ProfScope ps(h, FC_K_PASS1, st);
     fast::k_p1<T, R1B, CPW, fast::LD_CHIRP><<<g1, CPW * R1B, sm1, st>>>(
-        kp, vp, kv->stride_token, kv->stride_head, h0, d, Nseq, N2, ncol, ws, h->master, h->master_len, ptot);
+        kp, vp, kv->stride_token, kv->stride_head, h0, dcols, Nseq, N2, ncol, ws, h->master, h->master_len, ptot);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
@@ -933,7 +935,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   {
     ProfScope ps(h, FC_K_PASS3, st);
     fast::k_p3<R1B, CPW, fast::OUT_SPEC><<<g3, CPW * R1B, sm1, st>>>(
-        Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, h0, d, 0, 0.f, nullptr, nullptr, 0u, nullptr, 0, nullptr, 0,
+        Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, h0, dcols, 0, 0.f, nullptr, nullptr, 0u, nullptr, 0, nullptr, 0,
         nullptr, spec);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
@@ -952,8 +954,8 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
     ProfScope ps(h, FC_K_PASS3, st);
     const float inv = (float)(1.0 / ((double)Nseq * (double)Nseq * (double)d));
     fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP><<<g3, CPW * R1B, sm1, st>>>(
-        Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, d, total_tokens, inv, phi, nullptr, 0u, nullptr, 0,
-        nullptr, 0, nullptr, nullptr);
+        Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, dcols, total_tokens, inv, phi, nullptr, 0u, nullptr, 0,
+        nullptr, 0, nullptr, nullptr, (float)d, accumulate);
   }
   return fc_after_launch(h);
 }
@@ -971,19 +973,19 @@ inline void fast_factors(int M, int *r1b, int *r2b) {
 template <typename T>
 fc_status launch_chirp(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq, int M,
                        int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
-                       double *phi, float *scores, long long total_tokens) {
+                       double *phi, float *scores, long long total_tokens, int dcols, int accumulate) {
   int a, b;
   fast_factors(M, &a, &b);
 #define FC_CHIRP_CASE(A, B)                                                                                  \
   if (a == A && b == B)                                                                                      \
     return launch_chirp_impl<T, A, B>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, scores, \
-                                      total_tokens);
+                                      total_tokens, dcols, accumulate);
   FC_CHIRP_CASE(2, 2) FC_CHIRP_CASE(2, 4) FC_CHIRP_CASE(4, 4) FC_CHIRP_CASE(4, 8)
   FC_CHIRP_CASE(8, 8) FC_CHIRP_CASE(8, 16) FC_CHIRP_CASE(16, 16)
 #undef FC_CHIRP_CASE
   if (a == 16 && b == 32)
     return launch_chirp_impl<T, 16, 16, true>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, scores,
-                                              total_tokens);
+                                              total_tokens, dcols, accumulate);
   return FC_ERR_INTERNAL;
 }
 
@@ -1224,11 +1226,17 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       // stream order and the last pass adds their contributions to the score in that order.
       int fa, fb;
       fast_factors(sp.Nfft, &fa, &fb);
-      if (fa != 0 && !h->generic_only && L.sub_cols == d) {      // whole heads, a length the specialised kernels take
-        if ((s = launch_chirp<T>(h, st, kv, kp, vp, N, sp.Nfft, h0, hg, omega, ws, spec, hhat, ptot, phi,
-                                 scores + start, total_tokens)) != FC_OK) return s;
-        tot_slots += (size_t)(16 * fb) * (ncol_ws / 64);
-        hi_slots += (size_t)(16 * fb) * hg;
+      if (fa != 0 && !h->generic_only && L.sub_cols % 64 == 0) {   // a length and a width the specialised kernels take
+        const int sub = L.sub_cols, ngr = (hg == 1) ? d / sub : 1, n2f = 16 * fb;
+        const int ncol = (hg == 1) ? sub : ncol_ws;
+        for (int cg = 0; cg < ngr; ++cg) {                        // column groups of one head, else one pass
+          if ((s = launch_chirp<T>(h, st, kv, kp + cg * sub, vp + cg * sub, N, sp.Nfft, h0, hg, omega, ws, spec, hhat,
+                                   ptot + 2 * (size_t)cg * n2f * (ncol / 64), phi + 2 * (size_t)cg * n2f * hg,
+                                   scores + start, total_tokens, (hg == 1) ? sub : d, cg > 0 ? 1 : 0)) != FC_OK)
+            return s;
+        }
+        tot_slots += (size_t)n2f * (ncol / 64) * ngr;
+        hi_slots += (size_t)n2f * hg * ngr;
         continue;
       }
       const float invM = 1.f / (float)sp.Nfft;

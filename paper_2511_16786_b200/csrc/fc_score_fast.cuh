@@ -435,7 +435,9 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
      float inv_scale, double *__restrict__ partial, unsigned *__restrict__ done_counter,
      unsigned total_blocks, const double *__restrict__ part_tot, int n_tot,
      const double *__restrict__ part_hi, int n_hi, double *__restrict__ energy,
-     float2 *__restrict__ spec = nullptr) {
+     float2 *__restrict__ spec = nullptr, float energy_scale = 0.f, int accumulate = 0) {
+  // OUT_SCORE_CHIRP with a head transformed in column groups: head_dim is the group's width, energy_scale the
+  // head's true channel count, and every group after the first adds to the stored score (accumulate).
   constexpr int N1 = 16 * R1B, NT = CPW * R1B, IT = 16 / R1B, NW = (NT + 31) / 32;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                        // [N1][CPW]
@@ -533,8 +535,12 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
   constexpr int DUP = CPW / 16;                             // lanes that end with the same row sum
   if ((cp & (DUP - 1)) == 0) {
     const int p = (j + R1B * (cp / DUP)) * N2 + n2;
-    if (OUT == OUT_SCORE || p < N)
+    if (OUT == OUT_SCORE) {
       scores[(long long)(head0 + hh) * score_stride + perm_token(p, N)] = acc[0] * inv_scale;
+    } else if (p < N) {
+      float *dst = scores + (long long)(head0 + hh) * score_stride + perm_token(p, N);
+      *dst = accumulate ? *dst + acc[0] * inv_scale : acc[0] * inv_scale;
+    }
   }
   const double dk = warp_sum_d((double)(totK * inv_scale));
   const double dv = warp_sum_d((double)(totV * inv_scale));
@@ -545,8 +551,9 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
 #pragma unroll
     for (int i = 0; i < NW; ++i) { sa += red[0][i]; sb += red[1][i]; }
     const size_t slot = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
-    partial[2 * slot] = sa * (double)head_dim;
-    partial[2 * slot + 1] = sb * (double)head_dim;
+    const double es = (OUT == OUT_SCORE_CHIRP) ? (double)energy_scale : (double)head_dim;
+    partial[2 * slot] = sa * es;
+    partial[2 * slot + 1] = sb * es;
   }
   // The last block of the sequence (over all head groups, on either stream) adds up the
   // per-block partial sums in a fixed order: energy = (hiK, totK, hiV, totV).
