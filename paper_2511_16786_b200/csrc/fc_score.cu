@@ -686,6 +686,8 @@ struct ScoreLayout {
   size_t ws_buf_bytes;       // one group buffer; the fast path keeps two and alternates
   int heads_per_group;
   int sub_cols;              // chirp path: columns of one head transformed together (head_dim = all of them)
+  int chirp_streams;         // chirp path: internal streams the head groups alternate over (1 = the caller's stream)
+  size_t spec_buf_bytes;     // chirp path: one group's N-point spectrum; one copy per stream
 };
 
 // Workspace carve-up for one sequence plan (all sequences share the regions; the
@@ -703,6 +705,7 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
       L.total = f.ring_bytes + 2 * f.part_bytes + f.partial_bytes;
       L.ws_buf_bytes = f.ring_bytes;
       L.heads_per_group = num_heads;
+      L.chirp_streams = 1;
       return L;
     }
   }
@@ -711,9 +714,14 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   if (hg < 1) hg = 1;
   if (hg > num_heads) hg = num_heads;
   int groups = (num_heads + hg - 1) / hg;
-  if (sp.fast && groups < h->num_aux && num_heads >= h->num_aux) groups = h->num_aux;   // keep every internal stream busy
+  // Chirp transforms of up to 32768 points on the specialised kernels also alternate over the internal streams:
+  // a group's intermediate and spectrum (at most 50 MB) then stay in the L2 twice over.
+  const bool chirp_multi = sp.bluestein && !h->generic_only && h->aux[0] != nullptr && sp.Nfft >= 1024 &&
+                           sp.Nfft <= 32768 && num_heads >= h->num_aux && h->num_aux > 1;
+  if ((sp.fast || chirp_multi) && groups < h->num_aux && num_heads >= h->num_aux) groups = h->num_aux;   // keep every internal stream busy
   hg = (num_heads + groups - 1) / groups;                      // balanced groups
   L.heads_per_group = hg;
+  L.chirp_streams = chirp_multi ? h->num_aux : 1;
   // Chirp path, one head per group: the head is split into column groups only when its intermediates
   // pass four times the budget.  Narrower tiles cost time (measured: +2 % at 64 columns, +8 % at 32 for
   // 131072-point transforms) and the generic kernels do not wait on DRAM, so below that the split
@@ -725,8 +733,9 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   L.sub_cols = sub;
   L.ws_buf_bytes = align_up((size_t)sp.Nfft * sub * hg * sizeof(float2), 256);
   size_t off = 0;
-  L.off_ws = off;       off += L.ws_buf_bytes * (sp.fast ? h->num_aux : 1);
-  L.off_spec = off;     off += sp.bluestein ? align_up((size_t)sp.N * sub * hg * sizeof(float2), 256) : 0;
+  L.off_ws = off;       off += L.ws_buf_bytes * (sp.fast ? h->num_aux : L.chirp_streams);
+  L.spec_buf_bytes = sp.bluestein ? align_up((size_t)sp.N * sub * hg * sizeof(float2), 256) : 0;
+  L.off_spec = off;     off += L.spec_buf_bytes * L.chirp_streams;
   L.off_hhat = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * sizeof(float2), 256) : 0;
   L.off_hcol = off;     off += sp.bluestein ? align_up((size_t)sp.Nfft * 8 * sizeof(float2), 256) : 0;
   const size_t slices = (size_t)num_heads * head_dim / 32;   // finest slicing any kernel variant uses
@@ -1195,6 +1204,11 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     }
     h->last_sig = sig;
   }
+  const bool chirp_fork = sp.bluestein && L.chirp_streams > 1;
+  if (chirp_fork) {                     // the internal streams start after the chirp kernel's spectrum is ready
+    FC_CUDA_TRY(cudaEventRecord(h->ev_fork, st));
+    for (int i = 0; i < L.chirp_streams; ++i) FC_CUDA_TRY(cudaStreamWaitEvent(h->aux[i], h->ev_fork, 0));
+  }
   size_t tot_slots = 0, hi_slots = 0;
   int group = 0;
   for (int h0 = 0; h0 < H; h0 += L.heads_per_group, ++group) {
@@ -1229,8 +1243,12 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       if (fa != 0 && !h->generic_only && L.sub_cols % 64 == 0) {   // a length and a width the specialised kernels take
         const int sub = L.sub_cols, ngr = (hg == 1) ? d / sub : 1, n2f = 16 * fb;
         const int ncol = (hg == 1) ? sub : ncol_ws;
+        const int si = group % L.chirp_streams;                   // head groups alternate over the internal streams
+        cudaStream_t sx = L.chirp_streams > 1 ? h->aux[si] : st;
+        float2 *ws_s = reinterpret_cast<float2 *>(wsb + L.off_ws + (size_t)si * L.ws_buf_bytes);
+        float2 *spec_s = reinterpret_cast<float2 *>(wsb + L.off_spec + (size_t)si * L.spec_buf_bytes);
         for (int cg = 0; cg < ngr; ++cg) {                        // column groups of one head, else one pass
-          if ((s = launch_chirp<T>(h, st, kv, kp + cg * sub, vp + cg * sub, N, sp.Nfft, h0, hg, omega, ws, spec, hhat,
+          if ((s = launch_chirp<T>(h, sx, kv, kp + cg * sub, vp + cg * sub, N, sp.Nfft, h0, hg, omega, ws_s, spec_s, hhat,
                                    ptot + 2 * (size_t)cg * n2f * (ncol / 64), phi + 2 * (size_t)cg * n2f * hg,
                                    scores + start, total_tokens, (hg == 1) ? sub : d, cg > 0 ? 1 : 0)) != FC_OK)
             return s;
@@ -1291,6 +1309,12 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     }
   }
   if (sp.fast) return FC_OK;          // the last pass-3 block of the sequence has written the energy sums
+  if (chirp_fork) {                     // the caller's stream takes over again for the energy sums
+    for (int i = 0; i < L.chirp_streams; ++i) {
+      FC_CUDA_TRY(cudaEventRecord(h->ev_join[i], h->aux[i]));
+      FC_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_join[i], 0));
+    }
+  }
   {
     ProfScope ps(h, FC_K_OTHER, st);
     k_energy_finalize<<<1, 256, 0, st>>>(part_tot, (int)tot_slots, part_hi, (int)hi_slots, energy_b);
