@@ -169,6 +169,25 @@ def test_scores_long_arbitrary_length(fc):
     _check_layer(fc, k, v, [0, N], 0.2)
 
 
+def test_scores_mixed_paths_in_one_call(fc):
+    # power-of-two and other lengths alternate in one batch: the specialised transform path (two internal
+    # streams, work left pending), the chirp path on the same streams (joined per sequence), a 131072-point chirp
+    # transform and a tiny generic one; results match the oracle and do not change from run to run
+    lens = [5000, 4096, 3000, 8192, 33000, 7, 2048]
+    cu = [0] + [int(x) for x in np.cumsum(lens)]
+    k, v = _rand_kv(cu[-1], 4, 128, torch.bfloat16, 12)
+    g1, e1 = _check_layer(fc, k, v, cu, 0.2, max_seqlen=65536)
+    g2, e2 = _gpu_scores(fc, k, v, cu, 0.2, max_seqlen=65536)
+    assert np.array_equal(g1, g2) and np.array_equal(e1, e2)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
+def test_scores_131072_point_chirp_transform(fc, dtype):
+    N = 33001
+    k, v = _rand_kv(N, 2, 128, dtype, 13)
+    _check_layer(fc, k, v, [0, N], 0.2)
+
+
 @pytest.mark.parametrize("d,group_bytes", [(128, 1), (128, 1 << 20), (192, 1), (64, 1)])
 def test_scores_arbitrary_length_in_column_groups(fc, d, group_bytes):
     # a small cache budget makes the chirp path transform each head in groups of 32..96 columns
