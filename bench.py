@@ -255,7 +255,7 @@ def run_decode(args):
             graph = torch.cuda.CUDAGraph()
             side = torch.cuda.Stream(device=dev)
             side.wait_stream(torch.cuda.current_stream(dev))
-            with torch.cuda.graph(graph, stream=side):
+            with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
                 step()
             for e0, e1 in ev:
                 flush.zero_()
@@ -433,7 +433,7 @@ def main():
 
     # the same step replayed from a CUDA graph (reported beside the headline, which stays the plain call
     # sequence because only that one carries the per-kernel event timing)
-    if not args.no_graph:
+    if not args.no_graph and world == 1:
         graph = comp.capture(Kd, Vd)
         for _ in range(3):
             graph.replay()

@@ -532,7 +532,8 @@ class Compressor:
         side.wait_stream(torch.cuda.current_stream(self.device))
         fc_reset_ordering(self.handle)
         try:
-            with torch.cuda.graph(graph, stream=side):
+            # only this thread's calls belong to the capture (a collective library's watchdog thread may query events meanwhile)
+            with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
                 self.compress(K_layers, V_layers)
         finally:
             fc_reset_ordering(self.handle)
