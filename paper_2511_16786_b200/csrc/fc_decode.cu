@@ -24,7 +24,8 @@ constexpr int kStageBytes = 4 * kBoxBytes;   // K low/high halves, V low/high ha
 // 2 and 3 (three and two blocks per SM) and 5..7 were slower (1.05, 0.98, 0.84..0.91 against 0.82 ms for
 // 28 layers of 65536 rows)
 constexpr int kStages = 4;
-constexpr unsigned kSpinLimit = 1u << 20;    // blocking tests of an mbarrier before a wait gives up
+constexpr unsigned kSuspendNs = 2000u;        // a blocking test of an mbarrier sleeps at most about this long
+constexpr unsigned kSpinLimit = 1u << 17;    // such tests before a wait gives up (a quarter of a second)
 
 struct DecodeParams {
   const void *q;
@@ -51,8 +52,8 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned
 // One potentially blocking test: the thread sleeps until the phase completes or a hardware time limit passes.
 __device__ __forceinline__ bool mbar_try(unsigned long long *bar, unsigned parity) {
   unsigned ok;
-  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-               : "=r"(ok) : "r"((unsigned)__cvta_generic_to_shared(bar)), "r"(parity) : "memory");
+  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"((unsigned)__cvta_generic_to_shared(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
   return ok != 0u;
 }
 // Bounded wait; false = gave up.
@@ -189,7 +190,7 @@ k_decode_partial(const DecodeParams P, const __grid_constant__ DecodeMaps M) {
   float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
   const unsigned sbase = (unsigned)__cvta_generic_to_shared(smem);
   bool failed = false;
-  int issued = 0;
+  int issued = 0, consumed = 0;
 
   if (tid == 0)
     for (int ti = 0; ti < kStages - 1 && ti < ntiles; ++ti) { issue(ti, ti); issued = ti + 1; }
@@ -201,7 +202,7 @@ k_decode_partial(const DecodeParams P, const __grid_constant__ DecodeMaps M) {
       issued = ti + kStages;
     }
     const bool got = mbar_wait(&full[s], (unsigned)(ti / kStages) & 1u);
-    if (__syncthreads_or(got ? 0 : 1)) { failed = true; break; }
+    if (__syncthreads_or(got ? 0 : 1)) { failed = true; consumed = ti; break; }
     const int row0 = lo + ti * kTile;
     int valid = (row0 < n_main_pad ? n_main : total) - row0;
     valid = valid > kTile ? kTile : valid;
@@ -273,7 +274,7 @@ k_decode_partial(const DecodeParams P, const __grid_constant__ DecodeMaps M) {
     // (they write this block's shared memory), and report an empty share
     if (tid == 0) {
       atomicOr(P.status, FC_DEV_FLAG_TIMEOUT);
-      for (int ti = 0; ti < issued; ++ti) mbar_wait(&full[ti % kStages], (unsigned)(ti / kStages) & 1u);
+      for (int ti = consumed; ti < issued; ++ti) mbar_wait(&full[ti % kStages], (unsigned)(ti / kStages) & 1u);
     }
     m[0] = m[1] = -INFINITY;
     l[0] = l[1] = 0.f;
