@@ -286,6 +286,46 @@ def run_decode(args):
         "points": points}))
 
 
+# --------------------------------------------------------------------------- spectrum diagnostics
+def run_spectrum(args):
+    """Time of fc_power_spectrum (Eq. 11 per layer) over all layers of a config; a diagnostic, reported beside
+    the transform work it repeats (pass 1 and half of pass 2 of the scoring)."""
+    import torch
+    from paper_2511_16786_b200 import binding, synth_kv as S
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    cfg = S.paper_configs()[args.config]
+    L = cfg.num_layers
+    Kd, Vd = zip(*[S.make_layer(cfg, l, dev) for l in range(L)])
+    handle = binding.fc_create(0, max(cfg.seqlens))
+    spec = torch.empty((L, cfg.total_tokens, 2), dtype=torch.float64, device=dev)
+    ws = torch.empty(binding.fc_power_spectrum_workspace_bytes(handle, Kd[0], Vd[0], cfg.cu_seqlens),
+                     dtype=torch.uint8, device=dev)
+
+    def step():
+        for l in range(L):
+            binding.fc_power_spectrum(handle, Kd[l], Vd[l], cfg.cu_seqlens, spec[l], ws)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    binding._check(binding.fc_last_device_status(handle), "device status")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    steps = max(3, min(args.steps, 20))
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    binding.fc_destroy(handle)
+    print(json.dumps({"metric": "power_spectrum_ms_per_pass", "value": ms, "unit": "ms", "higher_is_better": False,
+                      "n_gpus": 1, "steps": steps, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": cfg.name + ": " + cfg.note, "layers": L,
+                                 "l2_policy": "inputs exceed L2; no flush"},
+                      "tokens_per_s": cfg.total_tokens / (ms / 1000.0)}))
+
+
 # --------------------------------------------------------------------------- main arm
 def main():
     ap = argparse.ArgumentParser()
@@ -304,6 +344,7 @@ def main():
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--decode", action="store_true",
                     help="time the decoding-step attention on full and compressed caches instead of the compressor")
+    ap.add_argument("--spectrum", action="store_true", help="time fc_power_spectrum over all layers of the config")
     ap.add_argument("--decode-n", type=int, default=0, help="--decode: only this context length")
     ap.add_argument("--decode-rho", type=float, default=0.0, help="--decode: only this cache ratio")
     args = ap.parse_args()
@@ -312,6 +353,9 @@ def main():
         return
     if args.decode:
         run_decode(args)
+        return
+    if args.spectrum:
+        run_spectrum(args)
         return
 
     import torch
