@@ -100,6 +100,20 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
     fc_destroy(h);
     return FC_ERR_CUDA;
   }
+  {
+    // room for the chirp kernel's spectrum of the longest sequence that is not a power of two (transform
+    // length: the power of two from 2N-1 up, at most 131072)
+    int m = 64;
+    const int nmax = max_seqlen < 65536 ? max_seqlen : 65536;
+    while (m < 2 * nmax - 1) m <<= 1;
+    h->hhat_cache_len = m;
+    for (int i = 0; i < FC_HHAT_SLOTS; ++i) h->hhat_cache_n[i] = 0;
+    h->hhat_cache_next = 0;
+    if (cudaMalloc(&h->hhat_cache, (size_t)FC_HHAT_SLOTS * m * sizeof(float2)) != cudaSuccess) {
+      fc_destroy(h);
+      return FC_ERR_CUDA;
+    }
+  }
   k_fill_master<<<(h->master_len + 255) / 256, 256>>>(h->master, h->master_len);
   if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
     fc_destroy(h);
@@ -177,6 +191,7 @@ extern "C" void fc_destroy(fc_handle *h) {
   for (int i = 0; i < h->host_ev_cap; ++i) cudaEventDestroy(h->host_ev[i]);
   delete[] h->host_ev;
   if (h->ev_inputs_free) cudaEventDestroy(h->ev_inputs_free);
+  if (h->hhat_cache) cudaFree(h->hhat_cache);
   if (h->master) cudaFree(h->master);
   if (h->status_word) cudaFree(h->status_word);
   if (h->done_counter) cudaFree(h->done_counter);
@@ -247,6 +262,7 @@ extern "C" fc_status fc_reset_ordering(fc_handle *h) {
   h->last_sig = 0;
   h->pending_join = false;
   h->host_last_arena = nullptr;
+  for (int i = 0; i < FC_HHAT_SLOTS; ++i) h->hhat_cache_n[i] = 0;
   return FC_OK;
 }
 

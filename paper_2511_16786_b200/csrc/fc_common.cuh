@@ -14,6 +14,7 @@
 
 #define FC_MAX_STAGES 4
 #define FC_MAX_AUX 4     // internal streams a handle may use
+#define FC_HHAT_SLOTS 8  // chirp-kernel spectra a handle keeps (one per sequence length)
 
 // Bits of the device status word.
 #define FC_DEV_FLAG_INTERNAL 1
@@ -67,6 +68,11 @@ struct fc_handle {
   // fc_compress_host (created on its first call): the stream the host-to-device copies run on, one
   // event per layer (that layer's copies have landed), and the point of the previous job after
   // which the staged inputs of its arena may be overwritten
+  // spectra of the chirp kernel of the last FC_HHAT_SLOTS sequence lengths that took the chirp path (DEVICE,
+  // allocated by fc_create: FC_HHAT_SLOTS x hhat_cache_len points; hhat_cache_n[i] = length in slot i, 0 = none;
+  // slots are reused round robin)
+  float2 *hhat_cache;
+  int hhat_cache_len, hhat_cache_n[FC_HHAT_SLOTS], hhat_cache_next;
   cudaStream_t host_copy;
   cudaEvent_t *host_ev;
   int host_ev_cap;

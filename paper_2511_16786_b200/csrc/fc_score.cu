@@ -1159,10 +1159,35 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   }
 
   if (sp.bluestein) {
-    // spectrum of the chirp kernel, once per sequence
-    ChirpKernelLoader cl{N, sp.Nfft};
-    if ((s = launch_pass1(h, st, cl, sp, 8, 8, hcol, nullptr)) != FC_OK) return s;
-    if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
+    // Spectrum of the chirp kernel.  It depends on the sequence length only, so the handle keeps the last few
+    // (layers of a prefill share their lengths).  While the stream is being captured the spectrum goes to the
+    // workspace instead, every time: a graph must not depend on what the handle holds when it is replayed.
+    bool cached = false;
+    if (h->hhat_cache && !h->generic_only && sp.Nfft <= h->hhat_cache_len) {
+      cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+      if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusActive; }
+      cached = (cap == cudaStreamCaptureStatusNone);
+    }
+    bool have = false;
+    int slot = 0;
+    if (cached) {
+      for (int i = 0; i < FC_HHAT_SLOTS && !have; ++i)
+        if (h->hhat_cache_n[i] == N) { have = true; slot = i; }
+      if (!have) {
+        // the slot taken over was last read by a sequence that has been joined to `st` since (the chirp path
+        // joins the internal streams before it returns), so stream order protects it
+        slot = h->hhat_cache_next;
+        h->hhat_cache_next = (slot + 1) % FC_HHAT_SLOTS;
+        h->hhat_cache_n[slot] = 0;                          // not valid until both launches are in the stream
+      }
+      hhat = h->hhat_cache + (size_t)slot * h->hhat_cache_len;
+    }
+    if (!have) {
+      ChirpKernelLoader cl{N, sp.Nfft};
+      if ((s = launch_pass1(h, st, cl, sp, 8, 8, hcol, nullptr)) != FC_OK) return s;
+      if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
+      if (cached) h->hhat_cache_n[slot] = N;
+    }
   }
 
   // fc_score_layer has claimed the persisting part of L2 if any sequence of the call takes this path
