@@ -62,7 +62,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
     if (mbar_try(bar, parity)) return true;
   return false;
 }
-// Tiled loads into this block's shared memory; completion is counted in bytes on `bar`.  No multicast.
+// Tiled loads into this block's shared memory; completion is counted in bytes on `bar`.  One destination block only.
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2,
                                             unsigned long long *bar) {
   asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"

@@ -270,7 +270,7 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned
   asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}\n"
                ::"r"((unsigned)__cvta_generic_to_shared(bar)), "r"(bytes) : "memory");
 }
-// Tiled loads into this block's shared memory; completion is counted in bytes on `bar`.  No multicast.
+// Tiled loads into this block's shared memory; completion is counted in bytes on `bar`.  One destination block only.
 __device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *map, int c0, int c1, int c2,
                                             unsigned long long *bar) {
   asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n"
