@@ -376,6 +376,7 @@ fc_status fc_score_layer_static(const fc_kv_view *kv, double gamma, float *score
  *                    index entries); fc_compress_host_rows() gives the number needed.
  * budgets_host, offsets_host and layer_rows_host are already valid when the call returns: the call
  * blocks the host once, after the budgets are known, to learn the sizes of the copies back.
+ * (For that reason the call cannot be captured into a CUDA graph; the per-stage entry points can.)
  *
  * Errors: FC_ERR_INVALID_ARG, FC_ERR_UNSUPPORTED (as fc_score_layer), FC_ERR_WORKSPACE (arena
  * too small or misaligned; more rows than out_capacity_rows, in which case nothing is copied
