@@ -117,7 +117,7 @@ def step_accounting(binding, handle, cfg):
     algorithm has to compute and move, not what the hardware happened to do)."""
     d, H, L = cfg.head_dim, cfg.num_heads, cfg.num_layers
     s = 4 if cfg.dtype == "f32" else 2
-    acc = {k: dict(flops=0.0, bytes=0.0) for k in ("pass1", "pass2", "pass3", "select", "gather", "fused")}
+    acc = {k: dict(flops=0.0, bytes=0.0) for k in ("pass1", "pass2", "pass3", "select", "gather")}
     rows = 0
     for N in cfg.seqlens:
         if N == 0:
@@ -134,10 +134,6 @@ def step_accounting(binding, handle, cfg):
         acc["select"]["bytes"] += N * H * L * 4.0                      # score read
         acc["gather"]["bytes"] += cfg.rho * N * H * L * (4.0 * d * s + 4.0)
         rows += N * H * L
-    # the fused transform kernel does the work of the three passes in one launch
-    for k in ("pass1", "pass2", "pass3"):
-        acc["fused"]["flops"] += acc[k]["flops"]
-        acc["fused"]["bytes"] += acc[k]["bytes"]
     return acc, rows
 
 
@@ -456,7 +452,7 @@ def main():
                 class_ms_per_step={k: v["ms"] for k, v in shares.items()})
     s = 4 if cfg.dtype == "f32" else 2
     step_bytes = rows * (2.0 * cfg.head_dim * s + 8.0 + cfg.rho * (4.0 * cfg.head_dim * s + 4.0))
-    step_flops = sum(v["flops"] for k, v in acc.items() if k != "fused")
+    step_flops = sum(v["flops"] for v in acc.values())
     t_bound = max(step_bytes / (peaks["hbm_gbs"] * 1e9), step_flops / (alu_peak * 1e12))
     roof_step = dict(bound="alu" if step_flops / (alu_peak * 1e12) >= step_bytes / (peaks["hbm_gbs"] * 1e9) else "hbm",
                      t_bound_ms=1000.0 * t_bound, frac=t_bound / (ms_per_step / 1000.0),

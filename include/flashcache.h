@@ -95,14 +95,6 @@ fc_status fc_profile_begin(fc_handle *h, int32_t kernel_class, int32_t max_launc
 fc_status fc_profile_stride(fc_handle *h, int32_t stride);
 fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *launches);
 
-/* Chooses how power-of-two sequences of 4096..65536 tokens are transformed: enabled = 0 (default)
- * runs the three passes as separate launches per head group, enabled = 1 runs ONE persistent
- * kernel per (layer, sequence) that hands out tiles of all three passes in dependency order;
- * stage_lag (1..4) is the distance, in units of about 8 MB of intermediate, between the passes
- * of a unit.  Same results up to fp32 rounding; affects speed and workspace size only, so call
- * it before fc_score_workspace_bytes. */
-fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_lag);
-
 /* enabled = 1: fc_score_layer calls for power-of-two lengths of 1024..65536 tokens leave their
  * work on the library's two internal streams instead of making `stream` wait for it, so that the
  * next layer starts while the last kernels of this one drain.  Inputs are still taken in stream
@@ -129,14 +121,6 @@ fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled);
  * Everything enqueued earlier through the handle must already be complete, or be ordered before the
  * next call by the stream that call is given (a graph launch on that stream is). */
 fc_status fc_reset_ordering(fc_handle *h);
-
-/* Running totals of the fused transform kernel since fc_create (diagnostic; synchronises the
- * device): out = { tiles processed, tiles whose inputs were not finished when they were looked
- * when the scheduler warp first looked, unused, clock cycles (thread 0 of every block, summed) inside
- * pass-1, pass-2 and pass-3 tiles, cycles waiting for tile data, cycles inside the tile loop,
- * scheduler-warp cycles waiting for a buffer to come back, waiting for dependencies, issuing loads,
- * and compute-warp cycles between the end of an issue and the buffer being full (waits only) }. */
-fc_status fc_fused_stats(fc_handle *h, uint64_t out[12]);
 
 /* Target size in bytes of the transform intermediates processed per kernel group
  * (kept below the L2 capacity so they are re-read from cache, not HBM).

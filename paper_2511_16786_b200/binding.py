@@ -23,7 +23,7 @@ _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
     "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count",
-    "fc_set_group_bytes", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_set_fused", "fc_fused_stats", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
+    "fc_set_group_bytes", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
     "fc_power_spectrum_workspace_bytes", "fc_power_spectrum",
@@ -100,10 +100,6 @@ def _load() -> ctypes.CDLL:
     lib.fc_set_score_overlap.restype = c_int
     lib.fc_set_select_overlap.argtypes = [c_void_p, c_int32]
     lib.fc_set_select_overlap.restype = c_int
-    lib.fc_set_fused.argtypes = [c_void_p, c_int32, c_int32]
-    lib.fc_set_fused.restype = c_int
-    lib.fc_fused_stats.argtypes = [c_void_p, POINTER(c_uint64)]
-    lib.fc_fused_stats.restype = c_int
     lib.fc_profile_begin.argtypes = [c_void_p, c_int32, c_int32]
     lib.fc_profile_begin.restype = c_int
     lib.fc_profile_stride.argtypes = [c_void_p, c_int32]
@@ -217,21 +213,7 @@ def fc_set_select_overlap(handle, enabled: bool) -> None:
     _check(_lib.fc_set_select_overlap(handle, 1 if enabled else 0), "fc_set_select_overlap")
 
 
-def fc_set_fused(handle, mode, stage_lag: int = 2) -> None:
-    """mode: 0 separate launches, 1 fused kernel with two packed columns per thread, 2 fused kernel
-    with one column per thread."""
-    _check(_lib.fc_set_fused(handle, int(mode), int(stage_lag)), "fc_set_fused")
-
-
-def fc_fused_stats(handle) -> dict:
-    out = (c_uint64 * 12)()
-    _check(_lib.fc_fused_stats(handle, out), "fc_fused_stats")
-    keys = ("tiles", "late_tiles", "unused", "cycles_pass1", "cycles_pass2", "cycles_pass3",
-            "cycles_data_wait", "cycles_loop", "sched_buffer_wait", "sched_dep_wait", "sched_issue", "landing_wait")
-    return {k: int(v) for k, v in zip(keys, out)}
-
-
-KERNEL_CLASSES = {"pass1": 1, "pass2": 2, "pass3": 3, "select": 4, "gather": 5, "other": 6, "fused": 7}
+KERNEL_CLASSES = {"pass1": 1, "pass2": 2, "pass3": 3, "select": 4, "gather": 5, "other": 6}
 
 
 def fc_profile_begin(handle, kernel_class: int, max_launches: int = 16384) -> None:

@@ -1,6 +1,5 @@
 // Handle life cycle, status reporting and the twiddle table of the FlashCache library.
 #include "fc_common.cuh"
-#include "fc_score_fused.cuh"
 
 #include <new>
 #include <stdlib.h>
@@ -64,21 +63,12 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->prof_stride = 1;
   h->prof_seen = 0;
   h->generic_only = false;
-  h->fused_sched = nullptr;
-  h->fused_enabled = 0;   // the separate-launch kernels are still faster; FC_FUSED=1 switches the fused kernel on
-  h->fused_blocks_per_sm = 0;
-  h->fused_lag = 1;
-  h->fused_unit_shift = 20;
-  if (const char *e = getenv("FC_FUSED_UNIT_SHIFT")) { const int v = atoi(e); if (v >= 18 && v <= 23) h->fused_unit_shift = v; }
   h->select_overlap = 0;
   h->score_overlap = 0;
   h->step = 0;
   h->last_sig = -1;
   h->pending_join = false;
   for (int a = 0; a < 2; ++a) for (int b = 0; b < FC_MAX_AUX; ++b) h->ev_done[a][b] = nullptr;
-  if (const char *e = getenv("FC_FUSED_LAG")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_lag = v; }
-  if (const char *e = getenv("FC_FUSED")) { const int v = atoi(e); if (v >= 0 && v <= 2) h->fused_enabled = v; }
-  if (const char *e = getenv("FC_FUSED_BPS")) { const int v = atoi(e); if (v >= 1 && v <= 4) h->fused_blocks_per_sm = v; }
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return FC_ERR_CUDA; }
   h->num_sms = prop.multiProcessorCount;
@@ -93,8 +83,6 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
       cudaMemset(h->status_word, 0, sizeof(int)) != cudaSuccess ||
       cudaMalloc(&h->done_counter, 2 * sizeof(unsigned)) != cudaSuccess ||
       cudaMemset(h->done_counter, 0, 2 * sizeof(unsigned)) != cudaSuccess ||
-      cudaMalloc(&h->fused_sched, sizeof(fused::Sched)) != cudaSuccess ||
-      cudaMemset(h->fused_sched, 0, sizeof(fused::Sched)) != cudaSuccess ||
       cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       !create_streams(h)) {
     fc_destroy(h);
@@ -134,7 +122,7 @@ static void free_prof(fc_handle *h) {
 }
 
 extern "C" fc_status fc_profile_begin(fc_handle *h, int32_t kernel_class, int32_t max_launches) {
-  if (!h || kernel_class < FC_K_PASS1 || kernel_class > FC_K_FUSED || max_launches < 1) return FC_ERR_INVALID_ARG;
+  if (!h || kernel_class < FC_K_PASS1 || kernel_class > FC_K_OTHER || max_launches < 1) return FC_ERR_INVALID_ARG;
   free_prof(h);
   h->prof_events = new (std::nothrow) cudaEvent_t[2 * (size_t)max_launches];
   if (!h->prof_events) return FC_ERR_INTERNAL;
@@ -195,7 +183,6 @@ extern "C" void fc_destroy(fc_handle *h) {
   if (h->master) cudaFree(h->master);
   if (h->status_word) cudaFree(h->status_word);
   if (h->done_counter) cudaFree(h->done_counter);
-  if (h->fused_sched) cudaFree(h->fused_sched);
   delete h;
 }
 
@@ -227,22 +214,7 @@ extern "C" fc_status fc_last_device_status(fc_handle *h, fc_stream stream) {
   return (word & FC_DEV_FLAG_INTERNAL) ? FC_ERR_INTERNAL : FC_ERR_TIMEOUT;
 }
 
-extern "C" fc_status fc_fused_stats(fc_handle *h, uint64_t out[12]) {
-  if (!h || !out || !h->fused_sched) return FC_ERR_INVALID_ARG;
-  FC_CUDA_TRY(cudaDeviceSynchronize());
-  const fused::Sched *sc = static_cast<const fused::Sched *>(h->fused_sched);
-  FC_CUDA_TRY(cudaMemcpy(out, sc->stats, 12 * sizeof(uint64_t), cudaMemcpyDeviceToHost));   // stats and stats2 are adjacent
-  return FC_OK;
-}
-
 extern "C" uint64_t fc_launch_count(const fc_handle *h) { return h ? (uint64_t)h->launches : 0; }
-
-extern "C" fc_status fc_set_fused(fc_handle *h, int32_t enabled, int32_t stage_lag) {
-  if (!h || stage_lag < 1 || stage_lag > 4 || enabled < 0 || enabled > 2) return FC_ERR_INVALID_ARG;
-  h->fused_enabled = enabled;
-  h->fused_lag = stage_lag;
-  return FC_OK;
-}
 
 extern "C" fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled) {
   if (!h) return FC_ERR_INVALID_ARG;

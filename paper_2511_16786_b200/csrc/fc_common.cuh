@@ -51,12 +51,6 @@ struct fc_handle {
   // true only for the stack handle of fc_score_layer_static: every length takes the generic
   // single-stream kernels (no internal streams or events exist there)
   bool generic_only;
-  // scheduler state of the fused persistent kernel (DEVICE, all zero between launches) and knobs
-  void *fused_sched;
-  int fused_enabled;       // 0 separate launches, 1 fused kernel (two packed columns per thread), 2 fused, one column per thread
-  int fused_blocks_per_sm; // 0 = as many as fit
-  int fused_lag;           // stages between pass 1, pass 2 and pass 3 of a unit
-  int fused_unit_shift;    // log2 of (unit columns x N): 20 = 8 MB units (developer knob FC_FUSED_UNIT_SHIFT)
   int select_overlap;      // 1: consecutive fc_select_compact launches may overlap (fc_set_select_overlap)
   // fc_set_score_overlap: consecutive fc_score_layer calls keep running on the two internal streams
   // without rejoining the caller's stream; the join is made by the next call that consumes their results
@@ -81,7 +75,7 @@ struct fc_handle {
 };
 
 // Kernel classes for fc_profile_begin.
-enum { FC_K_NONE = 0, FC_K_PASS1 = 1, FC_K_PASS2 = 2, FC_K_PASS3 = 3, FC_K_SELECT = 4, FC_K_GATHER = 5, FC_K_OTHER = 6, FC_K_FUSED = 7 };
+enum { FC_K_NONE = 0, FC_K_PASS1 = 1, FC_K_PASS2 = 2, FC_K_PASS3 = 3, FC_K_SELECT = 4, FC_K_GATHER = 5, FC_K_OTHER = 6 };
 
 // Brackets one launch with an event pair when its class is being profiled.
 struct ProfScope {

@@ -24,7 +24,6 @@
 // chirp convolution on a power-of-two length M >= 2N-1 with the same three passes.
 #include "fc_common.cuh"
 #include "fc_score_fast.cuh"
-#include "fc_score_fused.cuh"
 
 #include <math.h>
 #include <mutex>
@@ -642,44 +641,6 @@ SeqPlan plan_sequence(int N, bool allow_fast = true) {
   return s;
 }
 
-// Plan of the fused persistent kernel for one power-of-two sequence (see fc_score_fused.cuh).
-struct FusedPlan {
-  bool ok;
-  int r1b, r2b;                 // N1 = 16*r1b, N2 = 16*r2b
-  int UC, U, R, lag, TPU, ncb1, ncb2, nparts;
-  size_t ring_bytes, part_bytes, partial_bytes;
-};
-
-FusedPlan plan_fused(const fc_handle *h, const SeqPlan &sp, int H, int d) {
-  FusedPlan f = {};
-  if (!sp.fast || !h->fused_enabled || sp.N < 4096 || sp.N > 65536) return f;
-  f.r1b = sp.N1 / 16;
-  f.r2b = sp.N2 / 16;
-  const int cpw = fused::NT / f.r1b, cp = fused::NT / (2 * f.r2b);
-  const int min_uc = 2 * cpw > 2 * cp ? 2 * cpw : 2 * cp;
-  int uc = (1 << h->fused_unit_shift) / sp.N;      // 2^20: about 8 MB of intermediate per unit
-  if (uc < min_uc) uc = min_uc;
-  while (uc > min_uc && (uc > d || d % uc != 0)) uc >>= 1;
-  if (uc > d || d % uc != 0 || uc % (2 * cpw) != 0 || uc % (2 * cp) != 0) return f;
-  f.UC = uc;
-  f.U = H * (d / uc);
-  f.nparts = d / (2 * cpw);
-  if (f.U > 1024 || (f.nparts > 1 && (long long)H * sp.N2 > fused::kMaxCnt3)) return f;
-  // pass 3 of unit u-R is handed out in stage u-R+2*lag; pass 1 of unit u rewrites its slot in stage u:
-  // R = 2*lag + 3 puts three stages between them
-  f.lag = h->fused_lag;
-  f.R = 2 * f.lag + 3;
-  if (f.R > f.U) f.R = f.U;
-  f.TPU = (int)((long long)sp.N * uc / 4096);
-  f.ncb1 = uc / (2 * cpw);
-  f.ncb2 = uc / (2 * cp);
-  f.ring_bytes = align_up((size_t)f.R * sp.N * uc * sizeof(float2), 256);
-  f.part_bytes = align_up((size_t)f.U * f.TPU * 2 * sizeof(double), 256);
-  f.partial_bytes = f.nparts > 1 ? align_up((size_t)f.nparts * H * sp.N * sizeof(float), 256) : 0;
-  f.ok = true;
-  return f;
-}
-
 struct ScoreLayout {
   size_t off_ws, off_spec, off_hhat, off_hcol, off_part_tot, off_part_hi, total;
   size_t part_tot_bytes, part_hi_bytes;   // one copy; the specialised path keeps two and alternates (step parity)
@@ -694,21 +655,6 @@ struct ScoreLayout {
 // query takes the maximum over the sequences of the view).
 ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int head_dim) {
   ScoreLayout L;
-  {
-    const FusedPlan f = plan_fused(h, sp, num_heads, head_dim);
-    if (f.ok) {                                      // ring | pass-1 energy sums | pass-3 energy sums | partial scores
-      L = ScoreLayout{};
-      L.off_ws = 0;
-      L.off_part_tot = f.ring_bytes;
-      L.off_part_hi = f.ring_bytes + f.part_bytes;
-      L.off_spec = f.ring_bytes + 2 * f.part_bytes;
-      L.total = f.ring_bytes + 2 * f.part_bytes + f.partial_bytes;
-      L.ws_buf_bytes = f.ring_bytes;
-      L.heads_per_group = num_heads;
-      L.chirp_streams = 1;
-      return L;
-    }
-  }
   const size_t per_head = (size_t)sp.Nfft * head_dim * sizeof(float2);
   int hg = (int)(h->group_bytes / per_head);
   if (hg < 1) hg = 1;
@@ -764,7 +710,7 @@ void claim_persisting_l2(fc_handle *h, const fc_kv_view *kv, cudaStream_t st) {
     const int N = kv->cu_seqlens[b + 1] - kv->cu_seqlens[b];
     if (N == 0) continue;
     const SeqPlan sp = plan_sequence(N);
-    if (!sp.fast || plan_fused(h, sp, kv->num_heads, kv->head_dim).ok) continue;
+    if (!sp.fast) continue;
     claim = window_fits(h, layout_for(h, sp, kv->num_heads, kv->head_dim));
   }
   if (claim == (h->persist_on != 0)) return;
@@ -999,101 +945,6 @@ fc_status launch_chirp(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, cons
   return FC_ERR_INTERNAL;
 }
 
-// cuTensorMapEncodeTiled, looked up through the runtime (no link against the driver library).
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void *p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-fc_status encode_map(CUtensorMap *m, CUtensorMapDataType dt, int rank, const void *base, const cuuint64_t *dims,
-                     const cuuint64_t *strides_b, const cuuint32_t *box) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return FC_ERR_CUDA;
-  const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-  const CUresult r = fn(m, dt, (cuuint32_t)rank, const_cast<void *>(base), dims, strides_b, box, ones,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? FC_OK : FC_ERR_INTERNAL;
-}
-
-// The four tensor maps of one fused launch (see fused::TmaMaps).
-template <typename T>
-fc_status make_tma_maps(const fused::Params &P, int N1, int N2, int cpw, int cp, fused::TmaMaps *M) {
-  const CUtensorMapDataType dt = sizeof(T) == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
-                               : (std::is_same<T, __half>::value ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
-                                                                 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
-  fc_status s;
-  {
-    const cuuint64_t dims[4] = {(cuuint64_t)P.head_dim, (cuuint64_t)P.num_heads, (cuuint64_t)(2 * N2), (cuuint64_t)(N1 / 2)};
-    const cuuint64_t str[3] = {(cuuint64_t)P.stride_head_b, (cuuint64_t)P.stride_token_b,
-                               (cuuint64_t)(2 * N2) * (cuuint64_t)P.stride_token_b};
-    const cuuint32_t box[4] = {(cuuint32_t)(2 * cpw), 1, 1, (cuuint32_t)(N1 / 2)};
-    if ((s = encode_map(&M->k, dt, 4, P.k, dims, str, box)) != FC_OK) return s;
-    if ((s = encode_map(&M->v, dt, 4, P.v, dims, str, box)) != FC_OK) return s;
-  }
-  {
-    const cuuint64_t dims[3] = {(cuuint64_t)(2 * P.UC), (cuuint64_t)N2, (cuuint64_t)P.R * (cuuint64_t)N1};
-    const cuuint64_t str[2] = {(cuuint64_t)P.UC * 8, (cuuint64_t)N2 * (cuuint64_t)P.UC * 8};
-    const cuuint32_t box2[3] = {(cuuint32_t)(4 * cp), (cuuint32_t)N2, 1};
-    const cuuint32_t box3[3] = {(cuuint32_t)(4 * cpw), 1, (cuuint32_t)N1};
-    if ((s = encode_map(&M->ws2, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, P.ws, dims, str, box2)) != FC_OK) return s;
-    if ((s = encode_map(&M->ws3, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, P.ws, dims, str, box3)) != FC_OK) return s;
-  }
-  return FC_OK;
-}
-
-template <typename T, int R1B, int R2B, int ONE>
-fc_status launch_fused_impl(fc_handle *h, cudaStream_t st, const fused::Params &P) {
-  auto kern = fused::k_fused<T, R1B, R2B, ONE>;
-  const size_t sm = fused::Smem<R1B, R2B, ONE>::bytes;
-  constexpr int threads = fused::Threads<ONE>::all;
-  fc_status s = set_smem(kern, sm);
-  if (s != FC_OK) return s;
-  static int blocks_per_sm = 0;                     // per instantiation; the answer does not change
-  if (blocks_per_sm == 0) {
-    int n = 0;
-    FC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, threads, sm));
-    if (n < 1) return FC_ERR_INTERNAL;
-    blocks_per_sm = n;
-  }
-  int bps = blocks_per_sm;
-  if (h->fused_blocks_per_sm > 0 && h->fused_blocks_per_sm < bps) bps = h->fused_blocks_per_sm;
-  unsigned grid = (unsigned)(h->num_sms * bps);
-  if (grid > P.total_tiles) grid = P.total_tiles;
-  fused::TmaMaps M;
-  if ((s = make_tma_maps<T>(P, 16 * R1B, 16 * R2B, fused::NT / R1B, fused::NT / (2 * R2B), &M)) != FC_OK) return s;
-  ProfScope ps(h, FC_K_FUSED, st);
-  kern<<<grid, threads, sm, st>>>(P, M);
-  return fc_after_launch(h);
-}
-
-template <typename T>
-fc_status launch_fused(fc_handle *h, cudaStream_t st, const FusedPlan &f, const fused::Params &P) {
-  if (h->fused_enabled == 2 && f.r1b >= 8) {        // one column per thread (needs N1 >= 128)
-#define FC_FUSED_CASE1(A, B) \
-  if (f.r1b == A && f.r2b == B) return launch_fused_impl<T, A, B, 1>(h, st, P);
-    FC_FUSED_CASE1(8, 8) FC_FUSED_CASE1(8, 16) FC_FUSED_CASE1(16, 16)
-#undef FC_FUSED_CASE1
-  }
-#define FC_FUSED_CASE(A, B) \
-  if (f.r1b == A && f.r2b == B) return launch_fused_impl<T, A, B, 0>(h, st, P);
-  FC_FUSED_CASE(4, 4) FC_FUSED_CASE(4, 8) FC_FUSED_CASE(8, 8) FC_FUSED_CASE(8, 16) FC_FUSED_CASE(16, 16)
-#undef FC_FUSED_CASE
-  return FC_ERR_INTERNAL;
-}
-
 template <typename T>
 fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, int b, double gamma,
                          float *scores, double *energy, char *wsb) {
@@ -1120,7 +971,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   float2 *hcol = reinterpret_cast<float2 *>(wsb + L.off_hcol);
   double *part_tot = reinterpret_cast<double *>(wsb + L.off_part_tot);
   double *part_hi = reinterpret_cast<double *>(wsb + L.off_part_hi);
-  const bool separate_fast = sp.fast && !plan_fused(h, sp, H, d).ok;
+  const bool separate_fast = sp.fast;
   if (separate_fast) {                 // consecutive steps alternate between two copies of the partial sums
     part_tot = reinterpret_cast<double *>(wsb + L.off_part_tot + (h->step & 1u) * L.part_tot_bytes);
     part_hi = reinterpret_cast<double *>(wsb + L.off_part_hi + (h->step & 1u) * L.part_hi_bytes);
@@ -1131,32 +982,6 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   const T *vp = static_cast<const T *>(kv->v) + (long long)start * kv->stride_token;
   const FftPlan p1 = make_plan(sp.N1);
   fc_status s;
-
-  {
-    const FusedPlan f = plan_fused(h, sp, H, d);
-    if (f.ok) {
-      const int es = (int)sizeof(T);
-      fused::Params P = {};
-      P.k = kp; P.v = vp;
-      P.stride_token_b = (long long)kv->stride_token * es;
-      P.stride_head_b = (long long)kv->stride_head * es;
-      P.N = N; P.omega = omega; P.head_dim = d; P.num_heads = H;
-      P.UC = f.UC; P.U = f.U; P.R = f.R; P.lag = f.lag;
-      P.TPU = f.TPU; P.ncb1 = f.ncb1; P.ncb2 = f.ncb2; P.nparts = f.nparts;
-      P.total_tiles = (unsigned)(3ll * f.U * f.TPU);
-      P.ws = ws;
-      P.partial = reinterpret_cast<float *>(spec);
-      P.master = h->master; P.master_len = h->master_len;
-      P.scores = scores + start; P.score_stride = total_tokens;
-      P.inv_scale = (float)(1.0 / ((double)N * (double)N * (double)d));
-      P.part_tot = part_tot; P.part_hi = part_hi;
-      P.energy = energy_b;
-      P.sched = static_cast<fused::Sched *>(h->fused_sched);
-      P.status = h->status_word;
-      P.spin_limit = 1u << 22;
-      return launch_fused<T>(h, st, f, P);
-    }
-  }
 
   if (sp.bluestein) {
     // Spectrum of the chirp kernel.  It depends on the sequence length only, so the handle keeps the last few

@@ -40,15 +40,13 @@ def _rand_kv(T, H, d, dtype, seed, smooth=True):
     return k.to(dtype), v.to(dtype)
 
 
-def _gpu_scores(fc, k, v, cu, gamma, max_seqlen=None, group_bytes=None, fused=None, fused_mode=1):
+def _gpu_scores(fc, k, v, cu, gamma, max_seqlen=None, group_bytes=None):
     T, H, d = k.shape
     seqlens = [cu[i + 1] - cu[i] for i in range(len(cu) - 1)]
     h = fc.fc_create(0, max_seqlen or max(1, max(seqlens, default=1)))
     try:
         if group_bytes:
             fc.fc_set_group_bytes(h, group_bytes)
-        if fused is not None:
-            fc.fc_set_fused(h, fused_mode, fused)
         kd, vd = (k if k.is_cuda else k.cuda()), (v if v.is_cuda else v.cuda())
         scores = torch.full((H, max(T, 1)), -1.0, dtype=torch.float32, device="cuda")
         energy = torch.full((len(cu) - 1, 4), -1.0, dtype=torch.float64, device="cuda")
@@ -239,27 +237,6 @@ def test_power_spectrum_matches_oracle(fc, lens, H, d, dtype):
         om = O.cutoff_index(n, 0.2)
         np.testing.assert_allclose(got[s + om + 1:e, 0].sum(), en[b, 0], rtol=2e-3, atol=1e-6 * en[b, 1])
         np.testing.assert_allclose(got[s + om + 1:e, 1].sum(), en[b, 2], rtol=2e-3, atol=1e-6 * en[b, 3])
-
-
-@pytest.mark.parametrize("mode", [1, 2])
-@pytest.mark.parametrize("lag", [1, 2, 3])
-@pytest.mark.parametrize("N,H,dtype", [(4096, 3, torch.float32), (8192, 2, torch.bfloat16), (16384, 1, torch.float16),
-                                       (32768, 2, torch.bfloat16), (65536, 1, torch.bfloat16)])
-def test_scores_fused_persistent_kernel(fc, N, H, dtype, lag, mode):
-    # the one-launch persistent form of the three passes, every supported length and stage distance,
-    # with two packed columns per thread (1) and with one column per thread (2)
-    k, v = _rand_kv(N, H, 128, dtype, N + lag)
-    g, en = _check_layer(fc, k, v, [0, N], 0.2, fused=lag, fused_mode=mode)
-    g2, en2 = _gpu_scores(fc, k, v, [0, N], 0.2, fused=lag, fused_mode=mode)
-    assert np.array_equal(g, g2) and np.array_equal(en, en2)          # deterministic
-
-
-def test_scores_fused_ragged_batch(fc):
-    lens = [4096, 300, 8192, 0, 1024, 4096]
-    cu = [0] + [int(x) for x in np.cumsum(lens)]
-    k, v = _rand_kv(cu[-1], 4, 128, torch.bfloat16, 21)
-    _check_layer(fc, k, v, cu, 0.2, max_seqlen=8192, fused=2)
-    _check_layer(fc, k, v, cu, 0.2, max_seqlen=8192, fused=2, fused_mode=2)
 
 
 # ---------------------------------------------------------------- budgets
