@@ -282,6 +282,41 @@ fc_status fc_select_compact_ex(fc_handle *h, const fc_kv_view *kv, const float *
                                void *workspace, size_t workspace_bytes, fc_stream stream);
 
 /*
+ * fc_select_compact_ex for several layers in ONE launch (Sec. 3.2.1, last sentence; same selection, same
+ * results bit for bit).  After fc_allocate_budgets every layer's scores, budgets and offsets are known, and
+ * one layer's selection fills only a fraction of the GPU (8 blocks per sequence and head), so the layers
+ * are best selected side by side.
+ *
+ *   shape        the layout all layers share: strides, dtype, num_heads, head_dim, batch, cu_seqlens
+ *                (its k and v are not read)
+ *   layers       HOST array [num_layers] of per-layer DEVICE pointers and the rows available in that
+ *                layer's outputs (copied into the launch arguments; free to reuse on return)
+ *   budgets      DEVICE int32[num_layers][B], out_offsets DEVICE int64[num_layers][B+1]: the arrays
+ *                fc_allocate_budgets wrote (row l belongs to layers[l])
+ *   opt          as fc_select_compact_ex (NULL: defaults); the protect mask is shared by all layers
+ * Layers are launched 32 at a time.  Errors: as fc_select_compact_ex.
+ */
+typedef struct {
+  const void *k, *v;           /* DEVICE: the layer's K and V                      */
+  const float *scores;         /* DEVICE float[num_heads][T] from fc_score_layer   */
+  void *out_k, *out_v;         /* DEVICE [out_capacity_rows][h][c]                 */
+  int32_t *out_idx;            /* DEVICE int32[num_heads][out_capacity_rows]       */
+  int64_t out_capacity_rows;
+} fc_layer_buffers;
+
+fc_status fc_select_compact_layers(fc_handle *h, const fc_kv_view *shape, const fc_layer_buffers *layers,
+                                   int32_t num_layers, const int32_t *budgets, const int64_t *out_offsets,
+                                   const fc_select_options *opt, void *workspace, size_t workspace_bytes,
+                                   fc_stream stream);
+
+/* Rows one layer's compacted cache can receive at most: the sum over sequences of
+ * min(N_b, B_tot(b)), B_tot = clamp(floor(rho*N*L + 1/2), L*lo, L*N) (Sec. 3.2.2; the total the
+ * budgets of a sequence add up to).  Sizes out_k / out_v / out_idx before the budgets are known.
+ * -1 on bad input. */
+int64_t fc_layer_capacity_rows(int32_t num_layers, int32_t batch, const int32_t *cu_seqlens,
+                               double rho, int32_t min_keep);
+
+/*
  * fc_score_layer without any allocation (the paper has no counterpart: this is a
  * packaging variant of the same computation, added for integration reasons).
  *

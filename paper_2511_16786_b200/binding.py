@@ -26,6 +26,7 @@ EXPORTS = (
     "fc_set_group_bytes", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
+    "fc_select_compact_layers", "fc_layer_capacity_rows",
     "fc_power_spectrum_workspace_bytes", "fc_power_spectrum",
     "fc_decode_workspace_bytes", "fc_decode_attention",
     "fc_static_scratch_bytes", "fc_score_layer_static",
@@ -44,6 +45,11 @@ class fc_kv_view(ctypes.Structure):
 
 class fc_select_options(ctypes.Structure):
     _fields_ = [("per_layer", c_int32), ("protect", c_void_p)]
+
+
+class fc_layer_buffers(ctypes.Structure):
+    _fields_ = [("k", c_void_p), ("v", c_void_p), ("scores", c_void_p), ("out_k", c_void_p), ("out_v", c_void_p),
+                ("out_idx", c_void_p), ("out_capacity_rows", c_int64)]
 
 
 class fc_decode_args(ctypes.Structure):
@@ -125,6 +131,12 @@ def _load() -> ctypes.CDLL:
                                          c_void_p, c_void_p, c_void_p, c_int64, POINTER(fc_select_options),
                                          c_void_p, c_size_t, c_void_p]
     lib.fc_select_compact_ex.restype = c_int
+    lib.fc_select_compact_layers.argtypes = [c_void_p, POINTER(fc_kv_view), POINTER(fc_layer_buffers), c_int32,
+                                             c_void_p, c_void_p, POINTER(fc_select_options), c_void_p, c_size_t,
+                                             c_void_p]
+    lib.fc_select_compact_layers.restype = c_int
+    lib.fc_layer_capacity_rows.argtypes = [c_int32, c_int32, POINTER(c_int32), c_double, c_int32]
+    lib.fc_layer_capacity_rows.restype = c_int64
     lib.fc_power_spectrum_workspace_bytes.argtypes = [c_void_p, POINTER(fc_kv_view)]
     lib.fc_power_spectrum_workspace_bytes.restype = c_size_t
     lib.fc_power_spectrum.argtypes = [c_void_p, POINTER(fc_kv_view), c_void_p, c_void_p, c_size_t, c_void_p]
@@ -370,6 +382,36 @@ def fc_select_compact_ex(handle, k, v, cu_seqlens, scores, budgets, out_offsets,
            "fc_select_compact_ex")
 
 
+def fc_layer_capacity_rows(num_layers: int, cu_seqlens, rho: float, min_keep: int = 1) -> int:
+    """Rows one layer's compacted cache can receive at most (sizes out_k / out_v / out_idx)."""
+    cu = _cu_array(cu_seqlens)
+    r = int(_lib.fc_layer_capacity_rows(int(num_layers), len(cu) - 1, ctypes.cast(cu, POINTER(c_int32)),
+                                        float(rho), int(min_keep)))
+    if r < 0:
+        raise FlashCacheError(1, "fc_layer_capacity_rows")
+    return r
+
+
+def fc_select_compact_layers(handle, K_layers, V_layers, cu_seqlens, scores, budgets, out_offsets, out_k, out_v,
+                             out_idx, workspace, per_layer: bool = False, protect=None) -> None:
+    """All layers in one launch.  scores [L, H, T]; budgets [L, B]; out_offsets [L, B+1];
+    out_k / out_v [L, capacity, H, d]; out_idx [L, H, capacity]."""
+    L = len(K_layers)
+    cu = _cu_array(cu_seqlens)
+    view = make_view(K_layers[0], V_layers[0], cu)
+    cap = int(out_k.shape[1])
+    tab = (fc_layer_buffers * L)()
+    for l in range(L):
+        tab[l] = fc_layer_buffers(K_layers[l].data_ptr(), V_layers[l].data_ptr(), scores[l].data_ptr(),
+                                  out_k[l].data_ptr(), out_v[l].data_ptr(), out_idx[l].data_ptr(), cap)
+    opt = fc_select_options(per_layer=1 if per_layer else 0,
+                            protect=protect.data_ptr() if protect is not None else None)
+    _check(_lib.fc_select_compact_layers(handle, byref(view), tab, L, c_void_p(budgets.data_ptr()),
+                                         c_void_p(out_offsets.data_ptr()), byref(opt), c_void_p(workspace.data_ptr()),
+                                         workspace.numel() * workspace.element_size(), _stream()),
+           "fc_select_compact_layers")
+
+
 # ----------------------------------------------------------------------------
 # convenience: buffers for a whole model and the three-phase pass
 # ----------------------------------------------------------------------------
@@ -407,14 +449,8 @@ class Compressor:
         self.energy = torch.empty((self.L, self.B, 4), dtype=torch.float64, device=dev)
         self.budgets = torch.empty((self.L, self.B), dtype=torch.int32, device=dev)
         self.offsets = torch.empty((self.L, self.B + 1), dtype=torch.int64, device=dev)
-        # rows any one layer can receive: every sequence is capped at its own length and at its total
-        import math
-        self.capacity = 0
-        for n in seqlens:
-            lo = min(self.min_keep, n)
-            tot = max(self.L * lo, min(self.L * n, int(math.floor(self.rho * n * self.L + 0.5))))
-            self.capacity += min(n, tot)
-        self.capacity = max(self.capacity, 1)
+        # rows any one layer can receive (the library's own bound)
+        self.capacity = max(fc_layer_capacity_rows(self.L, self.cu, self.rho, self.min_keep), 1)
         self.out_k = None
         self.out_v = None
         self.out_idx = None
@@ -470,6 +506,12 @@ class Compressor:
             out_v=[P(self.out_v[l].data_ptr()) for l in range(self.L)],
             out_idx=[P(self.out_idx[l].data_ptr()) for l in range(self.L)],
             cap=int(self.out_k.shape[1]))
+        tab = (fc_layer_buffers * self.L)()
+        for l in range(self.L):
+            tab[l] = fc_layer_buffers(K_layers[l].data_ptr(), V_layers[l].data_ptr(), self.scores[l].data_ptr(),
+                                      self.out_k[l].data_ptr(), self.out_v[l].data_ptr(),
+                                      self.out_idx[l].data_ptr(), m["cap"])
+        m["layers"] = tab
         self._m, self._mkey, self._m_out = m, key, (id(self.out_k), id(self._ws))
         return m
 
@@ -486,10 +528,17 @@ class Compressor:
         fc_allocate_budgets(self.handle, self.energy, self.cu, self.rho, self.min_keep,
                             self.budgets, self.offsets)
 
-    def select_compact(self, K_layers, V_layers):
+    def select_compact(self, K_layers, V_layers, one_launch: bool = True):
         m = self._marshal(K_layers, V_layers)
         st, h = _stream(), self.handle
-        call, opt = _lib.fc_select_compact_ex, byref(self._opt)
+        opt = byref(self._opt)
+        if one_launch:         # every layer side by side (fc_select_compact_layers)
+            rc = _lib.fc_select_compact_layers(h, m["refs"][0], m["layers"], self.L, c_void_p(self.budgets.data_ptr()),
+                                               c_void_p(self.offsets.data_ptr()), opt, m["ws"], m["ws_bytes"], st)
+            if rc != FC_OK:
+                raise FlashCacheError(rc, "fc_select_compact_layers")
+            return
+        call = _lib.fc_select_compact_ex
         for l in range(self.L):
             rc = call(h, m["refs"][l], m["scores"][l], m["budgets"][l], m["offsets"][l], m["out_k"][l],
                       m["out_v"][l], m["out_idx"][l], m["cap"], opt, m["ws"], m["ws_bytes"], st)

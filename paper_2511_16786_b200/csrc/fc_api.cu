@@ -179,6 +179,7 @@ extern "C" void fc_destroy(fc_handle *h) {
   for (int i = 0; i < h->host_ev_cap; ++i) cudaEventDestroy(h->host_ev[i]);
   delete[] h->host_ev;
   if (h->ev_inputs_free) cudaEventDestroy(h->ev_inputs_free);
+  if (h->ev_outputs_done) cudaEventDestroy(h->ev_outputs_done);
   if (h->hhat_cache) cudaFree(h->hhat_cache);
   if (h->master) cudaFree(h->master);
   if (h->status_word) cudaFree(h->status_word);

@@ -71,6 +71,7 @@ struct fc_handle {
   cudaEvent_t *host_ev;
   int host_ev_cap;
   cudaEvent_t ev_inputs_free;
+  cudaEvent_t ev_outputs_done;      // the previous fc_compress_host job has copied its rows back to the host
   const void *host_last_arena;
 };
 

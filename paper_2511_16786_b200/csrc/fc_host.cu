@@ -4,7 +4,7 @@
 //   copy stream :  H2D K_0 V_0 | H2D K_1 V_1 | ...                    (one event per layer)
 //   caller's    :  wait ev_0, score 0 | wait ev_1, score 1 | ... | allocate | D2H budgets
 //                  -- host waits here once, learns the rows of every layer --
-//                  select 0 .. select L-1 | (inputs free) | D2H K rows, V rows, indices
+//                  select (all layers, one launch) | (inputs free) | D2H K rows, V rows, indices | (outputs done)
 //
 // The next job on the same arena starts its H2D copies at "inputs free", so they run while the
 // previous job's rows travel back: both directions of the link are busy in steady state.
@@ -85,6 +85,7 @@ Arena carve(const fc_handle *h, const fc_host_job *j) {
 fc_status ensure_pipeline(fc_handle *h, int L) {
   if (!h->host_copy) FC_CUDA_TRY(cudaStreamCreateWithFlags(&h->host_copy, cudaStreamNonBlocking));
   if (!h->ev_inputs_free) FC_CUDA_TRY(cudaEventCreateWithFlags(&h->ev_inputs_free, cudaEventDisableTiming));
+  if (!h->ev_outputs_done) FC_CUDA_TRY(cudaEventCreateWithFlags(&h->ev_outputs_done, cudaEventDisableTiming));
   if (h->host_ev_cap < L) {
     cudaEvent_t *ev = new (std::nothrow) cudaEvent_t[L];
     if (!ev) return FC_ERR_INTERNAL;
@@ -174,7 +175,8 @@ extern "C" fc_status fc_compress_host(fc_handle *h, const fc_host_job *job, fc_s
   const size_t in_bytes = (size_t)a.T * a.row_bytes;
 
   // the copies may start once whatever read or wrote this arena before is through with it
-  if (h->host_last_arena == job->arena) {
+  const bool same_arena = (h->host_last_arena == job->arena);
+  if (same_arena) {
     FC_CUDA_TRY(cudaStreamWaitEvent(h->host_copy, h->ev_inputs_free, 0));
   } else {
     FC_CUDA_TRY(cudaEventRecord(h->ev_inputs_free, st));
@@ -222,14 +224,25 @@ extern "C" fc_status fc_compress_host(fc_handle *h, const fc_host_job *job, fc_s
 
   char *ok = base + a.off_out_k, *ov = base + a.off_out_v;
   int32_t *oi = reinterpret_cast<int32_t *>(base + a.off_out_idx);
-  for (int l = 0; l < L; ++l) {
-    const int64_t r0 = job->layer_rows_host[l], r = job->layer_rows_host[l + 1] - r0;
-    if (r == 0) continue;
-    const fc_kv_view kv = view_of(job, base + a.off_k + (size_t)l * a.layer_in_bytes,
-                                  base + a.off_v + (size_t)l * a.layer_in_bytes);
-    s = fc_select_compact_ex(h, &kv, scores + (size_t)l * H * a.T, budgets + (size_t)l * B,
-                             offsets + (size_t)l * (B + 1), ok + (size_t)r0 * a.row_bytes, ov + (size_t)r0 * a.row_bytes,
-                             oi + (size_t)r0 * H, r, &opt, ws, a.ws_bytes, st);
+  // the previous job on this arena may still be copying its rows back (possibly on another stream)
+  if (same_arena) FC_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_outputs_done, 0));
+  {
+    // every layer in one launch (a layer without rows keeps its entry: its budgets are zero, nothing is written)
+    fc_layer_buffers *lb = new (std::nothrow) fc_layer_buffers[L];
+    if (!lb) return FC_ERR_INTERNAL;
+    for (int l = 0; l < L; ++l) {
+      const int64_t r0 = job->layer_rows_host[l], r = job->layer_rows_host[l + 1] - r0;
+      lb[l].k = base + a.off_k + (size_t)l * a.layer_in_bytes;
+      lb[l].v = base + a.off_v + (size_t)l * a.layer_in_bytes;
+      lb[l].scores = scores + (size_t)l * H * a.T;
+      lb[l].out_k = ok + (size_t)r0 * a.row_bytes;
+      lb[l].out_v = ov + (size_t)r0 * a.row_bytes;
+      lb[l].out_idx = oi + (size_t)r0 * H;
+      lb[l].out_capacity_rows = r;
+    }
+    const fc_kv_view shape = view_of(job, nullptr, nullptr);
+    s = fc_select_compact_layers(h, &shape, lb, L, budgets, offsets, &opt, ws, a.ws_bytes, st);
+    delete[] lb;
     if (s != FC_OK) return s;
   }
   FC_CUDA_TRY(cudaEventRecord(h->ev_inputs_free, st));
@@ -239,5 +252,6 @@ extern "C" fc_status fc_compress_host(fc_handle *h, const fc_host_job *job, fc_s
     FC_CUDA_TRY(cudaMemcpyAsync(job->out_v_host, ov, (size_t)rows * a.row_bytes, cudaMemcpyDeviceToHost, st));
     FC_CUDA_TRY(cudaMemcpyAsync(job->out_idx_host, oi, (size_t)rows * H * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
   }
+  FC_CUDA_TRY(cudaEventRecord(h->ev_outputs_done, st));
   return FC_OK;
 }

@@ -17,6 +17,14 @@ constexpr int kSeqChunk = 64;          // sequences described per launch (kernel
 struct SeqTable {
   int start[kSeqChunk + 1];            // token offsets of the chunk's sequences (cu_seqlens slice)
 };
+constexpr int kLayerChunk = 32;        // layers selected by one launch (kernel-argument table)
+struct LayerTable {                    // per layer of the chunk: where its scores, rows and outputs live (DEVICE pointers)
+  const float *scores[kLayerChunk];
+  const char *k[kLayerChunk], *v[kLayerChunk];
+  char *out_k[kLayerChunk], *out_v[kLayerChunk];
+  int *out_idx[kLayerChunk];
+  long long cap[kLayerChunk];          // rows available in the layer's outputs
+};
 
 // ---------------------------------------------------------------------------
 // budgets
@@ -375,21 +383,23 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
   }
 }
 
-// The kernel.  overlap != 0 (launched with the programmatic-serialisation attribute): the next
-// launch in the stream may start as soon as every block of this one has begun, and this grid
-// does not finish before its predecessor has, so "the last launch is complete" still means
-// "all of them are".
+// The kernel: grid (kSelCluster * sequences in chunk, heads or 1, layers in chunk); blockIdx.z picks the
+// layer's pointers from the table and the layer's rows of budgets [L][B] and out_offsets [L][B+1].
+// overlap != 0 (launched with the programmatic-serialisation attribute): the next launch in the stream
+// may start as soon as every block of this one has begun, and this grid does not finish before its
+// predecessor has, so "the last launch is complete" still means "all of them are".
 template <int kSelKpt, bool PER_LAYER>
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
-k_select_gather(const float *__restrict__ scores, long long T, const __grid_constant__ SeqTable st, int b0,
+k_select_gather(const __grid_constant__ LayerTable lt, long long T, const __grid_constant__ SeqTable st, int b0, int B,
                 const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
-                int *__restrict__ out_idx, long long cap, int *__restrict__ status,
-                const char *__restrict__ kin, const char *__restrict__ vin, long long stride_token_b,
-                long long stride_head_b, int row_bytes, int H, char *__restrict__ out_k,
-                char *__restrict__ out_v, int overlap, const unsigned char *__restrict__ protect) {
+                int *__restrict__ status, long long stride_token_b,
+                long long stride_head_b, int row_bytes, int H, int overlap,
+                const unsigned char *__restrict__ protect) {
   if (overlap) asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
-  select_gather_body<kSelKpt, PER_LAYER>(scores, T, st, b0, budgets, out_offsets, out_idx, cap, status, kin, vin,
-                                         stride_token_b, stride_head_b, row_bytes, H, out_k, out_v, protect);
+  const int z = blockIdx.z;
+  select_gather_body<kSelKpt, PER_LAYER>(lt.scores[z], T, st, b0, budgets + (size_t)z * B,
+                                         out_offsets + (size_t)z * (B + 1), lt.out_idx[z], lt.cap[z], status, lt.k[z], lt.v[z],
+                                         stride_token_b, stride_head_b, row_bytes, H, lt.out_k[z], lt.out_v[z], protect);
   if (overlap) asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
 
@@ -444,16 +454,12 @@ extern "C" fc_status fc_select_compact(fc_handle *h, const fc_kv_view *kv, const
                               nullptr, workspace, workspace_bytes, stream);
 }
 
-extern "C" fc_status fc_select_compact_ex(fc_handle *h, const fc_kv_view *kv, const float *scores,
-                                          const int32_t *budgets, const int64_t *out_offsets,
-                                          void *out_k, void *out_v, int32_t *out_idx,
-                                          int64_t out_capacity_rows, const fc_select_options *opt,
-                                          void *workspace, size_t workspace_bytes, fc_stream stream) {
-  const bool per_layer = opt && opt->per_layer != 0;
-  const unsigned char *protect = opt ? static_cast<const unsigned char *>(opt->protect) : nullptr;
-  if (!h || !kv || !kv->k || !kv->v || !scores || !budgets || !out_offsets || !out_k || !out_v || !out_idx)
-    return FC_ERR_INVALID_ARG;
-  if (kv->num_heads <= 0 || kv->head_dim <= 0 || out_capacity_rows < 0) return FC_ERR_INVALID_ARG;
+namespace {
+
+// Argument checks shared by the selection entry points (everything but the per-layer pointers).
+fc_status check_select_shape(const fc_handle *h, const fc_kv_view *kv, const void *workspace, size_t workspace_bytes) {
+  if (!h || !kv) return FC_ERR_INVALID_ARG;
+  if (kv->num_heads <= 0 || kv->head_dim <= 0) return FC_ERR_INVALID_ARG;
   if (kv->dtype != FC_F32 && kv->dtype != FC_F16 && kv->dtype != FC_BF16) return FC_ERR_UNSUPPORTED;
   const int es = kv->dtype == FC_F32 ? 4 : 2;
   if ((kv->head_dim * es) % 16) return FC_ERR_UNSUPPORTED;
@@ -461,17 +467,20 @@ extern "C" fc_status fc_select_compact_ex(fc_handle *h, const fc_kv_view *kv, co
   if (s != FC_OK) return s;
   for (int b = 0; b < kv->batch; ++b)
     if (kv->cu_seqlens[b + 1] - kv->cu_seqlens[b] > kSelCluster * kSelThreads * kSelKptMax) return FC_ERR_UNSUPPORTED;
-  if (((uintptr_t)kv->k & 15) || ((uintptr_t)kv->v & 15) || ((uintptr_t)out_k & 15) || ((uintptr_t)out_v & 15))
-    return FC_ERR_INVALID_ARG;
   if ((kv->stride_token * es) % 16 || (kv->stride_head * es) % 16) return FC_ERR_INVALID_ARG;
   if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < fc_select_workspace_bytes(h, kv))
     return FC_ERR_WORKSPACE;
-  int dev = -1;
-  FC_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if ((s = fc_flush_pending(h, st)) != FC_OK) return s;
+  return FC_OK;
+}
+
+// Launches the selection for `nl` (<= kLayerChunk) layers whose pointers are in `lt`; budgets and
+// out_offsets point at the first of these layers' rows.
+fc_status launch_select(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const LayerTable &lt, int nl,
+                        const int32_t *budgets, const int64_t *out_offsets, bool per_layer,
+                        const unsigned char *protect) {
+  const int es = kv->dtype == FC_F32 ? 4 : 2;
   const long long T = kv->cu_seqlens[kv->batch];
+  fc_status s;
   for (int b0 = 0; b0 < kv->batch; b0 += kSeqChunk) {
     const int nseq = kv->batch - b0 < kSeqChunk ? kv->batch - b0 : kSeqChunk;
     SeqTable tab;
@@ -484,7 +493,7 @@ extern "C" fc_status fc_select_compact_ex(fc_handle *h, const fc_kv_view *kv, co
 #define FC_SEL_LAUNCH(KPT, PL)                                                                          \
   do {                                                                                                  \
     cudaLaunchConfig_t lc = {};                                                                         \
-    lc.gridDim = dim3(kSelCluster * nseq, (PL) ? 1 : kv->num_heads);                                    \
+    lc.gridDim = dim3(kSelCluster * nseq, (PL) ? 1 : kv->num_heads, nl);                                \
     lc.blockDim = dim3(kSelThreads);                                                                    \
     lc.stream = st;                                                                                     \
     cudaLaunchAttribute at[1];                                                                          \
@@ -492,12 +501,10 @@ extern "C" fc_status fc_select_compact_ex(fc_handle *h, const fc_kv_view *kv, co
     at[0].val.programmaticStreamSerializationAllowed = 1;                                               \
     lc.attrs = at;                                                                                      \
     lc.numAttrs = h->select_overlap ? 1 : 0;                                                            \
-    launch_err = cudaLaunchKernelEx(&lc, k_select_gather<KPT, PL>, scores, (long long)T, tab, b0, budgets, \
-        reinterpret_cast<const long long *>(out_offsets), out_idx, (long long)out_capacity_rows,        \
-        h->status_word, static_cast<const char *>(kv->k), static_cast<const char *>(kv->v),             \
-        (long long)(kv->stride_token * es), (long long)(kv->stride_head * es), (int)(kv->head_dim * es), \
-        (int)kv->num_heads, static_cast<char *>(out_k), static_cast<char *>(out_v),                     \
-        (int)h->select_overlap, protect);                                                               \
+    launch_err = cudaLaunchKernelEx(&lc, k_select_gather<KPT, PL>, lt, (long long)T, tab, b0, (int)kv->batch, \
+        budgets, reinterpret_cast<const long long *>(out_offsets),                                      \
+        h->status_word, (long long)(kv->stride_token * es), (long long)(kv->stride_head * es),          \
+        (int)(kv->head_dim * es), (int)kv->num_heads, (int)h->select_overlap, protect);                 \
   } while (0)
       cudaError_t launch_err = cudaSuccess;
       if (per_layer) {
@@ -517,4 +524,92 @@ extern "C" fc_status fc_select_compact_ex(fc_handle *h, const fc_kv_view *kv, co
     if ((s = fc_after_launch(h)) != FC_OK) return s;
   }
   return FC_OK;
+}
+
+}  // namespace
+
+extern "C" fc_status fc_select_compact_ex(fc_handle *h, const fc_kv_view *kv, const float *scores,
+                                          const int32_t *budgets, const int64_t *out_offsets,
+                                          void *out_k, void *out_v, int32_t *out_idx,
+                                          int64_t out_capacity_rows, const fc_select_options *opt,
+                                          void *workspace, size_t workspace_bytes, fc_stream stream) {
+  if (!h || !kv || !kv->k || !kv->v || !scores || !budgets || !out_offsets || !out_k || !out_v || !out_idx)
+    return FC_ERR_INVALID_ARG;
+  if (out_capacity_rows < 0) return FC_ERR_INVALID_ARG;
+  fc_status s = check_select_shape(h, kv, workspace, workspace_bytes);
+  if (s != FC_OK) return s;
+  if (((uintptr_t)kv->k & 15) || ((uintptr_t)kv->v & 15) || ((uintptr_t)out_k & 15) || ((uintptr_t)out_v & 15))
+    return FC_ERR_INVALID_ARG;
+  int dev = -1;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if ((s = fc_flush_pending(h, st)) != FC_OK) return s;
+  LayerTable lt = {};
+  lt.scores[0] = scores;
+  lt.k[0] = static_cast<const char *>(kv->k);
+  lt.v[0] = static_cast<const char *>(kv->v);
+  lt.out_k[0] = static_cast<char *>(out_k);
+  lt.out_v[0] = static_cast<char *>(out_v);
+  lt.out_idx[0] = out_idx;
+  lt.cap[0] = out_capacity_rows;
+  return launch_select(h, st, kv, lt, 1, budgets, out_offsets, opt && opt->per_layer != 0,
+                       opt ? static_cast<const unsigned char *>(opt->protect) : nullptr);
+}
+
+extern "C" fc_status fc_select_compact_layers(fc_handle *h, const fc_kv_view *shape, const fc_layer_buffers *layers,
+                                              int32_t num_layers, const int32_t *budgets, const int64_t *out_offsets,
+                                              const fc_select_options *opt,
+                                              void *workspace, size_t workspace_bytes, fc_stream stream) {
+  if (!h || !shape || !layers || !budgets || !out_offsets || num_layers < 1) return FC_ERR_INVALID_ARG;
+  fc_status s = check_select_shape(h, shape, workspace, workspace_bytes);
+  if (s != FC_OK) return s;
+  for (int l = 0; l < num_layers; ++l) {
+    const fc_layer_buffers &b = layers[l];
+    if (!b.k || !b.v || !b.scores || !b.out_k || !b.out_v || !b.out_idx || b.out_capacity_rows < 0) return FC_ERR_INVALID_ARG;
+    if (((uintptr_t)b.k & 15) || ((uintptr_t)b.v & 15) || ((uintptr_t)b.out_k & 15) || ((uintptr_t)b.out_v & 15))
+      return FC_ERR_INVALID_ARG;
+  }
+  int dev = -1;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if ((s = fc_flush_pending(h, st)) != FC_OK) return s;
+  const int B = shape->batch;
+  for (int l0 = 0; l0 < num_layers; l0 += kLayerChunk) {
+    const int nl = num_layers - l0 < kLayerChunk ? num_layers - l0 : kLayerChunk;
+    LayerTable lt = {};
+    for (int i = 0; i < nl; ++i) {
+      const fc_layer_buffers &b = layers[l0 + i];
+      lt.scores[i] = b.scores;
+      lt.k[i] = static_cast<const char *>(b.k);
+      lt.v[i] = static_cast<const char *>(b.v);
+      lt.out_k[i] = static_cast<char *>(b.out_k);
+      lt.out_v[i] = static_cast<char *>(b.out_v);
+      lt.out_idx[i] = b.out_idx;
+      lt.cap[i] = b.out_capacity_rows;
+    }
+    s = launch_select(h, st, shape, lt, nl, budgets + (size_t)l0 * B, out_offsets + (size_t)l0 * (B + 1),
+                      opt && opt->per_layer != 0,
+                      opt ? static_cast<const unsigned char *>(opt->protect) : nullptr);
+    if (s != FC_OK) return s;
+  }
+  return FC_OK;
+}
+
+extern "C" int64_t fc_layer_capacity_rows(int32_t num_layers, int32_t batch, const int32_t *cu_seqlens,
+                                          double rho, int32_t min_keep) {
+  if (num_layers < 1 || batch < 0 || !cu_seqlens || min_keep < 0 || !(rho >= 0.0) || isinf(rho)) return -1;
+  if (check_cu(cu_seqlens, batch) != FC_OK) return -1;
+  long long rows = 0;
+  for (int b = 0; b < batch; ++b) {
+    const long long N = cu_seqlens[b + 1] - cu_seqlens[b];
+    if (N == 0) continue;
+    const double lo = (double)(min_keep < N ? min_keep : N), hi = (double)N, L = (double)num_layers;
+    double bt = floor(rho * (double)N * L + 0.5);        // B_tot of the sequence, as k_allocate computes it
+    if (bt < L * lo) bt = L * lo;
+    if (bt > L * hi) bt = L * hi;
+    rows += bt < hi ? (long long)bt : N;                  // one layer gets at most N and at most B_tot
+  }
+  return rows;
 }

@@ -533,6 +533,32 @@ def test_overlapping_launches_give_the_same_results(fc):
                                y.view(torch.uint8) if y.dtype != torch.int32 else y)
 
 
+@pytest.mark.parametrize("per_layer", [False, True])
+def test_one_selection_launch_for_all_layers_is_bit_identical(fc, per_layer):
+    # fc_select_compact_layers against one fc_select_compact_ex call per layer: same indices, same rows; more layers
+    # than one launch takes (32) so the chunking is exercised, ragged batch with an empty sequence
+    from paper_2511_16786_b200.binding import Compressor
+    cfg = S.scaled(S.paper_configs()["cfg2"], "cfg2_layers", num_layers=35, seqlens=(1000, 0, 2048, 517))
+    Kd, Vd = zip(*(S.make_layer(cfg, l, "cuda") for l in range(cfg.num_layers)))
+    comp = Compressor(cfg.num_layers, cfg.num_heads, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho,
+                      cfg.gamma, cfg.min_keep, per_layer=per_layer)
+    comp.score(Kd, Vd)
+    comp.allocate()
+    res = []
+    for one_launch in (False, True):
+        comp.out_k.fill_(0)
+        comp.out_v.fill_(0)
+        comp.out_idx.fill_(-1)
+        comp.select_compact(Kd, Vd, one_launch=one_launch)
+        comp.check_device_status()
+        res.append((comp.out_k.cpu().view(torch.uint8).clone(), comp.out_v.cpu().view(torch.uint8).clone(),
+                    comp.out_idx.cpu().clone()))
+    assert int(comp.offsets[:, -1].sum()) > 0
+    for a, b in zip(res[0], res[1]):
+        assert torch.equal(a, b)
+    comp.close()
+
+
 # ---------------------------------------------------------------- full-size shapes, sampled
 def test_head_sharded_pass_equals_the_whole_pass(fc):
     # two shards of the KV heads, run one after the other on this GPU, with the energy sums added by hand
