@@ -12,13 +12,36 @@
  *
  * Conventions
  *   - Every pointer is marked HOST or DEVICE.  The caller owns every buffer;
- *     the library allocates device memory only in fc_create and never frees or
- *     writes caller inputs.
- *   - All work is enqueued on the caller's stream (a cudaStream_t passed as
- *     void*); no entry point except fc_last_device_status synchronises.
- *   - Argument errors are found on the host before anything is launched and
- *     are returned as fc_status; nothing traps or aborts.
- *   - One handle serves one stream at a time.
+ *     the library allocates device memory only in fc_create (and, for its host
+ *     pipeline, two streams and a few events on the first fc_compress_host call)
+ *     and never frees or writes caller inputs.
+ *   - Streams.  `stream` is a cudaStream_t passed as void*.  Results are ordered
+ *     on it: work enqueued on `stream` after a call sees that call's outputs.
+ *     fc_score_layer runs power-of-two sequences of 1024..65536 tokens and long
+ *     sequences of other lengths on the handle's internal streams (two by
+ *     default), which wait for everything enqueued on `stream` before the call
+ *     and which `stream` waits for before the call returns, through events; no
+ *     host synchronisation is involved (see fc_set_score_overlap for the
+ *     variant that defers the second wait).  Nothing uses the default stream.
+ *   - Calls that block the host: fc_create and fc_destroy (device
+ *     synchronisation), fc_last_device_status and fc_static_last_device_status
+ *     (they synchronise `stream`), fc_profile_end (waits for its events),
+ *     fc_compress_host (once, to learn the row counts), the first
+ *     fc_score_layer_static call on a device.  Every other call only enqueues.
+ *   - Context-wide state.  While a handle scores power-of-two sequences it
+ *     raises the context's persisting-L2 limit (cudaLimitPersistingL2CacheSize)
+ *     to the device maximum and marks its transform workspace as a persisting
+ *     access window on its internal streams; the handles of a device share the
+ *     claim and the last one to let go restores the value found.  No persisting
+ *     line of anyone else is reset.  fc_set_l2_persist(h, 0) opts a handle out.
+ *   - Errors.  Argument errors are found on the host before anything is
+ *     launched and are returned as fc_status; nothing traps or aborts.  Device-
+ *     side problems (capacity overflow, a bounded wait that ran out) set a bit
+ *     in the handle's status word, read with fc_last_device_status.  After each
+ *     launch the library takes the runtime's pending error (cudaGetLastError):
+ *     a non-sticky error left pending by the caller's own earlier CUDA calls is
+ *     therefore reported as FC_ERR_CUDA by, and cleared by, the next launch.
+ *   - One handle serves one host thread and one stream at a time.
  *   - KV layout: element [t][h][c] at  base + t*stride_token + h*stride_head + c
  *     (strides in elements, channel stride 1).  The sequences of a batch are
  *     packed along t; sequence b owns tokens [cu_seqlens[b], cu_seqlens[b+1]).
@@ -41,7 +64,7 @@ typedef enum {
   FC_ERR_UNSUPPORTED = 2,   /* dtype / head_dim / sequence length outside what was built */
   FC_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or smaller than the query says */
   FC_ERR_CUDA = 4,          /* a CUDA runtime call failed */
-  FC_ERR_TIMEOUT = 5,       /* reserved: a bounded device-side wait ran out */
+  FC_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out (set in the status word by the decoding kernel) */
   FC_ERR_INTERNAL = 6       /* a device-side self check failed (see fc_last_device_status) */
 } fc_status;
 
@@ -79,6 +102,12 @@ const char *fc_status_string(fc_status s);
  * the handle's device status word since the last call (and clears it). */
 fc_status fc_last_device_status(fc_handle *h, fc_stream stream);
 
+/* Self test of the failure path of the bounded device-side waits (diagnostic; the paper has no
+ * counterpart): enqueues one small kernel that waits, at most 1000 tries, on a barrier nothing will ever
+ * complete, gives up, and records it.  The next fc_last_device_status returns FC_ERR_TIMEOUT; the
+ * context stays usable (nothing traps, nothing spins without a limit). */
+fc_status fc_selftest_bounded_wait(fc_handle *h, fc_stream stream);
+
 /* Number of kernels this handle has launched since fc_create (diagnostic). */
 uint64_t fc_launch_count(const fc_handle *h);
 
@@ -114,6 +143,15 @@ fc_status fc_set_score_overlap(fc_handle *h, int32_t enabled);
  * call waits for the one before it. */
 fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled);
 
+/* Number of internal streams fc_score_layer spreads the head groups of a sequence over (1..4,
+ * default 2, the measured best: two transforms in flight fill the GPU, three no longer fit the L2).
+ * Call it between passes, not while deferred work is pending (fc_set_score_overlap).  Speed only. */
+fc_status fc_set_internal_streams(fc_handle *h, int32_t count);
+
+/* enabled = 0: this handle never touches the context's persisting-L2 limit nor sets access windows
+ * (see Conventions); costs a few percent on long power-of-two sequences.  Default 1. */
+fc_status fc_set_l2_persist(fc_handle *h, int32_t enabled);
+
 /* Forgets the ordering state the handle keeps between calls (which of its internal events the next
  * call would wait on).  Call it right before cudaStreamBeginCapture and right after
  * cudaStreamEndCapture when a sequence of calls on this handle is captured into a CUDA graph: an
@@ -144,6 +182,11 @@ size_t fc_select_workspace_bytes(const fc_handle *h, const fc_kv_view *kv);
  * (Eq. 9), and every token is scored by
  *     Dev[x] = mean_c (K[x,c]-K_base[x,c])^2 + mean_c (V[x,c]-V_base[x,c])^2   (Eq. 10).
  * Arithmetic is fp32 on the stored values.
+ * Values that are not finite: the transform of a channel mixes all tokens of its sequence, so one NaN
+ * or Inf element of K or V makes every score of that (sequence, head) NaN and that sequence's energy
+ * sums NaN, exactly as the definition does; other heads' scores and other sequences are unaffected.
+ * fc_allocate_budgets then treats the sequence's weights as uniform and fc_select_compact ranks NaN as
+ * +inf, ties by token index: the affected head keeps its first tokens.
  *
  *   gamma      cutoff factor, 0 <= gamma <= 1.
  *   scores     DEVICE float[num_heads][T], T = cu_seqlens[B]; written for every token.
@@ -358,6 +401,9 @@ int64_t fc_layer_capacity_rows(int32_t num_layers, int32_t batch, const int32_t 
 size_t fc_static_scratch_bytes(void);
 fc_status fc_score_layer_static(const fc_kv_view *kv, double gamma, float *scores,
                                 double *energy, fc_stream stream);
+/* fc_last_device_status for the calls above (they have no handle): synchronises `stream`, returns and
+ * clears what the kernels of fc_score_layer_static recorded in the status word of the current device. */
+fc_status fc_static_last_device_status(fc_stream stream);
 
 /*
  * The whole compressor for one prefill, from HOST memory to HOST memory (Sec. 3.2, Fig. 2):

@@ -22,14 +22,14 @@ FC_F32, FC_F16, FC_BF16 = 0, 1, 2
 _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
-    "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count",
-    "fc_set_group_bytes", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
+    "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count", "fc_selftest_bounded_wait",
+    "fc_set_group_bytes", "fc_set_internal_streams", "fc_set_l2_persist", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
     "fc_select_compact_layers", "fc_layer_capacity_rows",
     "fc_power_spectrum_workspace_bytes", "fc_power_spectrum",
     "fc_decode_workspace_bytes", "fc_decode_attention",
-    "fc_static_scratch_bytes", "fc_score_layer_static",
+    "fc_static_scratch_bytes", "fc_score_layer_static", "fc_static_last_device_status",
     "fc_compress_host_rows", "fc_compress_host_arena_bytes", "fc_compress_host",
 )
 
@@ -102,6 +102,14 @@ def _load() -> ctypes.CDLL:
     lib.fc_set_group_bytes.restype = c_int
     lib.fc_reset_ordering.argtypes = [c_void_p]
     lib.fc_reset_ordering.restype = c_int
+    lib.fc_selftest_bounded_wait.argtypes = [c_void_p, c_void_p]
+    lib.fc_selftest_bounded_wait.restype = c_int
+    lib.fc_set_internal_streams.argtypes = [c_void_p, c_int32]
+    lib.fc_set_internal_streams.restype = c_int
+    lib.fc_set_l2_persist.argtypes = [c_void_p, c_int32]
+    lib.fc_set_l2_persist.restype = c_int
+    lib.fc_static_last_device_status.argtypes = [c_void_p]
+    lib.fc_static_last_device_status.restype = c_int
     lib.fc_set_score_overlap.argtypes = [c_void_p, c_int32]
     lib.fc_set_score_overlap.restype = c_int
     lib.fc_set_select_overlap.argtypes = [c_void_p, c_int32]
@@ -217,6 +225,18 @@ def fc_set_group_bytes(handle, nbytes: int) -> None:
     _check(_lib.fc_set_group_bytes(handle, int(nbytes)), "fc_set_group_bytes")
 
 
+def fc_selftest_bounded_wait(handle) -> None:
+    _check(_lib.fc_selftest_bounded_wait(handle, _stream()), "fc_selftest_bounded_wait")
+
+
+def fc_set_internal_streams(handle, count: int) -> None:
+    _check(_lib.fc_set_internal_streams(handle, int(count)), "fc_set_internal_streams")
+
+
+def fc_set_l2_persist(handle, enabled: bool) -> None:
+    _check(_lib.fc_set_l2_persist(handle, 1 if enabled else 0), "fc_set_l2_persist")
+
+
 def fc_set_score_overlap(handle, enabled: bool) -> None:
     _check(_lib.fc_set_score_overlap(handle, 1 if enabled else 0), "fc_set_score_overlap")
 
@@ -282,6 +302,11 @@ def fc_score_layer_static(k, v, cu_seqlens, gamma: float, scores, energy) -> Non
     view = make_view(k, v, cu)
     _check(_lib.fc_score_layer_static(byref(view), float(gamma), c_void_p(scores.data_ptr()),
                                       c_void_p(energy.data_ptr()), _stream()), "fc_score_layer_static")
+
+
+def fc_static_last_device_status() -> int:
+    """Synchronises the current stream; status recorded by fc_score_layer_static calls on this device."""
+    return int(_lib.fc_static_last_device_status(_stream()))
 
 
 def fc_compress_host_rows(num_layers: int, cu_seqlens, rho: float, min_keep: int) -> int:

@@ -1,6 +1,7 @@
 // Handle life cycle, status reporting and the twiddle table of the FlashCache library.
 #include "fc_common.cuh"
 
+#include <mutex>
 #include <new>
 #include <stdlib.h>
 
@@ -15,7 +16,73 @@ __global__ void k_fill_master(float2 *master, int len) {
   master[i] = make_float2((float)c, (float)s);
 }
 
+// Self test of the failure path every bounded device-side wait takes: one block waits on a shared-memory
+// barrier that nothing ever arrives on, gives up after `limit` tries, records the timeout in the status
+// word and returns normally.
+__global__ void k_selftest_bounded_wait(int *status, unsigned limit) {
+  __shared__ unsigned long long bar;
+  const unsigned addr = (unsigned)__cvta_generic_to_shared(&bar);
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(addr) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncthreads();
+  bool done = false;
+  for (unsigned it = 0; it < limit && !done; ++it) {
+    unsigned ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], 0;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(addr) : "memory");
+    done = ok != 0;
+  }
+  if (!done && threadIdx.x == 0) atomicOr(status, FC_DEV_FLAG_TIMEOUT);
+}
+
 }  // namespace
+
+// The persisting part of L2 is a setting of the whole context.  The handles of a device share one claim:
+// the first handle that needs it raises the limit (never lowers what the application had set), the last one
+// to let go puts the application's value back.  Lines are never reset: only the handle's own stream windows
+// are cleared, so another user of persisting L2 in the process keeps what it has.
+namespace {
+constexpr int kMaxPersistDevices = 64;
+std::mutex g_persist_mutex;
+int g_persist_claims[kMaxPersistDevices];
+size_t g_persist_prev[kMaxPersistDevices];
+}  // namespace
+
+bool fc_persist_acquire(fc_handle *h) {
+  if (h->persist_on) return true;
+  if (h->device < 0 || h->device >= kMaxPersistDevices) return false;
+  std::lock_guard<std::mutex> lock(g_persist_mutex);
+  if (g_persist_claims[h->device] == 0) {
+    size_t prev = 0;
+    if (cudaDeviceGetLimit(&prev, cudaLimitPersistingL2CacheSize) != cudaSuccess) { cudaGetLastError(); return false; }
+    if (prev < h->persist_max &&
+        cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, h->persist_max) != cudaSuccess) { cudaGetLastError(); return false; }
+    g_persist_prev[h->device] = prev;
+  }
+  g_persist_claims[h->device]++;
+  h->persist_on = 1;
+  return true;
+}
+
+void fc_persist_release(fc_handle *h) {
+  if (!h->persist_on) return;
+  for (int i = 0; i < FC_MAX_AUX; ++i) {
+    if (h->aux[i] && h->window_base[i]) {
+      cudaStreamAttrValue av = {};
+      av.accessPolicyWindow.num_bytes = 0;
+      if (cudaStreamSetAttribute(h->aux[i], cudaStreamAttributeAccessPolicyWindow, &av) != cudaSuccess) cudaGetLastError();
+    }
+    h->window_base[i] = nullptr;
+    h->window_bytes[i] = 0;
+  }
+  h->persist_on = 0;
+  if (h->device < 0 || h->device >= kMaxPersistDevices) return;
+  std::lock_guard<std::mutex> lock(g_persist_mutex);
+  if (--g_persist_claims[h->device] == 0 && g_persist_prev[h->device] < h->persist_max)
+    if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, g_persist_prev[h->device]) != cudaSuccess) cudaGetLastError();
+}
 
 static bool create_streams(fc_handle *h) {
   for (int i = 0; i < FC_MAX_AUX; ++i) {
@@ -46,14 +113,10 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->status_word = nullptr;
   h->done_counter = nullptr;
   h->group_bytes = (size_t)32 << 20;
-  // Developer tuning knobs (tile widths in channel pairs); the defaults are the measured best.
-  h->tune_cpw = 32;
+  h->tune_cpw = 32;        // tile widths of the specialised kernels in channel pairs (the measured best)
   h->tune_cp = 8;
-  if (const char *e = getenv("FC_TUNE_CPW")) { const int v = atoi(e); if (v == 16 || v == 32) h->tune_cpw = v; }
-  if (const char *e = getenv("FC_TUNE_CP")) { const int v = atoi(e); if (v == 4 || v == 8) h->tune_cp = v; }
   h->launches = 0;
   h->num_aux = 2;
-  if (const char *e = getenv("FC_NUM_AUX")) { const int v = atoi(e); if (v >= 1 && v <= FC_MAX_AUX) h->num_aux = v; }
   h->ev_fork = nullptr;
   for (int i = 0; i < FC_MAX_AUX; ++i) { h->aux[i] = nullptr; h->ev_join[i] = nullptr; }
   h->prof_class = FC_K_NONE;
@@ -73,7 +136,6 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return FC_ERR_CUDA; }
   h->num_sms = prop.multiProcessorCount;
   h->l2_persist = 1;
-  if (const char *e = getenv("FC_L2_PERSIST")) h->l2_persist = atoi(e) != 0 ? 1 : 0;
   h->persist_max = (size_t)prop.persistingL2CacheMaxSize;
   h->window_max = (size_t)prop.accessPolicyMaxWindowSize;
   for (int i = 0; i < FC_MAX_AUX; ++i) { h->window_base[i] = nullptr; h->window_bytes[i] = 0; }
@@ -167,7 +229,7 @@ extern "C" fc_status fc_profile_end(fc_handle *h, double *total_ms, uint64_t *la
 extern "C" void fc_destroy(fc_handle *h) {
   if (!h) return;
   free_prof(h);
-  if (h->persist_on) { cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, 0); cudaCtxResetPersistingL2Cache(); }
+  fc_persist_release(h);
   for (int i = 0; i < FC_MAX_AUX; ++i) {
     if (h->aux[i]) cudaStreamSynchronize(h->aux[i]);
     for (int a = 0; a < 2; ++a) if (h->ev_done[a][i]) cudaEventDestroy(h->ev_done[a][i]);
@@ -215,6 +277,12 @@ extern "C" fc_status fc_last_device_status(fc_handle *h, fc_stream stream) {
   return (word & FC_DEV_FLAG_INTERNAL) ? FC_ERR_INTERNAL : FC_ERR_TIMEOUT;
 }
 
+extern "C" fc_status fc_selftest_bounded_wait(fc_handle *h, fc_stream stream) {
+  if (!h) return FC_ERR_INVALID_ARG;
+  k_selftest_bounded_wait<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(h->status_word, 1000u);
+  return fc_after_launch(h);
+}
+
 extern "C" uint64_t fc_launch_count(const fc_handle *h) { return h ? (uint64_t)h->launches : 0; }
 
 extern "C" fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled) {
@@ -226,6 +294,21 @@ extern "C" fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled) {
 extern "C" fc_status fc_set_score_overlap(fc_handle *h, int32_t enabled) {
   if (!h) return FC_ERR_INVALID_ARG;
   h->score_overlap = enabled ? 1 : 0;
+  return FC_OK;
+}
+
+extern "C" fc_status fc_set_internal_streams(fc_handle *h, int32_t count) {
+  if (!h || count < 1 || count > FC_MAX_AUX) return FC_ERR_INVALID_ARG;
+  if (h->pending_join) return FC_ERR_INVALID_ARG;        // work of an earlier call is still on the internal streams
+  fc_persist_release(h);                                 // the windows belong to the old set of streams
+  h->num_aux = count;
+  return FC_OK;
+}
+
+extern "C" fc_status fc_set_l2_persist(fc_handle *h, int32_t enabled) {
+  if (!h) return FC_ERR_INVALID_ARG;
+  h->l2_persist = enabled ? 1 : 0;
+  if (!enabled) fc_persist_release(h);
   return FC_OK;
 }
 

@@ -31,7 +31,7 @@ struct fc_handle {
   int tune_cpw, tune_cp;   // tile widths of the specialised kernels (channel pairs), see fc_create
   int num_sms;
   // L2 residency of the transform intermediates: the per-stream workspace buffers are declared a
-  // persisting access window on the internal streams (0 switches it off, FC_L2_PERSIST)
+  // persisting access window on the internal streams (0 switches it off, fc_set_l2_persist)
   int l2_persist;
   int persist_on;                      // the context's persisting-L2 set-aside is currently claimed by this handle
   size_t persist_max, window_max;      // device limits (bytes)
@@ -41,7 +41,7 @@ struct fc_handle {
   // internal streams: consecutive head groups of one fc_score_layer call are transformed
   // concurrently, round robin over the streams, each with its own workspace buffer
   cudaStream_t aux[FC_MAX_AUX];
-  int num_aux;             // how many of them are used (2 by default, FC_NUM_AUX)
+  int num_aux;             // how many of them are used (2 by default, fc_set_internal_streams)
   cudaEvent_t ev_fork, ev_join[FC_MAX_AUX];
   // optional per-kernel-class timing (fc_profile_begin / fc_profile_end)
   int prof_class;
@@ -341,7 +341,13 @@ inline fc_status fc_flush_pending(fc_handle *h, cudaStream_t st) {
   return FC_OK;
 }
 
+// After every launch: takes (and so clears) the runtime's pending error, so a failed launch is reported by
+// the call that made it and does not linger for the caller's next CUDA call.
 inline fc_status fc_after_launch(fc_handle *h) {
   h->launches++;
-  return cudaPeekAtLastError() == cudaSuccess ? FC_OK : FC_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? FC_OK : FC_ERR_CUDA;
 }
+
+// Shared claim on the context's persisting-L2 limit (fc_api.cu).
+bool fc_persist_acquire(fc_handle *h);
+void fc_persist_release(fc_handle *h);

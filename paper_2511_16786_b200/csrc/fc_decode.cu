@@ -254,6 +254,15 @@ k_decode_partial(const DecodeParams P, const __grid_constant__ DecodeMaps M) {
         oacc[j][0] *= corr[0]; oacc[j][1] *= corr[0];
         oacc[j][2] *= corr[1]; oacc[j][3] *= corr[1];
       }
+      // rows at or past `valid` (another sequence's rows, or memory nobody wrote) have probability 0, but
+      // 0 x NaN is NaN: their value rows are cleared before the product.  k0 = first of the two rows a
+      // fragment register holds (low half k0, high half k0 + 1).
+      const int rem = valid - wrow;
+      unsigned vm0 = 0xffffffffu, vm1 = 0xffffffffu;
+      if (rem < 16) {
+        vm0 = (2 * t < rem ? 0x0000ffffu : 0u) | (2 * t + 1 < rem ? 0xffff0000u : 0u);
+        vm1 = (2 * t + 8 < rem ? 0x0000ffffu : 0u) | (2 * t + 9 < rem ? 0xffff0000u : 0u);
+      }
       unsigned pa[4];
       pa[0] = Mma<T>::pack(sacc[0][0], sacc[0][1]);
       pa[1] = Mma<T>::pack(sacc[0][2], sacc[0][3]);
@@ -263,6 +272,8 @@ k_decode_partial(const DecodeParams P, const __grid_constant__ DecodeMaps M) {
       for (int jj = 0; jj < kD / 16; ++jj) {
         unsigned r[4];
         ldmatrix_x4_trans(sb + 2 * kBoxBytes + tile_offset(wrow + (mi & 1) * 8 + (lane & 7), 2 * jj + (mi >> 1)), r);
+        r[0] &= vm0; r[2] &= vm0;
+        r[1] &= vm1; r[3] &= vm1;
         Mma<T>::run(oacc[2 * jj], pa, r[0], r[1]);
         Mma<T>::run(oacc[2 * jj + 1], pa, r[2], r[3]);
       }

@@ -28,6 +28,7 @@
 #include <math.h>
 #include <mutex>
 #include <type_traits>
+#include <unordered_map>
 
 namespace {
 
@@ -699,10 +700,10 @@ bool window_fits(const fc_handle *h, const ScoreLayout &L) {
   return h->l2_persist && L.ws_buf_bytes <= h->window_max && L.ws_buf_bytes * (size_t)h->num_aux <= h->persist_max;
 }
 
-// The persisting part of L2 is a set-aside of this process's context (gone with it): claimed while calls
-// contain a sequence for the specialised path, given back to ordinary caching when a call has none (the
-// generic kernels lose about a tenth of their speed to a set-aside they do not use).  Decided once per call;
-// left as it is while `st` is being captured into a graph, where device-wide settings cannot change.
+// The persisting part of L2 is a limit of the whole context, shared by the handles of a device (fc_persist_acquire):
+// held while calls contain a sequence for the specialised path, let go when a call has none (the generic kernels
+// lose about a tenth of their speed to a set-aside they do not use).  Decided once per call; left as it is while
+// `st` is being captured into a graph, where device-wide settings cannot change.
 void claim_persisting_l2(fc_handle *h, const fc_kv_view *kv, cudaStream_t st) {
   if (!h->l2_persist || h->generic_only) return;
   bool claim = false;
@@ -717,13 +718,11 @@ void claim_persisting_l2(fc_handle *h, const fc_kv_view *kv, cudaStream_t st) {
   cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) { cudaGetLastError(); return; }
   if (cap != cudaStreamCaptureStatusNone) return;
-  if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, claim ? h->persist_max : 0) != cudaSuccess) {
-    cudaGetLastError();
-    h->l2_persist = 0;
-    return;
+  if (claim) {
+    if (!fc_persist_acquire(h)) h->l2_persist = 0;      // not available here: never try again
+  } else {
+    fc_persist_release(h);
   }
-  h->persist_on = claim ? 1 : 0;
-  if (!claim) cudaCtxResetPersistingL2Cache();
 }
 
 fc_status validate_view(const fc_handle *h, const fc_kv_view *kv) {
@@ -746,11 +745,24 @@ fc_status validate_view(const fc_handle *h, const fc_kv_view *kv) {
   return FC_OK;
 }
 
+// Function attributes are set once per kernel and device (and again only if a launch needs more shared
+// memory than the last time), not before every launch.
 template <class Kern>
 fc_status set_smem(Kern kern, size_t bytes) {
+  static std::mutex mu;
+  static std::unordered_map<unsigned long long, size_t> done;     // (device, kernel) -> bytes already allowed
+  int dev = 0;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  const unsigned long long key = (unsigned long long)reinterpret_cast<uintptr_t>(reinterpret_cast<const void *>(kern)) ^
+                                 ((unsigned long long)dev << 56);
+  std::lock_guard<std::mutex> lock(mu);
+  auto it = done.find(key);
+  if (it != done.end() && it->second >= bytes) return FC_OK;
   if (bytes > 48 * 1024) FC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
   // as much of the L1/shared array as shared memory as the device offers: these kernels do not rely on L1
-  FC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+  if (it == done.end())
+    FC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+  done[key] = bytes;
   return FC_OK;
 }
 
@@ -849,7 +861,7 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
   if (h->tune_cpw == W && h->tune_cp == C)                                                              \
     return launch_fast_tuned<T, W, C>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores,       \
                                       total_tokens, part_tot, part_hi, energy_b);
-  FC_TUNE_CASE(32, 8) FC_TUNE_CASE(32, 4) FC_TUNE_CASE(16, 8) FC_TUNE_CASE(16, 4)
+  FC_TUNE_CASE(32, 8)
 #undef FC_TUNE_CASE
   return FC_ERR_INTERNAL;
 }
@@ -1366,6 +1378,7 @@ struct StaticSetup {
   float2 *master;
   int *status;
   unsigned *counter;
+  int num_sms;
 };
 constexpr int kMaxDevices = 64;
 StaticSetup g_setup[kMaxDevices];
@@ -1388,6 +1401,7 @@ fc_status static_setup(int dev, StaticSetup *out) {
     s.master = static_cast<float2 *>(p_master);
     s.status = static_cast<int *>(p_status);
     s.counter = static_cast<unsigned *>(p_counter);
+    FC_CUDA_TRY(cudaDeviceGetAttribute(&s.num_sms, cudaDevAttrMultiProcessorCount, dev));
     s.ready = true;
   }
   *out = s;
@@ -1421,9 +1435,7 @@ extern "C" fc_status fc_score_layer_static(const fc_kv_view *kv, double gamma, f
   hs.tune_cp = 8;
   hs.prof_class = FC_K_NONE;
   hs.generic_only = true;
-  cudaDeviceProp prop;
-  FC_CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
-  hs.num_sms = prop.multiProcessorCount;
+  hs.num_sms = su.num_sms;
   s = validate_view(&hs, kv);         // lengths above kStaticMaxSeqlen come back as FC_ERR_UNSUPPORTED
   if (s != FC_OK) return s;
   const size_t need = fc_score_workspace_bytes(&hs, kv);
@@ -1438,4 +1450,19 @@ extern "C" fc_status fc_score_layer_static(const fc_kv_view *kv, double gamma, f
     }
   }
   return s;
+}
+
+extern "C" fc_status fc_static_last_device_status(fc_stream stream) {
+  int dev = -1;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  StaticSetup su;
+  fc_status s = static_setup(dev, &su);
+  if (s != FC_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  FC_CUDA_TRY(cudaStreamSynchronize(st));
+  int word = 0;
+  FC_CUDA_TRY(cudaMemcpy(&word, su.status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (word != 0) FC_CUDA_TRY(cudaMemset(su.status, 0, sizeof(int)));
+  if (word == 0) return FC_OK;
+  return (word & FC_DEV_FLAG_INTERNAL) ? FC_ERR_INTERNAL : FC_ERR_TIMEOUT;
 }

@@ -94,6 +94,38 @@ def test_decode_with_uncompressed_tail_and_peaked_scores(fc):
     _check(got2, want)
 
 
+def test_decode_ignores_what_lies_past_the_valid_rows(fc):
+    # rows after a sequence's last kept row (the next sequence's rows, rows after offsets[B]) and tail rows at or past
+    # tail_len may hold anything, NaN and Inf bit patterns included: they have no weight and must not reach the output
+    lens = [70, 1, 130]
+    tail_len = [5, 0, 33]
+    offsets = [0] + [int(x) for x in np.cumsum(lens)]
+    B, H, G, d = 3, 2, 4, 128
+    for dtype in (torch.bfloat16, torch.float16):
+        q, ck, cv = _inputs(offsets[-1] + 100, B, H, G, dtype, 77)
+        g = torch.Generator().manual_seed(78)
+        tk = torch.randn((B, 64, H, d), generator=g).to(dtype)
+        tv = torch.randn((B, 64, H, d), generator=g).to(dtype)
+        want = O.decode_attention(q.double().numpy(), ck.double().numpy(), cv.double().numpy(), offsets,
+                                  tk.double().numpy(), tv.double().numpy(), tail_len)
+        poison = torch.tensor([float("nan"), float("inf"), -float("inf"), 1e30], dtype=torch.float32).to(dtype)
+        ck[offsets[-1]:] = poison[0]
+        cv[offsets[-1]:] = poison[torch.arange(cv[offsets[-1]:].numel()) % 4].view_as(cv[offsets[-1]:])
+        for b in range(B):
+            tk[b, tail_len[b]:] = poison[1]
+            tv[b, tail_len[b]:] = poison[torch.arange(tv[b, tail_len[b]:].numel()) % 4].view_as(tv[b, tail_len[b]:])
+        got = _run(fc, q, ck, cv, offsets, tail=(tk, tv, tail_len))
+        assert np.isfinite(got).all()
+        _check(got, want)
+    # the last sequence's neighbour inside the cache: sequence 0's last tile also holds rows of sequence 1 and 2;
+    # make those non-finite for a run that only looks at sequence 0
+    q, ck, cv = _inputs(200, 1, 1, 2, torch.bfloat16, 79)
+    want = O.decode_attention(q.double().numpy(), ck[:70].double().numpy(), cv[:70].double().numpy(), [0, 70])
+    ck[70:] = float("nan")
+    cv[70:] = float("inf")
+    _check(_run(fc, q, ck, cv, [0, 70]), want)
+
+
 def test_decode_closed_forms_on_the_device(fc):
     # zero query: the mean of the value rows; one row: that row
     g = torch.Generator().manual_seed(9)

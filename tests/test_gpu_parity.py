@@ -717,18 +717,68 @@ def test_config2_full_size_sampled(fc):
 
 
 def test_config3_full_size_sampled(fc):
+    # every head of four layers against the oracle, the any-size properties on all 28
     cfg = S.paper_configs()["cfg3"]
-    _compare_sampled(fc, cfg, [(0, 0, 1), (27, 0, 3)])
+    _compare_sampled(fc, cfg, [(l, 0, h) for l in (0, 9, 18, 27) for h in range(4)])
 
 
-def test_config4_shape_full_length_sampled(fc):
-    cfg = S.scaled(S.paper_configs()["cfg4"], "cfg4", num_layers=3)       # 32 heads x 16384 tokens, 3 of the 32 layers
-    _compare_sampled(fc, cfg, [(0, 0, 0), (2, 0, 31)])
+def test_config4_full_size_sampled(fc):
+    # all 32 layers x 32 heads x 16384 tokens on the device; eight (layer, head) pairs against the oracle
+    cfg = S.paper_configs()["cfg4"]
+    _compare_sampled(fc, cfg, [(0, 0, 0), (3, 0, 17), (8, 0, 31), (13, 0, 5), (19, 0, 22), (24, 0, 9), (28, 0, 30),
+                               (31, 0, 12)])
 
 
-def test_config5_full_lengths_sampled(fc):
-    cfg = S.scaled(S.paper_configs()["cfg5"], "cfg5", num_layers=2)       # the 8 ragged lengths, 2 of the 28 layers
-    _compare_sampled(fc, cfg, [(0, 6, 0), (1, 7, 3), (1, 3, 2)])
+def test_config5_full_size_sampled(fc):
+    # all 28 layers of the eight ragged sequences; the longest and the shortest sequence are among the samples
+    cfg = S.paper_configs()["cfg5"]
+    lens = list(cfg.seqlens)
+    longest, shortest = lens.index(max(lens)), lens.index(min(lens))
+    _compare_sampled(fc, cfg, [(0, longest, 0), (27, shortest, 3), (5, 0, 1), (11, 1, 2), (14, 2, 0), (17, 3, 3),
+                               (21, 4, 1), (25, 5, 2), (9, 6, 0), (2, 7, 3)])
+
+
+# ---------------------------------------------------------------- failure reporting
+def test_bounded_wait_that_runs_out_is_reported(fc):
+    # a wait nothing will ever satisfy gives up after its limit, the status word says so, and the handle and the
+    # context go on working (no trap, no hang)
+    h = fc.fc_create(0, 1024)
+    try:
+        assert fc.fc_last_device_status(h) == 0
+        fc.fc_selftest_bounded_wait(h)
+        assert fc.fc_last_device_status(h) == 5                     # FC_ERR_TIMEOUT
+        assert fc.fc_last_device_status(h) == 0                     # reading clears it
+    finally:
+        fc.fc_destroy(h)
+    k, v = _rand_kv(1024, 1, 128, torch.float32, 3)
+    _check_layer(fc, k, v, [0, 1024], 0.2)
+
+
+@pytest.mark.parametrize("N", [1024, 300])
+def test_nonfinite_input_poisons_its_own_sequence_and_head_only(fc, N):
+    # a NaN or Inf element makes every score of its (sequence, head) NaN, as in the fp64 definition (the transform
+    # mixes all tokens of a column); other heads and other sequences are untouched; the selection then keeps the
+    # first tokens by index for that head (NaN ranks as +inf, ties by index)
+    k, v = _rand_kv(2 * N, 3, 128, torch.float32, 91)
+    cu = [0, N, 2 * N]
+    kc, vc = k.clone(), v.clone()
+    k[N // 3, 1, 7] = float("nan")              # sequence 0, head 1
+    v[N + 5, 2, 100] = float("inf")             # sequence 1, head 2
+    g, en = _gpu_scores(fc, k, v, cu, 0.2)
+    o, _ = O.score_layer(kc.double().numpy(), vc.double().numpy(), cu, 0.2, "fft")
+    assert np.isnan(g[1, :N]).all() and np.isnan(g[2, N:]).all()
+    ok = np.ones_like(g, dtype=bool)
+    ok[1, :N] = False
+    ok[2, N:] = False
+    assert np.isfinite(g[ok]).all()
+    np.testing.assert_allclose(g[ok], o[ok], rtol=2e-3, atol=1e-6 * o.mean())
+    # the oracle agrees on which scores are lost
+    on, _ = O.score_layer(k.double().numpy(), v.double().numpy(), cu, 0.2, "fft")
+    assert np.array_equal(np.isnan(on), ~ok)
+    scores = torch.from_numpy(g.astype(np.float32))
+    got = _gpu_select(fc, k, v, cu, scores, [5, 7], [0, 5, 12], 12)[2]
+    np.testing.assert_array_equal(got[1, 0:5], np.arange(5))
+    np.testing.assert_array_equal(got[2, 5:12], np.arange(7))
 
 
 # ---------------------------------------------------------------- ABI error paths (host-side checks only)

@@ -6,7 +6,7 @@ every call shares that array and finds the previous call's leftovers in it.
 
 The test calls it through the C ABI twice in a row on different inputs and checks each
 result against fc_score_layer (the entry point with a caller-provided workspace) within
-the score tolerances of the parity tests.  It is collected last so that a failure here
+the score tolerances of the parity tests; a further test holds it to the fp64 oracle directly.  It is collected last so that a failure here
 cannot hide another test's result in a run that stops at the first failure, and it makes
 no assumption about what ran before it in the process.
 """
@@ -88,6 +88,30 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(fc):
     _compare(fc, [4096, 777], 2, 128, torch.float32, 2)
     # and once more with the first shape: results do not depend on what the scratch held
     _compare(fc, [300, 0, 1024, 17, 2048], 3, 128, torch.bfloat16, 1)
+
+
+def test_static_entry_point_matches_the_oracle(fc):
+    # the same check the workspace entry point gets: element by element against the fp64 oracle on a small ragged
+    # batch (chirp path, empty sequence, power of two), and the status word of the static calls reads clean
+    from oracle import flashcache_oracle as O
+    for dtype, seed in ((torch.float32, 11), (torch.bfloat16, 12)):
+        k, v, cu = _inputs([257, 0, 512, 33], 2, 128, dtype, seed)
+        got, got_e = _static(fc, k, v, cu, 0.2)
+        assert fc.fc_static_last_device_status() == 0
+        kk, vv = k.double().cpu().numpy(), v.double().cpu().numpy()
+        want, want_e = O.score_layer(kk, vv, cu, 0.2, "fft")
+        tol = TOL[dtype]
+        for b in range(len(cu) - 1):
+            s0, e0 = cu[b], cu[b + 1]
+            if e0 == s0:
+                continue
+            for h in range(2):
+                ebar = ((kk[s0:e0, h] ** 2).sum(1) + (vv[s0:e0, h] ** 2).sum(1)).mean() / 128
+                den = np.maximum(want[h, s0:e0], 1e-6 * ebar)
+                err = float((np.abs(got[h, s0:e0] - want[h, s0:e0]) / den).max())
+                assert err <= tol, "sequence %d head %d: score error %.3e" % (b, h, err)
+            np.testing.assert_allclose(got_e[b, [1, 3]], want_e[b, [1, 3]], rtol=1e-5)
+            np.testing.assert_allclose(got_e[b, [0, 2]], want_e[b, [0, 2]], rtol=max(tol, 1e-4), atol=1e-6 * want_e[b, 1])
 
 
 def test_sizes_beyond_the_fixed_scratch_are_refused(fc):
