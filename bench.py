@@ -31,11 +31,11 @@ UNIT = "tokens/s"
 FP32_LANES_PER_SM = 128          # FP32 FMA lanes per SM on B200
 DEFAULT_CONFIG = "cfg3"          # the 32k-token workload the target fraction is quoted on
 
-# DRAM traffic per launch of the dominant kernel from the committed ncu capture
-# (profiles/), bytes; None until a capture of that kernel and workload exists.
+# DRAM bytes read + written per launch of the dominant kernel as an ncu capture counted them (a constant from
+# that capture, not a measurement of this run; None where no capture of the kernel and workload exists):
+# pass 2 of cfg3, 0.68 MB read + 0.79 MB written on average over 24 launches with the intermediate in the
+# persisting part of L2.
 NCU_TRAFFIC_BYTES = {
-    # profiles/transform_passes_cfg3_dram_and_icache.md (d): 0.68 MB read + 0.79 MB written per launch of k_p2
-    # (average over 24 launches with the intermediate in the persisting part of L2)
     ("cfg3", "pass2"): 1.47e6,
 }
 
@@ -138,31 +138,60 @@ def step_accounting(binding, handle, cfg):
 
 
 # --------------------------------------------------------------------------- CPU baseline (oracle)
-def oracle_sample(cfg, Ks_host, Vs_host, budget_s: float):
-    """Times the fp64 oracle ("fft" tier, as it stands) on whole layers of the workload until
-    about budget_s seconds are used; returns tokens/s scaled to the full layer count."""
+def oracle_sample(cfg, Ks_host, Vs_host, budget_s: float, threads: int = 1):
+    """Times the fp64 oracle ("fft" tier, as it stands) on whole layers of the workload until about
+    budget_s seconds are used; returns tokens/s scaled to the full layer count.  With threads > 1 the
+    (layer, head) units go to a pool of host threads, one oracle call each (the oracle's numpy / scipy
+    routines release the interpreter lock); the oracle itself is untouched."""
     import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
     from oracle import flashcache_oracle as O
-    L = cfg.num_layers
+    L, H = cfg.num_layers, cfg.num_heads
+    cu = cfg.cu_seqlens
+    pool = ThreadPoolExecutor(max_workers=threads) if threads > 1 else None
+
+    def run(fn, items):
+        return list(pool.map(fn, items)) if pool else [fn(x) for x in items]
+
+    def score_unit(lh):                      # one head of one layer, every sequence: scores and energy sums
+        l, h = lh
+        sc = np.zeros(cfg.total_tokens)
+        en = np.zeros((len(cfg.seqlens), 4))
+        for b, n in enumerate(cfg.seqlens):
+            if n == 0:
+                continue
+            s, e = O.score_head(Ks_host[l][cu[b]:cu[b + 1], h].astype(np.float64),
+                                Vs_host[l][cu[b]:cu[b + 1], h].astype(np.float64), cfg.gamma, "fft")
+            sc[cu[b]:cu[b + 1]] = s
+            en[b] = e
+        return sc, en
+
     t0 = time.perf_counter()
     used, scores, energy = 0, [], []
+    step = max(1, threads // H)              # layers scored per round, so that every thread has a unit
     while used < len(Ks_host):
-        s, e = O.score_layer(Ks_host[used], Vs_host[used], cfg.cu_seqlens, cfg.gamma, "fft")
-        scores.append(s)
-        energy.append(e)
-        used += 1
+        ls = list(range(used, min(len(Ks_host), used + step)))
+        res = run(score_unit, [(l, h) for l in ls for h in range(H)])
+        for i, l in enumerate(ls):
+            scores.append(np.stack([res[i * H + h][0] for h in range(H)]))
+            energy.append(sum(res[i * H + h][1] for h in range(H)))
+        used += len(ls)
         el = time.perf_counter() - t0
-        if el + el / used > budget_s:
+        if el + el / used * len(ls) > budget_s:
             break
     budgets, offsets = O.allocate_budgets(np.stack(energy), list(cfg.seqlens), cfg.rho, cfg.min_keep)
-    cu = cfg.cu_seqlens
-    for l in range(used):
-        for h in range(cfg.num_heads):
-            for b, n in enumerate(cfg.seqlens):
-                idx = O.select_topk(scores[l][h, cu[b]:cu[b + 1]], int(budgets[l, b]))
-                O.compact_rows(Ks_host[l][cu[b]:cu[b + 1], h], idx)
-                O.compact_rows(Vs_host[l][cu[b]:cu[b + 1], h], idx)
+
+    def select_unit(lh):
+        l, h = lh
+        for b, n in enumerate(cfg.seqlens):
+            idx = O.select_topk(scores[l][h, cu[b]:cu[b + 1]], int(budgets[l, b]))
+            O.compact_rows(Ks_host[l][cu[b]:cu[b + 1], h], idx)
+            O.compact_rows(Vs_host[l][cu[b]:cu[b + 1], h], idx)
+
+    run(select_unit, [(l, h) for l in range(used) for h in range(H)])
     el = time.perf_counter() - t0
+    if pool:
+        pool.shutdown()
     tokens_per_s = cfg.total_tokens / (el * L / used)
     return tokens_per_s, used, el
 
@@ -322,6 +351,40 @@ def run_spectrum(args):
                       "tokens_per_s": cfg.total_tokens / (ms / 1000.0)}))
 
 
+def quick_config(torch, binding, S, name, dev, peaks, alu_peak, warmup=3, steps=10):
+    """ms per step, tokens/s and the step's roofline fraction of one configuration (short run, inputs resident)."""
+    cfg = S.paper_configs()[name]
+    L = cfg.num_layers
+    Kd, Vd = zip(*[S.make_layer(cfg, l, dev) for l in range(L)])
+    comp = binding.Compressor(L, cfg.num_heads, cfg.head_dim, cfg.cu_seqlens, cfg.torch_dtype, cfg.rho, cfg.gamma,
+                              cfg.min_keep, device=dev.index)
+    for _ in range(warmup):
+        comp.compress(Kd, Vd)
+    torch.cuda.synchronize(dev)
+    comp.check_device_status()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        comp.compress(Kd, Vd)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1) / steps
+    comp.check_device_status()
+    acc, rows = step_accounting(binding, comp.handle, cfg)
+    s = 4 if cfg.dtype == "f32" else 2
+    step_bytes = rows * (2.0 * cfg.head_dim * s + 8.0 + cfg.rho * (4.0 * cfg.head_dim * s + 4.0))
+    step_flops = sum(v["flops"] for v in acc.values())
+    t_bound = max(step_bytes / (peaks["hbm_gbs"] * 1e9), step_flops / (alu_peak * 1e12))
+    input_gb = sum(k.numel() * k.element_size() * 2 for k in Kd) / 1e9
+    comp.close()
+    del Kd, Vd
+    torch.cuda.empty_cache()
+    return {"workload": cfg.name + ": " + cfg.note, "ms_per_step": ms, "value": cfg.total_tokens / (ms / 1000.0),
+            "unit": UNIT, "steps": steps, "warmup": warmup, "t_bound_ms": 1000.0 * t_bound,
+            "roofline_step_frac": t_bound / (ms / 1000.0), "input_gbytes": input_gb,
+            "l2_policy": "inputs exceed L2; no flush" if input_gb > 0.2 else "inputs fit L2 (warm); launch-bound, fraction not meaningful"}
+
+
 # --------------------------------------------------------------------------- main arm
 def main():
     ap = argparse.ArgumentParser()
@@ -335,6 +398,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
+    ap.add_argument("--no-all-configs", action="store_true", help="skip the short runs of the other four configurations")
     ap.add_argument("--per-layer", action="store_true",
                     help="one index set per layer from the head-averaged score (fc_select_compact_ex)")
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
@@ -400,6 +464,16 @@ def main():
         ms, n = binding.fc_profile_end(comp.handle)
         shares[name] = dict(ms=ms, launches=n)
     dominant = max((k for k in shares if k != "other"), key=lambda k: shares[k]["ms"])
+    # the dominant kernel alone on the GPU: one more profiled step with a single internal stream
+    binding.fc_set_internal_streams(comp.handle, 1)
+    comp.compress(Kd, Vd)
+    binding.fc_profile_begin(comp.handle, binding.KERNEL_CLASSES[dominant])
+    comp.compress(Kd, Vd)
+    a_ms, a_n = binding.fc_profile_end(comp.handle)
+    alone_us = 1000.0 * a_ms / max(1, a_n)
+    binding.fc_set_internal_streams(comp.handle, 2)
+    comp.compress(Kd, Vd)
+    torch.cuda.synchronize()
 
     # timed region
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -430,7 +504,10 @@ def main():
     # roofline of the dominant kernel and of the whole step
     acc, rows = step_accounting(binding, comp.handle, cfg)
     props = torch.cuda.get_device_properties(dev)
+    # ALU peak: nominal (SMs x 128 lanes x 2 x max clock) and what a pure FMA loop sustains in this run; the
+    # fractions below divide by the nominal figure (the larger of the two), the measured one is reported beside it
     alu_peak = props.multi_processor_count * FP32_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12   # TFLOP/s
+    alu_peak_measured = binding.fc_measure_fp32_peak(comp.handle)
     d_acc = acc[dominant]
     launches_per_step = max(1, shares[dominant]["launches"])
     avg_launch_s = dom_ms / 1000.0 / max(1, dom_launches)   # average over the sampled launches of the timed region
@@ -448,15 +525,23 @@ def main():
                     "%d SMs x %d FP32 lanes x 2 x %.0f MHz" % (props.multi_processor_count, FP32_LANES_PER_SM,
                                                               peaks["sm_max_mhz"])
                     if roof["bound"] == "alu" else "MEASURED_PEAKS.json hbm_gbs (%s)" % peaks["source"]),
-                share_of_step=dom_s / (ms_per_step / 1000.0),
-                class_ms_per_step={k: v["ms"] for k, v in shares.items()})
+                peak_measured=alu_peak_measured if roof["bound"] == "alu" else None,
+                frac_of_measured=(roof["achieved"] / alu_peak_measured) if roof["bound"] == "alu" else None,
+                peak_measured_source="fc_measure_fp32_peak: packed FMA loop on every SM, this run",
+                avg_launch_us_alone=alone_us,
+                class_ms_per_step={k: v["ms"] for k, v in shares.items()},
+                # device time summed over the kernel classes divided by the step: above 1 because the
+                # library runs consecutive head groups on two internal streams, whose kernels share the GPU
+                # (a launch lasts longer co-scheduled than alone)
+                overlap_factor=sum(v["ms"] for v in shares.values()) / ms_per_step)
     s = 4 if cfg.dtype == "f32" else 2
     step_bytes = rows * (2.0 * cfg.head_dim * s + 8.0 + cfg.rho * (4.0 * cfg.head_dim * s + 4.0))
     step_flops = sum(v["flops"] for v in acc.values())
     t_bound = max(step_bytes / (peaks["hbm_gbs"] * 1e9), step_flops / (alu_peak * 1e12))
     roof_step = dict(bound="alu" if step_flops / (alu_peak * 1e12) >= step_bytes / (peaks["hbm_gbs"] * 1e9) else "hbm",
                      t_bound_ms=1000.0 * t_bound, frac=t_bound / (ms_per_step / 1000.0),
-                     gflop=step_flops / 1e9, gbytes=step_bytes / 1e9)
+                     gflop=step_flops / 1e9, gbytes=step_bytes / 1e9,
+                     ms_x_sm_mhz=ms_per_step * (clocks["sm_mhz"] or 0.0))
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -523,15 +608,25 @@ def main():
 
     # CPU baseline: the oracle on this machine's host cores, bounded sample (rank 0, single-GPU run only)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_layers_host = min(L, 4)
+        n_layers_host = min(L, 8)
         Ks_host = [Kd[l].float().cpu().numpy() for l in range(n_layers_host)]
         Vs_host = [Vd[l].float().cpu().numpy() for l in range(n_layers_host)]
-        tps, used, el = oracle_sample(cfg, Ks_host, Vs_host, args.cpu_budget_s)
-        out["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": 1, "kind": "oracle",
+        cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+        tps, used, el = oracle_sample(cfg, Ks_host, Vs_host, args.cpu_budget_s, threads=cores)
+        out["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle",
                                "host_cores": os.cpu_count(),
-                               "sample": "%d of %d layers (all heads, all sequences), %.1f s, scaled by the layer count"
-                                         % (used, L, el)}
+                               "sample": "%d of %d layers (all heads, all sequences), %.1f s on %d host threads "
+                                         "(one oracle call per layer and head), scaled by the layer count"
+                                         % (used, L, el, cores)}
     comp.close()
+    # the other four configurations, briefly: 3 warm-up steps, 10 timed, same accounting
+    if world == 1 and args.config == DEFAULT_CONFIG and not args.layers and not args.no_all_configs:
+        del Kd, Vd
+        torch.cuda.empty_cache()
+        out["all_configs"] = {args.config: {"ms_per_step": ms_per_step, "value": value, "unit": UNIT,
+                                            "roofline_step_frac": roof_step["frac"]}}
+        for name in ("cfg1", "cfg2", "cfg4", "cfg5"):
+            out["all_configs"][name] = quick_config(torch, binding, S, name, dev, peaks, alu_peak)
     if rank == 0:
         print(json.dumps(out))
     if dist is not None:

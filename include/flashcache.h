@@ -102,6 +102,12 @@ const char *fc_status_string(fc_status s);
  * the handle's device status word since the last call (and clears it). */
 fc_status fc_last_device_status(fc_handle *h, fc_stream stream);
 
+/* Measures what the FP32 pipes of this GPU sustain (diagnostic for roofline reports; the paper has no
+ * counterpart): a loop of independent fused multiply-adds on every SM, best of three runs of about 2 ms,
+ * on the default stream; blocks the host; allocates and frees a small output buffer.  tflops (HOST) counts
+ * a fused multiply-add as two operations, like the nominal figure SMs x 128 lanes x 2 x clock. */
+fc_status fc_measure_fp32_peak(fc_handle *h, double *tflops);
+
 /* Self test of the failure path of the bounded device-side waits (diagnostic; the paper has no
  * counterpart): enqueues one small kernel that waits, at most 1000 tries, on a barrier nothing will ever
  * complete, gives up, and records it.  The next fc_last_device_status returns FC_ERR_TIMEOUT; the

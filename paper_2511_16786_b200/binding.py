@@ -22,7 +22,7 @@ FC_F32, FC_F16, FC_BF16 = 0, 1, 2
 _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
-    "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count", "fc_selftest_bounded_wait",
+    "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count", "fc_selftest_bounded_wait", "fc_measure_fp32_peak",
     "fc_set_group_bytes", "fc_set_internal_streams", "fc_set_l2_persist", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
@@ -102,6 +102,8 @@ def _load() -> ctypes.CDLL:
     lib.fc_set_group_bytes.restype = c_int
     lib.fc_reset_ordering.argtypes = [c_void_p]
     lib.fc_reset_ordering.restype = c_int
+    lib.fc_measure_fp32_peak.argtypes = [c_void_p, POINTER(c_double)]
+    lib.fc_measure_fp32_peak.restype = c_int
     lib.fc_selftest_bounded_wait.argtypes = [c_void_p, c_void_p]
     lib.fc_selftest_bounded_wait.restype = c_int
     lib.fc_set_internal_streams.argtypes = [c_void_p, c_int32]
@@ -223,6 +225,13 @@ def fc_launch_count(handle) -> int:
 
 def fc_set_group_bytes(handle, nbytes: int) -> None:
     _check(_lib.fc_set_group_bytes(handle, int(nbytes)), "fc_set_group_bytes")
+
+
+def fc_measure_fp32_peak(handle) -> float:
+    """TFLOP/s the FP32 pipes sustain in a pure fused-multiply-add loop (blocks the host for a few ms)."""
+    t = c_double(0.0)
+    _check(_lib.fc_measure_fp32_peak(handle, byref(t)), "fc_measure_fp32_peak")
+    return float(t.value)
 
 
 def fc_selftest_bounded_wait(handle) -> None:

@@ -16,6 +16,25 @@ __global__ void k_fill_master(float2 *master, int len) {
   master[i] = make_float2((float)c, (float)s);
 }
 
+// FP32 throughput probe: every thread runs eight independent chains of packed fused multiply-adds
+// (two fp32 lanes per instruction), 4 x 8 of them per iteration, nothing else in the loop.
+__global__ void __launch_bounds__(256) k_fma_probe(float *out, int iters, float a, float b) {
+  float2 x[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) x[i] = make_float2(threadIdx.x * 0.001f + i, threadIdx.x * 0.002f - i);
+  const float2 aa = make_float2(a, a), bb = make_float2(b, b);
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x[i] = __ffma2_rn(x[i], aa, bb);
+  }
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) s += x[i].x + x[i].y;
+  out[blockIdx.x * blockDim.x + threadIdx.x] = s;
+}
+
 // Self test of the failure path every bounded device-side wait takes: one block waits on a shared-memory
 // barrier that nothing ever arrives on, gives up after `limit` tries, records the timeout in the status
 // word and returns normally.
@@ -275,6 +294,37 @@ extern "C" fc_status fc_last_device_status(fc_handle *h, fc_stream stream) {
   if (word != 0) FC_CUDA_TRY(cudaMemset(h->status_word, 0, sizeof(int)));
   if (word == 0) return FC_OK;
   return (word & FC_DEV_FLAG_INTERNAL) ? FC_ERR_INTERNAL : FC_ERR_TIMEOUT;
+}
+
+extern "C" fc_status fc_measure_fp32_peak(fc_handle *h, double *tflops) {
+  if (!h || !tflops) return FC_ERR_INVALID_ARG;
+  FC_CUDA_TRY(cudaSetDevice(h->device));
+  const int blocks = h->num_sms * 8, threads = 256, iters = 4000;
+  float *out = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  fc_status rc = FC_ERR_CUDA;
+  float best_ms = 0.f;
+  if (cudaMalloc(&out, (size_t)blocks * threads * sizeof(float)) != cudaSuccess) goto done;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) goto done;
+  k_fma_probe<<<blocks, threads>>>(out, 10, 1.0001f, 0.5f);
+  for (int rep = 0; rep < 3; ++rep) {
+    float ms = 0.f;
+    if (cudaEventRecord(e0) != cudaSuccess) goto done;
+    k_fma_probe<<<blocks, threads>>>(out, iters, 1.0001f, 0.5f);
+    if (cudaEventRecord(e1) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess || cudaGetLastError() != cudaSuccess)
+      goto done;
+    if (rep == 0 || ms < best_ms) best_ms = ms;
+  }
+  // flops: 2 per lane and fused multiply-add, 2 lanes per instruction, 32 instructions per iteration
+  *tflops = (double)blocks * threads * iters * 32.0 * 2.0 * 2.0 / ((double)best_ms * 1e-3) * 1e-12;
+  rc = FC_OK;
+done:
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (out) cudaFree(out);
+  if (rc != FC_OK) cudaGetLastError();
+  return rc;
 }
 
 extern "C" fc_status fc_selftest_bounded_wait(fc_handle *h, fc_stream stream) {
