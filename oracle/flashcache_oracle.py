@@ -212,6 +212,32 @@ def power_spectrum(K: np.ndarray, V: np.ndarray, cu_seqlens, tier: str = "litera
     return out
 
 
+def cutoff_for_energy_share(P: np.ndarray, share: float):
+    """Cutoff read from a power spectrum (Eq. 11-12; the energy-distribution figures and the gamma
+    ablation of Sec. 4.3): the smallest omega whose kept band 0..omega (Eq. 8) holds at least `share`
+    of the total energy sum_m P_k[m] + P_v[m], i.e. the smallest omega for which the outlier-energy
+    part of Eq. 12, taken over K and V together, is at most 1 - share.
+
+    P: [N, 2] rows (P_k[m], P_v[m]) of one sequence.  Returns (omega, gamma) with
+    gamma = (omega + 1/2) / N, so that min(N-1, floor(gamma*N)) == omega.  A spectrum without
+    energy gives omega = 0."""
+    P = np.asarray(P, dtype=np.float64)
+    N = P.shape[0]
+    tot = 0.0
+    for m in range(N):
+        tot += P[m, 0] + P[m, 1]
+    omega = 0
+    if tot > 0.0:
+        acc = 0.0
+        omega = N - 1
+        for m in range(N):
+            acc += P[m, 0] + P[m, 1]
+            if acc >= share * tot:
+                omega = m
+                break
+    return omega, (omega + 0.5) / N
+
+
 def energy_ratio(energy_row) -> float:
     """R^l = R_k^l + R_v^l of Eq. 12 from (hiK, totK, hiV, totV); a matrix with
     zero total energy contributes 0."""

@@ -276,3 +276,47 @@ def test_power_spectrum_tiers_agree():
         V = rng.standard_normal((n, 1, 5))
         np.testing.assert_allclose(O.power_spectrum(K, V, [0, n], "fft"), O.power_spectrum(K, V, [0, n], "literal"),
                                    rtol=1e-9, atol=1e-12)
+
+
+# ---------------------------------------------------------------- cutoff from the spectrum (Eq. 11-12)
+def test_cutoff_from_spectrum_single_basis_vector_steps_at_its_frequency():
+    # all the energy sits in bin m0: every share in (0, 1] gives omega = m0, and min(N-1, floor(gamma*N)) gives it back
+    N, d, m0 = 96, 3, 17
+    X = np.outer(O.phi(N)[m0], np.array([1.0, -2.0, 0.5]))
+    P = O.power_spectrum(X.reshape(N, 1, d), np.zeros((N, 1, d)), [0, N], "literal")
+    for share in (1e-6, 0.3, 0.999):
+        omega, gamma = O.cutoff_for_energy_share(P, share)
+        assert omega == m0
+        assert O.cutoff_index(N, gamma) == omega
+
+
+def test_cutoff_from_spectrum_white_noise_tracks_the_share():
+    # flat expected spectrum: the kept band must hold the share, so omega + 1 is close to share * N
+    rng = np.random.default_rng(5)
+    N, d = 2048, 64
+    K, V = rng.standard_normal((N, 1, d)), rng.standard_normal((N, 1, d))
+    P = O.power_spectrum(K, V, [0, N], "fft")
+    for share in (0.1, 0.5, 0.9):
+        omega, _ = O.cutoff_for_energy_share(P, share)
+        assert abs((omega + 1) / N - share) < 0.02
+
+
+def test_cutoff_from_spectrum_is_the_eq12_threshold_and_monotone():
+    # by its definition: outlier-energy share (Eq. 12 over K and V together) <= 1 - share at omega and > 1 - share at omega - 1
+    rng = np.random.default_rng(6)
+    N = 301
+    P = rng.random((N, 2)) * np.exp(-np.arange(N) / 40.0)[:, None]
+    tot = P.sum()
+    prev = -1
+    for share in (0.0, 0.2, 0.5, 0.8, 0.95, 1.0):
+        omega, gamma = O.cutoff_for_energy_share(P, share)
+        assert omega >= prev
+        prev = omega
+        assert P[omega + 1:].sum() / tot <= 1.0 - share + 1e-12
+        if omega > 0:
+            assert P[omega:].sum() / tot > 1.0 - share - 1e-12
+        assert O.cutoff_index(N, gamma) == omega
+    assert O.cutoff_for_energy_share(np.zeros((8, 2)), 0.5)[0] == 0
+    # brute force on a tiny spectrum
+    P = np.array([[1.0, 0.0], [0.0, 1.0], [2.0, 0.0], [0.0, 0.0]])
+    assert [O.cutoff_for_energy_share(P, s)[0] for s in (0.25, 0.26, 0.5, 0.51, 1.0)] == [0, 1, 1, 2, 2]
