@@ -268,6 +268,24 @@ fc_status fc_power_spectrum(fc_handle *h, const fc_kv_view *kv, double *spectrum
                             void *workspace, size_t workspace_bytes, fc_stream stream);
 
 /*
+ * Cutoff read from the spectrum (Sec. 3.2.2, Eq. 11-12; the energy-distribution figures; the gamma
+ * ablation of Sec. 4.3): for every sequence the smallest omega whose kept band 0..omega (Eq. 8) holds at
+ * least `share` of the total energy sum_m P_k[m] + P_v[m], i.e. the smallest cutoff that leaves at most
+ * 1 - share of the energy to the outlier band of Eq. 12.
+ *
+ *   spectrum    DEVICE double[T][2] as written by fc_power_spectrum
+ *   cu_seqlens  HOST int32[batch+1]
+ *   share       0 <= share <= 1
+ *   omega       DEVICE int32[batch]
+ *   gamma       DEVICE double[batch] = (omega + 1/2) / N: passed to fc_score_layer it gives exactly this
+ *               omega (min(N-1, floor(gamma*N))); an empty sequence gets 0, a spectrum without energy omega 0
+ * fp64 running sums in a fixed order.  Errors: FC_ERR_INVALID_ARG, FC_ERR_CUDA.
+ */
+fc_status fc_cutoff_from_spectrum(fc_handle *h, const double *spectrum, int32_t batch,
+                                  const int32_t *cu_seqlens, double share, int32_t *omega,
+                                  double *gamma, fc_stream stream);
+
+/*
  * Decoding step on the compacted cache (Sec. 3.1, Eq. 3-4): for every sequence b and query head j
  *     out[b][j] = Softmax(q[b][j] K^T / sqrt(head_dim)) V
  * where K and V are, for KV head j / (num_q_heads / num_heads), the rows the compressor kept for

@@ -27,7 +27,7 @@ EXPORTS = (
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
     "fc_select_compact_layers", "fc_layer_capacity_rows",
-    "fc_power_spectrum_workspace_bytes", "fc_power_spectrum",
+    "fc_power_spectrum_workspace_bytes", "fc_power_spectrum", "fc_cutoff_from_spectrum",
     "fc_decode_workspace_bytes", "fc_decode_attention",
     "fc_static_scratch_bytes", "fc_score_layer_static", "fc_static_last_device_status",
     "fc_compress_host_rows", "fc_compress_host_arena_bytes", "fc_compress_host",
@@ -102,6 +102,9 @@ def _load() -> ctypes.CDLL:
     lib.fc_set_group_bytes.restype = c_int
     lib.fc_reset_ordering.argtypes = [c_void_p]
     lib.fc_reset_ordering.restype = c_int
+    lib.fc_cutoff_from_spectrum.argtypes = [c_void_p, c_void_p, c_int32, POINTER(c_int32), c_double, c_void_p,
+                                            c_void_p, c_void_p]
+    lib.fc_cutoff_from_spectrum.restype = c_int
     lib.fc_measure_fp32_peak.argtypes = [c_void_p, POINTER(c_double)]
     lib.fc_measure_fp32_peak.restype = c_int
     lib.fc_selftest_bounded_wait.argtypes = [c_void_p, c_void_p]
@@ -225,6 +228,15 @@ def fc_launch_count(handle) -> int:
 
 def fc_set_group_bytes(handle, nbytes: int) -> None:
     _check(_lib.fc_set_group_bytes(handle, int(nbytes)), "fc_set_group_bytes")
+
+
+def fc_cutoff_from_spectrum(handle, spectrum, cu_seqlens, share: float, omega, gamma) -> None:
+    """spectrum: float64 [T, 2] from fc_power_spectrum; omega: int32 [B]; gamma: float64 [B] (device)."""
+    cu = _cu_array(cu_seqlens)
+    _check(_lib.fc_cutoff_from_spectrum(handle, c_void_p(spectrum.data_ptr()), len(cu) - 1,
+                                        ctypes.cast(cu, POINTER(c_int32)), float(share),
+                                        c_void_p(omega.data_ptr()), c_void_p(gamma.data_ptr()), _stream()),
+           "fc_cutoff_from_spectrum")
 
 
 def fc_measure_fp32_peak(handle) -> float:

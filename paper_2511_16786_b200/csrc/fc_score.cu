@@ -1343,6 +1343,96 @@ extern "C" fc_status fc_score_layer(fc_handle *h, const fc_kv_view *kv, double g
 }
 
 // ---------------------------------------------------------------------------
+// fc_cutoff_from_spectrum: the smallest omega whose kept band holds a given share of the energy.
+// One block per sequence; thread t adds up a contiguous run of bins, a block scan of the run totals in
+// fp64 finds the run in which the running sum first reaches share * total, and the thread that owns the
+// run walks it.  Sums are taken in a fixed order (deterministic).
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int kCutThreads = 1024;
+struct CutTable { int start[65]; };
+
+__global__ void __launch_bounds__(kCutThreads)
+k_cutoff_from_spectrum(const double *__restrict__ spectrum, const __grid_constant__ CutTable st, int b0, double share,
+                       int *__restrict__ omega, double *__restrict__ gamma) {
+  __shared__ double run[kCutThreads];
+  __shared__ double s_total;
+  const int tid = threadIdx.x;
+  const int s0 = st.start[blockIdx.x], N = st.start[blockIdx.x + 1] - s0;
+  const int b = b0 + blockIdx.x;
+  if (N == 0) {
+    if (tid == 0) { omega[b] = 0; gamma[b] = 0.0; }
+    return;
+  }
+  const int per = (N + kCutThreads - 1) / kCutThreads;
+  const int lo = tid * per, hi = lo + per < N ? lo + per : N;
+  const double *P = spectrum + 2 * (size_t)s0;
+  double mine = 0.0;
+  for (int m = lo; m < hi; ++m) mine += P[2 * m] + P[2 * m + 1];
+  run[tid] = mine;
+  __syncthreads();
+  // inclusive scan of the run totals (Hillis-Steele, fp64)
+  for (int o = 1; o < kCutThreads; o <<= 1) {
+    const double add = tid >= o ? run[tid - o] : 0.0;
+    __syncthreads();
+    run[tid] += add;
+    __syncthreads();
+  }
+  if (tid == kCutThreads - 1) s_total = run[tid];
+  __syncthreads();
+  const double total = s_total, want = share * total;
+  if (!(total > 0.0)) {
+    if (tid == 0) { omega[b] = 0; gamma[b] = 0.5 / (double)N; }
+    return;
+  }
+  // the run that holds the crossing: the first non-empty one whose running sum has reached `want` (the
+  // scan's sums of one and the same set can differ in the last bit, so "the last run reaches the total"
+  // is not relied on: without a qualifying run the last non-empty one is taken)
+  __shared__ int s_owner;
+  if (tid == 0) s_owner = kCutThreads;
+  __syncthreads();
+  if (lo < hi && run[tid] >= want) atomicMin(&s_owner, tid);
+  __syncthreads();
+  const int owner = s_owner < kCutThreads ? s_owner : (N - 1) / per;
+  if (tid == owner) {
+    double acc = run[tid] - mine;
+    int m = lo;
+    for (; m < hi; ++m) {
+      acc += P[2 * m] + P[2 * m + 1];
+      if (acc >= want) break;
+    }
+    if (m >= hi) m = hi - 1;
+    omega[b] = m;
+    gamma[b] = ((double)m + 0.5) / (double)N;
+  }
+}
+
+}  // namespace
+
+extern "C" fc_status fc_cutoff_from_spectrum(fc_handle *h, const double *spectrum, int32_t batch,
+                                             const int32_t *cu_seqlens, double share, int32_t *omega,
+                                             double *gamma, fc_stream stream) {
+  if (!h || !spectrum || !cu_seqlens || !omega || !gamma || batch < 0) return FC_ERR_INVALID_ARG;
+  if (!(share >= 0.0 && share <= 1.0) || cu_seqlens[0] != 0) return FC_ERR_INVALID_ARG;
+  for (int b = 0; b < batch; ++b)
+    if (cu_seqlens[b + 1] < cu_seqlens[b]) return FC_ERR_INVALID_ARG;
+  int dev = -1;
+  FC_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev != h->device) FC_CUDA_TRY(cudaSetDevice(h->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  fc_status s;
+  for (int b0 = 0; b0 < batch; b0 += 64) {
+    const int nseq = batch - b0 < 64 ? batch - b0 : 64;
+    CutTable tab;
+    for (int i = 0; i <= nseq; ++i) tab.start[i] = cu_seqlens[b0 + i];
+    k_cutoff_from_spectrum<<<nseq, kCutThreads, 0, st>>>(spectrum, tab, b0, share, omega, gamma);
+    if ((s = fc_after_launch(h)) != FC_OK) return s;
+  }
+  return FC_OK;
+}
+
+// ---------------------------------------------------------------------------
 // fc_score_layer_static: the same scoring with every byte of scratch in arrays that are
 // part of the loaded library image, for callers that must not allocate device memory.
 // ---------------------------------------------------------------------------

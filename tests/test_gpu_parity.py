@@ -239,6 +239,58 @@ def test_power_spectrum_matches_oracle(fc, lens, H, d, dtype):
         np.testing.assert_allclose(got[s + om + 1:e, 1].sum(), en[b, 2], rtol=2e-3, atol=1e-6 * en[b, 3])
 
 
+@pytest.mark.parametrize("share", [0.0, 0.5, 0.9, 0.999, 1.0])
+def test_cutoff_from_spectrum_matches_oracle(fc, share):
+    # (a) on spectra given to both sides (exact integer agreement, sequences of every size incl. empty, zero energy,
+    # longer than one bin per thread), (b) end to end: spectrum and cutoff on the device, then scoring at the
+    # returned gamma uses exactly that omega
+    rng = np.random.default_rng(int(share * 1000) + 3)
+    lens = [1, 0, 7, 1000, 5000, 64, 131072]
+    cu = [0] + [int(x) for x in np.cumsum(lens)]
+    P = rng.random((cu[-1], 2)) * np.exp(-rng.random((cu[-1], 1)) * 8.0)
+    P[cu[5]:cu[6]] = 0.0                                         # a sequence without energy
+    P[cu[3]:cu[3] + 40] *= 1e4                                   # one with a dominant low band
+    h = fc.fc_create(0, 131072)
+    try:
+        om = torch.full((len(lens),), -7, dtype=torch.int32, device="cuda")
+        ga = torch.full((len(lens),), -7.0, dtype=torch.float64, device="cuda")
+        fc.fc_cutoff_from_spectrum(h, torch.from_numpy(P).cuda(), cu, share, om, ga)
+        assert fc.fc_last_device_status(h) == 0
+        om, ga = om.cpu().numpy(), ga.cpu().numpy()
+        for b, n in enumerate(lens):
+            if n == 0:
+                assert om[b] == 0 and ga[b] == 0.0
+                continue
+            wo, wg = O.cutoff_for_energy_share(P[cu[b]:cu[b + 1]], share)
+            if om[b] != wo:                                      # only where rounding of the running sum decides
+                tot = P[cu[b]:cu[b + 1]].sum()
+                c = np.cumsum(P[cu[b]:cu[b + 1]].sum(1))
+                assert abs(c[min(om[b], wo)] - share * tot) <= 1e-12 * tot
+            else:
+                assert ga[b] == wg
+            assert O.cutoff_index(n, float(ga[b])) == om[b]
+        # end to end on one layer
+        k, v = _rand_kv(3000, 2, 128, torch.float32, 5)
+        cu2 = [0, 1000, 3000]
+        kd, vd = k.cuda(), v.cuda()
+        spec = torch.empty((3000, 2), dtype=torch.float64, device="cuda")
+        ws = torch.empty(fc.fc_power_spectrum_workspace_bytes(h, kd, vd, cu2), dtype=torch.uint8, device="cuda")
+        fc.fc_power_spectrum(h, kd, vd, cu2, spec, ws)
+        om2 = torch.empty(2, dtype=torch.int32, device="cuda")
+        ga2 = torch.empty(2, dtype=torch.float64, device="cuda")
+        fc.fc_cutoff_from_spectrum(h, spec, cu2, share, om2, ga2)
+        assert fc.fc_last_device_status(h) == 0
+        want = O.power_spectrum(k.double().numpy(), v.double().numpy(), cu2, "fft")
+        for b in range(2):
+            wo, _ = O.cutoff_for_energy_share(want[cu2[b]:cu2[b + 1]], share)
+            seg = want[cu2[b]:cu2[b + 1]].sum(1)
+            got = int(om2[b])
+            if got != wo:                                        # fp32 spectrum against fp64: the kept share must still fit
+                assert abs(np.cumsum(seg)[min(got, wo)] / seg.sum() - share) <= 2e-3
+    finally:
+        fc.fc_destroy(h)
+
+
 # ---------------------------------------------------------------- budgets
 def _gpu_budgets(fc, energy, cu, rho, min_keep):
     L, B = energy.shape[:2]
