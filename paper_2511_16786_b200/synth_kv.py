@@ -18,7 +18,10 @@ Recipe for one (layer, sequence) of length N, every KV head h and channel c:
 (un-normalised cosines, so the smooth part carries most of the energy), then a
 set of round(f * N) token rows, drawn without replacement per head and shared
 by K and V, is replaced by 5 * N(0, 1), and the result is cast to the storage
-dtype.  K and V use independent draws of a and n.
+dtype.  K and V use independent draws of a and n.  Every draw comes from a
+counter-based generator written in exactly defined tensor operations (see
+_normal), so a configuration, layer and seed name the same bytes on the CPU and
+on a GPU; the normal draws are sums of twelve uniforms.
 """
 from __future__ import annotations
 
@@ -93,6 +96,74 @@ def _stream(cfg: KVConfig, device, *key) -> torch.Generator:
     return g
 
 
+# ---------------------------------------------------------------------------
+# Counter-based draws that give the same bytes on every device.  Only operations whose
+# results are fixed by their definition are used on tensors: wrapping 64-bit integer
+# arithmetic, exact integer-to-float conversion, and single correctly rounded float64
+# multiplies, adds and subtractions (one torch call each, so nothing is fused).  No
+# library random generator, no transcendental function and no matrix product touches a
+# tensor; the few sines and cosines needed are Python floats computed on the host.
+# ---------------------------------------------------------------------------
+def _signed64(x: int) -> int:
+    x &= (1 << 64) - 1
+    return x - (1 << 64) if x >= (1 << 63) else x
+
+
+_M1, _M2, _GOLD = _signed64(0xBF58476D1CE4E5B9), _signed64(0x94D049BB133111EB), _signed64(0x9E3779B97F4A7C15)
+
+
+def _key(cfg: KVConfig, *key) -> int:
+    h = zlib.crc32(repr((cfg.name, cfg.seed) + tuple(key)).encode())
+    return _signed64(h * 0x9E3779B97F4A7C15 + cfg.seed * 0xD1B54A32D192ED03 + 0x632BE59BD9B4E019)
+
+
+def _mix(x: torch.Tensor) -> torch.Tensor:
+    """The splitmix64 finaliser on an int64 tensor (logical shifts, wrapping products)."""
+    x = x ^ ((x >> 30) & 0x3FFFFFFFF)
+    x = x * _M1
+    x = x ^ ((x >> 27) & 0x1FFFFFFFFF)
+    x = x * _M2
+    return x ^ ((x >> 31) & 0x1FFFFFFFF)
+
+
+def _normal(key: int, count: int, device) -> torch.Tensor:
+    """count draws, float64: the sum of twelve independent 16-bit uniforms, centred and scaled to unit
+    variance (Irwin-Hall; within 6 standard deviations, kurtosis 2.9)."""
+    idx = torch.arange(count, dtype=torch.int64, device=device) * 3
+    total = torch.zeros(count, dtype=torch.int64, device=device)
+    for r in range(3):
+        h = _mix((idx + r) * _GOLD + key)
+        for sh in (0, 16, 32, 48):
+            total += (h >> sh) & 0xFFFF
+    return (total - 6 * 65535).to(torch.float64) * (1.0 / 65536.0)
+
+
+def _cos_basis(N: int, M: int, device) -> list:
+    """[cos(pi * m * (2 i + 1) / (2 N)) for m < M] as float64 vectors over i: e^{j theta_i} by products of
+    host-computed rotations chosen by the bits of i, then the three-term recurrence in m."""
+    i = torch.arange(N, dtype=torch.int64, device=device)
+    t0 = math.pi / (2.0 * N)
+    zr = torch.full((N,), math.cos(t0), dtype=torch.float64, device=device)
+    zi = torch.full((N,), math.sin(t0), dtype=torch.float64, device=device)
+    k = 0
+    while (1 << k) < N:
+        ang = (math.pi / N) * (1 << k)
+        rr, ri = math.cos(ang), math.sin(ang)
+        on = ((i >> k) & 1).bool()
+        nr = zr * rr - zi * ri
+        ni = zr * ri + zi * rr
+        zr = torch.where(on, nr, zr)
+        zi = torch.where(on, ni, zi)
+        k += 1
+    out = [torch.ones(N, dtype=torch.float64, device=device)]
+    if M > 1:
+        out.append(zr)
+    two_c = zr * 2.0
+    for m in range(2, M):
+        out.append(two_c * out[m - 1] - out[m - 2])
+    return out[:M]
+
+
 def outlier_fraction(cfg: KVConfig, layer: int, seq: int) -> float:
     kind = cfg.outlier[0]
     if kind == "fixed":
@@ -104,8 +175,9 @@ def outlier_fraction(cfg: KVConfig, layer: int, seq: int) -> float:
 
 
 def make_layer(cfg: KVConfig, layer: int, device="cpu"):
-    """K, V of one layer: [T, H, d] tensors of cfg.torch_dtype on `device`,
-    the sequences of the batch packed along the token axis."""
+    """K, V of one layer: [T, H, d] tensors of cfg.torch_dtype on `device`, the sequences of the batch
+    packed along the token axis.  The same configuration, layer and seed give the same bytes on every
+    device."""
     device = torch.device(device)
     H, d, M = cfg.num_heads, cfg.head_dim, cfg.num_low
     T = cfg.total_tokens
@@ -115,23 +187,22 @@ def make_layer(cfg: KVConfig, layer: int, device="cpu"):
     for b, N in enumerate(cfg.seqlens):
         if N == 0:
             continue
-        g = _stream(cfg, device, "kv", layer, b)
-        i = torch.arange(N, device=device, dtype=torch.float64)
-        m = torch.arange(M, device=device, dtype=torch.float64)
-        basis = torch.cos(math.pi * (2.0 * i[:, None] + 1.0) * m[None, :] / (2.0 * N)).to(torch.float32)
+        basis = _cos_basis(N, M, device)
         f = outlier_fraction(cfg, layer, b)
         n_out = int(round(f * N))
         rows = None
-        if n_out > 0:
-            rows = torch.stack([torch.randperm(N, generator=g, device=device)[:n_out]
-                                for _ in range(H)])          # [H, n_out]
-        for dst in (K, V):
-            a = torch.randn((M, H * d), generator=g, device=device, dtype=torch.float32)
-            x = basis @ a
-            x.add_(torch.randn((N, H * d), generator=g, device=device, dtype=torch.float32), alpha=0.1)
+        if n_out > 0:          # n_out distinct tokens per head: the smallest of N hashed keys
+            pos = torch.arange(N, dtype=torch.int64, device=device)
+            rows = [torch.sort(_mix(pos * _GOLD + _key(cfg, "rows", layer, b, h)), stable=True).indices[:n_out]
+                    for h in range(H)]
+        for which, dst in (("k", K), ("v", V)):
+            a = _normal(_key(cfg, "coef", which, layer, b), M * H * d, device).view(M, H * d)
+            x = _normal(_key(cfg, "noise", which, layer, b), N * H * d, device).view(N, H * d) * 0.1
+            for m in range(M):
+                x = x + basis[m][:, None] * a[m][None, :]
             x = x.view(N, H, d)
             if rows is not None:
-                repl = 5.0 * torch.randn((H, n_out, d), generator=g, device=device, dtype=torch.float32)
+                repl = (_normal(_key(cfg, "outl", which, layer, b), H * n_out * d, device) * 5.0).view(H, n_out, d)
                 for h in range(H):
                     x[rows[h], h, :] = repl[h]
             dst[cu[b]:cu[b + 1]] = x.to(cfg.torch_dtype)

@@ -790,6 +790,20 @@ def test_config5_full_size_sampled(fc):
                                (21, 4, 1), (25, 5, 2), (9, 6, 0), (2, 7, 3)])
 
 
+# ---------------------------------------------------------------- inputs
+def test_generator_gives_the_same_bytes_on_cpu_and_gpu(fc):
+    # "seed 0" names one tensor: the oracle side (CPU) and the bench side (GPU) see identical inputs
+    for name, changes in (("cfg1", {}), ("cfg2", dict(num_layers=2, seqlens=(1000, 0, 333))),
+                          ("cfg4", dict(num_layers=1, num_heads=3, seqlens=(2048,))),
+                          ("cfg5", dict(num_layers=1, seqlens=(517, 4099)))):
+        cfg = S.scaled(S.paper_configs()[name], name + "_bytes", **changes)
+        for l in range(cfg.num_layers):
+            kc, vc = S.make_layer(cfg, l, "cpu")
+            kg, vg = S.make_layer(cfg, l, "cuda")
+            assert torch.equal(kc.view(torch.uint8), kg.cpu().view(torch.uint8))
+            assert torch.equal(vc.view(torch.uint8), vg.cpu().view(torch.uint8))
+
+
 # ---------------------------------------------------------------- failure reporting
 def test_bounded_wait_that_runs_out_is_reported(fc):
     # a wait nothing will ever satisfy gives up after its limit, the status word says so, and the handle and the
