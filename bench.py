@@ -311,6 +311,45 @@ def run_decode(args):
         "points": points}))
 
 
+# --------------------------------------------------------------------------- FP32 pipes against the tensor pipe
+def run_proto(args):
+    """One radix-16 transform stage on an L2-resident tile (16 x 65536 complex columns, 8.4 MB each way), on the
+    FP32 pipes, on the tensor pipe (3 x TF32) and as a plain copy; then the arithmetic alone (64 repetitions on the
+    loaded registers).  Median of 20 launches each, CUDA events."""
+    import torch
+    from paper_2511_16786_b200 import binding
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    h = binding.fc_create(0, 1024)
+    ncols = 65536
+    x = torch.randn((16, ncols, 2), device=dev)
+    y = torch.empty_like(x)
+    res = {}
+    for rep in (1, 64):
+        for variant, name in ((0, "fp32_pipes"), (1, "tensor_pipe_3xtf32"), (2, "copy_only")):
+            if variant == 2 and rep > 1:
+                continue
+            for _ in range(3):
+                binding.fc_proto_dft16_stage(h, x, y, variant, rep)
+            torch.cuda.synchronize()
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+            for e0, e1 in ev:
+                e0.record()
+                binding.fc_proto_dft16_stage(h, x, y, variant, rep)
+                e1.record()
+            torch.cuda.synchronize()
+            res["%s_repeat%d_us" % (name, rep)] = 1000.0 * sorted(a.elapsed_time(b) for a, b in ev)[10]
+    binding._check(binding.fc_last_device_status(h), "device status")
+    binding.fc_destroy(h)
+    a, t = res["fp32_pipes_repeat64_us"], res["tensor_pipe_3xtf32_repeat64_us"]
+    res["arithmetic_us_per_stage_fp32_pipes"] = (a - res["fp32_pipes_repeat1_us"]) / 63.0
+    res["arithmetic_us_per_stage_tensor_pipe"] = (t - res["tensor_pipe_3xtf32_repeat1_us"]) / 63.0
+    print(json.dumps({"metric": "dft16_stage_us", "unit": "us", "higher_is_better": False, "n_gpus": 1,
+                      "dtype": "f32 / tf32x3", "data": "synthetic",
+                      "config": {"workload": "one radix-16 stage over 65536 complex columns (16 points each), "
+                                             "tile resident in L2", "median_of": 20}, "times": res}))
+
+
 # --------------------------------------------------------------------------- spectrum diagnostics
 def run_spectrum(args):
     """Time of fc_power_spectrum (Eq. 11 per layer) over all layers of a config; a diagnostic, reported beside
@@ -405,6 +444,8 @@ def main():
     ap.add_argument("--decode", action="store_true",
                     help="time the decoding-step attention on full and compressed caches instead of the compressor")
     ap.add_argument("--spectrum", action="store_true", help="time fc_power_spectrum over all layers of the config")
+    ap.add_argument("--proto", action="store_true",
+                    help="time one transform stage on the FP32 pipes and on the tensor pipe (measurement aid)")
     ap.add_argument("--decode-n", type=int, default=0, help="--decode: only this context length")
     ap.add_argument("--decode-rho", type=float, default=0.0, help="--decode: only this cache ratio")
     args = ap.parse_args()
@@ -416,6 +457,9 @@ def main():
         return
     if args.spectrum:
         run_spectrum(args)
+        return
+    if args.proto:
+        run_proto(args)
         return
 
     import torch

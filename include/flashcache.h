@@ -108,6 +108,18 @@ fc_status fc_last_device_status(fc_handle *h, fc_stream stream);
  * a fused multiply-add as two operations, like the nominal figure SMs x 128 lanes x 2 x clock. */
 fc_status fc_measure_fp32_peak(fc_handle *h, double *tflops);
 
+/* Measurement aid, not on the compression path (the paper has no counterpart): one radix-16 stage of the
+ * token-axis transform, y[k][c] = sum_p x[p][c] exp(-2*pi*j*p*k/16), on DEVICE float2 [16][ncols] arrays
+ * (ncols a multiple of 8, 16-byte aligned), computed
+ *   variant 0  on the FP32 pipes, as the shipped passes do (register-resident butterfly, two columns a thread),
+ *   variant 1  on the tensor pipe: the stage as a 32 x 32 real matrix product in TF32 with fp32 accumulation,
+ *              operands split in two TF32 terms, three products (about 21 significant bits),
+ *   variant 2  not at all (load and store only).
+ * repeat > 1 reruns the arithmetic on the loaded registers (timing only; results are then meaningless).
+ * Kept so that "FP32 pipes or tensor pipe for a transform stage" stays a measured statement. */
+fc_status fc_proto_dft16_stage(fc_handle *h, const void *x, void *y, int32_t ncols, int32_t variant,
+                               int32_t repeat, fc_stream stream);
+
 /* Self test of the failure path of the bounded device-side waits (diagnostic; the paper has no
  * counterpart): enqueues one small kernel that waits, at most 1000 tries, on a barrier nothing will ever
  * complete, gives up, and records it.  The next fc_last_device_status returns FC_ERR_TIMEOUT; the

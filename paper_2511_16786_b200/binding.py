@@ -22,7 +22,7 @@ FC_F32, FC_F16, FC_BF16 = 0, 1, 2
 _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
-    "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count", "fc_selftest_bounded_wait", "fc_measure_fp32_peak",
+    "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count", "fc_selftest_bounded_wait", "fc_measure_fp32_peak", "fc_proto_dft16_stage",
     "fc_set_group_bytes", "fc_set_internal_streams", "fc_set_l2_persist", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
@@ -105,6 +105,8 @@ def _load() -> ctypes.CDLL:
     lib.fc_cutoff_from_spectrum.argtypes = [c_void_p, c_void_p, c_int32, POINTER(c_int32), c_double, c_void_p,
                                             c_void_p, c_void_p]
     lib.fc_cutoff_from_spectrum.restype = c_int
+    lib.fc_proto_dft16_stage.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p]
+    lib.fc_proto_dft16_stage.restype = c_int
     lib.fc_measure_fp32_peak.argtypes = [c_void_p, POINTER(c_double)]
     lib.fc_measure_fp32_peak.restype = c_int
     lib.fc_selftest_bounded_wait.argtypes = [c_void_p, c_void_p]
@@ -237,6 +239,12 @@ def fc_cutoff_from_spectrum(handle, spectrum, cu_seqlens, share: float, omega, g
                                         ctypes.cast(cu, POINTER(c_int32)), float(share),
                                         c_void_p(omega.data_ptr()), c_void_p(gamma.data_ptr()), _stream()),
            "fc_cutoff_from_spectrum")
+
+
+def fc_proto_dft16_stage(handle, x, y, variant: int, repeat: int = 1) -> None:
+    """x, y: float32 device tensors [16, ncols, 2] (complex as pairs); variant 0 FP32 pipes, 1 tensor pipe, 2 copy."""
+    _check(_lib.fc_proto_dft16_stage(handle, c_void_p(x.data_ptr()), c_void_p(y.data_ptr()), int(x.shape[1]),
+                                     int(variant), int(repeat), _stream()), "fc_proto_dft16_stage")
 
 
 def fc_measure_fp32_peak(handle) -> float:

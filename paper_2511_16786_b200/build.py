@@ -12,7 +12,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libflashcache.so")
-SOURCES = ["fc_api.cu", "fc_score.cu", "fc_select.cu", "fc_host.cu", "fc_decode.cu"]
+SOURCES = ["fc_api.cu", "fc_score.cu", "fc_select.cu", "fc_host.cu", "fc_decode.cu", "fc_proto.cu"]
 EXTRA = {"fc_select.cu": ["-fmad=false"]}
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]

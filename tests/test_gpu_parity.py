@@ -790,6 +790,33 @@ def test_config5_full_size_sampled(fc):
                                (21, 4, 1), (25, 5, 2), (9, 6, 0), (2, 7, 3)])
 
 
+# ---------------------------------------------------------------- tensor-pipe stage (measurement aid)
+def test_dft16_stage_on_both_pipes_matches_fp64(fc):
+    # both variants against the 16-point DFT in fp64; the tensor form keeps about 21 bits per operand, which
+    # carries through a whole transform at the 1e-3 score tolerance of fp32 inputs (here: 1e-5 of the column's norm)
+    g = torch.Generator().manual_seed(4)
+    ncols = 4096 + 8
+    x = torch.randn((16, ncols, 2), generator=g) * torch.rand((1, ncols, 1), generator=g) * 10.0
+    xc = x[..., 0].double().numpy() + 1j * x[..., 1].double().numpy()
+    want = np.fft.fft(xc, axis=0)
+    h = fc.fc_create(0, 1024)
+    try:
+        xd = x.cuda()
+        for variant, tol in ((0, 2e-6), (1, 1e-5)):
+            yd = torch.zeros_like(xd)
+            fc.fc_proto_dft16_stage(h, xd, yd, variant)
+            assert fc.fc_last_device_status(h) == 0
+            y = yd.cpu().double().numpy()
+            got = y[..., 0] + 1j * y[..., 1]
+            err = np.abs(got - want).max(axis=0) / np.linalg.norm(xc, axis=0)
+            assert err.max() <= tol, "variant %d: %.3e" % (variant, err.max())
+        yd = torch.zeros_like(xd)
+        fc.fc_proto_dft16_stage(h, xd, yd, 2)
+        assert torch.equal(yd, xd)
+    finally:
+        fc.fc_destroy(h)
+
+
 # ---------------------------------------------------------------- inputs
 def test_generator_gives_the_same_bytes_on_cpu_and_gpu(fc):
     # "seed 0" names one tensor: the oracle side (CPU) and the bench side (GPU) see identical inputs
