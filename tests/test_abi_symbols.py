@@ -65,3 +65,27 @@ def test_oracle_is_not_imported_by_the_product():
         for fn in files:
             if fn.endswith((".py", ".cu", ".cuh", ".h")):
                 assert "oracle" not in open(os.path.join(dirpath, fn)).read().replace("CPU oracle", ""), fn
+
+
+def test_host_side_queries_and_checks_of_the_new_entry_points(lib):
+    # the capacity query is the budget total of Sec. 3.2.2 capped at the sequence length, summed over sequences:
+    # checked against the oracle's total_budget on a ragged batch, without a device
+    from oracle import flashcache_oracle as O
+    lib.fc_layer_capacity_rows.restype = ctypes.c_int64
+    lib.fc_layer_capacity_rows.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32),
+                                           ctypes.c_double, ctypes.c_int32]
+    for lens, L, rho, mk in (([32768], 28, 0.1, 1), ([1024], 1, 0.2, 1), ([5, 0, 100, 7], 3, 0.9, 4),
+                             ([10, 20], 4, 0.0, 2), ([8], 2, 1.0, 1)):
+        cu = (ctypes.c_int32 * (len(lens) + 1))(*([0] + [sum(lens[:i + 1]) for i in range(len(lens))]))
+        want = sum(min(n, O.total_budget(n, L, rho, mk)) for n in lens if n > 0)
+        assert lib.fc_layer_capacity_rows(L, len(lens), cu, rho, mk) == want
+    assert lib.fc_layer_capacity_rows(0, 1, cu, 0.5, 1) == -1
+    assert lib.fc_layer_capacity_rows(1, 1, None, 0.5, 1) == -1
+    # null handles and pointers are refused before any CUDA call
+    assert lib.fc_select_compact_layers(None, None, None, 1, None, None, None, None, 0, None) == 1
+    assert lib.fc_cutoff_from_spectrum(None, None, 0, None, ctypes.c_double(0.5), None, None, None) == 1
+    assert lib.fc_proto_dft16_stage(None, None, None, 8, 0, 1, None) == 1
+    assert lib.fc_measure_fp32_peak(None, None) == 1
+    assert lib.fc_selftest_bounded_wait(None, None) == 1
+    assert lib.fc_set_internal_streams(None, 2) == 1
+    assert lib.fc_set_l2_persist(None, 1) == 1
