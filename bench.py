@@ -433,6 +433,7 @@ def main():
     ap.add_argument("--config", default=DEFAULT_CONFIG)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--group-mib", type=int, default=0, help="transform group size override (MiB)")
+    ap.add_argument("--streams", type=int, default=0, help="internal streams of the scoring calls (default: the library's 2)")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first LAYERS layers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -488,6 +489,8 @@ def main():
                               cfg.gamma, cfg.min_keep, device=local_rank,
                               group_bytes=(args.group_mib << 20) if args.group_mib else None,
                               per_layer=args.per_layer)
+    if args.streams:
+        binding.fc_set_internal_streams(comp.handle, args.streams)
     input_bytes = sum(k.numel() * k.element_size() * 2 for k in Kd)
 
     def barrier():
@@ -515,7 +518,7 @@ def main():
     comp.compress(Kd, Vd)
     a_ms, a_n = binding.fc_profile_end(comp.handle)
     alone_us = 1000.0 * a_ms / max(1, a_n)
-    binding.fc_set_internal_streams(comp.handle, 2)
+    binding.fc_set_internal_streams(comp.handle, args.streams or 2)
     comp.compress(Kd, Vd)
     torch.cuda.synchronize()
 
