@@ -161,6 +161,14 @@ fc_status fc_set_score_overlap(fc_handle *h, int32_t enabled);
  * call waits for the one before it. */
 fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled);
 
+/* Sequences whose length is not a power of two are transformed by chirp convolutions of a padded
+ * power-of-two length (>= 2N - 1).  enabled = 1 (default): where the cutoff index omega of Eq. 8
+ * allows a shorter padded length (>= N + 2*omega + 1), only the bins -omega .. omega of the
+ * spectrum are computed, the low-pass part (the Base KV of Eq. 9) is transformed back and the
+ * score of Eq. 10 is taken against the input rows.  Same result to fp32 rounding; speed only.
+ * enabled = 0: always the full-length form (all N bins, residual formed in the frequency domain). */
+fc_status fc_set_chirp_band(fc_handle *h, int32_t enabled);
+
 /* Number of internal streams fc_score_layer spreads the head groups of a sequence over (1..4,
  * default 2, the measured best: two transforms in flight fill the GPU, three no longer fit the L2).
  * Call it between passes, not while deferred work is pending (fc_set_score_overlap).  Speed only. */

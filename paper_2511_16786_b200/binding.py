@@ -23,7 +23,7 @@ _DTYPE = {torch.float32: FC_F32, torch.float16: FC_F16, torch.bfloat16: FC_BF16}
 
 EXPORTS = (
     "fc_create", "fc_destroy", "fc_status_string", "fc_last_device_status", "fc_launch_count", "fc_selftest_bounded_wait", "fc_measure_fp32_peak", "fc_proto_dft16_stage",
-    "fc_set_group_bytes", "fc_set_internal_streams", "fc_set_l2_persist", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
+    "fc_set_group_bytes", "fc_set_chirp_band", "fc_set_internal_streams", "fc_set_l2_persist", "fc_reset_ordering", "fc_set_score_overlap", "fc_set_select_overlap", "fc_profile_begin", "fc_profile_stride", "fc_profile_end", "fc_describe_plan",
     "fc_score_workspace_bytes", "fc_select_workspace_bytes",
     "fc_score_layer", "fc_allocate_budgets", "fc_select_compact", "fc_select_compact_ex",
     "fc_select_compact_layers", "fc_layer_capacity_rows",
@@ -111,6 +111,8 @@ def _load() -> ctypes.CDLL:
     lib.fc_measure_fp32_peak.restype = c_int
     lib.fc_selftest_bounded_wait.argtypes = [c_void_p, c_void_p]
     lib.fc_selftest_bounded_wait.restype = c_int
+    lib.fc_set_chirp_band.argtypes = [c_void_p, c_int32]
+    lib.fc_set_chirp_band.restype = c_int
     lib.fc_set_internal_streams.argtypes = [c_void_p, c_int32]
     lib.fc_set_internal_streams.restype = c_int
     lib.fc_set_l2_persist.argtypes = [c_void_p, c_int32]
@@ -256,6 +258,10 @@ def fc_measure_fp32_peak(handle) -> float:
 
 def fc_selftest_bounded_wait(handle) -> None:
     _check(_lib.fc_selftest_bounded_wait(handle, _stream()), "fc_selftest_bounded_wait")
+
+
+def fc_set_chirp_band(handle, enabled: bool) -> None:
+    _check(_lib.fc_set_chirp_band(handle, 1 if enabled else 0), "fc_set_chirp_band")
 
 
 def fc_set_internal_streams(handle, count: int) -> None:

@@ -147,6 +147,7 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
   h->generic_only = false;
   h->select_overlap = 0;
   h->score_overlap = 0;
+  h->band_form = 1;
   h->step = 0;
   h->last_sig = -1;
   h->pending_join = false;
@@ -344,6 +345,12 @@ extern "C" fc_status fc_set_select_overlap(fc_handle *h, int32_t enabled) {
 extern "C" fc_status fc_set_score_overlap(fc_handle *h, int32_t enabled) {
   if (!h) return FC_ERR_INVALID_ARG;
   h->score_overlap = enabled ? 1 : 0;
+  return FC_OK;
+}
+
+extern "C" fc_status fc_set_chirp_band(fc_handle *h, int32_t enabled) {
+  if (!h) return FC_ERR_INVALID_ARG;
+  h->band_form = enabled ? 1 : 0;
   return FC_OK;
 }
 

@@ -55,6 +55,7 @@ struct fc_handle {
   // fc_set_score_overlap: consecutive fc_score_layer calls keep running on the two internal streams
   // without rejoining the caller's stream; the join is made by the next call that consumes their results
   int score_overlap;
+  int band_form;           // 1: the chirp path may use its band form (fc_set_chirp_band)
   unsigned step;                 // specialised-path sequences scored so far (parity picks partial-sum buffers)
   long long last_sig;            // (N, heads, head_dim) of the previous specialised-path step
   bool pending_join;             // internal streams hold work the caller's stream has not waited for
@@ -66,7 +67,8 @@ struct fc_handle {
   // allocated by fc_create: FC_HHAT_SLOTS x hhat_cache_len points; hhat_cache_n[i] = length in slot i, 0 = none;
   // slots are reused round robin)
   float2 *hhat_cache;
-  int hhat_cache_len, hhat_cache_n[FC_HHAT_SLOTS], hhat_cache_next;
+  int hhat_cache_len, hhat_cache_next;
+  long long hhat_cache_n[FC_HHAT_SLOTS];   // key of slot i: length + ((band + 1) << 32), 0 = none
   cudaStream_t host_copy;
   cudaEvent_t *host_ev;
   int host_ev_cap;

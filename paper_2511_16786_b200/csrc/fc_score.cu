@@ -148,15 +148,22 @@ struct FilterLoader {
 };
 
 // Bluestein convolution kernel h[p] = chirp(|p|) wrapped to length M, in column 0.
+// band >= 0: the kernel of the band form, g[j] = chirp(|j - band|) for j = -(N-1) .. 2*band, wrapped (outputs
+// 0 .. 2*band of the convolution are the bins -band .. band; needs M >= N + 2*band).
 struct ChirpKernelLoader {
   static constexpr int VEC = 2;
-  int N, M;
+  int N, M, band;
   __device__ void init() {}
   __device__ void load(int p, int gc, float2 (&out)[2]) {
     out[0] = out[1] = make_float2(0.f, 0.f);
     if (gc != 0) return;
-    if (p < N) out[0] = chirp(p, N);
-    else if (p > M - N) out[0] = chirp(M - p, N);
+    if (band < 0) {
+      if (p < N) out[0] = chirp(p, N);
+      else if (p > M - N) out[0] = chirp(M - p, N);
+    } else {
+      if (p <= 2 * band) out[0] = chirp(p < band ? band - p : p - band, N);
+      else if (p > M - N) out[0] = chirp(band + (M - p), N);
+    }
   }
 };
 
@@ -614,19 +621,9 @@ struct SeqPlan {
   int cs, cs2;               // columns per tile in pass 1/3 and pass 2
 };
 
-SeqPlan plan_sequence(int N, bool allow_fast = true) {
-  SeqPlan s;
-  s.N = N;
-  s.bluestein = !(is_pow2(N) && N >= 16);
-  if (s.bluestein) {
-    int M = 64;
-    while (M < 2 * N - 1) M <<= 1;
-    s.Nfft = M;
-  } else {
-    s.Nfft = N;
-  }
+// Factors and tile widths of the generic kernels for the transform length s.Nfft.
+void finish_plan(SeqPlan &s) {
   const int bits = ilog2(s.Nfft);
-  s.fast = allow_fast && !s.bluestein && N >= 1024 && N <= 65536;
   int b1 = bits / 2;
   if (b1 > 7 && !s.fast) b1 = 7;
   s.cs = 64;
@@ -639,7 +636,31 @@ SeqPlan plan_sequence(int N, bool allow_fast = true) {
   if (cs2 > 64) cs2 = 64;
   if (cs2 < 4) cs2 = 4;
   s.cs2 = cs2;
+}
+
+SeqPlan plan_sequence(int N, bool allow_fast = true) {
+  SeqPlan s;
+  s.N = N;
+  s.bluestein = !(is_pow2(N) && N >= 16);
+  if (s.bluestein) {
+    int M = 64;
+    while (M < 2 * N - 1) M <<= 1;
+    s.Nfft = M;
+  } else {
+    s.Nfft = N;
+  }
+  s.fast = allow_fast && !s.bluestein && N >= 1024 && N <= 65536;
+  finish_plan(s);
   return s;
+}
+
+// Transform length of the band form of the chirp path (bins -omega .. omega only), or 0 where it does not apply:
+// the band must not wrap (2*omega + 1 < N) and the shorter length must be one the specialised kernels take.
+int band_length(int N, int omega, int full) {
+  if (2 * (long long)omega + 1 >= N) return 0;
+  int M = 1024;
+  while (M < N + 2 * omega + 1) M <<= 1;
+  return M < full ? M : 0;
 }
 
 struct ScoreLayout {
@@ -873,7 +894,7 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
 template <typename T, int R1B, int R2B, bool DOUBLE = false>
 fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq,
                             int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
-                            double *phi, float *scores, long long total_tokens, int dcols, int accumulate) {
+                            double *phi, float *scores, long long total_tokens, int dcols, int accumulate, int band) {
   constexpr int CPW = 32, CP = 8, N1 = 16 * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
   constexpr int MIDV = DOUBLE ? fast::MID_CONV2 : fast::MID_CONV;
   // dcols: columns of a head in this launch (head_dim, or a column group of one head: kp/vp point at its
@@ -889,6 +910,10 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   if ((s = set_smem(fast::k_p2<R2B, CP, MIDV>, sm2)) != FC_OK) return s;
   if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SPEC>, sm1)) != FC_OK) return s;
   if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP>, sm1)) != FC_OK) return s;
+  if (band >= 0) {
+    if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_BAND>, sm1)) != FC_OK) return s;
+    if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T>, sm1)) != FC_OK) return s;
+  }
   {
     ProfScope ps(h, FC_K_PASS1, st);
     fast::k_p1<T, R1B, CPW, fast::LD_CHIRP><<<g1, CPW * R1B, sm1, st>>>(
@@ -904,26 +929,40 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
     ProfScope ps(h, FC_K_PASS3, st);
     fast::k_p3<R1B, CPW, fast::OUT_SPEC><<<g3, CPW * R1B, sm1, st>>>(
         Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, h0, dcols, 0, 0.f, nullptr, nullptr, 0u, nullptr, 0, nullptr, 0,
-        nullptr, spec);
+        nullptr, spec, 0.f, 0, band);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS1, st);
-    fast::k_p1<float, R1B, CPW, fast::LD_FILTER><<<g1, CPW * R1B, sm1, st>>>(
-        nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, omega);
+    if (band >= 0)
+      fast::k_p1<float, R1B, CPW, fast::LD_BAND><<<g1, CPW * R1B, sm1, st>>>(
+          nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, band);
+    else
+      fast::k_p1<float, R1B, CPW, fast::LD_FILTER><<<g1, CPW * R1B, sm1, st>>>(
+          nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, omega);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
+    // band form: the second convolution's kernel is the first one's read backwards, whose spectrum is hhat read
+    // backwards
     ProfScope ps(h, FC_K_PASS2, st);
-    fast::k_p2<R2B, CP, MIDV><<<g2, 2 * CP * R2B, sm2, st>>>(N1, ncol, ws, h->master, h->master_len, 0, hhat, invM);
+    fast::k_p2<R2B, CP, MIDV><<<g2, 2 * CP * R2B, sm2, st>>>(N1, ncol, ws, h->master, h->master_len, 0, hhat, invM,
+                                                             band >= 0 ? 1 : 0);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS3, st);
-    const float inv = (float)(1.0 / ((double)Nseq * (double)Nseq * (double)d));
-    fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP><<<g3, CPW * R1B, sm1, st>>>(
-        Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, dcols, total_tokens, inv, phi, nullptr, 0u, nullptr, 0,
-        nullptr, 0, nullptr, nullptr, (float)d, accumulate);
+    if (band >= 0) {
+      fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T><<<g3, CPW * R1B, sm1, st>>>(
+          Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, dcols, total_tokens, (float)(1.0 / (double)d), phi,
+          nullptr, 0u, nullptr, 0, nullptr, 0, nullptr, nullptr, (float)d, accumulate, band, kp, vp, kv->stride_token,
+          kv->stride_head);
+    } else {
+      const float inv = (float)(1.0 / ((double)Nseq * (double)Nseq * (double)d));
+      fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP><<<g3, CPW * R1B, sm1, st>>>(
+          Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, dcols, total_tokens, inv, phi, nullptr, 0u, nullptr, 0,
+          nullptr, 0, nullptr, nullptr, (float)d, accumulate);
+    }
   }
   return fc_after_launch(h);
 }
@@ -941,19 +980,19 @@ inline void fast_factors(int M, int *r1b, int *r2b) {
 template <typename T>
 fc_status launch_chirp(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq, int M,
                        int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
-                       double *phi, float *scores, long long total_tokens, int dcols, int accumulate) {
+                       double *phi, float *scores, long long total_tokens, int dcols, int accumulate, int band) {
   int a, b;
   fast_factors(M, &a, &b);
 #define FC_CHIRP_CASE(A, B)                                                                                  \
   if (a == A && b == B)                                                                                      \
     return launch_chirp_impl<T, A, B>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, scores, \
-                                      total_tokens, dcols, accumulate);
+                                      total_tokens, dcols, accumulate, band);
   FC_CHIRP_CASE(2, 2) FC_CHIRP_CASE(2, 4) FC_CHIRP_CASE(4, 4) FC_CHIRP_CASE(4, 8)
   FC_CHIRP_CASE(8, 8) FC_CHIRP_CASE(8, 16) FC_CHIRP_CASE(16, 16)
 #undef FC_CHIRP_CASE
   if (a == 16 && b == 32)
     return launch_chirp_impl<T, 16, 16, true>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, scores,
-                                              total_tokens, dcols, accumulate);
+                                              total_tokens, dcols, accumulate, band);
   return FC_ERR_INTERNAL;
 }
 
@@ -995,6 +1034,19 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   const FftPlan p1 = make_plan(sp.N1);
   fc_status s;
 
+  // Band form of the chirp path: only the bins -omega .. omega of the spectrum are needed (the low-pass part; the
+  // score is taken against the input rows), which lets the convolutions run at a length >= N + 2*omega + 1 instead
+  // of 2N - 1.  Used where that length is a shorter power of two and the specialised kernels take the shape.
+  int band = -1, Mc = sp.Nfft;
+  if (sp.bluestein && !h->generic_only && L.sub_cols % 64 == 0) {
+    int fa = 0, fb = 0;
+    const int Mb = band_length(N, omega, sp.Nfft);
+    if (Mb != 0) fast_factors(Mb, &fa, &fb);
+    if (fa != 0 && h->band_form) { band = omega; Mc = Mb; }
+  }
+  SeqPlan spc = sp;                      // plan of the convolution length
+  if (band >= 0) { spc.Nfft = Mc; finish_plan(spc); }
+
   if (sp.bluestein) {
     // Spectrum of the chirp kernel.  It depends on the sequence length only, so the handle keeps the last few
     // (layers of a prefill share their lengths).  While the stream is being captured the spectrum goes to the
@@ -1007,9 +1059,10 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
     }
     bool have = false;
     int slot = 0;
+    const long long hkey = (long long)N + ((long long)(band + 1) << 32);
     if (cached) {
       for (int i = 0; i < FC_HHAT_SLOTS && !have; ++i)
-        if (h->hhat_cache_n[i] == N) { have = true; slot = i; }
+        if (h->hhat_cache_n[i] == hkey) { have = true; slot = i; }
       if (!have) {
         // the slot taken over was last read by a sequence that has been joined to `st` since (the chirp path
         // joins the internal streams before it returns), so stream order protects it
@@ -1020,10 +1073,10 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       hhat = h->hhat_cache + (size_t)slot * h->hhat_cache_len;
     }
     if (!have) {
-      ChirpKernelLoader cl{N, sp.Nfft};
-      if ((s = launch_pass1(h, st, cl, sp, 8, 8, hcol, nullptr)) != FC_OK) return s;
-      if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
-      if (cached) h->hhat_cache_n[slot] = N;
+      ChirpKernelLoader cl{N, Mc, band};
+      if ((s = launch_pass1(h, st, cl, spc, 8, 8, hcol, nullptr)) != FC_OK) return s;
+      if ((s = launch_pass2<MID_SPEC>(h, st, spc, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
+      if (cached) h->hhat_cache_n[slot] = hkey;
     }
   }
 
@@ -1102,7 +1155,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       // length-Nfft intermediates of a group stay within the cache budget; the groups run in
       // stream order and the last pass adds their contributions to the score in that order.
       int fa, fb;
-      fast_factors(sp.Nfft, &fa, &fb);
+      fast_factors(Mc, &fa, &fb);
       if (fa != 0 && !h->generic_only && L.sub_cols % 64 == 0) {   // a length and a width the specialised kernels take
         const int sub = L.sub_cols, ngr = (hg == 1) ? d / sub : 1, n2f = 16 * fb;
         const int ncol = (hg == 1) ? sub : ncol_ws;
@@ -1111,9 +1164,9 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
         float2 *ws_s = reinterpret_cast<float2 *>(wsb + L.off_ws + (size_t)si * L.ws_buf_bytes);
         float2 *spec_s = reinterpret_cast<float2 *>(wsb + L.off_spec + (size_t)si * L.spec_buf_bytes);
         for (int cg = 0; cg < ngr; ++cg) {                        // column groups of one head, else one pass
-          if ((s = launch_chirp<T>(h, sx, kv, kp + cg * sub, vp + cg * sub, N, sp.Nfft, h0, hg, omega, ws_s, spec_s, hhat,
+          if ((s = launch_chirp<T>(h, sx, kv, kp + cg * sub, vp + cg * sub, N, Mc, h0, hg, omega, ws_s, spec_s, hhat,
                                    ptot + 2 * (size_t)cg * n2f * (ncol / 64), phi + 2 * (size_t)cg * n2f * hg,
-                                   scores + start, total_tokens, (hg == 1) ? sub : d, cg > 0 ? 1 : 0)) != FC_OK)
+                                   scores + start, total_tokens, (hg == 1) ? sub : d, cg > 0 ? 1 : 0, band)) != FC_OK)
             return s;
         }
         tot_slots += (size_t)n2f * (ncol / 64) * ngr;
@@ -1210,7 +1263,7 @@ fc_status power_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   const FftPlan p1 = make_plan(sp.N1);
   fc_status s;
   if (sp.bluestein) {
-    ChirpKernelLoader cl{N, sp.Nfft};
+    ChirpKernelLoader cl{N, sp.Nfft, -1};
     if ((s = launch_pass1(h, st, cl, sp, 8, 8, hcol, nullptr)) != FC_OK) return s;
     if ((s = launch_pass2<MID_SPEC>(h, st, sp, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
   }

@@ -56,7 +56,11 @@ __device__ __forceinline__ float2 chirp_f(int n, int N) {
 //   LD_FILTER : chirp convolution, second half: the N-point spectrum spec[q][col] through the low-pass
 //               residual filter, conjugated (an inverse DFT is the conjugate of the forward DFT of the
 //               conjugate) and times conj(chirp), zeros behind.
-enum { LD_KV = 0, LD_CHIRP = 1, LD_FILTER = 2 };
+//   LD_BAND   : as LD_FILTER for the band form of the chirp path: spec holds only the 2*band+1 bins q = -band..band
+//               of the N-point spectrum (row q + band); the input is conj(Wb[q]) * conj(chirp(q)) with the low-pass
+//               part Wb[q] = (W[q] + exp(j*pi*q/N) W[-q]) / 2 (one formula for both signs of q and for q = 0),
+//               zeros behind.  `omega` carries the band.
+enum { LD_KV = 0, LD_CHIRP = 1, LD_FILTER = 2, LD_BAND = 3 };
 // What pass 2 does between its forward and inverse halves: the DCT/low-pass residual filter on paired rows,
 // or a multiplication by the spectrum of the chirp kernel (rows 2x and 2x+1, unrelated).  MID_CONV2 is the
 // convolution for rows of 2*N2 points: the two halves of the block take the even and the odd samples of ONE
@@ -65,7 +69,9 @@ enum { LD_KV = 0, LD_CHIRP = 1, LD_FILTER = 2 };
 enum { MID_FILTER = 0, MID_CONV = 1, MID_CONV2 = 2 };
 // What pass 3 does with the rows it gets back: scores of a power-of-two sequence, the N-point spectrum of
 // the chirp path (rows < N times conj(chirp)), or the scores at the end of the chirp path.
-enum { OUT_SCORE = 0, OUT_SPEC = 1, OUT_SCORE_CHIRP = 2 };
+// OUT_SCORE_BAND: end of the band form: the rows are N times the conjugate of the Base KV (low-pass part) in the
+// reordered domain; the K/V rows are read again and the score is |z - z_base|^2.
+enum { OUT_SCORE = 0, OUT_SPEC = 1, OUT_SCORE_CHIRP = 2, OUT_SCORE_BAND = 3 };
 
 template <int R>
 __device__ __forceinline__ void dft_fwd(float2 (&x)[R]) { dft_small<R, -1>(x); }
@@ -114,6 +120,22 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
         const float2 ch = chirp_f(n, N);
         x0[p] = cmul_conj(make_float2(kk.x, vv.x), ch);
         x1[p] = cmul_conj(make_float2(kk.y, vv.y), ch);
+      }
+    } else if (LD == LD_BAND) {
+      x0[p] = x1[p] = make_float2(0.f, 0.f);
+      const int band = omega;
+      if (n <= 2 * band) {
+        const int q = n - band;
+        const float4 P4 = *reinterpret_cast<const float4 *>(spec + (size_t)n * ncol_ws + gc0 + 2 * cp);
+        const float4 Q4 = *reinterpret_cast<const float4 *>(spec + (size_t)(2 * band - n) * ncol_ws + gc0 + 2 * cp);
+        float sn, cs;
+        sincospif(__fdiv_rn((float)q, (float)N), &sn, &cs);
+        const float2 u = make_float2(cs, sn);
+        const float2 ch = chirp_f(q < 0 ? -q : q, N);
+        const float2 W0 = cscale(cadd(make_float2(P4.x, P4.y), cmul(make_float2(Q4.x, Q4.y), u)), 0.5f);
+        const float2 W1 = cscale(cadd(make_float2(P4.z, P4.w), cmul(make_float2(Q4.z, Q4.w), u)), 0.5f);
+        x0[p] = cmul_conj(cconj(W0), ch);
+        x1[p] = cmul_conj(cconj(W1), ch);
       }
     } else {
       x0[p] = x1[p] = make_float2(0.f, 0.f);
@@ -177,7 +199,7 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
       *dst = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
     }
   }
-  if (LD == LD_FILTER) return;
+  if (LD == LD_FILTER || LD == LD_BAND) return;
   // per-block sums of squares (total energy of Eq. 12, by Parseval)
   const double a = warp_sum_d((double)accK), b = warp_sum_d((double)accV);
   if ((tid & 31) == 0) { red[0][tid >> 5] = a; red[1][tid >> 5] = b; }
@@ -201,7 +223,8 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
 template <int R2B, int CP, int MID = MID_FILTER>
 __global__ void __launch_bounds__(2 * CP * R2B, 512 / (2 * CP * R2B > 32 ? 2 * CP * R2B : 32))
 k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ master, int master_len,
-     int omega, const float2 *__restrict__ hhat = nullptr, float scale = 1.f) {
+     int omega, const float2 *__restrict__ hhat = nullptr, float scale = 1.f, int hrev = 0) {
+  // hrev (convolution variants): multiply by the spectrum of the index-reversed kernel, hhat[(-bin) mod N]
   constexpr int N2 = 16 * R2B, NT = 2 * CP * R2B, IT = 16 / R2B;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                         // [2][N2][CP]
@@ -306,7 +329,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
         const int k2 = pp + 16 * q;
         const int bin = k1 + N1 * k2;
         if (MID == MID_CONV) {
-          const float2 hq = cscale(__ldg(hhat + bin), scale);
+          const float2 hq = cscale(__ldg(hhat + (hrev ? ((N - bin) & (N - 1)) : bin)), scale);
           x0[it * R2B + q] = cmul(x0[it * R2B + q], hq);
           x1[it * R2B + q] = cmul(x1[it * R2B + q], hq);
           continue;
@@ -318,7 +341,8 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
           float2 &m0 = x0[it * R2B + q], &m1 = x1[it * R2B + q];
           const float2 e0 = hf ? make_float2(t.x, t.y) : m0, e1 = hf ? make_float2(t.z, t.w) : m1;
           const float2 o0 = cmul(hf ? m0 : make_float2(t.x, t.y), w), o1 = cmul(hf ? m1 : make_float2(t.z, t.w), w);
-          const float2 hq = cscale(__ldg(hhat + k1 + N1 * (k2 + hf * N2)), scale);
+          const int binh = k1 + N1 * (k2 + hf * N2);
+          const float2 hq = cscale(__ldg(hhat + (hrev ? ((N - binh) & (N - 1)) : binh)), scale);
           m0 = cmul(hf ? csub(e0, o0) : cadd(e0, o0), hq);
           m1 = cmul(hf ? csub(e1, o1) : cadd(e1, o1), hq);
           continue;
@@ -428,14 +452,19 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
 // OUT_SPEC and OUT_SCORE_CHIRP: N is the sequence length (< N1*N2), rows at or past it are dropped;
 // OUT_SPEC stores to spec[row][col] and returns; OUT_SCORE_CHIRP is given done_counter == nullptr and
 // leaves the final energy sums to the caller.
-template <int R1B, int CPW, int OUT = OUT_SCORE>
+// band >= 0 (band form of the chirp path): OUT_SPEC keeps rows 0 .. 2*band (bin q = row - band, rotated by
+// conj(chirp(|q|))); OUT_SCORE_BAND reads the K/V rows again (kin/vin: first token of the sequence, first channel of
+// the column group) and scores |z - z_base|^2 with z_base = conj(row * conj(chirp)) / N.
+template <int R1B, int CPW, int OUT = OUT_SCORE, typename T = float>
 __global__ void __launch_bounds__(CPW * R1B)
 k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__restrict__ master,
      int master_len, float *__restrict__ scores, int head0, int head_dim, long long score_stride,
      float inv_scale, double *__restrict__ partial, unsigned *__restrict__ done_counter,
      unsigned total_blocks, const double *__restrict__ part_tot, int n_tot,
      const double *__restrict__ part_hi, int n_hi, double *__restrict__ energy,
-     float2 *__restrict__ spec = nullptr, float energy_scale = 0.f, int accumulate = 0) {
+     float2 *__restrict__ spec = nullptr, float energy_scale = 0.f, int accumulate = 0, int band = -1,
+     const T *__restrict__ kin = nullptr, const T *__restrict__ vin = nullptr, long long stride_token = 0,
+     long long stride_head = 0) {
   // OUT_SCORE_CHIRP with a head transformed in column groups: head_dim is the group's width, energy_scale the
   // head's true channel count, and every group after the first adds to the stored score (accumulate).
   constexpr int N1 = 16 * R1B, NT = CPW * R1B, IT = 16 / R1B, NW = (NT + 31) / 32;
@@ -492,14 +521,29 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
     for (int p = 0; p < 16; ++p) {
       if (OUT != OUT_SCORE) {
         const int pos = (j + R1B * p) * N2 + n2;
-        if (pos >= N) continue;
-        const float2 ch = chirp_f(pos, N);
+        if (OUT == OUT_SPEC && band >= 0) {
+          if (pos > 2 * band) continue;
+        } else if (pos >= N) {
+          continue;
+        }
+        const int cpos = (OUT == OUT_SPEC && band >= 0) ? (pos < band ? band - pos : pos - band) : pos;
+        const float2 ch = chirp_f(cpos, N);
         x0[p] = cmul_conj(x0[p], ch);
         x1[p] = cmul_conj(x1[p], ch);
         if (OUT == OUT_SPEC) {
           *reinterpret_cast<float4 *>(spec + (size_t)pos * ncol_ws + gc0 + 2 * cp) =
               make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
           continue;
+        }
+        if (OUT == OUT_SCORE_BAND) {
+          // residual against the input rows: z_base = conj(x) / N (inv_scale carries 1/d only)
+          const int col = gc0 + 2 * cp;
+          const long long off = (long long)perm_token(pos, N) * stride_token +
+                                (long long)(head0 + col / head_dim) * stride_head + col % head_dim;
+          const float2 kk = Load2<T>::ld(kin + off), vv = Load2<T>::ld(vin + off);
+          const float rn = 1.f / (float)N;
+          x0[p] = make_float2(fmaf(-x0[p].x, rn, kk.x), fmaf(x0[p].y, rn, vv.x));
+          x1[p] = make_float2(fmaf(-x1[p].x, rn, kk.y), fmaf(x1[p].y, rn, vv.y));
         }
       }
       const float ek = fmaf(x0[p].x, x0[p].x, x1[p].x * x1[p].x);
@@ -551,13 +595,13 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
 #pragma unroll
     for (int i = 0; i < NW; ++i) { sa += red[0][i]; sb += red[1][i]; }
     const size_t slot = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
-    const double es = (OUT == OUT_SCORE_CHIRP) ? (double)energy_scale : (double)head_dim;
+    const double es = (OUT == OUT_SCORE_CHIRP || OUT == OUT_SCORE_BAND) ? (double)energy_scale : (double)head_dim;
     partial[2 * slot] = sa * es;
     partial[2 * slot + 1] = sb * es;
   }
   // The last block of the sequence (over all head groups, on either stream) adds up the
   // per-block partial sums in a fixed order: energy = (hiK, totK, hiV, totV).
-  if (OUT == OUT_SCORE_CHIRP) return;
+  if (OUT == OUT_SCORE_CHIRP || OUT == OUT_SCORE_BAND) return;
   __shared__ bool is_last;
   if (tid == 0) {
     __threadfence();

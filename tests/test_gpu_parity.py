@@ -40,13 +40,15 @@ def _rand_kv(T, H, d, dtype, seed, smooth=True):
     return k.to(dtype), v.to(dtype)
 
 
-def _gpu_scores(fc, k, v, cu, gamma, max_seqlen=None, group_bytes=None):
+def _gpu_scores(fc, k, v, cu, gamma, max_seqlen=None, group_bytes=None, band=None):
     T, H, d = k.shape
     seqlens = [cu[i + 1] - cu[i] for i in range(len(cu) - 1)]
     h = fc.fc_create(0, max_seqlen or max(1, max(seqlens, default=1)))
     try:
         if group_bytes:
             fc.fc_set_group_bytes(h, group_bytes)
+        if band is not None:
+            fc.fc_set_chirp_band(h, band)
         kd, vd = (k if k.is_cuda else k.cuda()), (v if v.is_cuda else v.cuda())
         scores = torch.full((H, max(T, 1)), -1.0, dtype=torch.float32, device="cuda")
         energy = torch.full((len(cu) - 1, 4), -1.0, dtype=torch.float64, device="cuda")
@@ -181,9 +183,38 @@ def test_scores_mixed_paths_in_one_call(fc):
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.float16])
 def test_scores_131072_point_chirp_transform(fc, dtype):
+    # full-length form (all N bins): 2N - 1 pads to 131072
     N = 33001
     k, v = _rand_kv(N, 2, 128, dtype, 13)
-    _check_layer(fc, k, v, [0, N], 0.2)
+    _check_layer(fc, k, v, [0, N], 0.2, band=False)
+
+
+@pytest.mark.parametrize("N,gamma,d,group_bytes", [
+    (2500, 0.2, 128, None),      # N + 2*omega + 1 = 3501 -> 4096 points instead of 8192
+    (2500, 0.0, 64, None),       # band of one bin (the mean)
+    (5000, 0.3, 128, None),      # 8001 -> 8192 instead of 16384
+    (5000, 0.1, 192, 1),         # heads in column groups
+    (1367, 0.25, 64, None),      # 2051 -> 4096: band form does not apply (same length), full form runs
+    (33001, 0.2, 128, None),     # 46202 -> 65536 instead of 131072
+    (46800, 0.2, 64, None),      # 65521 -> 65536: the longest sequence the band form shortens at this cutoff
+])
+def test_scores_chirp_band_form(fc, N, gamma, d, group_bytes):
+    # The band form of the chirp path (bins -omega .. omega, Base KV transformed back, score against the input
+    # rows) and the full-length form both match the oracle, and each other.
+    k, v = _rand_kv(N, 2, d, torch.float32, 500 + N)
+    g1, e1 = _check_layer(fc, k, v, [0, N], gamma, band=True, group_bytes=group_bytes)
+    g2, e2 = _check_layer(fc, k, v, [0, N], gamma, band=False, group_bytes=group_bytes)
+    np.testing.assert_allclose(g1, g2, rtol=2e-3, atol=1e-6 * float(g2.max()))
+    np.testing.assert_allclose(e1, e2, rtol=1e-4)
+
+
+def test_scores_chirp_band_form_16bit_ragged(fc):
+    lens = [2500, 1024, 5000, 40961, 300]
+    cu = [0] + [int(x) for x in np.cumsum(lens)]
+    k, v = _rand_kv(cu[-1], 4, 128, torch.bfloat16, 77)
+    g1, e1 = _check_layer(fc, k, v, cu, 0.2, max_seqlen=65536)
+    g2, e2 = _gpu_scores(fc, k, v, cu, 0.2, max_seqlen=65536)
+    assert np.array_equal(g1, g2) and np.array_equal(e1, e2)
 
 
 @pytest.mark.parametrize("d,group_bytes", [(128, 1), (128, 1 << 20), (192, 1), (64, 1)])
