@@ -200,12 +200,106 @@ __device__ __forceinline__ void dft16(float2 (&x)[16]) {
   for (int k = 0; k < 8; ++k) { x[k] = cadd(e[k], t[k]); x[k + 8] = csub(e[k], t[k]); }
 }
 
+// Odd lengths by the symmetric form: with a_m = x[m] + x[P-m], b_m = x[m] - x[P-m],
+//   y[k], y[P-k] = x[0] + sum_m cos(2*pi*k*m/P) a_m  +/-  DIR*j * sum_m sin(2*pi*k*m/P) b_m.
+template <int DIR>
+__device__ __forceinline__ void dft3(float2 &x0, float2 &x1, float2 &x2) {
+  const float s = 0.86602540378443864676f;
+  const float2 a = cadd(x1, x2), b = csub(x1, x2);
+  const float2 r = make_float2(fmaf(-0.5f, a.x, x0.x), fmaf(-0.5f, a.y, x0.y));
+  const float2 i = mul_j<DIR>(cscale(b, s));
+  x0 = cadd(x0, a);
+  x1 = cadd(r, i);
+  x2 = csub(r, i);
+}
+
+template <int DIR>
+__device__ __forceinline__ void dft5(float2 (&x)[5]) {
+  const float c1 = 0.30901699437494742410f, c2 = -0.80901699437494742410f;
+  const float s1 = 0.95105651629515357212f, s2 = 0.58778525229247312917f;
+  const float2 a1 = cadd(x[1], x[4]), a2 = cadd(x[2], x[3]), b1 = csub(x[1], x[4]), b2 = csub(x[2], x[3]);
+  const float2 r1 = make_float2(fmaf(c1, a1.x, fmaf(c2, a2.x, x[0].x)), fmaf(c1, a1.y, fmaf(c2, a2.y, x[0].y)));
+  const float2 r2 = make_float2(fmaf(c2, a1.x, fmaf(c1, a2.x, x[0].x)), fmaf(c2, a1.y, fmaf(c1, a2.y, x[0].y)));
+  const float2 i1 = mul_j<DIR>(make_float2(fmaf(s1, b1.x, s2 * b2.x), fmaf(s1, b1.y, s2 * b2.y)));
+  const float2 i2 = mul_j<DIR>(make_float2(fmaf(s2, b1.x, -s1 * b2.x), fmaf(s2, b1.y, -s1 * b2.y)));
+  x[0] = cadd(x[0], cadd(a1, a2));
+  x[1] = cadd(r1, i1); x[4] = csub(r1, i1);
+  x[2] = cadd(r2, i2); x[3] = csub(r2, i2);
+}
+
+template <int DIR>
+__device__ __forceinline__ void dft7(float2 (&x)[7]) {
+  // cos and sin of 2*pi*i/7, i = 1..3
+  const float c[3] = {0.62348980185873353053f, -0.22252093395631440429f, -0.90096886790241912624f};
+  const float s[3] = {0.78183148246802980871f, 0.97492791218182360702f, 0.43388373911755812048f};
+  float2 a[3], b[3];
+#pragma unroll
+  for (int m = 0; m < 3; ++m) { a[m] = cadd(x[m + 1], x[6 - m]); b[m] = csub(x[m + 1], x[6 - m]); }
+  const float2 x0 = x[0];
+  x[0] = cadd(x0, cadd(a[0], cadd(a[1], a[2])));
+#pragma unroll
+  for (int k = 1; k <= 3; ++k) {
+    float2 r = x0, im = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int m = 1; m <= 3; ++m) {
+      const int idx = (k * m) % 7;                       // 1..6; cos is even, sin odd about 7/2
+      const float cc = idx <= 3 ? c[idx - 1] : c[6 - idx];
+      const float ss = idx <= 3 ? s[idx - 1] : -s[6 - idx];
+      r = make_float2(fmaf(cc, a[m - 1].x, r.x), fmaf(cc, a[m - 1].y, r.y));
+      im = make_float2(fmaf(ss, b[m - 1].x, im.x), fmaf(ss, b[m - 1].y, im.y));
+    }
+    const float2 i = mul_j<DIR>(im);
+    x[k] = cadd(r, i);
+    x[7 - k] = csub(r, i);
+  }
+}
+
+template <int R, int DIR>
+__device__ __forceinline__ void dft_small(float2 (&x)[R]);
+
+// R = R1*R2 with coprime factors (prime-factor mapping, no twiddles between the two stages):
+// input n = (n1*R2 + n2*R1) mod R, output k with k = k1 (mod R1) and k = k2 (mod R2).
+template <int R1, int R2, int DIR>
+__device__ __forceinline__ void dft_coprime(float2 (&x)[R1 * R2]) {
+  constexpr int R = R1 * R2;
+  float2 t[R1][R2];
+#pragma unroll
+  for (int n1 = 0; n1 < R1; ++n1) {
+#pragma unroll
+    for (int n2 = 0; n2 < R2; ++n2) t[n1][n2] = x[(n1 * R2 + n2 * R1) % R];
+    dft_small<R2, DIR>(t[n1]);
+  }
+#pragma unroll
+  for (int k2 = 0; k2 < R2; ++k2) {
+    float2 col[R1];
+#pragma unroll
+    for (int n1 = 0; n1 < R1; ++n1) col[n1] = t[n1][k2];
+    dft_small<R1, DIR>(col);
+#pragma unroll
+    for (int k1 = 0; k1 < R1; ++k1) {
+      int k = k1;                                        // smallest k = k1 (mod R1) with k = k2 (mod R2)
+#pragma unroll
+      for (int i = 0; i < R2; ++i) if (k % R2 != k2) k += R1;
+      x[k] = col[k1];
+    }
+  }
+}
+
 template <int R, int DIR>
 __device__ __forceinline__ void dft_small(float2 (&x)[R]) {
   if constexpr (R == 2) dft2<DIR>(x[0], x[1]);
+  else if constexpr (R == 3) dft3<DIR>(x[0], x[1], x[2]);
   else if constexpr (R == 4) dft4<DIR>(x[0], x[1], x[2], x[3]);
+  else if constexpr (R == 5) dft5<DIR>(x);
+  else if constexpr (R == 7) dft7<DIR>(x);
   else if constexpr (R == 8) dft8<DIR>(x);
-  else dft16<DIR>(x);
+  else if constexpr (R == 10) dft_coprime<2, 5, DIR>(x);
+  else if constexpr (R == 12) dft_coprime<4, 3, DIR>(x);
+  else if constexpr (R == 14) dft_coprime<2, 7, DIR>(x);
+  else {
+    static_assert(R == 16, "unsupported small DFT length");
+    dft16<DIR>(x);
+  }
 }
 
 // ------------------------------------------------------------------ batched stages in shared memory

@@ -654,15 +654,6 @@ SeqPlan plan_sequence(int N, bool allow_fast = true) {
   return s;
 }
 
-// Transform length of the band form of the chirp path (bins -omega .. omega only), or 0 where it does not apply:
-// the band must not wrap (2*omega + 1 < N) and the shorter length must be one the specialised kernels take.
-int band_length(int N, int omega, int full) {
-  if (2 * (long long)omega + 1 >= N) return 0;
-  int M = 1024;
-  while (M < N + 2 * omega + 1) M <<= 1;
-  return M < full ? M : 0;
-}
-
 struct ScoreLayout {
   size_t off_ws, off_spec, off_hhat, off_hcol, off_part_tot, off_part_hi, total;
   size_t part_tot_bytes, part_hi_bytes;   // one copy; the specialised path keeps two and alternates (step parity)
@@ -887,36 +878,92 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
   return FC_ERR_INTERNAL;
 }
 
-// The chirp path on the specialised kernels, for transform lengths M = N1*N2 of 1024..65536 (sequence
-// lengths that are not a power of two, up to 32768): two circular convolutions with the chirp kernel, each
-// pass 1 -> pass 2 (multiply by the kernel's spectrum) -> pass 3, on the caller's stream.  Tile widths fixed.
-// DOUBLE: rows of 2 * 16 * R2B points, pass 2 joins two half-length transforms per row (131072 = 256 x 512).
-template <typename T, int R1B, int R2B, bool DOUBLE = false>
+// Shape of a chirp transform on the specialised kernels: M = N1 * N2 with N1 = a * r1b (first-stage radix a of
+// passes 1 and 3, then radix r1b) and N2 = 16 * r2b, or 2 * 16 * r2b when pass 2 takes its rows in two halves (dbl).
+// Powers of two 1024..131072 have a = 16; 2^k * {5, 3, 7} have a = 10, 12, 14 with r1b = 16.  a == 0: no such shape.
+struct ChirpShape {
+  int a, r1b, r2b;
+  bool dbl;
+  int n1() const { return a * r1b; }
+  int n2() const { return (dbl ? 32 : 16) * r2b; }
+};
+
+inline ChirpShape chirp_shape(int M) {
+  ChirpShape c{0, 0, 0, false};
+  if (M == 131072) return ChirpShape{16, 16, 16, true};          // 256 x 512
+  if (is_pow2(M)) {
+    if (M < 1024 || M > 65536) return c;
+    const int bits = ilog2(M), b1 = bits / 2;
+    return ChirpShape{16, (1 << b1) / 16, (M >> b1) / 16, false};
+  }
+  const int a = (M % 5 == 0) ? 10 : (M % 3 == 0) ? 12 : (M % 7 == 0) ? 14 : 0;
+  if (a == 0 || M % (16 * a) != 0) return c;
+  const int n2 = M / (16 * a);
+  if (!is_pow2(n2) || n2 < 32 || n2 > 512) return c;
+  return n2 == 512 ? ChirpShape{a, 16, 16, true} : ChirpShape{a, 16, n2 / 16, false};
+}
+
+// Smallest transform length >= need the specialised kernels take (0 if none up to 131072).
+inline int chirp_length(long long need) {
+  int best = 0;
+  for (int M = 1024; M <= 131072; M <<= 1)
+    if (M >= need) { best = M; break; }
+  for (int n1 = 160; n1 <= 224; n1 += 32)
+    for (int n2 = 32; n2 <= 512; n2 <<= 1) {
+      const int M = n1 * n2;
+      if (M >= need && (best == 0 || M < best)) best = M;
+    }
+  return best;
+}
+
+// The chirp path on the specialised kernels: two circular convolutions with the chirp kernel, each
+// pass 1 -> pass 2 (multiply by the kernel's spectrum) -> pass 3, on one stream.  Tile widths fixed.
+// DOUBLE: rows of 2 * 16 * R2B points, pass 2 joins two half-length transforms per row.
+// hout != nullptr: only the spectrum of the convolution kernel itself is computed (pass 1 with the kernel in column
+// 0 of a 64-column tile, the forward half of pass 2) and written to hout[0 .. M).
+template <typename T, int A, int R1B, int R2B, bool DOUBLE>
 fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq,
                             int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
-                            double *phi, float *scores, long long total_tokens, int dcols, int accumulate, int band) {
-  constexpr int CPW = 32, CP = 8, N1 = 16 * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
+                            double *phi, float *scores, long long total_tokens, int dcols, int accumulate, int band,
+                            float2 *hout) {
+  constexpr int CPW = 32, CP = 8, N1 = A * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
   constexpr int MIDV = DOUBLE ? fast::MID_CONV2 : fast::MID_CONV;
+  const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
+  const size_t sm2 = (size_t)2 * (16 * R2B) * CP * sizeof(float4) + 5 * (16 * R2B) * sizeof(float2);
+  fc_status s;
+  if ((s = set_smem(fast::k_p2<R2B, CP, MIDV>, sm2)) != FC_OK) return s;
+  if (hout != nullptr) {
+    if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_KERNEL, A>, sm1)) != FC_OK) return s;
+    {
+      ProfScope ps(h, FC_K_PASS1, st);
+      fast::k_p1<float, R1B, CPW, fast::LD_KERNEL, A><<<dim3(N2, 1), CPW * R1B, sm1, st>>>(
+          nullptr, nullptr, 0, 0, 0, 2 * CPW, Nseq, N2, 2 * CPW, ws, h->master, h->master_len, nullptr, nullptr, band);
+    }
+    if ((s = fc_after_launch(h)) != FC_OK) return s;
+    {
+      ProfScope ps(h, FC_K_PASS2, st);
+      fast::k_p2<R2B, CP, MIDV><<<dim3(DOUBLE ? N1 : N1 / 2, 1), 2 * CP * R2B, sm2, st>>>(
+          N1, 2 * CPW, ws, h->master, h->master_len, 0, nullptr, 1.f, 0, hout);
+    }
+    return fc_after_launch(h);
+  }
   // dcols: columns of a head in this launch (head_dim, or a column group of one head: kp/vp point at its
   // first channel and hg is 1)
   const int d = kv->head_dim, ncol = hg * dcols;
-  const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
-  const size_t sm2 = (size_t)2 * (16 * R2B) * CP * sizeof(float4) + 5 * (16 * R2B) * sizeof(float2);
   const float invM = 1.f / (float)(N1 * N2);
   const dim3 g1(N2, ncol / (2 * CPW)), g2(DOUBLE ? N1 : N1 / 2, ncol / (2 * CP)), g3(N2, hg);
-  fc_status s;
-  if ((s = set_smem(fast::k_p1<T, R1B, CPW, fast::LD_CHIRP>, sm1)) != FC_OK) return s;
-  if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_FILTER>, sm1)) != FC_OK) return s;
-  if ((s = set_smem(fast::k_p2<R2B, CP, MIDV>, sm2)) != FC_OK) return s;
-  if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SPEC>, sm1)) != FC_OK) return s;
-  if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP>, sm1)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p1<T, R1B, CPW, fast::LD_CHIRP, A>, sm1)) != FC_OK) return s;
+  if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SPEC, float, A>, sm1)) != FC_OK) return s;
   if (band >= 0) {
-    if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_BAND>, sm1)) != FC_OK) return s;
-    if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T>, sm1)) != FC_OK) return s;
+    if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_BAND, A>, sm1)) != FC_OK) return s;
+    if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T, A>, sm1)) != FC_OK) return s;
+  } else {
+    if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_FILTER, A>, sm1)) != FC_OK) return s;
+    if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP, float, A>, sm1)) != FC_OK) return s;
   }
   {
     ProfScope ps(h, FC_K_PASS1, st);
-    fast::k_p1<T, R1B, CPW, fast::LD_CHIRP><<<g1, CPW * R1B, sm1, st>>>(
+    fast::k_p1<T, R1B, CPW, fast::LD_CHIRP, A><<<g1, CPW * R1B, sm1, st>>>(
         kp, vp, kv->stride_token, kv->stride_head, h0, dcols, Nseq, N2, ncol, ws, h->master, h->master_len, ptot);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
@@ -927,7 +974,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS3, st);
-    fast::k_p3<R1B, CPW, fast::OUT_SPEC><<<g3, CPW * R1B, sm1, st>>>(
+    fast::k_p3<R1B, CPW, fast::OUT_SPEC, float, A><<<g3, CPW * R1B, sm1, st>>>(
         Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, h0, dcols, 0, 0.f, nullptr, nullptr, 0u, nullptr, 0, nullptr, 0,
         nullptr, spec, 0.f, 0, band);
   }
@@ -935,10 +982,10 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   {
     ProfScope ps(h, FC_K_PASS1, st);
     if (band >= 0)
-      fast::k_p1<float, R1B, CPW, fast::LD_BAND><<<g1, CPW * R1B, sm1, st>>>(
+      fast::k_p1<float, R1B, CPW, fast::LD_BAND, A><<<g1, CPW * R1B, sm1, st>>>(
           nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, band);
     else
-      fast::k_p1<float, R1B, CPW, fast::LD_FILTER><<<g1, CPW * R1B, sm1, st>>>(
+      fast::k_p1<float, R1B, CPW, fast::LD_FILTER, A><<<g1, CPW * R1B, sm1, st>>>(
           nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, omega);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
@@ -953,13 +1000,13 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   {
     ProfScope ps(h, FC_K_PASS3, st);
     if (band >= 0) {
-      fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T><<<g3, CPW * R1B, sm1, st>>>(
+      fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T, A><<<g3, CPW * R1B, sm1, st>>>(
           Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, dcols, total_tokens, (float)(1.0 / (double)d), phi,
           nullptr, 0u, nullptr, 0, nullptr, 0, nullptr, nullptr, (float)d, accumulate, band, kp, vp, kv->stride_token,
           kv->stride_head);
     } else {
       const float inv = (float)(1.0 / ((double)Nseq * (double)Nseq * (double)d));
-      fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP><<<g3, CPW * R1B, sm1, st>>>(
+      fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP, float, A><<<g3, CPW * R1B, sm1, st>>>(
           Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, dcols, total_tokens, inv, phi, nullptr, 0u, nullptr, 0,
           nullptr, 0, nullptr, nullptr, (float)d, accumulate);
     }
@@ -967,32 +1014,25 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   return fc_after_launch(h);
 }
 
-// Factors of the specialised kernels for a transform length (0, 0 when it has none).
-inline void fast_factors(int M, int *r1b, int *r2b) {
-  *r1b = *r2b = 0;
-  if (M == 131072) { *r1b = 16; *r2b = 32; return; }           // 256 x 512: pass 2 takes its rows in two halves
-  if (!is_pow2(M) || M < 1024 || M > 65536) return;
-  const int bits = ilog2(M), b1 = bits / 2;
-  *r1b = (1 << b1) / 16;
-  *r2b = (M >> b1) / 16;
-}
-
 template <typename T>
 fc_status launch_chirp(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq, int M,
                        int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
-                       double *phi, float *scores, long long total_tokens, int dcols, int accumulate, int band) {
-  int a, b;
-  fast_factors(M, &a, &b);
-#define FC_CHIRP_CASE(A, B)                                                                                  \
-  if (a == A && b == B)                                                                                      \
-    return launch_chirp_impl<T, A, B>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, scores, \
-                                      total_tokens, dcols, accumulate, band);
-  FC_CHIRP_CASE(2, 2) FC_CHIRP_CASE(2, 4) FC_CHIRP_CASE(4, 4) FC_CHIRP_CASE(4, 8)
-  FC_CHIRP_CASE(8, 8) FC_CHIRP_CASE(8, 16) FC_CHIRP_CASE(16, 16)
+                       double *phi, float *scores, long long total_tokens, int dcols, int accumulate, int band,
+                       float2 *hout = nullptr) {
+  const ChirpShape c = chirp_shape(M);
+#define FC_CHIRP_CASE(A, B, C, D)                                                                               \
+  if (c.a == A && c.r1b == B && c.r2b == C && c.dbl == D)                                                       \
+    return launch_chirp_impl<T, A, B, C, D>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, \
+                                            scores, total_tokens, dcols, accumulate, band, hout);
+  FC_CHIRP_CASE(16, 2, 2, false) FC_CHIRP_CASE(16, 2, 4, false) FC_CHIRP_CASE(16, 4, 4, false)
+  FC_CHIRP_CASE(16, 4, 8, false) FC_CHIRP_CASE(16, 8, 8, false) FC_CHIRP_CASE(16, 8, 16, false)
+  FC_CHIRP_CASE(16, 16, 16, false) FC_CHIRP_CASE(16, 16, 16, true)
+#define FC_CHIRP_MIXED(A)                                                                                       \
+  FC_CHIRP_CASE(A, 16, 2, false) FC_CHIRP_CASE(A, 16, 4, false) FC_CHIRP_CASE(A, 16, 8, false)                  \
+  FC_CHIRP_CASE(A, 16, 16, false) FC_CHIRP_CASE(A, 16, 16, true)
+  FC_CHIRP_MIXED(10) FC_CHIRP_MIXED(12) FC_CHIRP_MIXED(14)
+#undef FC_CHIRP_MIXED
 #undef FC_CHIRP_CASE
-  if (a == 16 && b == 32)
-    return launch_chirp_impl<T, 16, 16, true>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, scores,
-                                              total_tokens, dcols, accumulate, band);
   return FC_ERR_INTERNAL;
 }
 
@@ -1034,18 +1074,22 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   const FftPlan p1 = make_plan(sp.N1);
   fc_status s;
 
-  // Band form of the chirp path: only the bins -omega .. omega of the spectrum are needed (the low-pass part; the
-  // score is taken against the input rows), which lets the convolutions run at a length >= N + 2*omega + 1 instead
-  // of 2N - 1.  Used where that length is a shorter power of two and the specialised kernels take the shape.
+  // Convolution length of the chirp path.  Full form: M >= 2N - 1.  Band form: only the bins -omega .. omega of the
+  // spectrum are needed (the low-pass part; the score is taken against the input rows), M >= N + 2*omega + 1.  The
+  // specialised kernels take powers of two and 2^k * {3, 5, 7}; whichever form gives the shorter M runs, and the
+  // generic kernels (M = sp.Nfft, a power of two) remain for what the specialised ones do not take.
   int band = -1, Mc = sp.Nfft;
+  bool chirp_fast = false;
   if (sp.bluestein && !h->generic_only && L.sub_cols % 64 == 0) {
-    int fa = 0, fb = 0;
-    const int Mb = band_length(N, omega, sp.Nfft);
-    if (Mb != 0) fast_factors(Mb, &fa, &fb);
-    if (fa != 0 && h->band_form) { band = omega; Mc = Mb; }
+    const int Mf = chirp_length(2LL * N - 1);
+    if (Mf != 0 && Mf <= sp.Nfft) { Mc = Mf; chirp_fast = true; }
+    if (h->band_form && 2LL * omega + 1 < N) {
+      const int Mb = chirp_length((long long)N + 2LL * omega + 1);
+      if (Mb != 0 && Mb < Mc) { band = omega; Mc = Mb; chirp_fast = true; }
+    }
   }
-  SeqPlan spc = sp;                      // plan of the convolution length
-  if (band >= 0) { spc.Nfft = Mc; finish_plan(spc); }
+  SeqPlan spc = sp;                      // plan of the convolution length, for the generic kernels
+  if (is_pow2(Mc)) { spc.Nfft = Mc; finish_plan(spc); }
 
   if (sp.bluestein) {
     // Spectrum of the chirp kernel.  It depends on the sequence length only, so the handle keeps the last few
@@ -1073,9 +1117,16 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       hhat = h->hhat_cache + (size_t)slot * h->hhat_cache_len;
     }
     if (!have) {
-      ChirpKernelLoader cl{N, Mc, band};
-      if ((s = launch_pass1(h, st, cl, spc, 8, 8, hcol, nullptr)) != FC_OK) return s;
-      if ((s = launch_pass2<MID_SPEC>(h, st, spc, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
+      if (is_pow2(Mc)) {
+        ChirpKernelLoader cl{N, Mc, band};
+        if ((s = launch_pass1(h, st, cl, spc, 8, 8, hcol, nullptr)) != FC_OK) return s;
+        if ((s = launch_pass2<MID_SPEC>(h, st, spc, 8, 8, hcol, 0, hhat, 1.f)) != FC_OK) return s;
+      } else {
+        // lengths with an odd factor: the specialised kernels transform the kernel themselves (64 columns of the
+        // workspace, which no head group uses yet)
+        if ((s = launch_chirp<T>(h, st, kv, nullptr, nullptr, N, Mc, 0, 1, 0, ws, nullptr, nullptr, nullptr, nullptr,
+                                 nullptr, 0, 64, 0, band, hhat)) != FC_OK) return s;
+      }
       if (cached) h->hhat_cache_n[slot] = hkey;
     }
   }
@@ -1154,10 +1205,8 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       // One head may be transformed in several column groups (sub < d) so that the padded
       // length-Nfft intermediates of a group stay within the cache budget; the groups run in
       // stream order and the last pass adds their contributions to the score in that order.
-      int fa, fb;
-      fast_factors(Mc, &fa, &fb);
-      if (fa != 0 && !h->generic_only && L.sub_cols % 64 == 0) {   // a length and a width the specialised kernels take
-        const int sub = L.sub_cols, ngr = (hg == 1) ? d / sub : 1, n2f = 16 * fb;
+      if (chirp_fast) {                         // a length and a width the specialised kernels take
+        const int sub = L.sub_cols, ngr = (hg == 1) ? d / sub : 1, n2f = chirp_shape(Mc).n2();
         const int ncol = (hg == 1) ? sub : ncol_ws;
         const int si = group % L.chirp_streams;                   // head groups alternate over the internal streams
         cudaStream_t sx = L.chirp_streams > 1 ? h->aux[si] : st;

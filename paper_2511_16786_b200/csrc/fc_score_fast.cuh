@@ -43,6 +43,13 @@ template <> struct Load2<__nv_bfloat16> {
 
 // exp(+j*pi*n*n/N), the chirp of the convolution form of an N-point DFT; n*n is reduced modulo 2N
 // (one period) in integers first.
+// exp(-2*pi*j*r/n) for table lengths the master table has no entries for (not a power of two)
+__device__ __forceinline__ float2 root_of_unity(int r, int n) {
+  double sn, cs;
+  sincospi(-2.0 * (double)r / (double)n, &sn, &cs);
+  return make_float2((float)cs, (float)sn);
+}
+
 __device__ __forceinline__ float2 chirp_f(int n, int N) {
   const unsigned long long r = ((unsigned long long)n * (unsigned long long)n) % (2ull * (unsigned long long)N);
   float s, c;
@@ -60,7 +67,10 @@ __device__ __forceinline__ float2 chirp_f(int n, int N) {
 //               of the N-point spectrum (row q + band); the input is conj(Wb[q]) * conj(chirp(q)) with the low-pass
 //               part Wb[q] = (W[q] + exp(j*pi*q/N) W[-q]) / 2 (one formula for both signs of q and for q = 0),
 //               zeros behind.  `omega` carries the band.
-enum { LD_KV = 0, LD_CHIRP = 1, LD_FILTER = 2, LD_BAND = 3 };
+//   LD_KERNEL : the chirp kernel of the convolution itself in column 0 (other columns zero), wrapped to the transform
+//               length: chirp(|n|) for |n| < N, or for the band form (`omega` carries the band, else -1)
+//               chirp(|n - band|) for n = -(N-1) .. 2*band.
+enum { LD_KV = 0, LD_CHIRP = 1, LD_FILTER = 2, LD_BAND = 3, LD_KERNEL = 4 };
 // What pass 2 does between its forward and inverse halves: the DCT/low-pass residual filter on paired rows,
 // or a multiplication by the spectrum of the chirp kernel (rows 2x and 2x+1, unrelated).  MID_CONV2 is the
 // convolution for rows of 2*N2 points: the two halves of the block take the even and the odd samples of ONE
@@ -81,15 +91,16 @@ __device__ __forceinline__ void dft_inv(float2 (&x)[R]) { dft_small<R, +1>(x); }
 // ---------------------------------------------------------------------------
 // pass 1: grid (N2, group columns / (2*CPW)), block CPW*R1B.
 // Thread (cp = tid % CPW, j = tid / CPW): channels 2cp, 2cp+1 of the slice; first
-// stage points n1 = j + R1B*p, p = 0..15, loaded from the K/V rows.
+// stage points n1 = j + R1B*p, p = 0..A-1, loaded from the K/V rows.  N1 = A*R1B: A = 16 with R1B = 2..16 for
+// power-of-two lengths, A = 10, 12 or 14 with R1B = 16 for the chirp path's lengths 2^a * {5, 3, 7}.
 // ---------------------------------------------------------------------------
-template <typename T, int R1B, int CPW, int LD = LD_KV>
+template <typename T, int R1B, int CPW, int LD = LD_KV, int A = 16>
 __global__ void __launch_bounds__(CPW * R1B)
 k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, long long stride_head,
      int head0, int head_dim, int N, int N2, int ncol_ws, float2 *__restrict__ ws,
      const float2 *__restrict__ master, int master_len, double *__restrict__ partial,
      const float2 *__restrict__ spec = nullptr, int omega = 0) {
-  constexpr int N1 = 16 * R1B, NT = CPW * R1B, IT = 16 / R1B, NW = (NT + 31) / 32;
+  constexpr int N1 = A * R1B, NT = CPW * R1B, IT = (A + R1B - 1) / R1B, NW = (NT + 31) / 32;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                        // [N1][CPW]
   float2 *tw = reinterpret_cast<float2 *>(S + N1 * CPW);    // [N1]
@@ -100,10 +111,10 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
   const T *kb = k + (long long)h * stride_head + c;
   const T *vb = v + (long long)h * stride_head + c;
 
-  float2 x0[16], x1[16];
+  float2 x0[A], x1[A];
   float accK = 0.f, accV = 0.f;
 #pragma unroll
-  for (int p = 0; p < 16; ++p) {
+  for (int p = 0; p < A; ++p) {
     const int n = (j + R1B * p) * N2 + n2;
     if (LD == LD_KV) {
       const long long off = (long long)perm_token(n, N) * stride_token;
@@ -120,6 +131,20 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
         const float2 ch = chirp_f(n, N);
         x0[p] = cmul_conj(make_float2(kk.x, vv.x), ch);
         x1[p] = cmul_conj(make_float2(kk.y, vv.y), ch);
+      }
+    } else if (LD == LD_KERNEL) {
+      x0[p] = x1[p] = make_float2(0.f, 0.f);
+      if (gc0 == 0 && cp == 0) {
+        const int M = N1 * N2, band = omega;
+        int a = -1;                                  // argument of the chirp; -1: outside the kernel's support
+        if (band < 0) {
+          if (n < N) a = n;
+          else if (n > M - N) a = M - n;
+        } else {
+          if (n <= 2 * band) a = n < band ? band - n : n - band;
+          else if (n > M - N) a = band + (M - n);
+        }
+        if (a >= 0) x0[p] = chirp_f(a, N);
       }
     } else if (LD == LD_BAND) {
       x0[p] = x1[p] = make_float2(0.f, 0.f);
@@ -158,19 +183,19 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
       }
     }
   }
-  for (int i = tid; i < N1; i += NT) tw[i] = master[(size_t)i * (master_len / N1)];
+  for (int i = tid; i < N1; i += NT) tw[i] = (A == 16) ? master[(size_t)i * (master_len / N1)] : root_of_unity(i, N1);
   __syncthreads();
   if (LD == LD_KV) {
 #pragma unroll
-    for (int p = 0; p < 16; ++p) {
+    for (int p = 0; p < A; ++p) {
       accK = fmaf(x0[p].x, x0[p].x, fmaf(x1[p].x, x1[p].x, accK));
       accV = fmaf(x0[p].y, x0[p].y, fmaf(x1[p].y, x1[p].y, accV));
     }
   }
-  dft_fwd<16>(x0);
-  dft_fwd<16>(x1);
+  dft_fwd<A>(x0);
+  dft_fwd<A>(x1);
 #pragma unroll
-  for (int p = 0; p < 16; ++p) {
+  for (int p = 0; p < A; ++p) {
     if (p > 0) {
       const float2 w = tw[j * p];
       x0[p] = cmul(x0[p], w);
@@ -183,6 +208,7 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
 #pragma unroll
   for (int it = 0; it < IT; ++it) {
     const int pp = j + R1B * it;
+    if (A % R1B != 0 && pp >= A) break;
     float2 y0[R1B], y1[R1B];
 #pragma unroll
     for (int q = 0; q < R1B; ++q) {
@@ -194,12 +220,12 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
     dft_fwd<R1B>(y1);
 #pragma unroll
     for (int q = 0; q < R1B; ++q) {
-      const int k1 = pp + 16 * q;
+      const int k1 = pp + A * q;
       float4 *dst = reinterpret_cast<float4 *>(ws + ((size_t)k1 * N2 + n2) * ncol_ws + gc0 + 2 * cp);
       *dst = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
     }
   }
-  if (LD == LD_FILTER || LD == LD_BAND) return;
+  if (LD == LD_FILTER || LD == LD_BAND || LD == LD_KERNEL) return;
   // per-block sums of squares (total energy of Eq. 12, by Parseval)
   const double a = warp_sum_d((double)accK), b = warp_sum_d((double)accV);
   if ((tid & 31) == 0) { red[0][tid >> 5] = a; red[1][tid >> 5] = b; }
@@ -223,8 +249,11 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
 template <int R2B, int CP, int MID = MID_FILTER>
 __global__ void __launch_bounds__(2 * CP * R2B, 512 / (2 * CP * R2B > 32 ? 2 * CP * R2B : 32))
 k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ master, int master_len,
-     int omega, const float2 *__restrict__ hhat = nullptr, float scale = 1.f, int hrev = 0) {
+     int omega, const float2 *__restrict__ hhat = nullptr, float scale = 1.f, int hrev = 0,
+     float2 *__restrict__ hout = nullptr) {
   // hrev (convolution variants): multiply by the spectrum of the index-reversed kernel, hhat[(-bin) mod N]
+  // hout (convolution variants): forward half only; the spectrum of column 0 goes to hout[bin] (the chirp kernel's
+  // spectrum for transform lengths the generic kernels do not take)
   constexpr int N2 = 16 * R2B, NT = 2 * CP * R2B, IT = 16 / R2B;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                         // [2][N2][CP]
@@ -244,13 +273,20 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   const bool active = !(self && hf);
 
   {
-    const int mstepN = master_len / N, ustep = master_len / (2 * N);
+    // N is a power of two (every root is in the master table) or, on the chirp path, 2^a * {3, 5, 7}
+    const bool tab = (master_len % N) == 0;
+    const int mstepN = tab ? master_len / N : 0, ustep = master_len / (2 * N);
     for (int i = tid; i < N2; i += NT) {
       tw[i] = master[(size_t)i * (master_len / N2)];
       if (MID == MID_CONV2) {
-        twN[i] = master[(size_t)(((2 * i) * k1a) & (N - 1)) * mstepN];           // even samples: n2 = 2i
-        twN[N2 + i] = master[(size_t)(((2 * i + 1) * k1a) & (N - 1)) * mstepN];   // odd samples: n2 = 2i + 1
+        const int ra = ((2 * i) * k1a) % N, rb = ((2 * i + 1) * k1a) % N;
+        twN[i] = tab ? master[(size_t)ra * mstepN] : root_of_unity(ra, N);        // even samples: n2 = 2i
+        twN[N2 + i] = tab ? master[(size_t)rb * mstepN] : root_of_unity(rb, N);   // odd samples: n2 = 2i + 1
         uT[i] = master[(size_t)i * (master_len / ROW)];                          // w_ROW^k of the radix-2 step
+      } else if (MID == MID_CONV) {
+        const int ra = (i * k1a) % N, rb = (i * k1b) % N;
+        twN[i] = tab ? master[(size_t)ra * mstepN] : root_of_unity(ra, N);
+        twN[N2 + i] = tab ? master[(size_t)rb * mstepN] : root_of_unity(rb, N);
       } else {
         twN[i] = master[(size_t)((i * k1a) & (N - 1)) * mstepN];
         twN[N2 + i] = master[(size_t)((i * k1b) & (N - 1)) * mstepN];
@@ -329,7 +365,11 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
         const int k2 = pp + 16 * q;
         const int bin = k1 + N1 * k2;
         if (MID == MID_CONV) {
-          const float2 hq = cscale(__ldg(hhat + (hrev ? ((N - bin) & (N - 1)) : bin)), scale);
+          if (hout != nullptr) {
+            if (cp == 0 && blockIdx.y == 0) hout[bin] = x0[it * R2B + q];
+            continue;
+          }
+          const float2 hq = cscale(__ldg(hhat + ((hrev && bin != 0) ? N - bin : bin)), scale);
           x0[it * R2B + q] = cmul(x0[it * R2B + q], hq);
           x1[it * R2B + q] = cmul(x1[it * R2B + q], hq);
           continue;
@@ -342,7 +382,11 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
           const float2 e0 = hf ? make_float2(t.x, t.y) : m0, e1 = hf ? make_float2(t.z, t.w) : m1;
           const float2 o0 = cmul(hf ? m0 : make_float2(t.x, t.y), w), o1 = cmul(hf ? m1 : make_float2(t.z, t.w), w);
           const int binh = k1 + N1 * (k2 + hf * N2);
-          const float2 hq = cscale(__ldg(hhat + (hrev ? ((N - binh) & (N - 1)) : binh)), scale);
+          if (hout != nullptr) {
+            if (cp == 0 && blockIdx.y == 0) hout[binh] = hf ? csub(e0, o0) : cadd(e0, o0);
+            continue;
+          }
+          const float2 hq = cscale(__ldg(hhat + ((hrev && binh != 0) ? N - binh : binh)), scale);
           m0 = cmul(hf ? csub(e0, o0) : cadd(e0, o0), hq);
           m1 = cmul(hf ? csub(e1, o1) : cadd(e1, o1), hq);
           continue;
@@ -367,6 +411,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       }
     }
   }
+  if ((MID == MID_CONV || MID == MID_CONV2) && hout != nullptr) return;
   if (MID == MID_CONV2) {
     // B[k2] sits in half 0, B[k2 + N2] in half 1: even samples come back from B_lo + B_hi, odd samples from
     // (B_lo - B_hi) * conj(w)
@@ -455,7 +500,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
 // band >= 0 (band form of the chirp path): OUT_SPEC keeps rows 0 .. 2*band (bin q = row - band, rotated by
 // conj(chirp(|q|))); OUT_SCORE_BAND reads the K/V rows again (kin/vin: first token of the sequence, first channel of
 // the column group) and scores |z - z_base|^2 with z_base = conj(row * conj(chirp)) / N.
-template <int R1B, int CPW, int OUT = OUT_SCORE, typename T = float>
+template <int R1B, int CPW, int OUT = OUT_SCORE, typename T = float, int A = 16>
 __global__ void __launch_bounds__(CPW * R1B)
 k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__restrict__ master,
      int master_len, float *__restrict__ scores, int head0, int head_dim, long long score_stride,
@@ -467,14 +512,14 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
      long long stride_head = 0) {
   // OUT_SCORE_CHIRP with a head transformed in column groups: head_dim is the group's width, energy_scale the
   // head's true channel count, and every group after the first adds to the stored score (accumulate).
-  constexpr int N1 = 16 * R1B, NT = CPW * R1B, IT = 16 / R1B, NW = (NT + 31) / 32;
+  constexpr int N1 = A * R1B, NT = CPW * R1B, IT = (A + R1B - 1) / R1B, NW = (NT + 31) / 32;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                        // [N1][CPW]
   float2 *tw = reinterpret_cast<float2 *>(S + N1 * CPW);    // [N1]
   __shared__ double red[2][NW];
   const int tid = threadIdx.x, cp = tid % CPW, j = tid / CPW;
   const int n2 = blockIdx.x, hh = blockIdx.y;
-  for (int i = tid; i < N1; i += NT) tw[i] = master[(size_t)i * (master_len / N1)];
+  for (int i = tid; i < N1; i += NT) tw[i] = (A == 16) ? master[(size_t)i * (master_len / N1)] : root_of_unity(i, N1);
 
   float acc[16];            // |residual|^2 of rows j + R1B*p summed over this thread's channels (K and V)
 #pragma unroll
@@ -488,11 +533,12 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
       const int pp = j + R1B * it;
+      if (A % R1B != 0 && pp >= A) break;
       float2 y0[R1B], y1[R1B];
 #pragma unroll
       for (int q = 0; q < R1B; ++q) {
         const float4 t = *reinterpret_cast<const float4 *>(
-            ws + ((size_t)(pp + 16 * q) * N2 + n2) * ncol_ws + gc0 + 2 * cp);
+            ws + ((size_t)(pp + A * q) * N2 + n2) * ncol_ws + gc0 + 2 * cp);
         y0[q] = make_float2(t.x, t.y);
         y1[q] = make_float2(t.z, t.w);
       }
@@ -503,9 +549,9 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
         S[(q + R1B * pp) * CPW + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
     }
     __syncthreads();
-    float2 x0[16], x1[16];
+    float2 x0[A], x1[A];
 #pragma unroll
-    for (int p = 0; p < 16; ++p) {
+    for (int p = 0; p < A; ++p) {
       const float4 t = S[(j + R1B * p) * CPW + cp];
       x0[p] = make_float2(t.x, t.y);
       x1[p] = make_float2(t.z, t.w);
@@ -515,10 +561,10 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
         x1[p] = cmul_conj(x1[p], w);
       }
     }
-    dft_inv<16>(x0);
-    dft_inv<16>(x1);
+    dft_inv<A>(x0);
+    dft_inv<A>(x1);
 #pragma unroll
-    for (int p = 0; p < 16; ++p) {
+    for (int p = 0; p < A; ++p) {
       if (OUT != OUT_SCORE) {
         const int pos = (j + R1B * p) * N2 + n2;
         if (OUT == OUT_SPEC && band >= 0) {
@@ -577,7 +623,7 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
     }
   }
   constexpr int DUP = CPW / 16;                             // lanes that end with the same row sum
-  if ((cp & (DUP - 1)) == 0) {
+  if ((cp & (DUP - 1)) == 0 && cp / DUP < A) {            // rows A..15 of the reduction are padding
     const int p = (j + R1B * (cp / DUP)) * N2 + n2;
     if (OUT == OUT_SCORE) {
       scores[(long long)(head0 + hh) * score_stride + perm_token(p, N)] = acc[0] * inv_scale;

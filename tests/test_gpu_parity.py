@@ -208,6 +208,26 @@ def test_scores_chirp_band_form(fc, N, gamma, d, group_bytes):
     np.testing.assert_allclose(e1, e2, rtol=1e-4)
 
 
+@pytest.mark.parametrize("M", [5120, 6144, 7168, 10240, 12288, 14336, 20480, 24576, 28672, 40960, 49152, 57344,
+                               81920, 98304, 114688])
+def test_scores_chirp_lengths_with_an_odd_factor(fc, M):
+    # Full form of the chirp path at N = M/2 - 1: 2N - 1 = M - 3 pads to M = 2^k * {5, 3, 7}, every shape the
+    # specialised kernels have for such lengths (first-stage radix 10, 12, 14; rows of 32..512 points).  The band form
+    # of the same sequence picks another length; both match the oracle.
+    N = M // 2 - 1
+    k, v = _rand_kv(N, 1, 64, torch.float32, 900 + M % 1000)
+    g1, e1 = _check_layer(fc, k, v, [0, N], 0.2, band=False)
+    g2, e2 = _check_layer(fc, k, v, [0, N], 0.2, band=True)
+    np.testing.assert_allclose(g1, g2, rtol=2e-3, atol=1e-6 * float(g2.max()))
+
+
+@pytest.mark.parametrize("N", [5118, 20478, 29255, 35107, 40958, 58513])
+def test_scores_chirp_band_form_on_lengths_with_an_odd_factor(fc, N):
+    # N + 2*floor(0.2 N) + 1 lands just under 7168, 28672, 40960, 49152, 57344 and 81920
+    k, v = _rand_kv(N, 2, 128, torch.bfloat16, 30 + N % 100)
+    _check_layer(fc, k, v, [0, N], 0.2)
+
+
 def test_scores_chirp_band_form_16bit_ragged(fc):
     lens = [2500, 1024, 5000, 40961, 300]
     cu = [0] + [int(x) for x in np.cumsum(lens)]
