@@ -90,9 +90,9 @@ typedef struct {
 /* Create a handle on `device`.  max_seqlen bounds every N_b later passed in
  * (1 <= max_seqlen <= 131072; lengths that are not a power of two, or below 16,
  * are limited to 65536).  Allocates the twiddle table (8 bytes * 4 * next power of two of
- * max_seqlen), room for eight chirp-kernel spectra (each 8 bytes * the power of two from
- * 2*max_seqlen-1 up, at most 1 MiB; lengths that are not a power of two reuse theirs from layer to
- * layer) and a status word.  Returns FC_ERR_CUDA if the device cannot be
+ * max_seqlen), room for eight chirp-kernel spectra with their per-row chirp factors (each 8 bytes *
+ * (the power of two from 2*max_seqlen-1 up + 2*max_seqlen), at most 2 MiB; lengths that are not a
+ * power of two reuse theirs from layer to layer) and a status word.  Returns FC_ERR_CUDA if the device cannot be
  * used, FC_ERR_UNSUPPORTED if max_seqlen is out of range. */
 fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen);
 void fc_destroy(fc_handle *h);

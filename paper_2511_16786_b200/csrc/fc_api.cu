@@ -177,9 +177,10 @@ extern "C" fc_status fc_create(fc_handle **out, int device, int32_t max_seqlen) 
     const int nmax = max_seqlen < 65536 ? max_seqlen : 65536;
     while (m < 2 * nmax - 1) m <<= 1;
     h->hhat_cache_len = m;
+    h->hhat_slot_len = m + 2 * ((nmax + 31) / 32 * 32);
     for (int i = 0; i < FC_HHAT_SLOTS; ++i) h->hhat_cache_n[i] = 0;
     h->hhat_cache_next = 0;
-    if (cudaMalloc(&h->hhat_cache, (size_t)FC_HHAT_SLOTS * m * sizeof(float2)) != cudaSuccess) {
+    if (cudaMalloc(&h->hhat_cache, (size_t)FC_HHAT_SLOTS * h->hhat_slot_len * sizeof(float2)) != cudaSuccess) {
       fc_destroy(h);
       return FC_ERR_CUDA;
     }

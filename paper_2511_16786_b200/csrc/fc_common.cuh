@@ -68,6 +68,7 @@ struct fc_handle {
   // slots are reused round robin)
   float2 *hhat_cache;
   int hhat_cache_len, hhat_cache_next;
+  int hhat_slot_len;       // points per slot: the spectrum (hhat_cache_len) and 2N per-row chirp factors behind it
   long long hhat_cache_n[FC_HHAT_SLOTS];   // key of slot i: length + ((band + 1) << 32), 0 = none
   cudaStream_t host_copy;
   cudaEvent_t *host_ev;

@@ -925,7 +925,7 @@ template <typename T, int A, int R1B, int R2B, bool DOUBLE>
 fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq,
                             int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
                             double *phi, float *scores, long long total_tokens, int dcols, int accumulate, int band,
-                            float2 *hout) {
+                            float2 *hout, const float2 *ctab) {
   constexpr int CPW = 32, CP = 8, N1 = A * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
   constexpr int MIDV = DOUBLE ? fast::MID_CONV2 : fast::MID_CONV;
   const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
@@ -964,7 +964,8 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   {
     ProfScope ps(h, FC_K_PASS1, st);
     fast::k_p1<T, R1B, CPW, fast::LD_CHIRP, A><<<g1, CPW * R1B, sm1, st>>>(
-        kp, vp, kv->stride_token, kv->stride_head, h0, dcols, Nseq, N2, ncol, ws, h->master, h->master_len, ptot);
+        kp, vp, kv->stride_token, kv->stride_head, h0, dcols, Nseq, N2, ncol, ws, h->master, h->master_len, ptot,
+        nullptr, 0, ctab);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
@@ -976,17 +977,17 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
     ProfScope ps(h, FC_K_PASS3, st);
     fast::k_p3<R1B, CPW, fast::OUT_SPEC, float, A><<<g3, CPW * R1B, sm1, st>>>(
         Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, h0, dcols, 0, 0.f, nullptr, nullptr, 0u, nullptr, 0, nullptr, 0,
-        nullptr, spec, 0.f, 0, band);
+        nullptr, spec, 0.f, 0, band, nullptr, nullptr, 0, 0, ctab);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS1, st);
     if (band >= 0)
       fast::k_p1<float, R1B, CPW, fast::LD_BAND, A><<<g1, CPW * R1B, sm1, st>>>(
-          nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, band);
+          nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, band, ctab);
     else
       fast::k_p1<float, R1B, CPW, fast::LD_FILTER, A><<<g1, CPW * R1B, sm1, st>>>(
-          nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, omega);
+          nullptr, nullptr, 0, 0, 0, ncol, Nseq, N2, ncol, ws, h->master, h->master_len, nullptr, spec, omega, ctab);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;
   {
@@ -1003,12 +1004,12 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
       fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T, A><<<g3, CPW * R1B, sm1, st>>>(
           Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, dcols, total_tokens, (float)(1.0 / (double)d), phi,
           nullptr, 0u, nullptr, 0, nullptr, 0, nullptr, nullptr, (float)d, accumulate, band, kp, vp, kv->stride_token,
-          kv->stride_head);
+          kv->stride_head, ctab);
     } else {
       const float inv = (float)(1.0 / ((double)Nseq * (double)Nseq * (double)d));
       fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP, float, A><<<g3, CPW * R1B, sm1, st>>>(
           Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, dcols, total_tokens, inv, phi, nullptr, 0u, nullptr, 0,
-          nullptr, 0, nullptr, nullptr, (float)d, accumulate);
+          nullptr, 0, nullptr, nullptr, (float)d, accumulate, -1, nullptr, nullptr, 0, 0, ctab);
     }
   }
   return fc_after_launch(h);
@@ -1018,12 +1019,12 @@ template <typename T>
 fc_status launch_chirp(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp, int Nseq, int M,
                        int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
                        double *phi, float *scores, long long total_tokens, int dcols, int accumulate, int band,
-                       float2 *hout = nullptr) {
+                       const float2 *ctab, float2 *hout = nullptr) {
   const ChirpShape c = chirp_shape(M);
 #define FC_CHIRP_CASE(A, B, C, D)                                                                               \
   if (c.a == A && c.r1b == B && c.r2b == C && c.dbl == D)                                                       \
     return launch_chirp_impl<T, A, B, C, D>(h, st, kv, kp, vp, Nseq, h0, hg, omega, ws, spec, hhat, ptot, phi, \
-                                            scores, total_tokens, dcols, accumulate, band, hout);
+                                            scores, total_tokens, dcols, accumulate, band, hout, ctab);
   FC_CHIRP_CASE(16, 2, 2, false) FC_CHIRP_CASE(16, 2, 4, false) FC_CHIRP_CASE(16, 4, 4, false)
   FC_CHIRP_CASE(16, 4, 8, false) FC_CHIRP_CASE(16, 8, 8, false) FC_CHIRP_CASE(16, 8, 16, false)
   FC_CHIRP_CASE(16, 16, 16, false) FC_CHIRP_CASE(16, 16, 16, true)
@@ -1091,6 +1092,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   SeqPlan spc = sp;                      // plan of the convolution length, for the generic kernels
   if (is_pow2(Mc)) { spc.Nfft = Mc; finish_plan(spc); }
 
+  const float2 *ctab = nullptr;
   if (sp.bluestein) {
     // Spectrum of the chirp kernel.  It depends on the sequence length only, so the handle keeps the last few
     // (layers of a prefill share their lengths).  While the stream is being captured the spectrum goes to the
@@ -1114,7 +1116,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
         h->hhat_cache_next = (slot + 1) % FC_HHAT_SLOTS;
         h->hhat_cache_n[slot] = 0;                          // not valid until both launches are in the stream
       }
-      hhat = h->hhat_cache + (size_t)slot * h->hhat_cache_len;
+      hhat = h->hhat_cache + (size_t)slot * h->hhat_slot_len;
     }
     if (!have) {
       if (is_pow2(Mc)) {
@@ -1125,9 +1127,17 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
         // lengths with an odd factor: the specialised kernels transform the kernel themselves (64 columns of the
         // workspace, which no head group uses yet)
         if ((s = launch_chirp<T>(h, st, kv, nullptr, nullptr, N, Mc, 0, 1, 0, ws, nullptr, nullptr, nullptr, nullptr,
-                                 nullptr, 0, 64, 0, band, hhat)) != FC_OK) return s;
+                                 nullptr, 0, 64, 0, band, nullptr, hhat)) != FC_OK) return s;
       }
       if (cached) h->hhat_cache_n[slot] = hkey;
+    }
+    // per-row factors of the chirp modes (2N values): behind the spectrum in its cache slot, else in the column
+    // buffer of the workspace, which the spectrum's transform no longer needs
+    ctab = cached ? hhat + h->hhat_cache_len : hcol;
+    if (!have && chirp_fast) {
+      ProfScope ps(h, FC_K_OTHER, st);
+      fast::k_chirp_tables<<<(N + 255) / 256, 256, 0, st>>>(const_cast<float2 *>(ctab), N);
+      if ((s = fc_after_launch(h)) != FC_OK) return s;
     }
   }
 
@@ -1215,7 +1225,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
         for (int cg = 0; cg < ngr; ++cg) {                        // column groups of one head, else one pass
           if ((s = launch_chirp<T>(h, sx, kv, kp + cg * sub, vp + cg * sub, N, Mc, h0, hg, omega, ws_s, spec_s, hhat,
                                    ptot + 2 * (size_t)cg * n2f * (ncol / 64), phi + 2 * (size_t)cg * n2f * hg,
-                                   scores + start, total_tokens, (hg == 1) ? sub : d, cg > 0 ? 1 : 0, band)) != FC_OK)
+                                   scores + start, total_tokens, (hg == 1) ? sub : d, cg > 0 ? 1 : 0, band, ctab)) != FC_OK)
             return s;
         }
         tot_slots += (size_t)n2f * (ncol / 64) * ngr;

@@ -42,7 +42,7 @@ template <> struct Load2<__nv_bfloat16> {
 };
 
 // exp(+j*pi*n*n/N), the chirp of the convolution form of an N-point DFT; n*n is reduced modulo 2N
-// (one period) in integers first.
+// (one period) in integers first.  Costs a 64-bit division: the passes read it from a table (k_chirp_tables).
 // exp(-2*pi*j*r/n) for table lengths the master table has no entries for (not a power of two)
 __device__ __forceinline__ float2 root_of_unity(int r, int n) {
   double sn, cs;
@@ -55,6 +55,17 @@ __device__ __forceinline__ float2 chirp_f(int n, int N) {
   float s, c;
   sincospif(__fdiv_rn((float)(unsigned)r, (float)N), &s, &c);
   return make_float2(c, s);
+}
+
+// tab[n] = chirp(n), tab[N + q] = exp(j*pi*q/N) for n, q = 0..N-1: what the chirp modes of passes 1 and 3 need per
+// row, computed once per sequence length instead of once per thread and row.
+__global__ void k_chirp_tables(float2 *__restrict__ tab, int N) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N) return;
+  tab[i] = chirp_f(i, N);
+  float sn, cs;
+  sincospif(__fdiv_rn((float)i, (float)N), &sn, &cs);
+  tab[N + i] = make_float2(cs, sn);
 }
 
 // What pass 1 transforms.
@@ -99,7 +110,8 @@ __global__ void __launch_bounds__(CPW * R1B)
 k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, long long stride_head,
      int head0, int head_dim, int N, int N2, int ncol_ws, float2 *__restrict__ ws,
      const float2 *__restrict__ master, int master_len, double *__restrict__ partial,
-     const float2 *__restrict__ spec = nullptr, int omega = 0) {
+     const float2 *__restrict__ spec = nullptr, int omega = 0, const float2 *__restrict__ ctab = nullptr) {
+  // ctab (chirp modes): ctab[n] = chirp(n) and ctab[N + q] = exp(j*pi*q/N), n, q = 0..N-1
   constexpr int N1 = A * R1B, NT = CPW * R1B, IT = (A + R1B - 1) / R1B, NW = (NT + 31) / 32;
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                        // [N1][CPW]
@@ -128,7 +140,7 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
         const float2 kk = Load2<T>::ld(kb + off), vv = Load2<T>::ld(vb + off);
         accK = fmaf(kk.x, kk.x, fmaf(kk.y, kk.y, accK));
         accV = fmaf(vv.x, vv.x, fmaf(vv.y, vv.y, accV));
-        const float2 ch = chirp_f(n, N);
+        const float2 ch = __ldg(ctab + n);
         x0[p] = cmul_conj(make_float2(kk.x, vv.x), ch);
         x1[p] = cmul_conj(make_float2(kk.y, vv.y), ch);
       }
@@ -153,10 +165,10 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
         const int q = n - band;
         const float4 P4 = *reinterpret_cast<const float4 *>(spec + (size_t)n * ncol_ws + gc0 + 2 * cp);
         const float4 Q4 = *reinterpret_cast<const float4 *>(spec + (size_t)(2 * band - n) * ncol_ws + gc0 + 2 * cp);
-        float sn, cs;
-        sincospif(__fdiv_rn((float)q, (float)N), &sn, &cs);
-        const float2 u = make_float2(cs, sn);
-        const float2 ch = chirp_f(q < 0 ? -q : q, N);
+        const int aq = q < 0 ? -q : q;
+        float2 u = __ldg(ctab + N + aq);                         // exp(j*pi*q/N)
+        if (q < 0) u.y = -u.y;
+        const float2 ch = __ldg(ctab + aq);
         const float2 W0 = cscale(cadd(make_float2(P4.x, P4.y), cmul(make_float2(Q4.x, Q4.y), u)), 0.5f);
         const float2 W1 = cscale(cadd(make_float2(P4.z, P4.w), cmul(make_float2(Q4.z, Q4.w), u)), 0.5f);
         x0[p] = cmul_conj(cconj(W0), ch);
@@ -168,12 +180,10 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
         const int q = n, qp = (N - q) % N;
         const float4 P4 = *reinterpret_cast<const float4 *>(spec + (size_t)q * ncol_ws + gc0 + 2 * cp);
         const float4 Q4 = *reinterpret_cast<const float4 *>(spec + (size_t)qp * ncol_ws + gc0 + 2 * cp);
-        float sn, cs;
-        sincospif(__fdiv_rn((float)q, (float)N), &sn, &cs);
-        const float2 u = make_float2(cs, sn);
+        const float2 u = __ldg(ctab + N + q);
         const float inL = (q <= omega) ? 0.5f : 0.f;
         const float inH = (q != 0 && N - q <= omega) ? 0.5f : 0.f;
-        const float2 ch = chirp_f(n, N);
+        const float2 ch = __ldg(ctab + n);
         const float2 P0 = make_float2(P4.x, P4.y), P1 = make_float2(P4.z, P4.w);
         const float2 uQ0 = cmul(make_float2(Q4.x, Q4.y), u), uQ1 = cmul(make_float2(Q4.z, Q4.w), u);
         float2 E0 = csub(csub(P0, cscale(cadd(P0, uQ0), inL)), cscale(csub(P0, uQ0), inH));
@@ -509,7 +519,7 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
      const double *__restrict__ part_hi, int n_hi, double *__restrict__ energy,
      float2 *__restrict__ spec = nullptr, float energy_scale = 0.f, int accumulate = 0, int band = -1,
      const T *__restrict__ kin = nullptr, const T *__restrict__ vin = nullptr, long long stride_token = 0,
-     long long stride_head = 0) {
+     long long stride_head = 0, const float2 *__restrict__ ctab = nullptr) {
   // OUT_SCORE_CHIRP with a head transformed in column groups: head_dim is the group's width, energy_scale the
   // head's true channel count, and every group after the first adds to the stored score (accumulate).
   constexpr int N1 = A * R1B, NT = CPW * R1B, IT = (A + R1B - 1) / R1B, NW = (NT + 31) / 32;
@@ -573,7 +583,7 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
           continue;
         }
         const int cpos = (OUT == OUT_SPEC && band >= 0) ? (pos < band ? band - pos : pos - band) : pos;
-        const float2 ch = chirp_f(cpos, N);
+        const float2 ch = __ldg(ctab + cpos);                    // chirp(cpos), table of pass 1
         x0[p] = cmul_conj(x0[p], ch);
         x1[p] = cmul_conj(x1[p], ch);
         if (OUT == OUT_SPEC) {
