@@ -435,6 +435,7 @@ def main():
     ap.add_argument("--group-mib", type=int, default=0, help="transform group size override (MiB)")
     ap.add_argument("--streams", type=int, default=0, help="internal streams of the scoring calls (default: the library's 2)")
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first LAYERS layers")
+    ap.add_argument("--seqlens", default="", help="profiling aid: replace the config's sequence lengths (comma-separated)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
@@ -478,6 +479,9 @@ def main():
     cfg = S.paper_configs()[args.config]
     if args.layers:
         cfg = S.scaled(cfg, cfg.name, num_layers=args.layers, note=cfg.note + " (first %d layers only)" % args.layers)
+    if args.seqlens:
+        lens = tuple(int(x) for x in args.seqlens.split(","))
+        cfg = S.scaled(cfg, cfg.name, seqlens=lens, note=cfg.note + " (sequence lengths replaced: %s)" % args.seqlens)
     dev = torch.device("cuda", local_rank)
     L = cfg.num_layers
     Kd, Vd = [], []
@@ -667,7 +671,7 @@ def main():
                                          % (used, L, el, cores)}
     comp.close()
     # the other four configurations, briefly: 3 warm-up steps, 10 timed, same accounting
-    if world == 1 and args.config == DEFAULT_CONFIG and not args.layers and not args.no_all_configs:
+    if world == 1 and args.config == DEFAULT_CONFIG and not args.layers and not args.seqlens and not args.no_all_configs:
         del Kd, Vd
         torch.cuda.empty_cache()
         out["all_configs"] = {args.config: {"ms_per_step": ms_per_step, "value": value, "unit": UNIT,
