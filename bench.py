@@ -122,7 +122,7 @@ def step_accounting(binding, handle, cfg):
     for N in cfg.seqlens:
         if N == 0:
             continue
-        plan = binding.fc_describe_plan(handle, N)
+        plan = binding.fc_describe_plan(handle, N, cfg.gamma)
         M, n1, n2 = plan["nfft"], plan["n1"], plan["n2"]
         cols = H * d * L                       # complex columns (K + jV) of this sequence
         reps = 2 if plan["bluestein"] else 1   # chirp path: two convolutions, each a forward+inverse transform

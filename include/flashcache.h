@@ -191,10 +191,11 @@ fc_status fc_reset_ordering(fc_handle *h);
  * Default 32 MiB.  Affects speed only. */
 fc_status fc_set_group_bytes(fc_handle *h, size_t bytes);
 
-/* How a sequence of length seqlen is transformed (diagnostic, used for flop
- * accounting): out = { chirp-convolution path (1) or direct power-of-two path (0),
+/* How a sequence of length seqlen is transformed at cutoff ratio gamma (diagnostic, used for flop
+ * accounting; head_dim a multiple of 64 assumed): out = { direct power-of-two path (0), chirp
+ * convolutions in the full-length form (1) or in the band form (2, see fc_set_chirp_band),
  * transform length, first factor N1, second factor N2 }. */
-fc_status fc_describe_plan(const fc_handle *h, int32_t seqlen, int32_t out[4]);
+fc_status fc_describe_plan(const fc_handle *h, int32_t seqlen, double gamma, int32_t out[4]);
 
 /* Workspace sizes (bytes) the next two calls need for this view.  0 on bad input. */
 size_t fc_score_workspace_bytes(const fc_handle *h, const fc_kv_view *kv);

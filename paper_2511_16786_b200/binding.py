@@ -129,7 +129,7 @@ def _load() -> ctypes.CDLL:
     lib.fc_profile_stride.restype = c_int
     lib.fc_profile_end.argtypes = [c_void_p, POINTER(c_double), POINTER(c_uint64)]
     lib.fc_profile_end.restype = c_int
-    lib.fc_describe_plan.argtypes = [c_void_p, c_int32, POINTER(c_int32)]
+    lib.fc_describe_plan.argtypes = [c_void_p, c_int32, c_double, POINTER(c_int32)]
     lib.fc_describe_plan.restype = c_int
     lib.fc_score_workspace_bytes.argtypes = [c_void_p, POINTER(fc_kv_view)]
     lib.fc_score_workspace_bytes.restype = c_size_t
@@ -298,10 +298,10 @@ def fc_profile_end(handle):
     return float(ms.value), int(n.value)
 
 
-def fc_describe_plan(handle, seqlen: int) -> dict:
+def fc_describe_plan(handle, seqlen: int, gamma: float) -> dict:
     out = (c_int32 * 4)()
-    _check(_lib.fc_describe_plan(handle, int(seqlen), out), "fc_describe_plan")
-    return dict(bluestein=bool(out[0]), nfft=int(out[1]), n1=int(out[2]), n2=int(out[3]))
+    _check(_lib.fc_describe_plan(handle, int(seqlen), float(gamma), out), "fc_describe_plan")
+    return dict(bluestein=bool(out[0]), band_form=out[0] == 2, nfft=int(out[1]), n1=int(out[2]), n2=int(out[3]))
 
 
 def fc_score_workspace_bytes(handle, k, v, cu_seqlens) -> int:

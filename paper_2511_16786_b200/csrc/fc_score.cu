@@ -1046,6 +1046,37 @@ fc_status launch_chirp(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, cons
   return FC_ERR_INTERNAL;
 }
 
+// Cutoff index omega of Eq. 8 for a sequence of N tokens.
+inline int cutoff_index(double gamma, int N) {
+  long long om = (long long)floor(gamma * (double)N);
+  if (om > N - 1) om = N - 1;
+  if (om < 0) om = 0;
+  return (int)om;
+}
+
+// Convolution length of the chirp path.  Full form: M >= 2N - 1.  Band form: only the bins -omega .. omega of the
+// spectrum are needed (the low-pass part; the score is taken against the input rows), M >= N + 2*omega + 1.  The
+// specialised kernels take powers of two and 2^k * {3, 5, 7}; whichever form gives the shorter M runs, and the
+// generic kernels (M = sp.Nfft, a power of two, full form) remain for what the specialised ones do not take
+// (cols_ok: the column groups are multiples of 64 channels).
+struct ChirpChoice {
+  int band;      // omega when the band form runs, else -1
+  int M;         // convolution length
+  bool fast;     // specialised kernels
+};
+
+inline ChirpChoice choose_chirp(const fc_handle *h, const SeqPlan &sp, int N, int omega, bool cols_ok) {
+  ChirpChoice c{-1, sp.Nfft, false};
+  if (!sp.bluestein || h->generic_only || !cols_ok) return c;
+  const int Mf = chirp_length(2LL * N - 1);
+  if (Mf != 0 && Mf <= sp.Nfft) { c.M = Mf; c.fast = true; }
+  if (h->band_form && 2LL * omega + 1 < N) {
+    const int Mb = chirp_length((long long)N + 2LL * omega + 1);
+    if (Mb != 0 && Mb < c.M) { c.band = omega; c.M = Mb; c.fast = true; }
+  }
+  return c;
+}
+
 template <typename T>
 fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, int b, double gamma,
                          float *scores, double *energy, char *wsb) {
@@ -1060,10 +1091,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   const int d = kv->head_dim, H = kv->num_heads;
   const SeqPlan sp = plan_sequence(N, !h->generic_only);
   const ScoreLayout L = layout_for(h, sp, H, d);
-  long long om = (long long)floor(gamma * (double)N);
-  if (om > N - 1) om = N - 1;
-  if (om < 0) om = 0;
-  const int omega = (int)om;
+  const int omega = cutoff_index(gamma, N);
 
   fc_status s0 = FC_OK;
   float2 *ws = reinterpret_cast<float2 *>(wsb + L.off_ws);
@@ -1084,20 +1112,9 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
   const FftPlan p1 = make_plan(sp.N1);
   fc_status s;
 
-  // Convolution length of the chirp path.  Full form: M >= 2N - 1.  Band form: only the bins -omega .. omega of the
-  // spectrum are needed (the low-pass part; the score is taken against the input rows), M >= N + 2*omega + 1.  The
-  // specialised kernels take powers of two and 2^k * {3, 5, 7}; whichever form gives the shorter M runs, and the
-  // generic kernels (M = sp.Nfft, a power of two) remain for what the specialised ones do not take.
-  int band = -1, Mc = sp.Nfft;
-  bool chirp_fast = false;
-  if (sp.bluestein && !h->generic_only && L.sub_cols % 64 == 0) {
-    const int Mf = chirp_length(2LL * N - 1);
-    if (Mf != 0 && Mf <= sp.Nfft) { Mc = Mf; chirp_fast = true; }
-    if (h->band_form && 2LL * omega + 1 < N) {
-      const int Mb = chirp_length((long long)N + 2LL * omega + 1);
-      if (Mb != 0 && Mb < Mc) { band = omega; Mc = Mb; chirp_fast = true; }
-    }
-  }
+  const ChirpChoice cc = choose_chirp(h, sp, N, omega, L.sub_cols % 64 == 0);
+  const int band = cc.band, Mc = cc.M;
+  const bool chirp_fast = cc.fast;
   SeqPlan spc = sp;                      // plan of the convolution length, for the generic kernels
   if (is_pow2(Mc)) { spc.Nfft = Mc; finish_plan(spc); }
 
@@ -1416,14 +1433,24 @@ extern "C" fc_status fc_power_spectrum(fc_handle *h, const fc_kv_view *kv, doubl
   return s;
 }
 
-extern "C" fc_status fc_describe_plan(const fc_handle *h, int32_t seqlen, int32_t out[4]) {
-  if (!h || !out || seqlen < 1) return FC_ERR_INVALID_ARG;
+extern "C" fc_status fc_describe_plan(const fc_handle *h, int32_t seqlen, double gamma, int32_t out[4]) {
+  if (!h || !out || seqlen < 1 || !(gamma >= 0.0 && gamma <= 1.0)) return FC_ERR_INVALID_ARG;
   if (seqlen > h->max_seqlen || (seqlen > 65536 && !is_pow2(seqlen))) return FC_ERR_UNSUPPORTED;
   const SeqPlan sp = plan_sequence(seqlen);
   out[0] = sp.bluestein ? 1 : 0;
   out[1] = sp.Nfft;
   out[2] = sp.N1;
   out[3] = sp.N2;
+  if (sp.bluestein) {
+    const ChirpChoice c = choose_chirp(h, sp, seqlen, cutoff_index(gamma, seqlen), true);
+    out[0] = c.band >= 0 ? 2 : 1;
+    out[1] = c.M;
+    if (c.fast) {
+      const ChirpShape cs = chirp_shape(c.M);
+      out[2] = cs.n1();
+      out[3] = cs.n2();
+    }
+  }
   return FC_OK;
 }
 

@@ -228,6 +228,26 @@ def test_scores_chirp_band_form_on_lengths_with_an_odd_factor(fc, N):
     _check_layer(fc, k, v, [0, N], 0.2)
 
 
+def test_describe_plan_reports_the_convolution_length_in_use(fc):
+    h = fc.fc_create(0, 65536)
+    try:
+        p = fc.fc_describe_plan(h, 32768, 0.2)
+        assert (p["bluestein"], p["nfft"], p["n1"] * p["n2"]) == (False, 32768, 32768)
+        p = fc.fc_describe_plan(h, 2500, 0.2)                    # 2500 + 1000 + 1 -> 4096
+        assert (p["band_form"], p["nfft"], p["n1"] * p["n2"]) == (True, 4096, 4096)
+        p = fc.fc_describe_plan(h, 35107, 0.2)                   # 35107 + 14042 + 1 = 49150 -> 49152 = 96 x 512
+        assert (p["band_form"], p["nfft"], p["n1"], p["n2"]) == (True, 49152, 96, 512)
+        p = fc.fc_describe_plan(h, 33001, 0.6)                   # band wider than the spectrum: 2N - 1 -> 81920
+        assert (p["bluestein"], p["band_form"], p["nfft"], p["n1"], p["n2"]) == (True, False, 81920, 160, 512)
+        fc.fc_set_chirp_band(h, False)
+        p = fc.fc_describe_plan(h, 2500, 0.2)                    # 4999 -> 5120 = 160 x 32
+        assert (p["band_form"], p["nfft"], p["n1"], p["n2"]) == (False, 5120, 160, 32)
+        p = fc.fc_describe_plan(h, 300, 0.2)                     # short: generic kernels, power of two
+        assert (p["bluestein"], p["nfft"]) == (True, 1024)
+    finally:
+        fc.fc_destroy(h)
+
+
 def test_scores_chirp_band_form_16bit_ragged(fc):
     lens = [2500, 1024, 5000, 40961, 300]
     cu = [0] + [int(x) for x in np.cumsum(lens)]
