@@ -935,7 +935,9 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   constexpr int CPW = 32, CP = 8, N1 = A * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
   constexpr int MIDV = DOUBLE ? fast::MID_CONV2 : fast::MID_CONV;
   const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
-  const size_t sm2 = (size_t)2 * (16 * R2B) * CP * sizeof(float4) + 5 * (16 * R2B) * sizeof(float2);
+  const size_t sm2 = (size_t)2 * (16 * R2B) * CP * sizeof(float4) + 7 * (16 * R2B) * sizeof(float2);
+  // band form's last pass, 16-bit inputs: staging slots for the K/V rows it reads again
+  const size_t sm3b = sm1 + (sizeof(T) == 2 ? (size_t)2 * A * CPW * R1B * sizeof(unsigned) : 0);
   fc_status s;
   if ((s = set_smem(fast::k_p2<R2B, CP, MIDV>, sm2)) != FC_OK) return s;
   if (hout != nullptr) {
@@ -962,7 +964,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SPEC, float, A>, sm1)) != FC_OK) return s;
   if (band >= 0) {
     if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_BAND, A>, sm1)) != FC_OK) return s;
-    if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T, A>, sm1)) != FC_OK) return s;
+    if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T, A>, sm3b)) != FC_OK) return s;
   } else {
     if ((s = set_smem(fast::k_p1<float, R1B, CPW, fast::LD_FILTER, A>, sm1)) != FC_OK) return s;
     if ((s = set_smem(fast::k_p3<R1B, CPW, fast::OUT_SCORE_CHIRP, float, A>, sm1)) != FC_OK) return s;
@@ -1007,7 +1009,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   {
     ProfScope ps(h, FC_K_PASS3, st);
     if (band >= 0) {
-      fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T, A><<<g3, CPW * R1B, sm1, st>>>(
+      fast::k_p3<R1B, CPW, fast::OUT_SCORE_BAND, T, A><<<g3, CPW * R1B, sm3b, st>>>(
           Nseq, N2, ncol, ws, h->master, h->master_len, scores, h0, dcols, total_tokens, (float)(1.0 / (double)d), phi,
           nullptr, 0u, nullptr, 0, nullptr, 0, nullptr, nullptr, (float)d, accumulate, band, kp, vp, kv->stride_token,
           kv->stride_head, ctab);

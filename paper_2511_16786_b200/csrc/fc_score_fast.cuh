@@ -43,6 +43,20 @@ template <> struct Load2<__nv_bfloat16> {
 
 // exp(+j*pi*n*n/N), the chirp of the convolution form of an N-point DFT; n*n is reduced modulo 2N
 // (one period) in integers first.  Costs a 64-bit division: the passes read it from a table (k_chirp_tables).
+// 4-byte asynchronous copy global -> shared (two 16-bit channels), and the wait for this thread's copies
+__device__ __forceinline__ void cp_async4(void *smem_dst, const void *gsrc) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ float2 pair16_to_float2(unsigned u, const __half *) {
+  return __half22float2(*reinterpret_cast<const __half2 *>(&u));
+}
+__device__ __forceinline__ float2 pair16_to_float2(unsigned u, const __nv_bfloat16 *) {
+  return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+}
+__device__ __forceinline__ float2 pair16_to_float2(unsigned, const float *) { return make_float2(0.f, 0.f); }
+
 // exp(-2*pi*j*r/n) for table lengths the master table has no entries for (not a power of two)
 __device__ __forceinline__ float2 root_of_unity(int r, int n) {
   double sn, cs;
@@ -162,10 +176,9 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
       x0[p] = x1[p] = make_float2(0.f, 0.f);
       const int band = omega;
       if (n <= 2 * band) {
-        const int q = n - band;
+        const int q = n - band, aq = q < 0 ? -q : q;
         const float4 P4 = *reinterpret_cast<const float4 *>(spec + (size_t)n * ncol_ws + gc0 + 2 * cp);
         const float4 Q4 = *reinterpret_cast<const float4 *>(spec + (size_t)(2 * band - n) * ncol_ws + gc0 + 2 * cp);
-        const int aq = q < 0 ? -q : q;
         float2 u = __ldg(ctab + N + aq);                         // exp(j*pi*q/N)
         if (q < 0) u.y = -u.y;
         const float2 ch = __ldg(ctab + aq);
@@ -270,6 +283,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   float2 *tw = reinterpret_cast<float2 *>(S + 2 * N2 * CP);  // [N2]   w_N2^i
   float2 *twN = tw + N2;                                     // [2][N2] w_N^(n2*k1)
   float2 *uT = twN + 2 * N2;                                 // [2][N2] exp(-j*pi*(k1 + N1*k2)/N)
+  float2 *hs = uT + 2 * N2;                                  // [2][N2] convolution variants: scaled kernel spectrum of this block's bins
   const int tid = threadIdx.x, cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
   // MID_CONV: grid.x = N1/2, the two halves of the block are the unrelated rows 2x and 2x + 1
   const int k1a = (MID == MID_CONV) ? 2 * blockIdx.x : blockIdx.x;
@@ -304,6 +318,12 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       if (MID == MID_FILTER) {
         uT[i] = master[(size_t)(k1a + N1 * i) * ustep];
         uT[N2 + i] = master[(size_t)(k1b + N1 * i) * ustep];
+      }
+      if ((MID == MID_CONV || MID == MID_CONV2) && hout == nullptr) {
+        // bins of the two halves: rows k1a and k1b (MID_CONV) or the lower and upper half of row k1a (MID_CONV2)
+        const int ba = k1a + N1 * i, bb = (MID == MID_CONV2) ? k1a + N1 * (i + N2) : k1b + N1 * i;
+        hs[i] = cscale(__ldg(hhat + ((hrev && ba != 0) ? N - ba : ba)), scale);
+        hs[N2 + i] = cscale(__ldg(hhat + ((hrev && bb != 0) ? N - bb : bb)), scale);
       }
     }
   }
@@ -379,7 +399,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
             if (cp == 0 && blockIdx.y == 0) hout[bin] = x0[it * R2B + q];
             continue;
           }
-          const float2 hq = cscale(__ldg(hhat + ((hrev && bin != 0) ? N - bin : bin)), scale);
+          const float2 hq = hs[hf * N2 + k2];
           x0[it * R2B + q] = cmul(x0[it * R2B + q], hq);
           x1[it * R2B + q] = cmul(x1[it * R2B + q], hq);
           continue;
@@ -396,7 +416,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
             if (cp == 0 && blockIdx.y == 0) hout[binh] = hf ? csub(e0, o0) : cadd(e0, o0);
             continue;
           }
-          const float2 hq = cscale(__ldg(hhat + ((hrev && binh != 0) ? N - binh : binh)), scale);
+          const float2 hq = hs[hf * N2 + k2];
           m0 = cmul(hf ? csub(e0, o0) : cadd(e0, o0), hq);
           m1 = cmul(hf ? csub(e1, o1) : cadd(e1, o1), hq);
           continue;
@@ -511,7 +531,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
 // conj(chirp(|q|))); OUT_SCORE_BAND reads the K/V rows again (kin/vin: first token of the sequence, first channel of
 // the column group) and scores |z - z_base|^2 with z_base = conj(row * conj(chirp)) / N.
 template <int R1B, int CPW, int OUT = OUT_SCORE, typename T = float, int A = 16>
-__global__ void __launch_bounds__(CPW * R1B)
+__global__ void __launch_bounds__(CPW * R1B, 512 / (CPW * R1B))
 k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__restrict__ master,
      int master_len, float *__restrict__ scores, int head0, int head_dim, long long score_stride,
      float inv_scale, double *__restrict__ partial, unsigned *__restrict__ done_counter,
@@ -526,10 +546,25 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                        // [N1][CPW]
   float2 *tw = reinterpret_cast<float2 *>(S + N1 * CPW);    // [N1]
+  // band form, 16-bit inputs: the K/V rows the residual is taken against are copied asynchronously into
+  // stg[2*A][NT] (this thread's slots only) while the two inverse stages run
+  constexpr bool STAGE = (OUT == OUT_SCORE_BAND) && sizeof(T) == 2;
+  unsigned *stg = reinterpret_cast<unsigned *>(tw + N1);
   __shared__ double red[2][NW];
   const int tid = threadIdx.x, cp = tid % CPW, j = tid / CPW;
   const int n2 = blockIdx.x, hh = blockIdx.y;
   for (int i = tid; i < N1; i += NT) tw[i] = (A == 16) ? master[(size_t)i * (master_len / N1)] : root_of_unity(i, N1);
+  // chirp factor of each row of this block (row n1 is position n1*N2 + n2), visible after the first barrier
+  __shared__ float2 cts[OUT != OUT_SCORE ? N1 : 1];
+  if (OUT != OUT_SCORE) {
+    for (int i = tid; i < N1; i += NT) {
+      const int pos = i * N2 + n2;
+      const bool spec_band = (OUT == OUT_SPEC && band >= 0);
+      const bool valid = spec_band ? pos <= 2 * band : pos < N;
+      const int cpos = spec_band ? (pos < band ? band - pos : pos - band) : pos;
+      cts[i] = valid ? __ldg(ctab + cpos) : make_float2(0.f, 0.f);
+    }
+  }
 
   float acc[16];            // |residual|^2 of rows j + R1B*p summed over this thread's channels (K and V)
 #pragma unroll
@@ -539,6 +574,19 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
   const int nslices = head_dim / (2 * CPW);
   for (int sl = 0; sl < nslices; ++sl) {
     const int gc0 = hh * head_dim + sl * (2 * CPW);
+    if (STAGE) {
+      const int col = gc0 + 2 * cp;
+      const long long coff = (long long)(head0 + col / head_dim) * stride_head + col % head_dim;
+#pragma unroll
+      for (int p = 0; p < A; ++p) {
+        const int pos = (j + R1B * p) * N2 + n2;
+        if (pos < N) {
+          const long long off = (long long)perm_token(pos, N) * stride_token + coff;
+          cp_async4(stg + (2 * p) * NT + tid, kin + off);
+          cp_async4(stg + (2 * p + 1) * NT + tid, vin + off);
+        }
+      }
+    }
     // inverse radix-R1B stage on bins k1 = pp + 16*q, straight from the workspace
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
@@ -573,6 +621,7 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
     }
     dft_inv<A>(x0);
     dft_inv<A>(x1);
+    if (STAGE) cp_async_wait_all();
 #pragma unroll
     for (int p = 0; p < A; ++p) {
       if (OUT != OUT_SCORE) {
@@ -582,8 +631,7 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
         } else if (pos >= N) {
           continue;
         }
-        const int cpos = (OUT == OUT_SPEC && band >= 0) ? (pos < band ? band - pos : pos - band) : pos;
-        const float2 ch = __ldg(ctab + cpos);                    // chirp(cpos), table of pass 1
+        const float2 ch = cts[j + R1B * p];                      // chirp of this row
         x0[p] = cmul_conj(x0[p], ch);
         x1[p] = cmul_conj(x1[p], ch);
         if (OUT == OUT_SPEC) {
@@ -593,10 +641,17 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
         }
         if (OUT == OUT_SCORE_BAND) {
           // residual against the input rows: z_base = conj(x) / N (inv_scale carries 1/d only)
-          const int col = gc0 + 2 * cp;
-          const long long off = (long long)perm_token(pos, N) * stride_token +
-                                (long long)(head0 + col / head_dim) * stride_head + col % head_dim;
-          const float2 kk = Load2<T>::ld(kin + off), vv = Load2<T>::ld(vin + off);
+          float2 kk, vv;
+          if (STAGE) {
+            kk = pair16_to_float2(stg[(2 * p) * NT + tid], kin);
+            vv = pair16_to_float2(stg[(2 * p + 1) * NT + tid], vin);
+          } else {
+            const int col = gc0 + 2 * cp;
+            const long long off = (long long)perm_token(pos, N) * stride_token +
+                                  (long long)(head0 + col / head_dim) * stride_head + col % head_dim;
+            kk = Load2<T>::ld(kin + off);
+            vv = Load2<T>::ld(vin + off);
+          }
           const float rn = 1.f / (float)N;
           x0[p] = make_float2(fmaf(-x0[p].x, rn, kk.x), fmaf(x0[p].y, rn, vv.x));
           x1[p] = make_float2(fmaf(-x1[p].x, rn, kk.y), fmaf(x1[p].y, rn, vv.y));
