@@ -137,6 +137,13 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
   const T *kb = k + (long long)h * stride_head + c;
   const T *vb = v + (long long)h * stride_head + c;
 
+  __shared__ float2 cts[LD == LD_CHIRP ? N1 : 1];           // chirp of row n1 of this block (position n1*N2 + n2)
+  if (LD == LD_CHIRP) {
+    for (int i = tid; i < N1; i += NT) {
+      const int n = i * N2 + n2;
+      cts[i] = n < N ? __ldg(ctab + n) : make_float2(1.f, 0.f);
+    }
+  }
   float2 x0[A], x1[A];
   float accK = 0.f, accV = 0.f;
 #pragma unroll
@@ -148,16 +155,13 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
       x0[p] = make_float2(kk.x, vv.x);
       x1[p] = make_float2(kk.y, vv.y);
     } else if (LD == LD_CHIRP) {
-      x0[p] = x1[p] = make_float2(0.f, 0.f);
-      if (n < N) {
-        const long long off = (long long)perm_token(n, N) * stride_token;
-        const float2 kk = Load2<T>::ld(kb + off), vv = Load2<T>::ld(vb + off);
-        accK = fmaf(kk.x, kk.x, fmaf(kk.y, kk.y, accK));
-        accV = fmaf(vv.x, vv.x, fmaf(vv.y, vv.y, accV));
-        const float2 ch = __ldg(ctab + n);
-        x0[p] = cmul_conj(make_float2(kk.x, vv.x), ch);
-        x1[p] = cmul_conj(make_float2(kk.y, vv.y), ch);
-      }
+      // loads only (rows past the sequence read row 0 and are zeroed): the sums of squares and the rotation by the
+      // conjugate chirp follow the barrier, with the chirp factors of this block's rows in shared memory by then
+      const long long off = (long long)perm_token(n < N ? n : 0, N) * stride_token;
+      const float2 kk = Load2<T>::ld(kb + off), vv = Load2<T>::ld(vb + off);
+      const float keep = n < N ? 1.f : 0.f;
+      x0[p] = make_float2(kk.x * keep, vv.x * keep);
+      x1[p] = make_float2(kk.y * keep, vv.y * keep);
     } else if (LD == LD_KERNEL) {
       x0[p] = x1[p] = make_float2(0.f, 0.f);
       if (gc0 == 0 && cp == 0) {
@@ -208,11 +212,19 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
   }
   for (int i = tid; i < N1; i += NT) tw[i] = (A == 16) ? master[(size_t)i * (master_len / N1)] : root_of_unity(i, N1);
   __syncthreads();
-  if (LD == LD_KV) {
+  if (LD == LD_KV || LD == LD_CHIRP) {
 #pragma unroll
     for (int p = 0; p < A; ++p) {
       accK = fmaf(x0[p].x, x0[p].x, fmaf(x1[p].x, x1[p].x, accK));
       accV = fmaf(x0[p].y, x0[p].y, fmaf(x1[p].y, x1[p].y, accV));
+    }
+  }
+  if (LD == LD_CHIRP) {
+#pragma unroll
+    for (int p = 0; p < A; ++p) {
+      const float2 ch = cts[j + R1B * p];
+      x0[p] = cmul_conj(x0[p], ch);
+      x1[p] = cmul_conj(x1[p], ch);
     }
   }
   dft_fwd<A>(x0);
