@@ -392,11 +392,13 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       for (int q = 0; q < R2B; ++q) {
         x0[it * R2B + q] = y0[q];
         x1[it * R2B + q] = y1[q];
-        Sh[(q + R2B * pp) * CP + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
+        // MID_CONV keeps its bins in registers: nobody else reads them, and the rows of this sub-block are written
+        // again only by this thread (first inverse stage), so neither the store nor the two barriers are needed
+        if (MID != MID_CONV) Sh[(q + R2B * pp) * CP + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
       }
     }
   }
-  __syncthreads();       // full spectra of both halves are in shared memory
+  if (MID != MID_CONV) __syncthreads();       // full spectra of both halves are in shared memory
   if (active) {
     const float4 *Sp = S + (self ? hf : 1 - hf) * (N2 * CP);
 #pragma unroll
@@ -496,7 +498,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       for (int q = 0; q < R2B; ++q) { x0[it * R2B + q] = y0[q]; x1[it * R2B + q] = y1[q]; }
     }
   }
-  __syncthreads();       // all partner reads are done
+  if (MID != MID_CONV) __syncthreads();       // all partner reads are done
   if (active) {
 #pragma unroll
     for (int it = 0; it < IT; ++it) {
