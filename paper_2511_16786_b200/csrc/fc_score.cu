@@ -654,6 +654,50 @@ SeqPlan plan_sequence(int N, bool allow_fast = true) {
   return s;
 }
 
+// Shape of a chirp transform on the specialised kernels: M = N1 * N2 with N1 = a * r1b (first-stage radix a of
+// passes 1 and 3, then radix r1b) and N2 = 16 * r2b, or 2 * 16 * r2b when pass 2 takes its rows in two halves (dbl).
+// Powers of two 1024..131072 have a = 16; 2^k * {5, 3, 7} have a = 10, 12, 14 with r1b = 8 or 16.  a == 0: no such
+// shape.
+struct ChirpShape {
+  int a, r1b, r2b;
+  bool dbl;
+  int n1() const { return a * r1b; }
+  int n2() const { return (dbl ? 32 : 16) * r2b; }
+};
+
+inline ChirpShape chirp_shape(int M) {
+  ChirpShape c{0, 0, 0, false};
+  if (M == 131072) return ChirpShape{16, 16, 16, true};          // 256 x 512
+  if (is_pow2(M)) {
+    if (M < 1024 || M > 65536) return c;
+    const int bits = ilog2(M), b1 = bits / 2;
+    return ChirpShape{16, (1 << b1) / 16, (M >> b1) / 16, false};
+  }
+  const int a = (M % 5 == 0) ? 10 : (M % 3 == 0) ? 12 : (M % 7 == 0) ? 14 : 0;
+  if (a == 0 || M % (16 * a) != 0) return c;
+  // a = 10 and 12 run faster with a radix-8 second stage (256-thread blocks, two or three per SM) where the rows
+  // then have 128..512 points; measured 5..11 % on the whole chirp path, while a = 14 loses 8 % that way
+  const int n2w = M / (8 * a);
+  if (a != 14 && is_pow2(n2w) && n2w >= 128 && n2w <= 512)
+    return n2w == 512 ? ChirpShape{a, 8, 16, true} : ChirpShape{a, 8, n2w / 16, false};
+  const int n2 = M / (16 * a);
+  if (!is_pow2(n2) || n2 < 32 || n2 > 512) return c;
+  return n2 == 512 ? ChirpShape{a, 16, 16, true} : ChirpShape{a, 16, n2 / 16, false};
+}
+
+// Smallest transform length >= need the specialised kernels take (0 if none up to 131072).
+inline int chirp_length(long long need) {
+  int best = 0;
+  for (int M = 1024; M <= 131072; M <<= 1)
+    if (M >= need) { best = M; break; }
+  for (int n1 = 160; n1 <= 224; n1 += 32)
+    for (int n2 = 32; n2 <= 512; n2 <<= 1) {
+      const int M = n1 * n2;
+      if (M >= need && (best == 0 || M < best)) best = M;
+    }
+  return best;
+}
+
 struct ScoreLayout {
   size_t off_ws, off_spec, off_hhat, off_hcol, off_part_tot, off_part_hi, total;
   size_t part_tot_bytes, part_hi_bytes;   // one copy; the specialised path keeps two and alternates (step parity)
@@ -688,8 +732,16 @@ ScoreLayout layout_for(const fc_handle *h, const SeqPlan &sp, int num_heads, int
   // would only save workspace.
   int sub = head_dim;
   const size_t split_above = h->group_bytes > ((size_t)1 << 60) ? h->group_bytes : 4 * h->group_bytes;
-  if (sp.bluestein && hg == 1)
+  if (sp.bluestein && hg == 1) {
+    // specialised kernels: the intermediates of the groups in flight (one per internal stream) should stay in the
+    // cache, so a head is halved down to 64 columns while they exceed three times the budget (measured on eight
+    // ragged sequences of 7k..54k tokens: 1.6 % of the step; the length is the full form's, the band form's is shorter)
+    const int Mf = h->generic_only ? 0 : chirp_length(2LL * sp.N - 1);
+    if (Mf != 0 && Mf <= sp.Nfft)
+      while (sub % 128 == 0 && (size_t)(chirp_multi ? h->num_aux : 1) * Mf * sub * sizeof(float2) > 3 * h->group_bytes)
+        sub /= 2;
     while (sub % 64 == 0 && (size_t)sp.Nfft * sub * sizeof(float2) > split_above) sub /= 2;
+  }
   L.sub_cols = sub;
   L.ws_buf_bytes = align_up((size_t)sp.Nfft * sub * hg * sizeof(float2), 256);
   size_t off = 0;
@@ -876,50 +928,6 @@ fc_status launch_fast(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const
   FC_TUNE_CASE(32, 8)
 #undef FC_TUNE_CASE
   return FC_ERR_INTERNAL;
-}
-
-// Shape of a chirp transform on the specialised kernels: M = N1 * N2 with N1 = a * r1b (first-stage radix a of
-// passes 1 and 3, then radix r1b) and N2 = 16 * r2b, or 2 * 16 * r2b when pass 2 takes its rows in two halves (dbl).
-// Powers of two 1024..131072 have a = 16; 2^k * {5, 3, 7} have a = 10, 12, 14 with r1b = 8 or 16.  a == 0: no such
-// shape.
-struct ChirpShape {
-  int a, r1b, r2b;
-  bool dbl;
-  int n1() const { return a * r1b; }
-  int n2() const { return (dbl ? 32 : 16) * r2b; }
-};
-
-inline ChirpShape chirp_shape(int M) {
-  ChirpShape c{0, 0, 0, false};
-  if (M == 131072) return ChirpShape{16, 16, 16, true};          // 256 x 512
-  if (is_pow2(M)) {
-    if (M < 1024 || M > 65536) return c;
-    const int bits = ilog2(M), b1 = bits / 2;
-    return ChirpShape{16, (1 << b1) / 16, (M >> b1) / 16, false};
-  }
-  const int a = (M % 5 == 0) ? 10 : (M % 3 == 0) ? 12 : (M % 7 == 0) ? 14 : 0;
-  if (a == 0 || M % (16 * a) != 0) return c;
-  // a = 10 and 12 run faster with a radix-8 second stage (256-thread blocks, two or three per SM) where the rows
-  // then have 128..512 points; measured 5..11 % on the whole chirp path, while a = 14 loses 8 % that way
-  const int n2w = M / (8 * a);
-  if (a != 14 && is_pow2(n2w) && n2w >= 128 && n2w <= 512)
-    return n2w == 512 ? ChirpShape{a, 8, 16, true} : ChirpShape{a, 8, n2w / 16, false};
-  const int n2 = M / (16 * a);
-  if (!is_pow2(n2) || n2 < 32 || n2 > 512) return c;
-  return n2 == 512 ? ChirpShape{a, 16, 16, true} : ChirpShape{a, 16, n2 / 16, false};
-}
-
-// Smallest transform length >= need the specialised kernels take (0 if none up to 131072).
-inline int chirp_length(long long need) {
-  int best = 0;
-  for (int M = 1024; M <= 131072; M <<= 1)
-    if (M >= need) { best = M; break; }
-  for (int n1 = 160; n1 <= 224; n1 += 32)
-    for (int n2 = 32; n2 <= 512; n2 <<= 1) {
-      const int M = n1 * n2;
-      if (M >= need && (best == 0 || M < best)) best = M;
-    }
-  return best;
 }
 
 // The chirp path on the specialised kernels: two circular convolutions with the chirp kernel, each
