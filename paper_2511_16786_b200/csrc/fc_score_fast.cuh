@@ -119,8 +119,9 @@ __device__ __forceinline__ void dft_inv(float2 (&x)[R]) { dft_small<R, +1>(x); }
 // stage points n1 = j + R1B*p, p = 0..A-1, loaded from the K/V rows.  N1 = A*R1B: A = 16 with R1B = 2..16 for
 // power-of-two lengths, A = 10, 12 or 14 with R1B = 16 for the chirp path's lengths 2^a * {5, 3, 7}.
 // ---------------------------------------------------------------------------
+// Launch bounds: three resident blocks of 256 threads (80 registers), the measured best for the power-of-two path.
 template <typename T, int R1B, int CPW, int LD = LD_KV, int A = 16>
-__global__ void __launch_bounds__(CPW * R1B)
+__global__ void __launch_bounds__(CPW * R1B, (768 / (CPW * R1B)) > 0 ? 768 / (CPW * R1B) : 1)
 k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, long long stride_head,
      int head0, int head_dim, int N, int N2, int ncol_ws, float2 *__restrict__ ws,
      const float2 *__restrict__ master, int master_len, double *__restrict__ partial,
