@@ -108,6 +108,27 @@ enum { MID_FILTER = 0, MID_CONV = 1, MID_CONV2 = 2 };
 // reordered domain; the K/V rows are read again and the score is |z - z_base|^2.
 enum { OUT_SCORE = 0, OUT_SPEC = 1, OUT_SCORE_CHIRP = 2, OUT_SCORE_BAND = 3 };
 
+// x[p] *= w^p (CONJ: conj(w)^p), p = 1..15, for both channels, from w and w^4 alone: the other powers are products of
+// at most three table values (w^p = w^(4g) * w^r), which replaces 13 of 15 shared-memory reads per use by arithmetic.
+template <bool CONJ>
+__device__ __forceinline__ void twiddle_powers16(float2 (&x0)[16], float2 (&x1)[16], float2 c1, float2 c4) {
+  if (CONJ) { c1.y = -c1.y; c4.y = -c4.y; }
+  const float2 c2 = cmul(c1, c1), c3 = cmul(c2, c1);
+  float2 base = c4;
+  x0[1] = cmul(x0[1], c1); x1[1] = cmul(x1[1], c1);
+  x0[2] = cmul(x0[2], c2); x1[2] = cmul(x1[2], c2);
+  x0[3] = cmul(x0[3], c3); x1[3] = cmul(x1[3], c3);
+#pragma unroll
+  for (int g = 1; g < 4; ++g) {
+    const float2 b1 = cmul(base, c1), b2 = cmul(base, c2), b3 = cmul(base, c3);
+    x0[4 * g] = cmul(x0[4 * g], base);     x1[4 * g] = cmul(x1[4 * g], base);
+    x0[4 * g + 1] = cmul(x0[4 * g + 1], b1); x1[4 * g + 1] = cmul(x1[4 * g + 1], b1);
+    x0[4 * g + 2] = cmul(x0[4 * g + 2], b2); x1[4 * g + 2] = cmul(x1[4 * g + 2], b2);
+    x0[4 * g + 3] = cmul(x0[4 * g + 3], b3); x1[4 * g + 3] = cmul(x1[4 * g + 3], b3);
+    if (g < 3) base = cmul(base, c4);
+  }
+}
+
 template <int R>
 __device__ __forceinline__ void dft_fwd(float2 (&x)[R]) { dft_small<R, -1>(x); }
 template <int R>
@@ -363,15 +384,10 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
     }
     dft_fwd<16>(x0);
     dft_fwd<16>(x1);
+    twiddle_powers16<false>(x0, x1, tw[j], tw[4 * j]);
 #pragma unroll
-    for (int p = 0; p < 16; ++p) {
-      if (p > 0) {
-        const float2 w = tw[j * p];
-        x0[p] = cmul(x0[p], w);
-        x1[p] = cmul(x1[p], w);
-      }
+    for (int p = 0; p < 16; ++p)
       Sh[(j + R2B * p) * CP + cp] = make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
-    }
   }
   __syncthreads();
   // second forward stage, written back in place (each sub-block is touched by one thread only);
@@ -395,7 +411,14 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
         x1[it * R2B + q] = y1[q];
         // MID_CONV keeps its bins in registers: nobody else reads them, and the rows of this sub-block are written
         // again only by this thread (first inverse stage), so neither the store nor the two barriers are needed
-        if (MID != MID_CONV) Sh[(q + R2B * pp) * CP + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
+        // MID_FILTER: only bins inside the two bands are read by their partners (the partner of an in-band bin is
+        // in the other band), so the rest, 1 - 2*gamma of them, is not written back
+        bool wanted = (MID != MID_CONV);
+        if (MID == MID_FILTER) {
+          const int bin = k1 + N1 * (pp + 16 * q);
+          wanted = bin <= omega || N - bin <= omega;
+        }
+        if (wanted) Sh[(q + R2B * pp) * CP + cp] = make_float4(y0[q].x, y0[q].y, y1[q].x, y1[q].y);
       }
     }
   }
@@ -517,12 +540,8 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       const float4 t = Sh[(j + R2B * p) * CP + cp];
       x0[p] = make_float2(t.x, t.y);
       x1[p] = make_float2(t.z, t.w);
-      if (p > 0) {
-        const float2 w = tw[j * p];
-        x0[p] = cmul_conj(x0[p], w);
-        x1[p] = cmul_conj(x1[p], w);
-      }
     }
+    twiddle_powers16<true>(x0, x1, tw[j], tw[4 * j]);
     dft_inv<16>(x0);
     dft_inv<16>(x1);
 #pragma unroll
