@@ -129,6 +129,23 @@ __device__ __forceinline__ void twiddle_powers16(float2 (&x0)[16], float2 (&x1)[
   }
 }
 
+// x[p] *= b * s^p (CONJ: the conjugate of that), p = 0..15, from b, s and s^4.
+template <bool CONJ>
+__device__ __forceinline__ void twiddle_affine16(float2 (&x0)[16], float2 (&x1)[16], float2 b, float2 s1, float2 s4) {
+  if (CONJ) { b.y = -b.y; s1.y = -s1.y; s4.y = -s4.y; }
+  const float2 s2 = cmul(s1, s1), s3 = cmul(s2, s1);
+  float2 base = b;
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const float2 b1 = cmul(base, s1), b2 = cmul(base, s2), b3 = cmul(base, s3);
+    x0[4 * g] = cmul(x0[4 * g], base);     x1[4 * g] = cmul(x1[4 * g], base);
+    x0[4 * g + 1] = cmul(x0[4 * g + 1], b1); x1[4 * g + 1] = cmul(x1[4 * g + 1], b1);
+    x0[4 * g + 2] = cmul(x0[4 * g + 2], b2); x1[4 * g + 2] = cmul(x1[4 * g + 2], b2);
+    x0[4 * g + 3] = cmul(x0[4 * g + 3], b3); x1[4 * g + 3] = cmul(x1[4 * g + 3], b3);
+    if (g < 3) base = cmul(base, s4);
+  }
+}
+
 template <int R>
 __device__ __forceinline__ void dft_fwd(float2 (&x)[R]) { dft_small<R, -1>(x); }
 template <int R>
@@ -362,6 +379,9 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
     }
   }
   float4 *Sh = S + hf * (N2 * CP);
+  // row twiddles: entry j + R2B*p of this half's table is entry j times the p-th power of a step that the table
+  // holds at R2B (MID_CONV2: both halves belong to one row, the step sits in the even samples' table)
+  const int so = (MID == MID_CONV2) ? 0 : hf * N2;
   float2 x0[16], x1[16];
   // element n2 of the row: MID_CONV2 interleaves the halves (n2 = 2i + hf)
   float2 *base = ws + ((size_t)k1 * ROW + (MID == MID_CONV2 ? hf : 0)) * ncol_ws + gc0 + 2 * cp;
@@ -376,12 +396,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   }
   __syncthreads();
   if (active) {
-#pragma unroll
-    for (int p = 0; p < 16; ++p) {
-      const float2 w = twN[hf * N2 + j + R2B * p];
-      x0[p] = cmul(x0[p], w);
-      x1[p] = cmul(x1[p], w);
-    }
+    twiddle_affine16<false>(x0, x1, twN[hf * N2 + j], twN[so + R2B], twN[so + 4 * R2B]);
     dft_fwd<16>(x0);
     dft_fwd<16>(x1);
     twiddle_powers16<false>(x0, x1, tw[j], tw[4 * j]);
@@ -544,12 +559,11 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
     twiddle_powers16<true>(x0, x1, tw[j], tw[4 * j]);
     dft_inv<16>(x0);
     dft_inv<16>(x1);
+    twiddle_affine16<true>(x0, x1, twN[hf * N2 + j], twN[so + R2B], twN[so + 4 * R2B]);
 #pragma unroll
-    for (int p = 0; p < 16; ++p) {
-      const float2 w = twN[hf * N2 + j + R2B * p];
-      const float2 a = cmul_conj(x0[p], w), b = cmul_conj(x1[p], w);
-      *reinterpret_cast<float4 *>(base + (size_t)(j + R2B * p) * rstride) = make_float4(a.x, a.y, b.x, b.y);
-    }
+    for (int p = 0; p < 16; ++p)
+      *reinterpret_cast<float4 *>(base + (size_t)(j + R2B * p) * rstride) =
+          make_float4(x0[p].x, x0[p].y, x1[p].x, x1[p].y);
   }
 }
 
