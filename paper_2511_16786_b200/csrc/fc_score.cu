@@ -873,7 +873,7 @@ fc_status launch_fast_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, 
   constexpr int N1 = 16 * R1B, N2 = 16 * R2B;
   const int d = kv->head_dim, ncol_ws = hg * d;
   const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
-  const size_t sm2 = (size_t)2 * N2 * CP * sizeof(float4) + 5 * N2 * sizeof(float2);
+  const size_t sm2 = (size_t)2 * N2 * CP * sizeof(float4) + (5 * N2 + 16) * sizeof(float2);
   fc_status s;
   if ((s = set_smem(fast::k_p1<T, R1B, CPW>, sm1)) != FC_OK) return s;
   {
@@ -943,7 +943,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
   constexpr int CPW = 32, CP = 8, N1 = A * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
   constexpr int MIDV = DOUBLE ? fast::MID_CONV2 : fast::MID_CONV;
   const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
-  const size_t sm2 = (size_t)2 * (16 * R2B) * CP * sizeof(float4) + 7 * (16 * R2B) * sizeof(float2);
+  const size_t sm2 = (size_t)2 * (16 * R2B) * CP * sizeof(float4) + (7 * (16 * R2B) + 16) * sizeof(float2);
   // band form's last pass, 16-bit inputs: staging slots for the K/V rows it reads again
   const size_t sm3b = sm1 + (sizeof(T) == 2 ? (size_t)2 * A * CPW * R1B * sizeof(unsigned) : 0);
   fc_status s;

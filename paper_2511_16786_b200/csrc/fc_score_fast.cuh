@@ -332,9 +332,12 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   extern __shared__ float4 smem4[];
   float4 *S = smem4;                                         // [2][N2][CP]
   float2 *tw = reinterpret_cast<float2 *>(S + 2 * N2 * CP);  // [N2]   w_N2^i
+  // tables with one part per half: the second half starts H2 = N2 + 4 entries in, so that threads of the two halves
+  // reading the same index hit different banks
+  constexpr int H2 = N2 + 4;
   float2 *twN = tw + N2;                                     // [2][N2] w_N^(n2*k1)
-  float2 *uT = twN + 2 * N2;                                 // [2][N2] exp(-j*pi*(k1 + N1*k2)/N)
-  float2 *hs = uT + 2 * N2;                                  // [2][N2] convolution variants: scaled kernel spectrum of this block's bins
+  float2 *uT = twN + H2 + N2;                                // [2][N2] exp(-j*pi*(k1 + N1*k2)/N)
+  float2 *hs = uT + H2 + N2;                                  // [2][N2] convolution variants: scaled kernel spectrum of this block's bins
   const int tid = threadIdx.x, cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
   // MID_CONV: grid.x = N1/2, the two halves of the block are the unrelated rows 2x and 2x + 1
   const int k1a = (MID == MID_CONV) ? 2 * blockIdx.x : blockIdx.x;
@@ -356,32 +359,32 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
       if (MID == MID_CONV2) {
         const int ra = ((2 * i) * k1a) % N, rb = ((2 * i + 1) * k1a) % N;
         twN[i] = tab ? master[(size_t)ra * mstepN] : root_of_unity(ra, N);        // even samples: n2 = 2i
-        twN[N2 + i] = tab ? master[(size_t)rb * mstepN] : root_of_unity(rb, N);   // odd samples: n2 = 2i + 1
+        twN[H2 + i] = tab ? master[(size_t)rb * mstepN] : root_of_unity(rb, N);   // odd samples: n2 = 2i + 1
         uT[i] = master[(size_t)i * (master_len / ROW)];                          // w_ROW^k of the radix-2 step
       } else if (MID == MID_CONV) {
         const int ra = (i * k1a) % N, rb = (i * k1b) % N;
         twN[i] = tab ? master[(size_t)ra * mstepN] : root_of_unity(ra, N);
-        twN[N2 + i] = tab ? master[(size_t)rb * mstepN] : root_of_unity(rb, N);
+        twN[H2 + i] = tab ? master[(size_t)rb * mstepN] : root_of_unity(rb, N);
       } else {
         twN[i] = master[(size_t)((i * k1a) & (N - 1)) * mstepN];
-        twN[N2 + i] = master[(size_t)((i * k1b) & (N - 1)) * mstepN];
+        twN[H2 + i] = master[(size_t)((i * k1b) & (N - 1)) * mstepN];
       }
       if (MID == MID_FILTER) {
         uT[i] = master[(size_t)(k1a + N1 * i) * ustep];
-        uT[N2 + i] = master[(size_t)(k1b + N1 * i) * ustep];
+        uT[H2 + i] = master[(size_t)(k1b + N1 * i) * ustep];
       }
       if ((MID == MID_CONV || MID == MID_CONV2) && hout == nullptr) {
         // bins of the two halves: rows k1a and k1b (MID_CONV) or the lower and upper half of row k1a (MID_CONV2)
         const int ba = k1a + N1 * i, bb = (MID == MID_CONV2) ? k1a + N1 * (i + N2) : k1b + N1 * i;
         hs[i] = cscale(__ldg(hhat + ((hrev && ba != 0) ? N - ba : ba)), scale);
-        hs[N2 + i] = cscale(__ldg(hhat + ((hrev && bb != 0) ? N - bb : bb)), scale);
+        hs[H2 + i] = cscale(__ldg(hhat + ((hrev && bb != 0) ? N - bb : bb)), scale);
       }
     }
   }
   float4 *Sh = S + hf * (N2 * CP);
   // row twiddles: entry j + R2B*p of this half's table is entry j times the p-th power of a step that the table
   // holds at R2B (MID_CONV2: both halves belong to one row, the step sits in the even samples' table)
-  const int so = (MID == MID_CONV2) ? 0 : hf * N2;
+  const int so = (MID == MID_CONV2) ? 0 : hf * H2;
   float2 x0[16], x1[16];
   // element n2 of the row: MID_CONV2 interleaves the halves (n2 = 2i + hf)
   float2 *base = ws + ((size_t)k1 * ROW + (MID == MID_CONV2 ? hf : 0)) * ncol_ws + gc0 + 2 * cp;
@@ -396,7 +399,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   }
   __syncthreads();
   if (active) {
-    twiddle_affine16<false>(x0, x1, twN[hf * N2 + j], twN[so + R2B], twN[so + 4 * R2B]);
+    twiddle_affine16<false>(x0, x1, twN[hf * H2 + j], twN[so + R2B], twN[so + 4 * R2B]);
     dft_fwd<16>(x0);
     dft_fwd<16>(x1);
     twiddle_powers16<false>(x0, x1, tw[j], tw[4 * j]);
@@ -452,7 +455,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
             if (cp == 0 && blockIdx.y == 0) hout[bin] = x0[it * R2B + q];
             continue;
           }
-          const float2 hq = hs[hf * N2 + k2];
+          const float2 hq = hs[hf * H2 + k2];
           x0[it * R2B + q] = cmul(x0[it * R2B + q], hq);
           x1[it * R2B + q] = cmul(x1[it * R2B + q], hq);
           continue;
@@ -469,7 +472,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
             if (cp == 0 && blockIdx.y == 0) hout[binh] = hf ? csub(e0, o0) : cadd(e0, o0);
             continue;
           }
-          const float2 hq = hs[hf * N2 + k2];
+          const float2 hq = hs[hf * H2 + k2];
           m0 = cmul(hf ? csub(e0, o0) : cadd(e0, o0), hq);
           m1 = cmul(hf ? csub(e1, o1) : cadd(e1, o1), hq);
           continue;
@@ -482,7 +485,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
         } else if (inL || inH) {
           const int k2p = (k1 == 0) ? ((N2 - k2) & (N2 - 1)) : (N2 - 1 - k2);
           const float4 t = Sp[((k2p >> 4) + R2B * (k2p & 15)) * CP + cp];
-          float2 u = uT[hf * N2 + k2];                             // exp(-j*pi*bin/N)
+          float2 u = uT[hf * H2 + k2];                             // exp(-j*pi*bin/N)
           const float sgn = inL ? -0.5f : 0.5f;                   // E = (P -/+ uQ)/2 with u = exp(+j*pi*bin/N)
           u = make_float2(u.x * sgn, -u.y * sgn);
           const float2 q0 = make_float2(t.x, t.y), q1 = make_float2(t.z, t.w);
@@ -559,7 +562,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
     twiddle_powers16<true>(x0, x1, tw[j], tw[4 * j]);
     dft_inv<16>(x0);
     dft_inv<16>(x1);
-    twiddle_affine16<true>(x0, x1, twN[hf * N2 + j], twN[so + R2B], twN[so + 4 * R2B]);
+    twiddle_affine16<true>(x0, x1, twN[hf * H2 + j], twN[so + R2B], twN[so + 4 * R2B]);
 #pragma unroll
     for (int p = 0; p < 16; ++p)
       *reinterpret_cast<float4 *>(base + (size_t)(j + R2B * p) * rstride) =
