@@ -658,6 +658,11 @@ SeqPlan plan_sequence(int N, bool allow_fast = true) {
 // passes 1 and 3, then radix r1b) and N2 = 16 * r2b, or 2 * 16 * r2b when pass 2 takes its rows in two halves (dbl).
 // Powers of two 1024..131072 have a = 16; 2^k * {5, 3, 7} have a = 10, 12, 14 with r1b = 8 or 16.  a == 0: no such
 // shape.
+// Channel pairs per block of passes 1 and 3 on the chirp path: with a radix-16 second stage and rows of 128 points
+// or more, 16 pairs (256-thread blocks, two or three per SM) instead of 32 (512 threads, one per SM): measured
+// 10..14 % on transforms of 57344..98304 points, 2 % at 28672, while 224 x 64 loses 4 % that way.
+constexpr int chirp_cpw(int r1b, int r2b, bool dbl) { return (r1b == 16 && (r2b >= 8 || dbl)) ? 16 : 32; }
+
 struct ChirpShape {
   int a, r1b, r2b;
   bool dbl;
@@ -675,11 +680,11 @@ inline ChirpShape chirp_shape(int M) {
   }
   const int a = (M % 5 == 0) ? 10 : (M % 3 == 0) ? 12 : (M % 7 == 0) ? 14 : 0;
   if (a == 0 || M % (16 * a) != 0) return c;
-  // a = 10 and 12 run faster with a radix-8 second stage (256-thread blocks, two or three per SM) where the rows
-  // then have 128..512 points; measured 5..11 % on the whole chirp path, while a = 14 loses 8 % that way
+  // a = 10 and 12 with rows of 128 or 256 points run faster on a radix-8 second stage (80 or 96 x N2) than on
+  // 160 or 192 x N2/2: measured 3..10 % on the whole chirp path; a = 14 loses 8 % that way, and rows of 512 points
+  // (two halves per row in pass 2) lose 14 % against 160 or 192 x 256
   const int n2w = M / (8 * a);
-  if (a != 14 && is_pow2(n2w) && n2w >= 128 && n2w <= 512)
-    return n2w == 512 ? ChirpShape{a, 8, 16, true} : ChirpShape{a, 8, n2w / 16, false};
+  if (a != 14 && (n2w == 128 || n2w == 256)) return ChirpShape{a, 8, n2w / 16, false};
   const int n2 = M / (16 * a);
   if (!is_pow2(n2) || n2 < 32 || n2 > 512) return c;
   return n2 == 512 ? ChirpShape{a, 16, 16, true} : ChirpShape{a, 16, n2 / 16, false};
@@ -864,6 +869,9 @@ fc_status launch_pass2(fc_handle *h, cudaStream_t st, const SeqPlan &sp, int nco
 }
 
 // The three specialised launches for one head group of a power-of-two sequence.
+// Channel pairs per block of passes 1 and 3 on the power-of-two path for a first factor n1.
+constexpr int fast_cpw(int n1, int cpw) { return n1 == 256 ? 16 : cpw; }
+
 // CPW: channel pairs per block in passes 1 and 3; CP: channel pairs per half tile in pass 2.
 template <typename T, int R1B, int R2B, int CPW, int CP>
 fc_status launch_fast_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, const T *kp, const T *vp,
@@ -911,8 +919,12 @@ fc_status launch_fast_tuned(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
     return launch_fast_impl<T, A, B, CPW, CP>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores, \
                                               total_tokens, part_tot, part_hi, energy_b);
   FC_FAST_CASE(2, 2) FC_FAST_CASE(2, 4) FC_FAST_CASE(4, 4) FC_FAST_CASE(4, 8)
-  FC_FAST_CASE(8, 8) FC_FAST_CASE(8, 16) FC_FAST_CASE(16, 16)
+  FC_FAST_CASE(8, 8) FC_FAST_CASE(8, 16)
 #undef FC_FAST_CASE
+  // 65536 = 256 x 256: 16 channel pairs per block keep passes 1 and 3 at 256 threads (see chirp_cpw)
+  if (sp.N1 == 256 && sp.N2 == 256)
+    return launch_fast_impl<T, 16, 16, fast_cpw(256, CPW), CP>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores,
+                                                               total_tokens, part_tot, part_hi, energy_b);
   return FC_ERR_INTERNAL;
 }
 
@@ -940,7 +952,7 @@ fc_status launch_chirp_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
                             int h0, int hg, int omega, float2 *ws, float2 *spec, const float2 *hhat, double *ptot,
                             double *phi, float *scores, long long total_tokens, int dcols, int accumulate, int band,
                             float2 *hout, const float2 *ctab) {
-  constexpr int CPW = 32, CP = 8, N1 = A * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
+  constexpr int CPW = chirp_cpw(R1B, R2B, DOUBLE), CP = 8, N1 = A * R1B, N2 = (DOUBLE ? 32 : 16) * R2B;
   constexpr int MIDV = DOUBLE ? fast::MID_CONV2 : fast::MID_CONV;
   const size_t sm1 = (size_t)N1 * CPW * sizeof(float4) + N1 * sizeof(float2);
   const size_t sm2 = (size_t)2 * (16 * R2B) * CP * sizeof(float4) + (7 * (16 * R2B) + 16) * sizeof(float2);
@@ -1047,11 +1059,11 @@ fc_status launch_chirp(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, cons
   // a = 14: 224 x {32 .. 512}
   FC_CHIRP_CASE(14, 16, 2, false) FC_CHIRP_CASE(14, 16, 4, false) FC_CHIRP_CASE(14, 16, 8, false)
   FC_CHIRP_CASE(14, 16, 16, false) FC_CHIRP_CASE(14, 16, 16, true)
-  // a = 10, 12: {160, 192} x 32, {80, 96} x {128, 256, 512}, {160, 192} x 512
+  // a = 10, 12: {160, 192} x 32, {80, 96} x {128, 256}, {160, 192} x {256, 512}
   FC_CHIRP_CASE(10, 16, 2, false) FC_CHIRP_CASE(10, 8, 8, false) FC_CHIRP_CASE(10, 8, 16, false)
-  FC_CHIRP_CASE(10, 8, 16, true) FC_CHIRP_CASE(10, 16, 16, true)
+  FC_CHIRP_CASE(10, 16, 16, false) FC_CHIRP_CASE(10, 16, 16, true)
   FC_CHIRP_CASE(12, 16, 2, false) FC_CHIRP_CASE(12, 8, 8, false) FC_CHIRP_CASE(12, 8, 16, false)
-  FC_CHIRP_CASE(12, 8, 16, true) FC_CHIRP_CASE(12, 16, 16, true)
+  FC_CHIRP_CASE(12, 16, 16, false) FC_CHIRP_CASE(12, 16, 16, true)
 #undef FC_CHIRP_CASE
   return FC_ERR_INTERNAL;
 }
@@ -1253,6 +1265,8 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       // stream order and the last pass adds their contributions to the score in that order.
       if (chirp_fast) {                         // a length and a width the specialised kernels take
         const int sub = L.sub_cols, ngr = (hg == 1) ? d / sub : 1, n2f = chirp_shape(Mc).n2();
+        const ChirpShape shp = chirp_shape(Mc);
+        const int tilew = 2 * chirp_cpw(shp.r1b, shp.r2b, shp.dbl);     // columns per block of passes 1 and 3
         const int ncol = (hg == 1) ? sub : ncol_ws;
         const int si = group % L.chirp_streams;                   // head groups alternate over the internal streams
         cudaStream_t sx = L.chirp_streams > 1 ? h->aux[si] : st;
@@ -1260,11 +1274,11 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
         float2 *spec_s = reinterpret_cast<float2 *>(wsb + L.off_spec + (size_t)si * L.spec_buf_bytes);
         for (int cg = 0; cg < ngr; ++cg) {                        // column groups of one head, else one pass
           if ((s = launch_chirp<T>(h, sx, kv, kp + cg * sub, vp + cg * sub, N, Mc, h0, hg, omega, ws_s, spec_s, hhat,
-                                   ptot + 2 * (size_t)cg * n2f * (ncol / 64), phi + 2 * (size_t)cg * n2f * hg,
+                                   ptot + 2 * (size_t)cg * n2f * (ncol / tilew), phi + 2 * (size_t)cg * n2f * hg,
                                    scores + start, total_tokens, (hg == 1) ? sub : d, cg > 0 ? 1 : 0, band, ctab)) != FC_OK)
             return s;
         }
-        tot_slots += (size_t)n2f * (ncol / 64) * ngr;
+        tot_slots += (size_t)n2f * (ncol / tilew) * ngr;
         hi_slots += (size_t)n2f * hg * ngr;
         continue;
       }
@@ -1308,7 +1322,7 @@ fc_status score_sequence(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, in
       hi_slots += (size_t)sp.N2 * hg * ngroups;
       continue;
     }
-    tot_slots += (size_t)sp.N2 * (ncol_ws / (sp.fast ? 2 * h->tune_cpw : sp.cs));
+    tot_slots += (size_t)sp.N2 * (ncol_ws / (sp.fast ? 2 * fast_cpw(sp.N1, h->tune_cpw) : sp.cs));
     hi_slots += (size_t)sp.N2 * hg;
   }
   if (sp.fast) {

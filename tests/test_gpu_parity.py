@@ -235,8 +235,8 @@ def test_describe_plan_reports_the_convolution_length_in_use(fc):
         assert (p["bluestein"], p["nfft"], p["n1"] * p["n2"]) == (False, 32768, 32768)
         p = fc.fc_describe_plan(h, 2500, 0.2)                    # 2500 + 1000 + 1 -> 4096
         assert (p["band_form"], p["nfft"], p["n1"] * p["n2"]) == (True, 4096, 4096)
-        p = fc.fc_describe_plan(h, 35107, 0.2)                   # 35107 + 14042 + 1 = 49150 -> 49152 = 96 x 512
-        assert (p["band_form"], p["nfft"], p["n1"], p["n2"]) == (True, 49152, 96, 512)
+        p = fc.fc_describe_plan(h, 35107, 0.2)                   # 35107 + 14042 + 1 = 49150 -> 49152 = 192 x 256
+        assert (p["band_form"], p["nfft"], p["n1"], p["n2"]) == (True, 49152, 192, 256)
         p = fc.fc_describe_plan(h, 33001, 0.6)                   # band wider than the spectrum: 2N - 1 -> 81920
         assert (p["bluestein"], p["band_form"], p["nfft"], p["n1"], p["n2"]) == (True, False, 81920, 160, 512)
         fc.fc_set_chirp_band(h, False)
