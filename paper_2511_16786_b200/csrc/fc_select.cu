@@ -366,19 +366,31 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
   tie_take = tie_take < 0 ? 0 : (tie_take > my_tie ? my_tie : tie_take);
   const int count = my_gt + tie_take;
   const int n16 = row_bytes >> 4;
-  for (int rr = warp; rr < count; rr += kSelThreads / 32) {
-    const long long row = off + first + rr;
-    const long long tok = (long long)s0 + dst[first + rr];
-    const int per_head = 2 * n16;
+  // a warp takes kGatherRows rows at a time: their indices, then their 16-byte pieces, are requested together, so
+  // that several independent round trips to DRAM are in flight per warp instead of one after the other
+  constexpr int kGatherRows = 4;
+  const int per_head = 2 * n16;
+  for (int rr0 = warp * kGatherRows; rr0 < count; rr0 += (kSelThreads / 32) * kGatherRows) {
+    long long tok[kGatherRows];
+#pragma unroll
+    for (int g = 0; g < kGatherRows; ++g) {
+      const int rr = rr0 + g < count ? rr0 + g : rr0;            // rows past the end repeat the first (not stored)
+      tok[g] = (long long)s0 + dst[first + rr];
+    }
     for (int w = lane; w < (PER_LAYER ? H * per_head : per_head); w += 32) {
       const int hh = PER_LAYER ? w / per_head : h;
       const int u = PER_LAYER ? w - hh * per_head : w;
-      const long long src = tok * stride_token_b + (long long)hh * stride_head_b;
-      const long long dsto = (row * H + hh) * (long long)row_bytes;
       const bool isv = u >= n16;
       const int uu = isv ? u - n16 : u;
-      const uint4 val = *reinterpret_cast<const uint4 *>((isv ? vin : kin) + src + 16ll * uu);
-      *reinterpret_cast<uint4 *>((isv ? out_v : out_k) + dsto + 16ll * uu) = val;
+      const char *in = (isv ? vin : kin) + (long long)hh * stride_head_b + 16ll * uu;
+      char *out = (isv ? out_v : out_k) + 16ll * uu;
+      uint4 val[kGatherRows];
+#pragma unroll
+      for (int g = 0; g < kGatherRows; ++g) val[g] = *reinterpret_cast<const uint4 *>(in + tok[g] * stride_token_b);
+#pragma unroll
+      for (int g = 0; g < kGatherRows; ++g)
+        if (rr0 + g < count)
+          *reinterpret_cast<uint4 *>(out + ((off + first + rr0 + g) * H + hh) * (long long)row_bytes) = val[g];
     }
   }
 }
