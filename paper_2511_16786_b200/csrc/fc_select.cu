@@ -174,22 +174,22 @@ __device__ __forceinline__ unsigned score_key(float x) {
 }
 
 constexpr int kSelThreads = 1024;   // threads per block of the selection kernel
-constexpr int kSelCluster = 8;      // blocks (one cluster) per (sequence, head)
+constexpr int kSelCluster = 8;      // blocks (one cluster) per (sequence, head) at most; 2 or 4 for shorter sequences
 constexpr int kSelKptMax = 16;      // scores per thread: 8 * 1024 * 16 = 131072 tokens at most
 
 // Selection + compaction + row gather for one (sequence, head), by one cluster of
-// kSelCluster blocks.  Block r of the cluster owns the contiguous token range
+// CL blocks (2, 4 or 8).  Block r of the cluster owns the contiguous token range
 // [r*chunk, (r+1)*chunk) and keeps its score keys in registers.  The k-th largest
 // key is found by a 4-pass MSB-first radix select whose 256-bin histograms are
 // summed across the cluster through distributed shared memory; the chosen tokens
 // are then ranked in token order (block prefix + cluster prefix), written as
 // ascending indices, and their K/V rows are copied by the same block.
-// grid (kSelCluster * sequences in chunk, heads), cluster (kSelCluster, 1, 1).
+// grid (CL * sequences in chunk, heads), cluster (CL, 1, 1).
 // PER_LAYER: one cluster per sequence (grid.y = 1) ranks the tokens by the sum over heads of their
 // scores (the order of the head-averaged deviation), writes the same indices for every head and
 // gathers the rows of all heads.  protect (may be null): a non-zero byte per token of the batch puts
 // that token before every unmarked one.
-template <int kSelKpt, bool PER_LAYER>
+template <int kSelKpt, bool PER_LAYER, int CL>
 __device__ __forceinline__ void
 select_gather_body(const float *__restrict__ scores, long long T, const SeqTable &st, int b0,
                 const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
@@ -201,13 +201,13 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ int lhist[4][256];          // this block's histograms, one per pass (read by the whole cluster)
   __shared__ int ghist[256];             // cluster-wide histogram of the current pass
-  __shared__ unsigned tot[kSelCluster];  // (ties << 16 | greater) of every block of the cluster
+  __shared__ unsigned tot[CL];  // (ties << 16 | greater) of every block of the cluster
   __shared__ unsigned wsum[kSelThreads / 32];
   __shared__ unsigned s_prefix;
   __shared__ int s_krem;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned r = cluster.block_rank();
-  const int bl = blockIdx.x / kSelCluster;
+  const int bl = blockIdx.x / CL;
   const int b = b0 + bl, h = PER_LAYER ? 0 : blockIdx.y;
   const int s0 = st.start[bl];
   const int n = st.start[bl + 1] - s0;
@@ -222,7 +222,7 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
   const float *sc = scores + (long long)h * T + s0;
   int *dst = out_idx + (long long)h * cap + off;
 
-  const int chunk = (n + kSelCluster - 1) / kSelCluster;
+  const int chunk = (n + CL - 1) / CL;
   const int lo = (int)r * chunk;
   const int hi = lo + chunk < n ? lo + chunk : n;
   const int base = lo + tid * kSelKpt;
@@ -265,7 +265,7 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
       if (tid < 256) {
         int v = 0;
 #pragma unroll
-        for (unsigned rr = 0; rr < kSelCluster; ++rr) v += *cluster.map_shared_rank(&lhist[pass][tid], rr);
+        for (unsigned rr = 0; rr < CL; ++rr) v += *cluster.map_shared_rank(&lhist[pass][tid], rr);
         ghist[tid] = v;
       }
       __syncthreads();
@@ -325,14 +325,14 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
     wsum[lane] = wi - v;                                 // exclusive prefix of the warp totals
     if (lane == 31) {
 #pragma unroll
-      for (unsigned rr = 0; rr < kSelCluster; ++rr) *cluster.map_shared_rank(&tot[r], rr) = wi;
+      for (unsigned rr = 0; rr < CL; ++rr) *cluster.map_shared_rank(&tot[r], rr) = wi;
     }
   }
   cluster.sync();                                        // also orders wsum for the block
   const unsigned excl = wsum[warp] + incl - cnt;
   int gt_before = 0, tie_before = 0, my_gt = 0, my_tie = 0;
 #pragma unroll
-  for (unsigned rr = 0; rr < kSelCluster; ++rr) {
+  for (unsigned rr = 0; rr < CL; ++rr) {
     const unsigned t = tot[rr];
     if (rr < r) { gt_before += (int)(t & 0xFFFFu); tie_before += (int)(t >> 16); }
     if (rr == r) { my_gt = (int)(t & 0xFFFFu); my_tie = (int)(t >> 16); }
@@ -395,13 +395,13 @@ select_gather_body(const float *__restrict__ scores, long long T, const SeqTable
   }
 }
 
-// The kernel: grid (kSelCluster * sequences in chunk, heads or 1, layers in chunk); blockIdx.z picks the
+// The kernel: grid (CL * sequences in chunk, heads or 1, layers in chunk); blockIdx.z picks the
 // layer's pointers from the table and the layer's rows of budgets [L][B] and out_offsets [L][B+1].
 // overlap != 0 (launched with the programmatic-serialisation attribute): the next launch in the stream
 // may start as soon as every block of this one has begun, and this grid does not finish before its
 // predecessor has, so "the last launch is complete" still means "all of them are".
-template <int kSelKpt, bool PER_LAYER>
-__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
+template <int kSelKpt, bool PER_LAYER, int CL>
+__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(kSelThreads)
 k_select_gather(const __grid_constant__ LayerTable lt, long long T, const __grid_constant__ SeqTable st, int b0, int B,
                 const int *__restrict__ budgets, const long long *__restrict__ out_offsets,
                 int *__restrict__ status, long long stride_token_b,
@@ -409,7 +409,7 @@ k_select_gather(const __grid_constant__ LayerTable lt, long long T, const __grid
                 const unsigned char *__restrict__ protect) {
   if (overlap) asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
   const int z = blockIdx.z;
-  select_gather_body<kSelKpt, PER_LAYER>(lt.scores[z], T, st, b0, budgets + (size_t)z * B,
+  select_gather_body<kSelKpt, PER_LAYER, CL>(lt.scores[z], T, st, b0, budgets + (size_t)z * B,
                                          out_offsets + (size_t)z * (B + 1), lt.out_idx[z], lt.cap[z], status, lt.k[z], lt.v[z],
                                          stride_token_b, stride_head_b, row_bytes, H, lt.out_k[z], lt.out_v[z], protect);
   if (overlap) asm volatile("griddepcontrol.wait;\n" ::: "memory");
@@ -499,13 +499,20 @@ fc_status launch_select(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, con
     for (int i = 0; i <= nseq; ++i) tab.start[i] = kv->cu_seqlens[b0 + i];
     int nmax = 0;
     for (int i = 0; i < nseq; ++i) nmax = tab.start[i + 1] - tab.start[i] > nmax ? tab.start[i + 1] - tab.start[i] : nmax;
-    const int per_thread = (nmax + kSelCluster * kSelThreads - 1) / (kSelCluster * kSelThreads);
+    // blocks per (sequence, head): the fewest of 2, 4, 8 that hold the longest sequence at 16 scores per thread.
+    // Fewer blocks per cluster let more clusters run at once (8 blocks of 1024 threads: 15 clusters on 148 SMs) and
+    // the phases of the radix select wait on cluster barriers, not on bandwidth: measured per step, 8 -> 2 blocks,
+    // 0.199 -> 0.158 ms at 28 x 4 heads of 32768 tokens, 1.70 -> 1.12 ms at 32 x 32 heads of 16384; one block is
+    // 2..9 % slower than two where it would fit.
+    int cl = 2;
+    while (cl < kSelCluster && nmax > cl * kSelThreads * kSelKptMax) cl *= 2;
+    const int per_thread = (nmax + cl * kSelThreads - 1) / (cl * kSelThreads);
     {
       ProfScope ps(h, FC_K_SELECT, st);
-#define FC_SEL_LAUNCH(KPT, PL)                                                                          \
+#define FC_SEL_LAUNCH(KPT, PL, CLV)                                                                     \
   do {                                                                                                  \
     cudaLaunchConfig_t lc = {};                                                                         \
-    lc.gridDim = dim3(kSelCluster * nseq, (PL) ? 1 : kv->num_heads, nl);                                \
+    lc.gridDim = dim3(CLV * nseq, (PL) ? 1 : kv->num_heads, nl);                                        \
     lc.blockDim = dim3(kSelThreads);                                                                    \
     lc.stream = st;                                                                                     \
     cudaLaunchAttribute at[1];                                                                          \
@@ -513,24 +520,26 @@ fc_status launch_select(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, con
     at[0].val.programmaticStreamSerializationAllowed = 1;                                               \
     lc.attrs = at;                                                                                      \
     lc.numAttrs = h->select_overlap ? 1 : 0;                                                            \
-    launch_err = cudaLaunchKernelEx(&lc, k_select_gather<KPT, PL>, lt, (long long)T, tab, b0, (int)kv->batch, \
+    launch_err = cudaLaunchKernelEx(&lc, k_select_gather<KPT, PL, CLV>, lt, (long long)T, tab, b0, (int)kv->batch, \
         budgets, reinterpret_cast<const long long *>(out_offsets),                                      \
         h->status_word, (long long)(kv->stride_token * es), (long long)(kv->stride_head * es),          \
         (int)(kv->head_dim * es), (int)kv->num_heads, (int)h->select_overlap, protect);                 \
   } while (0)
+#define FC_SEL_KPT(PL, CLV)                                                                             \
+  do {                                                                                                  \
+    if (per_thread <= 2) FC_SEL_LAUNCH(2, PL, CLV);                                                     \
+    else if (per_thread <= 4) FC_SEL_LAUNCH(4, PL, CLV);                                                \
+    else if (per_thread <= 8) FC_SEL_LAUNCH(8, PL, CLV);                                                \
+    else FC_SEL_LAUNCH(16, PL, CLV);                                                                    \
+  } while (0)
       cudaError_t launch_err = cudaSuccess;
       if (per_layer) {
-        if (per_thread <= 2) FC_SEL_LAUNCH(2, true);
-        else if (per_thread <= 4) FC_SEL_LAUNCH(4, true);
-        else if (per_thread <= 8) FC_SEL_LAUNCH(8, true);
-        else FC_SEL_LAUNCH(16, true);
+        if (cl == 2) FC_SEL_KPT(true, 2); else if (cl == 4) FC_SEL_KPT(true, 4); else FC_SEL_KPT(true, 8);
       } else {
-        if (per_thread <= 2) FC_SEL_LAUNCH(2, false);
-        else if (per_thread <= 4) FC_SEL_LAUNCH(4, false);
-        else if (per_thread <= 8) FC_SEL_LAUNCH(8, false);
-        else FC_SEL_LAUNCH(16, false);
+        if (cl == 2) FC_SEL_KPT(false, 2); else if (cl == 4) FC_SEL_KPT(false, 4); else FC_SEL_KPT(false, 8);
       }
       if (launch_err != cudaSuccess) return FC_ERR_CUDA;
+#undef FC_SEL_KPT
 #undef FC_SEL_LAUNCH
     }
     if ((s = fc_after_launch(h)) != FC_OK) return s;
