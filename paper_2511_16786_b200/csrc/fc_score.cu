@@ -630,6 +630,8 @@ void finish_plan(SeqPlan &s) {
   // 131072 points: 256 x 512 with 32-column tiles in passes 1 and 3 beats 128 x 1024, whose pass 2 has
   // room for only 4 columns per block (measured on the chirp path: 461 against 488 ms per step)
   if (bits == 17) { b1 = 8; s.cs = 32; }
+  // 8192 points on the specialised kernels: 128 x 64 keeps every pass at 256-thread blocks (2 % over 64 x 128)
+  if (s.fast && bits == 13) b1 = 7;
   s.N1 = 1 << b1;
   s.N2 = s.Nfft / s.N1;
   int cs2 = 4096 / s.N2;      // 2*N2*cs2*8 bytes = 64 KiB
@@ -914,17 +916,18 @@ fc_status launch_fast_tuned(fc_handle *h, cudaStream_t st, const fc_kv_view *kv,
                             const SeqPlan &sp, int h0, int hg, int omega, float2 *ws, double *ptot, double *phi,
                             float *scores, long long total_tokens, const double *part_tot,
                             const double *part_hi, double *energy_b) {
-#define FC_FAST_CASE(A, B)                                                                                \
+  // Every pass runs 256-thread blocks, the measured optimum: CPWV channel pairs per block in passes 1 and 3 and CPV
+  // per half tile in pass 2 follow from the factors (CPW and CP are the widths for 128 x 256).
+#define FC_FAST_CASE(A, B, CPWV, CPV)                                                                     \
   if (sp.N1 == 16 * A && sp.N2 == 16 * B)                                                                 \
-    return launch_fast_impl<T, A, B, CPW, CP>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores, \
-                                              total_tokens, part_tot, part_hi, energy_b);
-  FC_FAST_CASE(2, 2) FC_FAST_CASE(2, 4) FC_FAST_CASE(4, 4) FC_FAST_CASE(4, 8)
-  FC_FAST_CASE(8, 8) FC_FAST_CASE(8, 16)
+    return launch_fast_impl<T, A, B, CPWV, CPV>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores, \
+                                                total_tokens, part_tot, part_hi, energy_b);
+  FC_FAST_CASE(2, 2, CPW, CP) FC_FAST_CASE(2, 4, CPW, CP) FC_FAST_CASE(4, 4, CPW, CP) FC_FAST_CASE(4, 8, CPW, CP)
+  FC_FAST_CASE(8, 4, CPW, 4 * CP)                 // 8192 = 128 x 64
+  FC_FAST_CASE(8, 8, CPW, 2 * CP)                 // 16384 = 128 x 128
+  FC_FAST_CASE(8, 16, CPW, CP)                    // 32768 = 128 x 256
+  FC_FAST_CASE(16, 16, fast_cpw(256, CPW), CP)    // 65536 = 256 x 256
 #undef FC_FAST_CASE
-  // 65536 = 256 x 256: 16 channel pairs per block keep passes 1 and 3 at 256 threads (see chirp_cpw)
-  if (sp.N1 == 256 && sp.N2 == 256)
-    return launch_fast_impl<T, 16, 16, fast_cpw(256, CPW), CP>(h, st, kv, kp, vp, sp, h0, hg, omega, ws, ptot, phi, scores,
-                                                               total_tokens, part_tot, part_hi, energy_b);
   return FC_ERR_INTERNAL;
 }
 
