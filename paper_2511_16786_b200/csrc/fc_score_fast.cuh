@@ -220,8 +220,8 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
       const int band = omega;
       if (n <= 2 * band) {
         const int q = n - band, aq = q < 0 ? -q : q;
-        const float4 P4 = *reinterpret_cast<const float4 *>(spec + (size_t)n * ncol_ws + gc0 + 2 * cp);
-        const float4 Q4 = *reinterpret_cast<const float4 *>(spec + (size_t)(2 * band - n) * ncol_ws + gc0 + 2 * cp);
+        const float4 P4 = __ldcg(reinterpret_cast<const float4 *>(spec + (size_t)n * ncol_ws + gc0 + 2 * cp));
+        const float4 Q4 = __ldcg(reinterpret_cast<const float4 *>(spec + (size_t)(2 * band - n) * ncol_ws + gc0 + 2 * cp));
         float2 u = __ldg(ctab + N + aq);                         // exp(j*pi*q/N)
         if (q < 0) u.y = -u.y;
         const float2 ch = __ldg(ctab + aq);
@@ -234,8 +234,8 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
       x0[p] = x1[p] = make_float2(0.f, 0.f);
       if (n < N) {
         const int q = n, qp = (N - q) % N;
-        const float4 P4 = *reinterpret_cast<const float4 *>(spec + (size_t)q * ncol_ws + gc0 + 2 * cp);
-        const float4 Q4 = *reinterpret_cast<const float4 *>(spec + (size_t)qp * ncol_ws + gc0 + 2 * cp);
+        const float4 P4 = __ldcg(reinterpret_cast<const float4 *>(spec + (size_t)q * ncol_ws + gc0 + 2 * cp));
+        const float4 Q4 = __ldcg(reinterpret_cast<const float4 *>(spec + (size_t)qp * ncol_ws + gc0 + 2 * cp));
         const float2 u = __ldg(ctab + N + q);
         const float inL = (q <= omega) ? 0.5f : 0.f;
         const float inH = (q != 0 && N - q <= omega) ? 0.5f : 0.f;
@@ -392,7 +392,7 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   if (active) {
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
-      const float4 t = *reinterpret_cast<const float4 *>(base + (size_t)(j + R2B * p) * rstride);
+      const float4 t = __ldcg(reinterpret_cast<const float4 *>(base + (size_t)(j + R2B * p) * rstride));
       x0[p] = make_float2(t.x, t.y);
       x1[p] = make_float2(t.z, t.w);
     }
@@ -646,8 +646,8 @@ k_p3(int N, int N2, int ncol_ws, const float2 *__restrict__ ws, const float2 *__
       float2 y0[R1B], y1[R1B];
 #pragma unroll
       for (int q = 0; q < R1B; ++q) {
-        const float4 t = *reinterpret_cast<const float4 *>(
-            ws + ((size_t)(pp + A * q) * N2 + n2) * ncol_ws + gc0 + 2 * cp);
+        const float4 t = __ldcg(reinterpret_cast<const float4 *>(
+            ws + ((size_t)(pp + A * q) * N2 + n2) * ncol_ws + gc0 + 2 * cp));
         y0[q] = make_float2(t.x, t.y);
         y1[q] = make_float2(t.z, t.w);
       }
