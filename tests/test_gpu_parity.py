@@ -163,6 +163,13 @@ def test_scores_long_sequences_sampled_head(fc, N):
     _check_layer(fc, k, v, [0, N], 0.2)
 
 
+@pytest.mark.parametrize("N", [8192, 32768, 65536])
+def test_scores_long_power_of_two_fp32_inputs(fc, N):
+    # fp32 rows at the 1e-3 bar on the lengths whose twiddles are products of table values (up to three factors)
+    k, v = _rand_kv(N, 1, 64, torch.float32, 7 + N)
+    _check_layer(fc, k, v, [0, N], 0.2)
+
+
 def test_scores_long_arbitrary_length(fc):
     N = 40961
     k, v = _rand_kv(N, 1, 64, torch.bfloat16, N)
