@@ -901,7 +901,7 @@ fc_status launch_fast_impl(fc_handle *h, cudaStream_t st, const fc_kv_view *kv, 
   if ((s = set_smem(fast::k_p2<R2B, CP>, sm2)) != FC_OK) return s;
   {
     ProfScope ps(h, FC_K_PASS2, st);
-    fast::k_p2<R2B, CP><<<dim3(N1 / 2 + 1, ncol_ws / (2 * CP)), 2 * CP * R2B, sm2, st>>>(
+    fast::k_p2<R2B, CP><<<dim3(N1 / 2, ncol_ws / (2 * CP)), 2 * CP * R2B, sm2, st>>>(
         N1, ncol_ws, ws, h->master, h->master_len, omega);
   }
   if ((s = fc_after_launch(h)) != FC_OK) return s;

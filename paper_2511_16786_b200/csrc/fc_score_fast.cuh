@@ -315,7 +315,7 @@ k_p1(const T *__restrict__ k, const T *__restrict__ v, long long stride_token, l
 }
 
 // ---------------------------------------------------------------------------
-// pass 2: grid (N1/2 + 1, group columns / (2*CP)), block 2*CP*R2B.
+// pass 2: grid (N1/2, group columns / (2*CP)) for the filter and the plain convolution, (N1, ...) for MID_CONV2; block 2*CP*R2B.
 // Thread (cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2*CP)): channel pair cp of
 // the slice, half hf (k1 = blockIdx.x or N1 - blockIdx.x), first-stage points
 // n2 = j + R2B*p.
@@ -341,14 +341,16 @@ k_p2(int N1, int ncol_ws, float2 *__restrict__ ws, const float2 *__restrict__ ma
   const int tid = threadIdx.x, cp = tid % CP, hf = (tid / CP) & 1, j = tid / (2 * CP);
   // MID_CONV: grid.x = N1/2, the two halves of the block are the unrelated rows 2x and 2x + 1
   const int k1a = (MID == MID_CONV) ? 2 * blockIdx.x : blockIdx.x;
+  // MID_FILTER: grid.x = N1/2; block x > 0 holds the partner rows x and N1 - x, block 0 the two rows that are their
+  // own partners, 0 and N1/2 (each half then reads its partner bins from itself)
   const int k1b = (MID == MID_CONV) ? 2 * blockIdx.x + 1
-                : (MID == MID_CONV2) ? (int)blockIdx.x : ((N1 - k1a) & (N1 - 1));
-  const bool self = (MID == MID_FILTER) && (k1a == k1b);
+                : (MID == MID_CONV2) ? (int)blockIdx.x : (k1a == 0 ? N1 / 2 : N1 - k1a);
+  const bool self = (MID == MID_FILTER) && (k1a == 0);
   const int k1 = hf ? k1b : k1a;
   constexpr int ROW = (MID == MID_CONV2) ? 2 * N2 : N2;      // points of one row of the workspace
   const int N = N1 * ROW;
   const int gc0 = blockIdx.y * (2 * CP);
-  const bool active = !(self && hf);
+  constexpr bool active = true;
 
   {
     // N is a power of two (every root is in the master table) or, on the chirp path, 2^a * {3, 5, 7}
